@@ -1,0 +1,163 @@
+/*
+ * pearl_prb.h -- C ABI of the B200-native Prioritized Replay Buffer.
+ *
+ * The buffer is the Replay Manager + Data Storage pair of PEARL (arXiv 2311.09445):
+ * a K-ary sum tree over transition priorities (Section V-A) next to a struct-of-arrays
+ * store of the transitions {state, action, reward, next state, done} (Section II-A).
+ * The four operations are the requests the host runtime sends to the Replay Manager in
+ * the paper's training protocol (Section IV, Listing 2): insertion, priority sampling
+ * (Eq. 1) followed by the read of the sampled rows, and priority update.
+ *
+ * Conventions
+ *   - Every `d_*` argument is a DEVICE pointer owned by the caller, every `h_*` argument a
+ *     HOST pointer owned by the caller.  The library never frees or keeps them.
+ *   - Batches are dense and row-major: row k of a field with `fb` bytes per row starts at
+ *     byte k*fb.  A field pointer must be aligned to the largest power of two (<= 16) that
+ *     divides fb, otherwise PEARL_ERR_ALIGN.
+ *   - Calls validate their host-visible arguments, enqueue kernels on the handle's stream
+ *     and return; they are ordered by that stream.  The ring cursor, the fill count, the
+ *     sample-call counter and the status word live in device memory.
+ *   - Return value: PEARL_OK or a negative PEARL_ERR_* (nothing was enqueued).  Conditions
+ *     found on the device never trap; they set PEARL_ST_* bits in a device status word that
+ *     pearl_prb_sync() returns and clears.
+ *   - One handle is used from one host thread at a time.
+ */
+#ifndef PEARL_PRB_H_
+#define PEARL_PRB_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pearl_prb pearl_prb_t;
+
+/* Row sizes of the two caller-defined fields; reward is one binary32 and done one byte. */
+typedef struct pearl_layout {
+    uint32_t obs_bytes;   /* bytes of one observation (state and next state alike), may be 0 */
+    uint32_t act_bytes;   /* bytes of one action, may be 0 */
+} pearl_layout_t;
+
+#define PEARL_OK 0
+#define PEARL_ERR_NULL (-1)        /* a required pointer is NULL */
+#define PEARL_ERR_BAD_FANOUT (-2)  /* fanout not in {2, 4, 8, 16, 32} */
+#define PEARL_ERR_BAD_BATCH (-3)   /* batch is 0 or larger than max_batch */
+#define PEARL_ERR_TOO_MANY (-4)    /* insert of more rows than the capacity */
+#define PEARL_ERR_ALIGN (-5)       /* a field pointer is misaligned for its row size */
+#define PEARL_ERR_OOM (-6)         /* allocation failed or the slab is too small */
+#define PEARL_ERR_BAD_ARG (-7)     /* a scalar argument is out of range or not finite */
+#define PEARL_ERR_CUDA (-8)        /* a CUDA runtime call failed */
+
+#define PEARL_ST_BAD_INDEX 1u      /* update: index < 0 or >= fill count; entry skipped */
+#define PEARL_ST_BAD_PRIORITY 2u   /* NaN/Inf/negative priority or non-finite TD error; update skips
+                                      the entry, insert stores the row with priority 0 */
+#define PEARL_ST_EMPTY 4u          /* sample on an empty buffer or a non-positive total; outputs untouched */
+#define PEARL_ST_CLAMPED 8u        /* a descent met residual >= last prefix sum and took the last positive child */
+#define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out */
+
+/* Largest batch the update calls accept, whatever max_batch says. */
+#define PEARL_MAX_UPDATE_BATCH 4096u
+
+/* Bytes of device memory a buffer of this geometry needs (tree, storage, scratch and the
+ * staging areas of the *_host calls).  0 if the arguments are invalid. */
+uint64_t pearl_prb_slab_bytes(uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
+                              uint32_t max_batch);
+
+/* Creates a buffer of `capacity` slots (1 .. 2^30) with a sum tree of the given fanout
+ * (Section V-A: the tree is parameterised by depth and fanout).  Depth D is the smallest
+ * D >= 1 with fanout^D >= capacity; level 0 is the root, level D the leaves; each level is a
+ * binary32 array zero-padded to a multiple of the fanout.
+ *   device       CUDA device ordinal that owns the memory.
+ *   cuda_stream  a cudaStream_t (NULL = the legacy default stream) on which every call enqueues.
+ *   slab         optional caller-owned device memory of at least pearl_prb_slab_bytes() bytes,
+ *                256-byte aligned; NULL lets the library allocate (and free in destroy).
+ * The tree, the state and the scratch area are zeroed on the stream.  Returns PEARL_ERR_OOM if
+ * the slab is too small. */
+int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout,
+                     const pearl_layout_t* layout, uint32_t max_batch, int device,
+                     void* cuda_stream, void* slab, uint64_t slab_bytes);
+
+/* Synchronises the stream, frees library-owned memory and the handle. */
+int pearl_prb_destroy(pearl_prb_t* prb);
+
+/* Insertion (Section V-A: "priority retrievals followed by priority updates"; Listing 2: the
+ * collected experiences are added to the Data Storage and insertion requests sent to the RM).
+ * Writes n transitions to ring slots cursor .. cursor+n-1 (mod capacity), sets their leaves to
+ * d_prio and re-sums the ancestors; then cursor += n (mod capacity), fill = min(fill+n, capacity).
+ * The caller supplies each new transition's priority.  d_obs/d_next_obs: n rows of obs_bytes;
+ * d_act: n rows of act_bytes; d_rew: n binary32; d_done: n bytes; a NULL field pointer leaves
+ * that field of the slots unwritten.  1 <= n <= min(max_batch, capacity). */
+int pearl_prb_insert(pearl_prb_t* prb, uint32_t n, const void* d_obs, const void* d_act,
+                     const float* d_rew, const void* d_next_obs, const uint8_t* d_done,
+                     const float* d_prio);
+
+/* Priority sampling (Eq. 1, Section V-A) + the Data Storage read of the sampled rows
+ * (Listing 2: sampled_data = D_storage[sampled_indices]).
+ * The range [0, total) is cut into B equal strata; stratum k draws
+ *   x_k = (k + u_k) * total / B,  u_k = word 0 of Philox4x32-10(counter = (k, 0, call_lo, call_hi),
+ *   key = (seed_lo, seed_hi)) * 2^-32,
+ * where `call` counts this handle's earlier successful sample calls.  A root-to-leaf traversal
+ * finds the leaf i_k whose prefix interval holds x_k (binary32 left-to-right child prefix sums,
+ * binary64 target).  Outputs, each of B entries:
+ *   d_idx   leaf indices (int32);
+ *   d_w     importance-sampling weights (fill * p_i / total)^(-beta), divided by their maximum
+ *           over the batch (may be NULL);
+ *   d_obs, d_act, d_rew, d_next_obs, d_done   the gathered rows (each may be NULL to skip it).
+ * 1 <= B <= max_batch; beta finite and >= 0. */
+int pearl_prb_sample(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, int32_t* d_idx,
+                     float* d_w, void* d_obs, void* d_act, float* d_rew, void* d_next_obs,
+                     uint8_t* d_done);
+
+/* Priority update (Section V-A).  For b = 0 .. B-1 in batch order: p_b = (|d_td[b]| + eps)^alpha
+ * and leaf[d_idx[b]] <- p_b, so the last valid entry of a repeated index wins; then every
+ * ancestor of a written leaf is recomputed as the left-to-right binary32 sum of its children,
+ * deepest level first.  The power is evaluated in binary64 from IEEE basic operations only, so
+ * it is reproducible bit for bit.  1 <= B <= min(max_batch, PEARL_MAX_UPDATE_BATCH);
+ * alpha, eps finite and >= 0. */
+int pearl_prb_update(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_td,
+                     float alpha, float eps);
+
+/* As pearl_prb_update, with the priorities given directly (no power). */
+int pearl_prb_update_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx,
+                                const float* d_prio);
+
+/* Host-buffer forms of the three calls (the paper's host runtime exchanges requests and data
+ * with the Replay Manager over PCIe, Section IV-A).  They copy their inputs to the device and
+ * their outputs back on the handle's stream; sample_host returns after the stream has drained,
+ * insert_host and update_host once their host buffers may be reused.  Pinned host memory makes
+ * the copies asynchronous.  Output pointers of sample_host other than h_idx may be NULL. */
+int pearl_prb_insert_host(pearl_prb_t* prb, uint32_t n, const void* h_obs, const void* h_act,
+                          const float* h_rew, const void* h_next_obs, const uint8_t* h_done,
+                          const float* h_prio);
+int pearl_prb_sample_host(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, int32_t* h_idx,
+                          float* h_w, void* h_obs, void* h_act, float* h_rew, void* h_next_obs,
+                          uint8_t* h_done);
+int pearl_prb_update_host(pearl_prb_t* prb, uint32_t B, const int32_t* h_idx, const float* h_td,
+                          float alpha, float eps);
+
+/* Waits for the stream; returns the accumulated PEARL_ST_* bits in *status_bits (may be NULL)
+ * and clears them. */
+int pearl_prb_sync(pearl_prb_t* prb, uint32_t* status_bits);
+
+/* Read-back for tests and checkpoints; each synchronises the stream.  Any output may be NULL. */
+int pearl_prb_info(pearl_prb_t* prb, uint64_t* fill, uint64_t* cursor, uint64_t* sample_calls,
+                   uint32_t* depth);
+/* Copies the first `count` entries (padding included) of tree level `level` (0 = root). */
+int pearl_prb_read_level(pearl_prb_t* prb, uint32_t level, float* h_dst, uint64_t count);
+/* Number of entries of a level including its zero padding; 0 for an invalid level. */
+uint64_t pearl_prb_level_alloc(pearl_prb_t* prb, uint32_t level);
+/* Copies stored rows h_idx[0..n) (slot numbers < capacity) to host arrays. */
+int pearl_prb_read_rows(pearl_prb_t* prb, const int32_t* h_idx, uint32_t n, void* h_obs,
+                        void* h_act, float* h_rew, void* h_next_obs, uint8_t* h_done);
+
+/* Number of kernels this handle has launched so far. */
+uint64_t pearl_prb_kernel_launches(pearl_prb_t* prb);
+
+/* A short English name for a PEARL_ERR_* code. */
+const char* pearl_prb_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PEARL_PRB_H_ */

@@ -1,0 +1,114 @@
+// Internal declarations shared by the CUDA translation units of libpearl_prb.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define PRB_MAX_LEVELS 32       // level 0 (root) .. level D (leaves), D <= 30 for fanout 2
+#define PRB_NUM_FIELDS 5        // obs, next_obs, act, rew, done
+
+enum PrbField { F_OBS = 0, F_NEXT_OBS = 1, F_ACT = 2, F_REW = 3, F_DONE = 4 };
+
+// Mutable state of a buffer; lives in device memory so that enqueued work never depends on
+// host-side copies of it.
+struct PrbState {
+    unsigned long long cursor;        // next ring slot to be written
+    unsigned long long fill;          // transitions stored, <= capacity
+    unsigned long long sample_calls;  // successful sample calls so far (Philox counter words 2,3)
+    unsigned long long wmax_bits;     // batch maximum of the raw IS weights (bits of a positive double)
+    unsigned int status;              // PEARL_ST_* bits
+    unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
+    unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished
+    unsigned int reserved;
+};
+
+// Geometry and device addresses, passed to kernels by value.
+struct PrbView {
+    PrbState* state;
+    float* level[PRB_MAX_LEVELS];     // level[l] holds K * n_{l-1} entries (level[0]: 1)
+    unsigned char* store[PRB_NUM_FIELDS];
+    uint32_t field_bytes[PRB_NUM_FIELDS];
+    uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
+    double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
+    uint64_t capacity;
+    uint32_t fanout;                  // K
+    uint32_t log2_fanout;
+    uint32_t depth;                   // D
+    uint32_t max_batch;
+};
+
+// Dense caller-side batch, one pointer per field (NULL = field skipped).
+struct PrbBatch {
+    unsigned char* ptr[PRB_NUM_FIELDS];
+};
+
+// Kernel launchers; each returns the number of kernels launched, or -1 on a launch error.
+int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s);
+int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s);
+int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
+                      float alpha, float eps, cudaStream_t s);
+
+// ---- device helpers -------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// Left-to-right binary32 sum of the K children of one parent (children start at c, K-aligned).
+// Loads bypass L1: other threads of this kernel may have written the children.
+template <int K>
+__device__ __forceinline__ float prb_sum_children(const float* c)
+{
+    if (K == 2) {
+        float2 v = __ldcg(reinterpret_cast<const float2*>(c));
+        return __fadd_rn(v.x, v.y);
+    } else {
+        float4 v = __ldcg(reinterpret_cast<const float4*>(c));
+        float s = __fadd_rn(__fadd_rn(__fadd_rn(v.x, v.y), v.z), v.w);
+#pragma unroll
+        for (int q = 1; q < K / 4; ++q) {
+            float4 u = __ldcg(reinterpret_cast<const float4*>(c) + q);
+            s = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(s, u.x), u.y), u.z), u.w);
+        }
+        return s;
+    }
+}
+
+__device__ __forceinline__ float prb_sum_children_dyn(const float* c, uint32_t K)
+{
+    switch (K) {
+    case 2: return prb_sum_children<2>(c);
+    case 4: return prb_sum_children<4>(c);
+    case 8: return prb_sum_children<8>(c);
+    case 16: return prb_sum_children<16>(c);
+    default: return prb_sum_children<32>(c);
+    }
+}
+
+__device__ __forceinline__ bool prb_valid_priority(float p)
+{
+    return (p >= 0.0f) && (p <= 3.402823466e+38f);   // false for NaN, negative, +Inf
+}
+
+// Copies granules e in [e_begin, e_end) of a tile: granule e is read from src[src_at(e)] and
+// written to dst[dst_at(e)].  Each thread first issues up to 8 independent loads, then the
+// stores, with consecutive threads on consecutive granules.
+template <typename T, typename SrcAt, typename DstAt>
+__device__ __forceinline__ void prb_copy_granules(T* __restrict__ dst, const T* __restrict__ src,
+                                                  uint32_t e_begin, uint32_t e_end, SrcAt src_at, DstAt dst_at)
+{
+    constexpr int U = 8;
+    const uint32_t stride = blockDim.x;
+    for (uint32_t base = e_begin + threadIdx.x; base < e_end; base += stride * U) {
+        T tmp[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t e = base + u * stride;
+            if (e < e_end) tmp[u] = src[src_at(e)];
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t e = base + u * stride;
+            if (e < e_end) dst[dst_at(e)] = tmp[u];
+        }
+    }
+}
+
+#endif  // __CUDACC__
