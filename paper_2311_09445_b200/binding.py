@@ -1,0 +1,237 @@
+"""ctypes binding of libpearl_prb.so: argument marshalling only.
+
+Method names and arguments mirror the C ABI in include/pearl_prb.h.  torch supplies device
+memory and the stream; every step of the replay path runs in the library's CUDA kernels.
+There is no CPU fallback: if the library is missing or no CUDA device is present the
+constructor raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL = 1, 2, 4, 8, 16
+MAX_UPDATE_BATCH = 4096
+
+
+class PearlError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed: %s (%d)" % (what, _lib_error_string(code), code))
+        self.code = code
+
+
+class _Layout(C.Structure):
+    _fields_ = [("obs_bytes", C.c_uint32), ("act_bytes", C.c_uint32)]
+
+
+_lib = None
+
+# name -> (restype, argtypes); every symbol include/pearl_prb.h declares
+_vp, _u32, _u64, _f32, _i = C.c_void_p, C.c_uint32, C.c_uint64, C.c_float, C.c_int
+SIGNATURES = {
+    "pearl_prb_slab_bytes": (_u64, [_u64, _u32, C.POINTER(_Layout), _u32]),
+    "pearl_prb_create": (_i, [C.POINTER(_vp), _u64, _u32, C.POINTER(_Layout), _u32, _i, _vp, _vp, _u64]),
+    "pearl_prb_destroy": (_i, [_vp]),
+    "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
+    "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
+    "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample_host": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_update_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
+    "pearl_prb_sync": (_i, [_vp, C.POINTER(_u32)]),
+    "pearl_prb_info": (_i, [_vp, C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u32)]),
+    "pearl_prb_read_level": (_i, [_vp, _u32, _vp, _u64]),
+    "pearl_prb_level_alloc": (_u64, [_vp, _u32]),
+    "pearl_prb_read_rows": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_kernel_launches": (_u64, [_vp]),
+    "pearl_prb_error_string": (C.c_char_p, [_i]),
+}
+
+
+def load_library(path: Optional[str] = None):
+    """Loads libpearl_prb.so (built in-tree by build.py) and declares its signatures."""
+    global _lib
+    if _lib is None:
+        path = path or _build.LIB
+        if not os.path.exists(path):
+            raise ImportError("libpearl_prb.so is not built (%s); run paper_2311_09445_b200/build.py" % path)
+        lib = C.CDLL(path)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _lib_error_string(code: int) -> str:
+    try:
+        return load_library().pearl_prb_error_string(code).decode()
+    except Exception:
+        return "error"
+
+
+def _dptr(t: Optional[torch.Tensor], what: str):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA tensor" % what)
+    return C.c_void_p(t.data_ptr())
+
+
+def _hptr(t, what: str):
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous host tensor" % what)
+        return C.c_void_p(t.data_ptr())
+    return C.c_void_p(t.ctypes.data)      # numpy array
+
+
+def _row_bytes(t: torch.Tensor, n: int) -> int:
+    return t.numel() * t.element_size() // n
+
+
+class PrioritizedReplay:
+    """One prioritized replay buffer on one GPU.
+
+    capacity / fanout / obs_bytes / act_bytes / max_batch are pearl_prb_create's arguments.
+    Device memory is one torch uint8 slab; the handle enqueues on `stream` (default: the
+    current torch stream at construction).
+    """
+
+    def __init__(self, capacity: int, fanout: int, obs_bytes: int, act_bytes: int, max_batch: int,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        self._h = None
+        lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("PrioritizedReplay needs a CUDA device; there is no CPU path")
+        self.device = torch.device(device if device is not None else "cuda:%d" % torch.cuda.current_device())
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self.capacity, self.fanout, self.max_batch = capacity, fanout, max_batch
+        self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
+        lay = _Layout(obs_bytes, act_bytes)
+        need = lib.pearl_prb_slab_bytes(capacity, fanout, C.byref(lay), max_batch)
+        if need == 0:
+            raise PearlError(-7, "pearl_prb_slab_bytes")
+        self.slab_bytes = int(need)
+        self._slab = torch.empty(self.slab_bytes, dtype=torch.uint8, device=self.device)
+        h = C.c_void_p()
+        rc = lib.pearl_prb_create(C.byref(h), capacity, fanout, C.byref(lay), max_batch, self.device.index or 0,
+                                  C.c_void_p(self.stream.cuda_stream), C.c_void_p(self._slab.data_ptr()),
+                                  self.slab_bytes)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_create")
+        self._h = h
+        self.depth = self.info()[3]
+
+    # ---- the four calls, device buffers ------------------------------------------------
+    def insert(self, obs, act, rew, next_obs, done, prio) -> None:
+        n = prio.numel()
+        rc = load_library().pearl_prb_insert(self._h, n, _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                             _dptr(next_obs, "next_obs"), _dptr(done, "done"), _dptr(prio, "prio"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_insert")
+
+    def sample(self, B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None,
+               done=None) -> None:
+        rc = load_library().pearl_prb_sample(self._h, B, beta, seed, _dptr(idx, "idx"), _dptr(w, "w"),
+                                             _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                             _dptr(next_obs, "next_obs"), _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample")
+
+    def update(self, idx, td, alpha: float, eps: float) -> None:
+        rc = load_library().pearl_prb_update(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"), alpha, eps)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update")
+
+    def update_priorities(self, idx, prio) -> None:
+        rc = load_library().pearl_prb_update_priorities(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(prio, "prio"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update_priorities")
+
+    # ---- the same calls, host buffers (numpy arrays or host torch tensors) -----------------
+    def insert_host(self, obs, act, rew, next_obs, done, prio) -> None:
+        n = int(prio.shape[0])
+        rc = load_library().pearl_prb_insert_host(self._h, n, _hptr(obs, "obs"), _hptr(act, "act"), _hptr(rew, "rew"),
+                                                  _hptr(next_obs, "next_obs"), _hptr(done, "done"),
+                                                  _hptr(prio, "prio"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_insert_host")
+
+    def sample_host(self, B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None,
+                    done=None) -> None:
+        rc = load_library().pearl_prb_sample_host(self._h, B, beta, seed, _hptr(idx, "idx"), _hptr(w, "w"),
+                                                  _hptr(obs, "obs"), _hptr(act, "act"), _hptr(rew, "rew"),
+                                                  _hptr(next_obs, "next_obs"), _hptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample_host")
+
+    def update_host(self, idx, td, alpha: float, eps: float) -> None:
+        rc = load_library().pearl_prb_update_host(self._h, int(idx.shape[0]), _hptr(idx, "idx"), _hptr(td, "td"),
+                                                  alpha, eps)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update_host")
+
+    # ---- synchronisation and read-back -----------------------------------------------------
+    def sync(self) -> int:
+        st = C.c_uint32(0)
+        rc = load_library().pearl_prb_sync(self._h, C.byref(st))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sync")
+        return int(st.value)
+
+    def info(self):
+        f, c, n, d = C.c_uint64(), C.c_uint64(), C.c_uint64(), C.c_uint32()
+        rc = load_library().pearl_prb_info(self._h, C.byref(f), C.byref(c), C.byref(n), C.byref(d))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_info")
+        return f.value, c.value, n.value, d.value
+
+    def level_alloc(self, level: int) -> int:
+        return int(load_library().pearl_prb_level_alloc(self._h, level))
+
+    def read_level(self, level: int):
+        import numpy as np
+        n = self.level_alloc(level)
+        out = np.zeros(n, dtype=np.float32)
+        rc = load_library().pearl_prb_read_level(self._h, level, C.c_void_p(out.ctypes.data), n)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_read_level")
+        return out
+
+    def read_rows(self, idx):
+        import numpy as np
+        idx = np.ascontiguousarray(idx, dtype=np.int32)
+        n = idx.shape[0]
+        out = {"obs": np.zeros((n, self.obs_bytes), np.uint8), "act": np.zeros((n, self.act_bytes), np.uint8),
+               "rew": np.zeros(n, np.float32), "next_obs": np.zeros((n, self.obs_bytes), np.uint8),
+               "done": np.zeros(n, np.uint8)}
+        rc = load_library().pearl_prb_read_rows(self._h, _hptr(idx, "idx"), n, _hptr(out["obs"], "obs"),
+                                                _hptr(out["act"], "act"), _hptr(out["rew"], "rew"),
+                                                _hptr(out["next_obs"], "next_obs"), _hptr(out["done"], "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_read_rows")
+        return out
+
+    def kernel_launches(self) -> int:
+        return int(load_library().pearl_prb_kernel_launches(self._h))
+
+    def close(self) -> None:
+        if self._h is not None:
+            load_library().pearl_prb_destroy(self._h)
+            self._h = None
+            self._slab = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,417 @@
+// Host side of libpearl_prb: handle, device-memory layout, argument checks and the C ABI.
+// Every step of the replay path runs in the kernels of prb_insert.cu / prb_sample.cu /
+// prb_update.cu; this file only places memory and enqueues.
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/pearl_prb.h"
+#include "prb_internal.cuh"
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+
+inline uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+inline uint32_t granule_of(uint32_t bytes)
+{
+    uint32_t g = 16;
+    while (g > 1 && bytes % g != 0) g >>= 1;
+    return g;
+}
+
+// Offsets (bytes from the slab base) of every region of a buffer.
+struct Layout {
+    uint32_t depth;
+    uint64_t level_alloc[PRB_MAX_LEVELS];
+    uint64_t off_state;
+    uint64_t off_level[PRB_MAX_LEVELS];
+    uint64_t off_wraw;
+    uint64_t off_zero_end;                    // [0, off_zero_end) is zeroed at creation
+    uint64_t off_store[PRB_NUM_FIELDS];
+    uint64_t off_stage_in[PRB_NUM_FIELDS];    // staging of the *_host calls: inputs ...
+    uint64_t off_stage_prio, off_stage_idx, off_stage_td;
+    uint64_t off_stage_out[PRB_NUM_FIELDS];   // ... and outputs
+    uint64_t off_stage_out_idx, off_stage_out_w;
+    uint32_t field_bytes[PRB_NUM_FIELDS];
+    uint64_t total;
+};
+
+bool valid_fanout(uint32_t k) { return k == 2 || k == 4 || k == 8 || k == 16 || k == 32; }
+
+bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, uint32_t max_batch, Layout* L)
+{
+    if (!lay || !valid_fanout(fanout) || capacity < 1 || capacity > (1ull << 30) || max_batch < 1 ||
+        max_batch > (1u << 20))
+        return false;
+    uint32_t D = 1;
+    uint64_t span = fanout;
+    while (span < capacity) { span *= fanout; ++D; }
+    if (D >= PRB_MAX_LEVELS) return false;
+    L->depth = D;
+    uint64_t nodes[PRB_MAX_LEVELS];
+    nodes[D] = capacity;
+    for (int l = (int)D - 1; l >= 0; --l) nodes[l] = (nodes[l + 1] + fanout - 1) / fanout;
+    for (uint32_t l = 0; l <= D; ++l)
+        L->level_alloc[l] = (l == 0) ? 1 : (nodes[l] + fanout - 1) / fanout * fanout;
+
+    L->field_bytes[F_OBS] = lay->obs_bytes;
+    L->field_bytes[F_NEXT_OBS] = lay->obs_bytes;
+    L->field_bytes[F_ACT] = lay->act_bytes;
+    L->field_bytes[F_REW] = 4;
+    L->field_bytes[F_DONE] = 1;
+
+    uint64_t at = 0;
+    L->off_state = at; at = align_up(at + sizeof(PrbState));
+    for (uint32_t l = 0; l <= D; ++l) { L->off_level[l] = at; at = align_up(at + L->level_alloc[l] * sizeof(float)); }
+    L->off_wraw = at; at = align_up(at + (uint64_t)max_batch * sizeof(double));
+    L->off_zero_end = at;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_store[f] = at; at = align_up(at + capacity * L->field_bytes[f]); }
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_in[f] = at; at = align_up(at + (uint64_t)max_batch * L->field_bytes[f]); }
+    L->off_stage_prio = at; at = align_up(at + (uint64_t)max_batch * 4);
+    L->off_stage_idx = at; at = align_up(at + (uint64_t)max_batch * 4);
+    L->off_stage_td = at; at = align_up(at + (uint64_t)max_batch * 4);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_out[f] = at; at = align_up(at + (uint64_t)max_batch * L->field_bytes[f]); }
+    L->off_stage_out_idx = at; at = align_up(at + (uint64_t)max_batch * 4);
+    L->off_stage_out_w = at; at = align_up(at + (uint64_t)max_batch * 4);
+    L->total = at;
+    return true;
+}
+
+}  // namespace
+
+struct pearl_prb {
+    Layout lay;
+    PrbView view;
+    unsigned char* base;
+    bool owns_slab;
+    int device;
+    cudaStream_t stream;
+    uint32_t max_batch;
+    uint64_t launches;
+};
+
+namespace {
+
+inline bool misaligned(const void* p, uint32_t granule) { return ((uintptr_t)p & (granule - 1)) != 0; }
+
+int check_batch_ptrs(const pearl_prb* h, const void* const ptrs[PRB_NUM_FIELDS])
+{
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
+        if (ptrs[f] && h->view.field_bytes[f] && misaligned(ptrs[f], h->view.field_vec[f])) return PEARL_ERR_ALIGN;
+    return PEARL_OK;
+}
+
+struct DeviceGuard {
+    int prev;
+    bool ok;
+    explicit DeviceGuard(int dev) : prev(-1), ok(true)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline unsigned char* at(const pearl_prb* h, uint64_t off) { return h->base + off; }
+
+bool finite_nonneg(float x) { return isfinite(x) && x >= 0.0f; }
+
+}  // namespace
+
+extern "C" {
+
+uint64_t pearl_prb_slab_bytes(uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t max_batch)
+{
+    Layout L;
+    if (!make_layout(capacity, fanout, layout, max_batch, &L)) return 0;
+    return L.total;
+}
+
+int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
+                     uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
+{
+    if (!out || !layout) return PEARL_ERR_NULL;
+    if (!valid_fanout(fanout)) return PEARL_ERR_BAD_FANOUT;
+    if (max_batch < 1 || max_batch > (1u << 20)) return PEARL_ERR_BAD_BATCH;
+    Layout L;
+    if (!make_layout(capacity, fanout, layout, max_batch, &L)) return PEARL_ERR_BAD_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+
+    pearl_prb* h = new (std::nothrow) pearl_prb();
+    if (!h) return PEARL_ERR_OOM;
+    h->lay = L;
+    h->device = device;
+    h->stream = (cudaStream_t)cuda_stream;
+    h->max_batch = max_batch;
+    h->launches = 0;
+    if (slab) {
+        if (slab_bytes < L.total || ((uintptr_t)slab & (kAlign - 1))) { delete h; return slab_bytes < L.total ? PEARL_ERR_OOM : PEARL_ERR_ALIGN; }
+        h->base = (unsigned char*)slab;
+        h->owns_slab = false;
+    } else {
+        void* p = nullptr;
+        if (cudaMalloc(&p, L.total) != cudaSuccess) { cudaGetLastError(); delete h; return PEARL_ERR_OOM; }
+        h->base = (unsigned char*)p;
+        h->owns_slab = true;
+    }
+    if (cudaMemsetAsync(h->base, 0, L.off_zero_end, h->stream) != cudaSuccess) {
+        if (h->owns_slab) cudaFree(h->base);
+        delete h;
+        return PEARL_ERR_CUDA;
+    }
+    PrbView& v = h->view;
+    memset(&v, 0, sizeof(v));
+    v.state = (PrbState*)at(h, L.off_state);
+    for (uint32_t l = 0; l <= L.depth; ++l) v.level[l] = (float*)at(h, L.off_level[l]);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        v.store[f] = at(h, L.off_store[f]);
+        v.field_bytes[f] = L.field_bytes[f];
+        v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
+    }
+    v.wraw = (double*)at(h, L.off_wraw);
+    v.capacity = capacity;
+    v.fanout = fanout;
+    v.log2_fanout = 0;
+    while ((1u << v.log2_fanout) < fanout) ++v.log2_fanout;
+    v.depth = L.depth;
+    v.max_batch = max_batch;
+    *out = h;
+    return PEARL_OK;
+}
+
+int pearl_prb_destroy(pearl_prb_t* h)
+{
+    if (!h) return PEARL_ERR_NULL;
+    DeviceGuard guard(h->device);
+    int rc = PEARL_OK;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) rc = PEARL_ERR_CUDA;
+    if (h->owns_slab && cudaFree(h->base) != cudaSuccess) rc = PEARL_ERR_CUDA;
+    delete h;
+    return rc;
+}
+
+int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* d_act, const float* d_rew,
+                     const void* d_next_obs, const uint8_t* d_done, const float* d_prio)
+{
+    if (!h || !d_prio) return PEARL_ERR_NULL;
+    if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
+    int rc = check_batch_ptrs(h, ptrs);
+    if (rc != PEARL_OK) return rc;
+    if (misaligned(d_prio, 4)) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    PrbBatch b;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
+    const int k = prb_launch_insert(h->view, n, b, d_prio, h->stream);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
+}
+
+int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
+                     void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    if (!h || !d_idx) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (!finite_nonneg(beta)) return PEARL_ERR_BAD_ARG;
+    const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
+    int rc = check_batch_ptrs(h, ptrs);
+    if (rc != PEARL_OK) return rc;
+    if (misaligned(d_idx, 4) || (d_w && misaligned(d_w, 4))) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    PrbBatch b;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
+    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
+}
+
+static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_val, int raw, float alpha,
+                         float eps)
+{
+    if (!h || !d_idx || !d_val) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (!raw && (!finite_nonneg(alpha) || !finite_nonneg(eps))) return PEARL_ERR_BAD_ARG;
+    if (misaligned(d_idx, 4) || misaligned(d_val, 4)) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    const int k = prb_launch_update(h->view, B, d_idx, d_val, raw, alpha, eps, h->stream);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
+}
+
+int pearl_prb_update(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_td, float alpha, float eps)
+{
+    return update_common(h, B, d_idx, d_td, 0, alpha, eps);
+}
+
+int pearl_prb_update_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_prio)
+{
+    return update_common(h, B, d_idx, d_prio, 1, 0.0f, 0.0f);
+}
+
+// ---- host-buffer forms ---------------------------------------------------------------------
+
+int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const void* h_act, const float* h_rew,
+                          const void* h_next_obs, const uint8_t* h_done, const float* h_prio)
+{
+    if (!h || !h_prio) return PEARL_ERR_NULL;
+    if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    const void* src[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
+    void* dev[PRB_NUM_FIELDS];
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        dev[f] = nullptr;
+        const uint64_t bytes = (uint64_t)n * h->view.field_bytes[f];
+        if (!src[f] || bytes == 0) continue;
+        dev[f] = at(h, h->lay.off_stage_in[f]);
+        if (cudaMemcpyAsync(dev[f], src[f], bytes, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    }
+    float* d_prio = (float*)at(h, h->lay.off_stage_prio);
+    if (cudaMemcpyAsync(d_prio, h_prio, (uint64_t)n * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    int rc = pearl_prb_insert(h, n, dev[F_OBS], dev[F_ACT], (const float*)dev[F_REW], dev[F_NEXT_OBS],
+                              (const uint8_t*)dev[F_DONE], d_prio);
+    if (rc != PEARL_OK) return rc;
+    // the staging area is reused by the next host call: wait until this call's work has drained
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* h_idx, float* h_w, void* h_obs,
+                          void* h_act, float* h_rew, void* h_next_obs, uint8_t* h_done)
+{
+    if (!h || !h_idx) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    void* dst[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
+    void* dev[PRB_NUM_FIELDS];
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
+        dev[f] = (dst[f] && h->view.field_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
+    int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_out_idx);
+    float* d_w = h_w ? (float*)at(h, h->lay.off_stage_out_w) : nullptr;
+    int rc = pearl_prb_sample(h, B, beta, seed, d_idx, d_w, dev[F_OBS], dev[F_ACT], (float*)dev[F_REW],
+                              dev[F_NEXT_OBS], (uint8_t*)dev[F_DONE]);
+    if (rc != PEARL_OK) return rc;
+    if (cudaMemcpyAsync(h_idx, d_idx, (uint64_t)B * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (h_w && cudaMemcpyAsync(h_w, d_w, (uint64_t)B * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        if (!dev[f]) continue;
+        if (cudaMemcpyAsync(dst[f], dev[f], (uint64_t)B * h->view.field_bytes[f], cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+            return PEARL_ERR_CUDA;
+    }
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, const float* h_td, float alpha, float eps)
+{
+    if (!h || !h_idx || !h_td) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_idx);
+    float* d_td = (float*)at(h, h->lay.off_stage_td);
+    if (cudaMemcpyAsync(d_idx, h_idx, (uint64_t)B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (cudaMemcpyAsync(d_td, h_td, (uint64_t)B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    int rc = pearl_prb_update(h, B, d_idx, d_td, alpha, eps);
+    if (rc != PEARL_OK) return rc;
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+// ---- synchronisation and read-back ---------------------------------------------------------
+
+int pearl_prb_sync(pearl_prb_t* h, uint32_t* status_bits)
+{
+    if (!h) return PEARL_ERR_NULL;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    uint32_t st = 0;
+    if (cudaMemcpyAsync(&st, &h->view.state->status, 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (cudaMemsetAsync(&h->view.state->status, 0, 4, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (status_bits) *status_bits = st;
+    return PEARL_OK;
+}
+
+int pearl_prb_info(pearl_prb_t* h, uint64_t* fill, uint64_t* cursor, uint64_t* sample_calls, uint32_t* depth)
+{
+    if (!h) return PEARL_ERR_NULL;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    PrbState st;
+    if (cudaMemcpyAsync(&st, h->view.state, sizeof(st), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (fill) *fill = st.fill;
+    if (cursor) *cursor = st.cursor;
+    if (sample_calls) *sample_calls = st.sample_calls;
+    if (depth) *depth = h->view.depth;
+    return PEARL_OK;
+}
+
+uint64_t pearl_prb_level_alloc(pearl_prb_t* h, uint32_t level)
+{
+    if (!h || level > h->view.depth) return 0;
+    return h->lay.level_alloc[level];
+}
+
+int pearl_prb_read_level(pearl_prb_t* h, uint32_t level, float* h_dst, uint64_t count)
+{
+    if (!h || !h_dst) return PEARL_ERR_NULL;
+    if (level > h->view.depth || count > h->lay.level_alloc[level]) return PEARL_ERR_BAD_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    if (cudaMemcpyAsync(h_dst, h->view.level[level], count * sizeof(float), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+        return PEARL_ERR_CUDA;
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+int pearl_prb_read_rows(pearl_prb_t* h, const int32_t* h_idx, uint32_t n, void* h_obs, void* h_act, float* h_rew,
+                        void* h_next_obs, uint8_t* h_done)
+{
+    if (!h || !h_idx) return PEARL_ERR_NULL;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    void* dst[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
+    for (uint32_t k = 0; k < n; ++k)
+        if (h_idx[k] < 0 || (uint64_t)h_idx[k] >= h->view.capacity) return PEARL_ERR_BAD_ARG;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        const uint64_t fb = h->view.field_bytes[f];
+        if (!dst[f] || fb == 0) continue;
+        for (uint32_t k = 0; k < n; ++k) {
+            if (cudaMemcpyAsync((unsigned char*)dst[f] + k * fb, h->view.store[f] + (uint64_t)h_idx[k] * fb, fb,
+                                cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+                return PEARL_ERR_CUDA;
+        }
+    }
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+uint64_t pearl_prb_kernel_launches(pearl_prb_t* h) { return h ? h->launches : 0; }
+
+const char* pearl_prb_error_string(int code)
+{
+    switch (code) {
+    case PEARL_OK: return "ok";
+    case PEARL_ERR_NULL: return "a required pointer is NULL";
+    case PEARL_ERR_BAD_FANOUT: return "fanout must be 2, 4, 8, 16 or 32";
+    case PEARL_ERR_BAD_BATCH: return "batch is 0 or exceeds the maximum";
+    case PEARL_ERR_TOO_MANY: return "more rows than the capacity";
+    case PEARL_ERR_ALIGN: return "a pointer is misaligned for its row size";
+    case PEARL_ERR_OOM: return "out of device memory or slab too small";
+    case PEARL_ERR_BAD_ARG: return "a scalar argument is out of range or not finite";
+    case PEARL_ERR_CUDA: return "a CUDA runtime call failed";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"

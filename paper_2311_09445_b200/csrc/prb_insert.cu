@@ -22,50 +22,53 @@ struct InsertPlan {
     uint32_t chunks_per_row[PRB_NUM_FIELDS];  // > 0: row mode (CTA = one chunk of one row); 0: flat mode
 };
 
+// Row mode (rows of 16-byte granules, at least kRowMode of them): this CTA copies one chunk of
+// one row, contiguous on both sides.
+__device__ __forceinline__ void copy_row_chunk(const PrbView& v, int f, const PrbBatch& src, uint64_t cursor,
+                                               uint32_t local_cta, uint32_t chunks_per_row)
+{
+    const uint32_t W = v.field_bytes[f] / 16u;
+    const uint64_t N = v.capacity;
+    const uint32_t t = local_cta / chunks_per_row;
+    const uint32_t c = local_cta - t * chunks_per_row;
+    uint64_t slot = cursor + t;
+    if (slot >= N) slot -= N;
+    const uint32_t e0 = c * kTile;
+    const uint32_t cnt = min(W - e0, kTile);
+    prb_copy_span16<8>(reinterpret_cast<uint4*>(v.store[f]) + slot * W + e0,
+                       reinterpret_cast<const uint4*>(src.ptr[f]) + (uint64_t)t * W + e0, cnt);
+}
+
+// Flat mode: the tile is a range of the dense batch and may span many short rows.
 template <typename T>
-__device__ __forceinline__ void copy_field_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
-                                                uint64_t cursor, uint32_t local_cta, uint32_t chunks_per_row)
+__device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
+                                               uint64_t cursor, uint32_t local_cta)
 {
     const uint32_t W = v.field_bytes[f] / sizeof(T);
-    T* dst = reinterpret_cast<T*>(v.store[f]);
-    const T* s = reinterpret_cast<const T*>(src.ptr[f]);
     const uint64_t N = v.capacity;
-    if (chunks_per_row > 0) {
-        // row mode: this CTA copies one chunk of one row, no per-granule division
-        const uint32_t t = local_cta / chunks_per_row;
-        const uint32_t c = local_cta - t * chunks_per_row;
-        uint64_t slot = cursor + t;
-        if (slot >= N) slot -= N;
-        const uint32_t e0 = c * kTile;
-        const uint32_t e1 = min(W, e0 + kTile);
-        const uint64_t sbase = (uint64_t)t * W, dbase = slot * W;
-        prb_copy_granules<T>(dst, s, e0, e1,
-                             [=](uint32_t e) { return sbase + e; }, [=](uint32_t e) { return dbase + e; });
-    } else {
-        // flat mode: the tile is a range of the dense batch and may span many short rows
-        const uint64_t total = (uint64_t)n * W;
-        const uint64_t e0 = (uint64_t)local_cta * kTile;
-        const uint32_t e1 = (uint32_t)min(total, e0 + kTile);
-        prb_copy_granules<T>(dst, s, (uint32_t)e0, e1,
-                             [=](uint32_t e) { return (uint64_t)e; },
-                             [=](uint32_t e) {
-                                 const uint32_t r = e / W;
-                                 uint64_t slot = cursor + r;
-                                 if (slot >= N) slot -= N;
-                                 return slot * W + (e - r * W);
-                             });
-    }
+    const uint64_t total = (uint64_t)n * W;
+    const uint64_t e0 = (uint64_t)local_cta * kTile;
+    const uint32_t e1 = (uint32_t)min(total, e0 + kTile);
+    prb_copy_mapped<T>(reinterpret_cast<T*>(v.store[f]), reinterpret_cast<const T*>(src.ptr[f]), (uint32_t)e0, e1,
+                       [=](uint32_t e) { return (uint64_t)e; },
+                       [=](uint32_t e) {
+                           const uint32_t r = e / W;
+                           uint64_t slot = cursor + r;
+                           if (slot >= N) slot -= N;
+                           return slot * W + (e - r * W);
+                       });
 }
 
 __device__ __forceinline__ void copy_field_dispatch(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
                                                     uint64_t cursor, uint32_t local_cta, uint32_t cpr)
 {
+    if (cpr > 0) { copy_row_chunk(v, f, src, cursor, local_cta, cpr); return; }
     switch (v.field_vec[f]) {
-    case 16: copy_field_tile<uint4>(v, f, src, n, cursor, local_cta, cpr); break;
-    case 8: copy_field_tile<uint2>(v, f, src, n, cursor, local_cta, cpr); break;
-    case 4: copy_field_tile<uint32_t>(v, f, src, n, cursor, local_cta, cpr); break;
-    case 2: copy_field_tile<uint16_t>(v, f, src, n, cursor, local_cta, cpr); break;
-    default: copy_field_tile<uint8_t>(v, f, src, n, cursor, local_cta, cpr); break;
+    case 16: copy_flat_tile<uint4>(v, f, src, n, cursor, local_cta); break;
+    case 8: copy_flat_tile<uint2>(v, f, src, n, cursor, local_cta); break;
+    case 4: copy_flat_tile<uint32_t>(v, f, src, n, cursor, local_cta); break;
+    case 2: copy_flat_tile<uint16_t>(v, f, src, n, cursor, local_cta); break;
+    default: copy_flat_tile<uint8_t>(v, f, src, n, cursor, local_cta); break;
     }
 }
 
@@ -120,7 +123,7 @@ prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__
         insert_tree(v, n, prio, cursor);
     } else {
         const uint32_t cta = blockIdx.x - 1;
-#pragma unroll
+#pragma unroll 1
         for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
             if (cta >= plan.first_cta[f] && cta < plan.first_cta[f + 1])
                 copy_field_dispatch(v, f, src, n, cursor, cta - plan.first_cta[f], plan.chunks_per_row[f]);
@@ -155,7 +158,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         plan.chunks_per_row[f] = 0;
         if (v.field_bytes[f] == 0 || src.ptr[f] == nullptr) continue;
         const uint32_t W = v.field_bytes[f] / v.field_vec[f];
-        if (W >= kRowMode) {
+        if (v.field_vec[f] == 16 && W >= kRowMode) {
             plan.chunks_per_row[f] = (W + kTile - 1) / kTile;
             next += n * plan.chunks_per_row[f];
         } else {

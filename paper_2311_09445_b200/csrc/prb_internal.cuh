@@ -87,28 +87,37 @@ __device__ __forceinline__ bool prb_valid_priority(float p)
     return (p >= 0.0f) && (p <= 3.402823466e+38f);   // false for NaN, negative, +Inf
 }
 
-// Copies granules e in [e_begin, e_end) of a tile: granule e is read from src[src_at(e)] and
-// written to dst[dst_at(e)].  Each thread first issues up to 8 independent loads, then the
-// stores, with consecutive threads on consecutive granules.
-template <typename T, typename SrcAt, typename DstAt>
-__device__ __forceinline__ void prb_copy_granules(T* __restrict__ dst, const T* __restrict__ src,
-                                                  uint32_t e_begin, uint32_t e_end, SrcAt src_at, DstAt dst_at)
+// Contiguous copy of n 16-byte granules by all threads of the CTA (the bandwidth-critical path:
+// one chunk of a long row).  Each thread issues up to U independent loads before its stores;
+// consecutive threads touch consecutive granules.
+template <int U>
+__device__ __forceinline__ void prb_copy_span16(uint4* __restrict__ dst, const uint4* __restrict__ src, uint32_t n)
 {
-    constexpr int U = 8;
     const uint32_t stride = blockDim.x;
-    for (uint32_t base = e_begin + threadIdx.x; base < e_end; base += stride * U) {
-        T tmp[U];
+    for (uint32_t base = threadIdx.x; base < n; base += stride * U) {
+        uint4 tmp[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t e = base + u * stride;
-            if (e < e_end) tmp[u] = src[src_at(e)];
-        }
+        for (int u = 0; u < U; ++u)
+            if (base + u * stride < n) tmp[u] = __ldcs(src + base + u * stride);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t e = base + u * stride;
-            if (e < e_end) dst[dst_at(e)] = tmp[u];
-        }
+        for (int u = 0; u < U; ++u)
+            if (base + u * stride < n) __stcs(dst + base + u * stride, tmp[u]);
     }
+}
+
+// Copy of short rows: granule e of [0, n) is read from src[src_at(e)] and written to dst[dst_at(e)].
+template <typename T, typename SrcAt, typename DstAt>
+__device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __restrict__ src, uint32_t e_begin,
+                                                uint32_t e_end, SrcAt src_at, DstAt dst_at)
+{
+    const uint32_t stride = blockDim.x;
+    uint32_t e = e_begin + threadIdx.x;
+    for (; e + stride < e_end; e += 2 * stride) {
+        const T a = src[src_at(e)], b = src[src_at(e + stride)];
+        dst[dst_at(e)] = a;
+        dst[dst_at(e + stride)] = b;
+    }
+    if (e < e_end) dst[dst_at(e)] = src[src_at(e)];
 }
 
 #endif  // __CUDACC__

@@ -85,27 +85,28 @@ __device__ __forceinline__ void descend(const PrbView& v, double x, uint32_t lan
     leaf = (uint32_t)g;
 }
 
+// Row mode: this CTA (part `part` of its stratum) copies one chunk of the sampled row of field f.
+__device__ __forceinline__ void gather_row_chunk(const PrbView& v, int f, unsigned char* out, const SamplePlan& plan,
+                                                 uint32_t part, uint32_t k0, uint32_t leaf)
+{
+    if (part < plan.part_first[f] || part >= plan.part_first[f] + plan.parts[f]) return;
+    const uint32_t W = v.field_bytes[f] / 16u;
+    const uint32_t e0 = (part - plan.part_first[f]) * kTile;
+    const uint32_t cnt = min(W - e0, kTile);
+    prb_copy_span16<8>(reinterpret_cast<uint4*>(out) + (uint64_t)k0 * W + e0,
+                       reinterpret_cast<const uint4*>(v.store[f]) + (uint64_t)leaf * W + e0, cnt);
+}
+
+// Flat mode: the rows of all strata of this CTA, granule by granule.
 template <typename T>
-__device__ __forceinline__ void gather_field(const PrbView& v, int f, unsigned char* out, const SamplePlan& plan,
-                                             uint32_t part, uint32_t k0, uint32_t n_strata, const uint32_t* s_idx)
+__device__ __forceinline__ void gather_flat(const PrbView& v, int f, unsigned char* out, uint32_t k0,
+                                            uint32_t n_strata, const uint32_t* s_idx)
 {
     const uint32_t W = v.field_bytes[f] / sizeof(T);
-    const T* src = reinterpret_cast<const T*>(v.store[f]);
-    T* dst = reinterpret_cast<T*>(out);
-    if (plan.parts[f] > 0) {
-        if (part < plan.part_first[f] || part >= plan.part_first[f] + plan.parts[f]) return;
-        const uint32_t c = part - plan.part_first[f];
-        const uint32_t e0 = c * kTile, e1 = min(W, e0 + kTile);
-        const uint64_t sbase = (uint64_t)s_idx[0] * W, dbase = (uint64_t)k0 * W;
-        prb_copy_granules<T>(dst, src, e0, e1,
-                             [=](uint32_t e) { return sbase + e; }, [=](uint32_t e) { return dbase + e; });
-    } else {
-        if (part != 0) return;
-        const uint64_t dbase = (uint64_t)k0 * W;
-        prb_copy_granules<T>(dst, src, 0u, n_strata * W,
-                             [=](uint32_t e) { const uint32_t r = e / W; return (uint64_t)s_idx[r] * W + (e - r * W); },
-                             [=](uint32_t e) { return dbase + e; });
-    }
+    const uint64_t dbase = (uint64_t)k0 * W;
+    prb_copy_mapped<T>(reinterpret_cast<T*>(out), reinterpret_cast<const T*>(v.store[f]), 0u, n_strata * W,
+                       [=](uint32_t e) { const uint32_t r = e / W; return (uint64_t)s_idx[r] * W + (e - r * W); },
+                       [=](uint32_t e) { return dbase + e; });
 }
 
 template <int K>
@@ -171,15 +172,17 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         }
 
         // ---- gather: Data Storage rows of this CTA's strata ----
-#pragma unroll
+#pragma unroll 1
         for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
             if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
+            if (plan.parts[f] > 0) { gather_row_chunk(v, f, dst.ptr[f], plan, part, k0, s_idx[0]); continue; }
+            if (part != 0) continue;
             switch (v.field_vec[f]) {
-            case 16: gather_field<uint4>(v, f, dst.ptr[f], plan, part, k0, n_strata, s_idx); break;
-            case 8: gather_field<uint2>(v, f, dst.ptr[f], plan, part, k0, n_strata, s_idx); break;
-            case 4: gather_field<uint32_t>(v, f, dst.ptr[f], plan, part, k0, n_strata, s_idx); break;
-            case 2: gather_field<uint16_t>(v, f, dst.ptr[f], plan, part, k0, n_strata, s_idx); break;
-            default: gather_field<uint8_t>(v, f, dst.ptr[f], plan, part, k0, n_strata, s_idx); break;
+            case 16: gather_flat<uint4>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
+            case 8: gather_flat<uint2>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
+            case 4: gather_flat<uint32_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
+            case 2: gather_flat<uint16_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
+            default: gather_flat<uint8_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
             }
         }
     }
@@ -223,7 +226,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         plan.parts[f] = 0;
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
         const uint32_t W = v.field_bytes[f] / v.field_vec[f];
-        if (W >= kRowMode) {
+        if (v.field_vec[f] == 16 && W >= kRowMode) {
             row_mode = true;
             plan.part_first[f] = plan.S;
             plan.parts[f] = (W + kTile - 1) / kTile;
