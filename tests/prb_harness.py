@@ -1,0 +1,119 @@
+"""Drives the CPU oracle and the CUDA library with the same inputs and compares them.
+Integer/byte results and tree contents must match bit for bit; IS weights within 1e-5 relative."""
+import numpy as np
+import torch
+
+W_RTOL = 1e-5      # importance-sampling weights: relative tolerance (binary64 pow, two libraries)
+FIELDS = ("obs", "act", "rew", "next_obs", "done")
+
+
+def bits(a):
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+class Pair:
+    def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True):
+        from paper_2311_09445_b200 import PrioritizedReplay
+        self.gpu = PrioritizedReplay(capacity, fanout, obs_bytes, act_bytes, max_batch)
+        self.oracle_store = oracle_store
+        self.ora = oracle_mod.OraclePRB(capacity, fanout, obs_bytes if oracle_store else 0,
+                                        act_bytes if oracle_store else 0)
+        self.capacity, self.fanout = capacity, fanout
+        self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
+        self.dev = self.gpu.device
+        assert self.gpu.depth == self.ora.depth
+
+    def close(self):
+        self.gpu.close()
+        self.ora.close()
+
+    # ---- calls on both sides ----------------------------------------------------------
+    def insert(self, batch, dev_batch=None, host_call=False):
+        """batch: host arrays (obs, act, rew, next_obs, done, prio).  dev_batch: optional device tensors
+        to use on the GPU side instead of uploading `batch`."""
+        if self.oracle_store:
+            rc = self.ora.insert(batch.get("obs"), batch.get("act"), batch.get("rew"), batch.get("next_obs"),
+                                 batch.get("done"), batch["prio"])
+        else:
+            rc = self.ora.insert(None, None, batch.get("rew"), None, batch.get("done"), batch["prio"])
+        assert rc == 0
+        if host_call:
+            c = {k: (np.ascontiguousarray(v) if v is not None else None) for k, v in batch.items()}
+            self.gpu.insert_host(c.get("obs"), c.get("act"), c.get("rew"), c.get("next_obs"), c.get("done"), c["prio"])
+            return
+        if dev_batch is None:
+            dev_batch = {k: torch.from_numpy(np.ascontiguousarray(v)).to(self.dev) for k, v in batch.items()
+                         if v is not None}
+        self.gpu.insert(dev_batch.get("obs"), dev_batch.get("act"), dev_batch.get("rew"), dev_batch.get("next_obs"),
+                        dev_batch.get("done"), dev_batch["prio"])
+
+    def sample(self, B, beta, seed, check=True, host_call=False):
+        o = self.ora.sample(B, beta, seed, gather=self.oracle_store)
+        if host_call:
+            g = {"idx": np.full(B, -1, np.int32), "w": np.zeros(B, np.float32),
+                 "obs": np.zeros((B, self.obs_bytes), np.uint8), "act": np.zeros((B, self.act_bytes), np.uint8),
+                 "rew": np.zeros(B, np.float32), "next_obs": np.zeros((B, self.obs_bytes), np.uint8),
+                 "done": np.zeros(B, np.uint8)}
+            self.gpu.sample_host(B, beta, seed, g["idx"], g["w"], g["obs"], g["act"], g["rew"], g["next_obs"], g["done"])
+        else:
+            t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=self.dev),
+                 "w": torch.zeros(B, dtype=torch.float32, device=self.dev),
+                 "obs": torch.zeros((B, self.obs_bytes), dtype=torch.uint8, device=self.dev),
+                 "act": torch.zeros((B, self.act_bytes), dtype=torch.uint8, device=self.dev),
+                 "rew": torch.zeros(B, dtype=torch.float32, device=self.dev),
+                 "next_obs": torch.zeros((B, self.obs_bytes), dtype=torch.uint8, device=self.dev),
+                 "done": torch.zeros(B, dtype=torch.uint8, device=self.dev)}
+            self.gpu.sample(B, beta, seed, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+            torch.cuda.synchronize()
+            g = {k: v.cpu().numpy() for k, v in t.items()}
+        if check:
+            self.compare_sample(o, g)
+        return o, g
+
+    def compare_sample(self, o, g):
+        assert np.array_equal(o["idx"], g["idx"]), "sampled indices differ"
+        np.testing.assert_allclose(g["w"], o["w"], rtol=W_RTOL, atol=0)
+        if o["idx"][0] >= 0:
+            assert g["w"].max() == np.float32(1.0)
+        if self.oracle_store:
+            for f in FIELDS:
+                a, b = np.ascontiguousarray(o[f]).view(np.uint8), np.ascontiguousarray(g[f]).view(np.uint8)
+                assert np.array_equal(a.reshape(-1), b.reshape(-1)), "gathered %s differs" % f
+
+    def update(self, idx, td, alpha, eps, host_call=False):
+        assert self.ora.update(idx, td, alpha, eps) == 0
+        if host_call:
+            self.gpu.update_host(np.ascontiguousarray(idx, np.int32), np.ascontiguousarray(td, np.float32), alpha, eps)
+        else:
+            self.gpu.update(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                            torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps)
+
+    def update_priorities(self, idx, prio):
+        assert self.ora.update_priorities(idx, prio) == 0
+        self.gpu.update_priorities(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                                   torch.from_numpy(np.ascontiguousarray(prio, np.float32)).to(self.dev))
+
+    # ---- comparisons ------------------------------------------------------------------
+    def compare_tree(self, levels=None):
+        D = self.ora.depth
+        for l in (range(D + 1) if levels is None else levels):
+            a, b = self.ora.read_level(l), self.gpu.read_level(l)
+            assert a.shape == b.shape
+            if not np.array_equal(bits(a), bits(b)):
+                bad = np.nonzero(bits(a) != bits(b))[0]
+                raise AssertionError("tree level %d differs at %d entries, first %d: oracle %r gpu %r"
+                                     % (l, bad.size, bad[0], a[bad[0]], b[bad[0]]))
+
+    def compare_state(self):
+        assert self.gpu.info() == self.ora.info()
+
+    def compare_status(self):
+        s_g, s_o = self.gpu.sync(), self.ora.status()
+        assert s_g == s_o, "status bits differ: gpu %d oracle %d" % (s_g, s_o)
+        return s_g
+
+    def compare_rows(self, idx):
+        a, b = self.ora.read_rows(idx), self.gpu.read_rows(idx)
+        for f in FIELDS:
+            assert np.array_equal(np.ascontiguousarray(a[f]).view(np.uint8).reshape(-1),
+                                  np.ascontiguousarray(b[f]).view(np.uint8).reshape(-1)), f

@@ -1,0 +1,300 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from conftest import golden_lines
+from paper_2311_09445_b200 import workloads as wk
+from prb_harness import Pair
+
+pytestmark = pytest.mark.gpu
+
+P8 = np.array([3, 1, 4, 1, 5, 9, 2, 6], dtype=np.float32)
+FANOUTS = [2, 4, 8, 16, 32]
+
+
+def raw_fields(rng, n, obs_bytes, act_bytes):
+    return dict(obs=rng.integers(0, 256, size=(n, obs_bytes), dtype=np.uint8),
+                act=rng.integers(0, 256, size=(n, act_bytes), dtype=np.uint8),
+                rew=rng.standard_normal(n).astype(np.float32),
+                next_obs=rng.integers(0, 256, size=(n, obs_bytes), dtype=np.uint8),
+                done=rng.integers(0, 2, size=n, dtype=np.uint8))
+
+
+@pytest.mark.parametrize("K", [2, 4, 8])
+def test_hand_worked_tree(oracle_mod, K):
+    rows = golden_lines("eight_leaf_levels.txt")
+    pr = Pair(oracle_mod, 8, K, 0, 0, 16)
+    pr.insert(dict(prio=P8))
+    for case, k, level, *vals in rows:
+        if case == "init" and int(k) == K:
+            assert pr.gpu.read_level(int(level)).tolist() == [float(v) for v in vals]
+    pr.update_priorities(np.array([5, 5], np.int32), np.array([7.0, 2.0], np.float32))
+    for case, k, level, *vals in rows:
+        if case == "upd" and int(k) == K:
+            assert pr.gpu.read_level(int(level)).tolist() == [float(v) for v in vals]
+    pr.compare_tree()
+    pr.close()
+
+
+@pytest.mark.parametrize("K", FANOUTS)
+@pytest.mark.parametrize("N,obs_bytes,act_bytes", [(1, 16, 4), (7, 3, 1), (100, 68, 24), (1000, 16, 4), (4097, 40, 2)])
+def test_small_buffers_all_calls(oracle_mod, K, N, obs_bytes, act_bytes):
+    rng = np.random.default_rng(K * 10007 + N)
+    maxb = 300
+    pr = Pair(oracle_mod, N, K, obs_bytes, act_bytes, maxb)
+    # sampling an empty buffer
+    o, g = pr.sample(5, 0.4, 1)
+    assert g["idx"].tolist() == [-1] * 5
+    assert pr.compare_status() == 4
+    pr.compare_state()
+    inserted = 0
+    for step in range(12):
+        n = int(rng.integers(1, min(N, maxb) + 1))
+        b = raw_fields(rng, n, obs_bytes, act_bytes)
+        b["prio"] = (np.abs(rng.standard_normal(n)) + 1e-6).astype(np.float32) ** np.float32(0.6)
+        if step == 3:
+            b["prio"][0] = np.nan
+        pr.insert(b)
+        inserted += n
+        pr.compare_state()
+        pr.compare_tree()
+        B = int(rng.integers(1, maxb + 1))
+        o, g = pr.sample(B, 0.4, seed=77 + step)
+        fill = min(inserted, N)
+        idx = o["idx"].copy()
+        if B > 4:
+            idx[1] = idx[0]                # duplicates with different TD errors
+            idx[B // 2] = idx[B - 1]
+        if step % 3 == 1 and B > 6:
+            idx[2] = -1                    # invalid entries are skipped
+            idx[3] = fill
+        td = rng.standard_normal(B).astype(np.float32)
+        if step % 4 == 2:
+            td[B - 1] = np.inf
+        pr.update(idx, td, 0.6, 1e-6)
+        pr.compare_tree()
+        pr.compare_status()
+    pr.compare_rows(np.arange(min(inserted, N), dtype=np.int32))
+    pr.close()
+
+
+def test_tiny_workload_100_steps(oracle_mod):
+    wl = wk.TINY
+    rng = np.random.default_rng(wl.seed)
+    pr = Pair(oracle_mod, wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096)
+    pr.insert(wk.transitions(wl, rng, wl.capacity))
+    pr.compare_tree()
+    for step in range(wl.steps):
+        o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree()
+    pr.compare_state()
+    assert pr.compare_status() & ~8 == 0
+    pr.close()
+
+
+@pytest.mark.parametrize("wl,steps,prefill_chunk", [(wk.CARTPOLE, 60, 4096), (wk.DDPG, 40, 4096)])
+def test_full_size_mlp_workloads(oracle_mod, wl, steps, prefill_chunk):
+    rng = np.random.default_rng(wl.seed)
+    pr = Pair(oracle_mod, wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, prefill_chunk)
+    for first in range(0, wl.capacity, prefill_chunk):
+        pr.insert(wk.transitions(wl, rng, prefill_chunk, first))
+    pr.compare_tree()
+    pr.compare_state()
+    top = range(0, pr.ora.depth)
+    for step in range(steps):
+        pr.insert(wk.transitions(wl, rng, wl.n_insert))
+        o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        if wl.dup_frac:
+            assert len(set(idx.tolist())) < len(idx)
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree(None if step % 10 == 9 else top)
+    pr.compare_state()
+    assert pr.compare_status() & ~8 == 0
+    pr.compare_rows(rng.integers(0, wl.capacity, size=2000).astype(np.int32))
+    pr.close()
+
+
+def test_atari_shaped_reduced_capacity(oracle_mod):
+    # Full oracle mirror (storage included) at a capacity the host can hold; same row shape,
+    # fanout and batch as the Atari-shaped workload.
+    wl = wk.scaled(wk.ATARI, 2048)
+    rng = np.random.default_rng(wl.seed)
+    pr = Pair(oracle_mod, wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, 512)
+    next_id = 0
+    for _ in range(5):                       # 2560 rows: fills and wraps
+        pr.insert(wk.transitions(wl, rng, 512, next_id))
+        next_id += 512
+    pr.compare_tree()
+    for step in range(6):
+        pr.insert(wk.transitions(wl, rng, wl.n_insert if step % 2 == 0 else 100, next_id))
+        next_id += wl.n_insert if step % 2 == 0 else 100
+        o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree()
+    pr.compare_state()
+    pr.compare_rows(np.arange(0, 2048, 7, dtype=np.int32))
+    pr.close()
+
+
+def test_atari_shaped_full_size(oracle_mod):
+    # 2^19 slots x 56 457 B cannot be mirrored on the host: the oracle keeps the tree (and the
+    # small fields) only, and gathered observations are checked against rows regenerated from the
+    # global insert id of the sampled slot.  Launch configuration = the benchmark's.
+    wl = wk.ATARI
+    free, _ = torch.cuda.mem_get_info()
+    need = wl.capacity * wl.transition_bytes + (2 << 30)
+    if free < need:
+        pytest.skip("not enough free device memory for the full-size store")
+    rng = np.random.default_rng(wl.seed)
+    pr = Pair(oracle_mod, wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, 512, oracle_store=False)
+    dev = pr.dev
+    slot_id = np.full(wl.capacity, -1, dtype=np.int64)
+    next_id, cursor = 0, 0
+
+    def insert(n):
+        nonlocal next_id, cursor
+        small = wk.transitions(wl, rng, n, with_obs=False)
+        ids = torch.arange(next_id, next_id + n, dtype=torch.int64, device=dev)
+        d = {"obs": wk.counter_row_bytes(ids, 0, wl.obs_bytes), "next_obs": wk.counter_row_bytes(ids, 1, wl.obs_bytes)}
+        for k in ("act", "rew", "done", "prio"):
+            d[k] = torch.from_numpy(small[k]).to(dev)
+        pr.insert(dict(rew=small["rew"], done=small["done"], prio=small["prio"]), dev_batch=d)
+        slot_id[(cursor + np.arange(n)) % wl.capacity] = np.arange(next_id, next_id + n)
+        next_id += n
+        cursor = (cursor + n) % wl.capacity
+
+    for _ in range(wl.capacity // 512):
+        insert(512)
+    pr.compare_tree()
+    pr.compare_state()
+    for step in range(4):
+        insert(wl.n_insert)
+        o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)      # indices, weights checked inside
+        ids = torch.from_numpy(slot_id[o["idx"]])
+        assert np.array_equal(g["obs"], wk.counter_row_bytes(ids, 0, wl.obs_bytes).numpy())
+        assert np.array_equal(g["next_obs"], wk.counter_row_bytes(ids, 1, wl.obs_bytes).numpy())
+        rows = pr.ora.read_rows(o["idx"])
+        assert np.array_equal(g["rew"], rows["rew"]) and np.array_equal(g["done"], rows["done"])
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree()
+    pr.compare_state()
+    pr.close()
+
+
+@pytest.mark.parametrize("N,K,B", [(1 << 16, 2, 32), (1 << 16, 4, 1024), (1 << 16, 16, 4096), (1 << 18, 32, 256),
+                                   (1 << 20, 2, 4096), (1 << 22, 4, 1024), (1 << 22, 16, 16384), (1 << 22, 32, 65536)])
+def test_sweep_cells(oracle_mod, N, K, B):
+    wl = wk.sweep_cell(N, K, B, cell_id=N % 997 + K + B)
+    rng = np.random.default_rng(wl.seed)
+    chunk = 1 << 16
+    pr = Pair(oracle_mod, N, K, wl.obs_bytes, wl.act_bytes, max(chunk, B))
+    for first in range(0, N, chunk):
+        pr.insert(wk.transitions(wl, rng, chunk, first))
+    pr.compare_tree()
+    for step in range(3):
+        pr.insert(wk.transitions(wl, rng, wl.n_insert))
+        o, g = pr.sample(B, wl.beta, wl.philox_seed)
+        Bu = min(B, 4096)
+        idx, td = wk.update_batch(wl, rng, o["idx"][:Bu])
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree()
+    pr.compare_state()
+    pr.close()
+
+
+def test_priority_transform_bits(oracle_mod):
+    # The power is compared through the leaves it writes: 4096 TD errors x several exponents.
+    rng = np.random.default_rng(21)
+    N = 4096
+    pr = Pair(oracle_mod, N, 16, 0, 0, 4096)
+    pr.insert(dict(prio=np.ones(N, np.float32)))
+    idx = np.arange(N, dtype=np.int32)
+    for alpha, eps in [(0.6, 1e-6), (1.0, 0.0), (0.5, 1e-3), (0.0, 1e-6), (1.7, 1e-6), (0.123, 0.5)]:
+        td = np.concatenate([rng.standard_normal(N // 2), np.exp(2 * rng.standard_normal(N // 4)),
+                             rng.uniform(-1e-5, 1e-5, N // 4)]).astype(np.float32)
+        td[:4] = [0.0, -0.0, 1e-30, 3e38]
+        pr.update(idx, td, alpha, eps)
+        pr.compare_tree()
+        leaves = pr.gpu.read_level(pr.gpu.depth)[:N]
+        for i in (0, 5, 100, 4095):
+            assert leaves[i] == oracle_mod.priority_pow(td[i], eps, alpha)
+    pr.compare_status()
+    pr.close()
+
+
+def test_host_buffer_calls(oracle_mod):
+    wl = wk.scaled(wk.DDPG, 5000)
+    rng = np.random.default_rng(5)
+    pr = Pair(oracle_mod, wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, 1024)
+    for _ in range(7):
+        pr.insert(wk.transitions(wl, rng, 1000), host_call=True)
+        o, g = pr.sample(256, 0.4, 9, host_call=True)
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, 0.6, 1e-6, host_call=True)
+        pr.compare_tree()
+    pr.compare_state()
+    pr.close()
+
+
+def test_update_is_deterministic(oracle_mod):
+    # The same batch with many duplicates, replayed: identical tree bytes every time.
+    rng = np.random.default_rng(13)
+    N = 50_000
+    pr = Pair(oracle_mod, N, 8, 0, 0, 4096)
+    pr.insert(dict(prio=rng.uniform(0.1, 1, 4096).astype(np.float32)))
+    for _ in range(12):
+        pr.insert(dict(prio=rng.uniform(0.1, 1, 4096).astype(np.float32)))
+    idx = rng.integers(0, 300, size=4096).astype(np.int32)
+    td = rng.standard_normal(4096).astype(np.float32)
+    pr.update(idx, td, 0.6, 1e-6)
+    ref = [pr.gpu.read_level(l).copy() for l in range(pr.gpu.depth + 1)]
+    pr.compare_tree()
+    for _ in range(20):
+        pr.gpu.update(torch.from_numpy(idx).to(pr.dev), torch.from_numpy(td).to(pr.dev), 0.6, 1e-6)
+        for l, r in enumerate(ref):
+            assert np.array_equal(pr.gpu.read_level(l).view(np.uint32), r.view(np.uint32))
+    pr.close()
+
+
+def test_argument_errors_leave_state_untouched(oracle_mod):
+    from paper_2311_09445_b200 import PearlError
+    pr = Pair(oracle_mod, 64, 4, 16, 4, 32)
+    rng = np.random.default_rng(1)
+    b = raw_fields(rng, 32, 16, 4)
+    b["prio"] = rng.uniform(0.5, 1, 32).astype(np.float32)
+    pr.insert(b)
+    dev = pr.dev
+    idx = torch.zeros(64, dtype=torch.int32, device=dev)
+    td = torch.zeros(64, dtype=torch.float32, device=dev)
+    before = [pr.gpu.read_level(l).copy() for l in range(pr.gpu.depth + 1)]
+    with pytest.raises(PearlError) as e:
+        pr.gpu.sample(33, 0.4, 0, idx)                       # B > max_batch
+    assert e.value.code == -3
+    with pytest.raises(PearlError) as e:
+        pr.gpu.sample(0, 0.4, 0, idx)
+    assert e.value.code == -3
+    with pytest.raises(PearlError) as e:
+        pr.gpu.sample(8, float("nan"), 0, idx)
+    assert e.value.code == -7
+    with pytest.raises(PearlError) as e:
+        pr.gpu.update(idx[:8], td[:8], -0.5, 1e-6)
+    assert e.value.code == -7
+    with pytest.raises(PearlError) as e:
+        pr.gpu.sample(8, 0.4, 0, idx, obs=torch.zeros(8 * 16 + 16, dtype=torch.uint8, device=dev)[4:4 + 8 * 16])
+    assert e.value.code == -5                                # misaligned 16-byte rows
+    big = Pair(oracle_mod, 16, 2, 0, 0, 32)
+    with pytest.raises(PearlError) as e:
+        big.gpu.insert(None, None, None, None, None, torch.ones(17, device=dev))
+    assert e.value.code == -4                                # n > capacity
+    big.close()
+    for l, r in enumerate(before):
+        assert np.array_equal(pr.gpu.read_level(l), r)
+    pr.compare_state()
+    assert pr.gpu.kernel_launches() == 1
+    pr.close()
