@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the prioritized-replay hot path: one step = insert + sample (indices, IS weights,
+gather) + priority update on one batch of synthetic transitions.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is sampled-and-updated transitions per second through
+the whole step with all inputs resident in device memory; `e2e` is the same through the
+host-buffer calls (host->device and device->host copies inside the timed region); `roofline`
+is the achieved fraction of the measured HBM copy bandwidth of the sample+gather kernel;
+`cpu_baseline` is the CPU oracle timed on this machine's host cores on a bounded sample.
+With N > 1 every rank runs an independent replica (the buffer does not shard); time is the
+maximum over ranks.  `--impl reference` times the CPU oracle instead of the CUDA library.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "PRB sample+update transitions/s at batch B"
+UNIT = "transitions/s"
+ROTATE = 8           # distinct input/output batch buffers cycled through, so inputs exceed L2 where rows are long
+FALLBACK_HBM_GBS = 6650.0
+
+
+def load_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle arm (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------
+def oracle_capacity(wl):
+    """Capacity the oracle is timed at: the workload's, unless its store would not fit the host."""
+    cap = wl.capacity
+    while cap * wl.transition_bytes > (6 << 30):
+        cap //= 2
+    return cap
+
+
+def oracle_setup(wl, capacity):
+    import oracle
+    from paper_2311_09445_b200 import workloads as wk
+    oracle.build()
+    rng = np.random.default_rng(wl.seed)
+    o = oracle.OraclePRB(capacity, wl.fanout, wl.obs_bytes, wl.act_bytes)
+    plain = wk.scaled(wl, capacity, counter_rows=False)      # same shapes; bytes from numpy (content is irrelevant to time)
+    chunk = max(1, min(capacity, (64 << 20) // wl.transition_bytes))
+    for first in range(0, capacity, chunk):
+        b = wk.transitions(plain, rng, min(chunk, capacity - first))
+        o.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+    batches = [wk.transitions(plain, rng, max(wl.n_insert, 1)) for _ in range(ROTATE)]
+    tds = [wk.td_errors(wl, rng, wl.batch) for _ in range(ROTATE)]
+    return o, plain, batches, tds, rng
+
+
+def oracle_step(o, wl, batches, tds, rng, i):
+    from paper_2311_09445_b200 import workloads as wk
+    if wl.n_insert:
+        b = batches[i % ROTATE]
+        o.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+    out = o.sample(wl.batch, wl.beta, wl.philox_seed)
+    idx = out["idx"]
+    if wl.dup_frac:
+        idx, _ = wk.update_batch(wl, rng, idx)
+    o.update(idx, tds[i % ROTATE], wl.alpha, wl.eps)
+
+
+def time_oracle(wl, steps, warmup, budget_s=None):
+    cap = oracle_capacity(wl)
+    o, plain, batches, tds, rng = oracle_setup(wl, cap)
+    for i in range(warmup):
+        oracle_step(o, wl, batches, tds, rng, i)
+    t0 = time.perf_counter()
+    done = 0
+    for i in range(steps):
+        oracle_step(o, wl, batches, tds, rng, i)
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    o.close()
+    sample = "%d steps of the %s step (insert %d, sample %d, update %d)" % (done, wl.name, wl.n_insert, wl.batch, wl.batch)
+    if cap != wl.capacity:
+        sample += " at capacity %d of %d (host memory)" % (cap, wl.capacity)
+    return done, dt, sample
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            p = [t.strip() for t in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------
+def device_batches(wl, rng, dev, n, count, first_id):
+    """`count` insert batches of n transitions resident on the device."""
+    import torch
+    from paper_2311_09445_b200 import workloads as wk
+    out = []
+    for r in range(count):
+        if wl.counter_rows:
+            small = wk.transitions(wl, rng, n, with_obs=False)
+            ids = torch.arange(first_id + r * n, first_id + (r + 1) * n, dtype=torch.int64, device=dev)
+            d = {"obs": wk.counter_row_bytes(ids, 0, wl.obs_bytes), "next_obs": wk.counter_row_bytes(ids, 1, wl.obs_bytes)}
+            for k in ("act", "rew", "done", "prio"):
+                d[k] = torch.from_numpy(small[k]).to(dev)
+        else:
+            d = wk.to_device(wk.transitions(wl, rng, n), dev)
+        out.append(d)
+    return out
+
+
+def out_buffers(wl, dev, B, pinned=False):
+    import torch
+    kw = dict(device="cpu", pin_memory=True) if pinned else dict(device=dev)
+    return {"idx": torch.zeros(B, dtype=torch.int32, **kw), "w": torch.zeros(B, dtype=torch.float32, **kw),
+            "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, **kw),
+            "act": torch.zeros((B, max(wl.act_bytes, 1)), dtype=torch.uint8, **kw),
+            "rew": torch.zeros(B, dtype=torch.float32, **kw),
+            "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, **kw),
+            "done": torch.zeros(B, dtype=torch.uint8, **kw)}
+
+
+def time_loop(stream, fn, iters):
+    """Milliseconds for `iters` calls of fn(i), CUDA events on `stream`, synchronised on both sides."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(iters):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args, wl, rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2311_09445_b200 import PrioritizedReplay
+    from paper_2311_09445_b200 import workloads as wk
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda:%d" % local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    stream = torch.cuda.Stream(dev)
+    rng = np.random.default_rng(wl.seed + 7919 * rank)
+    B, n_ins = wl.batch, wl.n_insert
+    chunk = 512 if wl.counter_rows else min(wl.capacity, 1 << 16)
+    max_batch = max(B, n_ins, chunk)
+
+    with torch.cuda.stream(stream):
+        prb = PrioritizedReplay(wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, max_batch, device=dev, stream=stream)
+        # prefill the whole ring through the insert call
+        filled = 0
+        while filled < wl.capacity:
+            n = min(chunk, wl.capacity - filled)
+            b = device_batches(wl, rng, dev, n, 1, filled)[0]
+            prb.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+            filled += n
+        torch.cuda.synchronize()
+        batches = device_batches(wl, rng, dev, max(n_ins, 1), ROTATE, wl.capacity)
+        outs = [out_buffers(wl, dev, B) for _ in range(ROTATE)]
+        tds = [torch.from_numpy(wk.td_errors(wl, rng, B)).to(dev) for _ in range(ROTATE)]
+        n_dup = int(round(wl.dup_frac * B))
+        dup_pos = [torch.from_numpy(rng.choice(B, size=n_dup, replace=False)).to(dev) for _ in range(ROTATE)] if n_dup else None
+        dup_src = [torch.from_numpy(rng.integers(0, B, size=n_dup)).to(dev) for _ in range(ROTATE)] if n_dup else None
+
+        def do_insert(i):
+            b = batches[i % ROTATE]
+            prb.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+
+        def do_sample(i):
+            o = outs[i % ROTATE]
+            prb.sample(B, wl.beta, wl.philox_seed, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
+                       o["rew"], o["next_obs"], o["done"])
+
+        def do_update(i):
+            o = outs[i % ROTATE]
+            if n_dup:
+                o["idx"][dup_pos[i % ROTATE]] = o["idx"][dup_src[i % ROTATE]]
+            prb.update(o["idx"], tds[i % ROTATE], wl.alpha, wl.eps)
+
+        def eager_step(i):
+            if n_ins:
+                do_insert(i)
+            do_sample(i)
+            do_update(i)
+
+        for i in range(max(args.warmup, 3)):
+            eager_step(i)
+        torch.cuda.synchronize()
+        status = prb.sync()
+
+        # one CUDA graph per rotation slot (all buffer state lives on the device, so replays advance it)
+        graphs, kernels_per_step = None, None
+        l0 = prb.kernel_launches()
+        eager_step(0)
+        kernels_per_step = prb.kernel_launches() - l0
+        torch.cuda.synchronize()
+        if not args.no_graph:
+            graphs = []
+            for r in range(ROTATE):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    eager_step(r)
+                graphs.append(g)
+            step = lambda i: graphs[i % ROTATE].replay()
+        else:
+            step = eager_step
+        for i in range(max(args.warmup, 3)):
+            step(i)
+        torch.cuda.synchronize()
+
+        # ---- the timed region: exactly K steps -------------------------------------------
+        clocks = ClockSampler(local)
+        if rank == 0:
+            clocks.start()
+            time.sleep(0.3)
+        if world > 1:
+            dist.barrier()
+        ms = time_loop(stream, step, args.steps)
+        if world > 1:
+            dist.barrier()
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        clk = clocks.stop() if rank == 0 else None
+
+        # ---- per-call timings (device resident), used for the roofline and the rates -------
+        reps = max(20, min(args.steps, 400))
+        for i in range(3):
+            do_sample(i)
+        ms_sample = time_loop(stream, do_sample, reps) / reps
+        ms_update = time_loop(stream, do_update, reps) / reps
+        ms_insert = time_loop(stream, do_insert, reps) / reps if n_ins else None
+        status |= prb.sync()
+
+        # ---- end to end through the host-buffer calls ----------------------------------------
+        e2e_steps = max(5, min(args.steps, 100 if wl.counter_rows else 500))
+        hb = []
+        for r in range(ROTATE):
+            d = batches[r]
+            hb.append({k: v.cpu().pin_memory() for k, v in d.items()})
+        ho = out_buffers(wl, dev, B, pinned=True)
+        htd = [t.cpu().pin_memory() for t in tds]
+
+        def e2e_step(i):
+            if n_ins:
+                b = hb[i % ROTATE]
+                prb.insert_host(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+            prb.sample_host(B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
+                            ho["rew"], ho["next_obs"], ho["done"])
+            prb.update_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps)
+
+        for i in range(3):
+            e2e_step(i)
+        if world > 1:
+            dist.barrier()
+        ms_e2e = time_loop(stream, e2e_step, e2e_steps)
+        if world > 1:
+            dist.barrier()
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        status |= prb.sync()
+        fill, cursor, calls, depth = prb.info()
+        prb.close()
+
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return None
+
+    E = wl.transition_bytes
+    h2d = (n_ins * (E + 4) if n_ins else 0) + B * 8
+    d2h = B * (E + 8)
+    peak, peak_kind = load_peak()
+    # algorithmic bytes of one sample launch: D child groups of K binary32 per stratum, index and
+    # weight written, every field of the row read once and written once
+    sample_bytes = B * (depth * wl.fanout * 4 + 8 + 2 * E)
+    achieved = sample_bytes / (ms_sample * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * B * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
+        "config": {"workload": wl.name, "capacity": wl.capacity, "fanout": wl.fanout, "depth": depth, "batch": B,
+                   "insert_per_step": n_ins, "transition_bytes": E, "step": "insert+sample(idx,IS,gather)+update",
+                   "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph,
+                   "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
+        "rates": {"samples_per_s": B / (ms_sample * 1e-3), "updates_per_s": B / (ms_update * 1e-3),
+                  "inserts_per_s": (n_ins / (ms_insert * 1e-3)) if n_ins else None,
+                  "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3,
+                  "us_insert": ms_insert * 1e3 if n_ins else None},
+        "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+                     "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes, "traffic": None},
+        "e2e": {"value": world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(kernels_per_step * args.steps),
+        "kernels_per_step": int(kernels_per_step),
+        "status_bits": int(status),
+        "clocks": clk,
+    }
+    if n_ins:
+        ins_bytes = n_ins * (2 * E + 4)
+        line["roofline_insert"] = {"kernel": "prb_insert_kernel", "bound": "hbm", "bytes_per_launch": ins_bytes,
+                                   "achieved": ins_bytes / (ms_insert * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": ins_bytes / (ms_insert * 1e-3) / 1e9 / peak}
+    if world == 1 and not args.no_cpu_baseline:
+        done, dt, sample = time_oracle(wl, 10 ** 9, 2, budget_s=args.cpu_budget)
+        line["cpu_baseline"] = {"value": B * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                                "host_cpus": os.cpu_count()}
+    return line
+
+
+def run_reference(args, wl, rank, world):
+    """The CPU oracle as it stands, on this machine's host cores; rank 0 only."""
+    if rank != 0:
+        return None
+    warm = max(args.warmup, 1)
+    per_step_guess = 0.03 if wl.counter_rows else 0.001
+    steps = max(1, min(args.steps, int(120 / per_step_guess)))
+    done, dt, sample = time_oracle(wl, steps, warm, budget_s=150)
+    v = wl.batch * done / dt
+    return {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world, "steps": done,
+            "warmup": warm, "ms_per_step": dt / done * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
+            "config": {"workload": wl.name, "capacity": oracle_capacity(wl), "fanout": wl.fanout, "batch": wl.batch,
+                       "insert_per_step": wl.n_insert, "step": "insert+sample(idx,IS,gather)+update"},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="atari_dqn")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
+    args = ap.parse_args()
+
+    from paper_2311_09445_b200 import workloads as wk
+    wl = wk.WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    line = run_reference(args, wl, rank, world) if args.impl == "reference" else run_ours(args, wl, rank, world)
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
