@@ -136,6 +136,39 @@ int pearl_prb_sample_host(pearl_prb_t* prb, uint32_t B, float beta, uint64_t see
 int pearl_prb_update_host(pearl_prb_t* prb, uint32_t B, const int32_t* h_idx, const float* h_td,
                           float alpha, float eps);
 
+/* Largest batch pearl_prb_sample_static_scratch accepts. */
+#define PEARL_STATIC_SCRATCH_MAX_BATCH 4096u
+
+/* pearl_prb_sample with its per-call scratch in library-owned static device memory.
+ * (The paper has no counterpart; this exists for callers that cannot allocate.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- a plug-in inside a
+ * framework whose memory pool has already claimed the whole GPU, so that a cudaMalloc would fail
+ * or fragment it; a real-time control or serving loop whose rules forbid allocator calls after
+ * start-up; a process whose handle was built on a caller-provided slab sized without the sample
+ * call's scratch.  Such a caller hands in the same inputs and outputs as pearl_prb_sample, and the
+ * kernel's scratch (the batch's raw, un-normalised importance-sampling weights, one binary64 per
+ * stratum) lives in a fixed 32 KiB array that is part of the library image: every GPU on which
+ * the library runs this call holds that array until the process exits, whether or not it is used
+ * again.  The call itself performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ * Arguments, outputs, ordering on the handle's stream and error codes are those of
+ * pearl_prb_sample, except that B > PEARL_STATIC_SCRATCH_MAX_BATCH returns PEARL_ERR_BAD_BATCH
+ * ("batch is 0 or exceeds the maximum") and nothing is enqueued.
+ *
+ * Set-up: the first call on each device looks up the array's device address (one runtime query,
+ * made with that device current, remembered afterwards).  Make that first call outside any
+ * stream capture.
+ *
+ * Sharing: all handles and all streams of a device use the same array, and it keeps whatever the
+ * last call left in it.  Nothing in it has to start at zero -- every entry the kernel reads was
+ * written earlier in the same call -- so it is not cleared.  Two of these calls that overlap on
+ * one GPU (different streams, or different handles on different streams) race on the array and
+ * produce wrong weights; keep them ordered on one stream or serialise them yourself. */
+int pearl_prb_sample_static_scratch(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed,
+                                    int32_t* d_idx, float* d_w, void* d_obs, void* d_act,
+                                    float* d_rew, void* d_next_obs, uint8_t* d_done);
+
 /* Waits for the stream; returns the accumulated PEARL_ST_* bits in *status_bits (may be NULL)
  * and clears them. */
 int pearl_prb_sync(pearl_prb_t* prb, uint32_t* status_bits);

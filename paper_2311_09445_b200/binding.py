@@ -39,6 +39,7 @@ SIGNATURES = {
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
     "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -146,6 +147,17 @@ class PrioritizedReplay:
                                              _dptr(next_obs, "next_obs"), _dptr(done, "done"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_sample")
+
+    def sample_static_scratch(self, B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None,
+                              next_obs=None, done=None) -> None:
+        """pearl_prb_sample_static_scratch: the sample call for callers that cannot allocate device
+        memory (B <= 4096); its scratch is a static array inside the library, shared by every
+        handle on the device, so overlapping calls on one GPU race."""
+        rc = load_library().pearl_prb_sample_static_scratch(self._h, B, beta, seed, _dptr(idx, "idx"), _dptr(w, "w"),
+                                                            _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                                            _dptr(next_obs, "next_obs"), _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample_static_scratch")
 
     def update(self, idx, td, alpha: float, eps: float) -> None:
         rc = load_library().pearl_prb_update(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"), alpha, eps)

@@ -328,6 +328,54 @@ int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, cons
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }
 
+// ---- sampling with static scratch --------------------------------------------------------------
+// Scratch of the sample kernel (raw importance-sampling weights) for callers that cannot
+// allocate: a fixed array in the library image instead of the handle's slab.  In host code the
+// name below is only a stand-in for the symbol; the device address comes from
+// cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) double g_static_wraw[PEARL_STATIC_SCRATCH_MAX_BATCH];
+
+namespace {
+constexpr int kMaxDevices = 64;
+double* g_static_wraw_addr[kMaxDevices];   // per device ordinal; nullptr until the first call there
+
+// Device address of g_static_wraw on `device` (which must be current); nullptr on failure.
+double* static_wraw_on(int device)
+{
+    if (device < 0 || device >= kMaxDevices) return nullptr;
+    if (g_static_wraw_addr[device] == nullptr) {
+        double* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_static_wraw) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        g_static_wraw_addr[device] = p;
+    }
+    return g_static_wraw_addr[device];
+}
+}  // namespace
+
+int pearl_prb_sample_static_scratch(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
+                                    void* d_obs, void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    if (!h || !d_idx) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch || B > PEARL_STATIC_SCRATCH_MAX_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (!finite_nonneg(beta)) return PEARL_ERR_BAD_ARG;
+    const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
+    int rc = check_batch_ptrs(h, ptrs);
+    if (rc != PEARL_OK) return rc;
+    if (misaligned(d_idx, 4) || (d_w && misaligned(d_w, 4))) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    double* scratch = static_wraw_on(h->device);
+    if (!scratch) return PEARL_ERR_CUDA;
+    PrbView v = h->view;          // same tree, store and state; only the scratch pointer differs
+    v.wraw = scratch;
+    PrbBatch b;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
+    const int k = prb_launch_sample(v, B, beta, seed, d_idx, d_w, b, h->stream);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
+}
+
 // ---- synchronisation and read-back ---------------------------------------------------------
 
 int pearl_prb_sync(pearl_prb_t* h, uint32_t* status_bits)
