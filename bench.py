@@ -311,11 +311,11 @@ def run_ours(args, wl, rank, world):
                             ho["rew"], ho["next_obs"], ho["done"])
             prb.update_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps)
 
-        for i in range(3):
+        for i in range(0 if args.no_e2e else 3):
             e2e_step(i)
         if world > 1:
             dist.barrier()
-        ms_e2e = time_loop(stream, e2e_step, e2e_steps)
+        ms_e2e = time_loop(stream, e2e_step, e2e_steps) if not args.no_e2e else float("nan")
         if world > 1:
             dist.barrier()
             t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
@@ -354,7 +354,7 @@ def run_ours(args, wl, rank, world):
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes, "traffic": None},
-        "e2e": {"value": world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
+        "e2e": {"value": None if args.no_e2e else world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(kernels_per_step * args.steps),
         "kernels_per_step": int(kernels_per_step),
@@ -401,11 +401,15 @@ def main():
     ap.add_argument("--workload", default="atari_dqn")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
     args = ap.parse_args()
 
     from paper_2311_09445_b200 import workloads as wk
     wl = wk.WORKLOADS[args.workload]
+    if args.capacity:
+        wl = wk.scaled(wl, args.capacity)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     line = run_reference(args, wl, rank, world) if args.impl == "reference" else run_ours(args, wl, rank, world)
