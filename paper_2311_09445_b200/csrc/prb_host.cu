@@ -166,7 +166,10 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
     PrbView& v = h->view;
     memset(&v, 0, sizeof(v));
     v.state = (PrbState*)at(h, L.off_state);
-    for (uint32_t l = 0; l <= L.depth; ++l) v.level[l] = (float*)at(h, L.off_level[l]);
+    for (uint32_t l = 0; l <= L.depth; ++l) {
+        v.level[l] = (float*)at(h, L.off_level[l]);
+        v.level_alloc[l] = (uint32_t)L.level_alloc[l];
+    }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         v.store[f] = at(h, L.off_store[f]);
         v.field_bytes[f] = L.field_bytes[f];

@@ -14,40 +14,27 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr uint32_t kTile = kThreads * 8;   // granules per copy tile
-constexpr uint32_t kRowMode = 512;         // rows of at least this many granules get CTAs of their own
+constexpr int kCtasPerSm = 4;
+constexpr uint32_t kChunk = kThreads * 4;  // upper bound on granules per chunk of a long row
+constexpr uint32_t kTile = kThreads * 8;   // granules per tile of short rows
+constexpr uint32_t kRowMode = 512;         // rows of at least this many 16-byte granules are split into chunks
 
+// The copy is cut into tasks, numbered field by field; every copy CTA takes a contiguous range.
 struct InsertPlan {
-    uint32_t first_cta[PRB_NUM_FIELDS + 1];   // copy CTAs of field f: [first_cta[f], first_cta[f+1])
-    uint32_t chunks_per_row[PRB_NUM_FIELDS];  // > 0: row mode (CTA = one chunk of one row); 0: flat mode
+    uint32_t first_task[PRB_NUM_FIELDS + 1];  // tasks of field f: [first_task[f], first_task[f+1])
+    uint32_t chunks[PRB_NUM_FIELDS];          // > 0: long rows, task = one chunk of one row; 0: short rows, task = one tile
+    uint32_t chunk[PRB_NUM_FIELDS];           // granules per chunk
 };
 
-// Row mode (rows of 16-byte granules, at least kRowMode of them): this CTA copies one chunk of
-// one row, contiguous on both sides.
-__device__ __forceinline__ void copy_row_chunk(const PrbView& v, int f, const PrbBatch& src, uint64_t cursor,
-                                               uint32_t local_cta, uint32_t chunks_per_row)
-{
-    const uint32_t W = v.field_bytes[f] / 16u;
-    const uint64_t N = v.capacity;
-    const uint32_t t = local_cta / chunks_per_row;
-    const uint32_t c = local_cta - t * chunks_per_row;
-    uint64_t slot = cursor + t;
-    if (slot >= N) slot -= N;
-    const uint32_t e0 = c * kTile;
-    const uint32_t cnt = min(W - e0, kTile);
-    prb_copy_span16<8>(reinterpret_cast<uint4*>(v.store[f]) + slot * W + e0,
-                       reinterpret_cast<const uint4*>(src.ptr[f]) + (uint64_t)t * W + e0, cnt);
-}
-
-// Flat mode: the tile is a range of the dense batch and may span many short rows.
+// Short rows: tile `tile` of the dense batch of field f, which may span many rows.
 template <typename T>
 __device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
-                                               uint64_t cursor, uint32_t local_cta)
+                                               uint64_t cursor, uint32_t tile)
 {
     const uint32_t W = v.field_bytes[f] / sizeof(T);
     const uint64_t N = v.capacity;
     const uint64_t total = (uint64_t)n * W;
-    const uint64_t e0 = (uint64_t)local_cta * kTile;
+    const uint64_t e0 = (uint64_t)tile * kTile;
     const uint32_t e1 = (uint32_t)min(total, e0 + kTile);
     prb_copy_mapped<T>(reinterpret_cast<T*>(v.store[f]), reinterpret_cast<const T*>(src.ptr[f]), (uint32_t)e0, e1,
                        [=](uint32_t e) { return (uint64_t)e; },
@@ -59,16 +46,27 @@ __device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const Pr
                        });
 }
 
-__device__ __forceinline__ void copy_field_dispatch(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
-                                                    uint64_t cursor, uint32_t local_cta, uint32_t cpr)
+__device__ __forceinline__ void copy_task(const PrbView& v, const InsertPlan& plan, int f, const PrbBatch& src,
+                                          uint32_t n, uint64_t cursor, uint32_t local)
 {
-    if (cpr > 0) { copy_row_chunk(v, f, src, cursor, local_cta, cpr); return; }
+    if (plan.chunks[f] > 0) {
+        // long rows: one chunk of one row, contiguous on both sides
+        const uint32_t W = v.field_bytes[f] / 16u;
+        const uint32_t t = local / plan.chunks[f];
+        const uint32_t e0 = (local - t * plan.chunks[f]) * plan.chunk[f];
+        const uint32_t cnt = min(W - e0, plan.chunk[f]);
+        uint64_t slot = cursor + t;
+        if (slot >= v.capacity) slot -= v.capacity;
+        prb_copy_span16<4>(reinterpret_cast<uint4*>(v.store[f]) + slot * W + e0,
+                           reinterpret_cast<const uint4*>(src.ptr[f]) + (uint64_t)t * W + e0, cnt);
+        return;
+    }
     switch (v.field_vec[f]) {
-    case 16: copy_flat_tile<uint4>(v, f, src, n, cursor, local_cta); break;
-    case 8: copy_flat_tile<uint2>(v, f, src, n, cursor, local_cta); break;
-    case 4: copy_flat_tile<uint32_t>(v, f, src, n, cursor, local_cta); break;
-    case 2: copy_flat_tile<uint16_t>(v, f, src, n, cursor, local_cta); break;
-    default: copy_flat_tile<uint8_t>(v, f, src, n, cursor, local_cta); break;
+    case 16: copy_flat_tile<uint4>(v, f, src, n, cursor, local); break;
+    case 8: copy_flat_tile<uint2>(v, f, src, n, cursor, local); break;
+    case 4: copy_flat_tile<uint32_t>(v, f, src, n, cursor, local); break;
+    case 2: copy_flat_tile<uint16_t>(v, f, src, n, cursor, local); break;
+    default: copy_flat_tile<uint8_t>(v, f, src, n, cursor, local); break;
     }
 }
 
@@ -111,7 +109,7 @@ __device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restric
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
 {
     __shared__ unsigned long long s_cursor;
@@ -122,11 +120,14 @@ prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__
     if (blockIdx.x == 0) {
         insert_tree(v, n, prio, cursor);
     } else {
-        const uint32_t cta = blockIdx.x - 1;
-#pragma unroll 1
-        for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-            if (cta >= plan.first_cta[f] && cta < plan.first_cta[f + 1])
-                copy_field_dispatch(v, f, src, n, cursor, cta - plan.first_cta[f], plan.chunks_per_row[f]);
+        const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
+        const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
+        const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tasks) / copy_ctas);
+        const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tasks) / copy_ctas);
+        int f = 0;
+        for (uint32_t t = t_lo; t < t_hi; ++t) {
+            while (t >= plan.first_task[f + 1]) ++f;
+            copy_task(v, plan, f, src, n, cursor, t - plan.first_task[f]);
         }
     }
 
@@ -151,22 +152,33 @@ prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__
 
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s)
 {
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+            sm_count = 148;
+    }
     InsertPlan plan;
     uint32_t next = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        plan.first_cta[f] = next;
-        plan.chunks_per_row[f] = 0;
+        plan.first_task[f] = next;
+        plan.chunks[f] = 0;
+        plan.chunk[f] = 0;
         if (v.field_bytes[f] == 0 || src.ptr[f] == nullptr) continue;
         const uint32_t W = v.field_bytes[f] / v.field_vec[f];
         if (v.field_vec[f] == 16 && W >= kRowMode) {
-            plan.chunks_per_row[f] = (W + kTile - 1) / kTile;
-            next += n * plan.chunks_per_row[f];
+            plan.chunks[f] = (W + kChunk - 1) / kChunk;
+            plan.chunk[f] = (W + plan.chunks[f] - 1) / plan.chunks[f];
+            next += n * plan.chunks[f];
         } else {
             const uint64_t total = (uint64_t)n * W;
             next += (uint32_t)((total + kTile - 1) / kTile);
         }
     }
-    plan.first_cta[PRB_NUM_FIELDS] = next;
-    prb_insert_kernel<<<next + 1, kThreads, 0, s>>>(v, n, src, d_prio, plan);
+    plan.first_task[PRB_NUM_FIELDS] = next;
+    const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm - 1;     // CTA 0 is the tree CTA
+    const uint32_t copy_ctas = next < one_wave ? next : one_wave;
+    prb_insert_kernel<<<copy_ctas + 1, kThreads, 0, s>>>(v, n, src, d_prio, plan);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

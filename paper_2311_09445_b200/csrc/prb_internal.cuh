@@ -25,6 +25,7 @@ struct PrbState {
 struct PrbView {
     PrbState* state;
     float* level[PRB_MAX_LEVELS];     // level[l] holds K * n_{l-1} entries (level[0]: 1)
+    uint32_t level_alloc[PRB_MAX_LEVELS];   // entries of level l, zero padding included
     unsigned char* store[PRB_NUM_FIELDS];
     uint32_t field_bytes[PRB_NUM_FIELDS];
     uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes

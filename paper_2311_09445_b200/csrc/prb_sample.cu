@@ -6,29 +6,37 @@
 // fanout) owns one stratum: lane j loads child j, so a child group is one 8..128-byte request;
 // the left-to-right binary32 prefix sums are formed by K-1 broadcast-and-add steps (the same
 // association as the stored parent), a ballot counts the prefixes the binary64 target has
-// passed, and that count is the child to enter.  The read of the sampled rows is Listing 2's
-// `D_storage[sampled_indices]`.  Stratification, the Philox stream and the weights follow the
-// prioritized-replay reference the paper cites (Schaul et al.).
+// passed, and that count is the child to enter.  The top levels of the tree (up to 20 KB) are
+// staged in shared memory at kernel start, the rest is read from L2.  The read of the sampled
+// rows is Listing 2's `D_storage[sampled_indices]`.  Stratification, the Philox stream and the
+// weights follow the prioritized-replay reference the paper cites (Schaul et al.).
 //
-// CTA layout: a CTA serves G consecutive strata.  When rows are long (Atari-shaped) G = 1 and
-// S CTAs share one stratum: each repeats the cheap descent (L2 reads) and copies one chunk of
-// the stratum's rows, so the HBM-bound copy is spread evenly over all SMs without a second
-// launch.  The CTA that finishes last normalises the weights by the batch maximum and bumps
-// the sample-call counter; nothing ever waits on another CTA.
+// Work split: the batch is cut into tasks (a stratum, or one <= 16 KB chunk of one long row of
+// a stratum) and every CTA of a grid that fits the GPU in one wave takes a contiguous range of
+// tasks.  A CTA first walks the tree for the strata its tasks touch (a stratum shared by two
+// CTAs is walked by both: L2 reads only), then copies.  So the chain of dependent tree reads
+// is paid once, and from then on all SMs stream rows.  Raw weights go to scratch; the CTA that
+// is last to finish its descents normalises them by the batch maximum and bumps the call
+// counter while the others are already copying.  No CTA ever waits on another.
 #include "prb_internal.cuh"
 #include "../../include/pearl_prb.h"
 
 namespace {
 
 constexpr int kThreads = 256;
-constexpr uint32_t kTile = kThreads * 8;   // granules per row chunk in row mode
-constexpr uint32_t kRowMode = 512;         // rows of at least this many granules are split into chunks
+constexpr int kCtasPerSm = 4;
+constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per row chunk
+constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
+constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB)
 
 struct SamplePlan {
-    uint32_t G;                              // strata per CTA
-    uint32_t S;                              // CTAs per stratum group (parts); > 1 only if G == 1
-    uint32_t part_first[PRB_NUM_FIELDS];     // row mode: parts [part_first, part_first + parts) copy the chunks
-    uint32_t parts[PRB_NUM_FIELDS];          // 0 = flat mode (copied by part 0)
+    uint32_t tps;                            // tasks per stratum (1 unless some field is in row mode)
+    uint32_t n_tasks;                        // B * tps
+    uint32_t task_first[PRB_NUM_FIELDS];     // row mode: tasks [task_first, task_first + chunks) of a stratum
+    uint32_t chunks[PRB_NUM_FIELDS];         //   copy the chunks of field f; 0 = short rows, copied flat
+    uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
+    uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
+    uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level
 };
 
 // Philox4x32-10 (Salmon et al., SC'11), first output word only.
@@ -50,8 +58,8 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
 }
 
 template <int K>
-__device__ __forceinline__ void descend(const PrbView& v, double x, uint32_t lane, uint32_t& leaf, float& p_leaf,
-                                        unsigned& flags)
+__device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan, const float* s_top, double x,
+                                        uint32_t lane, uint32_t& leaf, float& p_leaf, unsigned& flags)
 {
     constexpr unsigned FULL = 0xFFFFFFFFu;
     const unsigned gshift = (K == 32) ? 0u : ((threadIdx.x & 31u) / K) * K;
@@ -60,7 +68,8 @@ __device__ __forceinline__ void descend(const PrbView& v, double x, uint32_t lan
     float c = 0.0f;
     int j = 0;
     for (uint32_t l = 1; l <= v.depth; ++l) {
-        c = __ldg(v.level[l] + g * K + lane);
+        c = (l <= plan.top_levels) ? s_top[plan.top_off[l] + (uint32_t)g * K + lane]
+                                   : __ldg(v.level[l] + g * K + lane);
         float acc = __shfl_sync(FULL, c, 0, K);
 #pragma unroll
         for (int i = 1; i < K; ++i) {
@@ -85,38 +94,40 @@ __device__ __forceinline__ void descend(const PrbView& v, double x, uint32_t lan
     leaf = (uint32_t)g;
 }
 
-// Row mode: this CTA (part `part` of its stratum) copies one chunk of the sampled row of field f.
-__device__ __forceinline__ void gather_row_chunk(const PrbView& v, int f, unsigned char* out, const SamplePlan& plan,
-                                                 uint32_t part, uint32_t k0, uint32_t leaf)
-{
-    if (part < plan.part_first[f] || part >= plan.part_first[f] + plan.parts[f]) return;
-    const uint32_t W = v.field_bytes[f] / 16u;
-    const uint32_t e0 = (part - plan.part_first[f]) * kTile;
-    const uint32_t cnt = min(W - e0, kTile);
-    prb_copy_span16<8>(reinterpret_cast<uint4*>(out) + (uint64_t)k0 * W + e0,
-                       reinterpret_cast<const uint4*>(v.store[f]) + (uint64_t)leaf * W + e0, cnt);
-}
-
-// Flat mode: the rows of all strata of this CTA, granule by granule.
+// Short rows: rows of strata [k_first, k_first + n_rows), granule by granule; s_idx[r] is the
+// leaf of stratum k_first + r.
 template <typename T>
-__device__ __forceinline__ void gather_flat(const PrbView& v, int f, unsigned char* out, uint32_t k0,
-                                            uint32_t n_strata, const uint32_t* s_idx)
+__device__ __forceinline__ void gather_flat(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
+                                            uint32_t n_rows, const uint32_t* s_idx)
 {
     const uint32_t W = v.field_bytes[f] / sizeof(T);
-    const uint64_t dbase = (uint64_t)k0 * W;
-    prb_copy_mapped<T>(reinterpret_cast<T*>(out), reinterpret_cast<const T*>(v.store[f]), 0u, n_strata * W,
+    const uint64_t dbase = (uint64_t)k_first * W;
+    prb_copy_mapped<T>(reinterpret_cast<T*>(out), reinterpret_cast<const T*>(v.store[f]), 0u, n_rows * W,
                        [=](uint32_t e) { const uint32_t r = e / W; return (uint64_t)s_idx[r] * W + (e - r * W); },
                        [=](uint32_t e) { return dbase + e; });
 }
 
+__device__ __forceinline__ void gather_flat_dispatch(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
+                                                     uint32_t n_rows, const uint32_t* s_idx)
+{
+    switch (v.field_vec[f]) {
+    case 16: gather_flat<uint4>(v, f, out, k_first, n_rows, s_idx); break;
+    case 8: gather_flat<uint2>(v, f, out, k_first, n_rows, s_idx); break;
+    case 4: gather_flat<uint32_t>(v, f, out, k_first, n_rows, s_idx); break;
+    case 2: gather_flat<uint16_t>(v, f, out, k_first, n_rows, s_idx); break;
+    default: gather_flat<uint8_t>(v, f, out, k_first, n_rows, s_idx); break;
+    }
+}
+
 template <int K>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __restrict__ out_idx,
                   float* __restrict__ out_w, PrbBatch dst, SamplePlan plan)
 {
-    constexpr int kGroups = kThreads / K;         // lane groups in a CTA
-    __shared__ uint32_t s_idx[kGroups];
-    __shared__ double s_wraw[kGroups];
+    constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
+    __shared__ float s_top[kTopFloats];
+    __shared__ uint32_t s_idx[R];
+    __shared__ double s_wraw[R];
     __shared__ unsigned long long s_calls, s_fill;
     __shared__ float s_total;
     __shared__ unsigned int s_last;
@@ -127,89 +138,119 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         s_fill = v.state->fill;
         s_total = __ldg(v.level[0]);
     }
+    for (uint32_t l = 1; l <= plan.top_levels; ++l) {
+        const float* src = v.level[l];
+        float* d = s_top + plan.top_off[l];
+        for (uint32_t i = tid; i < v.level_alloc[l]; i += kThreads) d[i] = __ldg(src + i);
+    }
     __syncthreads();
     const float total32 = s_total;
     const unsigned long long calls = s_calls;
     const bool empty = (s_fill == 0) || !(total32 > 0.0f);
 
-    const uint32_t group = blockIdx.x / plan.S;
-    const uint32_t part = blockIdx.x - group * plan.S;
-    const uint32_t k0 = group * plan.G;
-    const uint32_t n_strata = min(plan.G, B - k0);
+    // this CTA's tasks and the strata they touch
+    const uint32_t tps = plan.tps;
+    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * plan.n_tasks) / gridDim.x);
+    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * plan.n_tasks) / gridDim.x);
+    const uint32_t k_lo = t_lo / tps;
+    const uint32_t k_hi = (t_hi + tps - 1) / tps;
+    const uint32_t k_own = (t_lo + tps - 1) / tps;       // strata whose first task is here: this CTA writes their idx / weight
+    const uint32_t n_rounds = (empty || t_hi <= t_lo) ? 0u : (k_hi - k_lo + R - 1) / R;
+    bool ticket_taken = false;
 
-    if (!empty) {
-        // ---- targets and descents: one K-lane group per stratum ----
-        const uint32_t gi = tid / K, lane = tid % K;
-        const uint32_t warp_first_group = (tid / 32u) * (32u / K);
-        if (warp_first_group < n_strata) {          // warp-uniform: whole warps take part in the shuffles
-            const uint32_t k = min(k0 + gi, B - 1);  // surplus groups repeat a valid stratum and write nothing
-            const double total = (double)total32;
-            const double seg = __ddiv_rn(total, (double)B);
-            const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32),
-                                                    (uint32_t)seed, (uint32_t)(seed >> 32));
-            const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
-            double x = __dmul_rn(__dadd_rn((double)k, u), seg);
-            if (x >= total) x = __longlong_as_double(__double_as_longlong(total) - 1);   // next binary64 below total
-            uint32_t leaf; float p; unsigned flags = 0;
-            descend<K>(v, x, lane, leaf, p, flags);
-            if (lane == 0 && gi < n_strata) {
-                s_idx[gi] = leaf;
-                const double scaled = __ddiv_rn(__dmul_rn((double)s_fill, (double)p), total);
-                const double wr = pow(scaled, -(double)beta);
-                s_wraw[gi] = wr;
-                if (part == 0) {
-                    out_idx[k] = (int32_t)leaf;
-                    v.wraw[k] = wr;
-                    if (flags) atomicOr(&v.state->status, flags);
+    for (uint32_t round = 0; round <= n_rounds; ++round) {
+        const uint32_t kb = k_lo + round * R;
+        uint32_t n_round = 0;
+        if (round < n_rounds) {
+            // ---- targets and descents: one K-lane group per stratum ----
+            n_round = min(R, k_hi - kb);
+            const uint32_t gi = tid / K, lane = tid % K;
+            const uint32_t warp_first_group = (tid / 32u) * (32u / K);
+            if (warp_first_group < n_round) {            // warp-uniform: whole warps take part in the shuffles
+                const uint32_t k = min(kb + gi, B - 1);   // surplus groups repeat a valid stratum and write nothing
+                const double total = (double)total32;
+                const double seg = __ddiv_rn(total, (double)B);
+                const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32),
+                                                        (uint32_t)seed, (uint32_t)(seed >> 32));
+                const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
+                double x = __dmul_rn(__dadd_rn((double)k, u), seg);
+                if (x >= total) x = __longlong_as_double(__double_as_longlong(total) - 1);   // next binary64 below total
+                uint32_t leaf; float p; unsigned flags = 0;
+                descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
+                if (lane == 0 && gi < n_round) {
+                    s_idx[gi] = leaf;
+                    double wr = 0.0;
+                    if (kb + gi >= k_own) {
+                        const double scaled = __ddiv_rn(__dmul_rn((double)s_fill, (double)p), total);
+                        wr = pow(scaled, -(double)beta);
+                        out_idx[k] = (int32_t)leaf;
+                        v.wraw[k] = wr;
+                        if (flags) atomicOr(&v.state->status, flags);
+                    }
+                    s_wraw[gi] = wr;
+                }
+            }
+            __syncthreads();
+            if (tid == 0) {
+                double m = 0.0;
+                for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
+                if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
+            }
+        }
+
+        // ---- after this CTA's last descents: the last CTA to get here normalises the weights ----
+        if (!ticket_taken && round + 1 >= n_rounds) {
+            ticket_taken = true;
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                __threadfence();
+                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+            }
+            __syncthreads();
+            if (s_last) {
+                __threadfence();
+                if (empty) {
+                    if (tid == 0) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+                } else if (out_w != nullptr) {
+                    const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
+                    for (uint32_t k = tid; k < B; k += kThreads) out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    if (!empty) v.state->sample_calls = calls + 1;
+                    v.state->wmax_bits = 0ull;
+                    v.state->sample_ticket = 0u;
                 }
             }
         }
-        __syncthreads();
-        if (part == 0 && tid == 0) {
-            double m = s_wraw[0];
-            for (uint32_t i = 1; i < n_strata; ++i) m = fmax(m, s_wraw[i]);
-            atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
-        }
+        if (round >= n_rounds) break;
 
-        // ---- gather: Data Storage rows of this CTA's strata ----
+        // ---- gather: Data Storage rows of this round's strata ----
+        const uint32_t k_flat = max(kb, k_own);              // short fields: copied by the stratum's owner
 #pragma unroll 1
         for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
             if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
-            if (plan.parts[f] > 0) { gather_row_chunk(v, f, dst.ptr[f], plan, part, k0, s_idx[0]); continue; }
-            if (part != 0) continue;
-            switch (v.field_vec[f]) {
-            case 16: gather_flat<uint4>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
-            case 8: gather_flat<uint2>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
-            case 4: gather_flat<uint32_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
-            case 2: gather_flat<uint16_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
-            default: gather_flat<uint8_t>(v, f, dst.ptr[f], k0, n_strata, s_idx); break;
+            if (plan.chunks[f] == 0) {
+                if (k_flat < kb + n_round)
+                    gather_flat_dispatch(v, f, dst.ptr[f], k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb));
+                continue;
+            }
+            // long rows: the tasks of field f that fall in this CTA's range, one chunk each
+            const uint32_t W = v.field_bytes[f] / 16u;
+            const uint4* src = reinterpret_cast<const uint4*>(v.store[f]);
+            uint4* out = reinterpret_cast<uint4*>(dst.ptr[f]);
+            for (uint32_t k = kb; k < kb + n_round; ++k) {
+                const uint32_t first = k * tps + plan.task_first[f];
+                const uint32_t a = max(first, t_lo), b = min(first + plan.chunks[f], t_hi);
+                for (uint32_t t = a; t < b; ++t) {
+                    const uint32_t e0 = (t - first) * plan.chunk[f];
+                    const uint32_t cnt = min(W - e0, plan.chunk[f]);
+                    prb_copy_span16<4>(out + (uint64_t)k * W + e0, src + (uint64_t)s_idx[k - kb] * W + e0, cnt);
+                }
             }
         }
-    }
-
-    // ---- the last CTA to finish normalises the weights and advances the call counter ----
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
-    }
-    __syncthreads();
-    if (s_last) {
-        __threadfence();
-        if (empty) {
-            if (tid == 0) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-        } else {
-            const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
-            if (out_w != nullptr)
-                for (uint32_t k = tid; k < B; k += kThreads) out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
-        }
-        __syncthreads();
-        if (tid == 0) {
-            if (!empty) v.state->sample_calls = calls + 1;
-            v.state->wmax_bits = 0ull;
-            v.state->sample_ticket = 0u;
-        }
+        __syncthreads();        // s_idx is rewritten by the next round
     }
 }
 
@@ -218,29 +259,45 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s)
 {
+    static int sm_count = 0;
+    if (sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+            sm_count = 148;
+    }
     SamplePlan plan;
-    plan.S = 0;
-    bool row_mode = false;
+    plan.tps = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        plan.part_first[f] = 0;
-        plan.parts[f] = 0;
+        plan.task_first[f] = 0;
+        plan.chunks[f] = 0;
+        plan.chunk[f] = 0;
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
         const uint32_t W = v.field_bytes[f] / v.field_vec[f];
         if (v.field_vec[f] == 16 && W >= kRowMode) {
-            row_mode = true;
-            plan.part_first[f] = plan.S;
-            plan.parts[f] = (W + kTile - 1) / kTile;
-            plan.S += plan.parts[f];
+            plan.task_first[f] = plan.tps;
+            plan.chunks[f] = (W + kChunk - 1) / kChunk;
+            plan.chunk[f] = (W + plan.chunks[f] - 1) / plan.chunks[f];
+            plan.tps += plan.chunks[f];
         }
     }
-    if (row_mode) {
-        plan.G = 1;
-    } else {
-        plan.S = 1;
-        plan.G = kThreads / v.fanout;
+    const bool row_mode = plan.tps > 0;
+    if (!row_mode) plan.tps = 1;
+    plan.n_tasks = B * plan.tps;
+    // levels 1 .. top_levels staged in shared memory while they fit
+    plan.top_levels = 0;
+    uint32_t used = 0;
+    for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
+    for (uint32_t l = 1; l <= v.depth; ++l) {
+        if (used + v.level_alloc[l] > kTopFloats) break;
+        plan.top_off[l] = used;
+        used += v.level_alloc[l];
+        plan.top_levels = l;
     }
-    const uint32_t groups = (B + plan.G - 1) / plan.G;
-    const uint32_t grid = groups * plan.S;
+    const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
+    const uint32_t R = kThreads / v.fanout;
+    const uint32_t want = row_mode ? plan.n_tasks : (B + R - 1) / R;
+    const uint32_t grid = want < one_wave ? want : one_wave;
     switch (v.fanout) {
     case 2: prb_sample_kernel<2><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
     case 4: prb_sample_kernel<4><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;

@@ -36,12 +36,17 @@ __device__ bool priority_pow(float delta, float eps, float alpha, float& p)
     double m = __longlong_as_double((bits & 0x000FFFFFFFFFFFFFll) | 0x3FF0000000000000ll);
     if (m > 1.4142135623730951) { m = __dmul_rn(m, 0.5); E += 1; }
 
+    // series coefficients 1/(2n+1) and 1/n!: IEEE quotients of exact integers, folded at compile time
+    constexpr double kOdd[13] = { 1.0 / 1.0, 1.0 / 3.0, 1.0 / 5.0, 1.0 / 7.0, 1.0 / 9.0, 1.0 / 11.0, 1.0 / 13.0,
+                                  1.0 / 15.0, 1.0 / 17.0, 1.0 / 19.0, 1.0 / 21.0, 1.0 / 23.0, 1.0 / 25.0 };
+    constexpr double kRfact[15] = { 1.0 / 1.0, 1.0 / 1.0, 1.0 / 2.0, 1.0 / 6.0, 1.0 / 24.0, 1.0 / 120.0, 1.0 / 720.0,
+                                    1.0 / 5040.0, 1.0 / 40320.0, 1.0 / 362880.0, 1.0 / 3628800.0, 1.0 / 39916800.0,
+                                    1.0 / 479001600.0, 1.0 / 6227020800.0, 1.0 / 87178291200.0 };
     const double t = __ddiv_rn(__dadd_rn(m, -1.0), __dadd_rn(m, 1.0));
     const double t2 = __dmul_rn(t, t);
-    double S = __ddiv_rn(1.0, 25.0);
-#pragma unroll 1
-    for (int n = 11; n >= 0; --n)
-        S = __dadd_rn(__dmul_rn(S, t2), __ddiv_rn(1.0, (double)(2 * n + 1)));
+    double S = kOdd[12];
+#pragma unroll
+    for (int n = 11; n >= 0; --n) S = __dadd_rn(__dmul_rn(S, t2), kOdd[n]);
     const double lnm = __dmul_rn(__dmul_rn(2.0, t), S);
 
     const double L = __dadd_rn(__dmul_rn((double)E, 0.6931471805599453), lnm);
@@ -53,13 +58,9 @@ __device__ bool priority_pow(float delta, float eps, float alpha, float& p)
     double r = __dsub_rn(z, __dmul_rn(k, 0.693147180369123816490));
     r = __dsub_rn(r, __dmul_rn(k, 1.90821492927058770002e-10));
 
-    double fact = 87178291200.0;                       // 14!
-    double P = __ddiv_rn(1.0, fact);
-#pragma unroll 1
-    for (int n = 13; n >= 0; --n) {
-        fact = __ddiv_rn(fact, (double)(n + 1));       // n!
-        P = __dadd_rn(__dmul_rn(P, r), __ddiv_rn(1.0, fact));
-    }
+    double P = kRfact[14];
+#pragma unroll
+    for (int n = 13; n >= 0; --n) P = __dadd_rn(__dmul_rn(P, r), kRfact[n]);
     const double scale = __longlong_as_double(((long long)k + 1023ll) << 52);
     const float out = __double2float_rn(__dmul_rn(P, scale));
     if (!(out <= 3.402823466e+38f)) return false;
@@ -97,8 +98,13 @@ prb_update_kernel(PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict_
     if (flags) atomicOr(&v.state->status, flags);
     __syncthreads();
 
+    // Indices that come straight from a stratified sample are already in order; sort only if needed.
+    int unsorted = 0;
+    for (uint32_t b = tid; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
+    unsorted = __syncthreads_or(unsorted);
+
     // bitonic sort, ascending
-    for (uint32_t k = 2; k <= n2; k <<= 1) {
+    for (uint32_t k = 2; unsorted && k <= n2; k <<= 1) {
         for (uint32_t j = k >> 1; j > 0; j >>= 1) {
             for (uint32_t t = tid; t < (n2 >> 1); t += nt) {
                 const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
