@@ -250,24 +250,34 @@ def run_ours(args, wl, rank, world):
         torch.cuda.synchronize()
         status = prb.sync()
 
-        # one CUDA graph per rotation slot (all buffer state lives on the device, so replays advance it)
-        graphs, kernels_per_step = None, None
+        # CUDA graphs (all buffer state lives on the device, so replays advance it): one graph of
+        # ROTATE consecutive steps, plus single-step graphs for a remainder of K
         l0 = prb.kernel_launches()
         eager_step(0)
         kernels_per_step = prb.kernel_launches() - l0
         torch.cuda.synchronize()
+
+        def capture(calls):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for c in calls:
+                    c()
+            return g
+
         if not args.no_graph:
-            graphs = []
-            for r in range(ROTATE):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    eager_step(r)
-                graphs.append(g)
-            step = lambda i: graphs[i % ROTATE].replay()
+            g_all = capture([lambda r=r: eager_step(r) for r in range(ROTATE)])
+            g_one = [capture([lambda r=r: eager_step(r)]) for r in range(ROTATE)]
+
+            def run_steps(k):
+                for _ in range(k // ROTATE):
+                    g_all.replay()
+                for r in range(k % ROTATE):
+                    g_one[r].replay()
         else:
-            step = eager_step
-        for i in range(max(args.warmup, 3)):
-            step(i)
+            def run_steps(k):
+                for i in range(k):
+                    eager_step(i)
+        run_steps(max(args.warmup, 3))
         torch.cuda.synchronize()
 
         # ---- the timed region: exactly K steps -------------------------------------------
@@ -277,7 +287,7 @@ def run_ours(args, wl, rank, world):
             time.sleep(0.3)
         if world > 1:
             dist.barrier()
-        ms = time_loop(stream, step, args.steps)
+        ms = time_loop(stream, lambda i: run_steps(args.steps), 1)
         if world > 1:
             dist.barrier()
             t = torch.tensor([ms], device=dev, dtype=torch.float64)
@@ -285,13 +295,22 @@ def run_ours(args, wl, rank, world):
             ms = float(t.item())
         clk = clocks.stop() if rank == 0 else None
 
-        # ---- per-call timings (device resident), used for the roofline and the rates -------
-        reps = max(20, min(args.steps, 400))
-        for i in range(3):
-            do_sample(i)
-        ms_sample = time_loop(stream, do_sample, reps) / reps
-        ms_update = time_loop(stream, do_update, reps) / reps
-        ms_insert = time_loop(stream, do_insert, reps) / reps if n_ins else None
+        # ---- per-call timings (device resident), used for the roofline and the rates: a graph of
+        # ROTATE back-to-back calls of one kind, replayed, so that host launch cost is not in them
+        reps = max(3, min(args.steps, 400) // ROTATE)
+
+        def per_call_ms(fn):
+            if args.no_graph:
+                for i in range(3):
+                    fn(i)
+                return time_loop(stream, fn, reps * ROTATE) / (reps * ROTATE)
+            g = capture([lambda r=r: fn(r) for r in range(ROTATE)])
+            g.replay()
+            return time_loop(stream, lambda i: g.replay(), reps) / (reps * ROTATE)
+
+        ms_sample = per_call_ms(do_sample)
+        ms_update = per_call_ms(do_update)
+        ms_insert = per_call_ms(do_insert) if n_ins else None
         status |= prb.sync()
 
         # ---- end to end through the host-buffer calls ----------------------------------------

@@ -3,11 +3,17 @@
 // priority retrieval followed by priority update; Listing 2: experiences are added to the
 // Data Storage and insertion requests go to the Replay Manager).
 //
-// One kernel.  CTA 0 owns the tree: it writes the n leaves and then re-sums the dirty parents
-// level by level (a contiguous slot range dirties a contiguous parent range on every level,
-// so no sorting is needed).  The other CTAs copy rows from the dense batch to ring slots,
-// HBM-bound, 16-byte granules where the row size allows.  The CTA that finishes last advances
-// the cursor and the fill count, after every CTA has read them.
+// One kernel per call, in one of two shapes.
+//   Short rows: CTA 0 owns the tree, the other CTAs copy tiles of the dense batch to ring slots
+//   through registers.
+//   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; thread 0 of
+//   every CTA drives bulk asynchronous copies global -> shared -> global through a ~200 KB
+//   ring (row chunks of <= 16 KB), issuing its loads before the cursor has even arrived; the
+//   other warps copy the short fields, and in CTA 0 they first do the tree work.
+// Tree work: write the n leaves, then re-sum the dirty parents level by level (a contiguous
+// slot range dirties a contiguous parent range on every level, so no sorting is needed).
+// The CTA that finishes last advances the cursor and the fill count, after every CTA has read
+// them.  No CTA waits on another.
 #include "prb_internal.cuh"
 #include "../../include/pearl_prb.h"
 
@@ -15,68 +21,37 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kCtasPerSm = 4;
-constexpr uint32_t kChunk = kThreads * 4;  // upper bound on granules per chunk of a long row
-constexpr uint32_t kTile = kThreads * 8;   // granules per tile of short rows
-constexpr uint32_t kRowMode = 512;         // rows of at least this many 16-byte granules are split into chunks
+constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per chunk of a long row
+constexpr uint32_t kTile = kThreads * 8;     // granules per tile of short rows
+constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
+constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring (dynamic shared memory)
+constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
-// The copy is cut into tasks, numbered field by field; every copy CTA takes a contiguous range.
 struct InsertPlan {
-    uint32_t first_task[PRB_NUM_FIELDS + 1];  // tasks of field f: [first_task[f], first_task[f+1])
-    uint32_t chunks[PRB_NUM_FIELDS];          // > 0: long rows, task = one chunk of one row; 0: short rows, task = one tile
+    // short-row tiles, numbered field by field: tiles of field f are [first_tile[f], first_tile[f+1])
+    uint32_t first_tile[PRB_NUM_FIELDS + 1];
+    // long-row tasks (one chunk of one row), numbered field by field
+    uint32_t first_task[PRB_NUM_FIELDS + 1];
+    uint32_t chunks[PRB_NUM_FIELDS];          // chunks per row of a long-row field, else 0
     uint32_t chunk[PRB_NUM_FIELDS];           // granules per chunk
+    uint32_t ring_stages, ring_stage_bytes;
 };
 
-// Short rows: tile `tile` of the dense batch of field f, which may span many rows.
-template <typename T>
-__device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n,
-                                               uint64_t cursor, uint32_t tile)
+// Barrier among the `nthreads` threads that do the tree work (the whole CTA, or warps 1..7).
+__device__ __forceinline__ void tree_barrier(uint32_t nthreads)
 {
-    const uint32_t W = v.field_bytes[f] / sizeof(T);
-    const uint64_t N = v.capacity;
-    const uint64_t total = (uint64_t)n * W;
-    const uint64_t e0 = (uint64_t)tile * kTile;
-    const uint32_t e1 = (uint32_t)min(total, e0 + kTile);
-    prb_copy_mapped<T>(reinterpret_cast<T*>(v.store[f]), reinterpret_cast<const T*>(src.ptr[f]), (uint32_t)e0, e1,
-                       [=](uint32_t e) { return (uint64_t)e; },
-                       [=](uint32_t e) {
-                           const uint32_t r = e / W;
-                           uint64_t slot = cursor + r;
-                           if (slot >= N) slot -= N;
-                           return slot * W + (e - r * W);
-                       });
+    if (nthreads == blockDim.x) __syncthreads();
+    else asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
 }
 
-__device__ __forceinline__ void copy_task(const PrbView& v, const InsertPlan& plan, int f, const PrbBatch& src,
-                                          uint32_t n, uint64_t cursor, uint32_t local)
-{
-    if (plan.chunks[f] > 0) {
-        // long rows: one chunk of one row, contiguous on both sides
-        const uint32_t W = v.field_bytes[f] / 16u;
-        const uint32_t t = local / plan.chunks[f];
-        const uint32_t e0 = (local - t * plan.chunks[f]) * plan.chunk[f];
-        const uint32_t cnt = min(W - e0, plan.chunk[f]);
-        uint64_t slot = cursor + t;
-        if (slot >= v.capacity) slot -= v.capacity;
-        prb_copy_span16<4>(reinterpret_cast<uint4*>(v.store[f]) + slot * W + e0,
-                           reinterpret_cast<const uint4*>(src.ptr[f]) + (uint64_t)t * W + e0, cnt);
-        return;
-    }
-    switch (v.field_vec[f]) {
-    case 16: copy_flat_tile<uint4>(v, f, src, n, cursor, local); break;
-    case 8: copy_flat_tile<uint2>(v, f, src, n, cursor, local); break;
-    case 4: copy_flat_tile<uint32_t>(v, f, src, n, cursor, local); break;
-    case 2: copy_flat_tile<uint16_t>(v, f, src, n, cursor, local); break;
-    default: copy_flat_tile<uint8_t>(v, f, src, n, cursor, local); break;
-    }
-}
-
-__device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restrict__ prio, uint64_t cursor)
+__device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restrict__ prio, uint64_t cursor,
+                            uint32_t rank, uint32_t nthreads)
 {
     const uint64_t N = v.capacity;
     const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
     float* leaves = v.level[D];
     bool bad = false;
-    for (uint32_t t = threadIdx.x; t < n; t += blockDim.x) {
+    for (uint32_t t = rank; t < n; t += nthreads) {
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
         float p = prio[t];
@@ -84,7 +59,7 @@ __device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restric
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    __syncthreads();
+    tree_barrier(nthreads);
     // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;
     const uint64_t a1 = min(cursor + n, N) - 1;
@@ -101,37 +76,53 @@ __device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restric
         }
         const float* child = v.level[l + 1];
         float* par = v.level[l];
-        for (uint64_t i = threadIdx.x; i < cntA + cntB; i += blockDim.x) {
+        for (uint64_t i = rank; i < cntA + cntB; i += nthreads) {
             const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
             par[j] = prb_sum_children_dyn(child + j * K, K);
         }
-        __syncthreads();
+        tree_barrier(nthreads);
     }
 }
 
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
-prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+// Short rows: tile `tile` of the dense batch of field f, which may span many rows.
+template <typename T>
+__device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n, uint64_t cursor,
+                                               uint32_t tile, uint32_t rank, uint32_t nthreads)
 {
-    __shared__ unsigned long long s_cursor;
-    if (threadIdx.x == 0) s_cursor = v.state->cursor;
-    __syncthreads();
-    const uint64_t cursor = s_cursor;
+    const uint32_t W = v.field_bytes[f] / sizeof(T);
+    const uint64_t N = v.capacity;
+    const uint64_t total = (uint64_t)n * W;
+    const uint64_t e0 = (uint64_t)tile * kTile;
+    const uint32_t e1 = (uint32_t)min(total, e0 + kTile);
+    prb_copy_mapped<T>(reinterpret_cast<T*>(v.store[f]), reinterpret_cast<const T*>(src.ptr[f]), (uint32_t)e0, e1,
+                       [=](uint32_t e) { return (uint64_t)e; },
+                       [=](uint32_t e) {
+                           const uint32_t r = e / W;
+                           uint64_t slot = cursor + r;
+                           if (slot >= N) slot -= N;
+                           return slot * W + (e - r * W);
+                       },
+                       rank, nthreads);
+}
 
-    if (blockIdx.x == 0) {
-        insert_tree(v, n, prio, cursor);
-    } else {
-        const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-        const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
-        const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tasks) / copy_ctas);
-        const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tasks) / copy_ctas);
-        int f = 0;
-        for (uint32_t t = t_lo; t < t_hi; ++t) {
-            while (t >= plan.first_task[f + 1]) ++f;
-            copy_task(v, plan, f, src, n, cursor, t - plan.first_task[f]);
-        }
+__device__ __forceinline__ void copy_tile(const PrbView& v, const InsertPlan& plan, const PrbBatch& src, uint32_t n,
+                                          uint64_t cursor, uint32_t tile, uint32_t rank, uint32_t nthreads)
+{
+    int f = 0;
+    while (tile >= plan.first_tile[f + 1]) ++f;
+    const uint32_t local = tile - plan.first_tile[f];
+    switch (v.field_vec[f]) {
+    case 16: copy_flat_tile<uint4>(v, f, src, n, cursor, local, rank, nthreads); break;
+    case 8: copy_flat_tile<uint2>(v, f, src, n, cursor, local, rank, nthreads); break;
+    case 4: copy_flat_tile<uint32_t>(v, f, src, n, cursor, local, rank, nthreads); break;
+    case 2: copy_flat_tile<uint16_t>(v, f, src, n, cursor, local, rank, nthreads); break;
+    default: copy_flat_tile<uint8_t>(v, f, src, n, cursor, local, rank, nthreads); break;
     }
+}
 
-    // The last CTA to finish publishes the new cursor and fill count.
+// The last CTA to finish publishes the new cursor and fill count (every CTA has read them by then).
+__device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor)
+{
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -148,6 +139,73 @@ prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__
     }
 }
 
+// Short rows only: CTA 0 = tree, CTAs 1.. = a contiguous range of tiles each.
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+{
+    const uint64_t cursor = v.state->cursor;
+    if (blockIdx.x == 0) {
+        insert_tree(v, n, prio, cursor, threadIdx.x, kThreads);
+    } else {
+        const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
+        const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
+        const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tiles) / copy_ctas);
+        const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tiles) / copy_ctas);
+        for (uint32_t t = t_lo; t < t_hi; ++t) copy_tile(v, plan, src, n, cursor, t, threadIdx.x, kThreads);
+    }
+    publish_if_last(v, n, cursor);
+}
+
+// Long rows present: thread 0 drives the bulk ring over this CTA's row chunks; warps 1..7 do the
+// tree (CTA 0) and the short-field tiles (dealt round-robin, CTA 1 first).
+__global__ void __launch_bounds__(kThreads, 1)
+prb_insert_rows_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+{
+    extern __shared__ __align__(128) unsigned char s_ring[];
+    const uint32_t tid = threadIdx.x;
+    const uint64_t cursor = v.state->cursor;       // consumed late by thread 0: its loads go out first
+
+    if (tid == 0) {
+        PrbBulk ring;
+        ring.init(s_ring, s_ring + kRingBarBytes, plan.ring_stages, plan.ring_stage_bytes);
+        const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
+        const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
+        const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
+        auto locate = [&](uint32_t i, int& f, uint32_t& row, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
+            const uint32_t t = t_lo + i;
+            f = 0;
+            while (t >= plan.first_task[f + 1]) ++f;
+            const uint32_t local = t - plan.first_task[f];
+            row = local / plan.chunks[f];
+            W = v.field_bytes[f] / 16u;
+            e0 = (local - row * plan.chunks[f]) * plan.chunk[f];
+            bytes = min(W - e0, plan.chunk[f]) * 16u;
+        };
+        prb_bulk_run(ring, t_hi - t_lo,
+                     [&](uint32_t i, const void*& s, uint32_t& bytes) {
+                         int f; uint32_t row, W, e0;
+                         locate(i, f, row, W, e0, bytes);
+                         s = src.ptr[f] + ((uint64_t)row * W + e0) * 16u;
+                     },
+                     [&](uint32_t i, void*& d, uint32_t& bytes) {
+                         int f; uint32_t row, W, e0;
+                         locate(i, f, row, W, e0, bytes);
+                         uint64_t slot = cursor + row;
+                         if (slot >= v.capacity) slot -= v.capacity;
+                         d = v.store[f] + (slot * W + e0) * 16u;
+                     });
+        ring.finish();
+        if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
+    } else if (tid >= 32) {
+        const uint32_t rank = tid - 32u, nthreads = kThreads - 32u;
+        if (blockIdx.x == 0) insert_tree(v, n, prio, cursor, rank, nthreads);
+        const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
+        for (uint32_t t = (blockIdx.x + gridDim.x - 1) % gridDim.x; t < n_tiles; t += gridDim.x)
+            copy_tile(v, plan, src, n, cursor, t, rank, nthreads);
+    }
+    publish_if_last(v, n, cursor);
+}
+
 }  // namespace
 
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s)
@@ -160,9 +218,10 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
             sm_count = 148;
     }
     InsertPlan plan;
-    uint32_t next = 0;
+    uint32_t tiles = 0, tasks = 0, stage = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        plan.first_task[f] = next;
+        plan.first_tile[f] = tiles;
+        plan.first_task[f] = tasks;
         plan.chunks[f] = 0;
         plan.chunk[f] = 0;
         if (v.field_bytes[f] == 0 || src.ptr[f] == nullptr) continue;
@@ -170,15 +229,36 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         if (v.field_vec[f] == 16 && W >= kRowMode) {
             plan.chunks[f] = (W + kChunk - 1) / kChunk;
             plan.chunk[f] = (W + plan.chunks[f] - 1) / plan.chunks[f];
-            next += n * plan.chunks[f];
+            tasks += n * plan.chunks[f];
+            if (plan.chunk[f] * 16u > stage) stage = plan.chunk[f] * 16u;
         } else {
             const uint64_t total = (uint64_t)n * W;
-            next += (uint32_t)((total + kTile - 1) / kTile);
+            tiles += (uint32_t)((total + kTile - 1) / kTile);
         }
     }
-    plan.first_task[PRB_NUM_FIELDS] = next;
-    const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm - 1;     // CTA 0 is the tree CTA
-    const uint32_t copy_ctas = next < one_wave ? next : one_wave;
-    prb_insert_kernel<<<copy_ctas + 1, kThreads, 0, s>>>(v, n, src, d_prio, plan);
+    plan.first_tile[PRB_NUM_FIELDS] = tiles;
+    plan.first_task[PRB_NUM_FIELDS] = tasks;
+    plan.ring_stages = 0;
+    plan.ring_stage_bytes = 0;
+    if (tasks == 0) {
+        const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm - 1;     // CTA 0 is the tree CTA
+        const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
+        prb_insert_kernel<<<copy_ctas + 1, kThreads, 0, s>>>(v, n, src, d_prio, plan);
+    } else {
+        stage = (stage + 127u) / 128u * 128u;
+        plan.ring_stage_bytes = stage;
+        plan.ring_stages = kRingBytes / stage;
+        if (plan.ring_stages > kRingBarBytes / 8) plan.ring_stages = kRingBarBytes / 8;
+        const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
+        static bool big_smem = false;
+        if (!big_smem) {
+            if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
+                return -1;
+            big_smem = true;
+        }
+        const uint32_t grid = tasks < (uint32_t)sm_count ? tasks : (uint32_t)sm_count;
+        prb_insert_rows_kernel<<<grid, kThreads, smem, s>>>(v, n, src, d_prio, plan);
+    }
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

@@ -15,7 +15,10 @@
 // a stratum) and every CTA of a grid that fits the GPU in one wave takes a contiguous range of
 // tasks.  A CTA first walks the tree for the strata its tasks touch (a stratum shared by two
 // CTAs is walked by both: L2 reads only), then copies.  So the chain of dependent tree reads
-// is paid once, and from then on all SMs stream rows.  Raw weights go to scratch; the CTA that
+// is paid once, and from then on all SMs stream rows.  Long rows (Atari-shaped) move as bulk
+// asynchronous copies global -> shared -> global driven by one thread per CTA, one CTA per SM
+// with a ~200 KB ring, so that nearly the whole read set of a batch is in flight at once;
+// short rows are copied through registers.  Raw weights go to scratch; the CTA that
 // is last to finish its descents normalises them by the batch maximum and bumps the call
 // counter while the others are already copying.  No CTA ever waits on another.
 #include "prb_internal.cuh"
@@ -28,6 +31,8 @@ constexpr int kCtasPerSm = 4;
 constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per row chunk
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
 constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB)
+constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring of a long-row CTA (dynamic shared memory)
+constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
 struct SamplePlan {
     uint32_t tps;                            // tasks per stratum (1 unless some field is in row mode)
@@ -35,6 +40,7 @@ struct SamplePlan {
     uint32_t task_first[PRB_NUM_FIELDS];     // row mode: tasks [task_first, task_first + chunks) of a stratum
     uint32_t chunks[PRB_NUM_FIELDS];         //   copy the chunks of field f; 0 = short rows, copied flat
     uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
+    uint32_t ring_stages, ring_stage_bytes;  // bulk-copy ring (long rows only; 0 stages otherwise)
     uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
     uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level
 };
@@ -98,24 +104,25 @@ __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan
 // leaf of stratum k_first + r.
 template <typename T>
 __device__ __forceinline__ void gather_flat(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
-                                            uint32_t n_rows, const uint32_t* s_idx)
+                                            uint32_t n_rows, const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
 {
     const uint32_t W = v.field_bytes[f] / sizeof(T);
     const uint64_t dbase = (uint64_t)k_first * W;
     prb_copy_mapped<T>(reinterpret_cast<T*>(out), reinterpret_cast<const T*>(v.store[f]), 0u, n_rows * W,
                        [=](uint32_t e) { const uint32_t r = e / W; return (uint64_t)s_idx[r] * W + (e - r * W); },
-                       [=](uint32_t e) { return dbase + e; });
+                       [=](uint32_t e) { return dbase + e; }, rank, nthreads);
 }
 
 __device__ __forceinline__ void gather_flat_dispatch(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
-                                                     uint32_t n_rows, const uint32_t* s_idx)
+                                                     uint32_t n_rows, const uint32_t* s_idx, uint32_t rank,
+                                                     uint32_t nthreads)
 {
     switch (v.field_vec[f]) {
-    case 16: gather_flat<uint4>(v, f, out, k_first, n_rows, s_idx); break;
-    case 8: gather_flat<uint2>(v, f, out, k_first, n_rows, s_idx); break;
-    case 4: gather_flat<uint32_t>(v, f, out, k_first, n_rows, s_idx); break;
-    case 2: gather_flat<uint16_t>(v, f, out, k_first, n_rows, s_idx); break;
-    default: gather_flat<uint8_t>(v, f, out, k_first, n_rows, s_idx); break;
+    case 16: gather_flat<uint4>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
+    case 8: gather_flat<uint2>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
+    case 4: gather_flat<uint32_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
+    case 2: gather_flat<uint16_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
+    default: gather_flat<uint8_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
     }
 }
 
@@ -131,8 +138,12 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
     __shared__ unsigned long long s_calls, s_fill;
     __shared__ float s_total;
     __shared__ unsigned int s_last;
+    extern __shared__ __align__(128) unsigned char s_ring[];   // long rows: mbarriers, then the ring buffers
 
     const uint32_t tid = threadIdx.x;
+    const bool bulk = plan.ring_stages > 0;
+    PrbBulk ring;
+    if (bulk && tid == 0) ring.init(s_ring, s_ring + kRingBarBytes, plan.ring_stages, plan.ring_stage_bytes);
     if (tid == 0) {
         s_calls = v.state->sample_calls;
         s_fill = v.state->fill;
@@ -227,30 +238,46 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         if (round >= n_rounds) break;
 
         // ---- gather: Data Storage rows of this round's strata ----
-        const uint32_t k_flat = max(kb, k_own);              // short fields: copied by the stratum's owner
+        if (bulk && tid == 0) {
+            // long rows: this CTA's tasks of the round, one chunk each, through the bulk ring
+            const uint32_t a = max(t_lo, kb * tps), b = min(t_hi, (kb + n_round) * tps);
+            auto locate = [&](uint32_t i, int& f, uint32_t& k, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
+                const uint32_t t = a + i;
+                k = t / tps;
+                const uint32_t r = t - k * tps;
+                f = 0;
+                while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
+                W = v.field_bytes[f] / 16u;
+                e0 = (r - plan.task_first[f]) * plan.chunk[f];
+                bytes = min(W - e0, plan.chunk[f]) * 16u;
+            };
+            prb_bulk_run(ring, b > a ? b - a : 0u,
+                         [&](uint32_t i, const void*& src, uint32_t& bytes) {
+                             int f; uint32_t k, W, e0;
+                             locate(i, f, k, W, e0, bytes);
+                             src = v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u;
+                         },
+                         [&](uint32_t i, void*& out, uint32_t& bytes) {
+                             int f; uint32_t k, W, e0;
+                             locate(i, f, k, W, e0, bytes);
+                             out = dst.ptr[f] + ((uint64_t)k * W + e0) * 16u;
+                         });
+        }
+        // short rows: copied by the stratum's owner through registers (warp 0 is busy when there are long rows)
+        const uint32_t k_flat = max(kb, k_own);
+        if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
+            const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads - 32u : kThreads;
 #pragma unroll 1
-        for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-            if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
-            if (plan.chunks[f] == 0) {
-                if (k_flat < kb + n_round)
-                    gather_flat_dispatch(v, f, dst.ptr[f], k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb));
-                continue;
-            }
-            // long rows: the tasks of field f that fall in this CTA's range, one chunk each
-            const uint32_t W = v.field_bytes[f] / 16u;
-            const uint4* src = reinterpret_cast<const uint4*>(v.store[f]);
-            uint4* out = reinterpret_cast<uint4*>(dst.ptr[f]);
-            for (uint32_t k = kb; k < kb + n_round; ++k) {
-                const uint32_t first = k * tps + plan.task_first[f];
-                const uint32_t a = max(first, t_lo), b = min(first + plan.chunks[f], t_hi);
-                for (uint32_t t = a; t < b; ++t) {
-                    const uint32_t e0 = (t - first) * plan.chunk[f];
-                    const uint32_t cnt = min(W - e0, plan.chunk[f]);
-                    prb_copy_span16<4>(out + (uint64_t)k * W + e0, src + (uint64_t)s_idx[k - kb] * W + e0, cnt);
-                }
+            for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+                if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
+                gather_flat_dispatch(v, f, dst.ptr[f], k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
             }
         }
         __syncthreads();        // s_idx is rewritten by the next round
+    }
+    if (bulk && tid == 0) {
+        ring.finish();
+        if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
     }
 }
 
@@ -294,16 +321,46 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         used += v.level_alloc[l];
         plan.top_levels = l;
     }
-    const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
     const uint32_t R = kThreads / v.fanout;
-    const uint32_t want = row_mode ? plan.n_tasks : (B + R - 1) / R;
-    const uint32_t grid = want < one_wave ? want : one_wave;
-    switch (v.fanout) {
-    case 2: prb_sample_kernel<2><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
-    case 4: prb_sample_kernel<4><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
-    case 8: prb_sample_kernel<8><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
-    case 16: prb_sample_kernel<16><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
-    default: prb_sample_kernel<32><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+    uint32_t grid, smem = 0;
+    plan.ring_stages = 0;
+    plan.ring_stage_bytes = 0;
+    if (row_mode) {
+        // one CTA per SM, each with a ring of chunk-sized stages
+        uint32_t stage = 0;
+        for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
+        stage = (stage + 127u) / 128u * 128u;
+        plan.ring_stage_bytes = stage;
+        plan.ring_stages = kRingBytes / stage;
+        if (plan.ring_stages > kRingBarBytes / 8) plan.ring_stages = kRingBarBytes / 8;
+        smem = kRingBarBytes + plan.ring_stages * stage;
+        grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
+    } else {
+        const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
+        const uint32_t want = (B + R - 1) / R;
+        grid = want < one_wave ? want : one_wave;
     }
+    static bool big_smem[6] = { false, false, false, false, false, false };
+    const int ki = v.log2_fanout;
+    cudaError_t attr = cudaSuccess;
+#define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
+    do {                                                                                                          \
+        if (smem && !big_smem[ki]) {                                                                              \
+            attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
+                                        (int)(kRingBarBytes + kRingBytes));                                       \
+            big_smem[ki] = (attr == cudaSuccess);                                                                 \
+        }                                                                                                         \
+        if (attr == cudaSuccess)                                                                                  \
+            prb_sample_kernel<KK><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);          \
+    } while (0)
+    switch (v.fanout) {
+    case 2: PRB_LAUNCH_SAMPLE(2); break;
+    case 4: PRB_LAUNCH_SAMPLE(4); break;
+    case 8: PRB_LAUNCH_SAMPLE(8); break;
+    case 16: PRB_LAUNCH_SAMPLE(16); break;
+    default: PRB_LAUNCH_SAMPLE(32); break;
+    }
+#undef PRB_LAUNCH_SAMPLE
+    if (attr != cudaSuccess) return -1;
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
