@@ -27,7 +27,7 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kCtasPerSm = 4;
+constexpr int kCtasPerSm = 2;
 constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per row chunk
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
 constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB)
@@ -42,7 +42,8 @@ struct SamplePlan {
     uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
     uint32_t ring_stages, ring_stage_bytes;  // bulk-copy ring (long rows only; 0 stages otherwise)
     uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
-    uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level
+    uint32_t top_vec4;                       // 16-byte units staged, from the start of level 1
+    uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level from the start of level 1
 };
 
 // Philox4x32-10 (Salmon et al., SC'11), first output word only.
@@ -100,29 +101,66 @@ __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan
     leaf = (uint32_t)g;
 }
 
-// Short rows: rows of strata [k_first, k_first + n_rows), granule by granule; s_idx[r] is the
-// leaf of stratum k_first + r.
-template <typename T>
-__device__ __forceinline__ void gather_flat(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
-                                            uint32_t n_rows, const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
+__device__ __forceinline__ uint4 load_granule(const unsigned char* base, uint64_t g, uint32_t vec)
 {
-    const uint32_t W = v.field_bytes[f] / sizeof(T);
-    const uint64_t dbase = (uint64_t)k_first * W;
-    prb_copy_mapped<T>(reinterpret_cast<T*>(out), reinterpret_cast<const T*>(v.store[f]), 0u, n_rows * W,
-                       [=](uint32_t e) { const uint32_t r = e / W; return (uint64_t)s_idx[r] * W + (e - r * W); },
-                       [=](uint32_t e) { return dbase + e; }, rank, nthreads);
+    uint4 r = make_uint4(0u, 0u, 0u, 0u);
+    switch (vec) {
+    case 16: r = reinterpret_cast<const uint4*>(base)[g]; break;
+    case 8: { const uint2 t = reinterpret_cast<const uint2*>(base)[g]; r.x = t.x; r.y = t.y; break; }
+    case 4: r.x = reinterpret_cast<const uint32_t*>(base)[g]; break;
+    case 2: r.x = reinterpret_cast<const uint16_t*>(base)[g]; break;
+    default: r.x = base[g]; break;
+    }
+    return r;
 }
 
-__device__ __forceinline__ void gather_flat_dispatch(const PrbView& v, int f, unsigned char* out, uint32_t k_first,
-                                                     uint32_t n_rows, const uint32_t* s_idx, uint32_t rank,
-                                                     uint32_t nthreads)
+__device__ __forceinline__ void store_granule(unsigned char* base, uint64_t g, uint32_t vec, const uint4& r)
 {
-    switch (v.field_vec[f]) {
-    case 16: gather_flat<uint4>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
-    case 8: gather_flat<uint2>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
-    case 4: gather_flat<uint32_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
-    case 2: gather_flat<uint16_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
-    default: gather_flat<uint8_t>(v, f, out, k_first, n_rows, s_idx, rank, nthreads); break;
+    switch (vec) {
+    case 16: reinterpret_cast<uint4*>(base)[g] = r; break;
+    case 8: reinterpret_cast<uint2*>(base)[g] = make_uint2(r.x, r.y); break;
+    case 4: reinterpret_cast<uint32_t*>(base)[g] = r.x; break;
+    case 2: reinterpret_cast<uint16_t*>(base)[g] = (uint16_t)r.x; break;
+    default: base[g] = (unsigned char)r.x; break;
+    }
+}
+
+// Short rows of strata [k_first, k_first + n_rows): every short field of the batch, granule by
+// granule, by `nthreads` threads.  s_idx[r] is the leaf of stratum k_first + r.  The first two
+// granules per thread of ALL fields are loaded before anything is stored, so a small batch costs
+// one round trip instead of one per field; what is left goes field by field.
+__device__ __forceinline__ void gather_short_fields(const PrbView& v, const SamplePlan& plan, const PrbBatch& dst,
+                                                    uint32_t k_first, uint32_t n_rows, const uint32_t* s_idx,
+                                                    uint32_t rank, uint32_t nthreads)
+{
+    uint4 tmp[PRB_NUM_FIELDS][2];
+#pragma unroll
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint32_t e = rank + u * nthreads;
+            if (e < total) {
+                const uint32_t r = (W == 1) ? e : e / W;
+                tmp[f][u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
+            }
+        }
+    }
+#pragma unroll
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+        const uint64_t dbase = (uint64_t)k_first * W;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const uint32_t e = rank + u * nthreads;
+            if (e < total) store_granule(dst.ptr[f], dbase + e, vec, tmp[f][u]);
+        }
+        for (uint32_t e = rank + 2 * nthreads; e < total; e += nthreads) {     // the rest of a larger batch
+            const uint32_t r = e / W;
+            store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec));
+        }
     }
 }
 
@@ -149,10 +187,16 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         s_fill = v.state->fill;
         s_total = __ldg(v.level[0]);
     }
-    for (uint32_t l = 1; l <= plan.top_levels; ++l) {
-        const float* src = v.level[l];
-        float* d = s_top + plan.top_off[l];
-        for (uint32_t i = tid; i < v.level_alloc[l]; i += kThreads) d[i] = __ldg(src + i);
+    {
+        // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
+        const float4* src = reinterpret_cast<const float4*>(v.level[1]);
+        float4 t[kTopFloats / 4 / kThreads];
+#pragma unroll
+        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+            if (tid + u * kThreads < plan.top_vec4) t[u] = __ldg(src + tid + u * kThreads);
+#pragma unroll
+        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+            if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
     }
     __syncthreads();
     const float total32 = s_total;
@@ -167,7 +211,6 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
     const uint32_t k_hi = (t_hi + tps - 1) / tps;
     const uint32_t k_own = (t_lo + tps - 1) / tps;       // strata whose first task is here: this CTA writes their idx / weight
     const uint32_t n_rounds = (empty || t_hi <= t_lo) ? 0u : (k_hi - k_lo + R - 1) / R;
-    bool ticket_taken = false;
 
     for (uint32_t round = 0; round <= n_rounds; ++round) {
         const uint32_t kb = k_lo + round * R;
@@ -197,82 +240,81 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
                         out_idx[k] = (int32_t)leaf;
                         v.wraw[k] = wr;
                         if (flags) atomicOr(&v.state->status, flags);
+                        __threadfence();
                     }
                     s_wraw[gi] = wr;
                 }
             }
             __syncthreads();
-            if (tid == 0) {
+        }
+
+        // From here the CTA splits by role: threads 0..127 copy, threads 128..255 look after the weights.
+        const bool last_descents = round + 1 >= n_rounds;
+        if (tid >= kThreads / 2) {
+            if (tid == kThreads / 2) {
                 double m = 0.0;
                 for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
                 if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
-            }
-        }
-
-        // ---- after this CTA's last descents: the last CTA to get here normalises the weights ----
-        if (!ticket_taken && round + 1 >= n_rounds) {
-            ticket_taken = true;
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) {
-                __threadfence();
-                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
-            }
-            __syncthreads();
-            if (s_last) {
-                __threadfence();
-                if (empty) {
-                    if (tid == 0) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-                } else if (out_w != nullptr) {
-                    const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
-                    for (uint32_t k = tid; k < B; k += kThreads) out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
+                if (last_descents) {
+                    // every descent of this CTA is done: the last CTA to get here normalises the weights
+                    __threadfence();
+                    s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
                 }
-                __syncthreads();
-                if (tid == 0) {
-                    if (!empty) v.state->sample_calls = calls + 1;
-                    v.state->wmax_bits = 0ull;
-                    v.state->sample_ticket = 0u;
+            }
+            if (last_descents) {
+                asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+                if (s_last) {
+                    __threadfence();
+                    if (empty) {
+                        if (tid == kThreads / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+                    } else if (out_w != nullptr) {
+                        const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
+                        for (uint32_t k = tid - kThreads / 2; k < B; k += kThreads / 2)
+                            out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
+                    }
+                    asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+                    if (tid == kThreads / 2) {
+                        if (!empty) v.state->sample_calls = calls + 1;
+                        v.state->wmax_bits = 0ull;
+                        v.state->sample_ticket = 0u;
+                    }
                 }
+            }
+        } else if (round < n_rounds) {
+            // ---- gather: Data Storage rows of this round's strata ----
+            if (bulk && tid == 0) {
+                // long rows: this CTA's tasks of the round, one chunk each, through the bulk ring
+                const uint32_t a = max(t_lo, kb * tps), b = min(t_hi, (kb + n_round) * tps);
+                auto locate = [&](uint32_t i, int& f, uint32_t& k, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
+                    const uint32_t t = a + i;
+                    k = t / tps;
+                    const uint32_t r = t - k * tps;
+                    f = 0;
+                    while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
+                    W = v.field_bytes[f] / 16u;
+                    e0 = (r - plan.task_first[f]) * plan.chunk[f];
+                    bytes = min(W - e0, plan.chunk[f]) * 16u;
+                };
+                prb_bulk_run(ring, b > a ? b - a : 0u,
+                             [&](uint32_t i, const void*& src, uint32_t& bytes) {
+                                 int f; uint32_t k, W, e0;
+                                 locate(i, f, k, W, e0, bytes);
+                                 src = v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u;
+                             },
+                             [&](uint32_t i, void*& out, uint32_t& bytes) {
+                                 int f; uint32_t k, W, e0;
+                                 locate(i, f, k, W, e0, bytes);
+                                 out = dst.ptr[f] + ((uint64_t)k * W + e0) * 16u;
+                             });
+            }
+            // short rows: copied by the stratum's owner through registers (warp 0 drives the ring when there is one)
+            const uint32_t k_flat = max(kb, k_own);
+            if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
+                const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads / 2 - 32u : kThreads / 2;
+                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
             }
         }
         if (round >= n_rounds) break;
-
-        // ---- gather: Data Storage rows of this round's strata ----
-        if (bulk && tid == 0) {
-            // long rows: this CTA's tasks of the round, one chunk each, through the bulk ring
-            const uint32_t a = max(t_lo, kb * tps), b = min(t_hi, (kb + n_round) * tps);
-            auto locate = [&](uint32_t i, int& f, uint32_t& k, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
-                const uint32_t t = a + i;
-                k = t / tps;
-                const uint32_t r = t - k * tps;
-                f = 0;
-                while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
-                W = v.field_bytes[f] / 16u;
-                e0 = (r - plan.task_first[f]) * plan.chunk[f];
-                bytes = min(W - e0, plan.chunk[f]) * 16u;
-            };
-            prb_bulk_run(ring, b > a ? b - a : 0u,
-                         [&](uint32_t i, const void*& src, uint32_t& bytes) {
-                             int f; uint32_t k, W, e0;
-                             locate(i, f, k, W, e0, bytes);
-                             src = v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u;
-                         },
-                         [&](uint32_t i, void*& out, uint32_t& bytes) {
-                             int f; uint32_t k, W, e0;
-                             locate(i, f, k, W, e0, bytes);
-                             out = dst.ptr[f] + ((uint64_t)k * W + e0) * 16u;
-                         });
-        }
-        // short rows: copied by the stratum's owner through registers (warp 0 is busy when there are long rows)
-        const uint32_t k_flat = max(kb, k_own);
-        if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
-            const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads - 32u : kThreads;
-#pragma unroll 1
-            for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-                if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
-                gather_flat_dispatch(v, f, dst.ptr[f], k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
-            }
-        }
         __syncthreads();        // s_idx is rewritten by the next round
     }
     if (bulk && tid == 0) {
@@ -312,13 +354,15 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     if (!row_mode) plan.tps = 1;
     plan.n_tasks = B * plan.tps;
     // levels 1 .. top_levels staged in shared memory while they fit
+    // (the levels lie one after another in the slab, each start 256-byte aligned)
     plan.top_levels = 0;
-    uint32_t used = 0;
+    plan.top_vec4 = 0;
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
     for (uint32_t l = 1; l <= v.depth; ++l) {
-        if (used + v.level_alloc[l] > kTopFloats) break;
-        plan.top_off[l] = used;
-        used += v.level_alloc[l];
+        const uint64_t off = (uint64_t)(v.level[l] - v.level[1]);
+        if (off + v.level_alloc[l] > kTopFloats) break;
+        plan.top_off[l] = (uint32_t)off;
+        plan.top_vec4 = (uint32_t)((off + v.level_alloc[l] + 3) / 4);
         plan.top_levels = l;
     }
     const uint32_t R = kThreads / v.fanout;
