@@ -212,7 +212,7 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
     const uint32_t k_own = (t_lo + tps - 1) / tps;       // strata whose first task is here: this CTA writes their idx / weight
     const uint32_t n_rounds = (empty || t_hi <= t_lo) ? 0u : (k_hi - k_lo + R - 1) / R;
 
-    for (uint32_t round = 0; round <= n_rounds; ++round) {
+    for (uint32_t round = 0; round < max(n_rounds, 1u); ++round) {      // one pass even with nothing to do: the ticket
         const uint32_t kb = k_lo + round * R;
         uint32_t n_round = 0;
         if (round < n_rounds) {
@@ -249,7 +249,7 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         }
 
         // From here the CTA splits by role: threads 0..127 copy, threads 128..255 look after the weights.
-        const bool last_descents = round + 1 >= n_rounds;
+        const bool last_descents = round + 1 >= n_rounds;      // true exactly once per CTA
         if (tid >= kThreads / 2) {
             if (tid == kThreads / 2) {
                 double m = 0.0;
@@ -314,7 +314,6 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
                 gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
             }
         }
-        if (round >= n_rounds) break;
         __syncthreads();        // s_idx is rewritten by the next round
     }
     if (bulk && tid == 0) {
