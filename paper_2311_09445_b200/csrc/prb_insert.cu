@@ -6,25 +6,26 @@
 // One kernel per call, in one of two shapes.
 //   Short rows: CTA 0 owns the tree, the other CTAs copy tiles of the dense batch to ring slots
 //   through registers.
-//   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; thread 0 of
+//   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; warp 0 of
 //   every CTA drives bulk asynchronous copies global -> shared -> global through a ~200 KB
-//   ring (row chunks of <= 16 KB), issuing its loads before the cursor has even arrived; the
-//   other warps copy the short fields, and in CTA 0 they first do the tree work.
+//   ring (row chunks of <= 8 KB, one lane per stage), issuing its loads before the cursor has
+//   even arrived; the other warps copy the short fields, and in CTA 0 they first do the tree.
 // Tree work: write the n leaves, then re-sum the dirty parents level by level (a contiguous
 // slot range dirties a contiguous parent range on every level, so no sorting is needed).
-// The CTA that finishes last advances the cursor and the fill count, after every CTA has read
-// them.  No CTA waits on another.
+// The CTA that is last to have read the cursor advances it (and the fill count) while the copies
+// are still running.  No CTA waits on another.
 #include "prb_internal.cuh"
 #include "../../include/pearl_prb.h"
 
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kWorkers = 224;                // warps 0..6 move data / do the tree; thread kWorkers publishes the cursor
 constexpr int kCtasPerSm = 4;
-constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per chunk of a long row
-constexpr uint32_t kTile = kThreads * 8;     // granules per tile of short rows
+constexpr uint32_t kChunk = 512;             // upper bound on granules per chunk of a long row (8 KB)
+constexpr uint32_t kTile = kWorkers * 8;     // granules per tile of short rows
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
-constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring (dynamic shared memory)
+constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring (dynamic shared memory), <= 32 stages
 constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
 struct InsertPlan {
@@ -37,7 +38,7 @@ struct InsertPlan {
     uint32_t ring_stages, ring_stage_bytes;
 };
 
-// Barrier among the `nthreads` threads that do the tree work (the whole CTA, or warps 1..7).
+// Barrier among the `nthreads` threads that do the tree work (a whole number of warps).
 __device__ __forceinline__ void tree_barrier(uint32_t nthreads)
 {
     if (nthreads == blockDim.x) __syncthreads();
@@ -120,90 +121,111 @@ __device__ __forceinline__ void copy_tile(const PrbView& v, const InsertPlan& pl
     }
 }
 
-// The last CTA to finish publishes the new cursor and fill count (every CTA has read them by then).
+// Taken by one thread per CTA once the whole CTA holds the cursor: the last CTA to get here
+// publishes the new cursor and fill count.  Nothing later in the kernel reads them, so this
+// happens while the copies are still running.
 __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor)
 {
+    __threadfence();
+    const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
+    if (done == gridDim.x - 1) {
+        const uint64_t N = v.capacity;
+        uint64_t c = cursor + n;
+        if (c >= N) c -= N;
+        v.state->cursor = c;
+        const uint64_t fill = v.state->fill + n;
+        v.state->fill = fill > N ? N : fill;
+        v.state->insert_ticket = 0;
+    }
+}
+
+// Short rows only: CTA 0 = tree, CTAs 1.. = a contiguous range of tiles each.  Warps 0..6 work,
+// thread kWorkers reads the cursor for the CTA and takes the ticket.
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+{
+    __shared__ unsigned long long s_cursor;
+    const uint32_t tid = threadIdx.x;
+    if (tid == kWorkers) s_cursor = v.state->cursor;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
-        if (done == gridDim.x - 1) {
-            const uint64_t N = v.capacity;
-            uint64_t c = cursor + n;
-            if (c >= N) c -= N;
-            v.state->cursor = c;
-            const uint64_t fill = v.state->fill + n;
-            v.state->fill = fill > N ? N : fill;
-            v.state->insert_ticket = 0;
+    const uint64_t cursor = s_cursor;
+    if (tid == kWorkers) {
+        publish_if_last(v, n, cursor);
+    } else if (tid < kWorkers) {
+        if (blockIdx.x == 0) {
+            insert_tree(v, n, prio, cursor, tid, kWorkers);
+        } else {
+            const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
+            const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
+            const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tiles) / copy_ctas);
+            const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tiles) / copy_ctas);
+            for (uint32_t t = t_lo; t < t_hi; ++t) copy_tile(v, plan, src, n, cursor, t, tid, kWorkers);
         }
     }
 }
 
-// Short rows only: CTA 0 = tree, CTAs 1.. = a contiguous range of tiles each.
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
-prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
-{
-    const uint64_t cursor = v.state->cursor;
-    if (blockIdx.x == 0) {
-        insert_tree(v, n, prio, cursor, threadIdx.x, kThreads);
-    } else {
-        const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
-        const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
-        const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tiles) / copy_ctas);
-        const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tiles) / copy_ctas);
-        for (uint32_t t = t_lo; t < t_hi; ++t) copy_tile(v, plan, src, n, cursor, t, threadIdx.x, kThreads);
-    }
-    publish_if_last(v, n, cursor);
-}
-
-// Long rows present: thread 0 drives the bulk ring over this CTA's row chunks; warps 1..7 do the
-// tree (CTA 0) and the short-field tiles (dealt round-robin, CTA 1 first).
+// Long rows present.  Warp 0: lane s owns ring stage s and moves row chunks t_lo+s, t_lo+s+S, ...
+// of this CTA's range; the first loads go out before the cursor has arrived (a source address does
+// not depend on it).  Warps 1..6: the tree (CTA 0) and the short-field tiles (dealt round-robin,
+// CTA 1 first).  Thread kWorkers: cursor and ticket.
 __global__ void __launch_bounds__(kThreads, 1)
 prb_insert_rows_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
+    __shared__ unsigned long long s_cursor;
     const uint32_t tid = threadIdx.x;
-    const uint64_t cursor = v.state->cursor;       // consumed late by thread 0: its loads go out first
+    const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
+    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
+    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
+    const bool ring_lane = tid < plan.ring_stages;
 
-    if (tid == 0) {
-        PrbBulk ring;
-        ring.init(s_ring, s_ring + kRingBarBytes, plan.ring_stages, plan.ring_stage_bytes);
-        const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-        const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
-        const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
-        auto locate = [&](uint32_t i, int& f, uint32_t& row, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
-            const uint32_t t = t_lo + i;
-            f = 0;
-            while (t >= plan.first_task[f + 1]) ++f;
-            const uint32_t local = t - plan.first_task[f];
-            row = local / plan.chunks[f];
-            W = v.field_bytes[f] / 16u;
-            e0 = (local - row * plan.chunks[f]) * plan.chunk[f];
-            bytes = min(W - e0, plan.chunk[f]) * 16u;
-        };
-        prb_bulk_run(ring, t_hi - t_lo,
-                     [&](uint32_t i, const void*& s, uint32_t& bytes) {
-                         int f; uint32_t row, W, e0;
-                         locate(i, f, row, W, e0, bytes);
-                         s = src.ptr[f] + ((uint64_t)row * W + e0) * 16u;
-                     },
-                     [&](uint32_t i, void*& d, uint32_t& bytes) {
-                         int f; uint32_t row, W, e0;
-                         locate(i, f, row, W, e0, bytes);
-                         uint64_t slot = cursor + row;
-                         if (slot >= v.capacity) slot -= v.capacity;
-                         d = v.store[f] + (slot * W + e0) * 16u;
-                     });
+    // one row chunk: field, row in the batch, first granule, bytes
+    auto locate = [&](uint32_t t, int& f, uint32_t& row, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
+        f = 0;
+        while (t >= plan.first_task[f + 1]) ++f;
+        const uint32_t local = t - plan.first_task[f];
+        row = local / plan.chunks[f];
+        W = v.field_bytes[f] / 16u;
+        e0 = (local - row * plan.chunks[f]) * plan.chunk[f];
+        bytes = min(W - e0, plan.chunk[f]) * 16u;
+    };
+
+    PrbBulkLane ring;
+    int f = 0; uint32_t row = 0, W = 0, e0 = 0, bytes = 0;
+    uint32_t t = t_lo + tid;
+    if (tid == kWorkers) s_cursor = v.state->cursor;
+    if (ring_lane) {
+        ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
+        if (t < t_hi) {
+            locate(t, f, row, W, e0, bytes);
+            ring.load(src.ptr[f] + ((uint64_t)row * W + e0) * 16u, bytes);
+        }
+    }
+    __syncthreads();
+    const uint64_t cursor = s_cursor;
+
+    if (tid == kWorkers) {
+        publish_if_last(v, n, cursor);
+    } else if (ring_lane) {
+        while (t < t_hi) {
+            uint64_t slot = cursor + row;
+            if (slot >= v.capacity) slot -= v.capacity;
+            ring.store(v.store[f] + (slot * W + e0) * 16u, bytes);
+            t += plan.ring_stages;
+            if (t < t_hi) {
+                locate(t, f, row, W, e0, bytes);
+                ring.load(src.ptr[f] + ((uint64_t)row * W + e0) * 16u, bytes);
+            }
+        }
         ring.finish();
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
-    } else if (tid >= 32) {
-        const uint32_t rank = tid - 32u, nthreads = kThreads - 32u;
+    } else if (tid >= 32 && tid < kWorkers) {
+        const uint32_t rank = tid - 32u, nthreads = kWorkers - 32u;
         if (blockIdx.x == 0) insert_tree(v, n, prio, cursor, rank, nthreads);
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
-        for (uint32_t t = (blockIdx.x + gridDim.x - 1) % gridDim.x; t < n_tiles; t += gridDim.x)
-            copy_tile(v, plan, src, n, cursor, t, rank, nthreads);
+        for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
+            copy_tile(v, plan, src, n, cursor, tile, rank, nthreads);
     }
-    publish_if_last(v, n, cursor);
 }
 
 }  // namespace
@@ -248,7 +270,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
         plan.ring_stages = kRingBytes / stage;
-        if (plan.ring_stages > kRingBarBytes / 8) plan.ring_stages = kRingBarBytes / 8;
+        if (plan.ring_stages > 32) plan.ring_stages = 32;
         const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
         static bool big_smem = false;
         if (!big_smem) {

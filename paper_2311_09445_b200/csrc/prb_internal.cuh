@@ -123,96 +123,62 @@ __device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __
 }
 
 // ---- bulk asynchronous copies (TMA, non-tensor form, no multicast) ------------------------------
-// Long rows move global -> shared -> global as cp.async.bulk transfers driven by ONE thread of
-// the CTA: a load completes on an mbarrier, the store is tracked by a bulk group.  Up to the
-// whole ring (about 200 KB per SM) is in flight, which registers cannot hold.
-// Addresses and sizes are multiples of 16 bytes (rows of 16-byte granules, 256-byte aligned bases).
+// Long rows move global -> shared -> global as cp.async.bulk transfers.  Warp 0 of a CTA drives
+// a ring of up to 32 stages in shared memory, ONE LANE PER STAGE: a lane issues the load of its
+// chunk (completion on the stage's mbarrier), waits for it, issues the store (tracked by the
+// lane's own bulk group) and, if it has another chunk, waits until the store has read the stage
+// before loading again.  All stages of all SMs are in flight together, about 200 KB per SM,
+// which registers cannot hold.  Addresses and sizes are multiples of 16 bytes (rows of 16-byte
+// granules, 256-byte aligned bases).
 
 constexpr uint32_t kBulkSpinLimit = 1u << 20;   // mbarrier polls before a wait gives up
-constexpr int kBulkLag = 2;                     // bulk stores that may still be reading when a stage is refilled
 
 __device__ __forceinline__ uint32_t prb_smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-struct PrbBulk {
-    uint32_t bars;          // shared address of `stages` mbarriers (8 bytes each)
-    uint32_t buf;           // shared address of `stages` buffers of `stage_bytes`
-    uint32_t stages, stage_bytes;
-    uint32_t issued, drained;   // loads issued / stores issued so far, over the life of the kernel
-    bool failed;                // a bounded wait ran out
+struct PrbBulkLane {
+    uint32_t bar;        // shared address of this lane's mbarrier
+    uint32_t buf;        // shared address of this lane's stage
+    uint32_t parity;     // phase parity of the next load's completion
+    bool busy;           // a store issued from the stage may still be reading it
+    bool failed;         // a bounded wait ran out
 
-    __device__ __forceinline__ void init(void* bar_mem, void* buf_mem, uint32_t n_stages, uint32_t bytes)
+    __device__ __forceinline__ void init(void* bar_mem, void* buf_mem)
     {
-        bars = prb_smem_addr(bar_mem); buf = prb_smem_addr(buf_mem);
-        stages = n_stages; stage_bytes = bytes; issued = 0; drained = 0; failed = false;
-        for (uint32_t s = 0; s < n_stages; ++s)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bars + 8u * s));
+        bar = prb_smem_addr(bar_mem); buf = prb_smem_addr(buf_mem);
+        parity = 0; busy = false; failed = false;
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    // A stage is free if it was never used, or the store that last read it has finished reading.
-    __device__ __forceinline__ bool can_load() const
-    {
-        if (failed || issued - drained >= stages) return false;
-        return issued < stages || drained + stages >= issued + 1 + kBulkLag;
     }
     __device__ __forceinline__ void load(const void* gsrc, uint32_t bytes)
     {
-        if (issued >= stages) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kBulkLag) : "memory");
-        const uint32_t s = issued % stages;
-        const uint32_t bar = bars + 8u * s;
+        if (busy) { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); busy = false; }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(buf + s * stage_bytes), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
-        ++issued;
+                     ::"r"(buf), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
     }
-    // Waits (bounded) for the oldest undrained load; false if the wait ran out.
-    __device__ __forceinline__ bool wait_oldest()
+    // Waits (bounded) for the load, then stores the stage to gdst.  The store is issued inside the
+    // polling loop so that a lane whose data has landed does not wait for the other lanes.
+    __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
     {
-        const uint32_t s = drained % stages, parity = (drained / stages) & 1u;
-        const uint32_t bar = bars + 8u * s;
-        for (uint32_t spin = 0; spin < kBulkSpinLimit; ++spin) {
+        bool done = false;
+        for (uint32_t spin = 0; spin < kBulkSpinLimit && !done; ++spin) {
             uint32_t ok;
             asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-            if (ok) return true;
+            if (ok) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             ::"l"(gdst), "r"(buf), "r"(bytes) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                done = true;
+            }
         }
-        failed = true;
-        return false;
+        parity ^= 1u;
+        busy = done;
+        if (!done) failed = true;
     }
-    // Stores the oldest loaded stage to gdst (after waiting for its load).
-    __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
-    {
-        const bool ok = wait_oldest();
-        const uint32_t s = drained % stages;
-        if (ok) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                         ::"l"(gdst), "r"(buf + s * stage_bytes), "r"(bytes) : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        }
-        ++drained;
-    }
-    // Before the CTA exits: loads still in flight are waited for (bounded), stores are completed.
-    __device__ __forceinline__ void finish()
-    {
-        while (drained < issued) { wait_oldest(); ++drained; }
-        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    }
+    // Before the CTA exits: this lane's stores are complete.
+    __device__ __forceinline__ void finish() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 };
-
-// Runs tasks [0, n) through the ring.  src_of(i, src, bytes) names what task i reads,
-// dst_of(i, dst, bytes) where it goes (asked for only when the store is issued).  One thread.
-template <typename SrcOf, typename DstOf>
-__device__ __forceinline__ void prb_bulk_run(PrbBulk& ring, uint32_t n, SrcOf src_of, DstOf dst_of)
-{
-    uint32_t li = 0, di = 0;
-    const void* src; void* dst; uint32_t bytes;
-    while (li < n && ring.can_load()) { src_of(li, src, bytes); ring.load(src, bytes); ++li; }
-    while (di < li) {
-        dst_of(di, dst, bytes);
-        ring.store(dst, bytes);
-        ++di;
-        while (li < n && ring.can_load()) { src_of(li, src, bytes); ring.load(src, bytes); ++li; }
-    }
-}
 
 #endif  // __CUDACC__

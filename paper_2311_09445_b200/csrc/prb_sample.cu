@@ -28,10 +28,10 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kCtasPerSm = 2;
-constexpr uint32_t kChunk = kThreads * 4;    // upper bound on granules per row chunk
+constexpr uint32_t kChunk = 512;             // upper bound on granules per row chunk (8 KB)
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
 constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB)
-constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring of a long-row CTA (dynamic shared memory)
+constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring of a long-row CTA (dynamic shared memory), <= 32 stages
 constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
 struct SamplePlan {
@@ -180,8 +180,9 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
 
     const uint32_t tid = threadIdx.x;
     const bool bulk = plan.ring_stages > 0;
-    PrbBulk ring;
-    if (bulk && tid == 0) ring.init(s_ring, s_ring + kRingBarBytes, plan.ring_stages, plan.ring_stage_bytes);
+    PrbBulkLane ring;            // lanes 0 .. ring_stages-1 of warp 0 own one stage each
+    const bool ring_lane = bulk && tid < plan.ring_stages;
+    if (ring_lane) ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
     if (tid == 0) {
         s_calls = v.state->sample_calls;
         s_fill = v.state->fill;
@@ -282,30 +283,19 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
             }
         } else if (round < n_rounds) {
             // ---- gather: Data Storage rows of this round's strata ----
-            if (bulk && tid == 0) {
-                // long rows: this CTA's tasks of the round, one chunk each, through the bulk ring
+            if (ring_lane) {
+                // long rows: this CTA's tasks of the round, one chunk each; lane s takes tasks a+s, a+s+S, ...
                 const uint32_t a = max(t_lo, kb * tps), b = min(t_hi, (kb + n_round) * tps);
-                auto locate = [&](uint32_t i, int& f, uint32_t& k, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
-                    const uint32_t t = a + i;
-                    k = t / tps;
-                    const uint32_t r = t - k * tps;
-                    f = 0;
+                for (uint32_t t = a + tid; t < b; t += plan.ring_stages) {
+                    const uint32_t k = t / tps, r = t - k * tps;
+                    int f = 0;
                     while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
-                    W = v.field_bytes[f] / 16u;
-                    e0 = (r - plan.task_first[f]) * plan.chunk[f];
-                    bytes = min(W - e0, plan.chunk[f]) * 16u;
-                };
-                prb_bulk_run(ring, b > a ? b - a : 0u,
-                             [&](uint32_t i, const void*& src, uint32_t& bytes) {
-                                 int f; uint32_t k, W, e0;
-                                 locate(i, f, k, W, e0, bytes);
-                                 src = v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u;
-                             },
-                             [&](uint32_t i, void*& out, uint32_t& bytes) {
-                                 int f; uint32_t k, W, e0;
-                                 locate(i, f, k, W, e0, bytes);
-                                 out = dst.ptr[f] + ((uint64_t)k * W + e0) * 16u;
-                             });
+                    const uint32_t W = v.field_bytes[f] / 16u;
+                    const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
+                    const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
+                    ring.load(v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u, bytes);
+                    ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
+                }
             }
             // short rows: copied by the stratum's owner through registers (warp 0 drives the ring when there is one)
             const uint32_t k_flat = max(kb, k_own);
@@ -316,7 +306,7 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         }
         __syncthreads();        // s_idx is rewritten by the next round
     }
-    if (bulk && tid == 0) {
+    if (ring_lane) {
         ring.finish();
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
     }
@@ -375,7 +365,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
         plan.ring_stages = kRingBytes / stage;
-        if (plan.ring_stages > kRingBarBytes / 8) plan.ring_stages = kRingBarBytes / 8;
+        if (plan.ring_stages > 32) plan.ring_stages = 32;
         smem = kRingBarBytes + plan.ring_stages * stage;
         grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
     } else {
