@@ -142,7 +142,8 @@ __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, ui
 // Short rows only: CTA 0 = tree, CTAs 1.. = a contiguous range of tiles each.  Warps 0..6 work,
 // thread kWorkers reads the cursor for the CTA and takes the ticket.
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
-prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
+                  const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
 {
     __shared__ unsigned long long s_cursor;
     const uint32_t tid = threadIdx.x;
@@ -169,7 +170,8 @@ prb_insert_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__
 // not depend on it).  Warps 1..6: the tree (CTA 0) and the short-field tiles (dealt round-robin,
 // CTA 1 first).  Thread kWorkers: cursor and ticket.
 __global__ void __launch_bounds__(kThreads, 1)
-prb_insert_rows_kernel(PrbView v, uint32_t n, PrbBatch src, const float* __restrict__ prio, InsertPlan plan)
+prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
+                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ unsigned long long s_cursor;

@@ -166,15 +166,14 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
 
 template <int K>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
-prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __restrict__ out_idx,
-                  float* __restrict__ out_w, PrbBatch dst, SamplePlan plan)
+prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uint64_t seed,
+                  int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
+                  const __grid_constant__ SamplePlan plan)
 {
     constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
     __shared__ float s_top[kTopFloats];
     __shared__ uint32_t s_idx[R];
     __shared__ double s_wraw[R];
-    __shared__ unsigned long long s_calls, s_fill;
-    __shared__ float s_total;
     __shared__ unsigned int s_last;
     extern __shared__ __align__(128) unsigned char s_ring[];   // long rows: mbarriers, then the ring buffers
 
@@ -183,11 +182,11 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
     PrbBulkLane ring;            // lanes 0 .. ring_stages-1 of warp 0 own one stage each
     const bool ring_lane = bulk && tid < plan.ring_stages;
     if (ring_lane) ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
-    if (tid == 0) {
-        s_calls = v.state->sample_calls;
-        s_fill = v.state->fill;
-        s_total = __ldg(v.level[0]);
-    }
+    // every thread reads the state it needs itself (same addresses: one request per warp), so the
+    // targets can be formed while the staged levels are still on their way
+    const unsigned long long calls = v.state->sample_calls;
+    const unsigned long long fill = v.state->fill;
+    const float total32 = __ldg(v.level[0]);
     {
         // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
         const float4* src = reinterpret_cast<const float4*>(v.level[1]);
@@ -199,10 +198,7 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
         for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
             if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
     }
-    __syncthreads();
-    const float total32 = s_total;
-    const unsigned long long calls = s_calls;
-    const bool empty = (s_fill == 0) || !(total32 > 0.0f);
+    const bool empty = (fill == 0) || !(total32 > 0.0f);
 
     // this CTA's tasks and the strata they touch
     const uint32_t tps = plan.tps;
@@ -216,27 +212,36 @@ prb_sample_kernel(PrbView v, uint32_t B, float beta, uint64_t seed, int32_t* __r
     for (uint32_t round = 0; round < max(n_rounds, 1u); ++round) {      // one pass even with nothing to do: the ticket
         const uint32_t kb = k_lo + round * R;
         uint32_t n_round = 0;
+        // ---- targets: stratum k of the batch draws x_k ----
+        const uint32_t gi = tid / K, lane = tid % K;
+        bool walks = false;
+        uint32_t k = 0;
+        double x = 0.0;
+        const double total = (double)total32;
         if (round < n_rounds) {
-            // ---- targets and descents: one K-lane group per stratum ----
             n_round = min(R, k_hi - kb);
-            const uint32_t gi = tid / K, lane = tid % K;
-            const uint32_t warp_first_group = (tid / 32u) * (32u / K);
-            if (warp_first_group < n_round) {            // warp-uniform: whole warps take part in the shuffles
-                const uint32_t k = min(kb + gi, B - 1);   // surplus groups repeat a valid stratum and write nothing
-                const double total = (double)total32;
+            walks = (tid / 32u) * (32u / K) < n_round;   // warp-uniform: whole warps take part in the shuffles
+            if (walks) {
+                k = min(kb + gi, B - 1);                  // surplus groups repeat a valid stratum and write nothing
                 const double seg = __ddiv_rn(total, (double)B);
                 const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32),
                                                         (uint32_t)seed, (uint32_t)(seed >> 32));
                 const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
-                double x = __dmul_rn(__dadd_rn((double)k, u), seg);
+                x = __dmul_rn(__dadd_rn((double)k, u), seg);
                 if (x >= total) x = __longlong_as_double(__double_as_longlong(total) - 1);   // next binary64 below total
+            }
+        }
+        if (round == 0) __syncthreads();                  // the staged levels are in shared memory
+        if (round < n_rounds) {
+            // ---- descents: one K-lane group per stratum ----
+            if (walks) {
                 uint32_t leaf; float p; unsigned flags = 0;
                 descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
                 if (lane == 0 && gi < n_round) {
                     s_idx[gi] = leaf;
                     double wr = 0.0;
                     if (kb + gi >= k_own) {
-                        const double scaled = __ddiv_rn(__dmul_rn((double)s_fill, (double)p), total);
+                        const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)p), total);
                         wr = pow(scaled, -(double)beta);
                         out_idx[k] = (int32_t)leaf;
                         v.wraw[k] = wr;

@@ -70,7 +70,7 @@ __device__ bool priority_pow(float delta, float eps, float alpha, float& p)
 
 // keys: (index << 32) | batch position, kInvalidKey for skipped entries; vals: priority by batch position.
 __global__ void __launch_bounds__(1024)
-prb_update_kernel(PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx, const float* __restrict__ val,
+prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx, const float* __restrict__ val,
                   int raw, float alpha, float eps)
 {
     extern __shared__ __align__(16) unsigned char smem[];
