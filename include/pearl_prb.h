@@ -122,6 +122,18 @@ int pearl_prb_update(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const f
 int pearl_prb_update_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx,
                                 const float* d_prio);
 
+/* Priority update followed by insertion, in one launch.  The result is exactly that of
+ * pearl_prb_update(prb, B, d_idx, d_td, alpha, eps) followed by pearl_prb_insert(prb, n, ...): the
+ * update's tree work is done first, the insertion's tree work after it, by the same thread block,
+ * while the other thread blocks already copy the new rows into the Data Storage (an update touches
+ * the tree only, so the two do not conflict).  This is the overlap of the paper's training
+ * protocol, where insertion runs beside the priority update (Section IV-C; Eq. 7:
+ * T_itr = T_samp + max(T_ins, T_upd + T_learner)).  Arguments and errors as for the two calls. */
+int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_td,
+                            float alpha, float eps, uint32_t n, const void* d_obs, const void* d_act,
+                            const float* d_rew, const void* d_next_obs, const uint8_t* d_done,
+                            const float* d_prio);
+
 /* Host-buffer forms of the three calls (the paper's host runtime exchanges requests and data
  * with the Replay Manager over PCIe, Section IV-A).  They copy their inputs to the device and
  * their outputs back on the handle's stream; sample_host returns after the stream has drained,

@@ -42,6 +42,7 @@ SIGNATURES = {
     "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
+    "pearl_prb_update_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_host": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
@@ -168,6 +169,14 @@ class PrioritizedReplay:
         rc = load_library().pearl_prb_update_priorities(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(prio, "prio"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_update_priorities")
+
+    def update_insert(self, idx, td, alpha: float, eps: float, obs, act, rew, next_obs, done, prio) -> None:
+        rc = load_library().pearl_prb_update_insert(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"), alpha, eps,
+                                                    prio.numel(), _dptr(obs, "obs"), _dptr(act, "act"),
+                                                    _dptr(rew, "rew"), _dptr(next_obs, "next_obs"),
+                                                    _dptr(done, "done"), _dptr(prio, "prio"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update_insert")
 
     # ---- the same calls, host buffers (numpy arrays or host torch tensors) -----------------
     def insert_host(self, obs, act, rew, next_obs, done, prio) -> None:

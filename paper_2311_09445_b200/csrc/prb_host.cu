@@ -262,6 +262,29 @@ int pearl_prb_update_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx
     return update_common(h, B, d_idx, d_prio, 1, 0.0f, 0.0f);
 }
 
+int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_td, float alpha, float eps,
+                            uint32_t n, const void* d_obs, const void* d_act, const float* d_rew, const void* d_next_obs,
+                            const uint8_t* d_done, const float* d_prio)
+{
+    if (!h || !d_idx || !d_td || !d_prio) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    if (!finite_nonneg(alpha) || !finite_nonneg(eps)) return PEARL_ERR_BAD_ARG;
+    const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
+    int rc = check_batch_ptrs(h, ptrs);
+    if (rc != PEARL_OK) return rc;
+    if (misaligned(d_prio, 4) || misaligned(d_idx, 4) || misaligned(d_td, 4)) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    PrbBatch b;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
+    const int k = prb_launch_insert(h->view, n, b, d_prio, h->stream, B, d_idx, d_td, 0, alpha, eps);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
+}
+
 // ---- host-buffer forms ---------------------------------------------------------------------
 
 int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const void* h_act, const float* h_rew,

@@ -14,14 +14,13 @@
 // slot range dirties a contiguous parent range on every level, so no sorting is needed).
 // The CTA that is last to have read the cursor advances it (and the fill count) while the copies
 // are still running.  No CTA waits on another.
-#include "prb_internal.cuh"
-#include "../../include/pearl_prb.h"
+#include "prb_tree.cuh"
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWorkers = 224;                // warps 0..6 move data / do the tree; thread kWorkers publishes the cursor
-constexpr int kCtasPerSm = 4;
+constexpr int kWorkers = 256;                // threads that copy short rows / do the tree work
+constexpr int kThreadsShort = kWorkers + 32;     // short-row kernel: workers, then the warp whose lane 0 publishes the cursor
+constexpr int kThreadsRows = 32 + kWorkers + 32; // long-row kernel: ring warp, workers, publishing warp
 constexpr uint32_t kChunk = 512;             // upper bound on granules per chunk of a long row (8 KB)
 constexpr uint32_t kTile = kWorkers * 8;     // granules per tile of short rows
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
@@ -37,53 +36,6 @@ struct InsertPlan {
     uint32_t chunk[PRB_NUM_FIELDS];           // granules per chunk
     uint32_t ring_stages, ring_stage_bytes;
 };
-
-// Barrier among the `nthreads` threads that do the tree work (a whole number of warps).
-__device__ __forceinline__ void tree_barrier(uint32_t nthreads)
-{
-    if (nthreads == blockDim.x) __syncthreads();
-    else asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
-}
-
-__device__ void insert_tree(const PrbView& v, uint32_t n, const float* __restrict__ prio, uint64_t cursor,
-                            uint32_t rank, uint32_t nthreads)
-{
-    const uint64_t N = v.capacity;
-    const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
-    float* leaves = v.level[D];
-    bool bad = false;
-    for (uint32_t t = rank; t < n; t += nthreads) {
-        uint64_t slot = cursor + t;
-        if (slot >= N) slot -= N;
-        float p = prio[t];
-        if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
-        leaves[slot] = p;
-    }
-    if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    tree_barrier(nthreads);
-    // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
-    const uint64_t a0 = cursor;
-    const uint64_t a1 = min(cursor + n, N) - 1;
-    const bool wrapped = cursor + n > N;
-    const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
-    for (int l = (int)D - 1; l >= 0; --l) {
-        const uint32_t sh = lg * (D - (uint32_t)l);
-        const uint64_t pa0 = a0 >> sh, pa1 = a1 >> sh;
-        const uint64_t cntA = pa1 - pa0 + 1;
-        uint64_t cntB = 0;
-        if (wrapped) {
-            const uint64_t pb1 = b1 >> sh;
-            cntB = (pa0 == 0) ? 0 : min(pb1, pa0 - 1) + 1;   // parents of B not already in A
-        }
-        const float* child = v.level[l + 1];
-        float* par = v.level[l];
-        for (uint64_t i = rank; i < cntA + cntB; i += nthreads) {
-            const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
-            par[j] = prb_sum_children_dyn(child + j * K, K);
-        }
-        tree_barrier(nthreads);
-    }
-}
 
 // Short rows: tile `tile` of the dense batch of field f, which may span many rows.
 template <typename T>
@@ -139,12 +91,23 @@ __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, ui
     }
 }
 
-// Short rows only: CTA 0 = tree, CTAs 1.. = a contiguous range of tiles each.  Warps 0..6 work,
-// thread kWorkers reads the cursor for the CTA and takes the ticket.
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+// A priority update to run before the insertion's tree work, by the same team (B == 0: none).
+struct FusedUpdate {
+    uint32_t B, n2;
+    const int32_t* idx;
+    const float* val;
+    int raw;
+    float alpha, eps;
+};
+
+// Short rows only: CTA 0 = tree (after the optional update), CTAs 1.. = a contiguous range of tiles
+// each.  Threads 0..kWorkers-1 work; thread kWorkers reads the cursor for the CTA and takes the ticket.
+__global__ void __launch_bounds__(kThreadsShort, 2)
 prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
-                  const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
+                  const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
+                  const __grid_constant__ FusedUpdate upd)
 {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ unsigned long long s_cursor;
     const uint32_t tid = threadIdx.x;
     if (tid == kWorkers) s_cursor = v.state->cursor;
@@ -154,7 +117,10 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
         publish_if_last(v, n, cursor);
     } else if (tid < kWorkers) {
         if (blockIdx.x == 0) {
-            insert_tree(v, n, prio, cursor, tid, kWorkers);
+            PrbTeam team;
+            team.rank = tid; team.size = kWorkers; team.whole_cta = false;
+            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_dyn);
+            prb_insert_tree_team(v, team, n, prio, cursor);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
@@ -167,19 +133,26 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
 
 // Long rows present.  Warp 0: lane s owns ring stage s and moves row chunks t_lo+s, t_lo+s+S, ...
 // of this CTA's range; the first loads go out before the cursor has arrived (a source address does
-// not depend on it).  Warps 1..6: the tree (CTA 0) and the short-field tiles (dealt round-robin,
-// CTA 1 first).  Thread kWorkers: cursor and ticket.
-__global__ void __launch_bounds__(kThreads, 1)
+// not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, after the optional update)
+// and the short-field tiles (dealt round-robin, CTA 1 first).  Thread 32+kWorkers: cursor and
+// ticket.  With an update fused in, CTA 0 moves no rows: its ring memory holds the update's keys.
+__global__ void __launch_bounds__(kThreadsRows, 1)
 prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
-                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
+                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
+                       const __grid_constant__ FusedUpdate upd)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ unsigned long long s_cursor;
     const uint32_t tid = threadIdx.x;
     const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
-    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
-    const bool ring_lane = tid < plan.ring_stages;
+    const uint32_t first_copy_cta = upd.B ? 1u : 0u;
+    const uint32_t copy_ctas = gridDim.x - first_copy_cta;
+    const bool copies = blockIdx.x >= first_copy_cta;
+    const uint32_t c = blockIdx.x - first_copy_cta;
+    const uint32_t t_lo = copies ? (uint32_t)(((uint64_t)c * n_tasks) / copy_ctas) : 0u;
+    const uint32_t t_hi = copies ? (uint32_t)(((uint64_t)(c + 1) * n_tasks) / copy_ctas) : 0u;
+    const bool ring_lane = copies && tid < plan.ring_stages;
+    constexpr uint32_t kPublisher = 32 + kWorkers;
 
     // one row chunk: field, row in the batch, first granule, bytes
     auto locate = [&](uint32_t t, int& f, uint32_t& row, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
@@ -195,7 +168,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     PrbBulkLane ring;
     int f = 0; uint32_t row = 0, W = 0, e0 = 0, bytes = 0;
     uint32_t t = t_lo + tid;
-    if (tid == kWorkers) s_cursor = v.state->cursor;
+    if (tid == kPublisher) s_cursor = v.state->cursor;
     if (ring_lane) {
         ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
         if (t < t_hi) {
@@ -206,7 +179,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     __syncthreads();
     const uint64_t cursor = s_cursor;
 
-    if (tid == kWorkers) {
+    if (tid == kPublisher) {
         publish_if_last(v, n, cursor);
     } else if (ring_lane) {
         while (t < t_hi) {
@@ -221,18 +194,23 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         }
         ring.finish();
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
-    } else if (tid >= 32 && tid < kWorkers) {
-        const uint32_t rank = tid - 32u, nthreads = kWorkers - 32u;
-        if (blockIdx.x == 0) insert_tree(v, n, prio, cursor, rank, nthreads);
+    } else if (tid >= 32 && tid < kPublisher) {
+        PrbTeam team;
+        team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
+        if (blockIdx.x == 0) {
+            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_ring);
+            prb_insert_tree_team(v, team, n, prio, cursor);
+        }
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
         for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
-            copy_tile(v, plan, src, n, cursor, tile, rank, nthreads);
+            copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
     }
 }
 
 }  // namespace
 
-int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s)
+int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
+                      uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps)
 {
     static int sm_count = 0;
     if (sm_count == 0) {
@@ -241,6 +219,11 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
             sm_count = 148;
     }
+    FusedUpdate upd;
+    upd.B = upd_B; upd.n2 = 2; upd.idx = upd_idx; upd.val = upd_val; upd.raw = upd_raw; upd.alpha = alpha; upd.eps = eps;
+    while (upd.n2 < upd_B) upd.n2 <<= 1;
+    const uint32_t upd_smem = upd_B ? (uint32_t)prb_update_smem_bytes(upd.n2) : 0u;
+
     InsertPlan plan;
     uint32_t tiles = 0, tasks = 0, stage = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
@@ -265,15 +248,21 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
     if (tasks == 0) {
-        const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm - 1;     // CTA 0 is the tree CTA
+        static bool big_smem = false;
+        if (upd_smem + 64 > 48 * 1024 && !big_smem) {
+            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
+                return -1;
+            big_smem = true;
+        }
+        const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        prb_insert_kernel<<<copy_ctas + 1, kThreads, 0, s>>>(v, n, src, d_prio, plan);
+        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem, s>>>(v, n, src, d_prio, plan, upd);
     } else {
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
         plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
-        const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
+        const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;     // >= the update's keys (<= 48 KB)
         static bool big_smem = false;
         if (!big_smem) {
             if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -281,8 +270,9 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
                 return -1;
             big_smem = true;
         }
-        const uint32_t grid = tasks < (uint32_t)sm_count ? tasks : (uint32_t)sm_count;
-        prb_insert_rows_kernel<<<grid, kThreads, smem, s>>>(v, n, src, d_prio, plan);
+        const uint32_t want = tasks + (upd_B ? 1u : 0u);           // with an update, CTA 0 moves no rows
+        const uint32_t grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
+        prb_insert_rows_kernel<<<grid, kThreadsRows, smem < upd_smem ? upd_smem : smem, s>>>(v, n, src, d_prio, plan, upd);
     }
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

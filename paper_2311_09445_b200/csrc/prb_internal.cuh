@@ -43,7 +43,10 @@ struct PrbBatch {
 };
 
 // Kernel launchers; each returns the number of kernels launched, or -1 on a launch error.
-int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s);
+// (upd_B > 0 runs a priority update of that batch before the insertion's tree work, in the same kernel)
+int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
+                      uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
+                      int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f);
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s);
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
@@ -177,8 +180,9 @@ struct PrbBulkLane {
         busy = done;
         if (!done) failed = true;
     }
-    // Before the CTA exits: this lane's stores are complete.
-    __device__ __forceinline__ void finish() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+    // Before the CTA exits: this lane's stores have read their stages (the writes themselves are
+    // complete when the kernel is, like any other store).
+    __device__ __forceinline__ void finish() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 };
 
 #endif  // __CUDACC__

@@ -88,6 +88,16 @@ class Pair:
             self.gpu.update(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
                             torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps)
 
+    def update_insert(self, idx, td, alpha, eps, batch):
+        """One fused launch on the GPU; update then insert on the oracle."""
+        assert self.ora.update(idx, td, alpha, eps) == 0
+        assert self.ora.insert(batch.get("obs"), batch.get("act"), batch.get("rew"), batch.get("next_obs"),
+                               batch.get("done"), batch["prio"]) == 0
+        d = {k: torch.from_numpy(np.ascontiguousarray(v)).to(self.dev) for k, v in batch.items() if v is not None}
+        self.gpu.update_insert(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                               torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps,
+                               d.get("obs"), d.get("act"), d.get("rew"), d.get("next_obs"), d.get("done"), d["prio"])
+
     def update_priorities(self, idx, prio):
         assert self.ora.update_priorities(idx, prio) == 0
         self.gpu.update_priorities(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),

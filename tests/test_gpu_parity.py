@@ -242,6 +242,34 @@ def test_host_buffer_calls(oracle_mod):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B,n", [(wk.CARTPOLE, 5000, 64, 64), (wk.DDPG, 70_000, 256, 256), (wk.DDPG, 3000, 1000, 777),
+                                      (wk.ATARI, 1500, 512, 512), (wk.ATARI, 700, 37, 1), (wk.ATARI, 700, 4096, 300)])
+def test_fused_update_insert(oracle_mod, wl, N, B, n):
+    # update + insert in one launch == update, then insert; the inserted slots overlap updated ones
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(B + n)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096)
+    chunk = min(N, 4096)
+    next_id = 0
+    for first in range(0, N + chunk, chunk):            # fill and wrap
+        m = min(chunk, N)
+        pr.insert(wk.transitions(wl, rng, m, next_id))
+        next_id += m
+    for step in range(5):
+        o, g = pr.sample(min(B, 4096), wl.beta, wl.philox_seed)
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        if step % 2 == 1:
+            rng.shuffle(idx)                               # unsorted batch: the sort path
+            idx[:3] = [(pr.ora.info()[1] + j) % N for j in range(3)]   # slots the insertion overwrites
+        pr.update_insert(idx, td, wl.alpha, wl.eps, wk.transitions(wl, rng, n, next_id))
+        next_id += n
+        pr.compare_tree()
+        pr.compare_state()
+    pr.compare_status()
+    pr.compare_rows(np.arange(0, N, max(1, N // 500), dtype=np.int32))
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)
