@@ -239,11 +239,24 @@ def run_ours(args, wl, rank, world):
                 o["idx"][dup_pos[i % ROTATE]] = o["idx"][dup_src[i % ROTATE]]
             prb.update(o["idx"], tds[i % ROTATE], wl.alpha, wl.eps)
 
+        def do_update_insert(i):
+            o, b = outs[i % ROTATE], batches[i % ROTATE]
+            if n_dup:
+                o["idx"][dup_pos[i % ROTATE]] = o["idx"][dup_src[i % ROTATE]]
+            prb.update_insert(o["idx"], tds[i % ROTATE], wl.alpha, wl.eps, b["obs"], b["act"], b["rew"], b["next_obs"],
+                              b["done"], b["prio"])
+
+        fused = bool(n_ins) and not args.unfused
+
         def eager_step(i):
-            if n_ins:
-                do_insert(i)
+            # the paper's schedule (Eq. 7): sample, then update with the insertion running beside it
             do_sample(i)
-            do_update(i)
+            if fused:
+                do_update_insert(i)
+            else:
+                do_update(i)
+                if n_ins:
+                    do_insert(i)
 
         for i in range(max(args.warmup, 3)):
             eager_step(i)
@@ -311,6 +324,7 @@ def run_ours(args, wl, rank, world):
         ms_sample = per_call_ms(do_sample)
         ms_update = per_call_ms(do_update)
         ms_insert = per_call_ms(do_insert) if n_ins else None
+        ms_fused = per_call_ms(do_update_insert) if fused else None
         status |= prb.sync()
 
         # ---- end to end through the host-buffer calls ----------------------------------------
@@ -363,13 +377,14 @@ def run_ours(args, wl, rank, world):
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
         "config": {"workload": wl.name, "capacity": wl.capacity, "fanout": wl.fanout, "depth": depth, "batch": B,
-                   "insert_per_step": n_ins, "transition_bytes": E, "step": "insert+sample(idx,IS,gather)+update",
+                   "insert_per_step": n_ins, "transition_bytes": E, "step": "sample(idx,IS,gather) + update_insert (one launch)" if fused else "sample(idx,IS,gather) + update + insert",
                    "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph,
                    "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
         "rates": {"samples_per_s": B / (ms_sample * 1e-3), "updates_per_s": B / (ms_update * 1e-3),
                   "inserts_per_s": (n_ins / (ms_insert * 1e-3)) if n_ins else None,
                   "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3,
-                  "us_insert": ms_insert * 1e3 if n_ins else None},
+                  "us_insert": ms_insert * 1e3 if n_ins else None,
+                  "us_update_insert": ms_fused * 1e3 if fused else None},
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes, "traffic": None},
@@ -419,6 +434,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="atari_dqn")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="update and insert as two launches instead of pearl_prb_update_insert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
