@@ -1,6 +1,6 @@
 // Sum-tree maintenance shared by the update and insert kernels: the priority transform, the
-// batched leaf update with last-writer-wins deduplication, and the re-sum of a contiguous range
-// of inserted leaves.  All of it is written for a "team": a whole number of warps of one CTA
+// batched leaf update with last-writer-wins deduplication, the leaves of an insertion, and the
+// level-by-level re-sum of every dirty ancestor.  All of it is written for a "team": a whole number of warps of one CTA
 // that synchronise on their own barrier, so that the same code runs as a full CTA (the update
 // kernel) or as a few warps beside the copy warps of an insert kernel.
 #pragma once
@@ -81,157 +81,225 @@ __device__ __forceinline__ bool prb_priority_pow(float delta, float eps, float a
 }
 
 constexpr unsigned long long kPrbInvalidKey = ~0ull;
+constexpr uint32_t kPrbNoParent = 0xFFFFFFFFu;
 
-// Shared memory an update of a batch padded to n2 entries needs: keys, then values.
-__host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
+// What the tree team does in one launch: an optional priority update (B > 0), then the tree part of
+// an optional insertion (n > 0).
+struct PrbTreeWork {
+    uint32_t B, n2;                 // update batch, and B rounded up to a power of two (>= 2)
+    const int32_t* idx;
+    const float* val;               // TD errors, or priorities if raw
+    int raw;
+    float alpha, eps;
+    uint32_t n;                     // inserted transitions
+    const float* prio;
+};
+
+// Shared memory the team needs: the update's keys and values, then per warp a 32 x (K+1) staging
+// area for the cooperative child loads (fanout >= 8 only).
+__host__ __device__ inline size_t prb_tree_smem_bytes(uint32_t n2_or_0, uint32_t fanout, uint32_t team_threads)
 {
-    return (size_t)n2 * (sizeof(unsigned long long) + sizeof(float));
+    size_t b = (size_t)n2_or_0 * (sizeof(unsigned long long) + sizeof(float));
+    b = (b + 15) / 16 * 16;
+    if (fanout >= 8) b += (size_t)(team_threads / 32) * 32 * (fanout + 1) * sizeof(float);
+    return b;
 }
 
-// Batched priority update by one team (PEARL Section V-A, "priority update", read as set +
-// re-sum).  Entries are keyed (index << 32) | batch position and sorted; the last entry of every
-// run of equal indices wins and writes its leaf; then, level by level from the deepest, the
-// first entry of every run of equal ancestors re-sums that ancestor from its children in
-// left-to-right order.  Sorted order survives dropping low digits of the index, so no list is
-// compacted and no lock is taken.  n2 = B rounded up to a power of two (>= 2); smem holds
-// prb_update_smem_bytes(n2) bytes.
-__device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam& team, uint32_t B, uint32_t n2,
-                                                const int32_t* __restrict__ idx, const float* __restrict__ val, int raw,
-                                                float alpha, float eps, unsigned char* smem)
+// Re-sums the parents named by slots [0, n_slots): slot_parent(slot) is a node of the parent level
+// or kPrbNoParent.  Each parent becomes the left-to-right binary32 sum of its K children.
+// Fanout >= 8: a warp takes 32 slots at a time, loads their child groups with coalesced 16-byte
+// loads (a group is K*4 contiguous bytes) into a padded staging area, and then every lane sums
+// its own group from shared memory; all the global loads of a pass are in flight together.
+template <int K, typename SlotParent>
+__device__ __forceinline__ void prb_resum_slots(const PrbTeam& team, const float* child, float* par, uint32_t n_slots,
+                                                SlotParent slot_parent, float* scratch)
 {
+    const uint32_t lane = team.rank & 31u, warp = team.rank >> 5, n_warps = team.size >> 5;
+    for (uint32_t base = warp * 32u; base < n_slots; base += n_warps * 32u) {
+        const uint32_t slot = base + lane;
+        const uint32_t a = slot < n_slots ? slot_parent(slot) : kPrbNoParent;
+        if constexpr (K <= 4) {
+            if (a != kPrbNoParent) par[a] = prb_sum_children<K>(child + (uint64_t)a * K);
+        } else {
+            if (!__any_sync(0xFFFFFFFFu, a != kPrbNoParent)) continue;
+            constexpr int G = K >= 8 ? K / 4 : 1;         // 16-byte units per child group
+            float* mine = scratch + (size_t)warp * 32 * (K + 1);
+            float4 c[G];
+            uint32_t loaded = 0;                          // bit t: unit t of this lane belongs to a live slot
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                const uint32_t u = (uint32_t)t * 32u + lane, job = u / G, part = u % G;
+                const uint32_t aj = __shfl_sync(0xFFFFFFFFu, a, job);
+                if (aj != kPrbNoParent) {
+                    c[t] = __ldcg(reinterpret_cast<const float4*>(child + (uint64_t)aj * K) + part);
+                    loaded |= 1u << t;
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                const uint32_t u = (uint32_t)t * 32u + lane, job = u / G, part = u % G;
+                if (loaded & (1u << t)) {
+                    float* d = mine + job * (K + 1) + part * 4;
+                    d[0] = c[t].x; d[1] = c[t].y; d[2] = c[t].z; d[3] = c[t].w;
+                }
+            }
+            __syncwarp();
+            if (a != kPrbNoParent) {
+                const float* g = mine + lane * (K + 1);
+                float sum = g[0];
+#pragma unroll
+                for (int j = 1; j < K; ++j) sum = __fadd_rn(sum, g[j]);
+                par[a] = sum;
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// The tree work of one launch by one team (PEARL Section V-A: priority update; insertion =
+// retrieval + update), read as SET + re-sum so that the result does not depend on scheduling.
+//   Update: entries are keyed (index << 32) | batch position and sorted (skipped if they already
+//   are, as indices straight from a stratified sample); the last entry of every run of equal
+//   indices wins and writes its leaf.
+//   Insertion: the n leaves of ring slots cursor .. cursor+n-1 (mod capacity) are written; they
+//   come after the update, so an updated leaf that is also inserted keeps the inserted priority.
+//   Then ONE pass per level, deepest first, re-sums every dirty parent: the first entry of every
+//   run of equal ancestors in the sorted update list (sorted order survives dropping low digits
+//   of the index, so nothing is compacted), and the contiguous parent range(s) of the inserted
+//   slots.  No lock is taken; a parent reached both ways is computed twice with the same result.
+// `fill` is the fill count before this launch (update indices must be below it).
+__device__ __forceinline__ void prb_tree_team(const PrbView& v, const PrbTeam& team, const PrbTreeWork& w,
+                                              uint64_t cursor, unsigned long long fill, unsigned char* smem)
+{
+    const uint32_t n2 = w.B ? w.n2 : 0u;
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
+    float* scratch = reinterpret_cast<float*>(smem + ((size_t)n2 * 12 + 15) / 16 * 16);
     const uint32_t rank = team.rank, nt = team.size;
-    const unsigned long long fill = v.state->fill;
-
-    unsigned flags = 0;
-    bool unsorted = false;
-    unsigned long long my_key = kPrbInvalidKey;      // the key of entry `rank` (one-key-per-thread case)
-    for (uint32_t b = rank; b < n2; b += nt) {
-        unsigned long long key = kPrbInvalidKey;
-        if (b < B) {
-            const int32_t i = idx[b];
-            float p = 0.0f;
-            bool ok_p;
-            if (raw) { p = val[b]; ok_p = prb_valid_priority(p); }
-            else ok_p = prb_priority_pow(val[b], eps, alpha, p);
-            if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
-            else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
-            else key = ((unsigned long long)(uint32_t)i << 32) | b;
-            vals[b] = p;
-        }
-        keys[b] = key;
-        my_key = key;
-    }
-    if (flags) atomicOr(&v.state->status, flags);
-    team.sync();
-
-    // Indices that come straight from a stratified sample are already in order; sort only if needed.
-    for (uint32_t b = rank; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
-    unsorted = team.sync_or(unsorted);
-
-    if (unsorted && n2 <= nt) {
-        // bitonic sort, one key per thread: exchanges across fewer than 32 positions are warp shuffles
-        unsigned long long key = (rank < n2) ? my_key : kPrbInvalidKey;
-        for (uint32_t k = 2; k <= n2; k <<= 1) {
-            for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-                unsigned long long other;
-                if (j >= 32) {
-                    if (rank < n2) keys[rank] = key;
-                    team.sync();
-                    other = (rank < n2) ? keys[rank ^ j] : kPrbInvalidKey;
-                    team.sync();
-                } else {
-                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
-                }
-                const bool keep_min = ((rank & k) == 0) == ((rank & j) == 0);
-                key = keep_min ? (key < other ? key : other) : (key > other ? key : other);
-            }
-        }
-        if (rank < n2) keys[rank] = key;
-        team.sync();
-    } else if (unsorted) {
-        // bitonic sort in shared memory, several keys per thread
-        for (uint32_t k = 2; k <= n2; k <<= 1) {
-            for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-                for (uint32_t t = rank; t < (n2 >> 1); t += nt) {
-                    const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
-                    const uint32_t hi = lo | j;
-                    const unsigned long long a = keys[lo], c = keys[hi];
-                    const bool up = (lo & k) == 0;
-                    if ((a > c) == up) { keys[lo] = c; keys[hi] = a; }
-                }
-                team.sync();
-            }
-        }
-    }
-
-    // winners write the leaves
-    float* leaves = v.level[v.depth];
-    for (uint32_t s = rank; s < n2; s += nt) {
-        const unsigned long long key = keys[s];
-        if (key == kPrbInvalidKey) continue;
-        const uint32_t i = (uint32_t)(key >> 32);
-        const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
-        if (last) leaves[i] = vals[(uint32_t)key];
-    }
-    team.sync();
-
-    // re-sum the ancestors, deepest level first
-    const uint32_t K = v.fanout, lg = v.log2_fanout;
-    for (int l = (int)v.depth - 1; l >= 0; --l) {
-        const uint32_t sh = lg * (v.depth - (uint32_t)l);
-        const float* child = v.level[l + 1];
-        float* par = v.level[l];
-        for (uint32_t s = rank; s < n2; s += nt) {
-            const unsigned long long key = keys[s];
-            if (key == kPrbInvalidKey) continue;
-            const uint32_t a = (uint32_t)(key >> 32) >> sh;
-            const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
-            if (first) par[a] = prb_sum_children_dyn(child + (uint64_t)a * K, K);
-        }
-        team.sync();
-    }
-}
-
-// Tree part of an insertion by one team: write the n leaves of ring slots cursor .. cursor+n-1
-// (mod capacity), then re-sum the dirty parents level by level.  A contiguous slot range dirties
-// a contiguous parent range on every level (two ranges if the ring wrapped), so nothing is sorted.
-__device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const PrbTeam& team, uint32_t n,
-                                                     const float* __restrict__ prio, uint64_t cursor)
-{
     const uint64_t N = v.capacity;
     const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
     float* leaves = v.level[D];
-    bool bad = false;
-    for (uint32_t t = team.rank; t < n; t += team.size) {
-        uint64_t slot = cursor + t;
-        if (slot >= N) slot -= N;
-        float p = prio[t];
-        if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
-        leaves[slot] = p;
+
+    if (w.B) {
+        unsigned flags = 0;
+        bool unsorted = false;
+        unsigned long long my_key = kPrbInvalidKey;      // the key of entry `rank` (one-key-per-thread case)
+        for (uint32_t b = rank; b < n2; b += nt) {
+            unsigned long long key = kPrbInvalidKey;
+            if (b < w.B) {
+                const int32_t i = w.idx[b];
+                float p = 0.0f;
+                bool ok_p;
+                if (w.raw) { p = w.val[b]; ok_p = prb_valid_priority(p); }
+                else ok_p = prb_priority_pow(w.val[b], w.eps, w.alpha, p);
+                if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
+                else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
+                else key = ((unsigned long long)(uint32_t)i << 32) | b;
+                vals[b] = p;
+            }
+            keys[b] = key;
+            my_key = key;
+        }
+        if (flags) atomicOr(&v.state->status, flags);
+        team.sync();
+
+        for (uint32_t b = rank; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
+        unsorted = team.sync_or(unsorted);
+
+        if (unsorted && n2 <= nt) {
+            // bitonic sort, one key per thread: exchanges across fewer than 32 positions are warp shuffles
+            unsigned long long key = (rank < n2) ? my_key : kPrbInvalidKey;
+            for (uint32_t k = 2; k <= n2; k <<= 1) {
+                for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+                    unsigned long long other;
+                    if (j >= 32) {
+                        if (rank < n2) keys[rank] = key;
+                        team.sync();
+                        other = (rank < n2) ? keys[rank ^ j] : kPrbInvalidKey;
+                        team.sync();
+                    } else {
+                        other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+                    }
+                    const bool keep_min = ((rank & k) == 0) == ((rank & j) == 0);
+                    key = keep_min ? (key < other ? key : other) : (key > other ? key : other);
+                }
+            }
+            if (rank < n2) keys[rank] = key;
+            team.sync();
+        } else if (unsorted) {
+            // bitonic sort in shared memory, several keys per thread
+            for (uint32_t k = 2; k <= n2; k <<= 1) {
+                for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+                    for (uint32_t t = rank; t < (n2 >> 1); t += nt) {
+                        const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
+                        const uint32_t hi = lo | j;
+                        const unsigned long long a = keys[lo], c = keys[hi];
+                        const bool up = (lo & k) == 0;
+                        if ((a > c) == up) { keys[lo] = c; keys[hi] = a; }
+                    }
+                    team.sync();
+                }
+            }
+        }
+
+        // winners write their leaves, unless the insertion below overwrites the slot anyway
+        for (uint32_t s = rank; s < n2; s += nt) {
+            const unsigned long long key = keys[s];
+            if (key == kPrbInvalidKey) continue;
+            const uint32_t i = (uint32_t)(key >> 32);
+            const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
+            const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;     // distance from the cursor along the ring
+            if (last && !(ahead < w.n)) leaves[i] = vals[(uint32_t)key];
+        }
     }
-    if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
+
+    if (w.n) {
+        bool bad = false;
+        for (uint32_t t = rank; t < w.n; t += nt) {
+            uint64_t slot = cursor + t;
+            if (slot >= N) slot -= N;
+            float p = w.prio[t];
+            if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+            leaves[slot] = p;
+        }
+        if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
+    }
     team.sync();
-    // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
+
+    // dirty leaf ranges of the insertion: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;
-    const uint64_t a1 = min(cursor + n, N) - 1;
-    const bool wrapped = cursor + n > N;
-    const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
+    const uint64_t a1 = (w.n ? min(cursor + w.n, N) : cursor + 1) - 1;
+    const bool wrapped = cursor + w.n > N;
+    const uint64_t b1 = wrapped ? cursor + w.n - N - 1 : 0;
+
     for (int l = (int)D - 1; l >= 0; --l) {
         const uint32_t sh = lg * (D - (uint32_t)l);
-        const uint64_t pa0 = a0 >> sh, pa1 = a1 >> sh;
-        const uint64_t cntA = pa1 - pa0 + 1;
-        uint64_t cntB = 0;
-        if (wrapped) {
-            const uint64_t pb1 = b1 >> sh;
-            cntB = (pa0 == 0) ? 0 : min(pb1, pa0 - 1) + 1;   // parents of B not already in A
+        uint32_t pa0 = 0, cntA = 0, cntB = 0;
+        if (w.n) {
+            pa0 = (uint32_t)(a0 >> sh);
+            cntA = (uint32_t)(a1 >> sh) - pa0 + 1;
+            if (wrapped) cntB = (pa0 == 0) ? 0u : min((uint32_t)(b1 >> sh), pa0 - 1) + 1;   // parents of B not already in A
         }
+        auto slot_parent = [&](uint32_t slot) -> uint32_t {
+            if (slot < n2) {
+                const unsigned long long key = keys[slot];
+                if (key == kPrbInvalidKey) return kPrbNoParent;
+                const uint32_t a = (uint32_t)(key >> 32) >> sh;
+                const bool first = (slot == 0) || (((uint32_t)(keys[slot - 1] >> 32) >> sh) != a);
+                return first ? a : kPrbNoParent;
+            }
+            const uint32_t i = slot - n2;
+            return i < cntA ? pa0 + i : i - cntA;
+        };
         const float* child = v.level[l + 1];
         float* par = v.level[l];
-        for (uint64_t i = team.rank; i < cntA + cntB; i += team.size) {
-            const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
-            par[j] = prb_sum_children_dyn(child + j * K, K);
+        const uint32_t n_slots = n2 + cntA + cntB;
+        switch (K) {
+        case 2: prb_resum_slots<2>(team, child, par, n_slots, slot_parent, scratch); break;
+        case 4: prb_resum_slots<4>(team, child, par, n_slots, slot_parent, scratch); break;
+        case 8: prb_resum_slots<8>(team, child, par, n_slots, slot_parent, scratch); break;
+        case 16: prb_resum_slots<16>(team, child, par, n_slots, slot_parent, scratch); break;
+        default: prb_resum_slots<32>(team, child, par, n_slots, slot_parent, scratch); break;
         }
         team.sync();
     }
