@@ -210,7 +210,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     }
     PrbTreeWork w;
     w.B = upd_B; w.n2 = 2; w.idx = upd_idx; w.val = upd_val; w.raw = upd_raw; w.alpha = alpha; w.eps = eps;
-    w.n = n; w.prio = d_prio;
+    w.n = n; w.prio = d_prio; w.forward = 0;
     while (w.n2 < upd_B) w.n2 <<= 1;
 
     InsertPlan plan;
@@ -237,7 +237,8 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
     if (tasks == 0) {
-        const uint32_t smem = (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamShort);
+        const uint32_t fwd = prb_fwd_plan(v, &w, kTeamShort, 96 * 1024);
+        const uint32_t smem = fwd ? fwd : (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamShort);
         static bool big_smem = false;
         if (smem + 64 > 48 * 1024 && !big_smem) {
             if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess)
@@ -253,7 +254,8 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
         uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
-        const uint32_t tree_smem = (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamRows);
+        const uint32_t fwd = prb_fwd_plan(v, &w, kTeamRows, kRingBarBytes + kRingBytes);
+        const uint32_t tree_smem = fwd ? fwd : (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamRows);
         if (tree_smem > smem) smem = tree_smem;
         static bool big_smem = false;
         if (!big_smem) {

@@ -27,10 +27,11 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
 {
     PrbTreeWork w;
     w.B = B; w.n2 = 2; w.idx = d_idx; w.val = d_val; w.raw = raw; w.alpha = alpha; w.eps = eps;
-    w.n = 0; w.prio = nullptr;
+    w.n = 0; w.prio = nullptr; w.forward = 0;
     while (w.n2 < B) w.n2 <<= 1;
     const uint32_t threads = w.n2 < 64 ? 64 : (w.n2 > 1024 ? 1024 : w.n2);
-    const size_t smem = prb_tree_smem_bytes(w.n2, v.fanout, threads);
+    const uint32_t fwd = prb_fwd_plan(v, &w, threads, 200 * 1024);
+    const size_t smem = fwd ? fwd : prb_tree_smem_bytes(w.n2, v.fanout, threads);
     static bool big_smem = false;
     if (smem > 48 * 1024 && !big_smem) {
         if (cudaFuncSetAttribute(prb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
