@@ -6,24 +6,23 @@
 // One kernel per call, in one of two shapes.
 //   Short rows: CTA 0 owns the tree, the other CTAs copy tiles of the dense batch to ring slots
 //   through registers.
-//   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; CTA 0 does the
-//   tree work, in every other CTA warp 0 drives bulk asynchronous copies global -> shared ->
-//   global through a ~200 KB ring (row chunks of <= 8 KB, one lane per stage), issuing its
-//   loads before the cursor has even arrived, and the other warps copy the short fields.
-// Tree work (prb_tree.cuh): an optional priority update first (pearl_prb_update_insert), then
-// the n leaves, then one re-sum pass per level over every dirty parent.
+//   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; warp 0 of
+//   every CTA drives bulk asynchronous copies global -> shared -> global through a ~200 KB
+//   ring (row chunks of <= 8 KB, one lane per stage), issuing its loads before the cursor has
+//   even arrived; the other warps copy the short fields, and in CTA 0 they first do the tree.
+// Tree work: write the n leaves, then re-sum the dirty parents level by level (a contiguous
+// slot range dirties a contiguous parent range on every level, so no sorting is needed).
 // The CTA that is last to have read the cursor advances it (and the fill count) while the copies
 // are still running.  No CTA waits on another.
 #include "prb_tree.cuh"
 
 namespace {
 
-constexpr int kTeamShort = 256;                  // short-row kernel: threads that copy tiles / do the tree work
-constexpr int kThreadsShort = kTeamShort + 32;   //   ... then the warp whose lane 0 publishes the cursor
-constexpr int kTeamRows = 960;                   // long-row kernel: warps 1..30 do the tree work / short fields
-constexpr int kThreadsRows = 32 + kTeamRows + 32;   //   warp 0 drives the ring, lane 0 of warp 31 publishes
+constexpr int kWorkers = 256;                // threads that copy short rows / do the tree work
+constexpr int kThreadsShort = kWorkers + 32;     // short-row kernel: workers, then the warp whose lane 0 publishes the cursor
+constexpr int kThreadsRows = 32 + kWorkers + 32; // long-row kernel: ring warp, workers, publishing warp
 constexpr uint32_t kChunk = 512;             // upper bound on granules per chunk of a long row (8 KB)
-constexpr uint32_t kTile = 2048;             // granules per tile of short rows
+constexpr uint32_t kTile = kWorkers * 8;     // granules per tile of short rows
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
 constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring (dynamic shared memory), <= 32 stages
 constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
@@ -74,9 +73,9 @@ __device__ __forceinline__ void copy_tile(const PrbView& v, const InsertPlan& pl
     }
 }
 
-// Taken by one thread per CTA once the whole CTA holds the cursor and the fill count: the last CTA
-// to get here publishes the new values.  Nothing later in the kernel reads them from global
-// memory, so this happens while the copies are still running.
+// Taken by one thread per CTA once the whole CTA holds the cursor: the last CTA to get here
+// publishes the new cursor and fill count.  Nothing later in the kernel reads them, so this
+// happens while the copies are still running.
 __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill)
 {
     __threadfence();
@@ -92,56 +91,68 @@ __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, ui
     }
 }
 
-// Short rows only: CTA 0 = the tree work (an optional priority update, then the insertion's leaves
-// and re-sum), CTAs 1.. = a contiguous range of tiles each.  Threads 0..kTeamShort-1 work; thread
-// kTeamShort reads cursor and fill for the CTA and takes the ticket.
+// A priority update to run before the insertion's tree work, by the same team (B == 0: none).
+struct FusedUpdate {
+    uint32_t B, n2;
+    const int32_t* idx;
+    const float* val;
+    int raw;
+    float alpha, eps;
+};
+
+// Short rows only: CTA 0 = tree (after the optional update), CTAs 1.. = a contiguous range of tiles
+// each.  Threads 0..kWorkers-1 work; thread kWorkers reads the cursor for the CTA and takes the ticket.
 __global__ void __launch_bounds__(kThreadsShort, 2)
-prb_insert_kernel(const __grid_constant__ PrbView v, const __grid_constant__ PrbBatch src,
-                  const __grid_constant__ InsertPlan plan, const __grid_constant__ PrbTreeWork work)
+prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
+                  const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
+                  const __grid_constant__ FusedUpdate upd)
 {
     extern __shared__ __align__(16) unsigned char s_dyn[];
-    __shared__ unsigned long long s_cursor, s_fill;
-    const uint32_t tid = threadIdx.x, n = work.n;
-    if (tid == kTeamShort) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
+    __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
+    const uint32_t tid = threadIdx.x;
+    if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
     __syncthreads();
     const uint64_t cursor = s_cursor;
-    if (tid == kTeamShort) {
+    if (tid == kWorkers) {
         publish_if_last(v, n, cursor, s_fill);
-    } else if (tid < kTeamShort) {
+    } else if (tid < kWorkers) {
         if (blockIdx.x == 0) {
             PrbTeam team;
-            team.rank = tid; team.size = kTeamShort; team.whole_cta = false;
-            prb_tree_team(v, team, work, cursor, s_fill, s_dyn);
+            team.rank = tid; team.size = kWorkers; team.whole_cta = false;
+            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn);
+            prb_insert_tree_team(v, team, n, prio, cursor);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
             const uint32_t t_lo = (uint32_t)(((uint64_t)c * n_tiles) / copy_ctas);
             const uint32_t t_hi = (uint32_t)(((uint64_t)(c + 1) * n_tiles) / copy_ctas);
-            for (uint32_t t = t_lo; t < t_hi; ++t) copy_tile(v, plan, src, n, cursor, t, tid, kTeamShort);
+            for (uint32_t t = t_lo; t < t_hi; ++t) copy_tile(v, plan, src, n, cursor, t, tid, kWorkers);
         }
     }
 }
 
-// Long rows present.  CTA 0 does the tree work (optional update, then the insertion) with warps
-// 1..30 and moves no rows.  In the other CTAs warp 0 drives the ring: lane s owns stage s and moves
-// row chunks t_lo+s, t_lo+s+S, ... of the CTA's range, its first load going out before the cursor
-// has arrived (a source address does not depend on it); warps 1..30 copy the short-field tiles,
-// dealt round-robin.  Lane 0 of warp 31: cursor, fill and ticket.
+// Long rows present.  Warp 0: lane s owns ring stage s and moves row chunks t_lo+s, t_lo+s+S, ...
+// of this CTA's range; the first loads go out before the cursor has arrived (a source address does
+// not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, after the optional update)
+// and the short-field tiles (dealt round-robin, CTA 1 first).  Thread 32+kWorkers: cursor and
+// ticket.  With an update fused in, CTA 0 moves no rows: its ring memory holds the update's keys.
 __global__ void __launch_bounds__(kThreadsRows, 1)
-prb_insert_rows_kernel(const __grid_constant__ PrbView v, const __grid_constant__ PrbBatch src,
-                       const __grid_constant__ InsertPlan plan, const __grid_constant__ PrbTreeWork work)
+prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
+                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
+                       const __grid_constant__ FusedUpdate upd)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
-    __shared__ unsigned long long s_cursor, s_fill;
-    const uint32_t tid = threadIdx.x, n = work.n;
+    __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
+    const uint32_t tid = threadIdx.x;
     const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-    const uint32_t copy_ctas = gridDim.x - 1;
-    const bool copies = blockIdx.x > 0;
-    const uint32_t c = blockIdx.x - 1;
+    const uint32_t first_copy_cta = upd.B ? 1u : 0u;
+    const uint32_t copy_ctas = gridDim.x - first_copy_cta;
+    const bool copies = blockIdx.x >= first_copy_cta;
+    const uint32_t c = blockIdx.x - first_copy_cta;
     const uint32_t t_lo = copies ? (uint32_t)(((uint64_t)c * n_tasks) / copy_ctas) : 0u;
     const uint32_t t_hi = copies ? (uint32_t)(((uint64_t)(c + 1) * n_tasks) / copy_ctas) : 0u;
     const bool ring_lane = copies && tid < plan.ring_stages;
-    constexpr uint32_t kPublisher = 32 + kTeamRows;
+    constexpr uint32_t kPublisher = 32 + kWorkers;
 
     // one row chunk: field, row in the batch, first granule, bytes
     auto locate = [&](uint32_t t, int& f, uint32_t& row, uint32_t& W, uint32_t& e0, uint32_t& bytes) {
@@ -185,14 +196,14 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, const __grid_constant_
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
     } else if (tid >= 32 && tid < kPublisher) {
         PrbTeam team;
-        team.rank = tid - 32u; team.size = kTeamRows; team.whole_cta = false;
+        team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
         if (blockIdx.x == 0) {
-            prb_tree_team(v, team, work, cursor, s_fill, s_ring);
-        } else {
-            const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
-            for (uint32_t tile = c; tile < n_tiles; tile += copy_ctas)
-                copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
+            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_ring);
+            prb_insert_tree_team(v, team, n, prio, cursor);
         }
+        const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
+        for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
+            copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
     }
 }
 
@@ -208,10 +219,9 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
             sm_count = 148;
     }
-    PrbTreeWork w;
-    w.B = upd_B; w.n2 = 2; w.idx = upd_idx; w.val = upd_val; w.raw = upd_raw; w.alpha = alpha; w.eps = eps;
-    w.n = n; w.prio = d_prio; w.forward = 0;
-    while (w.n2 < upd_B) w.n2 <<= 1;
+    FusedUpdate upd;
+    upd.B = upd_B; upd.n2 = 2; upd.idx = upd_idx; upd.val = upd_val; upd.raw = upd_raw; upd.alpha = alpha; upd.eps = eps;
+    while (upd.n2 < upd_B) upd.n2 <<= 1;
 
     InsertPlan plan;
     uint32_t tiles = 0, tasks = 0, stage = 0;
@@ -236,27 +246,31 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     plan.first_task[PRB_NUM_FIELDS] = tasks;
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
+    int launches = 1;
+    if (tasks > 0 && upd.B) {
+        // Long rows: measured faster as two launches.  Under the copy's memory traffic the update's
+        // chain of dependent tree reads runs at twice its idle latency and outlasts the copy.
+        if (prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, s) < 0) return -1;
+        upd.B = 0;
+        launches = 2;
+    }
+    const uint32_t upd_smem = upd.B ? (uint32_t)prb_update_smem_bytes(upd.n2) : 0u;
     if (tasks == 0) {
-        const uint32_t fwd = prb_fwd_plan(v, &w, kTeamShort, 96 * 1024);
-        const uint32_t smem = fwd ? fwd : (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamShort);
         static bool big_smem = false;
-        if (smem + 64 > 48 * 1024 && !big_smem) {
-            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess)
+        if (upd_smem + 64 > 48 * 1024 && !big_smem) {
+            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
                 return -1;
             big_smem = true;
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, src, plan, w);
+        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem, s>>>(v, n, src, d_prio, plan, upd);
     } else {
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
         plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
-        uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
-        const uint32_t fwd = prb_fwd_plan(v, &w, kTeamRows, kRingBarBytes + kRingBytes);
-        const uint32_t tree_smem = fwd ? fwd : (uint32_t)prb_tree_smem_bytes(upd_B ? w.n2 : 0u, v.fanout, kTeamRows);
-        if (tree_smem > smem) smem = tree_smem;
+        const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;     // >= the update's keys (<= 48 KB)
         static bool big_smem = false;
         if (!big_smem) {
             if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -264,9 +278,9 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
                 return -1;
             big_smem = true;
         }
-        const uint32_t want = tasks + 1;                           // CTA 0 is the tree CTA
+        const uint32_t want = tasks + (upd.B ? 1u : 0u);           // with an update, CTA 0 moves no rows
         const uint32_t grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
-        prb_insert_rows_kernel<<<grid, kThreadsRows, smem, s>>>(v, src, plan, w);
+        prb_insert_rows_kernel<<<grid, kThreadsRows, smem < upd_smem ? upd_smem : smem, s>>>(v, n, src, d_prio, plan, upd);
     }
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

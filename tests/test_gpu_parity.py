@@ -270,6 +270,25 @@ def test_fused_update_insert(oracle_mod, wl, N, B, n):
     pr.close()
 
 
+@pytest.mark.parametrize("wl", [wk.CARTPOLE, wk.ATARI])
+def test_fused_update_uses_fill_before_insert(oracle_mod, wl):
+    # In the fused call the update comes first: an index that only the insertion makes valid is refused.
+    wl = wk.scaled(wl, 400)
+    rng = np.random.default_rng(3)
+    pr = Pair(oracle_mod, 400, wl.fanout, wl.obs_bytes, wl.act_bytes, 256)
+    pr.insert(wk.transitions(wl, rng, 100, 0))
+    for rep in range(20):
+        idx = np.array([5, 99, 100, 120, 149, 7], dtype=np.int32)       # fill is 100 before, 150 after
+        td = rng.standard_normal(6).astype(np.float32)
+        pr.update_insert(idx, td, 0.6, 1e-6, wk.transitions(wl, rng, 50, 100))
+        pr.compare_tree()
+        assert pr.compare_status() == 1
+        pr.close()
+        pr = Pair(oracle_mod, 400, wl.fanout, wl.obs_bytes, wl.act_bytes, 256)
+        pr.insert(wk.transitions(wl, rng, 100, 0))
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)
