@@ -377,7 +377,7 @@ def run_ours(args, wl, rank, world):
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
         "config": {"workload": wl.name, "capacity": wl.capacity, "fanout": wl.fanout, "depth": depth, "batch": B,
-                   "insert_per_step": n_ins, "transition_bytes": E, "step": "sample(idx,IS,gather) + update_insert (one launch)" if fused else "sample(idx,IS,gather) + update + insert",
+                   "insert_per_step": n_ins, "transition_bytes": E, "step": "sample(idx,IS,gather) + update_insert" if fused else "sample(idx,IS,gather) + update + insert",
                    "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph,
                    "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
         "rates": {"samples_per_s": B / (ms_sample * 1e-3), "updates_per_s": B / (ms_update * 1e-3),
