@@ -31,6 +31,9 @@ METRIC = "PRB sample+update transitions/s at batch B"
 UNIT = "transitions/s"
 ROTATE = 8           # distinct input/output batch buffers cycled through, so inputs exceed L2 where rows are long
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one prb_sample_kernel launch on Atari-shaped rows with B = 512, from the
+# ncu capture summarised in profiles/prb_kernels_atari_N32768.md.  Null it if that kernel changes.
+SAMPLE_TRAFFIC_NCU = {"atari_dqn": 29.6e6}
 
 
 def load_peak():
@@ -387,7 +390,8 @@ def run_ours(args, wl, rank, world):
                   "us_update_insert": ms_fused * 1e3 if fused else None},
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
-                     "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes, "traffic": None},
+                     "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes,
+                     "traffic": SAMPLE_TRAFFIC_NCU.get(wl.name) if B == 512 else None},
         "e2e": {"value": None if args.no_e2e else world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(kernels_per_step * args.steps),
