@@ -1,6 +1,6 @@
 #!/usr/bin/env python
-"""Benchmark of the prioritized-replay hot path: one step = insert + sample (indices, IS weights,
-gather) + priority update on one batch of synthetic transitions.
+"""Benchmark of the prioritized-replay hot path: one step = sample (indices, IS weights, gather) +
+priority update + insert (pearl_prb_update_insert) on one batch of synthetic transitions.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
