@@ -180,6 +180,15 @@ def out_buffers(wl, dev, B, pinned=False):
             "done": torch.zeros(B, dtype=torch.uint8, **kw)}
 
 
+def max_over_ranks(value, device):
+    """The maximum of `value` over all ranks of the default process group (every rank gets it)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def time_loop(stream, fn, iters):
     """Milliseconds for `iters` calls of fn(i), CUDA events on `stream`, synchronised on both sides."""
     import torch
@@ -306,9 +315,7 @@ def run_ours(args, wl, rank, world):
         ms = time_loop(stream, lambda i: run_steps(args.steps), 1)
         if world > 1:
             dist.barrier()
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+            ms = max_over_ranks(ms, dev)
         clk = clocks.stop() if rank == 0 else None
 
         # ---- per-call timings (device resident), used for the roofline and the rates: a graph of
@@ -354,9 +361,7 @@ def run_ours(args, wl, rank, world):
         ms_e2e = time_loop(stream, e2e_step, e2e_steps) if not args.no_e2e else float("nan")
         if world > 1:
             dist.barrier()
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+            ms_e2e = max_over_ranks(ms_e2e, dev)
         status |= prb.sync()
         fill, cursor, calls, depth = prb.info()
         prb.close()

@@ -56,8 +56,10 @@ typedef struct pearl_layout {
 #define PEARL_ST_CLAMPED 8u        /* a descent met residual >= last prefix sum and took the last positive child */
 #define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out */
 
-/* Largest batch the update calls accept, whatever max_batch says. */
-#define PEARL_MAX_UPDATE_BATCH 4096u
+/* Update batches larger than this are applied as consecutive sub-batches of this many entries, in
+ * batch order, one launch each; the result is that of the whole batch (the last valid entry of a
+ * repeated index still wins, and the tree is re-summed after every sub-batch). */
+#define PEARL_UPDATE_SUBBATCH 4096u
 
 /* Bytes of device memory a buffer of this geometry needs (tree, storage, scratch and the
  * staging areas of the *_host calls).  0 if the arguments are invalid. */
@@ -113,7 +115,7 @@ int pearl_prb_sample(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, in
  * and leaf[d_idx[b]] <- p_b, so the last valid entry of a repeated index wins; then every
  * ancestor of a written leaf is recomputed as the left-to-right binary32 sum of its children,
  * deepest level first.  The power is evaluated in binary64 from IEEE basic operations only, so
- * it is reproducible bit for bit.  1 <= B <= min(max_batch, PEARL_MAX_UPDATE_BATCH);
+ * it is reproducible bit for bit.  1 <= B <= max_batch;
  * alpha, eps finite and >= 0. */
 int pearl_prb_update(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_td,
                      float alpha, float eps);

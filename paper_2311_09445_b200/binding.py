@@ -16,7 +16,6 @@ import torch
 from . import build as _build
 
 ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL = 1, 2, 4, 8, 16
-MAX_UPDATE_BATCH = 4096
 
 
 class PearlError(RuntimeError):

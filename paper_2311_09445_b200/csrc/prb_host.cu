@@ -241,7 +241,7 @@ static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const
                          float eps)
 {
     if (!h || !d_idx || !d_val) return PEARL_ERR_NULL;
-    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (!raw && (!finite_nonneg(alpha) || !finite_nonneg(eps))) return PEARL_ERR_BAD_ARG;
     if (misaligned(d_idx, 4) || misaligned(d_val, 4)) return PEARL_ERR_ALIGN;
     DeviceGuard guard(h->device);
@@ -267,7 +267,7 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
                             const uint8_t* d_done, const float* d_prio)
 {
     if (!h || !d_idx || !d_td || !d_prio) return PEARL_ERR_NULL;
-    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
     if (!finite_nonneg(alpha) || !finite_nonneg(eps)) return PEARL_ERR_BAD_ARG;
@@ -342,7 +342,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
 int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, const float* h_td, float alpha, float eps)
 {
     if (!h || !h_idx || !h_td) return PEARL_ERR_NULL;
-    if (B == 0 || B > h->max_batch || B > PEARL_MAX_UPDATE_BATCH) return PEARL_ERR_BAD_BATCH;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
     int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_idx);

@@ -247,12 +247,14 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
     int launches = 1;
-    if (tasks > 0 && upd.B) {
+    if (upd.B && (tasks > 0 || upd.B > PEARL_UPDATE_SUBBATCH)) {
         // Long rows: measured faster as two launches.  Under the copy's memory traffic the update's
         // chain of dependent tree reads runs at twice its idle latency and outlasts the copy.
-        if (prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, s) < 0) return -1;
+        // (A batch beyond one sub-batch is likewise updated by launches of its own.)
+        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, s);
+        if (k < 0) return -1;
         upd.B = 0;
-        launches = 2;
+        launches = 1 + k;
     }
     const uint32_t upd_smem = upd.B ? (uint32_t)prb_update_smem_bytes(upd.n2) : 0u;
     if (tasks == 0) {

@@ -26,9 +26,17 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s)
 {
-    uint32_t n2 = 2;
-    while (n2 < B) n2 <<= 1;
-    const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
-    prb_update_kernel<<<1, threads, prb_update_smem_bytes(n2), s>>>(v, B, n2, d_idx, d_val, raw, alpha, eps);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    // A batch beyond one CTA's reach goes sub-batch by sub-batch in batch order: every launch leaves
+    // a consistent tree and later entries overwrite earlier ones, as in the whole batch.
+    int launches = 0;
+    for (uint32_t first = 0; first < B; first += PEARL_UPDATE_SUBBATCH) {
+        const uint32_t b = B - first < PEARL_UPDATE_SUBBATCH ? B - first : PEARL_UPDATE_SUBBATCH;
+        uint32_t n2 = 2;
+        while (n2 < b) n2 <<= 1;
+        const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
+        prb_update_kernel<<<1, threads, prb_update_smem_bytes(n2), s>>>(v, b, n2, d_idx + first, d_val + first, raw, alpha, eps);
+        if (cudaGetLastError() != cudaSuccess) return -1;
+        ++launches;
+    }
+    return launches;
 }

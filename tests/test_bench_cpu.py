@@ -1,0 +1,65 @@
+"""bench.py pieces that need no GPU: the CPU-oracle arm, and the multi-rank plumbing over gloo."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from conftest import ROOT
+
+
+def _run(cmd, **kw):
+    return subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=600, **kw)
+
+
+def test_reference_arm_prints_one_contract_line():
+    r = _run([sys.executable, "bench.py", "--impl", "reference", "--workload", "tiny", "--steps", "50", "--warmup", "3"])
+    assert r.returncode == 0, r.stderr
+    lines = [ln for ln in r.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "transitions/s" and d["higher_is_better"] is True
+    assert d["value"] > 0 and d["steps"] == 50 and d["gpu_launches"] == 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["value"] == d["value"]
+    assert d["config"]["workload"] == "tiny"
+
+
+def test_reference_arm_under_torchrun_two_ranks():
+    # launched the way a multi-GPU run is: rank 0 alone works and prints, rank 1 exits 0 silently
+    r = _run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+              "127.0.0.1", "--master-port", "29541", "bench.py", "--impl", "reference", "--gpus", "2", "--workload", "tiny",
+              "--steps", "20", "--warmup", "2"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2
+
+
+def _rank_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    dist.barrier()
+    got = bench.max_over_ranks(10.0 + 5.0 * rank, torch.device("cpu"))       # each rank's own "time"
+    out.put((rank, got))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_time_is_max_over_ranks_gloo():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, 29543, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == {0: 15.0, 1: 15.0}

@@ -200,8 +200,7 @@ def test_sweep_cells(oracle_mod, N, K, B):
     for step in range(3):
         pr.insert(wk.transitions(wl, rng, wl.n_insert))
         o, g = pr.sample(B, wl.beta, wl.philox_seed)
-        Bu = min(B, 4096)
-        idx, td = wk.update_batch(wl, rng, o["idx"][:Bu])
+        idx, td = wk.update_batch(wl, rng, o["idx"])
         pr.update(idx, td, wl.alpha, wl.eps)
         pr.compare_tree()
     pr.compare_state()
@@ -286,6 +285,26 @@ def test_fused_update_uses_fill_before_insert(oracle_mod, wl):
         pr.close()
         pr = Pair(oracle_mod, 400, wl.fanout, wl.obs_bytes, wl.act_bytes, 256)
         pr.insert(wk.transitions(wl, rng, 100, 0))
+    pr.close()
+
+
+@pytest.mark.parametrize("K,B", [(2, 4097), (16, 10_000), (32, 65536)])
+def test_update_beyond_one_subbatch(oracle_mod, K, B):
+    # Sub-batches of 4096 in batch order: duplicates that span sub-batches, unsorted, some invalid.
+    rng = np.random.default_rng(K + B)
+    N = 30_000
+    pr = Pair(oracle_mod, N, K, 0, 0, 65536)
+    pr.insert(dict(prio=rng.uniform(0.1, 1, N).astype(np.float32)))
+    for _ in range(3):
+        idx = rng.integers(0, 2000, size=B).astype(np.int32)       # every index many times over
+        idx[::1000] = -1
+        td = rng.standard_normal(B).astype(np.float32)
+        pr.update(idx, td, 0.6, 1e-6)
+        pr.compare_tree()
+        pr.update_insert(idx[::-1].copy(), td, 0.6, 1e-6, dict(prio=rng.uniform(0.1, 1, 100).astype(np.float32)))
+        pr.compare_tree()
+        assert pr.compare_status() == 1
+    pr.compare_state()
     pr.close()
 
 
