@@ -207,6 +207,42 @@ def test_sweep_cells(oracle_mod, N, K, B):
     pr.close()
 
 
+@pytest.mark.parametrize("K", [2, 32])
+def test_largest_sweep_capacity(oracle_mod, K):
+    # 2^26 slots (depth 26 for fanout 2): the oracle mirrors the tree and the short fields; the 11 GB
+    # of observations live on the device only.
+    N, B = 1 << 26, 4096
+    free, _ = torch.cuda.mem_get_info()
+    if free < (14 << 30):
+        pytest.skip("not enough free device memory")
+    wl = wk.sweep_cell(N, K, B, cell_id=K)
+    rng = np.random.default_rng(wl.seed)
+    pr = Pair(oracle_mod, N, K, wl.obs_bytes, wl.act_bytes, 1 << 18, oracle_store=False)
+    dev = pr.dev
+    chunk = 1 << 18
+    obs = torch.zeros((chunk, wl.obs_bytes), dtype=torch.uint8, device=dev)      # same rows for every chunk
+    act = torch.zeros((chunk, wl.act_bytes), dtype=torch.uint8, device=dev)
+    for first in range(0, N, chunk):
+        prio = wk.priorities(wl, rng, chunk)
+        rew = rng.standard_normal(chunk).astype(np.float32)
+        done = np.zeros(chunk, np.uint8)
+        d = dict(obs=obs, next_obs=obs, act=act, rew=torch.from_numpy(rew).to(dev), done=torch.from_numpy(done).to(dev),
+                 prio=torch.from_numpy(prio).to(dev))
+        pr.insert(dict(rew=rew, done=done, prio=prio), dev_batch=d)
+    pr.compare_tree(range(0, pr.ora.depth - 1))
+    pr.compare_state()
+    assert pr.gpu.depth == (26 if K == 2 else 6)
+    for step in range(3):
+        o, g = pr.sample(B, wl.beta, wl.philox_seed)
+        rows = pr.ora.read_rows(o["idx"])
+        assert np.array_equal(g["rew"], rows["rew"])
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)
+        pr.compare_tree(range(0, pr.ora.depth - 1))
+    pr.compare_tree()
+    pr.close()
+
+
 def test_priority_transform_bits(oracle_mod):
     # The power is compared through the leaves it writes: 4096 TD errors x several exponents.
     rng = np.random.default_rng(21)
