@@ -174,6 +174,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     __shared__ float s_top[kTopFloats];
     __shared__ uint32_t s_idx[R];
     __shared__ double s_wraw[R];
+    __shared__ float s_p[R];
+    __shared__ unsigned s_flags[R];
     __shared__ unsigned int s_last;
     extern __shared__ __align__(128) unsigned char s_ring[];   // long rows: mbarriers, then the ring buffers
 
@@ -237,19 +239,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (walks) {
                 uint32_t leaf; float p; unsigned flags = 0;
                 descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
-                if (lane == 0 && gi < n_round) {
-                    s_idx[gi] = leaf;
-                    double wr = 0.0;
-                    if (kb + gi >= k_own) {
-                        const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)p), total);
-                        wr = pow(scaled, -(double)beta);
-                        out_idx[k] = (int32_t)leaf;
-                        v.wraw[k] = wr;
-                        if (flags) atomicOr(&v.state->status, flags);
-                        __threadfence();
-                    }
-                    s_wraw[gi] = wr;
-                }
+                if (lane == 0 && gi < n_round) { s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags; }
             }
             __syncthreads();
         }
@@ -257,6 +247,22 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         // From here the CTA splits by role: threads 0..127 copy, threads 128..255 look after the weights.
         const bool last_descents = round + 1 >= n_rounds;      // true exactly once per CTA
         if (tid >= kThreads / 2) {
+            // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path)
+            const uint32_t gi2 = tid - kThreads / 2;
+            if (gi2 < n_round) {
+                double wr = 0.0;
+                if (kb + gi2 >= k_own) {
+                    const uint32_t k2 = kb + gi2;
+                    const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
+                    wr = pow(scaled, -(double)beta);
+                    out_idx[k2] = (int32_t)s_idx[gi2];
+                    v.wraw[k2] = wr;
+                    if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
+                    __threadfence();
+                }
+                s_wraw[gi2] = wr;
+            }
+            asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
             if (tid == kThreads / 2) {
                 double m = 0.0;
                 for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
