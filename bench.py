@@ -202,6 +202,42 @@ def time_loop(stream, fn, iters):
     return e0.elapsed_time(e1)
 
 
+def copy_context(wl, store_rows, dev, stream):
+    """Library kernels on the same bytes, for context only (they are not on the product path): a dense
+    torch copy of one batch of observation rows, and torch.index_select of B random rows with the
+    indices already known.  Microseconds per batch, graphs of ROTATE calls like the per-call timings."""
+    import torch
+    B, W = wl.batch, wl.obs_bytes
+    rows = min(store_rows, 1 << 16)
+    with torch.cuda.stream(stream):
+        store = torch.empty((2, rows, W), dtype=torch.uint8, device=dev).random_(0, 255)
+        outs = [torch.empty((2, B, W), dtype=torch.uint8, device=dev) for _ in range(ROTATE)]
+        srcs = [torch.empty((2, B, W), dtype=torch.uint8, device=dev).random_(0, 255) for _ in range(ROTATE)]
+        idxs = [torch.sort(torch.randint(0, rows, (B,), device=dev))[0] for _ in range(ROTATE)]
+
+        def timed(fn):
+            for r in range(ROTATE):
+                fn(r)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for r in range(ROTATE):
+                    fn(r)
+            g.replay()
+            return time_loop(stream, lambda i: g.replay(), 25) * 1e3 / (25 * ROTATE)
+
+        def gather(r):
+            torch.index_select(store[0], 0, idxs[r], out=outs[r][0])
+            torch.index_select(store[1], 0, idxs[r], out=outs[r][1])
+
+        us_copy = timed(lambda r: outs[r].copy_(srcs[r]))
+        us_gather = timed(gather)
+    nbytes = 4 * B * W
+    return {"bytes": nbytes, "torch_dense_copy_us": us_copy, "torch_dense_copy_gbs": nbytes / us_copy / 1e3,
+            "torch_index_select_us": us_gather, "torch_index_select_gbs": nbytes / us_gather / 1e3,
+            "note": "library kernels on the same observation bytes (read+write), indices given; context, not the product path"}
+
+
 def run_ours(args, wl, rank, world):
     import torch
     import torch.distributed as dist
@@ -365,6 +401,9 @@ def run_ours(args, wl, rank, world):
         status |= prb.sync()
         fill, cursor, calls, depth = prb.info()
         prb.close()
+        ctx = None
+        if rank == 0 and world == 1 and wl.obs_bytes >= 8192 and not args.no_copy_context:
+            ctx = copy_context(wl, wl.capacity, dev, stream)
 
     if world > 1:
         dist.destroy_process_group()
@@ -409,6 +448,8 @@ def run_ours(args, wl, rank, world):
         line["roofline_insert"] = {"kernel": "prb_insert_kernel", "bound": "hbm", "bytes_per_launch": ins_bytes,
                                    "achieved": ins_bytes / (ms_insert * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                                    "frac": ins_bytes / (ms_insert * 1e-3) / 1e9 / peak}
+    if ctx is not None:
+        line["roofline"]["context"] = ctx
     if world == 1 and not args.no_cpu_baseline:
         done, dt, sample = time_oracle(wl, 10 ** 9, 2, budget_s=args.cpu_budget)
         line["cpu_baseline"] = {"value": B * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
@@ -446,6 +487,7 @@ def main():
     ap.add_argument("--unfused", action="store_true", help="update and insert as two launches instead of pearl_prb_update_insert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-copy-context", action="store_true", help="skip the torch copy / index_select context timings")
     ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
     args = ap.parse_args()
