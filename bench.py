@@ -208,7 +208,8 @@ def copy_context(wl, store_rows, dev, stream):
     indices already known.  Microseconds per batch, graphs of ROTATE calls like the per-call timings."""
     import torch
     B, W = wl.batch, wl.obs_bytes
-    rows = min(store_rows, 1 << 16)
+    free, _ = torch.cuda.mem_get_info(dev)
+    rows = store_rows if 2 * store_rows * W + (4 << 30) < free + torch.cuda.memory_reserved(dev) else min(store_rows, 1 << 16)
     with torch.cuda.stream(stream):
         store = torch.empty((2, rows, W), dtype=torch.uint8, device=dev).random_(0, 255)
         outs = [torch.empty((2, B, W), dtype=torch.uint8, device=dev) for _ in range(ROTATE)]
@@ -235,6 +236,7 @@ def copy_context(wl, store_rows, dev, stream):
     nbytes = 4 * B * W
     return {"bytes": nbytes, "torch_dense_copy_us": us_copy, "torch_dense_copy_gbs": nbytes / us_copy / 1e3,
             "torch_index_select_us": us_gather, "torch_index_select_gbs": nbytes / us_gather / 1e3,
+            "store_rows": rows,
             "note": "library kernels on the same observation bytes (read+write), indices given; context, not the product path"}
 
 
