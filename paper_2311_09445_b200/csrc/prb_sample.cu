@@ -11,16 +11,17 @@
 // rows is Listing 2's `D_storage[sampled_indices]`.  Stratification, the Philox stream and the
 // weights follow the prioritized-replay reference the paper cites (Schaul et al.).
 //
-// Work split: the batch is cut into tasks (a stratum, or one <= 16 KB chunk of one long row of
+// Work split: the batch is cut into tasks (a stratum, or one <= 8 KB chunk of one long row of
 // a stratum) and every CTA of a grid that fits the GPU in one wave takes a contiguous range of
 // tasks.  A CTA first walks the tree for the strata its tasks touch (a stratum shared by two
-// CTAs is walked by both: L2 reads only), then copies.  So the chain of dependent tree reads
-// is paid once, and from then on all SMs stream rows.  Long rows (Atari-shaped) move as bulk
-// asynchronous copies global -> shared -> global driven by one thread per CTA, one CTA per SM
-// with a ~200 KB ring, so that nearly the whole read set of a batch is in flight at once;
-// short rows are copied through registers.  Raw weights go to scratch; the CTA that
-// is last to finish its descents normalises them by the batch maximum and bumps the call
-// counter while the others are already copying.  No CTA ever waits on another.
+// CTAs is walked by both: L2 reads only), then splits by role: threads 0..127 copy, threads
+// 128..255 turn leaf priorities into raw weights.  So the chain of dependent tree reads is paid
+// once, and from then on all SMs stream rows.  Long rows (Atari-shaped) move as bulk
+// asynchronous copies global -> shared -> global driven by warp 0, one lane per stage of a
+// ~200 KB ring, one CTA per SM, so that nearly the whole read set of a batch is in flight at
+// once; short rows are copied through registers.  Raw weights go to scratch; the CTA that is
+// last to finish its descents normalises them by the batch maximum and bumps the call counter
+// while the others are already copying.  No CTA ever waits on another.
 #include "prb_internal.cuh"
 #include "../../include/pearl_prb.h"
 
