@@ -119,8 +119,10 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
         if (blockIdx.x == 0) {
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
-            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn);
-            prb_insert_tree_team(v, team, n, prio, cursor);
+            if (upd.B)      // update and insertion share one re-sum pass per level
+                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor);
+            else
+                prb_insert_tree_team(v, team, n, prio, cursor);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;

@@ -95,9 +95,16 @@ __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
 // left-to-right order.  Sorted order survives dropping low digits of the index, so no list is
 // compacted and no lock is taken.  n2 = B rounded up to a power of two (>= 2); smem holds
 // prb_update_smem_bytes(n2) bytes; fill = the fill count before this launch (indices must be below it).
+// With n > 0 the tree part of an insertion of n transitions at `cursor` follows in the same
+// passes: the inserted leaves are written after the update's (an updated leaf that is also
+// inserted keeps the inserted priority), and every level is re-summed once for both, the
+// insertion's parents being the contiguous range(s) above its slots.  A parent reached both ways
+// is computed twice with the same result.
 __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam& team, uint32_t B, uint32_t n2,
                                                 const int32_t* __restrict__ idx, const float* __restrict__ val, int raw,
-                                                float alpha, float eps, unsigned long long fill, unsigned char* smem)
+                                                float alpha, float eps, unsigned long long fill, unsigned char* smem,
+                                                uint32_t n = 0, const float* __restrict__ prio = nullptr,
+                                                uint64_t cursor = 0)
 {
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
@@ -165,19 +172,34 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         }
     }
 
-    // winners write the leaves
+    // winners write the leaves (unless the insertion overwrites the slot anyway), then the inserted leaves
+    const uint64_t N = v.capacity;
     float* leaves = v.level[v.depth];
     for (uint32_t s = rank; s < n2; s += nt) {
         const unsigned long long key = keys[s];
         if (key == kPrbInvalidKey) continue;
         const uint32_t i = (uint32_t)(key >> 32);
         const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
-        if (last) leaves[i] = vals[(uint32_t)key];
+        const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;     // distance from the cursor along the ring
+        if (last && !(ahead < n)) leaves[i] = vals[(uint32_t)key];
     }
+    bool bad = false;
+    for (uint32_t t = rank; t < n; t += nt) {
+        uint64_t slot = cursor + t;
+        if (slot >= N) slot -= N;
+        float p = prio[t];
+        if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+        leaves[slot] = p;
+    }
+    if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     team.sync();
 
-    // re-sum the ancestors, deepest level first
+    // re-sum the ancestors, deepest level first; the insertion dirties parent range A = [a0, a1] >> sh
+    // and, if the ring wrapped, B = [0, b1] >> sh
     const uint32_t K = v.fanout, lg = v.log2_fanout;
+    const uint64_t a0 = cursor, a1 = (n ? min(cursor + n, N) : cursor + 1) - 1;
+    const bool wrapped = cursor + n > N;
+    const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
     for (int l = (int)v.depth - 1; l >= 0; --l) {
         const uint32_t sh = lg * (v.depth - (uint32_t)l);
         const float* child = v.level[l + 1];
@@ -188,6 +210,15 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             const uint32_t a = (uint32_t)(key >> 32) >> sh;
             const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
             if (first) par[a] = prb_sum_children_dyn(child + (uint64_t)a * K, K);
+        }
+        if (n) {
+            const uint64_t pa0 = a0 >> sh, cntA = (a1 >> sh) - pa0 + 1;
+            uint64_t cntB = 0;
+            if (wrapped) cntB = (pa0 == 0) ? 0 : min(b1 >> sh, pa0 - 1) + 1;     // parents of B not already in A
+            for (uint64_t i = rank; i < cntA + cntB; i += nt) {
+                const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
+                par[j] = prb_sum_children_dyn(child + j * K, K);
+            }
         }
         team.sync();
     }
