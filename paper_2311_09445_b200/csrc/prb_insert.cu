@@ -111,6 +111,12 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
     const uint32_t tid = threadIdx.x;
     if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
+    // the tree CTA fetches its first inputs now, while the cursor is on its way
+    PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
+    if (blockIdx.x == 0 && tid < kWorkers) {
+        if (tid < upd.B) { pre.has_update = true; pre.idx = upd.idx[tid]; pre.val = upd.val[tid]; }
+        if (tid < n) { pre.has_prio = true; pre.prio = prio[tid]; }
+    }
     __syncthreads();
     const uint64_t cursor = s_cursor;
     if (tid == kWorkers) {
@@ -120,9 +126,9 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
             if (upd.B)      // update and insertion share one re-sum pass per level
-                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor);
+                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre);
             else
-                prb_insert_tree_team(v, team, n, prio, cursor);
+                prb_insert_tree_team(v, team, n, prio, cursor, pre);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;

@@ -9,6 +9,14 @@
 
 #ifdef __CUDACC__
 
+// Inputs of entry `rank` that a kernel may have fetched before the team's work starts (so that the
+// fetch overlaps an earlier wait); valid only where the matching flag is set.
+struct PrbPreloaded {
+    bool has_update, has_prio;
+    int32_t idx;
+    float val, prio;
+};
+
 struct PrbTeam {
     uint32_t rank, size;     // this thread's rank in the team, number of threads (multiple of 32)
     bool whole_cta;          // the team is the whole CTA: plain __syncthreads; otherwise named barrier 1
@@ -104,7 +112,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
                                                 const int32_t* __restrict__ idx, const float* __restrict__ val, int raw,
                                                 float alpha, float eps, unsigned long long fill, unsigned char* smem,
                                                 uint32_t n = 0, const float* __restrict__ prio = nullptr,
-                                                uint64_t cursor = 0)
+                                                uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f})
 {
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
@@ -116,11 +124,13 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     for (uint32_t b = rank; b < n2; b += nt) {
         unsigned long long key = kPrbInvalidKey;
         if (b < B) {
-            const int32_t i = idx[b];
+            const bool mine = pre.has_update && b == rank;
+            const int32_t i = mine ? pre.idx : idx[b];
+            const float x = mine ? pre.val : val[b];
             float p = 0.0f;
             bool ok_p;
-            if (raw) { p = val[b]; ok_p = prb_valid_priority(p); }
-            else ok_p = prb_priority_pow(val[b], eps, alpha, p);
+            if (raw) { p = x; ok_p = prb_valid_priority(p); }
+            else ok_p = prb_priority_pow(x, eps, alpha, p);
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
             else key = ((unsigned long long)(uint32_t)i << 32) | b;
@@ -187,7 +197,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     for (uint32_t t = rank; t < n; t += nt) {
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
-        float p = prio[t];
+        float p = (pre.has_prio && t == rank) ? pre.prio : prio[t];
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
         leaves[slot] = p;
     }
@@ -228,7 +238,8 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
 // (mod capacity), then re-sum the dirty parents level by level.  A contiguous slot range dirties
 // a contiguous parent range on every level (two ranges if the ring wrapped), so nothing is sorted.
 __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const PrbTeam& team, uint32_t n,
-                                                     const float* __restrict__ prio, uint64_t cursor)
+                                                     const float* __restrict__ prio, uint64_t cursor,
+                                                     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f})
 {
     const uint64_t N = v.capacity;
     const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
@@ -237,7 +248,7 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
     for (uint32_t t = team.rank; t < n; t += team.size) {
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
-        float p = prio[t];
+        float p = (pre.has_prio && t == team.rank) ? pre.prio : prio[t];
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
         leaves[slot] = p;
     }
