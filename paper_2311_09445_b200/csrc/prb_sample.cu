@@ -127,21 +127,20 @@ __device__ __forceinline__ void store_granule(unsigned char* base, uint64_t g, u
 }
 
 // Short rows of strata [k_first, k_first + n_rows): every short field of the batch, granule by
-// granule, by `nthreads` threads.  s_idx[r] is the leaf of stratum k_first + r.  The first U
+// granule, by `nthreads` threads.  s_idx[r] is the leaf of stratum k_first + r.  The first two
 // granules per thread of ALL fields are loaded before anything is stored, so a small batch costs
 // one round trip instead of one per field; what is left goes field by field.
-template <int U>
 __device__ __forceinline__ void gather_short_fields(const PrbView& v, const SamplePlan& plan, const PrbBatch& dst,
                                                     uint32_t k_first, uint32_t n_rows, const uint32_t* s_idx,
                                                     uint32_t rank, uint32_t nthreads)
 {
-    uint4 tmp[PRB_NUM_FIELDS][U];
+    uint4 tmp[PRB_NUM_FIELDS][2];
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
+        for (int u = 0; u < 2; ++u) {
             const uint32_t e = rank + u * nthreads;
             if (e < total) {
                 const uint32_t r = (W == 1) ? e : e / W;
@@ -155,29 +154,27 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
         const uint64_t dbase = (uint64_t)k_first * W;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
+        for (int u = 0; u < 2; ++u) {
             const uint32_t e = rank + u * nthreads;
             if (e < total) store_granule(dst.ptr[f], dbase + e, vec, tmp[f][u]);
         }
-        for (uint32_t e = rank + U * nthreads; e < total; e += nthreads) {     // the rest of a larger batch
+        for (uint32_t e = rank + 2 * nthreads; e < total; e += nthreads) {     // the rest of a larger batch
             const uint32_t r = e / W;
             store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec));
         }
     }
 }
 
-// T threads per CTA: 256 in general; 1024 for a short-row batch that one CTA can walk in one go
-// (B <= 1024 / K), which then needs neither scratch nor ticket: the weights are normalised in place.
-template <int K, int T>
-__global__ void __launch_bounds__(T, T == 1024 ? 1 : kCtasPerSm)
+template <int K>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uint64_t seed,
                   int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
                   const __grid_constant__ SamplePlan plan)
 {
-    constexpr uint32_t R = T / K;          // strata walked concurrently by one CTA
+    constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
     __shared__ float s_top[kTopFloats];
     __shared__ uint32_t s_idx[R];
-    __shared__ double s_wmax[T / 64];                // per-warp maxima of the weight threads
+    __shared__ double s_wraw[R];
     __shared__ float s_p[R];
     __shared__ unsigned s_flags[R];
     __shared__ unsigned int s_last;
@@ -196,13 +193,13 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     {
         // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
         const float4* src = reinterpret_cast<const float4*>(v.level[1]);
-        float4 t[(kTopFloats / 4 + T - 1) / T];
+        float4 t[kTopFloats / 4 / kThreads];
 #pragma unroll
-        for (uint32_t u = 0; u < (kTopFloats / 4 + T - 1) / T; ++u)
-            if (tid + u * T < plan.top_vec4) t[u] = __ldg(src + tid + u * T);
+        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+            if (tid + u * kThreads < plan.top_vec4) t[u] = __ldg(src + tid + u * kThreads);
 #pragma unroll
-        for (uint32_t u = 0; u < (kTopFloats / 4 + T - 1) / T; ++u)
-            if (tid + u * T < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * T] = t[u];
+        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+            if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
     }
     const bool empty = (fill == 0) || !(total32 > 0.0f);
 
@@ -250,60 +247,49 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 
         // From here the CTA splits by role: threads 0..127 copy, threads 128..255 look after the weights.
         const bool last_descents = round + 1 >= n_rounds;      // true exactly once per CTA
-        if (tid >= T / 2) {
+        if (tid >= kThreads / 2) {
             // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path)
-            const uint32_t gi2 = tid - T / 2;
-            const bool solo = gridDim.x == 1 && n_rounds <= 1;     // the whole batch is here: no scratch, no ticket
-            double wr = 0.0;
-            if (gi2 < n_round && kb + gi2 >= k_own) {
-                const uint32_t k2 = kb + gi2;
-                const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
-                wr = pow(scaled, -(double)beta);
-                out_idx[k2] = (int32_t)s_idx[gi2];
-                if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
-                if (!solo) { v.wraw[k2] = wr; __threadfence(); }
+            const uint32_t gi2 = tid - kThreads / 2;
+            if (gi2 < n_round) {
+                double wr = 0.0;
+                if (kb + gi2 >= k_own) {
+                    const uint32_t k2 = kb + gi2;
+                    const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
+                    wr = pow(scaled, -(double)beta);
+                    out_idx[k2] = (int32_t)s_idx[gi2];
+                    v.wraw[k2] = wr;
+                    if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
+                    __threadfence();
+                }
+                s_wraw[gi2] = wr;
             }
-            // maximum over the weight threads
-            double m = wr;
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) m = fmax(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-            if ((tid & 31u) == 0) s_wmax[gi2 >> 5] = m;
-            asm volatile("bar.sync 2, %0;" ::"n"(T / 2) : "memory");
-            m = s_wmax[0];
-#pragma unroll
-            for (int q = 1; q < T / 64; ++q) m = fmax(m, s_wmax[q]);
-            if (solo) {
-                if (!empty && out_w != nullptr && gi2 < n_round) out_w[kb + gi2] = (float)__ddiv_rn(wr, m);
-                if (tid == T / 2) {
-                    if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-                    else v.state->sample_calls = calls + 1;
-                }
-            } else {
-                if (tid == T / 2) {
-                    if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
-                    if (last_descents) {
-                        // every descent of this CTA is done: the last CTA to get here normalises the weights
-                        __threadfence();
-                        s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
-                    }
-                }
+            asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+            if (tid == kThreads / 2) {
+                double m = 0.0;
+                for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
+                if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
                 if (last_descents) {
-                    asm volatile("bar.sync 2, %0;" ::"n"(T / 2) : "memory");
-                    if (s_last) {
-                        __threadfence();
-                        if (empty) {
-                            if (tid == T / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-                        } else if (out_w != nullptr) {
-                            const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
-                            for (uint32_t k = tid - T / 2; k < B; k += T / 2)
-                                out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
-                        }
-                        asm volatile("bar.sync 2, %0;" ::"n"(T / 2) : "memory");
-                        if (tid == T / 2) {
-                            if (!empty) v.state->sample_calls = calls + 1;
-                            v.state->wmax_bits = 0ull;
-                            v.state->sample_ticket = 0u;
-                        }
+                    // every descent of this CTA is done: the last CTA to get here normalises the weights
+                    __threadfence();
+                    s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+                }
+            }
+            if (last_descents) {
+                asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+                if (s_last) {
+                    __threadfence();
+                    if (empty) {
+                        if (tid == kThreads / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+                    } else if (out_w != nullptr) {
+                        const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
+                        for (uint32_t k = tid - kThreads / 2; k < B; k += kThreads / 2)
+                            out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
+                    }
+                    asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+                    if (tid == kThreads / 2) {
+                        if (!empty) v.state->sample_calls = calls + 1;
+                        v.state->wmax_bits = 0ull;
+                        v.state->sample_ticket = 0u;
                     }
                 }
             }
@@ -326,8 +312,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             // short rows: copied by the stratum's owner through registers (warp 0 drives the ring when there is one)
             const uint32_t k_flat = max(kb, k_own);
             if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
-                const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? T / 2 - 32u : T / 2;
-                gather_short_fields<(T == 1024 ? 1 : 2)>(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
+                const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads / 2 - 32u : kThreads / 2;
+                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
             }
         }
         __syncthreads();        // s_idx is rewritten by the next round
@@ -380,9 +366,8 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         plan.top_vec4 = (uint32_t)((off + v.level_alloc[l] + 3) / 4);
         plan.top_levels = l;
     }
-    uint32_t R = kThreads / v.fanout;
+    const uint32_t R = kThreads / v.fanout;
     uint32_t grid, smem = 0;
-    bool one_cta = false;
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
     if (row_mode) {
@@ -395,10 +380,6 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         if (plan.ring_stages > 32) plan.ring_stages = 32;
         smem = kRingBarBytes + plan.ring_stages * stage;
         grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
-    } else if (B <= 1024u / v.fanout) {
-        one_cta = true;              // one 1024-thread CTA walks the whole batch at once
-        R = 1024u / v.fanout;
-        grid = 1;
     } else {
         const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
         const uint32_t want = (B + R - 1) / R;
@@ -410,14 +391,12 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
 #define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
     do {                                                                                                          \
         if (smem && !big_smem[ki]) {                                                                              \
-            attr = cudaFuncSetAttribute(prb_sample_kernel<KK, kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+            attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                         (int)(kRingBarBytes + kRingBytes));                                       \
             big_smem[ki] = (attr == cudaSuccess);                                                                 \
         }                                                                                                         \
-        if (attr == cudaSuccess && one_cta)                                                                       \
-            prb_sample_kernel<KK, 1024><<<1, 1024, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);              \
-        else if (attr == cudaSuccess)                                                                             \
-            prb_sample_kernel<KK, kThreads><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); \
+        if (attr == cudaSuccess)                                                                                  \
+            prb_sample_kernel<KK><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);          \
     } while (0)
     switch (v.fanout) {
     case 2: PRB_LAUNCH_SAMPLE(2); break;
