@@ -59,7 +59,7 @@ def load_library(path: Optional[str] = None):
     """Loads libpearl_prb.so (built in-tree by build.py) and declares its signatures."""
     global _lib
     if _lib is None:
-        path = path or _build.LIB
+        path = path or os.environ.get("PEARL_PRB_LIB") or _build.LIB      # PEARL_PRB_LIB: an alternate build of the library
         if not os.path.exists(path):
             raise ImportError("libpearl_prb.so is not built (%s); run paper_2311_09445_b200/build.py" % path)
         lib = C.CDLL(path)

@@ -259,7 +259,6 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     out_idx[k2] = (int32_t)s_idx[gi2];
                     v.wraw[k2] = wr;
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
-                    __threadfence();
                 }
                 s_wraw[gi2] = wr;
             }
@@ -270,6 +269,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                 if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
                 if (last_descents) {
                     // every descent of this CTA is done: the last CTA to get here normalises the weights
+                    // (the barrier above ordered the other threads' writes before this fence: it covers them)
                     __threadfence();
                     s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
                 }
@@ -381,8 +381,11 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         smem = kRingBarBytes + plan.ring_stages * stage;
         grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
     } else {
+        // a small batch is spread over more CTAs than it needs: its descents are chains of dependent
+        // L2 reads, and more SMs keep more of them in flight
         const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
-        const uint32_t want = (B + R - 1) / R;
+        const uint32_t per_cta = R >= 4 ? R / 4 : 1;
+        const uint32_t want = (B + per_cta - 1) / per_cta;
         grid = want < one_wave ? want : one_wave;
     }
     static bool big_smem[6] = { false, false, false, false, false, false };
