@@ -78,7 +78,8 @@ __device__ __forceinline__ void copy_tile(const PrbView& v, const InsertPlan& pl
 // happens while the copies are still running.
 __device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill)
 {
-    __threadfence();
+    // no fence: the cursor and fill reads that must precede this ticket have returned their values
+    // (they were stored to shared memory before the barrier this thread has passed)
     const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
     if (done == gridDim.x - 1) {
         const uint64_t N = v.capacity;
