@@ -20,11 +20,24 @@ struct PrbPreloaded {
 struct PrbTeam {
     uint32_t rank, size;     // this thread's rank in the team, number of threads (multiple of 32)
     bool whole_cta;          // the team is the whole CTA: plain __syncthreads; otherwise named barrier 1
+    // Several CTAs of one thread-block cluster may share the tree work: each holds the full sorted
+    // key list, CTA `part` of `parts` takes the slots whose warp-sized group number is congruent to
+    // it, and the phases are separated by the cluster's hardware barrier.  parts == 1: one CTA.
+    uint32_t part = 0, parts = 1;
 
     __device__ __forceinline__ void sync() const
     {
         if (whole_cta) __syncthreads();
         else asm volatile("bar.sync 1, %0;" ::"r"(size) : "memory");
+    }
+    __device__ __forceinline__ bool takes(uint32_t slot) const { return parts == 1 || ((slot >> 5) % parts) == part; }
+    // Between the phases of the tree work (leaves, then level by level): what the team -- or every
+    // CTA of the cluster -- wrote to global memory before is visible to all of it after.
+    __device__ __forceinline__ void phase_sync() const
+    {
+        if (parts == 1) { sync(); return; }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
     // barrier + OR-reduction of a predicate over the team
     __device__ __forceinline__ bool sync_or(bool pred) const
@@ -139,7 +152,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         keys[b] = key;
         my_key = key;
     }
-    if (flags) atomicOr(&v.state->status, flags);
+    if (flags && team.part == 0) atomicOr(&v.state->status, flags);
     team.sync();
 
     // Indices that come straight from a stratified sample are already in order; sort only if needed.
@@ -187,7 +200,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     float* leaves = v.level[v.depth];
     for (uint32_t s = rank; s < n2; s += nt) {
         const unsigned long long key = keys[s];
-        if (key == kPrbInvalidKey) continue;
+        if (key == kPrbInvalidKey || !team.takes(s)) continue;
         const uint32_t i = (uint32_t)(key >> 32);
         const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
         const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;     // distance from the cursor along the ring
@@ -195,6 +208,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     }
     bool bad = false;
     for (uint32_t t = rank; t < n; t += nt) {
+        if (!team.takes(t)) continue;
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
         float p = (pre.has_prio && t == rank) ? pre.prio : prio[t];
@@ -202,7 +216,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    team.sync();
+    team.phase_sync();
 
     // re-sum the ancestors, deepest level first; the insertion dirties parent range A = [a0, a1] >> sh
     // and, if the ring wrapped, B = [0, b1] >> sh
@@ -216,7 +230,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         float* par = v.level[l];
         for (uint32_t s = rank; s < n2; s += nt) {
             const unsigned long long key = keys[s];
-            if (key == kPrbInvalidKey) continue;
+            if (key == kPrbInvalidKey || !team.takes(s)) continue;
             const uint32_t a = (uint32_t)(key >> 32) >> sh;
             const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
             if (first) par[a] = prb_sum_children_dyn(child + (uint64_t)a * K, K);
@@ -226,11 +240,12 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             uint64_t cntB = 0;
             if (wrapped) cntB = (pa0 == 0) ? 0 : min(b1 >> sh, pa0 - 1) + 1;     // parents of B not already in A
             for (uint64_t i = rank; i < cntA + cntB; i += nt) {
+                if (!team.takes((uint32_t)i)) continue;
                 const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
                 par[j] = prb_sum_children_dyn(child + j * K, K);
             }
         }
-        team.sync();
+        team.phase_sync();
     }
 }
 

@@ -3,8 +3,8 @@
 // mutex; here the leaf is SET and the ancestors are re-summed, so the result does not depend
 // on scheduling (see prb_update_team in prb_tree.cuh for the steps).
 //
-// One CTA: the batch is at most a few thousand entries and the work is a chain of dependent
-// L2 round trips.
+// One CTA, or eight CTAs of one thread-block cluster that share every level: the batch is at most
+// a few thousand entries and the work is a chain of dependent L2 round trips, one per level.
 #include "prb_tree.cuh"
 
 namespace {
@@ -18,6 +18,8 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     team.rank = threadIdx.x;
     team.size = blockDim.x;
     team.whole_cta = true;
+    team.part = blockIdx.x;          // CTAs of one cluster share the work (one CTA: the whole of it)
+    team.parts = gridDim.x;
     prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, v.state->fill, smem);
 }
 
@@ -34,8 +36,23 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         uint32_t n2 = 2;
         while (n2 < b) n2 <<= 1;
         const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
-        prb_update_kernel<<<1, threads, prb_update_smem_bytes(n2), s>>>(v, b, n2, d_idx + first, d_val + first, raw, alpha, eps);
-        if (cudaGetLastError() != cudaSuccess) return -1;
+        // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
+        // one SM keeps in flight: then eight CTAs of one cluster share each level.
+        const uint32_t ctas = (v.fanout * b >= 8192u) ? 8u : 1u;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(ctas);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = ctas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps) != cudaSuccess)
+            return -1;
         ++launches;
     }
     return launches;
