@@ -243,6 +243,43 @@ def test_largest_sweep_capacity(oracle_mod, K):
     pr.close()
 
 
+def test_degenerate_sampling_cases(oracle_mod):
+    rng = np.random.default_rng(17)
+    pr = Pair(oracle_mod, 300, 16, 68, 24, 128)
+    b = raw_fields(rng, 100, 68, 24)
+    b["prio"] = np.zeros(100, np.float32)
+    pr.insert(b)                                         # stored, but the total is zero
+    o, g = pr.sample(16, 0.4, 3)
+    assert g["idx"].tolist() == [-1] * 16 and pr.compare_status() == 4
+    pr.compare_state()
+    pr.update_priorities(np.array([7], np.int32), np.array([2.5], np.float32))   # a single positive leaf
+    for beta in (0.0, 1.0, 0.4):
+        o, g = pr.sample(33, beta, 3)
+        assert np.all(g["idx"] == 7) and np.all(g["w"] == 1.0)
+    pr.update_priorities(np.arange(100, dtype=np.int32), rng.uniform(0.1, 1, 100).astype(np.float32))
+    for beta in (0.0, 1.0):
+        o, g = pr.sample(128, beta, 5)
+        if beta == 0.0:
+            assert np.all(g["w"] == 1.0)
+    o, g = pr.sample(1, 0.4, 5)                          # B = 1
+    assert g["w"][0] == 1.0
+    # outputs are optional: indices only, then indices + weights + one field
+    dev = pr.dev
+    idx = torch.full((64,), -1, dtype=torch.int32, device=dev)
+    o = pr.ora.sample(64, 0.4, 5)
+    pr.gpu.sample(64, 0.4, 5, idx)
+    assert np.array_equal(idx.cpu().numpy(), o["idx"])
+    w = torch.zeros(64, device=dev)
+    rew = torch.zeros(64, device=dev)
+    o = pr.ora.sample(64, 0.4, 5)
+    pr.gpu.sample(64, 0.4, 5, idx, w, rew=rew)
+    assert np.array_equal(idx.cpu().numpy(), o["idx"]) and np.array_equal(rew.cpu().numpy(), o["rew"])
+    np.testing.assert_allclose(w.cpu().numpy(), o["w"], rtol=1e-5)
+    pr.compare_state()
+    assert pr.compare_status() == 0
+    pr.close()
+
+
 def test_priority_transform_bits(oracle_mod):
     # The power is compared through the leaves it writes: 4096 TD errors x several exponents.
     rng = np.random.default_rng(21)
