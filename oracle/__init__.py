@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "prb_oracle.c")
 _LIB = os.path.join(_HERE, "libprb_oracle.so")
 
-ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL = 1, 2, 4, 8, 16
+ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL, ST_STALE = 1, 2, 4, 8, 16, 32
 
 
 def build(force: bool = False) -> str:
@@ -47,6 +47,8 @@ def lib():
         L.oracle_prb_insert.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp]
         L.oracle_prb_update_priorities.argtypes = [vp, u32, vp, vp]
         L.oracle_prb_update.argtypes = [vp, u32, vp, vp, f32, f32]
+        L.oracle_prb_update_after_insert.argtypes = [vp, u32, vp, vp, f32, f32, u32]
+        L.oracle_prb_get_priorities.argtypes = [vp, u32, vp, vp]
         L.oracle_prb_descend.argtypes = [vp, C.c_double, C.POINTER(f32)]
         L.oracle_prb_descend.restype = C.c_int64
         L.oracle_prb_targets.argtypes = [vp, u32, u64, u64, vp]
@@ -137,6 +139,17 @@ class OraclePRB:
     def update(self, idx, td, alpha: float, eps: float) -> int:
         idx, td = _host(idx, np.int32), _host(td, np.float32)
         return lib().oracle_prb_update(self._h, idx.shape[0], _ptr(idx), _ptr(td), alpha, eps)
+
+    def update_after_insert(self, idx, td, alpha: float, eps: float, inserted: int) -> int:
+        idx, td = _host(idx, np.int32), _host(td, np.float32)
+        return lib().oracle_prb_update_after_insert(self._h, idx.shape[0], _ptr(idx), _ptr(td), alpha, eps, inserted)
+
+    def get_priorities(self, idx) -> np.ndarray:
+        idx = _host(idx, np.int32)
+        out = np.zeros(idx.shape[0], dtype=np.float32)
+        rc = lib().oracle_prb_get_priorities(self._h, idx.shape[0], _ptr(idx), _ptr(out))
+        assert rc == 0
+        return out
 
     def update_priorities(self, idx, prio) -> int:
         idx, prio = _host(idx, np.int32), _host(prio, np.float32)

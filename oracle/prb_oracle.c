@@ -54,6 +54,7 @@
 #define ST_EMPTY 4u
 #define ST_CLAMPED 8u
 #define ST_INTERNAL 16u
+#define ST_STALE 32u
 
 #define MAX_LEVELS 64
 
@@ -352,6 +353,47 @@ int oracle_prb_update(oracle_prb_t *o, uint32_t B, const int32_t *idx, const flo
         mark_dirty(o, D, (uint64_t)idx[b]);
     }
     resum_dirty(o);
+    return ORACLE_OK;
+}
+
+/* Update that arrives after an insertion (Section IV-C, "Replay-Collision-Free Scheduling": the  */
+/* insertion index is compared against the sampled indices so that the Learner's update does not */
+/* contaminate a transition the Actors have written in the meantime).  `inserted` transitions    */
+/* were written since the batch was sampled: they occupy the ring slots cursor-inserted ..       */
+/* cursor-1 (mod capacity).  An entry that names one of them is stale: skipped, STALE raised.    */
+int oracle_prb_update_after_insert(oracle_prb_t *o, uint32_t B, const int32_t *idx, const float *td,
+                                   float alpha, float eps, uint32_t inserted)
+{
+    if (!o || !idx || !td) return ORACLE_ERR_NULL;
+    if (B == 0) return ORACLE_ERR_BAD_BATCH;
+    if (!isfinite(alpha) || alpha < 0.0f || !isfinite(eps) || eps < 0.0f) return ORACLE_ERR_BAD_ARG;
+    if (inserted > o->capacity) return ORACLE_ERR_BAD_ARG;
+    uint32_t D = o->depth;
+    for (uint32_t b = 0; b < B; ++b) {
+        if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
+        /* how many slots back from the most recently written one this index lies */
+        uint64_t i = (uint64_t)idx[b];
+        uint64_t back = (o->cursor + o->capacity - 1 - i) % o->capacity;
+        if (back < inserted) { o->status |= ST_STALE; continue; }
+        float p;
+        if (oracle_priority_pow(td[b], eps, alpha, &p)) { o->status |= ST_BAD_PRIORITY; continue; }
+        o->level[D][idx[b]] = p;
+        mark_dirty(o, D, i);
+    }
+    resum_dirty(o);
+    return ORACLE_OK;
+}
+
+/* Priority retrieval (Section V-A): the priorities stored at the given indices.  An index outside */
+/* [0, size) yields 0 and raises BAD_INDEX.                                                       */
+int oracle_prb_get_priorities(oracle_prb_t *o, uint32_t B, const int32_t *idx, float *out)
+{
+    if (!o || !idx || !out) return ORACLE_ERR_NULL;
+    if (B == 0) return ORACLE_ERR_BAD_BATCH;
+    for (uint32_t b = 0; b < B; ++b) {
+        if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; out[b] = 0.0f; continue; }
+        out[b] = o->level[o->depth][idx[b]];
+    }
     return ORACLE_OK;
 }
 

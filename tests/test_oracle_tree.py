@@ -224,3 +224,41 @@ def test_planted_mistake_is_caught(oracle_mod):
     assert o.descend(9.0 + 13.5)[0] != flat_scan(P8, 9.0 + 13.5)
     o.rebuild()
     check_invariant(o)
+
+
+def test_update_after_insert_equals_update_then_insert(oracle_mod):
+    # Collision-free scheduling (Section IV-C): sample, insert, then an update that skips the slots
+    # written since the sample must leave the same tree as update-then-insert on the same inputs.
+    rng = np.random.default_rng(31)
+    N, n, B = 200, 37, 64
+    for K in (2, 16):
+        a = oracle_mod.OraclePRB(N, K, 0, 0)
+        b = oracle_mod.OraclePRB(N, K, 0, 0)
+        first = rng.uniform(0.1, 1, 150).astype(np.float32)
+        for o in (a, b):
+            o.insert(None, None, None, None, None, first)
+        saw_stale = False
+        for step in range(30):
+            idx = a.sample(B, 0.4, 7, gather=False)["idx"]
+            assert np.array_equal(idx, b.sample(B, 0.4, 7, gather=False)["idx"])
+            td = rng.standard_normal(B).astype(np.float32)
+            newp = rng.uniform(0.1, 1, n).astype(np.float32)
+            a.insert(None, None, None, None, None, newp)
+            assert a.update_after_insert(idx, td, 0.6, 1e-6, n) == 0
+            assert b.update(idx, td, 0.6, 1e-6) == 0
+            b.insert(None, None, None, None, None, newp)
+            sa, sb = a.status(), b.status()
+            saw_stale |= bool(sa & oracle_mod.ST_STALE)
+            assert (sa & ~oracle_mod.ST_STALE) == sb
+            for l in range(a.depth + 1):
+                assert np.array_equal(a.read_level(l).view(np.uint32), b.read_level(l).view(np.uint32))
+            check_invariant(a)
+        assert saw_stale                       # the ring wrapped over sampled slots at least once
+    # inserted = 0 is the plain update; a stale index is exactly one of the last `inserted` slots
+    o = make(oracle_mod, P8, 2)
+    o.insert(None, None, None, None, None, np.array([7, 7, 7], np.float32))       # slots 0 1 2, cursor 3
+    assert o.update_after_insert([2, 3, 0, 7], [1.0, 1.0, 1.0, 1.0], 1.0, 0.0, 2) == 0
+    assert o.status() == oracle_mod.ST_STALE
+    assert o.read_level(3).tolist() == [1, 7, 7, 1, 5, 9, 2, 1]                      # 1 and 2 were skipped
+    assert o.get_priorities([0, 2, 7, 8, -1]).tolist() == [1, 7, 1, 0, 0]
+    assert o.status() == oracle_mod.ST_BAD_INDEX
