@@ -55,6 +55,7 @@ typedef struct pearl_layout {
 #define PEARL_ST_EMPTY 4u          /* sample on an empty buffer or a non-positive total; outputs untouched */
 #define PEARL_ST_CLAMPED 8u        /* a descent met residual >= last prefix sum and took the last positive child */
 #define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out */
+#define PEARL_ST_STALE 32u         /* update_after_insert: the index was overwritten since it was sampled; entry skipped */
 
 /* Update batches larger than this are applied as consecutive sub-batches of this many entries, in
  * batch order, one launch each; the result is that of the whole batch (the last valid entry of a
@@ -123,6 +124,20 @@ int pearl_prb_update(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const f
 /* As pearl_prb_update, with the priorities given directly (no power). */
 int pearl_prb_update_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx,
                                 const float* d_prio);
+
+/* Priority update that arrives after an insertion (Section IV-C, "Replay-Collision-Free
+ * Scheduling": the insertion index is compared against the sampled indices, so that the Learner's
+ * update does not contaminate a transition the Actors wrote in the meantime).  `inserted`
+ * transitions have been inserted since d_idx was sampled; they occupy the ring slots
+ * cursor-inserted .. cursor-1 (mod capacity).  An entry naming one of them is skipped and raises
+ * PEARL_ST_STALE; everything else is pearl_prb_update.  The sequence sample, insert,
+ * update_after_insert leaves the same tree as sample, update, insert.  inserted <= capacity. */
+int pearl_prb_update_after_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_td,
+                                  float alpha, float eps, uint32_t inserted);
+
+/* Priority retrieval (Section V-A): d_out[b] = the priority stored at d_idx[b], for b < B.  An
+ * index outside [0, fill) yields 0 and raises PEARL_ST_BAD_INDEX.  1 <= B <= max_batch. */
+int pearl_prb_get_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, float* d_out);
 
 /* Priority update followed by insertion, in one launch.  The result is exactly that of
  * pearl_prb_update(prb, B, d_idx, d_td, alpha, eps) followed by pearl_prb_insert(prb, n, ...): the

@@ -15,7 +15,7 @@ import torch
 
 from . import build as _build
 
-ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL = 1, 2, 4, 8, 16
+ST_BAD_INDEX, ST_BAD_PRIORITY, ST_EMPTY, ST_CLAMPED, ST_INTERNAL, ST_STALE = 1, 2, 4, 8, 16, 32
 
 
 class PearlError(RuntimeError):
@@ -41,6 +41,8 @@ SIGNATURES = {
     "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
+    "pearl_prb_update_after_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32]),
+    "pearl_prb_get_priorities": (_i, [_vp, _u32, _vp, _vp]),
     "pearl_prb_update_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_host": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -168,6 +170,17 @@ class PrioritizedReplay:
         rc = load_library().pearl_prb_update_priorities(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(prio, "prio"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_update_priorities")
+
+    def update_after_insert(self, idx, td, alpha: float, eps: float, inserted: int) -> None:
+        rc = load_library().pearl_prb_update_after_insert(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"),
+                                                          alpha, eps, inserted)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update_after_insert")
+
+    def get_priorities(self, idx, out) -> None:
+        rc = load_library().pearl_prb_get_priorities(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(out, "out"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_get_priorities")
 
     def update_insert(self, idx, td, alpha: float, eps: float, obs, act, rew, next_obs, done, prio) -> None:
         rc = load_library().pearl_prb_update_insert(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"), alpha, eps,

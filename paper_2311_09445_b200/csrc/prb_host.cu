@@ -238,7 +238,7 @@ int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int3
 }
 
 static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_val, int raw, float alpha,
-                         float eps)
+                         float eps, uint32_t stale = 0)
 {
     if (!h || !d_idx || !d_val) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
@@ -246,7 +246,8 @@ static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const
     if (misaligned(d_idx, 4) || misaligned(d_val, 4)) return PEARL_ERR_ALIGN;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
-    const int k = prb_launch_update(h->view, B, d_idx, d_val, raw, alpha, eps, h->stream);
+    if (stale > h->view.capacity) return PEARL_ERR_BAD_ARG;
+    const int k = prb_launch_update(h->view, B, d_idx, d_val, raw, alpha, eps, h->stream, stale);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
     return PEARL_OK;
@@ -260,6 +261,25 @@ int pearl_prb_update(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const flo
 int pearl_prb_update_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_prio)
 {
     return update_common(h, B, d_idx, d_prio, 1, 0.0f, 0.0f);
+}
+
+int pearl_prb_update_after_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_td, float alpha,
+                                  float eps, uint32_t inserted)
+{
+    return update_common(h, B, d_idx, d_td, 0, alpha, eps, inserted);
+}
+
+int pearl_prb_get_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, float* d_out)
+{
+    if (!h || !d_idx || !d_out) return PEARL_ERR_NULL;
+    if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (misaligned(d_idx, 4) || misaligned(d_out, 4)) return PEARL_ERR_ALIGN;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    const int k = prb_launch_get_priorities(h->view, B, d_idx, d_out, h->stream);
+    if (k < 0) return PEARL_ERR_CUDA;
+    h->launches += (uint64_t)k;
+    return PEARL_OK;
 }
 
 int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_td, float alpha, float eps,

@@ -49,8 +49,10 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
                       int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f);
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s);
+// (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
-                      float alpha, float eps, cudaStream_t s);
+                      float alpha, float eps, cudaStream_t s, uint32_t stale = 0);
+int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s);
 
 // ---- device helpers -------------------------------------------------------------------
 #ifdef __CUDACC__

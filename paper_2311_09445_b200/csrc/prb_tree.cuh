@@ -116,6 +116,8 @@ __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
 // left-to-right order.  Sorted order survives dropping low digits of the index, so no list is
 // compacted and no lock is taken.  n2 = B rounded up to a power of two (>= 2); smem holds
 // prb_update_smem_bytes(n2) bytes; fill = the fill count before this launch (indices must be below it).
+// With stale > 0 (and n == 0) entries that name one of the `stale` ring slots before `cursor` are
+// skipped: they were overwritten after they had been sampled.
 // With n > 0 the tree part of an insertion of n transitions at `cursor` follows in the same
 // passes: the inserted leaves are written after the update's (an updated leaf that is also
 // inserted keeps the inserted priority), and every level is re-summed once for both, the
@@ -125,7 +127,8 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
                                                 const int32_t* __restrict__ idx, const float* __restrict__ val, int raw,
                                                 float alpha, float eps, unsigned long long fill, unsigned char* smem,
                                                 uint32_t n = 0, const float* __restrict__ prio = nullptr,
-                                                uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f})
+                                                uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
+                                                uint32_t stale = 0)
 {
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
@@ -144,7 +147,10 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             bool ok_p;
             if (raw) { p = x; ok_p = prb_valid_priority(p); }
             else ok_p = prb_priority_pow(x, eps, alpha, p);
+            // stale: one of the `stale` slots written most recently, i.e. overwritten since it was sampled
+            const uint64_t back = (i >= 0 && stale) ? (cursor + v.capacity - 1 - (uint64_t)i) % v.capacity : ~0ull;
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
+            else if (back < stale) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
             else key = ((unsigned long long)(uint32_t)i << 32) | b;
             vals[b] = p;

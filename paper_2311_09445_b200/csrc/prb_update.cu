@@ -11,7 +11,7 @@ namespace {
 
 __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
-                  const float* __restrict__ val, int raw, float alpha, float eps)
+                  const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     PrbTeam team;
@@ -20,13 +20,33 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     team.whole_cta = true;
     team.part = blockIdx.x;          // CTAs of one cluster share the work (one CTA: the whole of it)
     team.parts = gridDim.x;
-    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, v.state->fill, smem);
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, v.state->fill, smem, 0, nullptr,
+                    stale ? v.state->cursor : 0ull, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale);
+}
+
+
+
+// Priority retrieval: one thread per entry.
+__global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
+                                          float* __restrict__ out)
+{
+    const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int32_t i = idx[b];
+    if (i < 0 || (unsigned long long)i >= v.state->fill) { out[b] = 0.0f; atomicOr(&v.state->status, PEARL_ST_BAD_INDEX); return; }
+    out[b] = __ldcg(v.level[v.depth] + i);
 }
 
 }  // namespace
 
+int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s)
+{
+    prb_get_priorities_kernel<<<(B + 255) / 256, 256, 0, s>>>(v, B, d_idx, d_out);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
-                      float alpha, float eps, cudaStream_t s)
+                      float alpha, float eps, cudaStream_t s, uint32_t stale)
 {
     // A batch beyond one CTA's reach goes sub-batch by sub-batch in batch order: every launch leaves
     // a consistent tree and later entries overwrite earlier ones, as in the whole batch.
@@ -51,7 +71,7 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps) != cudaSuccess)
+        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale) != cudaSuccess)
             return -1;
         ++launches;
     }

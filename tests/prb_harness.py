@@ -98,6 +98,18 @@ class Pair:
                                torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps,
                                d.get("obs"), d.get("act"), d.get("rew"), d.get("next_obs"), d.get("done"), d["prio"])
 
+    def update_after_insert(self, idx, td, alpha, eps, inserted):
+        assert self.ora.update_after_insert(idx, td, alpha, eps, inserted) == 0
+        self.gpu.update_after_insert(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                                     torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps,
+                                     inserted)
+
+    def compare_priorities(self, idx):
+        idx = np.ascontiguousarray(idx, np.int32)
+        out = torch.full((idx.shape[0],), -1.0, dtype=torch.float32, device=self.dev)
+        self.gpu.get_priorities(torch.from_numpy(idx).to(self.dev), out)
+        assert np.array_equal(out.cpu().numpy().view(np.uint32), self.ora.get_priorities(idx).view(np.uint32))
+
     def update_priorities(self, idx, prio):
         assert self.ora.update_priorities(idx, prio) == 0
         self.gpu.update_priorities(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),

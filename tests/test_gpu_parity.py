@@ -381,6 +381,32 @@ def test_update_beyond_one_subbatch(oracle_mod, K, B):
     pr.close()
 
 
+@pytest.mark.parametrize("K,N,B,n", [(2, 300, 64, 50), (16, 5000, 256, 700), (32, 900, 512, 512)])
+def test_update_after_insert_and_retrieval(oracle_mod, K, N, B, n):
+    # collision-free scheduling: sample, insert, then the update skips what the insertion overwrote
+    rng = np.random.default_rng(K * N)
+    pr = Pair(oracle_mod, N, K, 8, 4, 1024)
+    b = raw_fields(rng, N - 10, 8, 4)
+    b["prio"] = rng.uniform(0.1, 1, N - 10).astype(np.float32)
+    for first in range(0, N - 10, 1024):
+        pr.insert({k: v[first:first + 1024] for k, v in b.items()})
+    stale_seen = 0
+    for step in range(12):
+        o, g = pr.sample(B, 0.4, 11)
+        nb = raw_fields(rng, n, 8, 4)
+        nb["prio"] = rng.uniform(0.1, 1, n).astype(np.float32)
+        pr.insert(nb)
+        td = rng.standard_normal(B).astype(np.float32)
+        pr.update_after_insert(o["idx"], td, 0.6, 1e-6, n)
+        pr.compare_tree()
+        stale_seen |= pr.compare_status()
+        pr.compare_priorities(np.concatenate([o["idx"], [-1, N, N - 1, 0]]).astype(np.int32))
+        pr.compare_status()
+    assert stale_seen & 32
+    pr.compare_state()
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)
