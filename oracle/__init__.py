@@ -62,6 +62,8 @@ def lib():
         L.oracle_prb_read_level.argtypes = [vp, u32, vp, u64]
         L.oracle_prb_poke_level.argtypes = [vp, u32, u64, vp, u64]
         L.oracle_prb_read_rows.argtypes = [vp, vp, u32, vp, vp, vp, vp, vp]
+        L.oracle_prb_max_priority.argtypes = [vp]
+        L.oracle_prb_max_priority.restype = f32
         L.oracle_prb_status.argtypes = [vp]
         L.oracle_prb_status.restype = u32
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
@@ -128,9 +130,10 @@ class OraclePRB:
             pass
 
     # -- mutation -----------------------------------------------------------
-    def insert(self, obs, act, rew, next_obs, done, prio) -> int:
+    def insert(self, obs, act, rew, next_obs, done, prio, n=None) -> int:
+        """prio=None (with n given): every new transition gets the largest priority written so far."""
         prio = _host(prio, np.float32)
-        n = prio.shape[0]
+        n = prio.shape[0] if prio is not None else int(n)
         obs, act, next_obs = _host(obs), _host(act), _host(next_obs)
         rew, done = _host(rew, np.float32), _host(done, np.uint8)
         return lib().oracle_prb_insert(self._h, n, _ptr(obs), _ptr(act), _ptr(rew), _ptr(next_obs),
@@ -154,6 +157,9 @@ class OraclePRB:
     def update_priorities(self, idx, prio) -> int:
         idx, prio = _host(idx, np.int32), _host(prio, np.float32)
         return lib().oracle_prb_update_priorities(self._h, idx.shape[0], _ptr(idx), _ptr(prio))
+
+    def max_priority(self) -> np.float32:
+        return np.float32(lib().oracle_prb_max_priority(self._h))
 
     def rebuild(self):
         lib().oracle_prb_rebuild(self._h)

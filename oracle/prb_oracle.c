@@ -75,6 +75,7 @@ typedef struct oracle_prb {
     float *rew;
     uint64_t size, cursor, sample_calls;
     uint32_t status;
+    float max_priority;     /* largest priority written so far; 0 = none yet */
 } oracle_prb_t;
 
 /* ------------------------------------------------------------------------ */
@@ -282,22 +283,31 @@ static void resum_dirty(oracle_prb_t *o)
 
 static int valid_priority(float p) { return isfinite(p) && p >= 0.0f; }
 
+/* Running maximum of the priorities written (Schaul et al.: a new transition enters with the     */
+/* maximal priority seen so far, so that it is replayed at least once).                           */
+static void note_priority(oracle_prb_t *o, float p) { if (p > o->max_priority) o->max_priority = p; }
+static float default_priority(const oracle_prb_t *o) { return o->max_priority > 0.0f ? o->max_priority : 1.0f; }
+float oracle_prb_max_priority(const oracle_prb_t *o) { return o ? o->max_priority : 0.0f; }
+
 /* ------------------------------------------------------------------------ */
 /* Insert (Section V-A: insertion = retrieval + update; Listing 2: the new   */
 /* experiences are added to the Data Storage and insertion requests sent).   */
 /* Ring write at cursor .. cursor+n-1 (mod N).  The caller supplies the      */
-/* priority of each new transition (the paper is silent on its value).  An   */
-/* invalid priority (NaN, Inf, negative) stores the transition with leaf 0   */
-/* and raises BAD_PRIORITY.                                                  */
+/* priority of each new transition (the paper is silent on its value), or    */
+/* passes prio = NULL: then every new transition gets the largest priority   */
+/* written so far (1 if none), as in Schaul et al.  An invalid priority      */
+/* (NaN, Inf, negative) stores the transition with leaf 0 and raises         */
+/* BAD_PRIORITY.                                                             */
 /* ------------------------------------------------------------------------ */
 int oracle_prb_insert(oracle_prb_t *o, uint32_t n, const void *obs, const void *act,
                       const float *rew, const void *next_obs, const uint8_t *done,
                       const float *prio)
 {
-    if (!o || !prio) return ORACLE_ERR_NULL;
+    if (!o) return ORACLE_ERR_NULL;
     if (n == 0) return ORACLE_ERR_BAD_BATCH;
     if (n > o->capacity) return ORACLE_ERR_TOO_MANY;
     uint32_t D = o->depth;
+    const float dflt = default_priority(o);
     for (uint32_t t = 0; t < n; ++t) {
         uint64_t slot = (o->cursor + t) % o->capacity;
         if (obs) memcpy(o->obs + slot * o->obs_bytes, (const uint8_t *)obs + (size_t)t * o->obs_bytes, o->obs_bytes);
@@ -305,8 +315,9 @@ int oracle_prb_insert(oracle_prb_t *o, uint32_t n, const void *obs, const void *
         if (act) memcpy(o->act + slot * o->act_bytes, (const uint8_t *)act + (size_t)t * o->act_bytes, o->act_bytes);
         if (rew) o->rew[slot] = rew[t];
         if (done) o->done[slot] = done[t];
-        float p = prio[t];
+        float p = prio ? prio[t] : dflt;
         if (!valid_priority(p)) { p = 0.0f; o->status |= ST_BAD_PRIORITY; }
+        else note_priority(o, p);
         o->level[D][slot] = p;
         mark_dirty(o, D, slot);
     }
@@ -331,6 +342,7 @@ int oracle_prb_update_priorities(oracle_prb_t *o, uint32_t B, const int32_t *idx
     for (uint32_t b = 0; b < B; ++b) {
         if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
         if (!valid_priority(prio[b])) { o->status |= ST_BAD_PRIORITY; continue; }
+        note_priority(o, prio[b]);
         o->level[D][idx[b]] = prio[b];
         mark_dirty(o, D, (uint64_t)idx[b]);
     }
@@ -349,6 +361,7 @@ int oracle_prb_update(oracle_prb_t *o, uint32_t B, const int32_t *idx, const flo
         if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
         float p;
         if (oracle_priority_pow(td[b], eps, alpha, &p)) { o->status |= ST_BAD_PRIORITY; continue; }
+        note_priority(o, p);
         o->level[D][idx[b]] = p;
         mark_dirty(o, D, (uint64_t)idx[b]);
     }
@@ -377,6 +390,7 @@ int oracle_prb_update_after_insert(oracle_prb_t *o, uint32_t B, const int32_t *i
         if (back < inserted) { o->status |= ST_STALE; continue; }
         float p;
         if (oracle_priority_pow(td[b], eps, alpha, &p)) { o->status |= ST_BAD_PRIORITY; continue; }
+        note_priority(o, p);
         o->level[D][idx[b]] = p;
         mark_dirty(o, D, i);
     }

@@ -262,3 +262,25 @@ def test_update_after_insert_equals_update_then_insert(oracle_mod):
     assert o.read_level(3).tolist() == [1, 7, 7, 1, 5, 9, 2, 1]                      # 1 and 2 were skipped
     assert o.get_priorities([0, 2, 7, 8, -1]).tolist() == [1, 7, 1, 0, 0]
     assert o.status() == oracle_mod.ST_BAD_INDEX
+
+
+def test_default_insert_priority_is_running_maximum(oracle_mod):
+    # Schaul et al.: a new transition enters with the largest priority seen so far (1 before any).
+    o = oracle_mod.OraclePRB(16, 4, 0, 0)
+    assert o.max_priority() == 0
+    assert o.insert(None, None, None, None, None, None, n=2) == 0
+    assert o.read_level(2)[:2].tolist() == [1.0, 1.0] and o.max_priority() == 1.0
+    o.insert(None, None, None, None, None, np.array([3, 0.5, 4], np.float32))
+    assert o.max_priority() == 4.0
+    o.insert(None, None, None, None, None, None, n=2)
+    assert o.read_level(2)[:7].tolist() == [1, 1, 3, 0.5, 4, 4, 4]
+    o.update([0, 0], [100.0, 2.0], 0.5, 0.0)                 # 10 loses the duplicate race but was written
+    assert o.max_priority() == 10.0 and o.read_level(2)[0] == np.float32(2.0) ** np.float32(0.5)
+    o.update_priorities([1, 99], [50.0, 70.0])               # an invalid index does not count
+    assert o.max_priority() == 50.0
+    o.update([2], [np.nan], 0.5, 0.0)
+    o.insert(None, None, None, None, None, np.array([np.inf], np.float32))
+    assert o.max_priority() == 50.0 and o.status() == (oracle_mod.ST_BAD_INDEX | oracle_mod.ST_BAD_PRIORITY)
+    o.insert(None, None, None, None, None, None, n=1)
+    assert o.read_level(2)[8] == 50.0
+    check_invariant(o)
