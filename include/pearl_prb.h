@@ -88,7 +88,9 @@ int pearl_prb_destroy(pearl_prb_t* prb);
  * collected experiences are added to the Data Storage and insertion requests sent to the RM).
  * Writes n transitions to ring slots cursor .. cursor+n-1 (mod capacity), sets their leaves to
  * d_prio and re-sums the ancestors; then cursor += n (mod capacity), fill = min(fill+n, capacity).
- * The caller supplies each new transition's priority.  d_obs/d_next_obs: n rows of obs_bytes;
+ * d_prio gives each new transition's priority; with d_prio == NULL every new transition takes the
+ * largest priority written so far by any call (1 if none yet), the usual default of prioritized
+ * replay (Schaul et al.), so that it is replayed at least once.  d_obs/d_next_obs: n rows of obs_bytes;
  * d_act: n rows of act_bytes; d_rew: n binary32; d_done: n bytes; a NULL field pointer leaves
  * that field of the slots unwritten.  1 <= n <= min(max_batch, capacity). */
 int pearl_prb_insert(pearl_prb_t* prb, uint32_t n, const void* d_obs, const void* d_act,
@@ -205,6 +207,8 @@ int pearl_prb_sync(pearl_prb_t* prb, uint32_t* status_bits);
 /* Read-back for tests and checkpoints; each synchronises the stream.  Any output may be NULL. */
 int pearl_prb_info(pearl_prb_t* prb, uint64_t* fill, uint64_t* cursor, uint64_t* sample_calls,
                    uint32_t* depth);
+/* The largest priority written so far by insert or update calls (0 if none). */
+int pearl_prb_max_priority(pearl_prb_t* prb, float* h_out);
 /* Copies the first `count` entries (padding included) of tree level `level` (0 = root). */
 int pearl_prb_read_level(pearl_prb_t* prb, uint32_t level, float* h_dst, uint64_t count);
 /* Number of entries of a level including its zero padding; 0 for an invalid level. */

@@ -49,6 +49,7 @@ SIGNATURES = {
     "pearl_prb_update_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_sync": (_i, [_vp, C.POINTER(_u32)]),
     "pearl_prb_info": (_i, [_vp, C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u32)]),
+    "pearl_prb_max_priority": (_i, [_vp, C.POINTER(_f32)]),
     "pearl_prb_read_level": (_i, [_vp, _u32, _vp, _u64]),
     "pearl_prb_level_alloc": (_u64, [_vp, _u32]),
     "pearl_prb_read_rows": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp, _vp]),
@@ -135,8 +136,9 @@ class PrioritizedReplay:
         self.depth = self.info()[3]
 
     # ---- the four calls, device buffers ------------------------------------------------
-    def insert(self, obs, act, rew, next_obs, done, prio) -> None:
-        n = prio.numel()
+    def insert(self, obs, act, rew, next_obs, done, prio, n: Optional[int] = None) -> None:
+        """prio=None (with n given): the new transitions take the largest priority written so far."""
+        n = prio.numel() if prio is not None else int(n)
         rc = load_library().pearl_prb_insert(self._h, n, _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
                                              _dptr(next_obs, "next_obs"), _dptr(done, "done"), _dptr(prio, "prio"))
         if rc != 0:
@@ -182,17 +184,18 @@ class PrioritizedReplay:
         if rc != 0:
             raise PearlError(rc, "pearl_prb_get_priorities")
 
-    def update_insert(self, idx, td, alpha: float, eps: float, obs, act, rew, next_obs, done, prio) -> None:
+    def update_insert(self, idx, td, alpha: float, eps: float, obs, act, rew, next_obs, done, prio,
+                      n: Optional[int] = None) -> None:
         rc = load_library().pearl_prb_update_insert(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"), alpha, eps,
-                                                    prio.numel(), _dptr(obs, "obs"), _dptr(act, "act"),
+                                                    prio.numel() if prio is not None else int(n), _dptr(obs, "obs"), _dptr(act, "act"),
                                                     _dptr(rew, "rew"), _dptr(next_obs, "next_obs"),
                                                     _dptr(done, "done"), _dptr(prio, "prio"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_update_insert")
 
     # ---- the same calls, host buffers (numpy arrays or host torch tensors) -----------------
-    def insert_host(self, obs, act, rew, next_obs, done, prio) -> None:
-        n = int(prio.shape[0])
+    def insert_host(self, obs, act, rew, next_obs, done, prio, n: Optional[int] = None) -> None:
+        n = int(prio.shape[0]) if prio is not None else int(n)
         rc = load_library().pearl_prb_insert_host(self._h, n, _hptr(obs, "obs"), _hptr(act, "act"), _hptr(rew, "rew"),
                                                   _hptr(next_obs, "next_obs"), _hptr(done, "done"),
                                                   _hptr(prio, "prio"))
@@ -227,6 +230,13 @@ class PrioritizedReplay:
         if rc != 0:
             raise PearlError(rc, "pearl_prb_info")
         return f.value, c.value, n.value, d.value
+
+    def max_priority(self) -> float:
+        out = C.c_float(0.0)
+        rc = load_library().pearl_prb_max_priority(self._h, C.byref(out))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_max_priority")
+        return float(out.value)
 
     def level_alloc(self, level: int) -> int:
         return int(load_library().pearl_prb_level_alloc(self._h, level))

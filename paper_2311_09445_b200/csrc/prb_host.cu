@@ -200,13 +200,13 @@ int pearl_prb_destroy(pearl_prb_t* h)
 int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* d_act, const float* d_rew,
                      const void* d_next_obs, const uint8_t* d_done, const float* d_prio)
 {
-    if (!h || !d_prio) return PEARL_ERR_NULL;
+    if (!h) return PEARL_ERR_NULL;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
     const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
     int rc = check_batch_ptrs(h, ptrs);
     if (rc != PEARL_OK) return rc;
-    if (misaligned(d_prio, 4)) return PEARL_ERR_ALIGN;
+    if (d_prio && misaligned(d_prio, 4)) return PEARL_ERR_ALIGN;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
@@ -286,7 +286,7 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
                             uint32_t n, const void* d_obs, const void* d_act, const float* d_rew, const void* d_next_obs,
                             const uint8_t* d_done, const float* d_prio)
 {
-    if (!h || !d_idx || !d_td || !d_prio) return PEARL_ERR_NULL;
+    if (!h || !d_idx || !d_td) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
@@ -294,7 +294,7 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
     const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
     int rc = check_batch_ptrs(h, ptrs);
     if (rc != PEARL_OK) return rc;
-    if (misaligned(d_prio, 4) || misaligned(d_idx, 4) || misaligned(d_td, 4)) return PEARL_ERR_ALIGN;
+    if ((d_prio && misaligned(d_prio, 4)) || misaligned(d_idx, 4) || misaligned(d_td, 4)) return PEARL_ERR_ALIGN;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
@@ -310,7 +310,7 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
 int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const void* h_act, const float* h_rew,
                           const void* h_next_obs, const uint8_t* h_done, const float* h_prio)
 {
-    if (!h || !h_prio) return PEARL_ERR_NULL;
+    if (!h) return PEARL_ERR_NULL;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
     DeviceGuard guard(h->device);
@@ -324,8 +324,9 @@ int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const v
         dev[f] = at(h, h->lay.off_stage_in[f]);
         if (cudaMemcpyAsync(dev[f], src[f], bytes, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
     }
-    float* d_prio = (float*)at(h, h->lay.off_stage_prio);
-    if (cudaMemcpyAsync(d_prio, h_prio, (uint64_t)n * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    float* d_prio = h_prio ? (float*)at(h, h->lay.off_stage_prio) : nullptr;
+    if (h_prio && cudaMemcpyAsync(d_prio, h_prio, (uint64_t)n * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess)
+        return PEARL_ERR_CUDA;
     int rc = pearl_prb_insert(h, n, dev[F_OBS], dev[F_ACT], (const float*)dev[F_REW], dev[F_NEXT_OBS],
                               (const uint8_t*)dev[F_DONE], d_prio);
     if (rc != PEARL_OK) return rc;
@@ -449,6 +450,18 @@ int pearl_prb_info(pearl_prb_t* h, uint64_t* fill, uint64_t* cursor, uint64_t* s
     if (cursor) *cursor = st.cursor;
     if (sample_calls) *sample_calls = st.sample_calls;
     if (depth) *depth = h->view.depth;
+    return PEARL_OK;
+}
+
+int pearl_prb_max_priority(pearl_prb_t* h, float* out)
+{
+    if (!h || !out) return PEARL_ERR_NULL;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    unsigned int bits = 0;
+    if (cudaMemcpyAsync(&bits, &h->view.state->max_prio_bits, 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    memcpy(out, &bits, 4);
     return PEARL_OK;
 }
 

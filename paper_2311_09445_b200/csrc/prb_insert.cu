@@ -110,13 +110,14 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
 {
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
+    __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
     const uint32_t tid = threadIdx.x;
-    if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
+    if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; s_maxp = v.state->max_prio_bits; }
     // the tree CTA fetches its first inputs now, while the cursor is on its way
     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
     if (blockIdx.x == 0 && tid < kWorkers) {
         if (tid < upd.B) { pre.has_update = true; pre.idx = upd.idx[tid]; pre.val = upd.val[tid]; }
-        if (tid < n) { pre.has_prio = true; pre.prio = prio[tid]; }
+        if (tid < n && prio != nullptr) { pre.has_prio = true; pre.prio = prio[tid]; }
     }
     __syncthreads();
     const uint64_t cursor = s_cursor;
@@ -129,7 +130,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
             if (upd.B)      // update and insertion share one re-sum pass per level
                 prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre);
             else
-                prb_insert_tree_team(v, team, n, prio, cursor, pre);
+                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
@@ -152,6 +153,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
+    __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
     const uint32_t tid = threadIdx.x;
     const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
     const uint32_t first_copy_cta = upd.B ? 1u : 0u;
@@ -177,7 +179,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     PrbBulkLane ring;
     int f = 0; uint32_t row = 0, W = 0, e0 = 0, bytes = 0;
     uint32_t t = t_lo + tid;
-    if (tid == kPublisher) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
+    if (tid == kPublisher) { s_cursor = v.state->cursor; s_fill = v.state->fill; s_maxp = v.state->max_prio_bits; }
     if (ring_lane) {
         ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
         if (t < t_hi) {
@@ -208,7 +210,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
         if (blockIdx.x == 0) {
             if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_ring);
-            prb_insert_tree_team(v, team, n, prio, cursor);
+            prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp);
         }
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
         for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)

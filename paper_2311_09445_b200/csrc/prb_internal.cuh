@@ -18,7 +18,7 @@ struct PrbState {
     unsigned int status;              // PEARL_ST_* bits
     unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
     unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished
-    unsigned int reserved;
+    unsigned int max_prio_bits;       // bits of the largest priority written so far (0: none yet)
 };
 
 // Geometry and device addresses, passed to kernels by value.
@@ -86,6 +86,17 @@ __device__ __forceinline__ float prb_sum_children_dyn(const float* c, uint32_t K
     case 16: return prb_sum_children<16>(c);
     default: return prb_sum_children<32>(c);
     }
+}
+
+// The running maximum of written priorities: positive binary32 values order like their bit patterns.
+__device__ __forceinline__ void prb_note_priorities(PrbState* st, float local_max, bool report)
+{
+    const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(local_max));
+    if (report && (threadIdx.x & 31u) == 0 && m) atomicMax(&st->max_prio_bits, m);
+}
+__device__ __forceinline__ float prb_default_priority(unsigned max_bits)
+{
+    return max_bits ? __uint_as_float(max_bits) : 1.0f;
 }
 
 __device__ __forceinline__ bool prb_valid_priority(float p)

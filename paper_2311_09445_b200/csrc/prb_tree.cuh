@@ -135,6 +135,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     const uint32_t rank = team.rank, nt = team.size;
 
     unsigned flags = 0;
+    float wmax = 0.0f;                 // largest priority this thread accepted
     bool unsorted = false;
     unsigned long long my_key = kPrbInvalidKey;      // the key of entry `rank` (one-key-per-thread case)
     for (uint32_t b = rank; b < n2; b += nt) {
@@ -152,13 +153,14 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
             else if (back < stale) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
-            else key = ((unsigned long long)(uint32_t)i << 32) | b;
+            else { key = ((unsigned long long)(uint32_t)i << 32) | b; wmax = fmaxf(wmax, p); }
             vals[b] = p;
         }
         keys[b] = key;
         my_key = key;
     }
     if (flags && team.part == 0) atomicOr(&v.state->status, flags);
+    prb_note_priorities(v.state, wmax, team.part == 0);
     team.sync();
 
     // Indices that come straight from a stratified sample are already in order; sort only if needed.
@@ -213,15 +215,20 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         if (last && !(ahead < n)) leaves[i] = vals[(uint32_t)key];
     }
     bool bad = false;
+    float imax = 0.0f;
+    // without priorities the new transitions take the running maximum, this update's writes included
+    const float dflt = (n && prio == nullptr) ? prb_default_priority(__ldcg(&v.state->max_prio_bits)) : 0.0f;
     for (uint32_t t = rank; t < n; t += nt) {
         if (!team.takes(t)) continue;
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
-        float p = (pre.has_prio && t == rank) ? pre.prio : prio[t];
+        float p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+        else imax = fmaxf(imax, p);
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
+    if (n && prio != nullptr) prb_note_priorities(v.state, imax, team.part == 0);
     team.phase_sync();
 
     // re-sum the ancestors, deepest level first; the insertion dirties parent range A = [a0, a1] >> sh
@@ -260,20 +267,25 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
 // a contiguous parent range on every level (two ranges if the ring wrapped), so nothing is sorted.
 __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const PrbTeam& team, uint32_t n,
                                                      const float* __restrict__ prio, uint64_t cursor,
-                                                     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f})
+                                                     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
+                                                     unsigned max_bits = 0)
 {
     const uint64_t N = v.capacity;
     const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
     float* leaves = v.level[D];
     bool bad = false;
+    float imax = 0.0f;
+    const float dflt = prb_default_priority(max_bits);     // used when no priorities are given
     for (uint32_t t = team.rank; t < n; t += team.size) {
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
-        float p = (pre.has_prio && t == team.rank) ? pre.prio : prio[t];
+        float p = prio == nullptr ? dflt : ((pre.has_prio && t == team.rank) ? pre.prio : prio[t]);
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+        else imax = fmaxf(imax, p);
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
+    if (prio != nullptr) prb_note_priorities(v.state, imax, true);
     team.sync();
     // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;

@@ -128,6 +128,7 @@ class Pair:
 
     def compare_state(self):
         assert self.gpu.info() == self.ora.info()
+        assert np.float32(self.gpu.max_priority()) == self.ora.max_priority()
 
     def compare_status(self):
         s_g, s_o = self.gpu.sync(), self.ora.status()

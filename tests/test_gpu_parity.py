@@ -407,6 +407,46 @@ def test_update_after_insert_and_retrieval(oracle_mod, K, N, B, n):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N", [(wk.CARTPOLE, 3000), (wk.ATARI, 600)])
+def test_default_insert_priority(oracle_mod, wl, N):
+    # insertion without priorities: the running maximum of everything written so far (1 before any)
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(N)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 512)
+    dev = pr.dev
+
+    def insert_default(n, first, fused_with=None):
+        b = wk.transitions(wl, rng, n, first)
+        d = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in b.items() if k != "prio"}
+        if fused_with is None:
+            assert pr.ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], None, n=n) == 0
+            pr.gpu.insert(d["obs"], d["act"], d["rew"], d["next_obs"], d["done"], None, n=n)
+        else:
+            idx, td = fused_with
+            assert pr.ora.update(idx, td, 0.6, 1e-6) == 0
+            assert pr.ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], None, n=n) == 0
+            pr.gpu.update_insert(torch.from_numpy(idx).to(dev), torch.from_numpy(td).to(dev), 0.6, 1e-6, d["obs"], d["act"],
+                                 d["rew"], d["next_obs"], d["done"], None, n=n)
+
+    insert_default(100, 0)                        # nothing written yet: priority 1
+    pr.compare_tree()
+    pr.compare_state()
+    pr.insert(wk.transitions(wl, rng, 200, 100))  # explicit priorities raise the maximum
+    pr.compare_state()
+    for step in range(6):
+        o, g = pr.sample(128, 0.4, 1)
+        td = (rng.standard_normal(128) * (step + 1) * 3).astype(np.float32)
+        if step % 2 == 0:
+            pr.update(o["idx"], td, 0.6, 1e-6)
+            insert_default(77, 300 + 77 * step)
+        else:
+            insert_default(77, 300 + 77 * step, fused_with=(o["idx"], td))   # the update's writes count already
+        pr.compare_tree()
+        pr.compare_state()
+    pr.compare_status()
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)
