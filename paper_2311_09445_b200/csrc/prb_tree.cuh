@@ -228,7 +228,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    if (n && prio != nullptr) prb_note_priorities(v.state, imax, team.part == 0);
+    if (n) prb_note_priorities(v.state, imax, team.part == 0);      // (a first default insertion writes 1)
     team.phase_sync();
 
     // re-sum the ancestors, deepest level first; the insertion dirties parent range A = [a0, a1] >> sh
@@ -285,7 +285,7 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
         leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    if (prio != nullptr) prb_note_priorities(v.state, imax, true);
+    prb_note_priorities(v.state, imax, true);                       // (a first default insertion writes 1)
     team.sync();
     // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;
