@@ -114,6 +114,13 @@ int pearl_prb_sample(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, in
                      float* d_w, void* d_obs, void* d_act, float* d_rew, void* d_next_obs,
                      uint8_t* d_done);
 
+/* Uniform replay (the toolkit's other replay mode, Section III-B: set_replay(size, mode, fanout)):
+ * B independent draws i_k = floor(u_k * fill) from the transitions stored, u_k from the same Philox
+ * stream and call counter as pearl_prb_sample; the tree is not read.  d_w (may be NULL) is filled
+ * with 1; the gathered rows as in pearl_prb_sample.  An empty buffer raises PEARL_ST_EMPTY. */
+int pearl_prb_sample_uniform(pearl_prb_t* prb, uint32_t B, uint64_t seed, int32_t* d_idx, float* d_w,
+                             void* d_obs, void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done);
+
 /* Priority update (Section V-A).  For b = 0 .. B-1 in batch order: p_b = (|d_td[b]| + eps)^alpha
  * and leaf[d_idx[b]] <- p_b, so the last valid entry of a repeated index wins; then every
  * ancestor of a written leaf is recomputed as the left-to-right binary32 sum of its children,

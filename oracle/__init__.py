@@ -54,6 +54,7 @@ def lib():
         L.oracle_prb_targets.argtypes = [vp, u32, u64, u64, vp]
         L.oracle_prb_targets.restype = None
         L.oracle_prb_sample.argtypes = [vp, u32, f32, u64, vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_prb_sample_uniform.argtypes = [vp, u32, u64, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_prb_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64), C.POINTER(u32)]
         L.oracle_prb_level_nodes.argtypes = [vp, u32]
         L.oracle_prb_level_nodes.restype = u64
@@ -174,6 +175,16 @@ class OraclePRB:
         x = np.zeros(B, dtype=np.float64)
         lib().oracle_prb_targets(self._h, B, seed, call, _ptr(x))
         return x
+
+    def sample_uniform(self, B: int, seed: int):
+        out = {"idx": np.full(B, -1, dtype=np.int32), "w": np.zeros(B, dtype=np.float32),
+               "obs": np.zeros((B, self.obs_bytes), dtype=np.uint8), "act": np.zeros((B, self.act_bytes), dtype=np.uint8),
+               "rew": np.zeros(B, dtype=np.float32), "next_obs": np.zeros((B, self.obs_bytes), dtype=np.uint8),
+               "done": np.zeros(B, dtype=np.uint8)}
+        out["rc"] = lib().oracle_prb_sample_uniform(self._h, B, seed, _ptr(out["idx"]), _ptr(out["w"]), _ptr(out["obs"]),
+                                                    _ptr(out["act"]), _ptr(out["rew"]), _ptr(out["next_obs"]),
+                                                    _ptr(out["done"]))
+        return out
 
     def sample(self, B: int, beta: float, seed: int, gather: bool = True):
         """Returns a dict with idx, w and (if ``gather``) the gathered fields as raw bytes / f32."""

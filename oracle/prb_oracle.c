@@ -516,6 +516,32 @@ int oracle_prb_sample(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
     return ORACLE_OK;
 }
 
+int oracle_prb_read_rows(oracle_prb_t *o, const int32_t *idx, uint32_t n, void *obs, void *act,
+                         float *rew, void *next_obs, uint8_t *done);
+
+/* Uniform replay (Section III-B: the toolkit's replay mode besides "prioritized"): B independent */
+/* draws i_k = floor(u_k * size), u_k from the same Philox stream and call counter as the          */
+/* prioritized sample; weights are all 1; rows are gathered as usual.                              */
+int oracle_prb_sample_uniform(oracle_prb_t *o, uint32_t B, uint64_t seed, int32_t *idx, float *w, void *obs,
+                              void *act, float *rew, void *next_obs, uint8_t *done)
+{
+    if (!o || !idx) return ORACLE_ERR_NULL;
+    if (B == 0) return ORACLE_ERR_BAD_BATCH;
+    if (o->size == 0) { o->status |= ST_EMPTY; return ORACLE_OK; }
+    for (uint32_t k = 0; k < B; ++k) {
+        uint32_t ctr[4] = { k, 0u, (uint32_t)o->sample_calls, (uint32_t)(o->sample_calls >> 32) };
+        uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+        uint32_t r[4];
+        oracle_philox4x32_10(ctr, key, r);
+        idx[k] = (int32_t)(((uint64_t)r[0] * o->size) >> 32);        /* floor(r0 / 2^32 * size) */
+        if (w) w[k] = 1.0f;
+    }
+    int rc = oracle_prb_read_rows(o, idx, B, obs, act, rew, next_obs, done);
+    if (rc != ORACLE_OK) return rc;
+    o->sample_calls += 1;
+    return ORACLE_OK;
+}
+
 /* ------------------------------------------------------------------------ */
 /* Read-back                                                                 */
 /* ------------------------------------------------------------------------ */

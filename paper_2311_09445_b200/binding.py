@@ -38,6 +38,7 @@ SIGNATURES = {
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample_uniform": (_i, [_vp, _u32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
@@ -151,6 +152,13 @@ class PrioritizedReplay:
                                              _dptr(next_obs, "next_obs"), _dptr(done, "done"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_sample")
+
+    def sample_uniform(self, B: int, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None, done=None) -> None:
+        rc = load_library().pearl_prb_sample_uniform(self._h, B, seed, _dptr(idx, "idx"), _dptr(w, "w"), _dptr(obs, "obs"),
+                                                     _dptr(act, "act"), _dptr(rew, "rew"), _dptr(next_obs, "next_obs"),
+                                                     _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample_uniform")
 
     def sample_static_scratch(self, B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None,
                               next_obs=None, done=None) -> None:

@@ -217,8 +217,8 @@ int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* 
     return PEARL_OK;
 }
 
-int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
-                     void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
+                         void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done, int uniform)
 {
     if (!h || !d_idx) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
@@ -231,10 +231,22 @@ int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int3
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
-    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream);
+    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
     return PEARL_OK;
+}
+
+int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
+                     void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    return sample_common(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 0);
+}
+
+int pearl_prb_sample_uniform(pearl_prb_t* h, uint32_t B, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
+                             void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    return sample_common(h, B, 0.0f, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 1);
 }
 
 static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_val, int raw, float alpha,

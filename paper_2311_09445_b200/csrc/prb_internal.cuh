@@ -47,8 +47,9 @@ struct PrbBatch {
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
                       int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f);
+// (uniform != 0: uniform replay, no tree walk, all weights 1)
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s);
+                      const PrbBatch& dst, cudaStream_t s, int uniform = 0);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale = 0);

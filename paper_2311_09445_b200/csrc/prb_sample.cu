@@ -42,6 +42,7 @@ struct SamplePlan {
     uint32_t chunks[PRB_NUM_FIELDS];         //   copy the chunks of field f; 0 = short rows, copied flat
     uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
     uint32_t ring_stages, ring_stage_bytes;  // bulk-copy ring (long rows only; 0 stages otherwise)
+    uint32_t uniform;                        // 1: uniform replay (no tree walk): index = floor(u * fill)
     uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
     uint32_t top_vec4;                       // 16-byte units staged, from the start of level 1
     uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level from the start of level 1
@@ -201,7 +202,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
             if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
     }
-    const bool empty = (fill == 0) || !(total32 > 0.0f);
+    const bool empty = (fill == 0) || (!plan.uniform && !(total32 > 0.0f));
 
     // this CTA's tasks and the strata they touch
     const uint32_t tps = plan.tps;
@@ -218,7 +219,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         // ---- targets: stratum k of the batch draws x_k ----
         const uint32_t gi = tid / K, lane = tid % K;
         bool walks = false;
-        uint32_t k = 0;
+        uint32_t k = 0, r0 = 0;
         double x = 0.0;
         const double total = (double)total32;
         if (round < n_rounds) {
@@ -227,7 +228,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (walks) {
                 k = min(kb + gi, B - 1);                  // surplus groups repeat a valid stratum and write nothing
                 const double seg = __ddiv_rn(total, (double)B);
-                const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32),
+                r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32),
                                                         (uint32_t)seed, (uint32_t)(seed >> 32));
                 const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
                 x = __dmul_rn(__dadd_rn((double)k, u), seg);
@@ -239,7 +240,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             // ---- descents: one K-lane group per stratum ----
             if (walks) {
                 uint32_t leaf; float p; unsigned flags = 0;
-                descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
+                if (plan.uniform) { leaf = (uint32_t)(((unsigned long long)r0 * fill) >> 32); p = 1.0f; }   // floor(u * fill)
+                else descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
                 if (lane == 0 && gi < n_round) { s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags; }
             }
             __syncthreads();
@@ -255,7 +257,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                 if (kb + gi2 >= k_own) {
                     const uint32_t k2 = kb + gi2;
                     const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
-                    wr = pow(scaled, -(double)beta);
+                    wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
                     out_idx[k2] = (int32_t)s_idx[gi2];
                     v.wraw[k2] = wr;
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
@@ -327,7 +329,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 }  // namespace
 
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s)
+                      const PrbBatch& dst, cudaStream_t s, int uniform)
 {
     static int sm_count = 0;
     if (sm_count == 0) {
@@ -356,10 +358,11 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     plan.n_tasks = B * plan.tps;
     // levels 1 .. top_levels staged in shared memory while they fit
     // (the levels lie one after another in the slab, each start 256-byte aligned)
+    plan.uniform = uniform ? 1u : 0u;
     plan.top_levels = 0;
     plan.top_vec4 = 0;
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
-    for (uint32_t l = 1; l <= v.depth; ++l) {
+    for (uint32_t l = 1; l <= v.depth && !uniform; ++l) {
         const uint64_t off = (uint64_t)(v.level[l] - v.level[1]);
         if (off + v.level_alloc[l] > kTopFloats) break;
         plan.top_off[l] = (uint32_t)off;

@@ -447,6 +447,35 @@ def test_default_insert_priority(oracle_mod, wl, N):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B", [(wk.CARTPOLE, 3000, 64), (wk.DDPG, 100_000, 4096), (wk.ATARI, 700, 512)])
+def test_uniform_replay(oracle_mod, wl, N, B):
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(B)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096)
+    dev = pr.dev
+    first = 0
+    for _ in range(3):
+        m = min(N // 4, 4096)
+        pr.insert(wk.transitions(wl, rng, m, first))
+        first += m
+        for call in range(2):
+            o = pr.ora.sample_uniform(B, 9)
+            t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+                 "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+                 "act": torch.zeros((B, wl.act_bytes), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+                 "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+                 "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+            pr.gpu.sample_uniform(B, 9, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+            torch.cuda.synchronize()
+            g = {k: v.cpu().numpy() for k, v in t.items()}
+            assert g["idx"].max() < first
+            pr.compare_sample(o, g)
+        o, g = pr.sample(B, 0.4, 9)            # prioritized and uniform calls share the call counter
+    pr.compare_state()
+    assert pr.compare_status() == 0
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)

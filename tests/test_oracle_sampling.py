@@ -175,3 +175,28 @@ def test_gather_bytes(oracle_mod):
     i = out["idx"]
     for name in ("obs", "act", "rew", "next_obs", "done"):
         assert np.array_equal(out[name], f[name][i])
+
+
+def test_uniform_replay(oracle_mod):
+    # i_k = floor(u_k * size): in range, uniform (chi-square), independent of the priorities, rows gathered
+    rng = np.random.default_rng(12)
+    N = 50
+    f = dict(obs=rng.integers(0, 256, size=(N, 8), dtype=np.uint8), act=rng.integers(0, 256, size=(N, 2), dtype=np.uint8),
+             rew=rng.normal(size=N).astype(np.float32), next_obs=rng.integers(0, 256, size=(N, 8), dtype=np.uint8),
+             done=rng.integers(0, 2, size=N, dtype=np.uint8))
+    o = oracle_mod.OraclePRB(64, 4, 8, 2)
+    assert o.sample_uniform(4, 0)["idx"].tolist() == [-1] * 4 and o.status() == oracle_mod.ST_EMPTY
+    o.insert(f["obs"], f["act"], f["rew"], f["next_obs"], f["done"], np.exp(3 * rng.normal(size=N)).astype(np.float32))
+    counts = np.zeros(N, dtype=np.int64)
+    for call in range(400):
+        assert o.info()[2] == call
+        out = o.sample_uniform(100, 5)
+        i = out["idx"]
+        u = np.array([oracle_mod.stratum_uniform(5, call, k) for k in range(100)])
+        assert i.tolist() == np.floor(u * N).astype(np.int64).tolist()
+        assert np.all(out["w"] == 1.0)
+        for name in ("obs", "act", "rew", "next_obs", "done"):
+            assert np.array_equal(out[name], f[name][i])
+        counts += np.bincount(i, minlength=N)
+    chi2 = ((counts - 800.0) ** 2 / 800.0).sum()
+    assert stats.chi2.sf(chi2, N - 1) > 1e-4
