@@ -223,13 +223,8 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps)
 {
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            sm_count = 148;
-    }
+    const int sm_count = prb_sm_count();
+    const int dev = prb_current_device();
     FusedUpdate upd;
     upd.B = upd_B; upd.n2 = 2; upd.idx = upd_idx; upd.val = upd_val; upd.raw = upd_raw; upd.alpha = alpha; upd.eps = eps;
     while (upd.n2 < upd_B) upd.n2 <<= 1;
@@ -269,11 +264,11 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     }
     const uint32_t upd_smem = upd.B ? (uint32_t)prb_update_smem_bytes(upd.n2) : 0u;
     if (tasks == 0) {
-        static bool big_smem = false;
-        if (upd_smem + 64 > 48 * 1024 && !big_smem) {
+        static bool big_smem[kPrbMaxDevices];
+        if (upd_smem + 64 > 48 * 1024 && !big_smem[dev]) {
             if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
                 return -1;
-            big_smem = true;
+            big_smem[dev] = true;
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
@@ -284,12 +279,12 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
         const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;     // >= the update's keys (<= 48 KB)
-        static bool big_smem = false;
-        if (!big_smem) {
+        static bool big_rows[kPrbMaxDevices];
+        if (!big_rows[dev]) {
             if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
                 return -1;
-            big_smem = true;
+            big_rows[dev] = true;
         }
         const uint32_t want = tasks + (upd.B ? 1u : 0u);           // with an update, CTA 0 moves no rows
         const uint32_t grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;

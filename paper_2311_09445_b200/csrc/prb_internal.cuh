@@ -55,6 +55,27 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
                       float alpha, float eps, cudaStream_t s, uint32_t stale = 0);
 int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s);
 
+// Per-device facts the launchers cache: SM count, and which kernels already have their large
+// dynamic shared memory enabled (the attribute is per device).  One slot per device ordinal.
+constexpr int kPrbMaxDevices = 64;
+inline int prb_current_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kPrbMaxDevices) return 0;
+    return dev;
+}
+inline int prb_sm_count()
+{
+    static int cached[kPrbMaxDevices];
+    const int dev = prb_current_device();
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 // ---- device helpers -------------------------------------------------------------------
 #ifdef __CUDACC__
 

@@ -331,13 +331,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s, int uniform)
 {
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            sm_count = 148;
-    }
+    const int sm_count = prb_sm_count();
+    const int dev = prb_current_device();
     SamplePlan plan;
     plan.tps = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
@@ -391,15 +386,15 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         const uint32_t want = (B + per_cta - 1) / per_cta;
         grid = want < one_wave ? want : one_wave;
     }
-    static bool big_smem[6] = { false, false, false, false, false, false };
+    static bool big_smem[kPrbMaxDevices][6];
     const int ki = v.log2_fanout;
     cudaError_t attr = cudaSuccess;
 #define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
     do {                                                                                                          \
-        if (smem && !big_smem[ki]) {                                                                              \
+        if (smem && !big_smem[dev][ki]) {                                                                              \
             attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                         (int)(kRingBarBytes + kRingBytes));                                       \
-            big_smem[ki] = (attr == cudaSuccess);                                                                 \
+            big_smem[dev][ki] = (attr == cudaSuccess);                                                                 \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \
             prb_sample_kernel<KK><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);          \
