@@ -476,6 +476,75 @@ def test_uniform_replay(oracle_mod, wl, N, B):
     pr.close()
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_random_call_sequences(oracle_mod, seed):
+    # Random geometry and a random sequence of every call, compared with the oracle after each one.
+    rng = np.random.default_rng(9000 + seed)
+    K = int(rng.choice([2, 4, 8, 16, 32]))
+    N = int(rng.choice([1, 3, 17, 256, 1000, 4099, 20_000]))
+    obs_bytes = int(rng.choice([0, 1, 6, 16, 68, 100, 8192, 8208]))
+    act_bytes = int(rng.choice([0, 4, 24]))
+    maxb = 700
+    pr = Pair(oracle_mod, N, K, obs_bytes, act_bytes, maxb)
+    dev = pr.dev
+    inserted_since, last_idx = 0, None
+
+    def new_batch(n, with_prio=True):
+        b = raw_fields(rng, n, obs_bytes, act_bytes)
+        b["prio"] = np.exp(rng.standard_normal(n)).astype(np.float32) if with_prio else None
+        return b
+
+    for step in range(40):
+        op = rng.choice(["insert", "insert_default", "sample", "uniform", "update", "raw", "after", "fused", "get"],
+                        p=[0.2, 0.05, 0.2, 0.05, 0.15, 0.05, 0.1, 0.15, 0.05])
+        fill = pr.ora.info()[0]
+        n = int(rng.integers(1, min(N, maxb) + 1))
+        B = int(rng.integers(1, maxb + 1))
+        some_idx = (rng.integers(-1, max(fill, 1) + 1, size=B)).astype(np.int32)     # a few out of range
+        td = (rng.standard_normal(B) * 3).astype(np.float32)
+        if op == "insert":
+            pr.insert(new_batch(n))
+            inserted_since += n
+        elif op == "insert_default":
+            b = new_batch(n, with_prio=False)
+            assert pr.ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], None, n=n) == 0
+            d = {k: torch.from_numpy(v).to(dev) for k, v in b.items() if v is not None}
+            pr.gpu.insert(d["obs"], d["act"], d["rew"], d["next_obs"], d["done"], None, n=n)
+            inserted_since += n
+        elif op == "sample":
+            o, g = pr.sample(B, float(rng.choice([0.0, 0.4, 1.0])), seed)
+            if o["idx"][0] >= 0:
+                last_idx, inserted_since = o["idx"].copy(), 0
+        elif op == "uniform":
+            o = pr.ora.sample_uniform(B, seed)
+            t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+                 "obs": torch.zeros((B, obs_bytes), dtype=torch.uint8, device=dev),
+                 "act": torch.zeros((B, act_bytes), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+                 "next_obs": torch.zeros((B, obs_bytes), dtype=torch.uint8, device=dev),
+                 "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+            pr.gpu.sample_uniform(B, seed, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+            torch.cuda.synchronize()
+            pr.compare_sample(o, {k: v.cpu().numpy() for k, v in t.items()})
+        elif op == "update":
+            pr.update(some_idx, td, 0.6, 1e-6)
+        elif op == "raw":
+            pr.update_priorities(some_idx, np.abs(td))
+        elif op == "after" and last_idx is not None:
+            m = min(inserted_since, N)
+            pr.update_after_insert(last_idx, td[:len(last_idx)] if len(last_idx) <= B else np.resize(td, len(last_idx)),
+                                   0.6, 1e-6, m)
+        elif op == "fused":
+            pr.update_insert(some_idx, td, 0.6, 1e-6, new_batch(n))
+            inserted_since += n
+        elif op == "get":
+            pr.compare_priorities(some_idx)
+        pr.compare_tree()
+        pr.compare_state()
+        pr.compare_status()
+    pr.compare_rows(np.arange(min(pr.ora.info()[0], N), dtype=np.int32)[:2000])
+    pr.close()
+
+
 def test_update_is_deterministic(oracle_mod):
     # The same batch with many duplicates, replayed: identical tree bytes every time.
     rng = np.random.default_rng(13)
