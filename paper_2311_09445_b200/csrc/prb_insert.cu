@@ -108,7 +108,6 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
                   const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
                   const __grid_constant__ FusedUpdate upd)
 {
-    prb_grid_begin();
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
     __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
@@ -152,7 +151,6 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
                        const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
                        const __grid_constant__ FusedUpdate upd)
 {
-    prb_grid_begin();
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
     __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
@@ -274,7 +272,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        if (prb_launch(prb_insert_kernel, copy_ctas + 1, kThreadsShort, upd_smem, s, 1, v, n, src, d_prio, plan, upd) != cudaSuccess) return -1;
+        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem, s>>>(v, n, src, d_prio, plan, upd);
     } else {
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
@@ -290,7 +288,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         }
         const uint32_t want = tasks + (upd.B ? 1u : 0u);           // with an update, CTA 0 moves no rows
         const uint32_t grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
-        if (prb_launch(prb_insert_rows_kernel, grid, kThreadsRows, smem < upd_smem ? upd_smem : smem, s, 1, v, n, src, d_prio, plan, upd) != cudaSuccess) return -1;
+        prb_insert_rows_kernel<<<grid, kThreadsRows, smem < upd_smem ? upd_smem : smem, s>>>(v, n, src, d_prio, plan, upd);
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

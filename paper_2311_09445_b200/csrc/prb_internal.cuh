@@ -79,45 +79,6 @@ inline int prb_sm_count()
 // ---- device helpers -------------------------------------------------------------------
 #ifdef __CUDACC__
 
-// Programmatic dependent launch.  Every kernel of the library is launched with programmatic
-// stream serialisation and begins with prb_grid_begin(): it first waits (a hardware wait, not
-// a loop) until everything enqueued before it on the stream has completed and is visible, and
-// only then touches memory; then it lets the kernel enqueued after it be scheduled early, so
-// that the next kernel's launch latency hides behind this kernel's run.  The next kernel waits
-// in the same way before it reads anything, so the order of the results is the stream order.
-// Launched without the attribute, both instructions do nothing.
-__device__ __forceinline__ void prb_grid_begin()
-{
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-
-// Launch with programmatic stream serialisation (and, if cluster > 1, that cluster width).
-template <typename... KArgs, typename... Args>
-inline cudaError_t prb_launch(void (*kernel)(KArgs...), uint32_t grid, uint32_t block, size_t smem, cudaStream_t s,
-                              uint32_t cluster, Args... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    unsigned n_attr = 1;
-    if (cluster > 1) {
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = cluster;
-        attr[1].val.clusterDim.y = 1;
-        attr[1].val.clusterDim.z = 1;
-        n_attr = 2;
-    }
-    cfg.attrs = attr;
-    cfg.numAttrs = n_attr;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
-}
-
 // Left-to-right binary32 sum of the K children of one parent (children start at c, K-aligned).
 // Loads bypass L1: other threads of this kernel may have written the children.
 template <int K>

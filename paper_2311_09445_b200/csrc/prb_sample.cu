@@ -172,7 +172,6 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                   int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
                   const __grid_constant__ SamplePlan plan)
 {
-    prb_grid_begin();
     constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
     __shared__ float s_top[kTopFloats];
     __shared__ uint32_t s_idx[R];
@@ -398,7 +397,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
             big_smem[dev][ki] = (attr == cudaSuccess);                                                                 \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \
-            attr = prb_launch(prb_sample_kernel<KK>, grid, kThreads, smem, s, 1, v, B, beta, seed, d_idx, d_w, dst, plan); \
+            prb_sample_kernel<KK><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);          \
     } while (0)
     switch (v.fanout) {
     case 2: PRB_LAUNCH_SAMPLE(2); break;

@@ -13,7 +13,6 @@ __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
                   const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale)
 {
-    prb_grid_begin();
     extern __shared__ __align__(16) unsigned char smem[];
     PrbTeam team;
     team.rank = threadIdx.x;
@@ -31,7 +30,6 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 __global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
                                           float* __restrict__ out)
 {
-    prb_grid_begin();
     const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int32_t i = idx[b];
@@ -43,7 +41,8 @@ __global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uin
 
 int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s)
 {
-    return prb_launch(prb_get_priorities_kernel, (B + 255) / 256, 256, 0, s, 1, v, B, d_idx, d_out) == cudaSuccess ? 1 : -1;
+    prb_get_priorities_kernel<<<(B + 255) / 256, 256, 0, s>>>(v, B, d_idx, d_out);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
@@ -60,8 +59,19 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
         // one SM keeps in flight: then eight CTAs of one cluster share each level.
         const uint32_t ctas = (v.fanout * b >= 8192u) ? 8u : 1u;
-        if (prb_launch(prb_update_kernel, ctas, threads, prb_update_smem_bytes(n2), s, ctas, v, b, n2, d_idx + first,
-                       d_val + first, raw, alpha, eps, stale) != cudaSuccess)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(ctas);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = ctas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale) != cudaSuccess)
             return -1;
         ++launches;
     }
