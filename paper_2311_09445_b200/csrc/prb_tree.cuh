@@ -101,7 +101,10 @@ __device__ __forceinline__ bool prb_priority_pow(float delta, float eps, float a
     return true;
 }
 
+// A skipped entry keeps its batch position under an index of all ones: such keys sort last and, like
+// the valid ones, are all different.
 constexpr unsigned long long kPrbInvalidKey = ~0ull;
+__device__ __forceinline__ bool prb_key_invalid(unsigned long long key) { return (uint32_t)(key >> 32) == 0xFFFFFFFFu; }
 
 // Shared memory an update of a batch padded to n2 entries needs: keys, then values.
 __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
@@ -139,7 +142,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     bool unsorted = false;
     unsigned long long my_key = kPrbInvalidKey;      // the key of entry `rank` (one-key-per-thread case)
     for (uint32_t b = rank; b < n2; b += nt) {
-        unsigned long long key = kPrbInvalidKey;
+        unsigned long long key = 0xFFFFFFFF00000000ull | b;
         if (b < B) {
             const bool mine = pre.has_update && b == rank;
             const int32_t i = mine ? pre.idx : idx[b];
@@ -167,7 +170,20 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     for (uint32_t b = rank; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
     unsorted = team.sync_or(unsorted);
 
-    if (unsorted && n2 <= nt) {
+    if (unsorted && n2 <= nt && n2 <= 512) {
+        // a small batch is sorted by counting: the keys are all different, so the number of keys
+        // below a key is its place (every thread reads the same key at a time: one broadcast per step,
+        // no barrier between steps, against the dozens of dependent stages of a sorting network)
+        const unsigned long long key = my_key;
+        uint32_t place = 0;
+        if (rank < n2) {
+#pragma unroll 8
+            for (uint32_t j = 0; j < n2; ++j) place += (keys[j] < key) ? 1u : 0u;
+        }
+        team.sync();
+        if (rank < n2) keys[place] = key;
+        team.sync();
+    } else if (unsorted && n2 <= nt) {
         // bitonic sort, one key per thread: exchanges across fewer than 32 positions are warp shuffles
         unsigned long long key = (rank < n2) ? my_key : kPrbInvalidKey;
         for (uint32_t k = 2; k <= n2; k <<= 1) {
@@ -208,7 +224,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     float* leaves = v.level[v.depth];
     for (uint32_t s = rank; s < n2; s += nt) {
         const unsigned long long key = keys[s];
-        if (key == kPrbInvalidKey || !team.takes(s)) continue;
+        if (prb_key_invalid(key) || !team.takes(s)) continue;
         const uint32_t i = (uint32_t)(key >> 32);
         const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
         const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;     // distance from the cursor along the ring
@@ -243,7 +259,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         float* par = v.level[l];
         for (uint32_t s = rank; s < n2; s += nt) {
             const unsigned long long key = keys[s];
-            if (key == kPrbInvalidKey || !team.takes(s)) continue;
+            if (prb_key_invalid(key) || !team.takes(s)) continue;
             const uint32_t a = (uint32_t)(key >> 32) >> sh;
             const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
             if (first) par[a] = prb_sum_children_dyn(child + (uint64_t)a * K, K);
