@@ -182,6 +182,15 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
     while ((1u << v.log2_fanout) < fanout) ++v.log2_fanout;
     v.depth = L.depth;
     v.max_batch = max_batch;
+    // the levels that fit a CTA's staging area (the leaves are never staged)
+    v.top_levels = 0;
+    v.top_floats = 0;
+    for (uint32_t l = 1; l < L.depth; ++l) {
+        const uint64_t end = (uint64_t)(v.level[l] - v.level[1]) + v.level_alloc[l];
+        if (end > kPrbTopFloats) break;
+        v.top_levels = l;
+        v.top_floats = (uint32_t)((end + 3) / 4 * 4);
+    }
     *out = h;
     return PEARL_OK;
 }

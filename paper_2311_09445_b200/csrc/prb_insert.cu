@@ -114,10 +114,14 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
     const uint32_t tid = threadIdx.x;
     if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; s_maxp = v.state->max_prio_bits; }
     // the tree CTA fetches its first inputs now, while the cursor is on its way
+    // (and starts the copy of the tree's top into shared memory, behind the update's keys)
     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
+    PrbTop top;
     if (blockIdx.x == 0 && tid < kWorkers) {
         if (tid < upd.B) { pre.has_update = true; pre.idx = upd.idx[tid]; pre.val = upd.val[tid]; }
         if (tid < n && prio != nullptr) { pre.has_prio = true; pre.prio = prio[tid]; }
+        if (v.top_levels) top.mem = reinterpret_cast<float*>(s_dyn + (upd.B ? prb_update_smem_bytes(upd.n2) : 0));
+        prb_top_begin(v, top, tid, kWorkers);
     }
     __syncthreads();
     const uint64_t cursor = s_cursor;
@@ -128,9 +132,9 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
             if (upd.B)      // update and insertion share one re-sum pass per level
-                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre);
+                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top);
             else
-                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp);
+                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp, top);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
@@ -226,8 +230,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     const int sm_count = prb_sm_count();
     const int dev = prb_current_device();
     FusedUpdate upd;
-    upd.B = upd_B; upd.n2 = 2; upd.idx = upd_idx; upd.val = upd_val; upd.raw = upd_raw; upd.alpha = alpha; upd.eps = eps;
-    while (upd.n2 < upd_B) upd.n2 <<= 1;
+    upd.B = upd_B; upd.n2 = prb_update_n2(upd_B); upd.idx = upd_idx; upd.val = upd_val; upd.raw = upd_raw; upd.alpha = alpha; upd.eps = eps;
 
     InsertPlan plan;
     uint32_t tiles = 0, tasks = 0, stage = 0;
@@ -265,14 +268,15 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     const uint32_t upd_smem = upd.B ? (uint32_t)prb_update_smem_bytes(upd.n2) : 0u;
     if (tasks == 0) {
         static bool big_smem[kPrbMaxDevices];
-        if (upd_smem + 64 > 48 * 1024 && !big_smem[dev]) {
-            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
+        if (!big_smem[dev]) {
+            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float))) != cudaSuccess)
                 return -1;
             big_smem[dev] = true;
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem, s>>>(v, n, src, d_prio, plan, upd);
+        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem + v.top_floats * (uint32_t)sizeof(float), s>>>(v, n, src, d_prio, plan, upd);
     } else {
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;

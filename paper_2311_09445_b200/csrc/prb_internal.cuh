@@ -35,6 +35,10 @@ struct PrbView {
     uint32_t log2_fanout;
     uint32_t depth;                   // D
     uint32_t max_batch;
+    // levels 1 .. top_levels (< depth; 0: none) lie in the first top_floats entries from the start of
+    // level 1: the part of the tree a CTA may stage in shared memory (at most kPrbTopFloats entries)
+    uint32_t top_levels;
+    uint32_t top_floats;
 };
 
 // Dense caller-side batch, one pointer per field (NULL = field skipped).
@@ -58,6 +62,7 @@ int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx
 // Per-device facts the launchers cache: SM count, and which kernels already have their large
 // dynamic shared memory enabled (the attribute is per device).  One slot per device ordinal.
 constexpr int kPrbMaxDevices = 64;
+constexpr uint32_t kPrbTopFloats = 5120;     // 20 KB of shared memory
 inline int prb_current_device()
 {
     int dev = 0;

@@ -50,6 +50,84 @@ struct PrbTeam {
     }
 };
 
+// The top of the tree staged in shared memory for the re-sum passes: levels 1 .. v.top_levels as
+// they lie in global memory from the start of level 1 (v.top_floats entries).  Below the staged
+// levels a pass re-sums only the parents that the batch reaches; a re-summed parent of the deepest
+// staged level is written to the staged copy as well, and the levels above it are then re-summed
+// whole from shared memory (every parent always equals the sum of its children, so a parent none of
+// whose children changed comes out as it was): no sorted keys, no round trip through L2.
+// mem == nullptr: nothing is staged and every pass goes through global memory.
+struct PrbTop {
+    float* mem = nullptr;
+};
+__device__ __forceinline__ uint32_t prb_top_levels(const PrbView& v, const PrbTop& top) { return top.mem ? v.top_levels : 0u; }
+
+// Starts the copy of the staged levels (asynchronous 16-byte copies, `nthreads` threads share them);
+// prb_top_wait() by the same threads, then a barrier, before the first use.
+__device__ __forceinline__ void prb_top_begin(const PrbView& v, const PrbTop& top, uint32_t rank, uint32_t nthreads)
+{
+    if (top.mem == nullptr) return;
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(top.mem);
+    const float* src = v.level[1];
+    for (uint32_t q = rank; q < v.top_floats / 4u; q += nthreads)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + q * 16u), "l"(src + q * 4u) : "memory");
+}
+__device__ __forceinline__ void prb_top_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Re-sums parent `a` of level l >= T (T = staged levels) from its K children in global memory, left
+// to right in binary32.  A parent of level T >= 1 also goes to the staged copy: in a cluster
+// (team.parts > 1) the one of CTA 0, through distributed shared memory; the cluster barrier that
+// ends the pass makes it visible there.
+__device__ __forceinline__ void prb_resum(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T, uint32_t l, uint64_t a)
+{
+    const uint32_t K = v.fanout;
+    const float x = prb_sum_children_dyn(v.level[l + 1] + a * K, K);
+    v.level[l][a] = x;
+    if (l == T && l >= 1) {
+        float* t = top.mem + (v.level[l] - v.level[1]) + a;
+        if (team.parts == 1) {
+            *t = x;
+        } else {
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(t)), "r"(0u));
+            asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(x) : "memory");
+        }
+    }
+}
+
+// The passes over the staged levels, by one CTA: parents of level T-1, then T-2, ... then the root,
+// each level whole; a parent that comes out different is stored, staged copy and global memory.
+__device__ __forceinline__ void prb_top_passes(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T)
+{
+    const uint32_t K = v.fanout, lg = v.log2_fanout;
+    for (int l = (int)T - 1; l >= 0; --l) {
+        const uint32_t n_l = (uint32_t)((v.capacity - 1) >> (lg * (v.depth - (uint32_t)l))) + 1u;    // nodes of level l
+        const float* child = top.mem + (v.level[l + 1] - v.level[1]);
+        float* own = top.mem + (v.level[l] - v.level[1]);       // (not used for the root)
+        for (uint32_t i = team.rank; i < n_l; i += team.size) {
+            const float* c = child + (size_t)i * K;
+            float x;
+            if (K == 2) {
+                x = __fadd_rn(c[0], c[1]);
+            } else {
+                const float4 f = *reinterpret_cast<const float4*>(c);
+                x = __fadd_rn(__fadd_rn(__fadd_rn(f.x, f.y), f.z), f.w);
+                for (uint32_t q = 1; q < K / 4u; ++q) {
+                    const float4 u = reinterpret_cast<const float4*>(c)[q];
+                    x = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(x, u.x), u.y), u.z), u.w);
+                }
+            }
+            if (l == 0) {
+                v.level[0][0] = x;
+            } else if (__float_as_uint(x) != __float_as_uint(own[i])) {
+                own[i] = x;
+                v.level[l][i] = x;
+            }
+        }
+        if (l) team.sync();
+    }
+}
+
 // p = (|delta| + eps)^alpha from IEEE basic operations only (binary64, every operation rounded
 // once, no fused multiply-add), so that a CPU restatement reproduces it bit for bit:
 //   y = |delta| + eps (binary32);  y = m 2^E, m in (sqrt(1/2), sqrt(2)];  t = (m-1)/(m+1);
@@ -101,10 +179,87 @@ __device__ __forceinline__ bool prb_priority_pow(float delta, float eps, float a
     return true;
 }
 
-// A skipped entry keeps its batch position under an index of all ones: such keys sort last and, like
-// the valid ones, are all different.
+// Sort keys are (index, batch position) packed into one word, the index in the high bits: all
+// different.  A skipped entry keeps its position under an index field of all ones and sorts last.
 constexpr unsigned long long kPrbInvalidKey = ~0ull;
 __device__ __forceinline__ bool prb_key_invalid(unsigned long long key) { return (uint32_t)(key >> 32) == 0xFFFFFFFFu; }
+
+// One key per thread (threads rank < n2, whole warps): sorts them and returns the key of place
+// `rank`; keys[] holds the sorted order afterwards.  Every warp sorts its 32 keys with a bitonic
+// network of shuffles; a key's place in the whole is its place in its own run plus, for every other
+// run, the number of keys below it there -- a six-step binary search each, independent of one another.
+template <typename KeyT>
+__device__ __forceinline__ KeyT prb_sort_one_per_thread(const PrbTeam& team, KeyT key, KeyT* keys, uint32_t n2)
+{
+    const uint32_t rank = team.rank, lane = rank & 31u, run = rank >> 5;
+    const bool active = rank < n2;
+    if (active) {
+        for (uint32_t k = 2; k <= 32; k <<= 1) {
+            for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+                const KeyT other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
+                const bool keep_min = ((lane & k) == 0) == ((lane & j) == 0);
+                key = keep_min ? (key < other ? key : other) : (key > other ? key : other);
+            }
+        }
+        keys[rank] = key;
+    }
+    team.sync();
+    uint32_t place = lane;
+    if (active) {
+        const uint32_t runs = n2 >> 5;
+#pragma unroll 4
+        for (uint32_t r = 0; r < runs; ++r) {
+            const KeyT* other = keys + (r << 5);
+            uint32_t below = 0;
+#pragma unroll
+            for (uint32_t step = 16; step > 0; step >>= 1)
+                if (other[below + step - 1] < key) below += step;
+            below += (other[below] < key) ? 1u : 0u;
+            place += (r == run) ? 0u : below;
+        }
+    }
+    team.sync();
+    if (active) keys[place] = key;
+    team.sync();
+    return active ? keys[rank] : key;
+}
+
+// What one thread knows of the sorted batch when every thread holds one entry: the index and batch
+// position at its place, and the indices at the places before and after (0xFFFFFFFF: skipped entry,
+// or no such place -- no valid index equals it, nor any of its ancestors' numbers).
+struct PrbSlot {
+    uint32_t idx, pos, prev, next;
+};
+template <typename KeyT>
+__device__ __forceinline__ PrbSlot prb_sorted_slot(const PrbTeam& team, bool valid, uint32_t i, uint32_t n2, uint32_t shift, KeyT* keys)
+{
+    const uint32_t rank = team.rank;
+    const KeyT none = (KeyT)(~(KeyT)0) >> shift;          // index field of all ones
+    KeyT key = ((valid ? (KeyT)i : none) << shift) | (KeyT)rank;
+    if (rank < n2) keys[rank] = key;
+    team.sync();
+    // indices that come straight from a stratified sample are already in order; sort only if needed
+    bool unsorted = (rank + 1 < n2) && keys[rank] > keys[rank + 1];
+    unsorted = team.sync_or(unsorted);
+    if (unsorted) key = prb_sort_one_per_thread<KeyT>(team, key, keys, n2);
+    PrbSlot out = PrbSlot{0xFFFFFFFFu, 0u, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    if (rank < n2) {
+        const KeyT f = key >> shift;
+        if (f != none) out.idx = (uint32_t)f;
+        out.pos = (uint32_t)(key & (((KeyT)1 << shift) - 1));
+        if (rank > 0) { const KeyT g = keys[rank - 1] >> shift; if (g != none) out.prev = (uint32_t)g; }
+        if (rank + 1 < n2) { const KeyT g = keys[rank + 1] >> shift; if (g != none) out.next = (uint32_t)g; }
+    }
+    return out;
+}
+
+// A batch of B entries is padded to n2 = the smallest power of two >= max(B, 32): whole warps.
+__host__ __device__ inline uint32_t prb_update_n2(uint32_t B)
+{
+    uint32_t n2 = 32;
+    while (n2 < B) n2 <<= 1;
+    return n2;
+}
 
 // Shared memory an update of a batch padded to n2 entries needs: keys, then values.
 __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
@@ -117,7 +272,7 @@ __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
 // run of equal indices wins and writes its leaf; then, level by level from the deepest, the
 // first entry of every run of equal ancestors re-sums that ancestor from its children in
 // left-to-right order.  Sorted order survives dropping low digits of the index, so no list is
-// compacted and no lock is taken.  n2 = B rounded up to a power of two (>= 2); smem holds
+// compacted and no lock is taken.  n2 = prb_update_n2(B); smem holds
 // prb_update_smem_bytes(n2) bytes; fill = the fill count before this launch (indices must be below it).
 // With stale > 0 (and n == 0) entries that name one of the `stale` ring slots before `cursor` are
 // skipped: they were overwritten after they had been sampled.
@@ -131,16 +286,19 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
                                                 float alpha, float eps, unsigned long long fill, unsigned char* smem,
                                                 uint32_t n = 0, const float* __restrict__ prio = nullptr,
                                                 uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
-                                                uint32_t stale = 0)
+                                                uint32_t stale = 0, PrbTop top = PrbTop{})
 {
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
     const uint32_t rank = team.rank, nt = team.size;
+    const bool one_each = n2 <= nt;        // every thread holds one entry, in registers from the sort on
+    const uint64_t N = v.capacity;
 
+    // transform and validate; vals[b] = the priority entry b would write
     unsigned flags = 0;
     float wmax = 0.0f;                 // largest priority this thread accepted
-    bool unsorted = false;
-    unsigned long long my_key = kPrbInvalidKey;      // the key of entry `rank` (one-key-per-thread case)
+    bool my_valid = false;
+    uint32_t my_idx = 0;
     for (uint32_t b = rank; b < n2; b += nt) {
         unsigned long long key = 0xFFFFFFFF00000000ull | b;
         if (b < B) {
@@ -152,83 +310,64 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             if (raw) { p = x; ok_p = prb_valid_priority(p); }
             else ok_p = prb_priority_pow(x, eps, alpha, p);
             // stale: one of the `stale` slots written most recently, i.e. overwritten since it was sampled
-            const uint64_t back = (i >= 0 && stale) ? (cursor + v.capacity - 1 - (uint64_t)i) % v.capacity : ~0ull;
+            const uint64_t back = (i >= 0 && stale) ? (cursor + N - 1 - (uint64_t)i) % N : ~0ull;
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
             else if (back < stale) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
-            else { key = ((unsigned long long)(uint32_t)i << 32) | b; wmax = fmaxf(wmax, p); }
+            else { key = ((unsigned long long)(uint32_t)i << 32) | b; wmax = fmaxf(wmax, p); my_valid = true; my_idx = (uint32_t)i; }
             vals[b] = p;
         }
-        keys[b] = key;
-        my_key = key;
+        if (!one_each) keys[b] = key;
     }
     if (flags && team.part == 0) atomicOr(&v.state->status, flags);
     prb_note_priorities(v.state, wmax, team.part == 0);
-    team.sync();
+    prb_top_wait();                // (the staged top of the tree, if the kernel started a copy)
 
-    // Indices that come straight from a stratified sample are already in order; sort only if needed.
-    for (uint32_t b = rank; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
-    unsorted = team.sync_or(unsorted);
-
-    if (unsorted && n2 <= nt && n2 <= 512) {
-        // a small batch is sorted by counting: the keys are all different, so the number of keys
-        // below a key is its place (every thread reads the same key at a time: one broadcast per step,
-        // no barrier between steps, against the dozens of dependent stages of a sorting network)
-        const unsigned long long key = my_key;
-        uint32_t place = 0;
-        if (rank < n2) {
-#pragma unroll 8
-            for (uint32_t j = 0; j < n2; ++j) place += (keys[j] < key) ? 1u : 0u;
-        }
+    PrbSlot slot = PrbSlot{0xFFFFFFFFu, 0u, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    if (one_each) {
+        // index and position share a 32-bit key when they fit: half the shuffles and comparisons
+        const uint32_t pb = 31u - (uint32_t)__clz(n2);
+        if (N < (1ull << (32u - pb)))
+            slot = prb_sorted_slot<uint32_t>(team, my_valid, my_idx, n2, pb, reinterpret_cast<uint32_t*>(smem));
+        else
+            slot = prb_sorted_slot<unsigned long long>(team, my_valid, my_idx, n2, 32u, keys);
+    } else {
         team.sync();
-        if (rank < n2) keys[place] = key;
-        team.sync();
-    } else if (unsorted && n2 <= nt) {
-        // bitonic sort, one key per thread: exchanges across fewer than 32 positions are warp shuffles
-        unsigned long long key = (rank < n2) ? my_key : kPrbInvalidKey;
-        for (uint32_t k = 2; k <= n2; k <<= 1) {
-            for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-                unsigned long long other;
-                if (j >= 32) {
-                    if (rank < n2) keys[rank] = key;
+        bool unsorted = false;
+        for (uint32_t b = rank; b + 1 < n2; b += nt) unsorted |= (keys[b] > keys[b + 1]);
+        if (team.sync_or(unsorted)) {
+            // bitonic sort in shared memory, several keys per thread
+            for (uint32_t k = 2; k <= n2; k <<= 1) {
+                for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+                    for (uint32_t t = rank; t < (n2 >> 1); t += nt) {
+                        const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
+                        const uint32_t hi = lo | j;
+                        const unsigned long long a = keys[lo], c = keys[hi];
+                        const bool up = (lo & k) == 0;
+                        if ((a > c) == up) { keys[lo] = c; keys[hi] = a; }
+                    }
                     team.sync();
-                    other = (rank < n2) ? keys[rank ^ j] : kPrbInvalidKey;
-                    team.sync();
-                } else {
-                    other = __shfl_xor_sync(0xFFFFFFFFu, key, j);
                 }
-                const bool keep_min = ((rank & k) == 0) == ((rank & j) == 0);
-                key = keep_min ? (key < other ? key : other) : (key > other ? key : other);
-            }
-        }
-        if (rank < n2) keys[rank] = key;
-        team.sync();
-    } else if (unsorted) {
-        // bitonic sort in shared memory, several keys per thread
-        for (uint32_t k = 2; k <= n2; k <<= 1) {
-            for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-                for (uint32_t t = rank; t < (n2 >> 1); t += nt) {
-                    const uint32_t lo = ((t & ~(j - 1)) << 1) | (t & (j - 1));   // element with bit j clear
-                    const uint32_t hi = lo | j;
-                    const unsigned long long a = keys[lo], c = keys[hi];
-                    const bool up = (lo & k) == 0;
-                    if ((a > c) == up) { keys[lo] = c; keys[hi] = a; }
-                }
-                team.sync();
             }
         }
     }
 
     // winners write the leaves (unless the insertion overwrites the slot anyway), then the inserted leaves
-    const uint64_t N = v.capacity;
     float* leaves = v.level[v.depth];
-    for (uint32_t s = rank; s < n2; s += nt) {
-        const unsigned long long key = keys[s];
-        if (prb_key_invalid(key) || !team.takes(s)) continue;
-        const uint32_t i = (uint32_t)(key >> 32);
-        const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
-        const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;     // distance from the cursor along the ring
-        if (last && !(ahead < n)) leaves[i] = vals[(uint32_t)key];
+    if (one_each) {
+        if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
+            const uint64_t ahead = slot.idx >= cursor ? slot.idx - cursor : slot.idx + N - cursor;   // distance from the cursor along the ring
+            if (!(ahead < n)) leaves[slot.idx] = vals[slot.pos];
+        }
+    } else {
+        for (uint32_t s = rank; s < n2; s += nt) {
+            const unsigned long long key = keys[s];
+            if (prb_key_invalid(key) || !team.takes(s)) continue;
+            const uint32_t i = (uint32_t)(key >> 32);
+            const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
+            const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;
+            if (last && !(ahead < n)) leaves[i] = vals[(uint32_t)key];
+        }
     }
     bool bad = false;
     float imax = 0.0f;
@@ -236,33 +375,37 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     const float dflt = (n && prio == nullptr) ? prb_default_priority(__ldcg(&v.state->max_prio_bits)) : 0.0f;
     for (uint32_t t = rank; t < n; t += nt) {
         if (!team.takes(t)) continue;
-        uint64_t slot = cursor + t;
-        if (slot >= N) slot -= N;
+        uint64_t at = cursor + t;
+        if (at >= N) at -= N;
         float p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
         else imax = fmaxf(imax, p);
-        leaves[slot] = p;
+        leaves[at] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     if (n) prb_note_priorities(v.state, imax, team.part == 0);      // (a first default insertion writes 1)
     team.phase_sync();
 
-    // re-sum the ancestors, deepest level first; the insertion dirties parent range A = [a0, a1] >> sh
-    // and, if the ring wrapped, B = [0, b1] >> sh
-    const uint32_t K = v.fanout, lg = v.log2_fanout;
+    // re-sum the ancestors below the staged levels, deepest level first: the first entry of every run
+    // of equal ancestors does it; the insertion dirties parent range A = [a0, a1] >> sh and, if the
+    // ring wrapped, B = [0, b1] >> sh
+    const uint32_t lg = v.log2_fanout, T = prb_top_levels(v, top);
     const uint64_t a0 = cursor, a1 = (n ? min(cursor + n, N) : cursor + 1) - 1;
     const bool wrapped = cursor + n > N;
     const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
-    for (int l = (int)v.depth - 1; l >= 0; --l) {
-        const uint32_t sh = lg * (v.depth - (uint32_t)l);
-        const float* child = v.level[l + 1];
-        float* par = v.level[l];
-        for (uint32_t s = rank; s < n2; s += nt) {
-            const unsigned long long key = keys[s];
-            if (prb_key_invalid(key) || !team.takes(s)) continue;
-            const uint32_t a = (uint32_t)(key >> 32) >> sh;
-            const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
-            if (first) par[a] = prb_sum_children_dyn(child + (uint64_t)a * K, K);
+    for (int l = (int)v.depth - 1; l >= (int)T; --l) {
+        const uint32_t sh = min(lg * (v.depth - (uint32_t)l), 31u);      // (indices are below 2^31)
+        if (one_each) {
+            const uint32_t a = slot.idx >> sh;
+            if (slot.idx != 0xFFFFFFFFu && (slot.prev >> sh) != a && team.takes(rank)) prb_resum(v, top, team, T, (uint32_t)l, a);
+        } else {
+            for (uint32_t s = rank; s < n2; s += nt) {
+                const unsigned long long key = keys[s];
+                if (prb_key_invalid(key) || !team.takes(s)) continue;
+                const uint32_t a = (uint32_t)(key >> 32) >> sh;
+                const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
+                if (first) prb_resum(v, top, team, T, (uint32_t)l, a);
+            }
         }
         if (n) {
             const uint64_t pa0 = a0 >> sh, cntA = (a1 >> sh) - pa0 + 1;
@@ -270,12 +413,13 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             if (wrapped) cntB = (pa0 == 0) ? 0 : min(b1 >> sh, pa0 - 1) + 1;     // parents of B not already in A
             for (uint64_t i = rank; i < cntA + cntB; i += nt) {
                 if (!team.takes((uint32_t)i)) continue;
-                const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
-                par[j] = prb_sum_children_dyn(child + j * K, K);
+                prb_resum(v, top, team, T, (uint32_t)l, (i < cntA) ? pa0 + i : i - cntA);
             }
         }
         team.phase_sync();
     }
+    // the staged levels: CTA 0 alone
+    if (team.part == 0) prb_top_passes(v, top, team, T);
 }
 
 // Tree part of an insertion by one team: write the n leaves of ring slots cursor .. cursor+n-1
@@ -284,10 +428,10 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
 __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const PrbTeam& team, uint32_t n,
                                                      const float* __restrict__ prio, uint64_t cursor,
                                                      PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
-                                                     unsigned max_bits = 0)
+                                                     unsigned max_bits = 0, PrbTop top = PrbTop{})
 {
     const uint64_t N = v.capacity;
-    const uint32_t D = v.depth, K = v.fanout, lg = v.log2_fanout;
+    const uint32_t D = v.depth, lg = v.log2_fanout, T = prb_top_levels(v, top);
     float* leaves = v.level[D];
     bool bad = false;
     float imax = 0.0f;
@@ -302,13 +446,14 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     prb_note_priorities(v.state, imax, true);                       // (a first default insertion writes 1)
+    prb_top_wait();
     team.sync();
     // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;
     const uint64_t a1 = min(cursor + n, N) - 1;
     const bool wrapped = cursor + n > N;
     const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
-    for (int l = (int)D - 1; l >= 0; --l) {
+    for (int l = (int)D - 1; l >= (int)T; --l) {
         const uint32_t sh = lg * (D - (uint32_t)l);
         const uint64_t pa0 = a0 >> sh, pa1 = a1 >> sh;
         const uint64_t cntA = pa1 - pa0 + 1;
@@ -317,14 +462,11 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
             const uint64_t pb1 = b1 >> sh;
             cntB = (pa0 == 0) ? 0 : min(pb1, pa0 - 1) + 1;   // parents of B not already in A
         }
-        const float* child = v.level[l + 1];
-        float* par = v.level[l];
-        for (uint64_t i = team.rank; i < cntA + cntB; i += team.size) {
-            const uint64_t j = (i < cntA) ? pa0 + i : i - cntA;
-            par[j] = prb_sum_children_dyn(child + j * K, K);
-        }
+        for (uint64_t i = team.rank; i < cntA + cntB; i += team.size)
+            prb_resum(v, top, team, T, (uint32_t)l, (i < cntA) ? pa0 + i : i - cntA);
         team.sync();
     }
+    prb_top_passes(v, top, team, T);
 }
 
 #endif  // __CUDACC__

@@ -3,8 +3,9 @@
 // mutex; here the leaf is SET and the ancestors are re-summed, so the result does not depend
 // on scheduling (see prb_update_team in prb_tree.cuh for the steps).
 //
-// One CTA, or eight CTAs of one thread-block cluster that share every level: the batch is at most
-// a few thousand entries and the work is a chain of dependent L2 round trips, one per level.
+// One CTA, or eight CTAs of one thread-block cluster that share the deep levels: the batch is at most
+// a few thousand entries and the work is a chain of dependent L2 round trips, one per level below
+// the top of the tree, which is staged in shared memory.
 #include "prb_tree.cuh"
 
 namespace {
@@ -20,8 +21,11 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     team.whole_cta = true;
     team.part = blockIdx.x;          // CTAs of one cluster share the work (one CTA: the whole of it)
     team.parts = gridDim.x;
+    PrbTop top;
+    if (v.top_levels) top.mem = reinterpret_cast<float*>(smem + prb_update_smem_bytes(n2));
+    if (team.part == 0) prb_top_begin(v, top, team.rank, team.size);
     prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, v.state->fill, smem, 0, nullptr,
-                    stale ? v.state->cursor : 0ull, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale);
+                    stale ? v.state->cursor : 0ull, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale, top);
 }
 
 
@@ -48,13 +52,20 @@ int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale)
 {
+    static bool big_smem[kPrbMaxDevices];
+    const int dev = prb_current_device();
+    if (!big_smem[dev]) {
+        if (cudaFuncSetAttribute(prb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float))) != cudaSuccess)
+            return -1;
+        big_smem[dev] = true;
+    }
     // A batch beyond one CTA's reach goes sub-batch by sub-batch in batch order: every launch leaves
     // a consistent tree and later entries overwrite earlier ones, as in the whole batch.
     int launches = 0;
     for (uint32_t first = 0; first < B; first += PEARL_UPDATE_SUBBATCH) {
         const uint32_t b = B - first < PEARL_UPDATE_SUBBATCH ? B - first : PEARL_UPDATE_SUBBATCH;
-        uint32_t n2 = 2;
-        while (n2 < b) n2 <<= 1;
+        const uint32_t n2 = prb_update_n2(b);
         const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
         // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
         // one SM keeps in flight: then eight CTAs of one cluster share each level.
@@ -62,7 +73,7 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(ctas);
         cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2);
+        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2) + v.top_floats * sizeof(float);
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
