@@ -82,6 +82,17 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
 
 }  // namespace
 
+namespace {
+void destroy_fork(PrbFork& f)
+{
+    if (f.fork) cudaEventDestroy(f.fork);
+    if (f.join) cudaEventDestroy(f.join);
+    if (f.side) cudaStreamDestroy(f.side);
+    f = PrbFork{nullptr, nullptr, nullptr};
+    cudaGetLastError();
+}
+}  // namespace
+
 struct pearl_prb {
     Layout lay;
     PrbView view;
@@ -91,6 +102,8 @@ struct pearl_prb {
     cudaStream_t stream;
     uint32_t max_batch;
     uint64_t launches;
+    PrbFork fork = PrbFork{nullptr, nullptr, nullptr};   // side stream and events of pearl_prb_update_insert with long rows
+    ~pearl_prb() { destroy_fork(fork); }
 };
 
 namespace {
@@ -148,6 +161,12 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
     h->stream = (cudaStream_t)cuda_stream;
     h->max_batch = max_batch;
     h->launches = 0;
+    if (cudaStreamCreateWithFlags(&h->fork.side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->fork.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->fork.join, cudaEventDisableTiming) != cudaSuccess) {
+        delete h;
+        return PEARL_ERR_CUDA;
+    }
     if (slab) {
         if (slab_bytes < L.total || ((uintptr_t)slab & (kAlign - 1))) { delete h; return slab_bytes < L.total ? PEARL_ERR_OOM : PEARL_ERR_ALIGN; }
         h->base = (unsigned char*)slab;
@@ -201,6 +220,8 @@ int pearl_prb_destroy(pearl_prb_t* h)
     DeviceGuard guard(h->device);
     int rc = PEARL_OK;
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) rc = PEARL_ERR_CUDA;
+    if (h->fork.side && cudaStreamSynchronize(h->fork.side) != cudaSuccess) rc = PEARL_ERR_CUDA;
+    destroy_fork(h->fork);
     if (h->owns_slab && cudaFree(h->base) != cudaSuccess) rc = PEARL_ERR_CUDA;
     delete h;
     return rc;
@@ -320,7 +341,7 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
-    const int k = prb_launch_insert(h->view, n, b, d_prio, h->stream, B, d_idx, d_td, 0, alpha, eps);
+    const int k = prb_launch_insert(h->view, n, b, d_prio, h->stream, B, d_idx, d_td, 0, alpha, eps, &h->fork);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
     return PEARL_OK;

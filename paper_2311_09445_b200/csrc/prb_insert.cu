@@ -35,6 +35,9 @@ struct InsertPlan {
     uint32_t chunks[PRB_NUM_FIELDS];          // chunks per row of a long-row field, else 0
     uint32_t chunk[PRB_NUM_FIELDS];           // granules per chunk
     uint32_t ring_stages, ring_stage_bytes;
+    // CTAs of a tree kernel that runs beside this one and does the insertion's tree work (0: this
+    // kernel does it); they share the cursor ticket
+    uint32_t tree_ctas;
 };
 
 // Short rows: tile `tile` of the dense batch of field f, which may span many rows.
@@ -73,25 +76,6 @@ __device__ __forceinline__ void copy_tile(const PrbView& v, const InsertPlan& pl
     }
 }
 
-// Taken by one thread per CTA once the whole CTA holds the cursor: the last CTA to get here
-// publishes the new cursor and fill count.  Nothing later in the kernel reads them, so this
-// happens while the copies are still running.
-__device__ __forceinline__ void publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill)
-{
-    // no fence: the cursor and fill reads that must precede this ticket have returned their values
-    // (they were stored to shared memory before the barrier this thread has passed)
-    const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
-    if (done == gridDim.x - 1) {
-        const uint64_t N = v.capacity;
-        uint64_t c = cursor + n;
-        if (c >= N) c -= N;
-        v.state->cursor = c;
-        fill += n;
-        v.state->fill = fill > N ? N : fill;
-        v.state->insert_ticket = 0;
-    }
-}
-
 // A priority update to run before the insertion's tree work, by the same team (B == 0: none).
 struct FusedUpdate {
     uint32_t B, n2;
@@ -126,7 +110,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
     __syncthreads();
     const uint64_t cursor = s_cursor;
     if (tid == kWorkers) {
-        publish_if_last(v, n, cursor, s_fill);
+        prb_publish_if_last(v, n, cursor, s_fill, gridDim.x);
     } else if (tid < kWorkers) {
         if (blockIdx.x == 0) {
             PrbTeam team;
@@ -147,26 +131,21 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
 
 // Long rows present.  Warp 0: lane s owns ring stage s and moves row chunks t_lo+s, t_lo+s+S, ...
 // of this CTA's range; the first loads go out before the cursor has arrived (a source address does
-// not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, after the optional update)
-// and the short-field tiles (dealt round-robin, CTA 1 first).  Thread 32+kWorkers: cursor and
-// ticket.  With an update fused in, CTA 0 moves no rows: its ring memory holds the update's keys.
+// not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, unless a tree kernel beside
+// this one does it) and the short-field tiles (dealt round-robin, CTA 1 first).  Thread
+// 32+kWorkers: cursor and ticket.
 __global__ void __launch_bounds__(kThreadsRows, 1)
 prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
-                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
-                       const __grid_constant__ FusedUpdate upd)
+                       const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
     __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
     const uint32_t tid = threadIdx.x;
     const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-    const uint32_t first_copy_cta = upd.B ? 1u : 0u;
-    const uint32_t copy_ctas = gridDim.x - first_copy_cta;
-    const bool copies = blockIdx.x >= first_copy_cta;
-    const uint32_t c = blockIdx.x - first_copy_cta;
-    const uint32_t t_lo = copies ? (uint32_t)(((uint64_t)c * n_tasks) / copy_ctas) : 0u;
-    const uint32_t t_hi = copies ? (uint32_t)(((uint64_t)(c + 1) * n_tasks) / copy_ctas) : 0u;
-    const bool ring_lane = copies && tid < plan.ring_stages;
+    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
+    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
+    const bool ring_lane = tid < plan.ring_stages;
     constexpr uint32_t kPublisher = 32 + kWorkers;
 
     // one row chunk: field, row in the batch, first granule, bytes
@@ -195,7 +174,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     const uint64_t cursor = s_cursor;
 
     if (tid == kPublisher) {
-        publish_if_last(v, n, cursor, s_fill);
+        prb_publish_if_last(v, n, cursor, s_fill, gridDim.x + plan.tree_ctas);
     } else if (ring_lane) {
         while (t < t_hi) {
             uint64_t slot = cursor + row;
@@ -212,10 +191,8 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     } else if (tid >= 32 && tid < kPublisher) {
         PrbTeam team;
         team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
-        if (blockIdx.x == 0) {
-            if (upd.B) prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_ring);
+        if (blockIdx.x == 0 && plan.tree_ctas == 0)
             prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp);
-        }
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
         for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
             copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
@@ -225,7 +202,8 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
 }  // namespace
 
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
-                      uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps)
+                      uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps,
+                      const PrbFork* fork)
 {
     const int sm_count = prb_sm_count();
     const int dev = prb_current_device();
@@ -255,11 +233,34 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     plan.first_task[PRB_NUM_FIELDS] = tasks;
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
+    plan.tree_ctas = 0;
     int launches = 1;
-    if (upd.B && (tasks > 0 || upd.B > PEARL_UPDATE_SUBBATCH)) {
-        // Long rows: measured faster as two launches.  Under the copy's memory traffic the update's
-        // chain of dependent tree reads runs at twice its idle latency and outlasts the copy.
-        // (A batch beyond one sub-batch is likewise updated by launches of its own.)
+    bool forked = false;
+    uint32_t rows_grid = 0;
+    if (tasks > 0) {
+        stage = (stage + 127u) / 128u * 128u;
+        plan.ring_stage_bytes = stage;
+        plan.ring_stages = kRingBytes / stage;
+        if (plan.ring_stages > 32) plan.ring_stages = 32;
+        rows_grid = tasks < (uint32_t)sm_count ? tasks : (uint32_t)sm_count;
+    }
+    if (upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr) {
+        // Long rows: the update and the insertion's tree work are one kernel on the side stream, the
+        // row copy another on the caller's stream; neither waits for the other (the last CTA of
+        // the two to have read the cursor publishes the new one), and the caller's stream goes on
+        // when both are done.  (In one kernel the tree's chain of dependent reads, slowed by the
+        // copy's traffic, was measured to outlast the copy by far.)
+        plan.tree_ctas = prb_update_ctas(v, upd.B);
+        if (cudaEventRecord(fork->fork, s) != cudaSuccess || cudaStreamWaitEvent(fork->side, fork->fork, 0) != cudaSuccess)
+            return -1;
+        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, fork->side, 0, n, d_prio,
+                                        rows_grid + plan.tree_ctas);
+        if (k != 1 || cudaEventRecord(fork->join, fork->side) != cudaSuccess) return -1;
+        upd.B = 0;
+        launches = 2;
+        forked = true;
+    } else if (upd.B && (tasks > 0 || upd.B > PEARL_UPDATE_SUBBATCH)) {
+        // (a batch beyond one sub-batch, or no side stream: the update goes first, in launches of its own)
         const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, s);
         if (k < 0) return -1;
         upd.B = 0;
@@ -278,11 +279,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
         prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem + v.top_floats * (uint32_t)sizeof(float), s>>>(v, n, src, d_prio, plan, upd);
     } else {
-        stage = (stage + 127u) / 128u * 128u;
-        plan.ring_stage_bytes = stage;
-        plan.ring_stages = kRingBytes / stage;
-        if (plan.ring_stages > 32) plan.ring_stages = 32;
-        const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;     // >= the update's keys (<= 48 KB)
+        const uint32_t smem = kRingBarBytes + plan.ring_stages * plan.ring_stage_bytes;
         static bool big_rows[kPrbMaxDevices];
         if (!big_rows[dev]) {
             if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -290,9 +287,8 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
                 return -1;
             big_rows[dev] = true;
         }
-        const uint32_t want = tasks + (upd.B ? 1u : 0u);           // with an update, CTA 0 moves no rows
-        const uint32_t grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
-        prb_insert_rows_kernel<<<grid, kThreadsRows, smem < upd_smem ? upd_smem : smem, s>>>(v, n, src, d_prio, plan, upd);
+        prb_insert_rows_kernel<<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
+        if (forked && cudaStreamWaitEvent(s, fork->join, 0) != cudaSuccess) return -1;
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }

@@ -46,17 +46,32 @@ struct PrbBatch {
     unsigned char* ptr[PRB_NUM_FIELDS];
 };
 
+// A second stream of the handle and the two events that fork it off the caller's stream and join it
+// again: with long rows the tree work of an update + insertion runs there, beside the row copy.
+struct PrbFork {
+    cudaStream_t side;
+    cudaEvent_t fork, join;
+};
+
 // Kernel launchers; each returns the number of kernels launched, or -1 on a launch error.
-// (upd_B > 0 runs a priority update of that batch before the insertion's tree work, in the same kernel)
+// (upd_B > 0 runs a priority update of that batch before the insertion's tree work: in the same
+// kernel for short rows; for long rows in a tree kernel of its own on fork->side, or, without a
+// fork, in launches of its own before the insertion's)
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
-                      int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f);
+                      int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f, const PrbFork* fork = nullptr);
 // (uniform != 0: uniform replay, no tree walk, all weights 1)
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s, int uniform = 0);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
+// (ins_n > 0, B within one sub-batch: the tree part of an insertion of ins_n transitions follows
+// the update in the same kernel, whose CTAs take part in the insertion's cursor ticket with the
+// CTAs of the kernel that copies the rows: ticket_total in all)
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
-                      float alpha, float eps, cudaStream_t s, uint32_t stale = 0);
+                      float alpha, float eps, cudaStream_t s, uint32_t stale = 0,
+                      uint32_t ins_n = 0, const float* ins_prio = nullptr, uint32_t ticket_total = 0);
+// CTAs of the kernel that updates a batch (or sub-batch) of b entries
+uint32_t prb_update_ctas(const PrbView& v, uint32_t b);
 int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s);
 
 // Per-device facts the launchers cache: SM count, and which kernels already have their large

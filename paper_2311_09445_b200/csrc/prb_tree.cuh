@@ -50,6 +50,27 @@ struct PrbTeam {
     }
 };
 
+// Taken by one thread per CTA of an insertion once the whole CTA holds the cursor: the last of the
+// `participants` CTAs (of one kernel, or of the two kernels that share an insertion) to get here
+// publishes the new cursor and fill count.  Nothing later in those kernels reads them, so this
+// happens while the copies are still running; no CTA waits for another.
+__device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill,
+                                                    uint32_t participants)
+{
+    // no fence: the cursor and fill reads that must precede this ticket have returned their values
+    // (they were stored to shared memory before the barrier this thread has passed)
+    const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
+    if (done == participants - 1) {
+        const uint64_t N = v.capacity;
+        uint64_t c = cursor + n;
+        if (c >= N) c -= N;
+        v.state->cursor = c;
+        fill += n;
+        v.state->fill = fill > N ? N : fill;
+        v.state->insert_ticket = 0;
+    }
+}
+
 // The top of the tree staged in shared memory for the re-sum passes: levels 1 .. v.top_levels as
 // they lie in global memory from the start of level 1 (v.top_floats entries).  Below the staged
 // levels a pass re-sums only the parents that the batch reaches; a re-summed parent of the deepest
@@ -372,6 +393,8 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     bool bad = false;
     float imax = 0.0f;
     // without priorities the new transitions take the running maximum, this update's writes included
+    // (reported by CTA 0: in a cluster the others read it after a barrier)
+    if (n && prio == nullptr && team.parts > 1) { __threadfence(); team.phase_sync(); }
     const float dflt = (n && prio == nullptr) ? prb_default_priority(__ldcg(&v.state->max_prio_bits)) : 0.0f;
     for (uint32_t t = rank; t < n; t += nt) {
         if (!team.takes(t)) continue;
@@ -383,7 +406,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         leaves[at] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
-    if (n) prb_note_priorities(v.state, imax, team.part == 0);      // (a first default insertion writes 1)
+    if (n) prb_note_priorities(v.state, imax, true);      // (every CTA of a cluster wrote leaves of its own; a first default insertion writes 1)
     team.phase_sync();
 
     // re-sum the ancestors below the staged levels, deepest level first: the first entry of every run

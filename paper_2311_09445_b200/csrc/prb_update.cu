@@ -12,9 +12,11 @@ namespace {
 
 __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
-                  const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale)
+                  const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale,
+                  uint32_t ins_n, const float* __restrict__ ins_prio, uint32_t ticket_total)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ unsigned long long s_cursor, s_fill;
     PrbTeam team;
     team.rank = threadIdx.x;
     team.size = blockDim.x;
@@ -24,11 +26,21 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     PrbTop top;
     if (v.top_levels) top.mem = reinterpret_cast<float*>(smem + prb_update_smem_bytes(n2));
     if (team.part == 0) prb_top_begin(v, top, team.rank, team.size);
-    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, v.state->fill, smem, 0, nullptr,
-                    stale ? v.state->cursor : 0ull, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale, top);
+    unsigned long long fill, cursor = 0;
+    if (ins_n) {
+        // with an insertion: cursor and fill are read once per CTA, before anything is published
+        if (threadIdx.x == 0) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
+        __syncthreads();
+        cursor = s_cursor;
+        fill = s_fill;
+        if (threadIdx.x == 0) prb_publish_if_last(v, ins_n, cursor, fill, ticket_total);
+    } else {
+        fill = v.state->fill;
+        if (stale) cursor = v.state->cursor;
+    }
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor,
+                    PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale, top);
 }
-
-
 
 // Priority retrieval: one thread per entry.
 __global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
@@ -49,9 +61,18 @@ int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
-                      float alpha, float eps, cudaStream_t s, uint32_t stale)
+uint32_t prb_update_ctas(const PrbView& v, uint32_t b)
 {
+    // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
+    // one SM keeps in flight: then eight CTAs of one cluster share each level.
+    return (v.fanout * b >= 8192u) ? 8u : 1u;
+}
+
+int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
+                      float alpha, float eps, cudaStream_t s, uint32_t stale,
+                      uint32_t ins_n, const float* ins_prio, uint32_t ticket_total)
+{
+    if (ins_n && B > PEARL_UPDATE_SUBBATCH) return -1;
     static bool big_smem[kPrbMaxDevices];
     const int dev = prb_current_device();
     if (!big_smem[dev]) {
@@ -67,9 +88,7 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         const uint32_t b = B - first < PEARL_UPDATE_SUBBATCH ? B - first : PEARL_UPDATE_SUBBATCH;
         const uint32_t n2 = prb_update_n2(b);
         const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
-        // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
-        // one SM keeps in flight: then eight CTAs of one cluster share each level.
-        const uint32_t ctas = (v.fanout * b >= 8192u) ? 8u : 1u;
+        const uint32_t ctas = prb_update_ctas(v, b);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(ctas);
         cfg.blockDim = dim3(threads);
@@ -82,7 +101,8 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale) != cudaSuccess)
+        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale,
+                               ins_n, ins_prio, ticket_total) != cudaSuccess)
             return -1;
         ++launches;
     }
