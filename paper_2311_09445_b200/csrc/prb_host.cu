@@ -208,6 +208,7 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
         const uint64_t end = (uint64_t)(v.level[l] - v.level[1]) + v.level_alloc[l];
         if (end > kPrbTopFloats) break;
         v.top_levels = l;
+        v.top_off[l] = (uint32_t)(v.level[l] - v.level[1]);
         v.top_floats = (uint32_t)((end + 3) / 4 * 4);
     }
     *out = h;

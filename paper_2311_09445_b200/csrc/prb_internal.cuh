@@ -39,6 +39,7 @@ struct PrbView {
     // level 1: the part of the tree a CTA may stage in shared memory (at most kPrbTopFloats entries)
     uint32_t top_levels;
     uint32_t top_floats;
+    uint32_t top_off[PRB_MAX_LEVELS];     // entries from the start of level 1 to the start of staged level l (l >= 1)
 };
 
 // Dense caller-side batch, one pointer per field (NULL = field skipped).

@@ -31,7 +31,9 @@ constexpr int kThreads = 256;
 constexpr int kCtasPerSm = 2;
 constexpr uint32_t kChunk = 512;             // upper bound on granules per row chunk (8 KB)
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
-constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB)
+constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB) ...
+constexpr uint32_t kTopFloats32 = 1152;      // ... at fanout 32 only levels 1 and 2 can fit: 4.5 KB
+__host__ __device__ constexpr uint32_t top_floats_of(uint32_t K) { return K == 32 ? kTopFloats32 : kTopFloats; }
 constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring of a long-row CTA (dynamic shared memory), <= 32 stages
 constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
@@ -46,6 +48,9 @@ struct SamplePlan {
     uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
     uint32_t top_vec4;                       // 16-byte units staged, from the start of level 1
     uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level from the start of level 1
+    // leaf prefetch (when the level above the leaves is read from global memory): the first pf_groups
+    // lane groups of a CTA own K*K floats each at byte pf_off of the dynamic shared memory
+    uint32_t pf_groups, pf_off;
 };
 
 // Philox4x32-10 (Salmon et al., SC'11), first output word only.
@@ -66,9 +71,13 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
     return c0;
 }
 
+// Walks one stratum's target x from the root to a leaf; lane j of the group looks after child j.
+// pf != nullptr: while the group's K nodes of the level above the leaves come from global memory,
+// the K*K leaves below them are copied to pf (asynchronously, 16 bytes at a time), so that the last
+// level costs no second round trip: its K leaves are read from there.
 template <int K>
 __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan, const float* s_top, double x,
-                                        uint32_t lane, uint32_t& leaf, float& p_leaf, unsigned& flags)
+                                        uint32_t lane, uint32_t& leaf, float& p_leaf, unsigned& flags, float* pf)
 {
     constexpr unsigned FULL = 0xFFFFFFFFu;
     const unsigned gshift = (K == 32) ? 0u : ((threadIdx.x & 31u) / K) * K;
@@ -77,8 +86,27 @@ __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan
     float c = 0.0f;
     int j = 0;
     for (uint32_t l = 1; l <= v.depth; ++l) {
-        c = (l <= plan.top_levels) ? s_top[plan.top_off[l] + (uint32_t)g * K + lane]
-                                   : __ldg(v.level[l] + g * K + lane);
+        if (l <= plan.top_levels) {
+            c = s_top[plan.top_off[l] + (uint32_t)g * K + lane];
+        } else if (pf != nullptr && l == v.depth) {
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            __syncwarp();
+            c = pf[(uint32_t)j * K + lane];
+        } else {
+            c = __ldg(v.level[l] + g * K + lane);
+            if (pf != nullptr && l + 1 == v.depth) {
+                // the leaves under this group's K nodes: K*K/4 units of 16 bytes, dealt over the K lanes
+                // (fanout 2: one unit); units past the end of the leaf level are left out
+                const float* span = v.level[v.depth] + g * (K * K);
+                const uint64_t left = v.level_alloc[v.depth] - g * (K * K);        // entries from the span's start to the end
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(pf);
+                constexpr uint32_t kUnits = K * K / 4;
+#pragma unroll
+                for (uint32_t q = lane; q < kUnits; q += K)
+                    if ((uint64_t)q * 4u < left)
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + q * 16u), "l"(span + q * 4u) : "memory");
+            }
+        }
         float acc = __shfl_sync(FULL, c, 0, K);
 #pragma unroll
         for (int i = 1; i < K; ++i) {
@@ -173,7 +201,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                   const __grid_constant__ SamplePlan plan)
 {
     constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
-    __shared__ float s_top[kTopFloats];
+    __shared__ __align__(16) float s_top[top_floats_of(K)];
     __shared__ uint32_t s_idx[R];
     __shared__ double s_wraw[R];
     __shared__ float s_p[R];
@@ -194,12 +222,13 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     {
         // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
         const float4* src = reinterpret_cast<const float4*>(v.level[1]);
-        float4 t[kTopFloats / 4 / kThreads];
+        constexpr uint32_t kPerThread = (top_floats_of(K) / 4 + kThreads - 1) / kThreads;
+        float4 t[kPerThread];
 #pragma unroll
-        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+        for (uint32_t u = 0; u < kPerThread; ++u)
             if (tid + u * kThreads < plan.top_vec4) t[u] = __ldg(src + tid + u * kThreads);
 #pragma unroll
-        for (uint32_t u = 0; u < kTopFloats / 4 / kThreads; ++u)
+        for (uint32_t u = 0; u < kPerThread; ++u)
             if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
     }
     const bool empty = (fill == 0) || (!plan.uniform && !(total32 > 0.0f));
@@ -241,7 +270,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (walks) {
                 uint32_t leaf; float p; unsigned flags = 0;
                 if (plan.uniform) { leaf = (uint32_t)(((unsigned long long)r0 * fill) >> 32); p = 1.0f; }   // floor(u * fill)
-                else descend<K>(v, plan, s_top, x, lane, leaf, p, flags);
+                else descend<K>(v, plan, s_top, x, lane, leaf, p, flags,
+                                gi < plan.pf_groups ? reinterpret_cast<float*>(s_ring + plan.pf_off) + gi * (K * K) : nullptr);
                 if (lane == 0 && gi < n_round) { s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags; }
             }
             __syncthreads();
@@ -359,12 +389,38 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
     for (uint32_t l = 1; l <= v.depth && !uniform; ++l) {
         const uint64_t off = (uint64_t)(v.level[l] - v.level[1]);
-        if (off + v.level_alloc[l] > kTopFloats) break;
+        if (off + v.level_alloc[l] > top_floats_of(v.fanout)) break;
         plan.top_off[l] = (uint32_t)off;
         plan.top_vec4 = (uint32_t)((off + v.level_alloc[l] + 3) / 4);
         plan.top_levels = l;
     }
     const uint32_t R = kThreads / v.fanout;
+    const int ki = v.log2_fanout;
+    // dynamic shared memory a CTA of this kernel may have: what the device allows less its static part
+    static uint32_t dyn_max[kPrbMaxDevices][6];
+    if (dyn_max[dev][ki] == 0) {
+        cudaFuncAttributes fa;
+        int optin = 0;
+        cudaError_t e = cudaSuccess;
+        switch (v.fanout) {
+        case 2: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<2>); break;
+        case 4: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<4>); break;
+        case 8: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<8>); break;
+        case 16: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<16>); break;
+        default: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<32>); break;
+        }
+        if (e != cudaSuccess || cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return -1;
+        const long room = (long)optin - (long)fa.sharedSizeBytes - 256;
+        if (room < (long)(kRingBarBytes + 16 * 1024)) return -1;
+        dyn_max[dev][ki] = (uint32_t)room;
+    }
+    // leaf prefetch: when the level above the leaves is not staged, every walking lane group copies
+    // the K*K leaves under its K nodes to shared memory while those nodes are on their way
+    const bool prefetch = !uniform && v.depth >= 2 && plan.top_levels < v.depth - 1;
+    const uint32_t pf_group_bytes = v.fanout * v.fanout * (uint32_t)sizeof(float);
+    plan.pf_groups = 0;
+    plan.pf_off = 0;
     uint32_t grid, smem = 0;
     plan.ring_stages = 0;
     plan.ring_stage_bytes = 0;
@@ -373,11 +429,22 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         uint32_t stage = 0;
         for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
         stage = (stage + 127u) / 128u * 128u;
-        plan.ring_stage_bytes = stage;
-        plan.ring_stages = kRingBytes / stage;
-        if (plan.ring_stages > 32) plan.ring_stages = 32;
-        smem = kRingBarBytes + plan.ring_stages * stage;
         grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
+        // strata a CTA can touch: its share of the tasks, plus one for a range that straddles
+        const uint32_t tasks_per_cta = (plan.n_tasks + grid - 1) / grid;
+        uint32_t strata = (tasks_per_cta + plan.tps - 1) / plan.tps + 1;
+        if (strata > R) strata = R;
+        uint32_t pf_bytes = prefetch ? strata * pf_group_bytes : 0u;
+        uint32_t ring_bytes = dyn_max[dev][ki] - kRingBarBytes;
+        if (pf_bytes + 8u * stage > ring_bytes) pf_bytes = 0;      // (not at the price of the ring)
+        ring_bytes -= pf_bytes;
+        if (ring_bytes > kRingBytes) ring_bytes = kRingBytes;
+        plan.ring_stage_bytes = stage;
+        plan.ring_stages = ring_bytes / stage;
+        if (plan.ring_stages > 32) plan.ring_stages = 32;
+        plan.pf_off = kRingBarBytes + plan.ring_stages * stage;
+        plan.pf_groups = pf_bytes ? strata : 0u;
+        smem = plan.pf_off + pf_bytes;
     } else {
         // a small batch is spread over more CTAs than it needs: its descents are chains of dependent
         // L2 reads, and more SMs keep more of them in flight
@@ -385,15 +452,20 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         const uint32_t per_cta = R >= 4 ? R / 4 : 1;
         const uint32_t want = (B + per_cta - 1) / per_cta;
         grid = want < one_wave ? want : one_wave;
+        if (prefetch) {
+            uint32_t strata = (B + grid - 1) / grid;
+            if (strata > R) strata = R;
+            plan.pf_groups = strata;
+            smem = strata * pf_group_bytes;
+        }
     }
     static bool big_smem[kPrbMaxDevices][6];
-    const int ki = v.log2_fanout;
     cudaError_t attr = cudaSuccess;
 #define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
     do {                                                                                                          \
         if (smem && !big_smem[dev][ki]) {                                                                              \
             attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
-                                        (int)(kRingBarBytes + kRingBytes));                                       \
+                                        (int)dyn_max[dev][ki]);                                                   \
             big_smem[dev][ki] = (attr == cudaSuccess);                                                                 \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \

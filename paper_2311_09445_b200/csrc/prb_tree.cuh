@@ -105,7 +105,7 @@ __device__ __forceinline__ void prb_resum(const PrbView& v, const PrbTop& top, c
     const float x = prb_sum_children_dyn(v.level[l + 1] + a * K, K);
     v.level[l][a] = x;
     if (l == T && l >= 1) {
-        float* t = top.mem + (v.level[l] - v.level[1]) + a;
+        float* t = top.mem + v.top_off[l] + a;
         if (team.parts == 1) {
             *t = x;
         } else {
@@ -116,28 +116,38 @@ __device__ __forceinline__ void prb_resum(const PrbView& v, const PrbTop& top, c
     }
 }
 
+// Left-to-right binary32 sum of K staged children (all loads first, then the chain of additions).
+template <int K>
+__device__ __forceinline__ float prb_sum_staged(const float* c)
+{
+    if (K == 2) {
+        const float2 f = *reinterpret_cast<const float2*>(c);
+        return __fadd_rn(f.x, f.y);
+    } else {
+        float4 u[K / 4 > 0 ? K / 4 : 1];
+#pragma unroll
+        for (int q = 0; q < K / 4; ++q) u[q] = reinterpret_cast<const float4*>(c)[q];
+        float x = __fadd_rn(__fadd_rn(__fadd_rn(u[0].x, u[0].y), u[0].z), u[0].w);
+#pragma unroll
+        for (int q = 1; q < K / 4; ++q) x = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(x, u[q].x), u[q].y), u[q].z), u[q].w);
+        return x;
+    }
+}
+
 // The passes over the staged levels, by one CTA: parents of level T-1, then T-2, ... then the root,
 // each level whole; a parent that comes out different is stored, staged copy and global memory.
-__device__ __forceinline__ void prb_top_passes(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T)
+template <int K>
+__device__ __forceinline__ void prb_top_passes_k(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T)
 {
-    const uint32_t K = v.fanout, lg = v.log2_fanout;
+    constexpr uint32_t lg = K == 2 ? 1 : K == 4 ? 2 : K == 8 ? 3 : K == 16 ? 4 : 5;
+    // nodes of level T (then of the levels above, one division by K each, rounded up)
+    uint32_t n_l = (uint32_t)((v.capacity - 1) >> (lg * (v.depth - T))) + 1u;
     for (int l = (int)T - 1; l >= 0; --l) {
-        const uint32_t n_l = (uint32_t)((v.capacity - 1) >> (lg * (v.depth - (uint32_t)l))) + 1u;    // nodes of level l
-        const float* child = top.mem + (v.level[l + 1] - v.level[1]);
-        float* own = top.mem + (v.level[l] - v.level[1]);       // (not used for the root)
+        n_l = (n_l + K - 1) >> lg;
+        const float* child = top.mem + v.top_off[l + 1];
+        float* own = top.mem + v.top_off[l];       // (not used for the root)
         for (uint32_t i = team.rank; i < n_l; i += team.size) {
-            const float* c = child + (size_t)i * K;
-            float x;
-            if (K == 2) {
-                x = __fadd_rn(c[0], c[1]);
-            } else {
-                const float4 f = *reinterpret_cast<const float4*>(c);
-                x = __fadd_rn(__fadd_rn(__fadd_rn(f.x, f.y), f.z), f.w);
-                for (uint32_t q = 1; q < K / 4u; ++q) {
-                    const float4 u = reinterpret_cast<const float4*>(c)[q];
-                    x = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(x, u.x), u.y), u.z), u.w);
-                }
-            }
+            const float x = prb_sum_staged<K>(child + (size_t)i * K);
             if (l == 0) {
                 v.level[0][0] = x;
             } else if (__float_as_uint(x) != __float_as_uint(own[i])) {
@@ -146,6 +156,16 @@ __device__ __forceinline__ void prb_top_passes(const PrbView& v, const PrbTop& t
             }
         }
         if (l) team.sync();
+    }
+}
+__device__ __forceinline__ void prb_top_passes(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T)
+{
+    switch (v.fanout) {
+    case 2: prb_top_passes_k<2>(v, top, team, T); break;
+    case 4: prb_top_passes_k<4>(v, top, team, T); break;
+    case 8: prb_top_passes_k<8>(v, top, team, T); break;
+    case 16: prb_top_passes_k<16>(v, top, team, T); break;
+    default: prb_top_passes_k<32>(v, top, team, T); break;
     }
 }
 

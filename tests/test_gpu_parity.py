@@ -342,6 +342,64 @@ def test_fused_update_insert(oracle_mod, wl, N, B, n):
     pr.close()
 
 
+@pytest.mark.parametrize("B,n", [(512, 300), (40, 512)])
+def test_fused_long_rows_replayed_as_cuda_graph(oracle_mod, B, n):
+    # Long rows: update_insert runs its tree kernel on the handle's side stream beside the row copy.
+    # Captured into a CUDA graph with a sample between the calls and replayed, it must leave what the
+    # oracle leaves after the same sequence of calls.
+    from paper_2311_09445_b200 import PrioritizedReplay
+    N = 900
+    wl = wk.scaled(wk.ATARI, N)
+    rng = np.random.default_rng(B)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(dev)
+    ora = oracle_mod.OraclePRB(N, wl.fanout, wl.obs_bytes, wl.act_bytes)
+    with torch.cuda.stream(stream):
+        gpu = PrioritizedReplay(N, wl.fanout, wl.obs_bytes, wl.act_bytes, 512, device=dev, stream=stream)
+        first = wk.transitions(wl, rng, 512, 0)
+        assert ora.insert(first["obs"], first["act"], first["rew"], first["next_obs"], first["done"], first["prio"]) == 0
+        d = wk.to_device(first, dev)
+        gpu.insert(d["obs"], d["act"], d["rew"], d["next_obs"], d["done"], d["prio"])
+        calls = []
+        for c in range(3):
+            b = wk.transitions(wl, rng, n, 512 + c * n)
+            idx = rng.integers(0, 512, size=B).astype(np.int32)          # unsorted, with duplicates
+            td = rng.standard_normal(B).astype(np.float32)
+            calls.append((b, idx, td, wk.to_device(b, dev), torch.from_numpy(idx).to(dev), torch.from_numpy(td).to(dev)))
+        out_idx = torch.zeros(64, dtype=torch.int32, device=dev)
+        out_w = torch.zeros(64, device=dev)
+
+        def sequence():
+            for b, idx, td, db, didx, dtd in calls:
+                gpu.update_insert(didx, dtd, wl.alpha, wl.eps, db["obs"], db["act"], db["rew"], db["next_obs"], db["done"], db["prio"])
+                gpu.sample(64, wl.beta, 5, out_idx, out_w)
+
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            sequence()
+        for rep in range(2):
+            graph.replay()
+            torch.cuda.synchronize()
+            for b, idx, td, *_ in calls:
+                assert ora.update(idx, td, wl.alpha, wl.eps) == 0
+                assert ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"]) == 0
+                o = ora.sample(64, wl.beta, 5, gather=False)
+            assert np.array_equal(out_idx.cpu().numpy(), o["idx"])
+            np.testing.assert_allclose(out_w.cpu().numpy(), o["w"], rtol=1e-5, atol=0)
+            for l in range(ora.depth + 1):
+                assert np.array_equal(ora.read_level(l).view(np.uint32), gpu.read_level(l).view(np.uint32)), "level %d" % l
+            assert gpu.info() == ora.info()
+        assert gpu.sync() == ora.status()
+        rows = np.arange(0, N, 7, dtype=np.int32)
+        g_rows, o_rows = gpu.read_rows(rows), ora.read_rows(rows)
+        for f in g_rows:
+            assert np.array_equal(np.ascontiguousarray(g_rows[f]).view(np.uint8).reshape(-1),
+                                  np.ascontiguousarray(o_rows[f]).view(np.uint8).reshape(-1)), f
+    gpu.close()
+    ora.close()
+
+
 @pytest.mark.parametrize("wl", [wk.CARTPOLE, wk.ATARI])
 def test_fused_update_uses_fill_before_insert(oracle_mod, wl):
     # In the fused call the update comes first: an index that only the insertion makes valid is refused.
@@ -407,8 +465,8 @@ def test_update_after_insert_and_retrieval(oracle_mod, K, N, B, n):
     pr.close()
 
 
-@pytest.mark.parametrize("wl,N", [(wk.CARTPOLE, 3000), (wk.ATARI, 600)])
-def test_default_insert_priority(oracle_mod, wl, N):
+@pytest.mark.parametrize("wl,N,B", [(wk.CARTPOLE, 3000, 128), (wk.ATARI, 600, 128), (wk.ATARI, 600, 512)])
+def test_default_insert_priority(oracle_mod, wl, N, B):
     # insertion without priorities: the running maximum of everything written so far (1 before any)
     wl = wk.scaled(wl, N)
     rng = np.random.default_rng(N)
@@ -434,8 +492,8 @@ def test_default_insert_priority(oracle_mod, wl, N):
     pr.insert(wk.transitions(wl, rng, 200, 100))  # explicit priorities raise the maximum
     pr.compare_state()
     for step in range(6):
-        o, g = pr.sample(128, 0.4, 1)
-        td = (rng.standard_normal(128) * (step + 1) * 3).astype(np.float32)
+        o, g = pr.sample(B, 0.4, 1)          # (B = 512 at fanout 32: the update's CTAs form a cluster)
+        td = (rng.standard_normal(B) * (step + 1) * 3).astype(np.float32)
         if step % 2 == 0:
             pr.update(o["idx"], td, 0.6, 1e-6)
             insert_default(77, 300 + 77 * step)
