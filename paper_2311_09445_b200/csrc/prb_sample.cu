@@ -71,29 +71,58 @@ __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1
     return c0;
 }
 
+// The K children of one node lie in shared memory at `row`: every lane of the group reads all of them
+// (the same addresses: broadcasts) and forms the left-to-right binary32 prefix sums in registers, one
+// chain of K-1 additions; lane j keeps child j and the prefix that ends with it.  (Passing the
+// children from lane to lane by shuffles instead puts a shuffle's latency into every step of the chain.)
+template <int K>
+__device__ __forceinline__ void group_prefix(const float* row, uint32_t lane, float& c, float& acc)
+{
+    if (K == 2) {
+        const float2 v = *reinterpret_cast<const float2*>(row);
+        c = lane ? v.y : v.x;
+        acc = lane ? __fadd_rn(v.x, v.y) : v.x;
+    } else {
+        float run = 0.0f;
+#pragma unroll
+        for (int q = 0; q < K / 4; ++q) {
+            const float4 v = reinterpret_cast<const float4*>(row)[q];
+            const float e[4] = { v.x, v.y, v.z, v.w };
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int i = 4 * q + t;
+                run = (i == 0) ? e[t] : __fadd_rn(run, e[t]);
+                if ((int)lane == i) { c = e[t]; acc = run; }
+            }
+        }
+    }
+}
+
 // Walks one stratum's target x from the root to a leaf; lane j of the group looks after child j.
+// s_child: K floats of shared memory of the group's own, for a level that comes from global memory.
 // pf != nullptr: while the group's K nodes of the level above the leaves come from global memory,
 // the K*K leaves below them are copied to pf (asynchronously, 16 bytes at a time), so that the last
 // level costs no second round trip: its K leaves are read from there.
 template <int K>
-__device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan, const float* s_top, double x,
+__device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan, const float* s_top, float* s_child, double x,
                                         uint32_t lane, uint32_t& leaf, float& p_leaf, unsigned& flags, float* pf)
 {
     constexpr unsigned FULL = 0xFFFFFFFFu;
     const unsigned gshift = (K == 32) ? 0u : ((threadIdx.x & 31u) / K) * K;
     const unsigned gmask = (K == 32) ? FULL : ((1u << (K & 31)) - 1u);
     uint64_t g = 0;
-    float c = 0.0f;
+    float c = 0.0f, acc = 0.0f;
     int j = 0;
     for (uint32_t l = 1; l <= v.depth; ++l) {
+        const float* row;
         if (l <= plan.top_levels) {
-            c = s_top[plan.top_off[l] + (uint32_t)g * K + lane];
+            row = s_top + plan.top_off[l] + (uint32_t)g * K;
         } else if (pf != nullptr && l == v.depth) {
             asm volatile("cp.async.wait_all;" ::: "memory");
             __syncwarp();
-            c = pf[(uint32_t)j * K + lane];
+            row = pf + (uint32_t)j * K;
         } else {
-            c = __ldg(v.level[l] + g * K + lane);
+            const float mine = __ldg(v.level[l] + g * K + lane);
             if (pf != nullptr && l + 1 == v.depth) {
                 // the leaves under this group's K nodes: K*K/4 units of 16 bytes, dealt over the K lanes
                 // (fanout 2: one unit); units past the end of the leaf level are left out
@@ -106,13 +135,12 @@ __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan
                     if ((uint64_t)q * 4u < left)
                         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + q * 16u), "l"(span + q * 4u) : "memory");
             }
+            __syncwarp();              // (the group has read what the level before left in s_child)
+            s_child[lane] = mine;
+            __syncwarp();
+            row = s_child;
         }
-        float acc = __shfl_sync(FULL, c, 0, K);
-#pragma unroll
-        for (int i = 1; i < K; ++i) {
-            const float ci = __shfl_sync(FULL, c, i, K);
-            if ((int)lane >= i) acc = __fadd_rn(acc, ci);
-        }
+        group_prefix<K>(row, lane, c, acc);
         const unsigned passed = (__ballot_sync(FULL, x >= (double)acc) >> gshift) & gmask;
         const unsigned positive = (__ballot_sync(FULL, c > 0.0f) >> gshift) & gmask;
         const int cnt = __popc(passed);
@@ -202,6 +230,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 {
     constexpr uint32_t R = kThreads / K;          // strata walked concurrently by one CTA
     __shared__ __align__(16) float s_top[top_floats_of(K)];
+    __shared__ __align__(16) float s_child[kThreads];     // K floats per lane group: a level that came from global memory
     __shared__ uint32_t s_idx[R];
     __shared__ double s_wraw[R];
     __shared__ float s_p[R];
@@ -270,7 +299,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (walks) {
                 uint32_t leaf; float p; unsigned flags = 0;
                 if (plan.uniform) { leaf = (uint32_t)(((unsigned long long)r0 * fill) >> 32); p = 1.0f; }   // floor(u * fill)
-                else descend<K>(v, plan, s_top, x, lane, leaf, p, flags,
+                else descend<K>(v, plan, s_top, s_child + (tid - lane), x, lane, leaf, p, flags,
                                 gi < plan.pf_groups ? reinterpret_cast<float*>(s_ring + plan.pf_off) + gi * (K * K) : nullptr);
                 if (lane == 0 && gi < n_round) { s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags; }
             }
