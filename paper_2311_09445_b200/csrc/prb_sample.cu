@@ -309,7 +309,11 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         // From here the CTA splits by role: threads 0..127 copy, threads 128..255 look after the weights.
         const bool last_descents = round + 1 >= n_rounds;      // true exactly once per CTA
         if (tid >= kThreads / 2) {
-            // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path)
+            // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path).
+            // What other CTAs read -- the raw weights and the batch maximum -- is written by atomics
+            // whose results are waited for: when a thread goes on, its value is in L2.  A fence here
+            // instead would also wait for the bulk copies the ring has in flight, and so put the
+            // ticket, and the normalisation of the weights behind it, after the whole copy.
             const uint32_t gi2 = tid - kThreads / 2;
             if (gi2 < n_round) {
                 double wr = 0.0;
@@ -318,7 +322,9 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
                     wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
                     out_idx[k2] = (int32_t)s_idx[gi2];
-                    v.wraw[k2] = wr;
+                    const unsigned long long before = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
+                                                                 (unsigned long long)__double_as_longlong(wr));
+                    asm volatile("" ::"l"(before) : "memory");
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
                 }
                 s_wraw[gi2] = wr;
@@ -327,18 +333,19 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (tid == kThreads / 2) {
                 double m = 0.0;
                 for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
-                if (m > 0.0) atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
+                if (m > 0.0) {
+                    const unsigned long long before = atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
+                    asm volatile("" ::"l"(before) : "memory");
+                }
                 if (last_descents) {
-                    // every descent of this CTA is done: the last CTA to get here normalises the weights
-                    // (the barrier above ordered the other threads' writes before this fence: it covers them)
-                    __threadfence();
+                    // every descent of this CTA is done and its weights are in L2: the last CTA to get
+                    // here normalises the weights of the whole batch
                     s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
                 }
             }
             if (last_descents) {
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
                 if (s_last) {
-                    __threadfence();
                     if (empty) {
                         if (tid == kThreads / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
                     } else if (out_w != nullptr) {
