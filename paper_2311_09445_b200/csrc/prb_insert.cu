@@ -143,9 +143,15 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
     const uint32_t tid = threadIdx.x;
     const uint32_t n_tasks = plan.first_task[PRB_NUM_FIELDS];
-    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * n_tasks) / gridDim.x);
-    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * n_tasks) / gridDim.x);
-    const bool ring_lane = tid < plan.ring_stages;
+    // A CTA that does the tree work moves no rows: the answers to its tree reads would queue behind
+    // the data of its own bulk loads.
+    const uint32_t first_copy_cta = (plan.tree_ctas == 0 && gridDim.x > 1) ? 1u : 0u;
+    const uint32_t copy_ctas = gridDim.x - first_copy_cta;
+    const bool copies = blockIdx.x >= first_copy_cta;
+    const uint32_t cc = blockIdx.x - first_copy_cta;
+    const uint32_t t_lo = copies ? (uint32_t)(((uint64_t)cc * n_tasks) / copy_ctas) : 0u;
+    const uint32_t t_hi = copies ? (uint32_t)(((uint64_t)(cc + 1) * n_tasks) / copy_ctas) : 0u;
+    const bool ring_lane = copies && tid < plan.ring_stages;
     constexpr uint32_t kPublisher = 32 + kWorkers;
 
     // one row chunk: field, row in the batch, first granule, bytes
@@ -242,9 +248,13 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         plan.ring_stage_bytes = stage;
         plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
-        rows_grid = tasks < (uint32_t)sm_count ? tasks : (uint32_t)sm_count;
     }
-    if (upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr) {
+    const bool fork_tree = upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr;
+    if (tasks > 0) {
+        const uint32_t want = tasks + (fork_tree ? 0u : 1u);       // (without a tree kernel, CTA 0 does the tree work and no copies)
+        rows_grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
+    }
+    if (fork_tree) {
         // Long rows: the update and the insertion's tree work are one kernel on the side stream, the
         // row copy another on the caller's stream; neither waits for the other (the last CTA of
         // the two to have read the cursor publishes the new one), and the caller's stream goes on

@@ -233,6 +233,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     __shared__ __align__(16) float s_child[kThreads];     // K floats per lane group: a level that came from global memory
     __shared__ uint32_t s_idx[R];
     __shared__ double s_wraw[R];
+    __shared__ volatile unsigned long long s_seen[R];     // answers of the atomics that publish the weights
     __shared__ float s_p[R];
     __shared__ unsigned s_flags[R];
     __shared__ unsigned int s_last;
@@ -322,9 +323,9 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
                     wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
                     out_idx[k2] = (int32_t)s_idx[gi2];
-                    const unsigned long long before = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
-                                                                 (unsigned long long)__double_as_longlong(wr));
-                    asm volatile("" ::"l"(before) : "memory");
+                    // (the old value goes to shared memory: a store that cannot issue before the atomic has answered)
+                    s_seen[gi2] = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
+                                             (unsigned long long)__double_as_longlong(wr));
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
                 }
                 s_wraw[gi2] = wr;
@@ -334,8 +335,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                 double m = 0.0;
                 for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
                 if (m > 0.0) {
-                    const unsigned long long before = atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
-                    asm volatile("" ::"l"(before) : "memory");
+                    s_seen[0] = atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
                 }
                 if (last_descents) {
                     // every descent of this CTA is done and its weights are in L2: the last CTA to get
