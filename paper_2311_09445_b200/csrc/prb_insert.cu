@@ -251,8 +251,12 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     }
     const bool fork_tree = upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr;
     if (tasks > 0) {
-        const uint32_t want = tasks + (fork_tree ? 0u : 1u);       // (without a tree kernel, CTA 0 does the tree work and no copies)
-        rows_grid = want < (uint32_t)sm_count ? want : (uint32_t)sm_count;
+        // Without a tree kernel CTA 0 does the tree work and no copies; with one, its CTAs get SMs of
+        // their own: a copy CTA takes an SM's whole shared memory and would wait for them to leave.
+        const uint32_t want = tasks + (fork_tree ? 0u : 1u);
+        uint32_t room = (uint32_t)sm_count;
+        if (fork_tree && room > 2u * prb_update_ctas(v, upd.B)) room -= prb_update_ctas(v, upd.B);
+        rows_grid = want < room ? want : room;
     }
     if (fork_tree) {
         // Long rows: the update and the insertion's tree work are one kernel on the side stream, the
