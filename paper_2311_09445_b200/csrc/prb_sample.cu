@@ -4,10 +4,12 @@
 // Priority sampling is Eq. 1 of PEARL (Section II-A) carried out as Section V-A describes it:
 // "traversing the tree performing prefix sum from root to leaf".  A group of K lanes (K = the
 // fanout) owns one stratum: lane j loads child j, so a child group is one 8..128-byte request;
-// the left-to-right binary32 prefix sums are formed by K-1 broadcast-and-add steps (the same
-// association as the stored parent), a ballot counts the prefixes the binary64 target has
-// passed, and that count is the child to enter.  The top levels of the tree (up to 20 KB) are
-// staged in shared memory at kernel start, the rest is read from L2.  The read of the sampled
+// the children are put in shared memory (the staged levels are there already), every lane reads
+// all K and forms the left-to-right binary32 prefix sums in registers (the same association as
+// the stored parent), lane j keeping prefix j; a ballot counts the prefixes the binary64 target
+// has passed, and that count is the child to enter.  The top levels of the tree (up to 20 KB) are
+// staged in shared memory at kernel start, the rest is read from L2, the leaves ahead of time
+// while the level above them is on its way.  The read of the sampled
 // rows is Listing 2's `D_storage[sampled_indices]`.  Stratification, the Philox stream and the
 // weights follow the prioritized-replay reference the paper cites (Schaul et al.).
 //
