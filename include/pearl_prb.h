@@ -163,8 +163,11 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
 /* Host-buffer forms of the three calls (the paper's host runtime exchanges requests and data
  * with the Replay Manager over PCIe, Section IV-A).  They copy their inputs to the device and
  * their outputs back on the handle's stream; sample_host returns after the stream has drained,
- * insert_host and update_host once their host buffers may be reused.  Pinned host memory makes
- * the copies asynchronous.  Output pointers of sample_host other than h_idx may be NULL. */
+ * insert_host and update_host once their host buffers may be reused.  A call whose arrays come to
+ * at most 256 KB travels packed -- the arrays are gathered in a pinned buffer of the handle and cross
+ * PCIe in one copy (insert_host and update_host then leave their work on the stream and return at
+ * once); a larger call copies array by array, asynchronously if the caller's memory is pinned, and
+ * returns when the stream has drained.  Output pointers of sample_host other than h_idx may be NULL. */
 int pearl_prb_insert_host(pearl_prb_t* prb, uint32_t n, const void* h_obs, const void* h_act,
                           const float* h_rew, const void* h_next_obs, const uint8_t* h_done,
                           const float* h_prio);

@@ -93,6 +93,8 @@ void destroy_fork(PrbFork& f)
 }
 }  // namespace
 
+constexpr uint64_t kPackBytes = 256 * 1024;
+
 struct pearl_prb {
     Layout lay;
     PrbView view;
@@ -103,7 +105,17 @@ struct pearl_prb {
     uint32_t max_batch;
     uint64_t launches;
     PrbFork fork = PrbFork{nullptr, nullptr, nullptr};   // side stream and events of pearl_prb_update_insert with long rows
-    ~pearl_prb() { destroy_fork(fork); }
+    // Small batches of the *_host calls travel packed: all arrays of a call in one pinned buffer, one
+    // copy each way (2 x kPackBytes of pinned host memory; nullptr: every array is copied by itself).
+    unsigned char* pin = nullptr;
+    cudaEvent_t pin_read = nullptr;      // the last host-to-device copy out of `pin` has been made
+    ~pearl_prb()
+    {
+        destroy_fork(fork);
+        if (pin_read) cudaEventDestroy(pin_read);
+        if (pin) cudaFreeHost(pin);
+        cudaGetLastError();
+    }
 };
 
 namespace {
@@ -166,6 +178,12 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
         cudaEventCreateWithFlags(&h->fork.join, cudaEventDisableTiming) != cudaSuccess) {
         delete h;
         return PEARL_ERR_CUDA;
+    }
+    if (cudaHostAlloc((void**)&h->pin, 2 * kPackBytes, cudaHostAllocDefault) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->pin_read, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();                 // (not fatal: the host calls then copy array by array)
+        if (h->pin) cudaFreeHost(h->pin);
+        h->pin = nullptr;
     }
     if (slab) {
         if (slab_bytes < L.total || ((uintptr_t)slab & (kAlign - 1))) { delete h; return slab_bytes < L.total ? PEARL_ERR_OOM : PEARL_ERR_ALIGN; }
@@ -350,6 +368,40 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
 
 // ---- host-buffer forms ---------------------------------------------------------------------
 
+namespace {
+
+// Offsets of up to seven arrays packed one after another, each start 16-byte aligned.
+struct Packing {
+    uint64_t off[PRB_NUM_FIELDS + 2];
+    uint64_t bytes[PRB_NUM_FIELDS + 2];
+    uint64_t total = 0;
+    void add(int slot, uint64_t nbytes)
+    {
+        off[slot] = total;
+        bytes[slot] = nbytes;
+        total = (total + nbytes + 15) / 16 * 16;
+    }
+};
+
+// Host -> pinned buffer -> device arena in one copy; dev[i] = where array i landed (nullptr if absent).
+// The pinned buffer is written only after the copy that last read it has been made.
+int pack_to_device(pearl_prb* h, const Packing& pk, const void* const* src, int count, unsigned char* arena, void** dev)
+{
+    if (cudaEventSynchronize(h->pin_read) != cudaSuccess) return PEARL_ERR_CUDA;
+    for (int i = 0; i < count; ++i) {
+        dev[i] = nullptr;
+        if (!src[i] || pk.bytes[i] == 0) continue;
+        memcpy(h->pin + pk.off[i], src[i], pk.bytes[i]);
+        dev[i] = arena + pk.off[i];
+    }
+    if (cudaMemcpyAsync(arena, h->pin, pk.total, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaEventRecord(h->pin_read, h->stream) != cudaSuccess)
+        return PEARL_ERR_CUDA;
+    return PEARL_OK;
+}
+
+}  // namespace
+
 int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const void* h_act, const float* h_rew,
                           const void* h_next_obs, const uint8_t* h_done, const float* h_prio)
 {
@@ -358,8 +410,18 @@ int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const v
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
-    const void* src[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
-    void* dev[PRB_NUM_FIELDS];
+    const void* src[PRB_NUM_FIELDS + 1] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_prio };
+    void* dev[PRB_NUM_FIELDS + 1];
+    Packing pk;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, src[f] ? (uint64_t)n * h->view.field_bytes[f] : 0);
+    pk.add(PRB_NUM_FIELDS, h_prio ? (uint64_t)n * 4 : 0);
+    if (h->pin && pk.total <= kPackBytes) {
+        // small batch: one copy; the caller's arrays are free on return, the work is left on the stream
+        int rc = pack_to_device(h, pk, src, PRB_NUM_FIELDS + 1, at(h, h->lay.off_stage_in[0]), dev);
+        if (rc != PEARL_OK) return rc;
+        return pearl_prb_insert(h, n, dev[F_OBS], dev[F_ACT], (const float*)dev[F_REW], dev[F_NEXT_OBS],
+                                (const uint8_t*)dev[F_DONE], (const float*)dev[PRB_NUM_FIELDS]);
+    }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         dev[f] = nullptr;
         const uint64_t bytes = (uint64_t)n * h->view.field_bytes[f];
@@ -373,7 +435,7 @@ int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const v
     int rc = pearl_prb_insert(h, n, dev[F_OBS], dev[F_ACT], (const float*)dev[F_REW], dev[F_NEXT_OBS],
                               (const uint8_t*)dev[F_DONE], d_prio);
     if (rc != PEARL_OK) return rc;
-    // the staging area is reused by the next host call: wait until this call's work has drained
+    // (copies from pinned memory are asynchronous: the caller's arrays are free once the stream has drained)
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }
 
@@ -384,8 +446,27 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
-    void* dst[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
-    void* dev[PRB_NUM_FIELDS];
+    void* dst[PRB_NUM_FIELDS + 2] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_idx, h_w };
+    void* dev[PRB_NUM_FIELDS + 2];
+    Packing pk;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, dst[f] ? (uint64_t)B * h->view.field_bytes[f] : 0);
+    pk.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
+    pk.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
+    if (h->pin && pk.total <= kPackBytes) {
+        // small batch: the kernel writes its outputs packed, one copy brings them to the pinned buffer
+        unsigned char* arena = at(h, h->lay.off_stage_out[0]);
+        unsigned char* pin_out = h->pin + kPackBytes;
+        for (int i = 0; i < PRB_NUM_FIELDS + 2; ++i) dev[i] = (dst[i] && pk.bytes[i]) ? arena + pk.off[i] : nullptr;
+        int rc = pearl_prb_sample(h, B, beta, seed, (int32_t*)dev[PRB_NUM_FIELDS], (float*)dev[PRB_NUM_FIELDS + 1], dev[F_OBS],
+                                  dev[F_ACT], (float*)dev[F_REW], dev[F_NEXT_OBS], (uint8_t*)dev[F_DONE]);
+        if (rc != PEARL_OK) return rc;
+        if (cudaMemcpyAsync(pin_out, arena, pk.total, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+            cudaStreamSynchronize(h->stream) != cudaSuccess)
+            return PEARL_ERR_CUDA;
+        for (int i = 0; i < PRB_NUM_FIELDS + 2; ++i)
+            if (dev[i]) memcpy(dst[i], pin_out + pk.off[i], pk.bytes[i]);
+        return PEARL_OK;
+    }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f)
         dev[f] = (dst[f] && h->view.field_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
     int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_out_idx);
@@ -409,6 +490,16 @@ int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, cons
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
+    if (h->pin && (uint64_t)B * 8 + 16 <= kPackBytes) {
+        const void* src[2] = { h_idx, h_td };
+        void* dev[2];
+        Packing pk;
+        pk.add(0, (uint64_t)B * 4);
+        pk.add(1, (uint64_t)B * 4);
+        int rc = pack_to_device(h, pk, src, 2, at(h, h->lay.off_stage_in[0]), dev);
+        if (rc != PEARL_OK) return rc;
+        return pearl_prb_update(h, B, (const int32_t*)dev[0], (const float*)dev[1], alpha, eps);
+    }
     int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_idx);
     float* d_td = (float*)at(h, h->lay.off_stage_td);
     if (cudaMemcpyAsync(d_idx, h_idx, (uint64_t)B * 4, cudaMemcpyHostToDevice, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
