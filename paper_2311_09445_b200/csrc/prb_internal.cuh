@@ -14,7 +14,7 @@ struct PrbState {
     unsigned long long cursor;        // next ring slot to be written
     unsigned long long fill;          // transitions stored, <= capacity
     unsigned long long sample_calls;  // successful sample calls so far (Philox counter words 2,3)
-    unsigned long long wmax_bits;     // batch maximum of the raw IS weights (bits of a positive double)
+    unsigned long long reserved;      // (not used)
     unsigned int status;              // PEARL_ST_* bits
     unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
     unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished

@@ -234,7 +234,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     __shared__ __align__(16) float s_top[top_floats_of(K)];
     __shared__ __align__(16) float s_child[kThreads];     // K floats per lane group: a level that came from global memory
     __shared__ uint32_t s_idx[R];
-    __shared__ double s_wraw[R];
+    __shared__ double s_wmax[kThreads / 2 / 32];          // the last CTA's maximum of the raw weights, per warp
     __shared__ volatile unsigned long long s_seen[R];     // answers of the atomics that publish the weights
     __shared__ float s_p[R];
     __shared__ unsigned s_flags[R];
@@ -313,37 +313,28 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         const bool last_descents = round + 1 >= n_rounds;      // true exactly once per CTA
         if (tid >= kThreads / 2) {
             // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path).
-            // What other CTAs read -- the raw weights and the batch maximum -- is written by atomics
-            // whose results are waited for: when a thread goes on, its value is in L2.  A fence here
-            // instead would also wait for the bulk copies the ring has in flight, and so put the
-            // ticket, and the normalisation of the weights behind it, after the whole copy.
+            // What another CTA reads -- the raw weights -- is written by atomics whose results are
+            // waited for: when a thread goes on, its value is in L2.  A fence here instead would also
+            // wait for the bulk copies the ring has in flight, and so put the ticket, and the
+            // normalisation of the weights behind it, after the whole copy.
             const uint32_t gi2 = tid - kThreads / 2;
             if (gi2 < n_round) {
-                double wr = 0.0;
                 if (kb + gi2 >= k_own) {
                     const uint32_t k2 = kb + gi2;
                     const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
-                    wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
+                    const double wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
                     out_idx[k2] = (int32_t)s_idx[gi2];
                     // (the old value goes to shared memory: a store that cannot issue before the atomic has answered)
                     s_seen[gi2] = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
                                              (unsigned long long)__double_as_longlong(wr));
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
                 }
-                s_wraw[gi2] = wr;
             }
             asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
-            if (tid == kThreads / 2) {
-                double m = 0.0;
-                for (uint32_t i = 0; i < n_round; ++i) m = fmax(m, s_wraw[i]);
-                if (m > 0.0) {
-                    s_seen[0] = atomicMax(&v.state->wmax_bits, (unsigned long long)__double_as_longlong(m));
-                }
-                if (last_descents) {
-                    // every descent of this CTA is done and its weights are in L2: the last CTA to get
-                    // here normalises the weights of the whole batch
-                    s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
-                }
+            if (tid == kThreads / 2 && last_descents) {
+                // every descent of this CTA is done and its weights are in L2: the last CTA to get
+                // here normalises the weights of the whole batch
+                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
             }
             if (last_descents) {
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
@@ -351,14 +342,36 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     if (empty) {
                         if (tid == kThreads / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
                     } else if (out_w != nullptr) {
-                        const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wmax_bits));
-                        for (uint32_t k = tid - kThreads / 2; k < B; k += kThreads / 2)
+                        // the batch maximum, then the division: the first raw weights of every thread stay in registers
+                        constexpr uint32_t kHalf = kThreads / 2, kHeld = 4;
+                        const uint32_t j = tid - kHalf;
+                        double held[kHeld];
+                        double m = 0.0;
+#pragma unroll
+                        for (uint32_t u = 0; u < kHeld; ++u) {
+                            const uint32_t k = j + u * kHalf;
+                            held[u] = k < B ? __ldcg(v.wraw + k) : 0.0;
+                            m = fmax(m, held[u]);
+                        }
+                        for (uint32_t k = j + kHeld * kHalf; k < B; k += kHalf) m = fmax(m, __ldcg(v.wraw + k));
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+                        if ((tid & 31u) == 0) s_wmax[(tid - kHalf) >> 5] = m;
+                        asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
+                        double wmax = s_wmax[0];
+#pragma unroll
+                        for (uint32_t q = 1; q < kHalf / 32; ++q) wmax = fmax(wmax, s_wmax[q]);
+#pragma unroll
+                        for (uint32_t u = 0; u < kHeld; ++u) {
+                            const uint32_t k = j + u * kHalf;
+                            if (k < B) out_w[k] = (float)__ddiv_rn(held[u], wmax);
+                        }
+                        for (uint32_t k = j + kHeld * kHalf; k < B; k += kHalf)
                             out_w[k] = (float)__ddiv_rn(__ldcg(v.wraw + k), wmax);
                     }
                     asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
                     if (tid == kThreads / 2) {
                         if (!empty) v.state->sample_calls = calls + 1;
-                        v.state->wmax_bits = 0ull;
                         v.state->sample_ticket = 0u;
                     }
                 }
