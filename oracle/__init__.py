@@ -46,6 +46,8 @@ def lib():
         L.oracle_prb_rebuild.restype = None
         L.oracle_prb_insert.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp]
         L.oracle_prb_update_priorities.argtypes = [vp, u32, vp, vp]
+        L.oracle_prb_update_delta.restype = C.c_int
+        L.oracle_prb_update_delta.argtypes = [vp, u32, vp, vp]
         L.oracle_prb_update.argtypes = [vp, u32, vp, vp, f32, f32]
         L.oracle_prb_update_after_insert.argtypes = [vp, u32, vp, vp, f32, f32, u32]
         L.oracle_prb_get_priorities.argtypes = [vp, u32, vp, vp]
@@ -158,6 +160,10 @@ class OraclePRB:
     def update_priorities(self, idx, prio) -> int:
         idx, prio = _host(idx, np.int32), _host(prio, np.float32)
         return lib().oracle_prb_update_priorities(self._h, idx.shape[0], _ptr(idx), _ptr(prio))
+
+    def update_delta(self, idx, delta) -> int:
+        idx, delta = _host(idx, np.int32), _host(delta, np.float32)
+        return lib().oracle_prb_update_delta(self._h, idx.shape[0], _ptr(idx), _ptr(delta))
 
     def max_priority(self) -> np.float32:
         return np.float32(lib().oracle_prb_max_priority(self._h))

@@ -350,6 +350,33 @@ int oracle_prb_update_priorities(oracle_prb_t *o, uint32_t B, const int32_t *idx
     return ORACLE_OK;
 }
 
+/* The paper's own form of the priority update (Section V-A, "priority update": the inputs are   */
+/* indices and the change Delta of each priority).  Entry by entry, in batch order: the leaf      */
+/* becomes leaf + Delta, one binary32 addition; an entry whose Delta is not finite, or whose sum   */
+/* is not a valid priority (negative, not finite), is skipped with BAD_PRIORITY and leaves the     */
+/* leaf as it was.  Repeated indices therefore accumulate in batch order.  Where the paper adds    */
+/* Delta to every node of the root-leaf path, the ancestors here are re-summed from their          */
+/* children afterwards, like after any other write: the same tree up to rounding, with every        */
+/* parent still equal to the sum of its children.                                                   */
+int oracle_prb_update_delta(oracle_prb_t *o, uint32_t B, const int32_t *idx, const float *delta)
+{
+    if (!o || !idx || !delta) return ORACLE_ERR_NULL;
+    if (B == 0) return ORACLE_ERR_BAD_BATCH;
+    uint32_t D = o->depth;
+    for (uint32_t b = 0; b < B; ++b) {
+        if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
+        if (!isfinite(delta[b])) { o->status |= ST_BAD_PRIORITY; continue; }
+        volatile float sum = o->level[D][idx[b]] + delta[b];
+        float p = sum;
+        if (!valid_priority(p)) { o->status |= ST_BAD_PRIORITY; continue; }
+        note_priority(o, p);
+        o->level[D][idx[b]] = p;
+        mark_dirty(o, D, (uint64_t)idx[b]);
+    }
+    resum_dirty(o);
+    return ORACLE_OK;
+}
+
 int oracle_prb_update(oracle_prb_t *o, uint32_t B, const int32_t *idx, const float *td,
                       float alpha, float eps)
 {

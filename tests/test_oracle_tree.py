@@ -284,3 +284,52 @@ def test_default_insert_priority_is_running_maximum(oracle_mod):
     o.insert(None, None, None, None, None, None, n=1)
     assert o.read_level(2)[8] == 50.0
     check_invariant(o)
+
+
+@pytest.mark.parametrize("K", FANOUTS)
+def test_delta_update_with_exact_arithmetic_equals_setting_the_priority(oracle_mod, K):
+    # Section V-A gives the update as index + change.  On small integers every binary32 operation is
+    # exact, so adding new - old must leave the tree that writing `new` leaves, whatever the order.
+    rng = np.random.default_rng(K)
+    N = 777
+    old = rng.integers(0, 50, size=N).astype(np.float32)
+    a, b = make(oracle_mod, old, K), make(oracle_mod, old, K)
+    idx = rng.permutation(N)[:300].astype(np.int32)
+    new = rng.integers(0, 50, size=300).astype(np.float32)
+    assert a.update_delta(idx, new - old[idx]) == 0
+    assert b.update_priorities(idx, new) == 0
+    for l in range(a.depth + 1):
+        assert np.array_equal(a.read_level(l).view(np.uint32), b.read_level(l).view(np.uint32))
+    check_invariant(a)
+    assert a.status() == 0
+
+
+def test_delta_update_accumulates_repeats_in_batch_order(oracle_mod):
+    # 2^24 + 1 + 1 in binary32: each addition of 1 is lost to rounding, one addition of 2 is not --
+    # so the result tells whether the repeats were added one by one in batch order.
+    big = np.float32(2 ** 24)
+    o = make(oracle_mod, [big, 1, 1, 1], 2)
+    assert o.update_delta([0, 0], [1.0, 1.0]) == 0
+    assert o.read_level(2)[0] == big
+    assert o.update_delta([0], [2.0]) == 0
+    assert o.read_level(2)[0] == big + np.float32(2)
+    # order matters: (1 + 2^24) - 2^24 = 0 but (1 - 2^24) is refused (negative), then 1 + 2^24 = 2^24
+    o2 = make(oracle_mod, [1, 1, 1, 1], 2)
+    assert o2.update_delta([1, 1], [big, -big]) == 0
+    assert o2.read_level(2)[1] == 0.0 and o2.status() == 0
+    o3 = make(oracle_mod, [1, 1, 1, 1], 2)
+    assert o3.update_delta([1, 1], [-big, big]) == 0
+    assert o3.read_level(2)[1] == big and o3.status() == oracle_mod.ST_BAD_PRIORITY
+    check_invariant(o3)
+    assert o3.max_priority() == big
+
+
+def test_delta_update_skips_invalid_entries(oracle_mod):
+    o = make(oracle_mod, P8, 4)
+    before = [o.read_level(l).copy() for l in range(o.depth + 1)]
+    assert o.update_delta([-1, 8, 0, 1, 2], [1.0, 1.0, np.nan, np.inf, -5.0]) == 0
+    assert o.status() == (oracle_mod.ST_BAD_INDEX | oracle_mod.ST_BAD_PRIORITY)
+    for l in range(o.depth + 1):
+        assert np.array_equal(o.read_level(l), before[l])
+    assert o.update_delta([2], [-4.0]) == 0             # exactly to zero is allowed
+    assert o.read_level(o.depth)[2] == 0.0 and o.total() == 27.0
