@@ -134,6 +134,16 @@ int pearl_prb_update(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const f
 int pearl_prb_update_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx,
                                 const float* d_prio);
 
+/* The paper's own form of the priority update (Section V-A, "priority update": the inputs are the
+ * indices and the change Delta of each priority).  Entry by entry in batch order the leaf becomes
+ * leaf + Delta, one binary32 addition, so that repeated indices accumulate in batch order; an
+ * entry whose Delta is not finite, or whose sum is negative or not finite, is skipped with
+ * BAD_PRIORITY and leaves the leaf as it was.  Where the paper adds Delta to every node of the
+ * root-leaf path under a mutex, the ancestors here are re-summed from their children as after any
+ * other write: the same tree up to rounding, every parent still the sum of its children, and no
+ * lock.  Arguments and errors as for pearl_prb_update_priorities. */
+int pearl_prb_update_delta(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_delta);
+
 /* Priority update that arrives after an insertion (Section IV-C, "Replay-Collision-Free
  * Scheduling": the insertion index is compared against the sampled indices, so that the Learner's
  * update does not contaminate a transition the Actors wrote in the meantime).  `inserted`

@@ -42,6 +42,7 @@ SIGNATURES = {
     "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
     "pearl_prb_update_priorities": (_i, [_vp, _u32, _vp, _vp]),
+    "pearl_prb_update_delta": (_i, [_vp, _u32, _vp, _vp]),
     "pearl_prb_update_after_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32]),
     "pearl_prb_get_priorities": (_i, [_vp, _u32, _vp, _vp]),
     "pearl_prb_update_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -180,6 +181,11 @@ class PrioritizedReplay:
         rc = load_library().pearl_prb_update_priorities(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(prio, "prio"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_update_priorities")
+
+    def update_delta(self, idx, delta) -> None:
+        rc = load_library().pearl_prb_update_delta(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(delta, "delta"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_update_delta")
 
     def update_after_insert(self, idx, td, alpha: float, eps: float, inserted: int) -> None:
         rc = load_library().pearl_prb_update_after_insert(self._h, idx.numel(), _dptr(idx, "idx"), _dptr(td, "td"),

@@ -324,6 +324,11 @@ int pearl_prb_update_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx
     return update_common(h, B, d_idx, d_prio, 1, 0.0f, 0.0f);
 }
 
+int pearl_prb_update_delta(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_delta)
+{
+    return update_common(h, B, d_idx, d_delta, 2, 0.0f, 0.0f);
+}
+
 int pearl_prb_update_after_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const float* d_td, float alpha,
                                   float eps, uint32_t inserted)
 {

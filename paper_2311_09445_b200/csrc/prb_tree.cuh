@@ -348,14 +348,15 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             const float x = mine ? pre.val : val[b];
             float p = 0.0f;
             bool ok_p;
-            if (raw) { p = x; ok_p = prb_valid_priority(p); }
+            if (raw == 2) { p = x; ok_p = fabsf(x) <= 3.402823466e+38f; }      // a change: any finite value
+            else if (raw) { p = x; ok_p = prb_valid_priority(p); }
             else ok_p = prb_priority_pow(x, eps, alpha, p);
             // stale: one of the `stale` slots written most recently, i.e. overwritten since it was sampled
             const uint64_t back = (i >= 0 && stale) ? (cursor + N - 1 - (uint64_t)i) % N : ~0ull;
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
             else if (back < stale) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
-            else { key = ((unsigned long long)(uint32_t)i << 32) | b; wmax = fmaxf(wmax, p); my_valid = true; my_idx = (uint32_t)i; }
+            else { key = ((unsigned long long)(uint32_t)i << 32) | b; if (raw != 2) wmax = fmaxf(wmax, p); my_valid = true; my_idx = (uint32_t)i; }
             vals[b] = p;
         }
         if (!one_each) keys[b] = key;
@@ -393,9 +394,48 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         }
     }
 
-    // winners write the leaves (unless the insertion overwrites the slot anyway), then the inserted leaves
     float* leaves = v.level[v.depth];
-    if (one_each) {
+    if (raw == 2) {
+        // Changes instead of values (n == 0): the last entry of a run of equal indices adds the run's
+        // changes to the leaf one by one in batch order -- the order of the sorted run -- skipping a
+        // sum that is not a valid priority.
+        float dmax = 0.0f;
+        bool refused = false;
+        auto add_change = [&](float& p, float change) {
+            const float q = __fadd_rn(p, change);
+            if (prb_valid_priority(q)) { p = q; dmax = fmaxf(dmax, q); }
+            else refused = true;
+        };
+        if (one_each) {
+            // the sorted indices and positions of all slots, in place of the keys
+            uint32_t* sidx = reinterpret_cast<uint32_t*>(smem);
+            uint32_t* spos = sidx + n2;
+            team.sync();
+            if (rank < n2) { sidx[rank] = slot.idx; spos[rank] = slot.pos; }
+            team.sync();
+            if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
+                uint32_t s0 = rank;
+                while (s0 > 0 && sidx[s0 - 1] == slot.idx) --s0;
+                float p = __ldcg(leaves + slot.idx);
+                for (uint32_t s2 = s0; s2 <= rank; ++s2) add_change(p, vals[spos[s2]]);
+                leaves[slot.idx] = p;
+            }
+        } else {
+            for (uint32_t s1 = rank; s1 < n2; s1 += nt) {
+                const unsigned long long key = keys[s1];
+                if (prb_key_invalid(key) || !team.takes(s1)) continue;
+                const uint32_t i = (uint32_t)(key >> 32);
+                if (s1 + 1 < n2 && (uint32_t)(keys[s1 + 1] >> 32) == i) continue;      // not the last of its run
+                uint32_t s0 = s1;
+                while (s0 > 0 && (uint32_t)(keys[s0 - 1] >> 32) == i) --s0;
+                float p = __ldcg(leaves + i);
+                for (uint32_t s2 = s0; s2 <= s1; ++s2) add_change(p, vals[(uint32_t)keys[s2]]);
+                leaves[i] = p;
+            }
+        }
+        if (refused) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
+        prb_note_priorities(v.state, dmax, true);
+    } else if (one_each) {
         if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
             const uint64_t ahead = slot.idx >= cursor ? slot.idx - cursor : slot.idx + N - cursor;   // distance from the cursor along the ring
             if (!(ahead < n)) leaves[slot.idx] = vals[slot.pos];

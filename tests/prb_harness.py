@@ -115,6 +115,11 @@ class Pair:
         self.gpu.update_priorities(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
                                    torch.from_numpy(np.ascontiguousarray(prio, np.float32)).to(self.dev))
 
+    def update_delta(self, idx, delta):
+        assert self.ora.update_delta(idx, delta) == 0
+        self.gpu.update_delta(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                              torch.from_numpy(np.ascontiguousarray(delta, np.float32)).to(self.dev))
+
     # ---- comparisons ------------------------------------------------------------------
     def compare_tree(self, levels=None):
         D = self.ora.depth

@@ -534,6 +534,35 @@ def test_uniform_replay(oracle_mod, wl, N, B):
     pr.close()
 
 
+@pytest.mark.parametrize("K,N,B", [(2, 300, 64), (4, 5000, 700), (16, 70_000, 256), (32, 900, 512), (8, 20_000, 3000),
+                                   (16, 50_000, 9000)])
+def test_delta_update(oracle_mod, K, N, B):
+    # Section V-A's index + change form: repeats accumulate in batch order, refused sums leave the leaf alone.
+    rng = np.random.default_rng(K * 1000 + B)
+    pr = Pair(oracle_mod, N, K, 8, 4, max(B, 1024))
+    for first in range(0, N, 1024):
+        m = min(1024, N - first)
+        b = raw_fields(rng, m, 8, 4)
+        b["prio"] = np.exp(rng.standard_normal(m)).astype(np.float32)
+        pr.insert(b)
+    for step in range(4):
+        idx = rng.integers(0, N, size=B).astype(np.int32)
+        idx[: B // 4] = idx[B // 4: 2 * (B // 4)]                      # many repeats, far apart in the batch
+        delta = (rng.standard_normal(B) * (0.3 if step < 3 else 3.0)).astype(np.float32)    # last step: many sums go negative
+        if step == 1:
+            idx[3], idx[5] = -1, N
+            delta[7], delta[9] = np.nan, np.inf
+            big = np.float32(2 ** 24)
+            idx[11], idx[12], delta[11], delta[12] = 17, 17, big, -big   # rounding-order probe
+        if step == 2:
+            idx = np.sort(idx)                                            # already in order: no sort in the kernel
+        pr.update_delta(idx, delta)
+        pr.compare_tree()
+        pr.compare_state()
+        pr.compare_status()
+    pr.close()
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_random_call_sequences(oracle_mod, seed):
     # Random geometry and a random sequence of every call, compared with the oracle after each one.
