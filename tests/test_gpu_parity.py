@@ -184,6 +184,32 @@ def test_atari_shaped_full_size(oracle_mod):
         pr.update(idx, td, wl.alpha, wl.eps)
         pr.compare_tree()
     pr.compare_state()
+    # the benchmark's step: sample, then update and insertion in one call (for rows this long the tree
+    # work runs as a kernel of its own beside the row copy)
+    for step in range(3):
+        o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)
+        ids = torch.from_numpy(slot_id[o["idx"]])
+        assert np.array_equal(g["obs"], wk.counter_row_bytes(ids, 0, wl.obs_bytes).numpy())
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        n = wl.n_insert
+        small = wk.transitions(wl, rng, n, with_obs=False)
+        new_ids = torch.arange(next_id, next_id + n, dtype=torch.int64, device=dev)
+        assert pr.ora.update(idx, td, wl.alpha, wl.eps) == 0
+        assert pr.ora.insert(None, None, small["rew"], None, small["done"], small["prio"]) == 0
+        pr.gpu.update_insert(torch.from_numpy(idx).to(dev), torch.from_numpy(td).to(dev), wl.alpha, wl.eps,
+                             wk.counter_row_bytes(new_ids, 0, wl.obs_bytes), torch.from_numpy(small["act"]).to(dev),
+                             torch.from_numpy(small["rew"]).to(dev), wk.counter_row_bytes(new_ids, 1, wl.obs_bytes),
+                             torch.from_numpy(small["done"]).to(dev), torch.from_numpy(small["prio"]).to(dev))
+        slot_id[(cursor + np.arange(n)) % wl.capacity] = np.arange(next_id, next_id + n)
+        next_id += n
+        cursor = (cursor + n) % wl.capacity
+        pr.compare_tree()
+        pr.compare_state()
+    o, g = pr.sample(wl.batch, wl.beta, wl.philox_seed)
+    ids = torch.from_numpy(slot_id[o["idx"]])
+    assert np.array_equal(g["obs"], wk.counter_row_bytes(ids, 0, wl.obs_bytes).numpy())
+    assert np.array_equal(g["next_obs"], wk.counter_row_bytes(ids, 1, wl.obs_bytes).numpy())
+    pr.compare_status()
     pr.close()
 
 
