@@ -384,6 +384,12 @@ def run_ours(args, wl, rank, world):
         # the same update with its index batch in random order (the kernel has to sort it)
         shuffled = [(upd_idx[r] if upd_idx else outs[r]["idx"])[torch.randperm(B, device=dev)] for r in range(ROTATE)]
         ms_update_shuffled = per_call_ms(lambda i: prb.update(shuffled[i % ROTATE], tds[i % ROTATE], wl.alpha, wl.eps))
+        # the sample call issued as 4 sub-batches on 4 streams of the handle (whole call, all joined)
+        def do_sample_streamed(i):
+            o = outs[i % ROTATE]
+            prb.sample_streamed(B, wl.beta, wl.philox_seed, 4, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
+                                o["rew"], o["next_obs"], o["done"])
+        ms_streamed = per_call_ms(do_sample_streamed) if B >= 4 else None
         ms_insert = per_call_ms(do_insert) if n_ins else None
         ms_fused = per_call_ms(do_update_insert) if fused else None
         status |= prb.sync()
@@ -446,7 +452,8 @@ def run_ours(args, wl, rank, world):
                   "inserts_per_s": (n_ins / (ms_insert * 1e-3)) if n_ins else None,
                   "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3, "us_update_shuffled": ms_update_shuffled * 1e3,
                   "us_insert": ms_insert * 1e3 if n_ins else None,
-                  "us_update_insert": ms_fused * 1e3 if fused else None},
+                  "us_update_insert": ms_fused * 1e3 if fused else None,
+                  "us_sample_streamed4": ms_streamed * 1e3 if ms_streamed else None},
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes,

@@ -170,6 +170,20 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
                             const float* d_rew, const void* d_next_obs, const uint8_t* d_done,
                             const float* d_prio);
 
+/* pearl_prb_sample issued as n_sub (1..4, <= B) sub-batches of consecutive strata -- sub-batch i is
+ * strata [i*B/n_sub, (i+1)*B/n_sub) -- each a launch of its own on a stream of the handle, so that
+ * the Learner can start on the first sub-batch while the others are still being gathered (the
+ * paper's overlap of computation and communication by sub-batches on several streams, Section IV-C).
+ * Outputs, and the state left behind, are those of pearl_prb_sample.  The handle's stream continues
+ * when all sub-batches are done; the weights are normalised by the maximum of the whole batch and
+ * final only then.  pearl_prb_wait_sub_batch makes `cuda_stream` (a cudaStream_t) wait until the
+ * indices and gathered rows of sub-batch `sub_batch` of the most recent streamed call are in place
+ * (PEARL_ERR_BAD_ARG if there is no such sub-batch).  n_sub == 1 is pearl_prb_sample. */
+int pearl_prb_sample_streamed(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, uint32_t n_sub,
+                              int32_t* d_idx, float* d_w, void* d_obs, void* d_act, float* d_rew,
+                              void* d_next_obs, uint8_t* d_done);
+int pearl_prb_wait_sub_batch(pearl_prb_t* prb, uint32_t sub_batch, void* cuda_stream);
+
 /* Host-buffer forms of the three calls (the paper's host runtime exchanges requests and data
  * with the Replay Manager over PCIe, Section IV-A).  They copy their inputs to the device and
  * their outputs back on the handle's stream; sample_host returns after the stream has drained,

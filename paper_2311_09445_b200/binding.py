@@ -38,6 +38,8 @@ SIGNATURES = {
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample_streamed": (_i, [_vp, _u32, _f32, _u64, _u32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_wait_sub_batch": (_i, [_vp, _u32, _vp]),
     "pearl_prb_sample_uniform": (_i, [_vp, _u32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_static_scratch": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
@@ -153,6 +155,20 @@ class PrioritizedReplay:
                                              _dptr(next_obs, "next_obs"), _dptr(done, "done"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_sample")
+
+    def sample_streamed(self, B: int, beta: float, seed: int, n_sub: int, idx, w=None, obs=None, act=None, rew=None,
+                        next_obs=None, done=None) -> None:
+        rc = load_library().pearl_prb_sample_streamed(self._h, B, beta, seed, n_sub, _dptr(idx, "idx"), _dptr(w, "w"),
+                                                      _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                                      _dptr(next_obs, "next_obs"), _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample_streamed")
+
+    def wait_sub_batch(self, sub_batch: int, stream: torch.cuda.Stream) -> None:
+        """Makes `stream` wait for sub-batch `sub_batch` of the last sample_streamed call."""
+        rc = load_library().pearl_prb_wait_sub_batch(self._h, sub_batch, C.c_void_p(stream.cuda_stream))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_wait_sub_batch")
 
     def sample_uniform(self, B: int, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None, done=None) -> None:
         rc = load_library().pearl_prb_sample_uniform(self._h, B, seed, _dptr(idx, "idx"), _dptr(w, "w"), _dptr(obs, "obs"),

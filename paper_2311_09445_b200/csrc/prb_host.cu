@@ -105,6 +105,9 @@ struct pearl_prb {
     uint32_t max_batch;
     uint64_t launches;
     PrbFork fork = PrbFork{nullptr, nullptr, nullptr};   // side stream and events of pearl_prb_update_insert with long rows
+    // pearl_prb_sample_streamed: one stream and one event per sub-batch, created with the handle
+    PrbSubStreams subs = PrbSubStreams{{nullptr, nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr, nullptr}, nullptr};
+    uint32_t streamed_subs = 0;          // sub-batches of the last streamed call (0: none yet)
     // Small batches of the *_host calls travel packed: all arrays of a call in one pinned buffer, one
     // copy each way (2 x kPackBytes of pinned host memory; nullptr: every array is copied by itself).
     unsigned char* pin = nullptr;
@@ -112,6 +115,11 @@ struct pearl_prb {
     ~pearl_prb()
     {
         destroy_fork(fork);
+        for (uint32_t i = 0; i < kPrbMaxSubBatches; ++i) {
+            if (subs.done[i]) cudaEventDestroy(subs.done[i]);
+            if (subs.stream[i]) cudaStreamDestroy(subs.stream[i]);
+        }
+        if (subs.fork) cudaEventDestroy(subs.fork);
         if (pin_read) cudaEventDestroy(pin_read);
         if (pin) cudaFreeHost(pin);
         cudaGetLastError();
@@ -179,6 +187,14 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
         delete h;
         return PEARL_ERR_CUDA;
     }
+    for (uint32_t i = 0; i < kPrbMaxSubBatches; ++i) {
+        if (cudaStreamCreateWithFlags(&h->subs.stream[i], cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->subs.done[i], cudaEventDisableTiming) != cudaSuccess) {
+            delete h;
+            return PEARL_ERR_CUDA;
+        }
+    }
+    if (cudaEventCreateWithFlags(&h->subs.fork, cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
     if (cudaHostAlloc((void**)&h->pin, 2 * kPackBytes, cudaHostAllocDefault) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->pin_read, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();                 // (not fatal: the host calls then copy array by array)
@@ -267,10 +283,11 @@ int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* 
 }
 
 static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
-                         void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done, int uniform)
+                         void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done, int uniform, uint32_t n_sub = 1)
 {
     if (!h || !d_idx) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B) return PEARL_ERR_BAD_ARG;
     if (!finite_nonneg(beta)) return PEARL_ERR_BAD_ARG;
     const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
     int rc = check_batch_ptrs(h, ptrs);
@@ -280,9 +297,10 @@ static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, 
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
-    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform);
+    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform, n_sub, &h->subs);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
+    if (n_sub > 1) h->streamed_subs = n_sub;
     return PEARL_OK;
 }
 
@@ -290,6 +308,21 @@ int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int3
                      void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
 {
     return sample_common(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 0);
+}
+
+int pearl_prb_sample_streamed(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, uint32_t n_sub, int32_t* d_idx, float* d_w,
+                              void* d_obs, void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    return sample_common(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 0, n_sub);
+}
+
+int pearl_prb_wait_sub_batch(pearl_prb_t* h, uint32_t sub_batch, void* cuda_stream)
+{
+    if (!h) return PEARL_ERR_NULL;
+    if (sub_batch >= h->streamed_subs) return PEARL_ERR_BAD_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    return cudaStreamWaitEvent((cudaStream_t)cuda_stream, h->subs.done[sub_batch], 0) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }
 
 int pearl_prb_sample_uniform(pearl_prb_t* h, uint32_t B, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,

@@ -61,9 +61,20 @@ struct PrbFork {
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
                       int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f, const PrbFork* fork = nullptr);
-// (uniform != 0: uniform replay, no tree walk, all weights 1)
+// Streams and events of a sample call that is issued as sub-batches (the paper's sub-batch
+// streaming, Section IV-C): sub-batch i runs on stream[i]; done[i] fires when its rows are in place.
+constexpr uint32_t kPrbMaxSubBatches = 4;
+struct PrbSubStreams {
+    cudaStream_t stream[kPrbMaxSubBatches];
+    cudaEvent_t done[kPrbMaxSubBatches];
+    cudaEvent_t fork;
+};
+
+// (uniform != 0: uniform replay, no tree walk, all weights 1; n_sub > 1: as that many launches, one
+// per sub-batch of consecutive strata, each on a stream of `subs`, joined back into s)
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, int uniform = 0);
+                      const PrbBatch& dst, cudaStream_t s, int uniform = 0, uint32_t n_sub = 1,
+                      const PrbSubStreams* subs = nullptr);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
 // (ins_n > 0, B within one sub-batch: the tree part of an insertion of ins_n transitions follows
 // the update in the same kernel, whose CTAs take part in the insertion's cursor ticket with the

@@ -41,7 +41,9 @@ constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in
 
 struct SamplePlan {
     uint32_t tps;                            // tasks per stratum (1 unless some field is in row mode)
-    uint32_t n_tasks;                        // B * tps
+    uint32_t n_tasks;                        // tasks of this launch: a whole number of strata ...
+    uint32_t first_task;                     // ... starting with this task of the batch (sub-batch launches; else 0)
+    uint32_t ticket_total;                   // CTAs of all launches of the call: the last of them normalises the weights
     uint32_t task_first[PRB_NUM_FIELDS];     // row mode: tasks [task_first, task_first + chunks) of a stratum
     uint32_t chunks[PRB_NUM_FIELDS];         //   copy the chunks of field f; 0 = short rows, copied flat
     uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
@@ -267,8 +269,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 
     // this CTA's tasks and the strata they touch
     const uint32_t tps = plan.tps;
-    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * plan.n_tasks) / gridDim.x);
-    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * plan.n_tasks) / gridDim.x);
+    const uint32_t t_lo = plan.first_task + (uint32_t)(((uint64_t)blockIdx.x * plan.n_tasks) / gridDim.x);
+    const uint32_t t_hi = plan.first_task + (uint32_t)(((uint64_t)(blockIdx.x + 1) * plan.n_tasks) / gridDim.x);
     const uint32_t k_lo = t_lo / tps;
     const uint32_t k_hi = (t_hi + tps - 1) / tps;
     const uint32_t k_own = (t_lo + tps - 1) / tps;       // strata whose first task is here: this CTA writes their idx / weight
@@ -334,7 +336,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (tid == kThreads / 2 && last_descents) {
                 // every descent of this CTA is done and its weights are in L2: the last CTA to get
                 // here normalises the weights of the whole batch
-                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == plan.ticket_total - 1) ? 1u : 0u;
             }
             if (last_descents) {
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
@@ -410,8 +412,9 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 }  // namespace
 
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, int uniform)
+                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs)
 {
+    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
     const int sm_count = prb_sm_count();
     const int dev = prb_current_device();
     SamplePlan plan;
@@ -432,6 +435,8 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     const bool row_mode = plan.tps > 0;
     if (!row_mode) plan.tps = 1;
     plan.n_tasks = B * plan.tps;
+    plan.first_task = 0;
+    plan.ticket_total = 0;
     // levels 1 .. top_levels staged in shared memory while they fit
     // (the levels lie one after another in the slab, each start 256-byte aligned)
     plan.uniform = uniform ? 1u : 0u;
@@ -472,64 +477,98 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     const uint32_t pf_group_bytes = v.fanout * v.fanout * (uint32_t)sizeof(float);
     plan.pf_groups = 0;
     plan.pf_off = 0;
-    uint32_t grid, smem = 0;
-    plan.ring_stages = 0;
-    plan.ring_stage_bytes = 0;
-    if (row_mode) {
-        // one CTA per SM, each with a ring of chunk-sized stages
-        uint32_t stage = 0;
-        for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
-        stage = (stage + 127u) / 128u * 128u;
-        grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
-        // strata a CTA can touch: its share of the tasks, plus one for a range that straddles
-        const uint32_t tasks_per_cta = (plan.n_tasks + grid - 1) / grid;
-        uint32_t strata = (tasks_per_cta + plan.tps - 1) / plan.tps + 1;
-        if (strata > R) strata = R;
-        uint32_t pf_bytes = prefetch ? strata * pf_group_bytes : 0u;
-        uint32_t ring_bytes = dyn_max[dev][ki] - kRingBarBytes;
-        if (pf_bytes + 8u * stage > ring_bytes) pf_bytes = 0;      // (not at the price of the ring)
-        ring_bytes -= pf_bytes;
-        if (ring_bytes > kRingBytes) ring_bytes = kRingBytes;
-        plan.ring_stage_bytes = stage;
-        plan.ring_stages = ring_bytes / stage;
-        if (plan.ring_stages > 32) plan.ring_stages = 32;
-        plan.pf_off = kRingBarBytes + plan.ring_stages * stage;
-        plan.pf_groups = pf_bytes ? strata : 0u;
-        smem = plan.pf_off + pf_bytes;
-    } else {
-        // a small batch is spread over more CTAs than it needs: its descents are chains of dependent
-        // L2 reads, and more SMs keep more of them in flight
-        const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
-        const uint32_t per_cta = R >= 4 ? R / 4 : 1;
-        const uint32_t want = (B + per_cta - 1) / per_cta;
-        grid = want < one_wave ? want : one_wave;
-        if (prefetch) {
-            uint32_t strata = (B + grid - 1) / grid;
+    // One launch, or one per sub-batch of strata [k0, k1): sized like a call of its own, on a stream
+    // of its own, so that the first sub-batch is complete while the others are still being copied.
+    SamplePlan sub_plan[kPrbMaxSubBatches];
+    uint32_t sub_grid[kPrbMaxSubBatches], sub_smem[kPrbMaxSubBatches];
+    uint32_t ticket_total = 0, max_smem = 0;
+    for (uint32_t i = 0; i < n_sub; ++i) {
+        SamplePlan& sp = sub_plan[i];
+        sp = plan;
+        const uint32_t k0 = (uint32_t)((uint64_t)i * B / n_sub), k1 = (uint32_t)((uint64_t)(i + 1) * B / n_sub);
+        const uint32_t strata_here = k1 - k0;
+        sp.first_task = k0 * plan.tps;
+        sp.n_tasks = strata_here * plan.tps;
+        uint32_t grid, smem = 0;
+        sp.ring_stages = 0;
+        sp.ring_stage_bytes = 0;
+        if (row_mode) {
+            // one CTA per SM, each with a ring of chunk-sized stages
+            uint32_t stage = 0;
+            for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
+            stage = (stage + 127u) / 128u * 128u;
+            grid = sp.n_tasks < (uint32_t)sm_count ? sp.n_tasks : (uint32_t)sm_count;
+            // strata a CTA can touch: its share of the tasks, plus one for a range that straddles
+            const uint32_t tasks_per_cta = (sp.n_tasks + grid - 1) / grid;
+            uint32_t strata = (tasks_per_cta + plan.tps - 1) / plan.tps + 1;
             if (strata > R) strata = R;
-            plan.pf_groups = strata;
-            smem = strata * pf_group_bytes;
+            uint32_t pf_bytes = prefetch ? strata * pf_group_bytes : 0u;
+            uint32_t ring_bytes = dyn_max[dev][ki] - kRingBarBytes;
+            if (pf_bytes + 8u * stage > ring_bytes) pf_bytes = 0;      // (not at the price of the ring)
+            ring_bytes -= pf_bytes;
+            if (ring_bytes > kRingBytes) ring_bytes = kRingBytes;
+            sp.ring_stage_bytes = stage;
+            sp.ring_stages = ring_bytes / stage;
+            if (sp.ring_stages > 32) sp.ring_stages = 32;
+            sp.pf_off = kRingBarBytes + sp.ring_stages * stage;
+            sp.pf_groups = pf_bytes ? strata : 0u;
+            smem = sp.pf_off + pf_bytes;
+        } else {
+            // a small batch is spread over more CTAs than it needs: its descents are chains of dependent
+            // L2 reads, and more SMs keep more of them in flight
+            const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
+            const uint32_t per_cta = R >= 4 ? R / 4 : 1;
+            const uint32_t want = (strata_here + per_cta - 1) / per_cta;
+            grid = want < one_wave ? want : one_wave;
+            if (prefetch) {
+                uint32_t strata = (strata_here + grid - 1) / grid;
+                if (strata > R) strata = R;
+                sp.pf_groups = strata;
+                smem = strata * pf_group_bytes;
+            }
         }
+        sub_grid[i] = grid;
+        sub_smem[i] = smem;
+        ticket_total += grid;
+        if (smem > max_smem) max_smem = smem;
     }
+    for (uint32_t i = 0; i < n_sub; ++i) sub_plan[i].ticket_total = ticket_total;
     static bool big_smem[kPrbMaxDevices][6];
     cudaError_t attr = cudaSuccess;
+    if (n_sub > 1 && (cudaEventRecord(subs->fork, s) != cudaSuccess)) return -1;
+    for (uint32_t i = 0; i < n_sub; ++i) {
+        cudaStream_t at = s;
+        if (n_sub > 1) {
+            at = subs->stream[i];
+            if (cudaStreamWaitEvent(at, subs->fork, 0) != cudaSuccess) return -1;
+        }
+        const uint32_t grid = sub_grid[i], smem = sub_smem[i];
+        const SamplePlan& sp = sub_plan[i];
 #define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
     do {                                                                                                          \
-        if (smem && !big_smem[dev][ki]) {                                                                              \
+        if (max_smem && !big_smem[dev][ki]) {                                                                     \
             attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                                         (int)dyn_max[dev][ki]);                                                   \
-            big_smem[dev][ki] = (attr == cudaSuccess);                                                                 \
+            big_smem[dev][ki] = (attr == cudaSuccess);                                                            \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \
-            prb_sample_kernel<KK><<<grid, kThreads, smem, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan);          \
+            prb_sample_kernel<KK><<<grid, kThreads, smem, at>>>(v, B, beta, seed, d_idx, d_w, dst, sp);           \
     } while (0)
-    switch (v.fanout) {
-    case 2: PRB_LAUNCH_SAMPLE(2); break;
-    case 4: PRB_LAUNCH_SAMPLE(4); break;
-    case 8: PRB_LAUNCH_SAMPLE(8); break;
-    case 16: PRB_LAUNCH_SAMPLE(16); break;
-    default: PRB_LAUNCH_SAMPLE(32); break;
-    }
+        switch (v.fanout) {
+        case 2: PRB_LAUNCH_SAMPLE(2); break;
+        case 4: PRB_LAUNCH_SAMPLE(4); break;
+        case 8: PRB_LAUNCH_SAMPLE(8); break;
+        case 16: PRB_LAUNCH_SAMPLE(16); break;
+        default: PRB_LAUNCH_SAMPLE(32); break;
+        }
 #undef PRB_LAUNCH_SAMPLE
-    if (attr != cudaSuccess) return -1;
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+        if (attr != cudaSuccess) return -1;
+        if (n_sub > 1) {
+            // the sub-batch's rows and indices are in place when its event fires; the caller's stream
+            // goes on when all of them have (the weights are final only then)
+            if (cudaEventRecord(subs->done[i], at) != cudaSuccess || cudaStreamWaitEvent(s, subs->done[i], 0) != cudaSuccess)
+                return -1;
+        }
+    }
+    return cudaGetLastError() == cudaSuccess ? (int)n_sub : -1;
 }

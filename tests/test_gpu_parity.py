@@ -560,6 +560,52 @@ def test_uniform_replay(oracle_mod, wl, N, B):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B,n_sub", [(wk.CARTPOLE, 3000, 64, 2), (wk.DDPG, 100_000, 1000, 4), (wk.DDPG, 5000, 3, 3),
+                                          (wk.ATARI, 700, 512, 4), (wk.ATARI, 700, 37, 3)])
+def test_sample_streamed_as_sub_batches(oracle_mod, wl, N, B, n_sub):
+    # Sub-batch streaming (Section IV-C): the same sample, issued as launches on several streams.  A
+    # consumer stream that waits for sub-batch i alone must find that sub-batch's indices and rows.
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(N + B)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 1024)
+    dev = pr.dev
+    for first in range(0, N, 512):
+        pr.insert(wk.transitions(wl, rng, min(512, N - first), first))
+    consumer = torch.cuda.Stream(dev)
+    for call in range(3):
+        o = pr.ora.sample(B, wl.beta, wl.philox_seed)
+        t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+             "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "act": torch.zeros((B, max(wl.act_bytes, 1)), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+             "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+        torch.cuda.synchronize()
+        pr.gpu.sample_streamed(B, wl.beta, wl.philox_seed, n_sub, t["idx"], t["w"], t["obs"],
+                               t["act"] if wl.act_bytes else None, t["rew"], t["next_obs"], t["done"])
+        early = []
+        with torch.cuda.stream(consumer):
+            for i in range(n_sub):                  # each sub-batch is copied out as soon as it alone is ready
+                pr.gpu.wait_sub_batch(i, consumer)
+                k0, k1 = i * B // n_sub, (i + 1) * B // n_sub
+                early.append((k0, k1, t["idx"][k0:k1].clone(), t["obs"][k0:k1].clone(), t["done"][k0:k1].clone()))
+        torch.cuda.synchronize()
+        for k0, k1, idx_i, obs_i, done_i in early:
+            assert np.array_equal(idx_i.cpu().numpy(), o["idx"][k0:k1])
+            assert np.array_equal(obs_i.cpu().numpy().reshape(-1), np.ascontiguousarray(o["obs"][k0:k1]).view(np.uint8).reshape(-1))
+            assert np.array_equal(done_i.cpu().numpy(), o["done"][k0:k1])
+        g = {k: v.cpu().numpy() for k, v in t.items()}
+        if not wl.act_bytes:
+            g["act"] = o["act"]
+        pr.compare_sample(o, g)                    # the whole batch, weights included, after the join
+        pr.compare_state()
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)
+    with pytest.raises(Exception):
+        pr.gpu.wait_sub_batch(n_sub, consumer)
+    pr.compare_status()
+    pr.close()
+
+
 @pytest.mark.parametrize("K,N,B", [(2, 300, 64), (4, 5000, 700), (16, 70_000, 256), (32, 900, 512), (8, 20_000, 3000),
                                    (16, 50_000, 9000)])
 def test_delta_update(oracle_mod, K, N, B):
