@@ -56,6 +56,8 @@ def lib():
         L.oracle_prb_targets.argtypes = [vp, u32, u64, u64, vp]
         L.oracle_prb_targets.restype = None
         L.oracle_prb_sample.argtypes = [vp, u32, f32, u64, vp, vp, vp, vp, vp, vp, vp]
+        L.oracle_prb_sample_buffer_norm.restype = C.c_int
+        L.oracle_prb_sample_buffer_norm.argtypes = [vp, u32, f32, u64, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_prb_sample_uniform.argtypes = [vp, u32, u64, vp, vp, vp, vp, vp, vp, vp]
         L.oracle_prb_info.argtypes = [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64), C.POINTER(u32)]
         L.oracle_prb_level_nodes.argtypes = [vp, u32]
@@ -192,8 +194,9 @@ class OraclePRB:
                                                     _ptr(out["done"]))
         return out
 
-    def sample(self, B: int, beta: float, seed: int, gather: bool = True):
-        """Returns a dict with idx, w and (if ``gather``) the gathered fields as raw bytes / f32."""
+    def sample(self, B: int, beta: float, seed: int, gather: bool = True, buffer_norm: bool = False):
+        """Returns a dict with idx, w and (if ``gather``) the gathered fields as raw bytes / f32.
+        buffer_norm: weights divided by the largest weight in the whole buffer instead of the batch."""
         out = {
             "idx": np.full(B, -1, dtype=np.int32),
             "w": np.zeros(B, dtype=np.float32),
@@ -204,9 +207,10 @@ class OraclePRB:
             out["rew"] = np.zeros(B, dtype=np.float32)
             out["next_obs"] = np.zeros((B, self.obs_bytes), dtype=np.uint8)
             out["done"] = np.zeros(B, dtype=np.uint8)
-        rc = lib().oracle_prb_sample(self._h, B, beta, seed, _ptr(out["idx"]), _ptr(out["w"]),
-                                     _ptr(out.get("obs")), _ptr(out.get("act")), _ptr(out.get("rew")),
-                                     _ptr(out.get("next_obs")), _ptr(out.get("done")))
+        fn = lib().oracle_prb_sample_buffer_norm if buffer_norm else lib().oracle_prb_sample
+        rc = fn(self._h, B, beta, seed, _ptr(out["idx"]), _ptr(out["w"]),
+                _ptr(out.get("obs")), _ptr(out.get("act")), _ptr(out.get("rew")),
+                _ptr(out.get("next_obs")), _ptr(out.get("done")))
         out["rc"] = rc
         return out
 

@@ -506,9 +506,9 @@ void oracle_prb_targets(oracle_prb_t *o, uint32_t B, uint64_t seed, uint64_t cal
 /* non-positive total raises EMPTY and leaves outputs and the call counter   */
 /* untouched.                                                                */
 /* ------------------------------------------------------------------------ */
-int oracle_prb_sample(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
-                      int32_t *idx, float *w, void *obs, void *act, float *rew,
-                      void *next_obs, uint8_t *done)
+static int sample_impl(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
+                       int32_t *idx, float *w, void *obs, void *act, float *rew,
+                       void *next_obs, uint8_t *done, int buffer_norm)
 {
     if (!o || !idx) return ORACLE_ERR_NULL;
     if (B == 0) return ORACLE_ERR_BAD_BATCH;
@@ -529,6 +529,15 @@ int oracle_prb_sample(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
         wraw[k] = pow(prob_times_size, -(double)beta);
         if (wraw[k] > wmax) wmax = wraw[k];
     }
+    if (buffer_norm) {
+        /* the largest weight any stored transition could get: that of the smallest positive priority */
+        float pmin = 0.0f;
+        for (uint64_t i = 0; i < o->size; ++i) {
+            float p = o->level[o->depth][i];
+            if (p > 0.0f && (pmin == 0.0f || p < pmin)) pmin = p;
+        }
+        wmax = pow((double)o->size * (double)pmin / total, -(double)beta);
+    }
     if (w) for (uint32_t k = 0; k < B; ++k) w[k] = (float)(wraw[k] / wmax);
     for (uint32_t k = 0; k < B; ++k) {
         uint64_t i = (uint64_t)idx[k];
@@ -541,6 +550,25 @@ int oracle_prb_sample(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
     free(x); free(wraw);
     o->sample_calls += 1;
     return ORACLE_OK;
+}
+
+int oracle_prb_sample(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
+                      int32_t *idx, float *w, void *obs, void *act, float *rew,
+                      void *next_obs, uint8_t *done)
+{
+    return sample_impl(o, B, beta, seed, idx, w, obs, act, rew, next_obs, done, 0);
+}
+
+/* The same sample with the weights normalised as in the prioritized-replay paper the toolkit    */
+/* follows (Schaul et al., Algorithm 1: w_j = (N P(j))^-beta / max_i w_i with the maximum over the */
+/* whole memory): the divisor is the weight of the smallest positive priority in the buffer,     */
+/* (N p_min / total)^-beta, found by a plain scan.  Weights are then at most 1 and do not depend   */
+/* on which other transitions the batch happens to hold.                                           */
+int oracle_prb_sample_buffer_norm(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
+                                  int32_t *idx, float *w, void *obs, void *act, float *rew,
+                                  void *next_obs, uint8_t *done)
+{
+    return sample_impl(o, B, beta, seed, idx, w, obs, act, rew, next_obs, done, 1);
 }
 
 int oracle_prb_read_rows(oracle_prb_t *o, const int32_t *idx, uint32_t n, void *obs, void *act,

@@ -200,3 +200,30 @@ def test_uniform_replay(oracle_mod):
         counts += np.bincount(i, minlength=N)
     chi2 = ((counts - 800.0) ** 2 / 800.0).sum()
     assert stats.chi2.sf(chi2, N - 1) > 1e-4
+
+
+def test_buffer_wide_weight_normalisation(oracle_mod):
+    # Schaul et al., Algorithm 1: the weights are divided by the largest weight over the whole memory,
+    # i.e. that of the smallest positive priority.  Closed form: w_k = (p_min / p_k)^beta.
+    prio = np.array([3, 1, 4, 0, 5, 9, 0.5, 6], dtype=np.float32)
+    for K in (2, 4, 8):
+        a, b = make(oracle_mod, prio, K), make(oracle_mod, prio, K)
+        for beta in (0.0, 0.4, 1.0):
+            out = a.sample(4, beta, 7, buffer_norm=True)
+            ref = b.sample(4, beta, 7)
+            assert np.array_equal(out["idx"], ref["idx"])               # same draw, same counter
+            p = prio[out["idx"]].astype(np.float64)
+            assert np.allclose(out["w"], (0.5 / p) ** beta, rtol=1e-6)
+            assert np.all(out["w"] <= 1.0 + 1e-6)
+            # against the batch-normalised weights: one common factor, the batch's own largest weight
+            factor = (0.5 / p.min()) ** beta
+            assert np.allclose(out["w"], ref["w"].astype(np.float64) * factor, rtol=1e-6)
+        assert a.info() == b.info()
+    # uniform priorities: every weight is exactly 1 in either form
+    o = make(oracle_mod, np.full(64, 2.5, dtype=np.float32), 4)
+    assert np.all(o.sample(16, 0.7, 1, buffer_norm=True)["w"] == 1.0)
+    # zero priorities do not count as the minimum; slots not yet written neither
+    o = oracle_mod.OraclePRB(16, 2, 0, 0)
+    assert o.insert(None, None, None, None, None, np.array([0, 2, 8], dtype=np.float32)) == 0
+    out = o.sample(8, 1.0, 3, buffer_norm=True)
+    assert np.allclose(out["w"], 2.0 / np.array([0, 2, 8], dtype=np.float64)[out["idx"]], rtol=1e-6)
