@@ -170,6 +170,16 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
                             const float* d_rew, const void* d_next_obs, const uint8_t* d_done,
                             const float* d_prio);
 
+/* pearl_prb_sample with the weights normalised as in the prioritized-replay paper the toolkit
+ * follows (Schaul et al., Algorithm 1: w_j = (N P(j))^-beta / max_i w_i, the maximum over the whole
+ * memory): the divisor is the weight of the smallest positive priority stored,
+ * (N p_min / total)^-beta, found by a scan of the leaves in a launch of its own before the sample.
+ * Weights are then at most 1 and do not depend on which other transitions the batch holds.  PEARL
+ * itself does not say how the weights are normalised.  Everything else as pearl_prb_sample. */
+int pearl_prb_sample_buffer_norm(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, int32_t* d_idx,
+                                 float* d_w, void* d_obs, void* d_act, float* d_rew, void* d_next_obs,
+                                 uint8_t* d_done);
+
 /* pearl_prb_sample issued as n_sub (1..4, <= B) sub-batches of consecutive strata -- sub-batch i is
  * strata [i*B/n_sub, (i+1)*B/n_sub) -- each a launch of its own on a stream of the handle, so that
  * the Learner can start on the first sub-batch while the others are still being gathered (the

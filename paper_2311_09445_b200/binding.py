@@ -38,6 +38,7 @@ SIGNATURES = {
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_sample_buffer_norm": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_streamed": (_i, [_vp, _u32, _f32, _u64, _u32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_wait_sub_batch": (_i, [_vp, _u32, _vp]),
     "pearl_prb_sample_uniform": (_i, [_vp, _u32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -155,6 +156,14 @@ class PrioritizedReplay:
                                              _dptr(next_obs, "next_obs"), _dptr(done, "done"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_sample")
+
+    def sample_buffer_norm(self, B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None,
+                           done=None) -> None:
+        rc = load_library().pearl_prb_sample_buffer_norm(self._h, B, beta, seed, _dptr(idx, "idx"), _dptr(w, "w"),
+                                                         _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                                         _dptr(next_obs, "next_obs"), _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_sample_buffer_norm")
 
     def sample_streamed(self, B: int, beta: float, seed: int, n_sub: int, idx, w=None, obs=None, act=None, rew=None,
                         next_obs=None, done=None) -> None:

@@ -283,7 +283,8 @@ int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* 
 }
 
 static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
-                         void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done, int uniform, uint32_t n_sub = 1)
+                         void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done, int uniform, uint32_t n_sub = 1,
+                         int buffer_norm = 0)
 {
     if (!h || !d_idx) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
@@ -297,7 +298,7 @@ static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, 
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
-    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform, n_sub, &h->subs);
+    const int k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform, n_sub, &h->subs, buffer_norm);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
     if (n_sub > 1) h->streamed_subs = n_sub;
@@ -308,6 +309,12 @@ int pearl_prb_sample(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int3
                      void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
 {
     return sample_common(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 0);
+}
+
+int pearl_prb_sample_buffer_norm(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
+                                 void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
+{
+    return sample_common(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 0, 1, 1);
 }
 
 int pearl_prb_sample_streamed(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, uint32_t n_sub, int32_t* d_idx, float* d_w,

@@ -14,7 +14,7 @@ struct PrbState {
     unsigned long long cursor;        // next ring slot to be written
     unsigned long long fill;          // transitions stored, <= capacity
     unsigned long long sample_calls;  // successful sample calls so far (Philox counter words 2,3)
-    unsigned long long reserved;      // (not used)
+    unsigned long long pmin_bits;     // smallest positive leaf (bits of a binary32), filled in before a sample that normalises over the buffer
     unsigned int status;              // PEARL_ST_* bits
     unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
     unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished
@@ -70,11 +70,13 @@ struct PrbSubStreams {
     cudaEvent_t fork;
 };
 
-// (uniform != 0: uniform replay, no tree walk, all weights 1; n_sub > 1: as that many launches, one
+// (buffer_norm != 0: weights divided by the largest weight of the whole buffer, found by a scan of
+// the leaves in a launch of its own, instead of the batch's;
+// uniform != 0: uniform replay, no tree walk, all weights 1; n_sub > 1: as that many launches, one
 // per sub-batch of consecutive strata, each on a stream of `subs`, joined back into s)
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s, int uniform = 0, uint32_t n_sub = 1,
-                      const PrbSubStreams* subs = nullptr);
+                      const PrbSubStreams* subs = nullptr, int buffer_norm = 0);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
 // (ins_n > 0, B within one sub-batch: the tree part of an insertion of ins_n transitions follows
 // the update in the same kernel, whose CTAs take part in the insertion's cursor ticket with the

@@ -49,6 +49,7 @@ struct SamplePlan {
     uint32_t chunk[PRB_NUM_FIELDS];          // granules per chunk
     uint32_t ring_stages, ring_stage_bytes;  // bulk-copy ring (long rows only; 0 stages otherwise)
     uint32_t uniform;                        // 1: uniform replay (no tree walk): index = floor(u * fill)
+    uint32_t buffer_norm;                    // 1: weights divided by the largest weight over the buffer (state->pmin_bits), not the batch
     uint32_t top_levels;                     // levels 1 .. top_levels are staged in shared memory
     uint32_t top_vec4;                       // 16-byte units staged, from the start of level 1
     uint32_t top_off[PRB_MAX_LEVELS];        // offset (floats) of a staged level from the start of level 1
@@ -253,6 +254,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     const unsigned long long calls = v.state->sample_calls;
     const unsigned long long fill = v.state->fill;
     const float total32 = __ldg(v.level[0]);
+    const float pmin = plan.buffer_norm ? __uint_as_float((unsigned)v.state->pmin_bits) : 0.0f;
     {
         // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
         const float4* src = reinterpret_cast<const float4*>(v.level[1]);
@@ -326,9 +328,15 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
                     const double wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
                     out_idx[k2] = (int32_t)s_idx[gi2];
-                    // (the old value goes to shared memory: a store that cannot issue before the atomic has answered)
-                    s_seen[gi2] = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
-                                             (unsigned long long)__double_as_longlong(wr));
+                    if (plan.buffer_norm) {
+                        // the divisor is known already: the weight of the buffer's smallest positive priority
+                        const double wmax = pow(__ddiv_rn(__dmul_rn((double)fill, (double)pmin), total), -(double)beta);
+                        if (out_w != nullptr) out_w[k2] = (float)__ddiv_rn(wr, wmax);
+                    } else {
+                        // (the old value goes to shared memory: a store that cannot issue before the atomic has answered)
+                        s_seen[gi2] = atomicExch(reinterpret_cast<unsigned long long*>(v.wraw + k2),
+                                                 (unsigned long long)__double_as_longlong(wr));
+                    }
                     if (s_flags[gi2]) atomicOr(&v.state->status, s_flags[gi2]);
                 }
             }
@@ -343,7 +351,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                 if (s_last) {
                     if (empty) {
                         if (tid == kThreads / 2) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-                    } else if (out_w != nullptr) {
+                    } else if (out_w != nullptr && !plan.buffer_norm) {
                         // the batch maximum, then the division: the first raw weights of every thread stay in registers
                         constexpr uint32_t kHalf = kThreads / 2, kHeld = 4;
                         const uint32_t j = tid - kHalf;
@@ -409,10 +417,26 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     }
 }
 
+// The smallest positive leaf among the `fill` stored ones, into state->pmin_bits (set to all ones
+// beforehand): positive binary32 values order like their bit patterns.
+__global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
+{
+    const unsigned long long fill = v.state->fill;
+    const float* leaves = v.level[v.depth];
+    unsigned best = 0xFFFFFFFFu;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < fill;
+         i += (unsigned long long)gridDim.x * blockDim.x) {
+        const float p = __ldg(leaves + i);
+        if (p > 0.0f) best = min(best, __float_as_uint(p));
+    }
+    best = __reduce_min_sync(0xFFFFFFFFu, best);
+    if ((threadIdx.x & 31u) == 0 && best != 0xFFFFFFFFu) atomicMin(&v.state->pmin_bits, (unsigned long long)best);
+}
+
 }  // namespace
 
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs)
+                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs, int buffer_norm)
 {
     if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
     const int sm_count = prb_sm_count();
@@ -440,6 +464,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     // levels 1 .. top_levels staged in shared memory while they fit
     // (the levels lie one after another in the slab, each start 256-byte aligned)
     plan.uniform = uniform ? 1u : 0u;
+    plan.buffer_norm = (buffer_norm && !uniform) ? 1u : 0u;
     plan.top_levels = 0;
     plan.top_vec4 = 0;
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
@@ -533,6 +558,16 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         if (smem > max_smem) max_smem = smem;
     }
     for (uint32_t i = 0; i < n_sub; ++i) sub_plan[i].ticket_total = ticket_total;
+    int extra_launches = 0;
+    if (plan.buffer_norm) {
+        // the scan of the leaves goes first, on the caller's stream
+        if (cudaMemsetAsync(&v.state->pmin_bits, 0xFF, sizeof(unsigned long long), s) != cudaSuccess) return -1;
+        const uint64_t per_cta = 256ull * 16ull;
+        uint64_t ctas = (v.capacity + per_cta - 1) / per_cta;
+        if (ctas > (uint64_t)sm_count * 4) ctas = (uint64_t)sm_count * 4;
+        prb_leaf_min_kernel<<<(unsigned)ctas, 256, 0, s>>>(v);
+        extra_launches = 1;
+    }
     static bool big_smem[kPrbMaxDevices][6];
     cudaError_t attr = cudaSuccess;
     if (n_sub > 1 && (cudaEventRecord(subs->fork, s) != cudaSuccess)) return -1;
@@ -570,5 +605,5 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
                 return -1;
         }
     }
-    return cudaGetLastError() == cudaSuccess ? (int)n_sub : -1;
+    return cudaGetLastError() == cudaSuccess ? (int)n_sub + extra_launches : -1;
 }

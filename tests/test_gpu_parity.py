@@ -560,6 +560,43 @@ def test_uniform_replay(oracle_mod, wl, N, B):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B", [(wk.CARTPOLE, 3000, 64), (wk.DDPG, 100_000, 1000), (wk.ATARI, 700, 512), (wk.TINY, 9, 32)])
+def test_sample_normalised_over_the_buffer(oracle_mod, wl, N, B):
+    # Weights divided by the largest weight any stored transition could get (smallest positive priority).
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(N * 7 + B)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 1024)
+    dev = pr.dev
+    filled = 0
+    for first in range(0, N - N // 3, 512):                  # a third of the ring stays unwritten
+        m = min(512, N - N // 3 - first)
+        b = wk.transitions(wl, rng, m, first)
+        b["prio"][::7] = 0.0                                    # zero priorities are never the minimum
+        pr.insert(b)
+        filled += m
+    for call in range(4):
+        o = pr.ora.sample(B, wl.beta, wl.philox_seed, buffer_norm=True)
+        t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+             "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "act": torch.zeros((B, max(wl.act_bytes, 1)), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+             "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+        pr.gpu.sample_buffer_norm(B, wl.beta, wl.philox_seed, t["idx"], t["w"], t["obs"], t["act"] if wl.act_bytes else None,
+                                  t["rew"], t["next_obs"], t["done"])
+        torch.cuda.synchronize()
+        g = {k: v.cpu().numpy() for k, v in t.items()}
+        assert np.array_equal(o["idx"], g["idx"])
+        np.testing.assert_allclose(g["w"], o["w"], rtol=1e-5, atol=0)
+        assert g["w"].max() <= 1.0
+        assert np.array_equal(np.ascontiguousarray(o["obs"]).view(np.uint8).reshape(-1), g["obs"].reshape(-1))
+        pr.compare_state()
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        pr.update(idx, td, wl.alpha, wl.eps)                    # the minimum moves between calls
+        o2, g2 = pr.sample(B, wl.beta, wl.philox_seed)          # and the batch-normalised call still agrees
+    pr.compare_status()
+    pr.close()
+
+
 @pytest.mark.parametrize("wl,N,B,n_sub", [(wk.CARTPOLE, 3000, 64, 2), (wk.DDPG, 100_000, 1000, 4), (wk.DDPG, 5000, 3, 3),
                                           (wk.ATARI, 700, 512, 4), (wk.ATARI, 700, 37, 3)])
 def test_sample_streamed_as_sub_batches(oracle_mod, wl, N, B, n_sub):
