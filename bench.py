@@ -390,6 +390,13 @@ def run_ours(args, wl, rank, world):
             prb.sample_streamed(B, wl.beta, wl.philox_seed, 4, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
                                 o["rew"], o["next_obs"], o["done"])
         ms_streamed = per_call_ms(do_sample_streamed) if B >= 4 else None
+
+        # the sample call with weights normalised over the whole buffer (a scan of the leaves goes first)
+        def do_sample_buffer_norm(i):
+            o = outs[i % ROTATE]
+            prb.sample_buffer_norm(B, wl.beta, wl.philox_seed, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
+                                   o["rew"], o["next_obs"], o["done"])
+        ms_buffer_norm = per_call_ms(do_sample_buffer_norm)
         ms_insert = per_call_ms(do_insert) if n_ins else None
         ms_fused = per_call_ms(do_update_insert) if fused else None
         status |= prb.sync()
@@ -453,7 +460,8 @@ def run_ours(args, wl, rank, world):
                   "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3, "us_update_shuffled": ms_update_shuffled * 1e3,
                   "us_insert": ms_insert * 1e3 if n_ins else None,
                   "us_update_insert": ms_fused * 1e3 if fused else None,
-                  "us_sample_streamed4": ms_streamed * 1e3 if ms_streamed else None},
+                  "us_sample_streamed4": ms_streamed * 1e3 if ms_streamed else None,
+                  "us_sample_buffer_norm": ms_buffer_norm * 1e3},
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes,

@@ -219,6 +219,11 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
     PrbView& v = h->view;
     memset(&v, 0, sizeof(v));
     v.state = (PrbState*)at(h, L.off_state);
+    if (cudaMemsetAsync(&v.state->pmin_bits, 0xFF, sizeof(unsigned long long), h->stream) != cudaSuccess) {
+        if (h->owns_slab) cudaFree(h->base);
+        delete h;
+        return PEARL_ERR_CUDA;
+    }
     for (uint32_t l = 0; l <= L.depth; ++l) {
         v.level[l] = (float*)at(h, L.off_level[l]);
         v.level_alloc[l] = (uint32_t)L.level_alloc[l];

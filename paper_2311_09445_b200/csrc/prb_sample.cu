@@ -325,12 +325,17 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (gi2 < n_round) {
                 if (kb + gi2 >= k_own) {
                     const uint32_t k2 = kb + gi2;
-                    const double scaled = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
-                    const double wr = plan.uniform ? 1.0 : pow(scaled, -(double)beta);
+                    // (one call site for the power: with the buffer-wide divisor the loop runs twice)
+                    double base = __ddiv_rn(__dmul_rn((double)fill, (double)s_p[gi2]), total);
+                    double wr = 1.0, wmax = 1.0;
+#pragma unroll 1
+                    for (uint32_t q = 0; q < 1u + plan.buffer_norm; ++q) {
+                        const double r = plan.uniform ? 1.0 : pow(base, -(double)beta);
+                        if (q == 0) wr = r; else wmax = r;
+                        base = __ddiv_rn(__dmul_rn((double)fill, (double)pmin), total);     // the buffer's smallest positive priority
+                    }
                     out_idx[k2] = (int32_t)s_idx[gi2];
                     if (plan.buffer_norm) {
-                        // the divisor is known already: the weight of the buffer's smallest positive priority
-                        const double wmax = pow(__ddiv_rn(__dmul_rn((double)fill, (double)pmin), total), -(double)beta);
                         if (out_w != nullptr) out_w[k2] = (float)__ddiv_rn(wr, wmax);
                     } else {
                         // (the old value goes to shared memory: a store that cannot issue before the atomic has answered)
@@ -382,6 +387,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
                     if (tid == kThreads / 2) {
                         if (!empty) v.state->sample_calls = calls + 1;
+                        if (plan.buffer_norm) v.state->pmin_bits = ~0ull;      // (ready for the next scan)
                         v.state->sample_ticket = 0u;
                     }
                 }
@@ -417,8 +423,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     }
 }
 
-// The smallest positive leaf among the `fill` stored ones, into state->pmin_bits (set to all ones
-// beforehand): positive binary32 values order like their bit patterns.
+// The smallest positive leaf among the `fill` stored ones, into state->pmin_bits (all ones at creation and
+// again after every sample that used it): positive binary32 values order like their bit patterns.
 __global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
 {
     const unsigned long long fill = v.state->fill;
@@ -429,8 +435,14 @@ __global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
         const float p = __ldg(leaves + i);
         if (p > 0.0f) best = min(best, __float_as_uint(p));
     }
+    __shared__ unsigned s_best[8];
     best = __reduce_min_sync(0xFFFFFFFFu, best);
-    if ((threadIdx.x & 31u) == 0 && best != 0xFFFFFFFFu) atomicMin(&v.state->pmin_bits, (unsigned long long)best);
+    if ((threadIdx.x & 31u) == 0) s_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (unsigned w = 1; w < blockDim.x / 32u; ++w) best = min(best, s_best[w]);
+        if (best != 0xFFFFFFFFu) atomicMin(&v.state->pmin_bits, (unsigned long long)best);      // one atomic per CTA
+    }
 }
 
 }  // namespace
@@ -561,7 +573,6 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     int extra_launches = 0;
     if (plan.buffer_norm) {
         // the scan of the leaves goes first, on the caller's stream
-        if (cudaMemsetAsync(&v.state->pmin_bits, 0xFF, sizeof(unsigned long long), s) != cudaSuccess) return -1;
         const uint64_t per_cta = 256ull * 16ull;
         uint64_t ctas = (v.capacity + per_cta - 1) / per_cta;
         if (ctas > (uint64_t)sm_count * 4) ctas = (uint64_t)sm_count * 4;
