@@ -383,20 +383,21 @@ def run_ours(args, wl, rank, world):
         ms_update = per_call_ms(do_update)
         # the same update with its index batch in random order (the kernel has to sort it)
         shuffled = [(upd_idx[r] if upd_idx else outs[r]["idx"])[torch.randperm(B, device=dev)] for r in range(ROTATE)]
-        ms_update_shuffled = per_call_ms(lambda i: prb.update(shuffled[i % ROTATE], tds[i % ROTATE], wl.alpha, wl.eps))
+        ms_update_shuffled = per_call_ms(lambda i: prb.update(shuffled[i % ROTATE], tds[i % ROTATE], wl.alpha, wl.eps)) \
+            if not args.core_only else None
         # the sample call issued as 4 sub-batches on 4 streams of the handle (whole call, all joined)
         def do_sample_streamed(i):
             o = outs[i % ROTATE]
             prb.sample_streamed(B, wl.beta, wl.philox_seed, 4, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
                                 o["rew"], o["next_obs"], o["done"])
-        ms_streamed = per_call_ms(do_sample_streamed) if B >= 4 else None
+        ms_streamed = per_call_ms(do_sample_streamed) if (B >= 4 and not args.core_only) else None
 
         # the sample call with weights normalised over the whole buffer (a scan of the leaves goes first)
         def do_sample_buffer_norm(i):
             o = outs[i % ROTATE]
             prb.sample_buffer_norm(B, wl.beta, wl.philox_seed, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
                                    o["rew"], o["next_obs"], o["done"])
-        ms_buffer_norm = per_call_ms(do_sample_buffer_norm)
+        ms_buffer_norm = per_call_ms(do_sample_buffer_norm) if not args.core_only else None
         ms_insert = per_call_ms(do_insert) if n_ins else None
         ms_fused = per_call_ms(do_update_insert) if fused else None
         status |= prb.sync()
@@ -457,11 +458,11 @@ def run_ours(args, wl, rank, world):
                    "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
         "rates": {"samples_per_s": B / (ms_sample * 1e-3), "updates_per_s": B / (ms_update * 1e-3),
                   "inserts_per_s": (n_ins / (ms_insert * 1e-3)) if n_ins else None,
-                  "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3, "us_update_shuffled": ms_update_shuffled * 1e3,
+                  "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3, "us_update_shuffled": ms_update_shuffled * 1e3 if ms_update_shuffled else None,
                   "us_insert": ms_insert * 1e3 if n_ins else None,
                   "us_update_insert": ms_fused * 1e3 if fused else None,
                   "us_sample_streamed4": ms_streamed * 1e3 if ms_streamed else None,
-                  "us_sample_buffer_norm": ms_buffer_norm * 1e3},
+                  "us_sample_buffer_norm": ms_buffer_norm * 1e3 if ms_buffer_norm else None},
         "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes,
@@ -518,6 +519,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-copy-context", action="store_true", help="skip the torch copy / index_select context timings")
+    ap.add_argument("--core-only", action="store_true",
+                    help="time only the step and its three calls (no shuffled-update, streamed or buffer-normalised sample timings)")
     ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
     args = ap.parse_args()
