@@ -158,11 +158,14 @@ int pearl_prb_update_after_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d
  * index outside [0, fill) yields 0 and raises PEARL_ST_BAD_INDEX.  1 <= B <= max_batch. */
 int pearl_prb_get_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, float* d_out);
 
-/* Priority update followed by insertion, in one launch.  The result is exactly that of
+/* Priority update followed by insertion, in one call.  The result is exactly that of
  * pearl_prb_update(prb, B, d_idx, d_td, alpha, eps) followed by pearl_prb_insert(prb, n, ...): the
- * update's tree work is done first, the insertion's tree work after it, by the same thread block,
- * while the other thread blocks already copy the new rows into the Data Storage (an update touches
- * the tree only, so the two do not conflict).  This is the overlap of the paper's training
+ * update's tree work is done first, the insertion's tree work after it, by the same thread blocks,
+ * while other thread blocks already copy the new rows into the Data Storage (an update touches
+ * the tree only, so the two do not conflict).  Short rows: one launch.  Rows of 8 KB and more: the
+ * tree work is a kernel of its own on a second stream of the handle, beside the kernel that copies
+ * the rows; the handle's stream continues when both are done (capturable in a CUDA graph).  This
+ * is the overlap of the paper's training
  * protocol, where insertion runs beside the priority update (Section IV-C; Eq. 7:
  * T_itr = T_samp + max(T_ins, T_upd + T_learner)).  Arguments and errors as for the two calls. */
 int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, const float* d_td,
