@@ -534,7 +534,12 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
             uint32_t stage = 0;
             for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
             stage = (stage + 127u) / 128u * 128u;
-            grid = sp.n_tasks < (uint32_t)sm_count ? sp.n_tasks : (uint32_t)sm_count;
+            // (sub-batch launches take half the SMs' worth each way round: two of them run side by side,
+            // so a later one's prologue hides behind an earlier one's copy)
+            uint32_t room = (uint32_t)sm_count;
+            if (n_sub > 1) room = (room * 2u + n_sub - 1) / n_sub;
+            if (room > (uint32_t)sm_count) room = (uint32_t)sm_count;
+            grid = sp.n_tasks < room ? sp.n_tasks : room;
             // strata a CTA can touch: its share of the tasks, plus one for a range that straddles
             const uint32_t tasks_per_cta = (sp.n_tasks + grid - 1) / grid;
             uint32_t strata = (tasks_per_cta + plan.tps - 1) / plan.tps + 1;
