@@ -560,6 +560,38 @@ def test_uniform_replay(oracle_mod, wl, N, B):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B", [(wk.ATARI, 2000, 512), (wk.DDPG, 200_000, 256)])
+def test_weights_over_many_calls(oracle_mod, wl, N, B):
+    # The weights of a call are normalised by the last thread block to have published its raw weights,
+    # while the others are still copying rows: 150 calls in a row, every weight checked.
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(N)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 512, oracle_store=False)
+    dev = pr.dev
+    for first in range(0, N, 500):
+        m = min(500, N - first)
+        b = wk.transitions(wl, rng, m, first)
+        pr.insert(dict(rew=b["rew"], done=b["done"], prio=b["prio"]), dev_batch=wk.to_device(b, dev))
+    t = {"idx": torch.zeros(B, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+         "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+         "act": torch.zeros((B, max(wl.act_bytes, 1)), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+         "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+         "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+    for call in range(150):
+        o = pr.ora.sample(B, wl.beta, wl.philox_seed, gather=False)
+        t["w"].fill_(-1.0)
+        pr.gpu.sample(B, wl.beta, wl.philox_seed, t["idx"], t["w"], t["obs"], t["act"] if wl.act_bytes else None, t["rew"],
+                      t["next_obs"], t["done"])
+        assert np.array_equal(t["idx"].cpu().numpy(), o["idx"])
+        w = t["w"].cpu().numpy()
+        np.testing.assert_allclose(w, o["w"], rtol=1e-5, atol=0)
+        assert w.max() == np.float32(1.0)
+        if call % 10 == 0:
+            pr.update(o["idx"], (rng.standard_normal(B) * 2).astype(np.float32), wl.alpha, wl.eps)
+    pr.compare_status()
+    pr.close()
+
+
 @pytest.mark.parametrize("wl,N,B", [(wk.CARTPOLE, 3000, 64), (wk.DDPG, 100_000, 1000), (wk.ATARI, 700, 512), (wk.TINY, 9, 32)])
 def test_sample_normalised_over_the_buffer(oracle_mod, wl, N, B):
     # Weights divided by the largest weight any stored transition could get (smallest positive priority).
