@@ -27,8 +27,12 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     if (v.top_levels) top.mem = reinterpret_cast<float*>(smem + prb_update_smem_bytes(n2));
     if (team.part == 0) prb_top_begin(v, top, team.rank, team.size);
     unsigned long long fill, cursor = 0;
+    PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
     if (ins_n) {
-        // with an insertion: cursor and fill are read once per CTA, before anything is published
+        // with an insertion: cursor and fill are read once per CTA, before anything is published;
+        // every thread fetches its first inputs meanwhile (beside the row copy each round trip is long)
+        if (threadIdx.x < B) { pre.has_update = true; pre.idx = idx[threadIdx.x]; pre.val = val[threadIdx.x]; }
+        if (threadIdx.x < ins_n && ins_prio != nullptr) { pre.has_prio = true; pre.prio = ins_prio[threadIdx.x]; }
         if (threadIdx.x == 0) { s_cursor = v.state->cursor; s_fill = v.state->fill; }
         __syncthreads();
         cursor = s_cursor;
@@ -38,8 +42,7 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
         fill = v.state->fill;
         if (stale) cursor = v.state->cursor;
     }
-    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor,
-                    PrbPreloaded{false, false, 0, 0.0f, 0.0f}, stale, top);
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top);
 }
 
 // Priority retrieval: one thread per entry.
