@@ -201,7 +201,9 @@ __device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __
 // lane's own bulk group) and, if it has another chunk, waits until the store has read the stage
 // before loading again.  All stages of all SMs are in flight together, about 200 KB per SM,
 // which registers cannot hold.  Addresses and sizes are multiples of 16 bytes (rows of 16-byte
-// granules, 256-byte aligned bases).
+// granules, 256-byte aligned bases).  Rows that stream through -- everything but a sampled batch
+// on its way to the Learner -- carry the L2 hint "evict first", so that a step's ~100 MB of rows
+// do not push the few megabytes of the tree out of L2.
 
 constexpr uint32_t kBulkSpinLimit = 1u << 20;   // mbarrier polls before a wait gives up
 
@@ -213,6 +215,7 @@ struct PrbBulkLane {
     uint32_t parity;     // phase parity of the next load's completion
     bool busy;           // a store issued from the stage may still be reading it
     bool failed;         // a bounded wait ran out
+    uint64_t stream_policy;   // L2 policy "evict first" for rows that are not read again soon
 
     __device__ __forceinline__ void init(void* bar_mem, void* buf_mem)
     {
@@ -220,17 +223,20 @@ struct PrbBulkLane {
         parity = 0; busy = false; failed = false;
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
     }
+    // (the source is read once: always hinted "evict first")
     __device__ __forceinline__ void load(const void* gsrc, uint32_t bytes)
     {
         if (busy) { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); busy = false; }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(buf), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                     ::"r"(buf), "l"(gsrc), "r"(bytes), "r"(bar), "l"(stream_policy) : "memory");
     }
     // Waits (bounded) for the load, then stores the stage to gdst.  The store is issued inside the
     // polling loop so that a lane whose data has landed does not wait for the other lanes.
-    __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
+    // keep: the destination is read again soon (a sampled batch); otherwise it is hinted "evict first".
+    __device__ __forceinline__ void store(void* gdst, uint32_t bytes, bool keep)
     {
         bool done = false;
         for (uint32_t spin = 0; spin < kBulkSpinLimit && !done; ++spin) {
@@ -239,8 +245,12 @@ struct PrbBulkLane {
                          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
             if (ok) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             ::"l"(gdst), "r"(buf), "r"(bytes) : "memory");
+                if (keep)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 ::"l"(gdst), "r"(buf), "r"(bytes) : "memory");
+                else
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                                 ::"l"(gdst), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 done = true;
             }
