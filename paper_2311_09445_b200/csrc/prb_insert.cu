@@ -185,7 +185,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         while (t < t_hi) {
             uint64_t slot = cursor + row;
             if (slot >= v.capacity) slot -= v.capacity;
-            ring.store(v.store[f] + (slot * W + e0) * 16u, bytes, false);
+            ring.store(v.store[f] + (slot * W + e0) * 16u, bytes);
             t += plan.ring_stages;
             if (t < t_hi) {
                 locate(t, f, row, W, e0, bytes);

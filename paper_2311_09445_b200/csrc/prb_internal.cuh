@@ -201,9 +201,10 @@ __device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __
 // lane's own bulk group) and, if it has another chunk, waits until the store has read the stage
 // before loading again.  All stages of all SMs are in flight together, about 200 KB per SM,
 // which registers cannot hold.  Addresses and sizes are multiples of 16 bytes (rows of 16-byte
-// granules, 256-byte aligned bases).  Rows that stream through -- everything but a sampled batch
-// on its way to the Learner -- carry the L2 hint "evict first", so that a step's ~100 MB of rows
-// do not push the few megabytes of the tree out of L2.
+// granules, 256-byte aligned bases).  Every row is read or written once and not touched again
+// soon (a sampled batch is read once by the Learner, right after the call), so all these copies
+// carry the L2 hint "evict first": a step's ~100 MB of rows then do not push the few megabytes of
+// the tree out of L2, nor one another.
 
 constexpr uint32_t kBulkSpinLimit = 1u << 20;   // mbarrier polls before a wait gives up
 
@@ -215,7 +216,7 @@ struct PrbBulkLane {
     uint32_t parity;     // phase parity of the next load's completion
     bool busy;           // a store issued from the stage may still be reading it
     bool failed;         // a bounded wait ran out
-    uint64_t stream_policy;   // L2 policy "evict first" for rows that are not read again soon
+    uint64_t stream_policy;   // L2 policy "evict first"
 
     __device__ __forceinline__ void init(void* bar_mem, void* buf_mem)
     {
@@ -225,7 +226,6 @@ struct PrbBulkLane {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
     }
-    // (the source is read once: always hinted "evict first")
     __device__ __forceinline__ void load(const void* gsrc, uint32_t bytes)
     {
         if (busy) { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); busy = false; }
@@ -235,8 +235,7 @@ struct PrbBulkLane {
     }
     // Waits (bounded) for the load, then stores the stage to gdst.  The store is issued inside the
     // polling loop so that a lane whose data has landed does not wait for the other lanes.
-    // keep: the destination is read again soon (a sampled batch); otherwise it is hinted "evict first".
-    __device__ __forceinline__ void store(void* gdst, uint32_t bytes, bool keep)
+    __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
     {
         bool done = false;
         for (uint32_t spin = 0; spin < kBulkSpinLimit && !done; ++spin) {
@@ -245,12 +244,8 @@ struct PrbBulkLane {
                          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
             if (ok) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                if (keep)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                                 ::"l"(gdst), "r"(buf), "r"(bytes) : "memory");
-                else
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
-                                 ::"l"(gdst), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                             ::"l"(gdst), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 done = true;
             }

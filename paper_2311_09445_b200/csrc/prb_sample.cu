@@ -405,7 +405,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
                     const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
                     ring.load(v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u, bytes);
-                    ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes, true);
+                    ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
                 }
             }
             // short rows: copied by the stratum's owner through registers (warp 0 drives the ring when there is one)
