@@ -33,7 +33,7 @@ ROTATE = 8           # distinct input/output batch buffers cycled through, so in
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one prb_sample_kernel launch on Atari-shaped rows with B = 512, from the
 # ncu capture summarised in profiles/prb_kernels_atari_N32768.md.  Null it if that kernel changes.
-SAMPLE_TRAFFIC_NCU = {"atari_dqn": 29.7e6}      # dram read + write of one sample launch (profiles/)
+SAMPLE_TRAFFIC_NCU = {"atari_dqn": 29.6e6}      # dram read + write of one sample launch (profiles/)
 
 
 def load_peak():
