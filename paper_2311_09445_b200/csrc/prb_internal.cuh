@@ -194,7 +194,7 @@ __device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __
     if (e < e_end) dst[dst_at(e)] = src[src_at(e)];
 }
 
-// ---- bulk asynchronous copies (TMA, non-tensor form, no multicast) ------------------------------
+// ---- bulk asynchronous copies (TMA, non-tensor form, one destination each) ----------------------
 // Long rows move global -> shared -> global as cp.async.bulk transfers.  Warp 0 of a CTA drives
 // a ring of up to 32 stages in shared memory, ONE LANE PER STAGE: a lane issues the load of its
 // chunk (completion on the stage's mbarrier), waits for it, issues the store (tracked by the
