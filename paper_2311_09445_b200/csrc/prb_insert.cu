@@ -9,7 +9,9 @@
 //   Long rows (at least 8 KB of 16-byte granules, Atari-shaped): one CTA per SM; warp 0 of
 //   every CTA drives bulk asynchronous copies global -> shared -> global through a ~200 KB
 //   ring (row chunks of <= 8 KB, one lane per stage), issuing its loads before the cursor has
-//   even arrived; the other warps copy the short fields, and in CTA 0 they first do the tree.
+//   even arrived; the other warps copy the short fields.  CTA 0 does the tree and moves no rows;
+//   with a priority update in the same call the tree work is a kernel of its own on a second
+//   stream (prb_update.cu) and every CTA here copies.
 // Tree work: write the n leaves, then re-sum the dirty parents level by level (a contiguous
 // slot range dirties a contiguous parent range on every level, so no sorting is needed).
 // The CTA that is last to have read the cursor advances it (and the fill count) while the copies

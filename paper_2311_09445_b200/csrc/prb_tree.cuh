@@ -309,11 +309,16 @@ __host__ __device__ inline size_t prb_update_smem_bytes(uint32_t n2)
 }
 
 // Batched priority update by one team (PEARL Section V-A, "priority update", read as set +
-// re-sum).  Entries are keyed (index << 32) | batch position and sorted; the last entry of every
-// run of equal indices wins and writes its leaf; then, level by level from the deepest, the
-// first entry of every run of equal ancestors re-sums that ancestor from its children in
-// left-to-right order.  Sorted order survives dropping low digits of the index, so no list is
-// compacted and no lock is taken.  n2 = prb_update_n2(B); smem holds
+// re-sum).  Entries are keyed (index, batch position) and sorted -- with one entry per thread by
+// warp-wide sorting networks and a merge by rank, each thread then holding its place's index and
+// its neighbours' in registers; with more, by a bitonic network in shared memory.  The last entry
+// of every run of equal indices wins and writes its leaf (raw == 2: adds the run's changes to the
+// leaf in batch order); then, level by level from the deepest down to the staged top, the first
+// entry of every run of equal ancestors re-sums that ancestor from its children in left-to-right
+// order, and the staged levels are re-summed whole (prb_top_passes).  Sorted order survives
+// dropping low digits of the index, so no list is compacted and no lock is taken.
+// raw: 0 = val holds TD errors (transformed), 1 = priorities, 2 = changes of priorities.
+// n2 = prb_update_n2(B); smem holds
 // prb_update_smem_bytes(n2) bytes; fill = the fill count before this launch (indices must be below it).
 // With stale > 0 (and n == 0) entries that name one of the `stale` ring slots before `cursor` are
 // skipped: they were overwritten after they had been sampled.
