@@ -819,6 +819,19 @@ def test_argument_errors_leave_state_untouched(oracle_mod):
     with pytest.raises(PearlError) as e:
         pr.gpu.sample(8, 0.4, 0, idx, obs=torch.zeros(8 * 16 + 16, dtype=torch.uint8, device=dev)[4:4 + 8 * 16])
     assert e.value.code == -5                                # misaligned 16-byte rows
+    with pytest.raises(PearlError) as e:
+        pr.gpu.wait_sub_batch(0, torch.cuda.current_stream(dev))      # no streamed call yet
+    assert e.value.code == -7
+    for bad_subs in (0, 5, 9):                                        # 1..4 sub-batches, and not more than B
+        with pytest.raises(PearlError) as e:
+            pr.gpu.sample_streamed(8 if bad_subs != 9 else 3, 0.4, 0, bad_subs if bad_subs != 9 else 4, idx)
+        assert e.value.code == -7
+    with pytest.raises(PearlError) as e:
+        pr.gpu.sample_buffer_norm(8, -1.0, 0, idx)
+    assert e.value.code == -7
+    with pytest.raises(PearlError) as e:
+        pr.gpu.update_delta(idx[:40], td[:40])                        # B > max_batch
+    assert e.value.code == -3
     big = Pair(oracle_mod, 16, 2, 0, 0, 32)
     with pytest.raises(PearlError) as e:
         big.gpu.insert(None, None, None, None, None, torch.ones(17, device=dev))
