@@ -75,13 +75,16 @@ uint64_t pearl_prb_slab_bytes(uint64_t capacity, uint32_t fanout, const pearl_la
  *   cuda_stream  a cudaStream_t (NULL = the legacy default stream) on which every call enqueues.
  *   slab         optional caller-owned device memory of at least pearl_prb_slab_bytes() bytes,
  *                256-byte aligned; NULL lets the library allocate (and free in destroy).
- * The tree, the state and the scratch area are zeroed on the stream.  Returns PEARL_ERR_OOM if
- * the slab is too small. */
+ * The tree, the state and the scratch area are zeroed on the stream.  Besides the slab a handle
+ * owns five more streams with their events (the tree kernel of a long-row update_insert, the
+ * sub-batches of pearl_prb_sample_streamed; all joined back into cuda_stream before a call's work
+ * is over) and 512 KB of pinned host memory for the *_host calls (without it they copy array by
+ * array).  Returns PEARL_ERR_OOM if the slab is too small. */
 int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout,
                      const pearl_layout_t* layout, uint32_t max_batch, int device,
                      void* cuda_stream, void* slab, uint64_t slab_bytes);
 
-/* Synchronises the stream, frees library-owned memory and the handle. */
+/* Synchronises the handle's streams, frees library-owned memory, streams, events and the handle. */
 int pearl_prb_destroy(pearl_prb_t* prb);
 
 /* Insertion (Section V-A: "priority retrievals followed by priority updates"; Listing 2: the

@@ -261,6 +261,8 @@ int pearl_prb_destroy(pearl_prb_t* h)
     int rc = PEARL_OK;
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) rc = PEARL_ERR_CUDA;
     if (h->fork.side && cudaStreamSynchronize(h->fork.side) != cudaSuccess) rc = PEARL_ERR_CUDA;
+    for (uint32_t i = 0; i < kPrbMaxSubBatches; ++i)
+        if (h->subs.stream[i] && cudaStreamSynchronize(h->subs.stream[i]) != cudaSuccess) rc = PEARL_ERR_CUDA;
     destroy_fork(h->fork);
     if (h->owns_slab && cudaFree(h->base) != cudaSuccess) rc = PEARL_ERR_CUDA;
     delete h;
