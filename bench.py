@@ -488,6 +488,119 @@ def run_ours(args, wl, rank, world):
     return line
 
 
+# ------------------------------------------------------------------------------------------
+# Scaling sweep (capacity x fanout x batch): per-call times of every cell, one process
+# ------------------------------------------------------------------------------------------
+SWEEP_CAPACITIES = [1 << 16, 1 << 18, 1 << 20, 1 << 22, 1 << 24, 1 << 26]
+SWEEP_FANOUTS = [2, 4, 16, 32]
+SWEEP_BATCHES = [32, 256, 1024, 4096, 16384, 65536]
+
+
+def run_sweep(args):
+    """Times sample, update, insert and the step (sample + update_insert) on every cell of the scaling
+    sweep: 165-byte transitions, LogNormal(0, 2) priorities, 1024 insertions per step.  A buffer is
+    created and filled once per (capacity, fanout) and serves all its batch sizes; every timing is a
+    captured graph of ROTATE consecutive calls, replayed.  Prints one JSON line with a row per cell."""
+    import torch
+    from paper_2311_09445_b200 import PrioritizedReplay
+    from paper_2311_09445_b200 import workloads as wk
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(dev)
+    caps = [c for c in SWEEP_CAPACITIES if not args.capacity or c == args.capacity]
+    gen = torch.Generator(device=dev)
+    rows = []
+    clocks = ClockSampler(0)
+    clocks.start()
+    t_start = time.time()
+    with torch.cuda.stream(stream):
+        for N in caps:
+            for K in SWEEP_FANOUTS:
+                wl = wk.sweep_cell(N, K, 1024, cell_id=0)
+                gen.manual_seed(wl.seed + N % 997 + K)
+                batches_B = [b for b in SWEEP_BATCHES if b <= N // 2]
+                chunk = min(N, 1 << 16)
+                prb = PrioritizedReplay(N, K, wl.obs_bytes, wl.act_bytes, max(chunk, max(batches_B)), device=dev, stream=stream)
+
+                def lognormal_prio(n):
+                    d = torch.exp(2.0 * torch.randn(n, generator=gen, device=dev, dtype=torch.float64))
+                    return ((d + 1e-6) ** 0.6).to(torch.float32)
+
+                def make_batch(n):
+                    return {"obs": torch.randn((n, wl.obs_bytes // 4), generator=gen, device=dev).view(torch.uint8),
+                            "next_obs": torch.randn((n, wl.obs_bytes // 4), generator=gen, device=dev).view(torch.uint8),
+                            "act": (torch.rand((n, wl.act_bytes // 4), generator=gen, device=dev) * 2 - 1).view(torch.uint8),
+                            "rew": torch.randn(n, generator=gen, device=dev),
+                            "done": (torch.rand(n, generator=gen, device=dev) < 0.05).to(torch.uint8)}
+
+                rowsrc = make_batch(chunk)       # the same rows for every prefill chunk, fresh priorities
+                for first in range(0, N, chunk):
+                    prb.insert(rowsrc["obs"], rowsrc["act"], rowsrc["rew"], rowsrc["next_obs"], rowsrc["done"], lognormal_prio(chunk))
+                ins = []
+                for r in range(ROTATE):
+                    b = make_batch(wl.n_insert)
+                    b["prio"] = lognormal_prio(wl.n_insert)
+                    ins.append(b)
+                for B in batches_B:
+                    cw = wk.sweep_cell(N, K, B)
+                    outs = [out_buffers(cw, dev, B) for _ in range(ROTATE)]
+                    tds = [torch.exp(2.0 * torch.randn(B, generator=gen, device=dev)) for _ in range(ROTATE)]
+
+                    def do_sample(i):
+                        o = outs[i % ROTATE]
+                        prb.sample(B, cw.beta, cw.philox_seed, o["idx"], o["w"], o["obs"], o["act"], o["rew"], o["next_obs"], o["done"])
+
+                    def do_update(i):
+                        prb.update(outs[i % ROTATE]["idx"], tds[i % ROTATE], cw.alpha, cw.eps)
+
+                    def do_insert(i):
+                        b = ins[i % ROTATE]
+                        prb.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+
+                    def do_update_insert(i):
+                        b = ins[i % ROTATE]
+                        prb.update_insert(outs[i % ROTATE]["idx"], tds[i % ROTATE], cw.alpha, cw.eps, b["obs"], b["act"], b["rew"],
+                                          b["next_obs"], b["done"], b["prio"])
+
+                    def do_step(i):
+                        do_sample(i)
+                        do_update_insert(i)
+
+                    for i in range(ROTATE):       # every output buffer holds a sampled batch before updates are timed
+                        do_step(i)
+                    reps = 3 if B >= 16384 else 6
+
+                    def per_call_us(fn):
+                        g = torch.cuda.CUDAGraph()
+                        with torch.cuda.graph(g, stream=stream):
+                            for r in range(ROTATE):
+                                fn(r)
+                        g.replay()
+                        return time_loop(stream, lambda i: g.replay(), reps) / (reps * ROTATE) * 1e3
+
+                    row = {"N": N, "K": K, "B": B, "depth": prb.info()[3],
+                           "us_sample": per_call_us(do_sample), "us_update": per_call_us(do_update),
+                           "us_insert": per_call_us(do_insert), "us_update_insert": per_call_us(do_update_insert),
+                           "us_step": per_call_us(do_step)}
+                    row["transitions_per_s"] = B / (row["us_step"] * 1e-6)
+                    rows.append(row)
+                    print("sweep %6.1f s  %s" % (time.time() - t_start, json.dumps(row)), file=sys.stderr, flush=True)
+                    del outs, tds
+                status = prb.sync()
+                if status & ~0x8:          # anything but CLAMPED (informational)
+                    raise RuntimeError("status bits 0x%x in sweep cell N=%d K=%d" % (status, N, K))
+                prb.close()
+                del prb, rowsrc, ins
+                torch.cuda.empty_cache()
+    clk = clocks.stop()
+    return {"metric": METRIC, "unit": UNIT, "n_gpus": 1, "data": "synthetic",
+            "config": {"workload": "sweep", "transition_bytes": 165, "insert_per_step": 1024,
+                       "step": "sample(idx,IS,gather) + update_insert", "cuda_graph": True,
+                       "timing": "graphs of %d consecutive calls over rotating buffers, CUDA events" % ROTATE},
+            "cells": rows, "clocks": clk}
+
+
 def run_reference(args, wl, rank, world):
     """The CPU oracle as it stands, on this machine's host cores; rank 0 only."""
     if rank != 0:
@@ -523,9 +636,15 @@ def main():
                     help="time only the step and its three calls (no shuffled-update, streamed or buffer-normalised sample timings)")
     ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every cell of the capacity x fanout x batch sweep instead (one GPU; --capacity picks one capacity)")
     args = ap.parse_args()
 
     from paper_2311_09445_b200 import workloads as wk
+    if args.sweep:
+        if int(os.environ.get("RANK", 0)) == 0:
+            print(json.dumps(run_sweep(args)), flush=True)
+        return
     wl = wk.WORKLOADS[args.workload]
     if args.capacity:
         wl = wk.scaled(wl, args.capacity)

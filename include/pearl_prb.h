@@ -57,9 +57,11 @@ typedef struct pearl_layout {
 #define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out */
 #define PEARL_ST_STALE 32u         /* update_after_insert: the index was overwritten since it was sampled; entry skipped */
 
-/* Update batches larger than this are applied as consecutive sub-batches of this many entries, in
- * batch order, one launch each; the result is that of the whole batch (the last valid entry of a
- * repeated index still wins, and the tree is re-summed after every sub-batch). */
+/* The largest update batch one thread block handles.  A larger batch of priorities or TD errors is
+ * applied by one launch of many co-resident thread blocks (a cooperative launch; the last valid entry
+ * of a repeated index still wins); a larger batch of changes (pearl_prb_update_delta), or any larger
+ * batch on a device without cooperative launches, as consecutive sub-batches of this many entries in
+ * batch order, one launch each.  The result is that of the whole batch either way. */
 #define PEARL_UPDATE_SUBBATCH 4096u
 
 /* Bytes of device memory a buffer of this geometry needs (tree, storage, scratch and the

@@ -511,6 +511,9 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     // leaf prefetch: when the level above the leaves is not staged, every walking lane group copies
     // the K*K leaves under its K nodes to shared memory while those nodes are on their way
     const bool prefetch = !uniform && v.depth >= 2 && plan.top_levels < v.depth - 1;
+    // All lane groups of a warp take the same path through the descent (its warp-wide barriers and
+    // ballots are met by every lane): the groups that prefetch are a whole number of warps' worth.
+    const uint32_t groups_per_warp = 32u / v.fanout;       // (fanout 32: one)
     const uint32_t pf_group_bytes = v.fanout * v.fanout * (uint32_t)sizeof(float);
     plan.pf_groups = 0;
     plan.pf_off = 0;
@@ -543,6 +546,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
             // strata a CTA can touch: its share of the tasks, plus one for a range that straddles
             const uint32_t tasks_per_cta = (sp.n_tasks + grid - 1) / grid;
             uint32_t strata = (tasks_per_cta + plan.tps - 1) / plan.tps + 1;
+            strata = (strata + groups_per_warp - 1) / groups_per_warp * groups_per_warp;
             if (strata > R) strata = R;
             uint32_t pf_bytes = prefetch ? strata * pf_group_bytes : 0u;
             uint32_t ring_bytes = dyn_max[dev][ki] - kRingBarBytes;
@@ -564,6 +568,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
             grid = want < one_wave ? want : one_wave;
             if (prefetch) {
                 uint32_t strata = (strata_here + grid - 1) / grid;
+                strata = (strata + groups_per_warp - 1) / groups_per_warp * groups_per_warp;
                 if (strata > R) strata = R;
                 sp.pf_groups = strata;
                 smem = strata * pf_group_bytes;

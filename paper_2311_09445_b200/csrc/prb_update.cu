@@ -45,6 +45,168 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top);
 }
 
+// ---- large batches: one launch of many CTAs ------------------------------------------------------
+// A batch beyond one CTA's reach is updated by a grid of co-resident CTAs (a cooperative launch)
+// whose phases are separated by a grid-wide barrier.  Nothing is sorted and no scratch is used:
+//   1. every valid entry b raises the bits of its leaf to 0x80000000 | b with an atomic maximum --
+//      a pattern above every valid priority (those are non-negative), so after the barrier the
+//      leaf names the LAST valid entry of the batch that writes it;
+//   2. the entry that finds its own number there stores its priority (last writer wins);
+//   3. level by level, deepest first, the parents above the named leaves are re-summed from their
+//      children, left to right in binary32: per entry (the first of consecutive entries with the same
+//      parent) while a level has many more nodes than the batch has entries, the whole level once it
+//      has not.  Re-summing a parent none of whose children changed gives back what it held, so
+//      an entry that was refused for its priority may take part and duplicates only cost time;
+//   4. CTA 0 stages the top of the tree in shared memory and re-sums it whole (prb_top_passes).
+// The barrier's wait is bounded: a CTA that gives up raises PEARL_ST_INTERNAL and returns.
+constexpr uint32_t kWideThreads = 256;
+constexpr uint32_t kWideSpinLimit = 1u << 22;
+
+struct PrbWideEntry {
+    bool valid;
+    uint32_t i;
+    float p;
+    unsigned flags;
+};
+
+__device__ __forceinline__ PrbWideEntry prb_wide_classify(const PrbView& v, int32_t i, float x, int raw, float alpha, float eps,
+                                                          unsigned long long fill, uint64_t cursor, uint32_t stale)
+{
+    PrbWideEntry e = PrbWideEntry{false, 0u, 0.0f, 0u};
+    const uint64_t N = v.capacity;
+    if (i < 0 || (unsigned long long)i >= fill) { e.flags = PEARL_ST_BAD_INDEX; return e; }
+    // one of the `stale` slots written most recently: overwritten since it was sampled
+    if (stale && (cursor + N - 1 - (uint64_t)i) % N < stale) { e.flags = PEARL_ST_STALE; return e; }
+    float p = x;
+    const bool ok = raw ? prb_valid_priority(p) : prb_priority_pow(x, eps, alpha, p);
+    if (!ok) { e.flags = PEARL_ST_BAD_PRIORITY; return e; }
+    e.valid = true;
+    e.i = (uint32_t)i;
+    e.p = p;
+    return e;
+}
+
+// All CTAs of the (co-resident) grid meet; what any of them wrote to global memory before is
+// visible, through L2, to all of them after.  `passed` counts the barriers this CTA has been through.
+// Returns false if the wait ran out.
+__device__ __forceinline__ bool prb_grid_barrier(PrbState* st, uint32_t& passed, uint32_t nctas, int* s_ok)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&st->wide_arrived, 1u);
+        const uint32_t target = (passed + 1u) * nctas;
+        int ok = 1;
+        for (uint32_t spins = 0;; ++spins) {
+            uint32_t seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->wide_arrived) : "memory");
+            if (seen >= target) break;
+            if (spins >= kWideSpinLimit) { ok = 0; break; }
+            __nanosleep(32);
+        }
+        __threadfence();
+        *s_ok = ok;
+    }
+    __syncthreads();
+    ++passed;
+    return *s_ok != 0;
+}
+
+__global__ void __launch_bounds__(kWideThreads)
+prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
+                       const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ unsigned s_flags, s_maxbits;
+    __shared__ int s_ok;
+    const uint32_t tid = threadIdx.x, nctas = gridDim.x;
+    const uint32_t gthreads = nctas * kWideThreads, gtid = blockIdx.x * kWideThreads + tid;
+    const unsigned long long fill = v.state->fill;
+    const uint64_t cursor = stale ? v.state->cursor : 0ull;
+    const uint32_t K = v.fanout, lg = v.log2_fanout, D = v.depth, T = v.top_levels;
+    unsigned* leaf_bits = reinterpret_cast<unsigned*>(v.level[D]);
+    if (tid == 0) { s_flags = 0u; s_maxbits = 0u; }
+    __syncthreads();
+
+    // 1. validate, transform, name the last writer of every leaf (a thread's first entry stays in registers)
+    PrbWideEntry first = PrbWideEntry{false, 0u, 0.0f, 0u};
+    unsigned flags = 0u;
+    float wmax = 0.0f;
+    for (uint32_t b = gtid; b < B; b += gthreads) {
+        const PrbWideEntry e = prb_wide_classify(v, idx[b], val[b], raw, alpha, eps, fill, cursor, stale);
+        if (b == gtid) first = e;
+        flags |= e.flags;
+        if (e.valid) { wmax = fmaxf(wmax, e.p); atomicMax(leaf_bits + e.i, 0x80000000u | b); }
+    }
+    flags = __reduce_or_sync(0xFFFFFFFFu, flags);
+    const unsigned mbits = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(wmax));
+    if ((tid & 31u) == 0) {
+        if (flags) atomicOr(&s_flags, flags);
+        if (mbits) atomicMax(&s_maxbits, mbits);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (s_flags) atomicOr(&v.state->status, s_flags);
+        if (s_maxbits) atomicMax(&v.state->max_prio_bits, s_maxbits);
+    }
+    uint32_t passed = 0;
+    bool alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
+
+    // 2. the named entry writes the leaf
+    if (alive) {
+        for (uint32_t b = gtid; b < B; b += gthreads) {
+            const PrbWideEntry e = (b == gtid) ? first : prb_wide_classify(v, idx[b], val[b], raw, alpha, eps, fill, cursor, stale);
+            if (e.valid && __ldcg(leaf_bits + e.i) == (0x80000000u | b)) v.level[D][e.i] = e.p;
+        }
+        alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
+    }
+
+    // 3. the levels below the staged top, deepest first
+    for (int l = (int)D - 1; alive && l >= (int)T; --l) {
+        const uint32_t sh = lg * (D - (uint32_t)l);
+        const uint64_t n_l = ((v.capacity - 1) >> sh) + 1;        // nodes of level l
+        float* parents = v.level[l];
+        const float* children = v.level[l + 1];
+        if (n_l <= 2ull * B) {
+            for (uint64_t a = gtid; a < n_l; a += gthreads) parents[a] = prb_sum_children_dyn(children + a * K, K);
+        } else {
+            for (uint32_t b = gtid; b < B; b += gthreads) {
+                const int32_t i = idx[b];
+                if (i < 0 || (unsigned long long)i >= fill) continue;
+                const uint64_t a = (uint64_t)i >> sh;
+                if (b > 0) {
+                    const int32_t before = idx[b - 1];
+                    if (before >= 0 && (unsigned long long)before < fill && ((uint64_t)before >> sh) == a) continue;
+                }
+                parents[a] = prb_sum_children_dyn(children + a * K, K);
+            }
+        }
+        alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
+    }
+    if (!alive) {
+        if (tid == 0) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
+        return;
+    }
+    // every CTA is past its last barrier: the last one to say so clears the barrier for the next launch
+    if (tid == 0 && atomicAdd(&v.state->wide_done, 1u) == nctas - 1) {
+        v.state->wide_arrived = 0u;
+        v.state->wide_done = 0u;
+    }
+    // 4. the staged levels
+    if (blockIdx.x == 0 && T > 0) {
+        PrbTop top;
+        top.mem = reinterpret_cast<float*>(smem);
+        prb_top_begin(v, top, tid, kWideThreads);
+        prb_top_wait();
+        __syncthreads();
+        PrbTeam team;
+        team.rank = tid;
+        team.size = kWideThreads;
+        team.whole_cta = true;
+        prb_top_passes(v, top, team, T);
+    }
+}
+
 // Priority retrieval: one thread per entry.
 __global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
                                           float* __restrict__ out)
@@ -71,11 +233,53 @@ uint32_t prb_update_ctas(const PrbView& v, uint32_t b)
     return (v.fanout * b >= 8192u) ? 8u : 1u;
 }
 
+// The many-CTA update of a large batch: 1 launch, or 0 if this device cannot run it (no cooperative
+// launch), or -1 on a launch error.
+static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
+                                  float alpha, float eps, cudaStream_t s, uint32_t stale)
+{
+    static int ctas_per_sm[kPrbMaxDevices];      // 0: not asked yet, -1: not available
+    const int dev = prb_current_device();
+    const size_t smem = (size_t)kPrbTopFloats * sizeof(float);
+    if (ctas_per_sm[dev] == 0) {
+        int coop = 0, nb = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, prb_update_wide_kernel, (int)kWideThreads, smem) != cudaSuccess || nb < 1) {
+            cudaGetLastError();
+            ctas_per_sm[dev] = -1;
+        } else {
+            ctas_per_sm[dev] = nb > 2 ? 2 : nb;
+        }
+    }
+    if (ctas_per_sm[dev] < 0) return 0;
+    uint32_t grid = (B + kWideThreads - 1) / kWideThreads;
+    const uint32_t room = (uint32_t)(prb_sm_count() * ctas_per_sm[dev]);
+    if (grid > room) grid = room;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kWideThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, prb_update_wide_kernel, v, B, d_idx, d_val, raw, alpha, eps, stale) != cudaSuccess) return -1;
+    return 1;
+}
+
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale,
                       uint32_t ins_n, const float* ins_prio, uint32_t ticket_total)
 {
     if (ins_n && B > PEARL_UPDATE_SUBBATCH) return -1;
+    // a batch of more than one entry per thread of a CTA: one launch of many CTAs (values or TD errors;
+    // changes keep their batch order and go sub-batch by sub-batch below)
+    if (B > kPrbWideFrom && raw != 2 && ins_n == 0 && B < 0x80000000u) {
+        const int k = prb_launch_update_wide(v, B, d_idx, d_val, raw, alpha, eps, s, stale);
+        if (k != 0) return k;
+    }
     static bool big_smem[kPrbMaxDevices];
     const int dev = prb_current_device();
     if (!big_smem[dev]) {

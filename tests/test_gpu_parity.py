@@ -269,6 +269,24 @@ def test_largest_sweep_capacity(oracle_mod, K):
     pr.close()
 
 
+@pytest.mark.parametrize("K,N,B", [(2, 1 << 16, 16384), (2, 5000, 5), (4, 5000, 5), (4, 20_000, 2001), (8, 40_000, 3),
+                                   (8, 40_000, 1100), (16, 70_000, 3), (16, 70_000, 777)])
+def test_sample_with_a_ragged_last_warp(oracle_mod, K, N, B):
+    # The strata of a CTA need not fill its last warp of lane groups (several groups share a warp
+    # below fanout 32) while the leaves are prefetched: every group of the warp walks all the same.
+    rng = np.random.default_rng(K + N + B)
+    pr = Pair(oracle_mod, N, K, 8, 4, max(B, 4096))
+    for first in range(0, N, 4096):
+        n = min(4096, N - first)
+        b = raw_fields(rng, n, 8, 4)
+        b["prio"] = rng.uniform(0.01, 1, n).astype(np.float32)
+        pr.insert(b)
+    for _ in range(3):
+        pr.sample(B, 0.4, 3)
+    pr.compare_status()
+    pr.close()
+
+
 def test_degenerate_sampling_cases(oracle_mod):
     rng = np.random.default_rng(17)
     pr = Pair(oracle_mod, 300, 16, 68, 24, 128)
@@ -462,6 +480,49 @@ def test_update_beyond_one_subbatch(oracle_mod, K, B):
         pr.compare_tree()
         assert pr.compare_status() == 1
     pr.compare_state()
+    pr.close()
+
+
+@pytest.mark.parametrize("K,N,B", [(2, 1 << 20, 5000), (4, 300_000, 8192), (16, 1 << 20, 20_000), (32, 1 << 19, 65536),
+                                   (16, 9000, 4097), (8, 70_000, 30_011)])
+def test_many_cta_update(oracle_mod, K, N, B):
+    # Batches beyond one CTA's reach go to one launch of many CTAs: values and TD errors, sorted and
+    # shuffled, sparse (levels with far more nodes than entries) and dense, with repeated indices,
+    # refused priorities, indices out of range and entries made stale by an insertion.
+    rng = np.random.default_rng(K * 7 + N + B)
+    pr = Pair(oracle_mod, N, K, 0, 0, 65536)
+    fill = N - 37
+    for first in range(0, fill, 65536):
+        pr.insert(dict(prio=rng.uniform(0.1, 1, min(65536, fill - first)).astype(np.float32)))
+    pr.compare_tree()
+    seen = 0
+    for step in range(4):
+        idx = rng.integers(0, fill, size=B).astype(np.int32)
+        if step % 2 == 0:
+            idx.sort()                                   # as a stratified sample returns them
+        rep = rng.integers(0, B, size=B // 10)
+        idx[rep] = idx[rng.integers(0, B, size=B // 10)]          # repeats anywhere in the batch
+        idx[rng.integers(0, B, size=7)] = [-1, N, fill, N - 1, 2 ** 31 - 1, -2 ** 31, fill + 5]
+        td = (rng.standard_normal(B) * 3).astype(np.float32)
+        td[rng.integers(0, B, size=3)] = [np.nan, np.inf, -np.inf]
+        if step == 1:
+            prio = np.abs(td)
+            prio[rng.integers(0, B, size=2)] = [-1.0, np.nan]
+            pr.update_priorities(idx, prio)
+        elif step == 3:
+            pr.insert(dict(prio=rng.uniform(0.1, 1, 777).astype(np.float32)))
+            idx[rng.integers(0, B, size=50)] = (pr.ora.info()[1] - 1 - rng.integers(0, 777, size=50)) % N   # just overwritten
+            pr.update_after_insert(idx, td, 0.6, 1e-6, 777)
+        else:
+            pr.update(idx, td, 0.6, 1e-6)
+        pr.compare_tree()
+        seen |= pr.compare_status()
+        pr.compare_state()
+    assert seen & 1 and seen & 2 and seen & 32            # bad index, bad priority, stale
+    # and the buffer still samples identically afterwards (only priorities were stored: no rows to compare)
+    o, g = pr.sample(256, 0.4, 5, check=False)
+    assert np.array_equal(o["idx"], g["idx"])
+    np.testing.assert_allclose(g["w"], o["w"], rtol=1e-5, atol=0)
     pr.close()
 
 
