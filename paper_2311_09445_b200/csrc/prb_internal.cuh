@@ -21,6 +21,7 @@ struct PrbState {
     unsigned int max_prio_bits;       // bits of the largest priority written so far (0: none yet)
     unsigned int wide_arrived;        // grid barrier of the running many-CTA update: arrivals so far (0 between launches)
     unsigned int wide_done;           // its CTAs that have passed their last barrier
+    unsigned long long wide_wmax_bits; // largest raw weight of the running large-batch sample (bits of a binary64; 0 between calls)
 };
 
 // Geometry and device addresses, passed to kernels by value.

@@ -423,6 +423,182 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     }
 }
 
+// ---- large batches of short rows: one stratum per thread -------------------------------------------
+// With thousands of strata the K-lane groups above keep too few tree reads in flight (a CTA walks
+// 256 / K strata at a time, round after round).  Here every thread walks a stratum of its own: it
+// loads the K children of its node itself (one 8..128-byte group: whole sectors), forms the same
+// left-to-right binary32 prefix sums one after another and enters the first child whose prefix
+// exceeds the binary64 target -- the count of prefixes the target has passed, as the lanes' ballot
+// gives it.  A CTA takes a contiguous range of strata, 256 at a time: targets, descents, index and raw
+// weight per thread; then all its threads copy the rows, granule by granule (consecutive threads,
+// consecutive granules), eight loads in flight each.  Every CTA raises the batch's largest raw
+// weight with one atomic maximum (positive binary64 values order like their bit patterns); the last
+// CTA to finish (ticket) divides all raw weights by it.
+constexpr uint32_t kWideSampleFrom = 2048;      // batches of at least this many strata (short rows)
+constexpr uint32_t kWideSampleStrata = 32;      // ... spread over CTAs of at least this many strata
+
+template <int K>
+__device__ __forceinline__ void load_children(const float* src, bool global, float (&c)[K])
+{
+    if (K == 2) {
+        const float2 t = global ? __ldg(reinterpret_cast<const float2*>(src)) : *reinterpret_cast<const float2*>(src);
+        c[0] = t.x; c[1] = t.y;
+    } else {
+#pragma unroll
+        for (int q = 0; q < K / 4; ++q) {
+            const float4 t = global ? __ldg(reinterpret_cast<const float4*>(src) + q) : reinterpret_cast<const float4*>(src)[q];
+            c[4 * q] = t.x; c[4 * q + 1] = t.y; c[4 * q + 2] = t.z; c[4 * q + 3] = t.w;
+        }
+    }
+}
+
+template <int K>
+__device__ __forceinline__ void descend_alone(const PrbView& v, const SamplePlan& plan, const float* s_top, double x,
+                                              uint32_t& leaf, float& p_leaf, unsigned& flags)
+{
+    uint64_t g = 0;
+    float chosen = 0.0f;
+    for (uint32_t l = 1; l <= v.depth; ++l) {
+        float c[K];
+        const bool staged = l <= plan.top_levels;
+        load_children<K>(staged ? s_top + plan.top_off[l] + (uint32_t)g * K : v.level[l] + g * K, !staged, c);
+        int j = -1, last_pos = -1;
+        float run = 0.0f, before_j = 0.0f, before_last = 0.0f;
+#pragma unroll
+        for (int q = 0; q < K; ++q) {
+            const float before = run;                          // prefix q-1 (0 in front of the first child)
+            run = (q == 0) ? c[0] : __fadd_rn(run, c[q]);
+            if (j < 0 && !(x >= (double)run)) { j = q; before_j = before; chosen = c[q]; }
+            if (c[q] > 0.0f) { last_pos = q; before_last = before; }
+        }
+        if (j < 0) {
+            // the target has passed every prefix (possible only by binary32 rounding): last positive child
+            flags |= PEARL_ST_CLAMPED;
+            if (last_pos >= 0) { j = last_pos; before_j = before_last; }
+            else { j = 0; before_j = 0.0f; flags |= PEARL_ST_INTERNAL; }
+            chosen = 0.0f;
+#pragma unroll
+            for (int q = 0; q < K; ++q) if (q == j) chosen = c[q];
+        }
+        if (j > 0) x = __dsub_rn(x, (double)before_j);
+        g = g * K + (uint64_t)j;
+    }
+    p_leaf = chosen;
+    leaf = (uint32_t)g;
+}
+
+// Short rows of strata [k_first, k_first + n_rows) by all `nthreads` threads, field by field, up to
+// eight granules per thread loaded before the first is stored.
+__device__ __forceinline__ void gather_short_fields_deep(const PrbView& v, const PrbBatch& dst, uint32_t k_first, uint32_t n_rows,
+                                                         const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
+{
+    constexpr int U = 8;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+        const uint64_t dbase = (uint64_t)k_first * W;
+        for (uint32_t e0 = rank; e0 < total; e0 += nthreads * U) {
+            uint4 tmp[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t e = e0 + u * nthreads;
+                if (e < total) {
+                    const uint32_t r = (W == 1) ? e : e / W;
+                    tmp[u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t e = e0 + u * nthreads;
+                if (e < total) store_granule(dst.ptr[f], dbase + e, vec, tmp[u]);
+            }
+        }
+    }
+}
+
+template <int K>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uint64_t seed,
+                       int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
+                       const __grid_constant__ SamplePlan plan)
+{
+    __shared__ __align__(16) float s_top[top_floats_of(K)];
+    __shared__ uint32_t s_idx[kThreads];
+    __shared__ unsigned long long s_wmax;
+    __shared__ unsigned s_flags;
+    __shared__ unsigned int s_last;
+    const uint32_t tid = threadIdx.x;
+    const unsigned long long calls = v.state->sample_calls;
+    const unsigned long long fill = v.state->fill;
+    const float total32 = __ldg(v.level[0]);
+    {
+        const float4* src = reinterpret_cast<const float4*>(v.level[1]);
+        for (uint32_t q = tid; q < plan.top_vec4; q += kThreads) reinterpret_cast<float4*>(s_top)[q] = __ldg(src + q);
+    }
+    if (tid == 0) { s_wmax = 0ull; s_flags = 0u; }
+    const bool empty = (fill == 0) || !(total32 > 0.0f);
+    const double total = (double)total32;
+    const uint32_t k_lo = (uint32_t)(((uint64_t)blockIdx.x * B) / gridDim.x);
+    const uint32_t k_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * B) / gridDim.x);
+    __syncthreads();
+    unsigned long long my_wmax = 0ull;
+    unsigned my_flags = 0u;
+    for (uint32_t kb = k_lo; kb < k_hi && !empty; kb += kThreads) {
+        const uint32_t k = kb + tid, n_here = min(kThreads, k_hi - kb);
+        if (k < k_hi) {
+            // target of stratum k (Eq. 1's x, one per equal segment of the total), then the walk
+            const double seg = __ddiv_rn(total, (double)B);
+            const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32), (uint32_t)seed, (uint32_t)(seed >> 32));
+            const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
+            double x = __dmul_rn(__dadd_rn((double)k, u), seg);
+            if (x >= total) x = __longlong_as_double(__double_as_longlong(total) - 1);   // next binary64 below total
+            uint32_t leaf; float p;
+            descend_alone<K>(v, plan, s_top, x, leaf, p, my_flags);
+            s_idx[tid] = leaf;
+            out_idx[k] = (int32_t)leaf;
+            if (out_w != nullptr) {
+                const double wr = pow(__ddiv_rn(__dmul_rn((double)fill, (double)p), total), -(double)beta);
+                v.wraw[k] = wr;
+                my_wmax = max(my_wmax, (unsigned long long)__double_as_longlong(wr));
+            }
+        }
+        __syncthreads();
+        gather_short_fields_deep(v, dst, kb, n_here, s_idx, tid, kThreads);
+        __syncthreads();            // s_idx is rewritten by the next pass
+    }
+    if (my_wmax) atomicMax(&s_wmax, my_wmax);
+    if (my_flags) atomicOr(&s_flags, my_flags);
+    __threadfence();                // this thread's raw weights are in L2 before the CTA takes its ticket
+    __syncthreads();
+    if (tid == 0) {
+        if (s_flags) atomicOr(&v.state->status, s_flags);
+        if (s_wmax) atomicMax(&v.state->wide_wmax_bits, s_wmax);
+        __threadfence();
+        s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    // the last CTA: every raw weight and the batch maximum are in L2
+    if (empty) {
+        if (tid == 0) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+    } else if (out_w != nullptr) {
+        const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wide_wmax_bits));
+        for (uint32_t k0 = tid; k0 < B; k0 += kThreads * 4u) {
+            double held[4];
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) held[u] = __ldcg(v.wraw + k0 + u * kThreads);
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) out_w[k0 + u * kThreads] = (float)__ddiv_rn(held[u], wmax);
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (!empty) v.state->sample_calls = calls + 1;
+        v.state->wide_wmax_bits = 0ull;
+        v.state->sample_ticket = 0u;
+    }
+}
+
 // The smallest positive leaf among the `fill` stored ones, into state->pmin_bits (all ones at creation and
 // again after every sample that used it): positive binary32 values order like their bit patterns.
 __global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
@@ -489,6 +665,22 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     }
     const uint32_t R = kThreads / v.fanout;
     const int ki = v.log2_fanout;
+    if (!row_mode && n_sub == 1 && !uniform && !buffer_norm && B >= kWideSampleFrom) {
+        // a large batch of short rows: one stratum per thread
+        uint32_t grid = (B + kWideSampleStrata - 1) / kWideSampleStrata;
+        const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;
+        if (grid > one_wave) grid = one_wave;
+        plan.ring_stages = 0; plan.ring_stage_bytes = 0; plan.pf_groups = 0; plan.pf_off = 0;
+        plan.ticket_total = grid;
+        switch (v.fanout) {
+        case 2: prb_sample_wide_kernel<2><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+        case 4: prb_sample_wide_kernel<4><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+        case 8: prb_sample_wide_kernel<8><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+        case 16: prb_sample_wide_kernel<16><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+        default: prb_sample_wide_kernel<32><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
+        }
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    }
     // dynamic shared memory a CTA of this kernel may have: what the device allows less its static part
     static uint32_t dyn_max[kPrbMaxDevices][6];
     if (dyn_max[dev][ki] == 0) {

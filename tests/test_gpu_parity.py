@@ -270,7 +270,8 @@ def test_largest_sweep_capacity(oracle_mod, K):
 
 
 @pytest.mark.parametrize("K,N,B", [(2, 1 << 16, 16384), (2, 5000, 5), (4, 5000, 5), (4, 20_000, 2001), (8, 40_000, 3),
-                                   (8, 40_000, 1100), (16, 70_000, 3), (16, 70_000, 777)])
+                                   (8, 40_000, 1100), (16, 70_000, 3), (16, 70_000, 777), (4, 20_000, 2049), (8, 40_000, 5000),
+                                   (32, 100_000, 3333), (16, 70_000, 2048)])
 def test_sample_with_a_ragged_last_warp(oracle_mod, K, N, B):
     # The strata of a CTA need not fill its last warp of lane groups (several groups share a warp
     # below fanout 32) while the leaves are prefetched: every group of the warp walks all the same.
@@ -284,6 +285,34 @@ def test_sample_with_a_ragged_last_warp(oracle_mod, K, N, B):
     for _ in range(3):
         pr.sample(B, 0.4, 3)
     pr.compare_status()
+    pr.close()
+
+
+@pytest.mark.parametrize("K", FANOUTS)
+@pytest.mark.parametrize("B", [2048, 4099, 20_000])
+def test_large_batch_sample_cases(oracle_mod, K, B):
+    # Large batches of short rows take the one-stratum-per-thread kernel: most leaves zero, the rest
+    # spread over many orders of magnitude (prefix sums that round), every beta, weights optional.
+    rng = np.random.default_rng(K * 31 + B)
+    N = 50_000
+    pr = Pair(oracle_mod, N, K, 12, 4, max(B, 4096))
+    for first in range(0, N - 3, 4096):
+        n = min(4096, N - 3 - first)
+        b = raw_fields(rng, n, 12, 4)
+        p = np.exp(4.0 * rng.standard_normal(n)).astype(np.float32)
+        p[rng.random(n) < 0.9] = 0.0
+        b["prio"] = p
+        pr.insert(b)
+    for beta in (0.0, 0.4, 1.0):
+        pr.sample(B, beta, 17)
+    pr.compare_status()
+    # the same call without weights leaves the state as the oracle's
+    t = torch.full((B,), -1, dtype=torch.int32, device=pr.dev)
+    pr.gpu.sample(B, 0.4, 17, t)
+    o = pr.ora.sample(B, 0.4, 17, gather=False)
+    assert np.array_equal(o["idx"], t.cpu().numpy())
+    pr.sample(B, 0.4, 17)
+    pr.compare_state()
     pr.close()
 
 
