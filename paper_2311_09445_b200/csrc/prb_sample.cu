@@ -432,8 +432,8 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 // gives it.  A CTA takes a contiguous range of strata, 256 at a time: targets, descents, index and raw
 // weight per thread; then all its threads copy the rows, granule by granule (consecutive threads,
 // consecutive granules), eight loads in flight each.  Every CTA raises the batch's largest raw
-// weight with one atomic maximum (positive binary64 values order like their bit patterns); the last
-// CTA to finish (ticket) divides all raw weights by it.
+// weight with one atomic maximum (positive binary64 values order like their bit patterns); a second,
+// small launch divides all raw weights by it.
 constexpr uint32_t kWideSampleFrom = 2048;      // batches of at least this many strata (short rows)
 constexpr uint32_t kWideSampleStrata = 32;      // ... spread over CTAs of at least this many strata
 
@@ -568,32 +568,39 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
     }
     if (my_wmax) atomicMax(&s_wmax, my_wmax);
     if (my_flags) atomicOr(&s_flags, my_flags);
-    __threadfence();                // this thread's raw weights are in L2 before the CTA takes its ticket
     __syncthreads();
     if (tid == 0) {
         if (s_flags) atomicOr(&v.state->status, s_flags);
         if (s_wmax) atomicMax(&v.state->wide_wmax_bits, s_wmax);
-        __threadfence();
         s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
     }
     __syncthreads();
-    if (!s_last) return;
-    // the last CTA: every raw weight and the batch maximum are in L2
-    if (empty) {
-        if (tid == 0) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-    } else if (out_w != nullptr) {
-        const double wmax = __longlong_as_double((long long)__ldcg(&v.state->wide_wmax_bits));
-        for (uint32_t k0 = tid; k0 < B; k0 += kThreads * 4u) {
-            double held[4];
-#pragma unroll
-            for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) held[u] = __ldcg(v.wraw + k0 + u * kThreads);
-#pragma unroll
-            for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) out_w[k0 + u * kThreads] = (float)__ddiv_rn(held[u], wmax);
-        }
+    if (tid == 0 && s_last) {
+        // the last CTA to finish: the call's bookkeeping (the weights are divided by a launch of their own)
+        if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+        else v.state->sample_calls = calls + 1;
+        v.state->sample_ticket = 0u;
     }
-    __syncthreads();
-    if (tid == 0) {
-        if (!empty) v.state->sample_calls = calls + 1;
+}
+
+// Second launch of a large-batch sample: w_k = raw weight / the batch's largest, by as many CTAs as
+// it takes (one CTA would need B / 1024 dependent round trips).  The largest raw weight is zero only
+// if the buffer was empty: then nothing is written.  The last CTA to have read it clears it.
+__global__ void __launch_bounds__(kThreads)
+prb_normalise_weights_kernel(const __grid_constant__ PrbView v, uint32_t B, float* __restrict__ out_w)
+{
+    const unsigned long long bits = __ldcg(&v.state->wide_wmax_bits);
+    if (bits) {
+        const double wmax = __longlong_as_double((long long)bits);
+        const uint32_t k0 = blockIdx.x * kThreads * 4u + threadIdx.x;
+        double held[4];
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) held[u] = __ldcg(v.wraw + k0 + u * kThreads);
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) out_w[k0 + u * kThreads] = (float)__ddiv_rn(held[u], wmax);
+    }
+    __syncthreads();        // every thread of the CTA has read the maximum
+    if (threadIdx.x == 0 && atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) {
         v.state->wide_wmax_bits = 0ull;
         v.state->sample_ticket = 0u;
     }
@@ -679,7 +686,8 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         case 16: prb_sample_wide_kernel<16><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
         default: prb_sample_wide_kernel<32><<<grid, kThreads, 0, s>>>(v, B, beta, seed, d_idx, d_w, dst, plan); break;
         }
-        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+        if (d_w != nullptr) prb_normalise_weights_kernel<<<(B + kThreads * 4u - 1) / (kThreads * 4u), kThreads, 0, s>>>(v, B, d_w);
+        return cudaGetLastError() == cudaSuccess ? (d_w != nullptr ? 2 : 1) : -1;
     }
     // dynamic shared memory a CTA of this kernel may have: what the device allows less its static part
     static uint32_t dyn_max[kPrbMaxDevices][6];
