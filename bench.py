@@ -509,6 +509,7 @@ def run_sweep(args):
     dev = torch.device("cuda:0")
     stream = torch.cuda.Stream(dev)
     caps = [c for c in SWEEP_CAPACITIES if not args.capacity or c == args.capacity]
+    fanouts = [k for k in SWEEP_FANOUTS if not args.sweep_fanout or k == args.sweep_fanout]
     gen = torch.Generator(device=dev)
     rows = []
     clocks = ClockSampler(0)
@@ -516,10 +517,12 @@ def run_sweep(args):
     t_start = time.time()
     with torch.cuda.stream(stream):
         for N in caps:
-            for K in SWEEP_FANOUTS:
+            for K in fanouts:
                 wl = wk.sweep_cell(N, K, 1024, cell_id=0)
                 gen.manual_seed(wl.seed + N % 997 + K)
-                batches_B = [b for b in SWEEP_BATCHES if b <= N // 2]
+                batches_B = [b for b in SWEEP_BATCHES if b <= N // 2 and (not args.sweep_batch or b == args.sweep_batch)]
+                if not batches_B:
+                    continue
                 chunk = min(N, 1 << 16)
                 prb = PrioritizedReplay(N, K, wl.obs_bytes, wl.act_bytes, max(chunk, max(batches_B)), device=dev, stream=stream)
 
@@ -636,6 +639,8 @@ def main():
                     help="time only the step and its three calls (no shuffled-update, streamed or buffer-normalised sample timings)")
     ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
+    ap.add_argument("--sweep-fanout", type=int, default=0, help="with --sweep: this fanout only")
+    ap.add_argument("--sweep-batch", type=int, default=0, help="with --sweep: this batch size only")
     ap.add_argument("--sweep", action="store_true",
                     help="time every cell of the capacity x fanout x batch sweep instead (one GPU; --capacity picks one capacity)")
     args = ap.parse_args()
