@@ -167,7 +167,8 @@ int pearl_prb_get_priorities(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx,
  * pearl_prb_update(prb, B, d_idx, d_td, alpha, eps) followed by pearl_prb_insert(prb, n, ...): the
  * update's tree work is done first, the insertion's tree work after it, by the same thread blocks,
  * while other thread blocks already copy the new rows into the Data Storage (an update touches
- * the tree only, so the two do not conflict).  Short rows: one launch.  Rows of 8 KB and more: the
+ * the tree only, so the two do not conflict).  Short rows: one launch (update batches of 1024 entries
+ * and more: the update's launch, then the insertion's).  Rows of 8 KB and more: the
  * tree work is a kernel of its own on a second stream of the handle, beside the kernel that copies
  * the rows; the handle's stream continues when both are done (capturable in a CUDA graph).  This
  * is the overlap of the paper's training

@@ -431,7 +431,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 // exceeds the binary64 target -- the count of prefixes the target has passed, as the lanes' ballot
 // gives it.  A CTA takes a contiguous range of strata, 256 at a time: targets, descents, index and raw
 // weight per thread; then all its threads copy the rows, granule by granule (consecutive threads,
-// consecutive granules), eight loads in flight each.  Every CTA raises the batch's largest raw
+// consecutive granules), up to sixteen loads in flight each.  Every CTA raises the batch's largest raw
 // weight with one atomic maximum (positive binary64 values order like their bit patterns); a second,
 // small launch divides all raw weights by it.
 constexpr uint32_t kWideSampleFrom = 2048;      // batches of at least this many strata (short rows)
@@ -487,31 +487,44 @@ __device__ __forceinline__ void descend_alone(const PrbView& v, const SamplePlan
     leaf = (uint32_t)g;
 }
 
-// Short rows of strata [k_first, k_first + n_rows) by all `nthreads` threads, field by field, up to
-// eight granules per thread loaded before the first is stored.
+// Short rows of strata [k_first, k_first + n_rows) by all `nthreads` threads, field by field, in
+// granules of type T: up to U granules per thread are loaded before the first is stored.
+template <typename T, int U>
+__device__ __forceinline__ void gather_field_deep(const T* __restrict__ store, T* __restrict__ out, uint32_t W, uint32_t total,
+                                                  const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
+{
+    for (uint32_t e0 = rank; e0 < total; e0 += nthreads * U) {
+        T tmp[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t e = e0 + u * nthreads;
+            if (e < total) {
+                const uint32_t r = (W == 1) ? e : e / W;
+                tmp[u] = store[(uint64_t)s_idx[r] * W + (e - r * W)];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t e = e0 + u * nthreads;
+            if (e < total) out[e] = tmp[u];
+        }
+    }
+}
+
 __device__ __forceinline__ void gather_short_fields_deep(const PrbView& v, const PrbBatch& dst, uint32_t k_first, uint32_t n_rows,
                                                          const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
 {
-    constexpr int U = 8;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
-        const uint64_t dbase = (uint64_t)k_first * W;
-        for (uint32_t e0 = rank; e0 < total; e0 += nthreads * U) {
-            uint4 tmp[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t e = e0 + u * nthreads;
-                if (e < total) {
-                    const uint32_t r = (W == 1) ? e : e / W;
-                    tmp[u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t e = e0 + u * nthreads;
-                if (e < total) store_granule(dst.ptr[f], dbase + e, vec, tmp[u]);
-            }
+        const unsigned char* src = v.store[f];
+        unsigned char* out = dst.ptr[f] + (uint64_t)k_first * v.field_bytes[f];
+        switch (vec) {
+        case 16: gather_field_deep<uint4, 4>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(out), W, total, s_idx, rank, nthreads); break;
+        case 8: gather_field_deep<uint2, 8>(reinterpret_cast<const uint2*>(src), reinterpret_cast<uint2*>(out), W, total, s_idx, rank, nthreads); break;
+        case 4: gather_field_deep<uint32_t, 16>(reinterpret_cast<const uint32_t*>(src), reinterpret_cast<uint32_t*>(out), W, total, s_idx, rank, nthreads); break;
+        case 2: gather_field_deep<uint16_t, 8>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(out), W, total, s_idx, rank, nthreads); break;
+        default: gather_field_deep<unsigned char, 8>(src, out, W, total, s_idx, rank, nthreads); break;
         }
     }
 }
