@@ -93,8 +93,9 @@ __device__ __forceinline__ bool prb_grid_barrier(PrbState* st, uint32_t& passed,
 {
     __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(&st->wide_arrived, 1u);
+        // arrival with release semantics (the CTA's writes, ordered before it by the barrier above, are
+        // visible to whoever then reads the counter with acquire semantics); no fence, no returned value
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&st->wide_arrived) : "memory");
         const uint32_t target = (passed + 1u) * nctas;
         int ok = 1;
         for (uint32_t spins = 0;; ++spins) {
@@ -102,9 +103,7 @@ __device__ __forceinline__ bool prb_grid_barrier(PrbState* st, uint32_t& passed,
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&st->wide_arrived) : "memory");
             if (seen >= target) break;
             if (spins >= kWideSpinLimit) { ok = 0; break; }
-            __nanosleep(32);
         }
-        __threadfence();
         *s_ok = ok;
     }
     __syncthreads();
