@@ -52,7 +52,8 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 //      a pattern above every valid priority (those are non-negative), so after the barrier the
 //      leaf names the LAST valid entry of the batch that writes it;
 //   2. the entry that finds its own number there stores its priority (last writer wins);
-//   3. level by level, deepest first, the parents above the named leaves are re-summed from their
+//   3. level by level, deepest first (fanouts 2 and 4: up to five and two levels per pass, a thread
+//      re-summing a whole small subtree), the parents above the named leaves are re-summed from their
 //      children, left to right in binary32: per entry (the first of consecutive entries with the same
 //      parent) while a level has many more nodes than the batch has entries, the whole level once it
 //      has not.  Re-summing a parent none of whose children changed gives back what it held, so
@@ -84,6 +85,72 @@ __device__ __forceinline__ PrbWideEntry prb_wide_classify(const PrbView& v, int3
     e.i = (uint32_t)i;
     e.p = p;
     return e;
+}
+
+// Several levels in one pass, for small fanouts (a pass costs a grid barrier): node a of level lt and
+// everything below it down to level lt + H - 1 are re-summed from the K^H entries of level lt + H
+// under it (one contiguous run of at most 128 bytes), level by level in registers, every sum left to
+// right as in a single-level pass.  Nodes past the end of a level are not written; entries past the end
+// of the children's array count as zero.
+template <int K, int H>
+__device__ __forceinline__ void prb_resum_subtree(const PrbView& v, uint32_t lt, uint64_t a)
+{
+    constexpr int M = (K == 2) ? (1 << H) : (1 << (2 * H));      // K^H for K = 2, 4
+    const uint32_t lb = lt + H - 1, D = v.depth, lg = v.log2_fanout;
+    const float* ch = v.level[lb + 1];
+    const uint64_t base = a * M, alloc = v.level_alloc[lb + 1];
+    float c[M];
+    if (K == 2 && base + M > alloc) {
+        // (the run ends inside the children's array, whose length is a multiple of the fanout only)
+#pragma unroll
+        for (int q = 0; q < M / 2; ++q) {
+            const float2 t = (base + 2 * q < alloc) ? __ldcg(reinterpret_cast<const float2*>(ch + base) + q) : make_float2(0.0f, 0.0f);
+            c[2 * q] = t.x; c[2 * q + 1] = t.y;
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < M / 4; ++q) {
+            const float4 t = (base + 4 * q < alloc) ? __ldcg(reinterpret_cast<const float4*>(ch + base) + q) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            c[4 * q] = t.x; c[4 * q + 1] = t.y; c[4 * q + 2] = t.z; c[4 * q + 3] = t.w;
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < H; ++s) {
+        const uint32_t m = lb - s;                                   // the level written in this step
+        const int cnt = M >> ((s + 1) * (K == 2 ? 1 : 2));           // its nodes under a: K^(H-1-s)
+        const uint64_t n_m = ((v.capacity - 1) >> (lg * (D - m))) + 1;
+        const uint64_t first = a * cnt;
+#pragma unroll
+        for (int j = 0; j < M / K; ++j) {
+            if (j < cnt) {
+                float x = c[j * K];
+#pragma unroll
+                for (int t = 1; t < K; ++t) x = __fadd_rn(x, c[j * K + t]);
+                if (first + j < n_m) v.level[m][first + j] = x;
+                c[j] = x;
+            }
+        }
+    }
+}
+
+// levels one pass takes when `left` levels are still to do: up to 32 entries under a node; with
+// tens of thousands of batch entries only two levels (the wider subtrees' extra reads and scattered
+// stores then cost more than the barriers they save: measured at 65536 entries)
+__device__ __forceinline__ uint32_t prb_levels_per_pass(uint32_t K, uint32_t left, uint32_t B)
+{
+    const uint32_t most = (K == 2) ? (B > 16384u ? 2u : 5u) : (K == 4) ? 2u : 1u;
+    return left < most ? left : most;
+}
+
+__device__ __forceinline__ void prb_resum_levels(const PrbView& v, uint32_t h, uint32_t lt, uint64_t a)
+{
+    if (v.fanout == 4) { prb_resum_subtree<4, 2>(v, lt, a); return; }
+    switch (h) {
+    case 2: prb_resum_subtree<2, 2>(v, lt, a); break;
+    case 3: prb_resum_subtree<2, 3>(v, lt, a); break;
+    case 4: prb_resum_subtree<2, 4>(v, lt, a); break;
+    default: prb_resum_subtree<2, 5>(v, lt, a); break;
+    }
 }
 
 // All CTAs of the (co-resident) grid meet; what any of them wrote to global memory before is
@@ -160,14 +227,17 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
     }
 
-    // 3. the levels below the staged top, deepest first
-    for (int l = (int)D - 1; alive && l >= (int)T; --l) {
-        const uint32_t sh = lg * (D - (uint32_t)l);
-        const uint64_t n_l = ((v.capacity - 1) >> sh) + 1;        // nodes of level l
-        float* parents = v.level[l];
-        const float* children = v.level[l + 1];
-        if (n_l <= 2ull * B) {
-            for (uint64_t a = gtid; a < n_l; a += gthreads) parents[a] = prb_sum_children_dyn(children + a * K, K);
+    // 3. the levels below the staged top, deepest first; small fanouts take several levels per pass
+    for (int l = (int)D - 1; alive && l >= (int)T;) {
+        const uint32_t h = prb_levels_per_pass(K, (uint32_t)l - T + 1u, B);
+        const uint32_t lt = (uint32_t)l - h + 1u;                 // the highest level this pass writes
+        const uint32_t sh = lg * (D - lt);
+        const uint64_t n_lt = ((v.capacity - 1) >> sh) + 1;       // nodes of level lt
+        if (n_lt <= 2ull * B) {
+            for (uint64_t a = gtid; a < n_lt; a += gthreads) {
+                if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
+                else prb_resum_levels(v, h, lt, a);
+            }
         } else {
             for (uint32_t b = gtid; b < B; b += gthreads) {
                 const int32_t i = idx[b];
@@ -177,10 +247,12 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
                     const int32_t before = idx[b - 1];
                     if (before >= 0 && (unsigned long long)before < fill && ((uint64_t)before >> sh) == a) continue;
                 }
-                parents[a] = prb_sum_children_dyn(children + a * K, K);
+                if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
+                else prb_resum_levels(v, h, lt, a);
             }
         }
         alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
+        l -= (int)h;
     }
     if (!alive) {
         if (tid == 0) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
