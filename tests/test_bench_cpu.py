@@ -63,3 +63,15 @@ def test_time_is_max_over_ranks_gloo():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert got == {0: 15.0, 1: 15.0}
+
+
+def test_sweep_grid_is_the_stated_one():
+    # capacity x fanout x batch, batches above half the capacity left out: 140 cells
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    cells = [(n, k, b) for n in bench.SWEEP_CAPACITIES for k in bench.SWEEP_FANOUTS for b in bench.SWEEP_BATCHES if b <= n // 2]
+    assert len(cells) == 140
+    assert bench.SWEEP_CAPACITIES[0] == 1 << 16 and bench.SWEEP_CAPACITIES[-1] == 1 << 26
+    assert bench.SWEEP_FANOUTS == [2, 4, 16, 32] and max(bench.SWEEP_BATCHES) == 65536
