@@ -3,9 +3,10 @@
 // mutex; here the leaf is SET and the ancestors are re-summed, so the result does not depend
 // on scheduling (see prb_update_team in prb_tree.cuh for the steps).
 //
-// One CTA, or eight CTAs of one thread-block cluster that share the deep levels: the batch is at most
-// a few thousand entries and the work is a chain of dependent L2 round trips, one per level below
-// the top of the tree, which is staged in shared memory.
+// Up to 1024 entries (and every batch of changes): one CTA, or eight CTAs of one thread-block cluster
+// that share the deep levels -- the work is a chain of dependent L2 round trips, one per level below
+// the top of the tree, which is staged in shared memory.  More entries: one cooperative launch of
+// many CTAs (prb_update_wide_kernel, below).
 #include "prb_tree.cuh"
 
 namespace {
@@ -46,7 +47,7 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 }
 
 // ---- large batches: one launch of many CTAs ------------------------------------------------------
-// A batch beyond one CTA's reach is updated by a grid of co-resident CTAs (a cooperative launch)
+// A batch of more than one entry per thread of a CTA is updated by a grid of co-resident CTAs (a cooperative launch)
 // whose phases are separated by a grid-wide barrier.  Nothing is sorted and no scratch is used:
 //   1. every valid entry b raises the bits of its leaf to 0x80000000 | b with an atomic maximum --
 //      a pattern above every valid priority (those are non-negative), so after the barrier the
