@@ -54,14 +54,23 @@ typedef struct pearl_layout {
                                       the entry, insert stores the row with priority 0 */
 #define PEARL_ST_EMPTY 4u          /* sample on an empty buffer or a non-positive total; outputs untouched */
 #define PEARL_ST_CLAMPED 8u        /* a descent met residual >= last prefix sum and took the last positive child */
-#define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out */
+#define PEARL_ST_INTERNAL 16u      /* inconsistent tree met during a descent, or a bounded wait ran out.
+                                      Every wait on the device (a bulk copy's completion, the grid barrier of
+                                      a large update) gives up after a fixed number of polls instead of
+                                      hanging.  After a copy that gave up, rows of that call are missing or
+                                      partial.  After an update of more than 1024 entries that gave up, the
+                                      tree is not consistent: leaves named by the batch may hold the marker
+                                      bit pattern 0x80000000|entry instead of a priority, and parents may not
+                                      equal the sum of their children.  Treat the buffer as lost: destroy it
+                                      and build a new one.  No correct run raises this bit. */
 #define PEARL_ST_STALE 32u         /* update_after_insert: the index was overwritten since it was sampled; entry skipped */
 
-/* The largest update batch one thread block handles.  A larger batch of priorities or TD errors is
- * applied by one launch of many co-resident thread blocks (a cooperative launch; the last valid entry
- * of a repeated index still wins); a larger batch of changes (pearl_prb_update_delta), or any larger
- * batch on a device without cooperative launches, as consecutive sub-batches of this many entries in
- * batch order, one launch each.  The result is that of the whole batch either way. */
+/* The largest update batch one thread block handles.  A batch of more than 1024 priorities or TD
+ * errors is applied by one launch of many co-resident thread blocks (a cooperative launch; the last
+ * valid entry of a repeated index still wins); a batch of changes (pearl_prb_update_delta) of any
+ * size, or any batch on a device without cooperative launches, by one thread block per sub-batch of
+ * at most this many entries, sub-batches in batch order, one launch each.  The result is that of
+ * the whole batch either way. */
 #define PEARL_UPDATE_SUBBATCH 4096u
 
 /* Bytes of device memory a buffer of this geometry needs (tree, storage, scratch and the
@@ -81,7 +90,10 @@ uint64_t pearl_prb_slab_bytes(uint64_t capacity, uint32_t fanout, const pearl_la
  * owns five more streams with their events (the tree kernel of a long-row update_insert, the
  * sub-batches of pearl_prb_sample_streamed; all joined back into cuda_stream before a call's work
  * is over) and 512 KB of pinned host memory for the *_host calls (without it they copy array by
- * array).  Returns PEARL_ERR_OOM if the slab is too small. */
+ * array).  Returns PEARL_ERR_OOM if the slab is too small, and PEARL_ERR_BAD_ARG for a geometry out
+ * of range -- which includes a row whose size is not a multiple of 16 bytes (or is below 8 KB) when
+ * max_batch such rows hold 2^32 or more copy granules (the largest power of two, at most 16, that
+ * divides the row size): pad such rows to a multiple of 16 bytes or lower max_batch. */
 int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout,
                      const pearl_layout_t* layout, uint32_t max_batch, int device,
                      void* cuda_stream, void* slab, uint64_t slab_bytes);
@@ -229,8 +241,7 @@ int pearl_prb_update_host(pearl_prb_t* prb, uint32_t B, const int32_t* h_idx, co
  * Who needs it: code that runs where device allocation is off the table -- a plug-in inside a
  * framework whose memory pool has already claimed the whole GPU, so that a cudaMalloc would fail
  * or fragment it; a real-time control or serving loop whose rules forbid allocator calls after
- * start-up; a process whose handle was built on a caller-provided slab sized without the sample
- * call's scratch.  Such a caller hands in the same inputs and outputs as pearl_prb_sample, and the
+ * start-up.  Such a caller hands in the same inputs and outputs as pearl_prb_sample, and the
  * kernel's scratch (the batch's raw, un-normalised importance-sampling weights, one binary64 per
  * stratum) lives in a fixed 32 KiB array that is part of the library image: every GPU on which
  * the library runs this call holds that array until the process exits, whether or not it is used

@@ -62,6 +62,13 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     L->field_bytes[F_ACT] = lay->act_bytes;
     L->field_bytes[F_REW] = 4;
     L->field_bytes[F_DONE] = 1;
+    // A field that is copied granule by granule (anything but rows of at least 512 16-byte granules,
+    // which move as bulk copies) is indexed with 32-bit granule numbers within one batch.
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        const uint32_t g = L->field_bytes[f] ? granule_of(L->field_bytes[f]) : 1;
+        const uint64_t W = L->field_bytes[f] / g;
+        if (!(g == 16 && W >= 512) && (uint64_t)max_batch * W >= (1ull << 32)) return false;
+    }
 
     uint64_t at = 0;
     L->off_state = at; at = align_up(at + sizeof(PrbState));

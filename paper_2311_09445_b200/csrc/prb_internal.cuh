@@ -19,8 +19,8 @@ struct PrbState {
     unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
     unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished
     unsigned int max_prio_bits;       // bits of the largest priority written so far (0: none yet)
-    unsigned int wide_arrived;        // grid barrier of the running many-CTA update: arrivals so far (0 between launches)
-    unsigned int wide_done;           // its CTAs that have passed their last barrier
+    unsigned int wide_arrived;        // grid barrier of the running many-CTA update: arrivals so far (cleared on the stream before each launch)
+    unsigned int wide_spare;
     unsigned long long wide_wmax_bits; // largest raw weight of the running large-batch sample (bits of a binary64; 0 between calls)
 };
 
@@ -233,23 +233,33 @@ struct PrbBulkLane {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
     }
+    // (a lane whose wait ran out moves nothing more: its remaining chunks are skipped, see store())
     __device__ __forceinline__ void load(const void* gsrc, uint32_t bytes)
     {
+        if (failed) return;
         if (busy) { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); busy = false; }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                      ::"r"(buf), "l"(gsrc), "r"(bytes), "r"(bar), "l"(stream_policy) : "memory");
     }
+    __device__ __forceinline__ bool landed()
+    {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        return ok != 0;
+    }
     // Waits (bounded) for the load, then stores the stage to gdst.  The store is issued inside the
-    // polling loop so that a lane whose data has landed does not wait for the other lanes.
+    // polling loop so that a lane whose data has landed does not wait for the other lanes.  If the
+    // wait runs out the lane is marked failed: the phase parity stays as it is (the load is still
+    // outstanding), nothing is stored from the stage, and every later load and store of the lane is
+    // skipped; finish() then only waits, again with a limit, for what is in flight.
     __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
     {
+        if (failed) return;
         bool done = false;
         for (uint32_t spin = 0; spin < kBulkSpinLimit && !done; ++spin) {
-            uint32_t ok;
-            asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-            if (ok) {
+            if (landed()) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                              ::"l"(gdst), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
@@ -257,13 +267,18 @@ struct PrbBulkLane {
                 done = true;
             }
         }
-        parity ^= 1u;
-        busy = done;
-        if (!done) failed = true;
+        if (done) { parity ^= 1u; busy = true; }
+        else failed = true;
     }
     // Before the CTA exits: this lane's stores have read their stages (the writes themselves are
-    // complete when the kernel is, like any other store).
-    __device__ __forceinline__ void finish() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+    // complete when the kernel is, like any other store); a failed lane gives its outstanding load
+    // one more bounded wait, so that shared memory is not handed back under a copy still landing.
+    __device__ __forceinline__ void finish()
+    {
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        if (failed)
+            for (uint32_t spin = 0; spin < kBulkSpinLimit && !landed(); ++spin) { }
+    }
 };
 
 #endif  // __CUDACC__

@@ -60,7 +60,8 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 //      has not.  Re-summing a parent none of whose children changed gives back what it held, so
 //      an entry that was refused for its priority may take part and duplicates only cost time;
 //   4. CTA 0 stages the top of the tree in shared memory and re-sums it whole (prb_top_passes).
-// The barrier's wait is bounded: a CTA that gives up raises PEARL_ST_INTERNAL and returns.
+// The barrier's wait is bounded: a CTA that gives up raises PEARL_ST_INTERNAL and returns; the update
+// is then incomplete (see PEARL_ST_INTERNAL in the header for what that leaves in the tree).
 constexpr uint32_t kWideThreads = 256;
 constexpr uint32_t kWideSpinLimit = 1u << 22;
 
@@ -256,13 +257,10 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         l -= (int)h;
     }
     if (!alive) {
+        // (the barrier's counter is cleared on the stream before every launch: a launch that gave up
+        // leaves nothing behind that the next one would trip over)
         if (tid == 0) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
         return;
-    }
-    // every CTA is past its last barrier: the last one to say so clears the barrier for the next launch
-    if (tid == 0 && atomicAdd(&v.state->wide_done, 1u) == nctas - 1) {
-        v.state->wide_arrived = 0u;
-        v.state->wide_done = 0u;
     }
     // 4. the staged levels
     if (blockIdx.x == 0 && T > 0) {
@@ -337,6 +335,8 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // the grid barrier counts arrivals from zero: cleared here, on the stream, not by the launch before
+    if (cudaMemsetAsync(&v.state->wide_arrived, 0, sizeof(unsigned int), s) != cudaSuccess) return -1;
     if (cudaLaunchKernelEx(&cfg, prb_update_wide_kernel, v, B, d_idx, d_val, raw, alpha, eps, stale) != cudaSuccess) return -1;
     return 1;
 }

@@ -11,6 +11,41 @@ def bits(a):
     return np.ascontiguousarray(a).view(np.uint32)
 
 
+def sliver_leaves(K, D, lift=0):
+    """Leaves of a K^D-leaf tree that make one root-to-leaf walk fall off the end of a child group.
+
+    Two sibling nodes of level D-1 hold 2^24 (K leaves of 2^24/K each) and 3 (leaves 1, 2, 0, ...);
+    every other leaf is zero.  Their left-to-right binary32 prefix is fl(2^24 + 3) = 2^24 + 4 (a
+    tie, rounded to even), and so is every ancestor up to the root.  A target in
+    [2^24 + 3, 2^24 + 4) therefore enters the second node with a residual in [3, 4), which has
+    passed every prefix of (1, 3, 3, ...): the walk takes the last positive child, the leaf
+    holding 2.  With lift > 0 every leaf is pushed down `lift` more levels (leaf i of the small
+    tree becomes leaf i * K^lift of a tree of depth D + lift), so the walk falls off at an inner
+    level as well.  Returns (leaves, index of the leaf the walk ends in)."""
+    p = np.zeros(K ** D, np.float32)
+    a = (K ** (D - 1)) // 2
+    a -= a % K                               # a and a + 1 are children of one parent
+    p[a * K:(a + 1) * K] = np.float32(2 ** 24 / K)
+    p[(a + 1) * K], p[(a + 1) * K + 1] = 1.0, 2.0
+    leaf = (a + 1) * K + 1
+    if lift:
+        big = np.zeros(K ** (D + lift), np.float32)
+        big[::K ** lift] = p
+        p, leaf = big, leaf * K ** lift
+    return p, leaf
+
+
+def seed_for_sliver(oracle_mod, B, call=0, limit=1 << 22):
+    """The first Philox seed whose last stratum (of B, sample call `call`) draws a target in the last
+    unit of a total of 2^24 + 4, i.e. in [2^24 + 3, 2^24 + 4): found by scanning on the CPU."""
+    total = 2.0 ** 24 + 4
+    for seed in range(limit):
+        x = (B - 1 + oracle_mod.stratum_uniform(seed, call, B - 1)) * (total / B)
+        if 2.0 ** 24 + 3 <= x < total:
+            return seed
+    raise AssertionError("no seed found")
+
+
 class Pair:
     def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True):
         from paper_2311_09445_b200 import PrioritizedReplay

@@ -5,7 +5,7 @@ import torch
 
 from conftest import golden_lines
 from paper_2311_09445_b200 import workloads as wk
-from prb_harness import Pair
+from prb_harness import Pair, seed_for_sliver, sliver_leaves
 
 pytestmark = pytest.mark.gpu
 
@@ -213,59 +213,69 @@ def test_atari_shaped_full_size(oracle_mod):
     pr.close()
 
 
-@pytest.mark.parametrize("N,K,B", [(1 << 16, 2, 32), (1 << 16, 4, 1024), (1 << 16, 16, 4096), (1 << 18, 32, 256),
-                                   (1 << 20, 2, 4096), (1 << 22, 4, 1024), (1 << 22, 16, 16384), (1 << 22, 32, 65536)])
-def test_sweep_cells(oracle_mod, N, K, B):
-    wl = wk.sweep_cell(N, K, B, cell_id=N % 997 + K + B)
-    rng = np.random.default_rng(wl.seed)
-    chunk = 1 << 16
-    pr = Pair(oracle_mod, N, K, wl.obs_bytes, wl.act_bytes, max(chunk, B))
-    for first in range(0, N, chunk):
-        pr.insert(wk.transitions(wl, rng, chunk, first))
-    pr.compare_tree()
-    for step in range(3):
-        pr.insert(wk.transitions(wl, rng, wl.n_insert))
-        o, g = pr.sample(B, wl.beta, wl.philox_seed)
-        idx, td = wk.update_batch(wl, rng, o["idx"])
-        pr.update(idx, td, wl.alpha, wl.eps)
-        pr.compare_tree()
-    pr.compare_state()
-    pr.close()
+SWEEP_CAPACITIES = [1 << 16, 1 << 18, 1 << 20, 1 << 22, 1 << 24, 1 << 26]
+SWEEP_FANOUTS = [2, 4, 16, 32]
+SWEEP_BATCHES = [32, 256, 1024, 4096, 16384, 65536]
 
 
-@pytest.mark.parametrize("K", [2, 32])
-def test_largest_sweep_capacity(oracle_mod, K):
-    # 2^26 slots (depth 26 for fanout 2): the oracle mirrors the tree and the short fields; the 11 GB
-    # of observations live on the device only.
-    N, B = 1 << 26, 4096
-    free, _ = torch.cuda.mem_get_info()
-    if free < (14 << 30):
-        pytest.skip("not enough free device memory")
-    wl = wk.sweep_cell(N, K, B, cell_id=K)
+def test_sweep_grid_is_the_stated_one():
+    # capacity 2^16..2^26 x fanout {2,4,16,32} x batch {32..65536}, batches up to half the capacity: 140 cells
+    cells = [(N, K, B) for N in SWEEP_CAPACITIES for K in SWEEP_FANOUTS for B in SWEEP_BATCHES if B <= N // 2]
+    assert len(cells) == 140
+
+
+@pytest.mark.parametrize("K", SWEEP_FANOUTS)
+@pytest.mark.parametrize("N", SWEEP_CAPACITIES)
+def test_sweep_cells(oracle_mod, N, K):
+    # Every cell of the scaling sweep: one buffer per (capacity, fanout), filled once, then for every
+    # batch size of the grid two mixed steps (insert 1024, sample B, update B) compared with the oracle
+    # call by call -- indices, weights, rows, every tree level, counters, status bits.  Up to 2^22
+    # slots the oracle mirrors the whole store; above, the tree and the short fields (the
+    # observations then live on the device only and the reward stands in for the row).
+    full = N <= (1 << 22)
+    if not full:
+        free, _ = torch.cuda.mem_get_info()
+        if free < N * 165 + (3 << 30):
+            pytest.skip("not enough free device memory")
+    wl = wk.sweep_cell(N, K, 1024, cell_id=N % 997 + K)
     rng = np.random.default_rng(wl.seed)
-    pr = Pair(oracle_mod, N, K, wl.obs_bytes, wl.act_bytes, 1 << 18, oracle_store=False)
+    chunk = min(N, 1 << 18)
+    batches = [B for B in SWEEP_BATCHES if B <= N // 2]
+    pr = Pair(oracle_mod, N, K, wl.obs_bytes, wl.act_bytes, max(chunk, max(batches)), oracle_store=full)
     dev = pr.dev
-    chunk = 1 << 18
-    obs = torch.zeros((chunk, wl.obs_bytes), dtype=torch.uint8, device=dev)      # same rows for every chunk
-    act = torch.zeros((chunk, wl.act_bytes), dtype=torch.uint8, device=dev)
-    for first in range(0, N, chunk):
-        prio = wk.priorities(wl, rng, chunk)
-        rew = rng.standard_normal(chunk).astype(np.float32)
-        done = np.zeros(chunk, np.uint8)
-        d = dict(obs=obs, next_obs=obs, act=act, rew=torch.from_numpy(rew).to(dev), done=torch.from_numpy(done).to(dev),
-                 prio=torch.from_numpy(prio).to(dev))
+    zeros = None if full else {"obs": torch.zeros((chunk, wl.obs_bytes), dtype=torch.uint8, device=dev),
+                               "act": torch.zeros((chunk, wl.act_bytes), dtype=torch.uint8, device=dev)}
+
+    def insert(n, first):
+        if full:
+            pr.insert(wk.transitions(wl, rng, n, first))
+            return
+        prio = wk.priorities(wl, rng, n)
+        rew = rng.standard_normal(n).astype(np.float32)
+        done = (rng.random(n) < 0.05).astype(np.uint8)
+        d = dict(obs=zeros["obs"][:n], next_obs=zeros["obs"][:n], act=zeros["act"][:n], rew=torch.from_numpy(rew).to(dev),
+                 done=torch.from_numpy(done).to(dev), prio=torch.from_numpy(prio).to(dev))
         pr.insert(dict(rew=rew, done=done, prio=prio), dev_batch=d)
-    pr.compare_tree(range(0, pr.ora.depth - 1))
-    pr.compare_state()
-    assert pr.gpu.depth == (26 if K == 2 else 6)
-    for step in range(3):
-        o, g = pr.sample(B, wl.beta, wl.philox_seed)
-        rows = pr.ora.read_rows(o["idx"])
-        assert np.array_equal(g["rew"], rows["rew"])
-        idx, td = wk.update_batch(wl, rng, o["idx"])
-        pr.update(idx, td, wl.alpha, wl.eps)
-        pr.compare_tree(range(0, pr.ora.depth - 1))
+
+    for first in range(0, N, chunk):
+        insert(chunk, first)
+    D = pr.ora.depth
+    assert D == pr.gpu.depth
     pr.compare_tree()
+    pr.compare_state()
+    upper = range(0, D if full else max(1, D - 2))      # (the two widest levels of the largest trees: once per batch size)
+    for B in batches:
+        for step in range(2):
+            insert(wl.n_insert, N)
+            o, g = pr.sample(B, wl.beta, wl.philox_seed)
+            if not full:
+                rows = pr.ora.read_rows(o["idx"])
+                assert np.array_equal(g["rew"], rows["rew"]) and np.array_equal(g["done"], rows["done"])
+            idx, td = wk.update_batch(wl, rng, o["idx"])
+            pr.update(idx, td, wl.alpha, wl.eps)
+            pr.compare_tree(upper if step == 0 else None)
+        pr.compare_state()
+        assert pr.compare_status() & ~8 == 0
     pr.close()
 
 
@@ -312,6 +322,39 @@ def test_large_batch_sample_cases(oracle_mod, K, B):
     o = pr.ora.sample(B, 0.4, 17, gather=False)
     assert np.array_equal(o["idx"], t.cpu().numpy())
     pr.sample(B, 0.4, 17)
+    pr.compare_state()
+    pr.close()
+
+
+@pytest.mark.parametrize("K,D,lift,B", [
+    # a lane group per stratum (prb_sample_kernel<K>): the group falls off in a staged level, in a level
+    # read from global memory, in prefetched leaves, and at an inner level
+    (2, 10, 0, 1024), (2, 14, 0, 1024), (2, 9, 2, 1024), (4, 6, 1, 1024), (8, 4, 0, 1024), (16, 3, 0, 1024),
+    (16, 5, 0, 1024), (16, 3, 1, 1024), (32, 3, 0, 1024), (32, 4, 0, 1024), (32, 2, 1, 512),
+    # a thread per stratum (prb_sample_wide_kernel<K>, from 2048 strata of short rows)
+    (2, 14, 0, 4096), (2, 9, 2, 2048), (4, 6, 1, 4096), (8, 4, 0, 4096), (16, 5, 0, 4096), (16, 3, 1, 65536),
+    (32, 3, 0, 2048), (32, 2, 1, 4096)])
+def test_descent_falls_off_a_child_group(oracle_mod, K, D, lift, B):
+    # The rounding sliver: a prefix that rounded up leaves a residual no child group can hold, and the
+    # walk takes the last positive child (status CLAMPED).  The tree is built through insert alone and
+    # the Philox seed is found on the CPU so that the batch's last stratum draws such a target; the
+    # oracle must report the fall-off, and indices, weights, rows and status bits must agree.
+    p, leaf = sliver_leaves(K, D, lift)
+    N = p.shape[0]
+    rng = np.random.default_rng(K * 100 + D)
+    pr = Pair(oracle_mod, N, K, 12, 4, max(B, 4096))
+    for first in range(0, N, 4096):
+        n = min(4096, N - first)
+        b = raw_fields(rng, n, 12, 4)
+        b["prio"] = p[first:first + n]
+        pr.insert(b)
+    pr.compare_tree()
+    assert pr.ora.total() == np.float32(2 ** 24 + 4)
+    for call in range(2):                    # the call counter is part of the Philox counter
+        seed = seed_for_sliver(oracle_mod, B, call=call)
+        o, g = pr.sample(B, 0.4, seed)
+        assert o["idx"][-1] == leaf
+        assert pr.compare_status() == 8      # CLAMPED on both sides, nothing else
     pr.compare_state()
     pr.close()
 

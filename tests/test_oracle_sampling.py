@@ -163,6 +163,28 @@ def test_rounding_sliver_rule(oracle_mod):
     o.status()
 
 
+@pytest.mark.parametrize("K,D,lift", [(2, 2, 0), (2, 10, 0), (4, 3, 1), (16, 3, 0), (32, 2, 0), (32, 2, 1)])
+def test_rounding_sliver_reached_without_planting(oracle_mod, K, D, lift):
+    # The fall-off is reachable through the public calls alone: a level prefix fl(2^24 + 3) that
+    # rounds up to 2^24 + 4 leaves a residual of at least 3 under a node that holds 3.  Every other
+    # target of the batch behaves: the flat scan over the exact binary64 prefixes names its leaf.
+    from prb_harness import seed_for_sliver, sliver_leaves
+    p, leaf = sliver_leaves(K, D, lift)
+    o = make(oracle_mod, p, K)
+    assert float(o.total()) == 2.0 ** 24 + 4
+    i, pl = o.descend(2.0 ** 24 + 3.5)
+    assert (i, pl) == (leaf, 2.0) and o.status() == oracle_mod.ST_CLAMPED
+    assert o.descend(2.0 ** 24 + 2.5)[0] == leaf and o.status() == 0          # just below the sliver: no fall-off
+    B = 1024
+    seed = seed_for_sliver(oracle_mod, B)
+    x = o.targets(B, seed, 0)
+    out = o.sample(B, 0.4, seed, gather=False)
+    assert o.status() == oracle_mod.ST_CLAMPED
+    flat = np.cumsum(p.astype(np.float64))
+    expect = np.searchsorted(flat, x[:-1], side="right")
+    assert np.array_equal(out["idx"][:-1], expect) and out["idx"][-1] == leaf
+
+
 def test_gather_bytes(oracle_mod):
     rng = np.random.default_rng(6)
     N = 100
