@@ -191,6 +191,25 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
                             const float* d_rew, const void* d_next_obs, const uint8_t* d_done,
                             const float* d_prio);
 
+/* One iteration of the training protocol as one call (Listing 2; Section IV-C, Eq. 7): the priority
+ * update for the batch the Learner has just finished with and the insertion of the transitions the
+ * Actors have collected meanwhile -- exactly pearl_prb_update_insert(prb, B_upd, d_upd_idx, d_td, alpha,
+ * eps, n, d_new_*...) -- followed by the sample of the next batch -- exactly pearl_prb_sample(prb, B,
+ * beta, seed, d_idx, d_w, d_obs ...): same results, same state, same status bits as the two calls.
+ * What the one call buys: with rows of 8 KB and more, and an update of at most PEARL_UPDATE_SUBBATCH
+ * entries, the descents and weights of the sample are computed by the tree kernel itself as soon as its
+ * update and insertion work is done, on the handle's second stream, while the caller's stream is still
+ * copying the new rows; the caller's stream then only copies the sampled rows.  The sample's chain of
+ * dependent tree reads, which keeps HBM idle, thus leaves the critical path (the paper's sampling
+ * latency T_samp of Eq. 7 shrinks to the Data Storage read).  Otherwise the call is the two calls one
+ * after the other.  d_upd_idx may be the d_idx of the previous step: it is read before d_idx is written.
+ * Arguments and errors as for the two calls; nothing is enqueued if any argument is refused. */
+int pearl_prb_step(pearl_prb_t* prb, uint32_t B_upd, const int32_t* d_upd_idx, const float* d_td, float alpha,
+                   float eps, uint32_t n, const void* d_new_obs, const void* d_new_act, const float* d_new_rew,
+                   const void* d_new_next_obs, const uint8_t* d_new_done, const float* d_new_prio, uint32_t B,
+                   float beta, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs, void* d_act, float* d_rew,
+                   void* d_next_obs, uint8_t* d_done);
+
 /* pearl_prb_sample with the weights normalised as in the prioritized-replay paper the toolkit
  * follows (Schaul et al., Algorithm 1: w_j = (N P(j))^-beta / max_i w_i, the maximum over the whole
  * memory): the divisor is the weight of the smallest positive priority stored,

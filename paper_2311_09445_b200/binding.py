@@ -49,6 +49,8 @@ SIGNATURES = {
     "pearl_prb_update_after_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32]),
     "pearl_prb_get_priorities": (_i, [_vp, _u32, _vp, _vp]),
     "pearl_prb_update_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_step": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp,
+                            _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_host": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
@@ -231,6 +233,20 @@ class PrioritizedReplay:
                                                     _dptr(done, "done"), _dptr(prio, "prio"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_update_insert")
+
+    def step(self, upd_idx, td, alpha: float, eps: float, new_obs, new_act, new_rew, new_next_obs, new_done, new_prio,
+             B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None, done=None,
+             n: Optional[int] = None) -> None:
+        """pearl_prb_step: update_insert for the previous batch, then the sample of the next one, as one call."""
+        rc = load_library().pearl_prb_step(self._h, upd_idx.numel(), _dptr(upd_idx, "upd_idx"), _dptr(td, "td"), alpha, eps,
+                                           new_prio.numel() if new_prio is not None else int(n), _dptr(new_obs, "new_obs"),
+                                           _dptr(new_act, "new_act"), _dptr(new_rew, "new_rew"),
+                                           _dptr(new_next_obs, "new_next_obs"), _dptr(new_done, "new_done"),
+                                           _dptr(new_prio, "new_prio"), B, beta, seed, _dptr(idx, "idx"), _dptr(w, "w"),
+                                           _dptr(obs, "obs"), _dptr(act, "act"), _dptr(rew, "rew"),
+                                           _dptr(next_obs, "next_obs"), _dptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_step")
 
     # ---- the same calls, host buffers (numpy arrays or host torch tensors) -----------------
     def insert_host(self, obs, act, rew, next_obs, done, prio, n: Optional[int] = None) -> None:

@@ -24,8 +24,7 @@
 // once; short rows are copied through registers.  Raw weights go to scratch; the CTA that is
 // last to finish its descents normalises them by the batch maximum and bumps the call counter
 // while the others are already copying.  No CTA ever waits on another.
-#include "prb_internal.cuh"
-#include "../../include/pearl_prb.h"
+#include "prb_descend.cuh"
 
 namespace {
 
@@ -56,25 +55,8 @@ struct SamplePlan {
     // leaf prefetch (when the level above the leaves is read from global memory): the first pf_groups
     // lane groups of a CTA own K*K floats each at byte pf_off of the dynamic shared memory
     uint32_t pf_groups, pf_off;
+    unsigned int* found;                     // not nullptr: the call's last CTA stores 1 there (0 if the buffer was empty)
 };
-
-// Philox4x32-10 (Salmon et al., SC'11), first output word only.
-__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                        uint32_t k0, uint32_t k1)
-{
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-        c0 = hi1 ^ c1 ^ k0;
-        c1 = lo1;
-        c2 = hi0 ^ c3 ^ k1;
-        c3 = lo0;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
-    }
-    return c0;
-}
 
 // The K children of one node lie in shared memory at `row`: every lane of the group reads all of them
 // (the same addresses: broadcasts) and forms the left-to-right binary32 prefix sums in registers, one
@@ -388,6 +370,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     if (tid == kThreads / 2) {
                         if (!empty) v.state->sample_calls = calls + 1;
                         if (plan.buffer_norm) v.state->pmin_bits = ~0ull;      // (ready for the next scan)
+                        if (plan.found != nullptr) *plan.found = empty ? 0u : 1u;
                         v.state->sample_ticket = 0u;
                     }
                 }
@@ -436,56 +419,6 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
 // small launch divides all raw weights by it.
 constexpr uint32_t kWideSampleFrom = 2048;      // batches of at least this many strata (short rows)
 constexpr uint32_t kWideSampleStrata = 32;      // ... spread over CTAs of at least this many strata
-
-template <int K>
-__device__ __forceinline__ void load_children(const float* src, bool global, float (&c)[K])
-{
-    if (K == 2) {
-        const float2 t = global ? __ldg(reinterpret_cast<const float2*>(src)) : *reinterpret_cast<const float2*>(src);
-        c[0] = t.x; c[1] = t.y;
-    } else {
-#pragma unroll
-        for (int q = 0; q < K / 4; ++q) {
-            const float4 t = global ? __ldg(reinterpret_cast<const float4*>(src) + q) : reinterpret_cast<const float4*>(src)[q];
-            c[4 * q] = t.x; c[4 * q + 1] = t.y; c[4 * q + 2] = t.z; c[4 * q + 3] = t.w;
-        }
-    }
-}
-
-template <int K>
-__device__ __forceinline__ void descend_alone(const PrbView& v, const SamplePlan& plan, const float* s_top, double x,
-                                              uint32_t& leaf, float& p_leaf, unsigned& flags)
-{
-    uint64_t g = 0;
-    float chosen = 0.0f;
-    for (uint32_t l = 1; l <= v.depth; ++l) {
-        float c[K];
-        const bool staged = l <= plan.top_levels;
-        load_children<K>(staged ? s_top + plan.top_off[l] + (uint32_t)g * K : v.level[l] + g * K, !staged, c);
-        int j = -1, last_pos = -1;
-        float run = 0.0f, before_j = 0.0f, before_last = 0.0f;
-#pragma unroll
-        for (int q = 0; q < K; ++q) {
-            const float before = run;                          // prefix q-1 (0 in front of the first child)
-            run = (q == 0) ? c[0] : __fadd_rn(run, c[q]);
-            if (j < 0 && !(x >= (double)run)) { j = q; before_j = before; chosen = c[q]; }
-            if (c[q] > 0.0f) { last_pos = q; before_last = before; }
-        }
-        if (j < 0) {
-            // the target has passed every prefix (possible only by binary32 rounding): last positive child
-            flags |= PEARL_ST_CLAMPED;
-            if (last_pos >= 0) { j = last_pos; before_j = before_last; }
-            else { j = 0; before_j = 0.0f; flags |= PEARL_ST_INTERNAL; }
-            chosen = 0.0f;
-#pragma unroll
-            for (int q = 0; q < K; ++q) if (q == j) chosen = c[q];
-        }
-        if (j > 0) x = __dsub_rn(x, (double)before_j);
-        g = g * K + (uint64_t)j;
-    }
-    p_leaf = chosen;
-    leaf = (uint32_t)g;
-}
 
 // Short rows of strata [k_first, k_first + n_rows) by all `nthreads` threads, field by field, in
 // granules of type T: up to U granules per thread are loaded before the first is stored.
@@ -560,13 +493,9 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
         const uint32_t k = kb + tid, n_here = min(kThreads, k_hi - kb);
         if (k < k_hi) {
             // target of stratum k (Eq. 1's x, one per equal segment of the total), then the walk
-            const double seg = __ddiv_rn(total, (double)B);
-            const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32), (uint32_t)seed, (uint32_t)(seed >> 32));
-            const double u = __dmul_rn((double)r0, 2.3283064365386963e-10);     // * 2^-32, exact
-            double x = __dmul_rn(__dadd_rn((double)k, u), seg);
-            if (x >= total) x = __longlong_as_double(__double_as_longlong(total) - 1);   // next binary64 below total
+            const double x = prb_stratum_target(k, B, total, calls, seed);
             uint32_t leaf; float p;
-            descend_alone<K>(v, plan, s_top, x, leaf, p, my_flags);
+            prb_descend_alone<K, false>(v, plan.top_levels, plan.top_off, s_top, x, leaf, p, my_flags);
             s_idx[tid] = leaf;
             out_idx[k] = (int32_t)leaf;
             if (out_w != nullptr) {
@@ -592,6 +521,7 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
         // the last CTA to finish: the call's bookkeeping (the weights are divided by a launch of their own)
         if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
         else v.state->sample_calls = calls + 1;
+        if (plan.found != nullptr) *plan.found = empty ? 0u : 1u;
         v.state->sample_ticket = 0u;
     }
 }
@@ -641,15 +571,78 @@ __global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
     }
 }
 
+// ---- the row copy of a two-kernel sample ----------------------------------------------------------------
+// When a sample of long rows is part of a captured sequence of calls, its descents (the kernels above,
+// launched without fields) run on the handle's second stream, where they can overlap whatever the
+// caller's stream is still copying, and leave indices and normalised weights in a hand-off area of the
+// slab; this kernel, on the caller's stream, is then nothing but the indexed copy: one CTA per SM, warp 0
+// driving the bulk-copy ring (a lane's first load goes out one L2 read -- its row's index -- after the
+// kernel starts), four more warps copying the short fields, the indices and the weights of the strata
+// whose first chunk the CTA holds.  The task numbering is that of prb_sample_kernel.
+constexpr int kGatherWorkers = 128;
+constexpr int kGatherThreads = 32 + kGatherWorkers;
+
+__global__ void __launch_bounds__(kGatherThreads, 1)
+prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, const unsigned char* __restrict__ handoff,
+                       int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
+                       const __grid_constant__ SamplePlan plan)
+{
+    extern __shared__ __align__(128) unsigned char s_ring[];
+    __shared__ uint32_t s_idx[kGatherWorkers];
+    const uint32_t tid = threadIdx.x;
+    const int32_t* pre_idx = prb_handoff_idx(handoff);
+    const uint32_t tps = plan.tps;
+    const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * plan.n_tasks) / gridDim.x);
+    const uint32_t t_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * plan.n_tasks) / gridDim.x);
+    if (tid < plan.ring_stages) {
+        PrbBulkLane ring;
+        uint32_t t = t_lo + tid;
+        // (the index of the lane's first row is asked for before anything else)
+        int32_t leaf = t < t_hi ? __ldcg(pre_idx + t / tps) : 0;
+        ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
+        if (__ldcg(prb_handoff_found(handoff)) == 0u) return;          // the buffer was empty: nothing is written
+        while (t < t_hi) {
+            const uint32_t k = t / tps, r = t - k * tps;
+            int f = 0;
+            while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
+            const uint32_t W = v.field_bytes[f] / 16u;
+            const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
+            const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
+            ring.load(v.store[f] + ((uint64_t)(uint32_t)leaf * W + e0) * 16u, bytes);
+            const uint32_t t_next = t + plan.ring_stages;
+            const int32_t leaf_next = t_next < t_hi ? __ldcg(pre_idx + t_next / tps) : 0;
+            ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
+            t = t_next;
+            leaf = leaf_next;
+        }
+        ring.finish();
+        if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
+    } else if (tid >= 32) {
+        // strata whose first task lies in this CTA's range: indices, weights and short fields
+        const uint32_t rank = tid - 32u;
+        const uint32_t k_own = (t_lo + tps - 1) / tps, k_end = (t_hi + tps - 1) / tps;
+        if (__ldcg(prb_handoff_found(handoff)) == 0u) return;
+        const float* pre_w = prb_handoff_w(handoff, v.max_batch);
+        for (uint32_t kb = k_own; kb < k_end; kb += kGatherWorkers) {
+            const uint32_t n_here = min((uint32_t)kGatherWorkers, k_end - kb);
+            if (rank < n_here) {
+                const int32_t leaf = __ldcg(pre_idx + kb + rank);
+                s_idx[rank] = (uint32_t)leaf;
+                out_idx[kb + rank] = leaf;
+                if (out_w != nullptr) out_w[kb + rank] = __ldcg(pre_w + kb + rank);
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kGatherWorkers) : "memory");
+            gather_short_fields(v, plan, dst, kb, n_here, s_idx, rank, kGatherWorkers);
+            asm volatile("bar.sync 1, %0;" ::"n"(kGatherWorkers) : "memory");
+        }
+    }
+}
+
 }  // namespace
 
-int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs, int buffer_norm)
+// The row-mode part of a plan: which fields move as chunks of long rows, and how they are cut.
+static bool plan_row_mode(const PrbView& v, const PrbBatch& dst, SamplePlan& plan)
 {
-    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
-    const int sm_count = prb_sm_count();
-    const int dev = prb_current_device();
-    SamplePlan plan;
     plan.tps = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         plan.task_first[f] = 0;
@@ -666,6 +659,25 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     }
     const bool row_mode = plan.tps > 0;
     if (!row_mode) plan.tps = 1;
+    return row_mode;
+}
+
+bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst)
+{
+    SamplePlan plan;
+    return plan_row_mode(v, dst, plan);
+}
+
+int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs, int buffer_norm,
+                      unsigned int* found)
+{
+    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
+    const int sm_count = prb_sm_count();
+    const int dev = prb_current_device();
+    SamplePlan plan;
+    const bool row_mode = plan_row_mode(v, dst, plan);
+    plan.found = found;
     plan.n_tasks = B * plan.tps;
     plan.first_task = 0;
     plan.ticket_total = 0;
@@ -840,4 +852,37 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         }
     }
     return cudaGetLastError() == cudaSuccess ? (int)n_sub + extra_launches : -1;
+}
+
+int prb_launch_gather(const PrbView& v, uint32_t B, const unsigned char* handoff, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s)
+{
+    SamplePlan plan;
+    if (!plan_row_mode(v, dst, plan)) return -1;
+    const int sm_count = prb_sm_count();
+    const int dev = prb_current_device();
+    plan.n_tasks = B * plan.tps;
+    plan.first_task = 0;
+    plan.ticket_total = 0;
+    plan.uniform = 0; plan.buffer_norm = 0; plan.top_levels = 0; plan.top_vec4 = 0;
+    for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
+    plan.pf_groups = 0; plan.pf_off = 0;
+    plan.found = nullptr;
+    uint32_t stage = 0;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
+    stage = (stage + 127u) / 128u * 128u;
+    plan.ring_stage_bytes = stage;
+    plan.ring_stages = kRingBytes / stage;
+    if (plan.ring_stages > 32) plan.ring_stages = 32;
+    const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
+    static bool big_smem[kPrbMaxDevices];
+    if (!big_smem[dev]) {
+        if (cudaFuncSetAttribute(prb_gather_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
+            return -1;
+        big_smem[dev] = true;
+    }
+    const uint32_t grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
+    prb_gather_rows_kernel<<<grid, kGatherThreads, smem, s>>>(v, B, handoff, d_idx, d_w, dst, plan);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

@@ -51,23 +51,30 @@ struct PrbTeam {
 };
 
 // Taken by one thread per CTA of an insertion once the whole CTA holds the cursor: the last of the
-// `participants` CTAs (of one kernel, or of the two kernels that share an insertion) to get here
-// publishes the new cursor and fill count.  Nothing later in those kernels reads them, so this
-// happens while the copies are still running; no CTA waits for another.
+// `participants` CTAs to get here publishes the new cursor.  Nothing later in those kernels reads
+// it, so this happens while the copies are still running; no CTA waits for another.
+//   kPrbPublishAll   a one-kernel insertion: cursor, fill and row_cursor (ticket: insert_ticket)
+//   kPrbPublishTree  the tree kernel of a two-kernel insertion: cursor and fill (insert_ticket)
+//   kPrbPublishRows  its row kernel: row_cursor (row_ticket)
+constexpr int kPrbPublishTree = 1, kPrbPublishRows = 2, kPrbPublishAll = 3;
 __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill,
-                                                    uint32_t participants)
+                                                    uint32_t participants, int what = kPrbPublishAll)
 {
     // no fence: the cursor and fill reads that must precede this ticket have returned their values
     // (they were stored to shared memory before the barrier this thread has passed)
-    const unsigned int done = atomicAdd(&v.state->insert_ticket, 1u);
+    unsigned int* ticket = (what == kPrbPublishRows) ? &v.state->row_ticket : &v.state->insert_ticket;
+    const unsigned int done = atomicAdd(ticket, 1u);
     if (done == participants - 1) {
         const uint64_t N = v.capacity;
         uint64_t c = cursor + n;
         if (c >= N) c -= N;
-        v.state->cursor = c;
-        fill += n;
-        v.state->fill = fill > N ? N : fill;
-        v.state->insert_ticket = 0;
+        if (what & kPrbPublishRows) v.state->row_cursor = c;
+        if (what & kPrbPublishTree) {
+            v.state->cursor = c;
+            fill += n;
+            v.state->fill = fill > N ? N : fill;
+        }
+        *ticket = 0;
     }
 }
 

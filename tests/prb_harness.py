@@ -133,6 +133,30 @@ class Pair:
                                torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps,
                                d.get("obs"), d.get("act"), d.get("rew"), d.get("next_obs"), d.get("done"), d["prio"])
 
+    def step(self, idx, td, alpha, eps, batch, B, beta, seed, check=True):
+        """pearl_prb_step on the GPU; update, insert, sample on the oracle.  Returns both sides' samples."""
+        assert self.ora.update(idx, td, alpha, eps) == 0
+        assert self.ora.insert(batch.get("obs"), batch.get("act"), batch.get("rew"), batch.get("next_obs"),
+                               batch.get("done"), batch["prio"]) == 0
+        o = self.ora.sample(B, beta, seed, gather=self.oracle_store)
+        d = {k: torch.from_numpy(np.ascontiguousarray(v)).to(self.dev) for k, v in batch.items() if v is not None}
+        t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=self.dev),
+             "w": torch.zeros(B, dtype=torch.float32, device=self.dev),
+             "obs": torch.zeros((B, self.obs_bytes), dtype=torch.uint8, device=self.dev),
+             "act": torch.zeros((B, self.act_bytes), dtype=torch.uint8, device=self.dev),
+             "rew": torch.zeros(B, dtype=torch.float32, device=self.dev),
+             "next_obs": torch.zeros((B, self.obs_bytes), dtype=torch.uint8, device=self.dev),
+             "done": torch.zeros(B, dtype=torch.uint8, device=self.dev)}
+        self.gpu.step(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),
+                      torch.from_numpy(np.ascontiguousarray(td, np.float32)).to(self.dev), alpha, eps,
+                      d.get("obs"), d.get("act"), d.get("rew"), d.get("next_obs"), d.get("done"), d["prio"],
+                      B, beta, seed, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+        torch.cuda.synchronize()
+        g = {k: v.cpu().numpy() for k, v in t.items()}
+        if check:
+            self.compare_sample(o, g)
+        return o, g
+
     def update_after_insert(self, idx, td, alpha, eps, inserted):
         assert self.ora.update_after_insert(idx, td, alpha, eps, inserted) == 0
         self.gpu.update_after_insert(torch.from_numpy(np.ascontiguousarray(idx, np.int32)).to(self.dev),

@@ -516,6 +516,260 @@ def test_fused_long_rows_replayed_as_cuda_graph(oracle_mod, B, n):
     ora.close()
 
 
+@pytest.mark.parametrize("B,n,beta_mode", [(512, 512, "batch"), (37, 300, "buffer"), (2500, 64, "batch"), (64, 200, "uniform")])
+def test_captured_steps_with_two_kernel_sample(oracle_mod, B, n, beta_mode):
+    # Inside a stream capture a sample of long rows is two kernels -- the descents on the handle's second
+    # stream, the indexed row copy on the caller's -- so that in a replayed sequence of steps the descents
+    # of one call overlap the row copies of the calls before.  A captured sequence of back-to-back
+    # samples and of whole steps (sample, update + insertion), replayed, must give every call the
+    # outputs the oracle gives it, and leave the oracle's tree and state.
+    from paper_2311_09445_b200 import PrioritizedReplay
+    N = 3000
+    wl = wk.scaled(wk.ATARI, N)
+    rng = np.random.default_rng(B + n)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(dev)
+    ora = oracle_mod.OraclePRB(N, wl.fanout, wl.obs_bytes, wl.act_bytes)
+
+    def outputs():
+        return {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.full((B,), -1.0, device=dev),
+                "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+                "act": torch.zeros((B, wl.act_bytes), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+                "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+                "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+
+    def gpu_sample(gpu, o):
+        args = (o["idx"], o["w"], o["obs"], o["act"], o["rew"], o["next_obs"], o["done"])
+        if beta_mode == "uniform":
+            gpu.sample_uniform(B, 5, *args)
+        elif beta_mode == "buffer":
+            gpu.sample_buffer_norm(B, wl.beta, 5, *args)
+        else:
+            gpu.sample(B, wl.beta, 5, *args)
+
+    def ora_sample():
+        if beta_mode == "uniform":
+            return ora.sample_uniform(B, 5)
+        return ora.sample(B, wl.beta, 5, buffer_norm=(beta_mode == "buffer"))
+
+    def check(o, t):
+        g = {k: v.cpu().numpy() for k, v in t.items()}
+        assert np.array_equal(o["idx"], g["idx"])
+        np.testing.assert_allclose(g["w"], o["w"], rtol=1e-5, atol=0)
+        for f in ("obs", "act", "rew", "next_obs", "done"):
+            assert np.array_equal(np.ascontiguousarray(o[f]).view(np.uint8).reshape(-1), g[f].view(np.uint8).reshape(-1)), f
+
+    with torch.cuda.stream(stream):
+        gpu = PrioritizedReplay(N, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096, device=dev, stream=stream)
+        # a captured sample of an empty buffer writes nothing and raises EMPTY
+        t0 = outputs()
+        torch.cuda.synchronize()
+        g0 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g0, stream=stream):
+            gpu_sample(gpu, t0)
+        g0.replay()
+        torch.cuda.synchronize()
+        ora_sample()
+        assert t0["idx"].min().item() == -1 and t0["idx"].max().item() == -1 and t0["w"].max().item() == -1.0
+        assert gpu.sync() == ora.status() == 4
+        next_id = 0
+        for _ in range(5):
+            b = wk.transitions(wl, rng, 512, next_id)
+            next_id += 512
+            assert ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"]) == 0
+            d = wk.to_device(b, dev)
+            gpu.insert(d["obs"], d["act"], d["rew"], d["next_obs"], d["done"], d["prio"])
+        steps = []
+        for c in range(3):
+            b = wk.transitions(wl, rng, n, next_id + c * n)
+            td = (rng.standard_normal(B) * 2).astype(np.float32)
+            steps.append((b, td, wk.to_device(b, dev), torch.from_numpy(td).to(dev)))
+        outs = [outputs() for _ in range(3 + 4)]
+
+        def sequence():
+            for c, (b, td, db, dtd) in enumerate(steps):          # whole steps: the update names what the step sampled
+                gpu_sample(gpu, outs[c])
+                gpu.update_insert(outs[c]["idx"], dtd, wl.alpha, wl.eps, db["obs"], db["act"], db["rew"], db["next_obs"],
+                                  db["done"], db["prio"])
+            for c in range(3, 7):                                    # back-to-back samples: the hand-off areas take turns
+                gpu_sample(gpu, outs[c])
+
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            sequence()
+        for rep in range(3):
+            graph.replay()
+            torch.cuda.synchronize()
+            for c, (b, td, db, dtd) in enumerate(steps):
+                o = ora_sample()
+                check(o, outs[c])
+                assert ora.update(o["idx"], td, wl.alpha, wl.eps) == 0
+                assert ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"]) == 0
+            for c in range(3, 7):
+                check(ora_sample(), outs[c])
+            for l in range(ora.depth + 1):
+                assert np.array_equal(ora.read_level(l).view(np.uint32), gpu.read_level(l).view(np.uint32)), "level %d" % l
+            assert gpu.info() == ora.info()
+            # an eager call between replays (one kernel, on the caller's stream) sees what the replay left
+            t = outputs()
+            gpu_sample(gpu, t)
+            torch.cuda.synchronize()
+            check(ora_sample(), t)
+        assert gpu.sync() == ora.status()
+        rows = np.arange(0, N, 11, dtype=np.int32)
+        g_rows, o_rows = gpu.read_rows(rows), ora.read_rows(rows)
+        for f in g_rows:
+            assert np.array_equal(np.ascontiguousarray(g_rows[f]).view(np.uint8).reshape(-1),
+                                  np.ascontiguousarray(o_rows[f]).view(np.uint8).reshape(-1)), f
+    gpu.close()
+    ora.close()
+
+
+@pytest.mark.parametrize("wl,N,B_upd,n,B", [(wk.ATARI, 1500, 512, 512, 512), (wk.ATARI, 700, 37, 1, 64), (wk.ATARI, 3000, 300, 300, 3000),
+                                            (wk.ATARI, 700, 4096, 300, 512), (wk.ATARI, 900, 5000, 100, 128),
+                                            (wk.CARTPOLE, 5000, 64, 64, 64), (wk.DDPG, 70_000, 256, 256, 2500)])
+def test_step_is_update_insert_then_sample(oracle_mod, wl, N, B_upd, n, B):
+    # pearl_prb_step == pearl_prb_update_insert followed by pearl_prb_sample.  With long rows the sample's
+    # descents and weights come from the tree kernel (sampling ahead), its rows from the indexed copy;
+    # with short rows, or an update beyond one tree kernel, the call is the two calls.
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(B_upd + n + B)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 8192)
+    # a step on an empty buffer whose insertion carries zero priorities only: nothing to sample
+    first = wk.transitions(wl, rng, min(n, N), 0)
+    first["prio"][:] = 0.0
+    o, g = pr.step(np.zeros(3, np.int32), np.ones(3, np.float32), wl.alpha, wl.eps, first, 16, wl.beta, 1)
+    assert g["idx"].tolist() == [-1] * 16 and pr.compare_status() == 1 | 4      # BAD_INDEX (nothing stored yet), EMPTY
+    pr.compare_state()
+    next_id = first["prio"].shape[0]
+    chunk = min(N, 4096)
+    for _ in range(0, N + chunk, chunk):            # fill and wrap
+        m = min(chunk, N)
+        pr.insert(wk.transitions(wl, rng, m, next_id))
+        next_id += m
+    o, g = pr.sample(min(B_upd, 8192), wl.beta, wl.philox_seed)
+    for step in range(5):
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        if step % 2 == 1:
+            rng.shuffle(idx)                               # unsorted batch: the sort path
+            idx[:3] = [(pr.ora.info()[1] + j) % N for j in range(3)]   # slots the insertion overwrites
+            idx[3] = -1
+        o, g = pr.step(idx, td, wl.alpha, wl.eps, wk.transitions(wl, rng, n, next_id), B, wl.beta, wl.philox_seed + step)
+        next_id += n
+        pr.compare_tree()
+        pr.compare_state()
+        pr.compare_status()
+        if B != B_upd:
+            o, g = pr.sample(min(B_upd, 8192), wl.beta, wl.philox_seed)
+    pr.compare_rows(np.arange(0, N, max(1, N // 500), dtype=np.int32))
+    pr.close()
+
+
+def test_step_in_place_and_captured(oracle_mod):
+    # The loop as a trainer runs it: one set of buffers, the update naming the indices the previous step
+    # left in the very buffer the step's sample overwrites; captured once, replayed.
+    from paper_2311_09445_b200 import PrioritizedReplay
+    N, B, n = 2000, 512, 512
+    wl = wk.scaled(wk.ATARI, N)
+    rng = np.random.default_rng(77)
+    dev = torch.device("cuda:0")
+    stream = torch.cuda.Stream(dev)
+    ora = oracle_mod.OraclePRB(N, wl.fanout, wl.obs_bytes, wl.act_bytes)
+    with torch.cuda.stream(stream):
+        gpu = PrioritizedReplay(N, wl.fanout, wl.obs_bytes, wl.act_bytes, 512, device=dev, stream=stream)
+        next_id = 0
+        for _ in range(4):
+            b = wk.transitions(wl, rng, 512, next_id)
+            next_id += 512
+            assert ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"]) == 0
+            d = wk.to_device(b, dev)
+            gpu.insert(d["obs"], d["act"], d["rew"], d["next_obs"], d["done"], d["prio"])
+        t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+             "obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "act": torch.zeros((B, wl.act_bytes), dtype=torch.uint8, device=dev), "rew": torch.zeros(B, device=dev),
+             "next_obs": torch.zeros((B, wl.obs_bytes), dtype=torch.uint8, device=dev),
+             "done": torch.zeros(B, dtype=torch.uint8, device=dev)}
+        gpu.sample(B, wl.beta, 3, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+        last = ora.sample(B, wl.beta, 3)
+        new = wk.transitions(wl, rng, n, next_id)
+        dnew = wk.to_device(new, dev)
+        td = (rng.standard_normal(B) * 2).astype(np.float32)
+        dtd = torch.from_numpy(td).to(dev)
+
+        def one_step():
+            gpu.step(t["idx"], dtd, wl.alpha, wl.eps, dnew["obs"], dnew["act"], dnew["rew"], dnew["next_obs"], dnew["done"],
+                     dnew["prio"], B, wl.beta, 3, t["idx"], t["w"], t["obs"], t["act"], t["rew"], t["next_obs"], t["done"])
+
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            one_step()
+            one_step()
+        for rep in range(4):
+            if rep == 2:
+                one_step()                       # an eager step between replays
+                one_step()
+            else:
+                graph.replay()
+            torch.cuda.synchronize()
+            for _ in range(2):
+                assert ora.update(last["idx"], td, wl.alpha, wl.eps) == 0
+                assert ora.insert(new["obs"], new["act"], new["rew"], new["next_obs"], new["done"], new["prio"]) == 0
+                last = ora.sample(B, wl.beta, 3)
+            assert np.array_equal(t["idx"].cpu().numpy(), last["idx"])
+            np.testing.assert_allclose(t["w"].cpu().numpy(), last["w"], rtol=1e-5, atol=0)
+            assert np.array_equal(t["obs"].cpu().numpy().reshape(-1), np.ascontiguousarray(last["obs"]).reshape(-1))
+            assert np.array_equal(t["next_obs"].cpu().numpy().reshape(-1), np.ascontiguousarray(last["next_obs"]).reshape(-1))
+            assert np.array_equal(t["done"].cpu().numpy(), last["done"])
+            for l in range(ora.depth + 1):
+                assert np.array_equal(ora.read_level(l).view(np.uint32), gpu.read_level(l).view(np.uint32)), "level %d" % l
+            assert gpu.info() == ora.info()
+        assert gpu.sync() == ora.status()
+    gpu.close()
+    ora.close()
+
+
+def test_step_sample_falls_off_a_child_group(oracle_mod):
+    # the rounding sliver met by a tree kernel that samples ahead (long rows), both as a step and as the
+    # first kernel of a captured two-kernel sample
+    K, D, B = 32, 3, 512
+    p, leaf = sliver_leaves(K, D, 0)
+    N = p.shape[0]
+    rng = np.random.default_rng(5)
+    pr = Pair(oracle_mod, N, K, 8192, 4, 4096, oracle_store=False)
+    dev = pr.dev
+    for first in range(0, N, 4096):
+        b = dict(rew=rng.standard_normal(4096).astype(np.float32), done=np.zeros(4096, np.uint8), prio=p[first:first + 4096])
+        d = {k: torch.from_numpy(v).to(dev) for k, v in b.items()}
+        d["obs"] = torch.zeros((4096, 8192), dtype=torch.uint8, device=dev)
+        d["next_obs"], d["act"] = d["obs"], torch.zeros((4096, 4), dtype=torch.uint8, device=dev)
+        pr.insert(b, dev_batch=d)
+    # the step re-writes two zero leaves with zero (update_priorities form is not part of the step: use a
+    # TD error with alpha > 0 and eps = 0, |0|^alpha = 0) and inserts nothing that changes the total
+    seed = seed_for_sliver(oracle_mod, B, call=0)
+    z = np.zeros(1, np.float32)
+    cur = pr.ora.info()[1]
+    newb = dict(rew=z, done=np.zeros(1, np.uint8), prio=p[cur:cur + 1].copy())
+    dnew = {k: torch.from_numpy(v).to(dev) for k, v in newb.items()}
+    dnew["obs"] = torch.zeros((1, 8192), dtype=torch.uint8, device=dev)
+    dnew["next_obs"], dnew["act"] = dnew["obs"], torch.zeros((1, 4), dtype=torch.uint8, device=dev)
+    assert pr.ora.update(np.array([0, 1], np.int32), np.zeros(2, np.float32), 0.6, 0.0) == 0
+    assert pr.ora.insert(None, None, newb["rew"], None, newb["done"], newb["prio"]) == 0
+    o = pr.ora.sample(B, 0.4, seed, gather=False)
+    t = {"idx": torch.full((B,), -1, dtype=torch.int32, device=dev), "w": torch.zeros(B, device=dev),
+         "obs": torch.zeros((B, 8192), dtype=torch.uint8, device=dev)}
+    pr.gpu.step(torch.tensor([0, 1], dtype=torch.int32, device=dev), torch.zeros(2, device=dev), 0.6, 0.0, dnew["obs"], dnew["act"],
+                dnew["rew"], dnew["next_obs"], dnew["done"], dnew["prio"], B, 0.4, seed, t["idx"], t["w"], t["obs"])
+    torch.cuda.synchronize()
+    assert o["idx"][-1] == leaf and np.array_equal(t["idx"].cpu().numpy(), o["idx"])
+    np.testing.assert_allclose(t["w"].cpu().numpy(), o["w"], rtol=1e-5, atol=0)
+    assert pr.compare_status() == 8
+    pr.compare_tree()
+    pr.compare_state()
+    pr.close()
+
+
 @pytest.mark.parametrize("wl", [wk.CARTPOLE, wk.ATARI])
 def test_fused_update_uses_fill_before_insert(oracle_mod, wl):
     # In the fused call the update comes first: an index that only the insertion makes valid is refused.
