@@ -196,13 +196,10 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
  * Actors have collected meanwhile -- exactly pearl_prb_update_insert(prb, B_upd, d_upd_idx, d_td, alpha,
  * eps, n, d_new_*...) -- followed by the sample of the next batch -- exactly pearl_prb_sample(prb, B,
  * beta, seed, d_idx, d_w, d_obs ...): same results, same state, same status bits as the two calls.
- * What the one call buys: with rows of 8 KB and more, and an update of at most PEARL_UPDATE_SUBBATCH
- * entries, the descents and weights of the sample are computed by the tree kernel itself as soon as its
- * update and insertion work is done, on the handle's second stream, while the caller's stream is still
- * copying the new rows; the caller's stream then only copies the sampled rows.  The sample's chain of
- * dependent tree reads, which keeps HBM idle, thus leaves the critical path (the paper's sampling
- * latency T_samp of Eq. 7 shrinks to the Data Storage read).  Otherwise the call is the two calls one
- * after the other.  d_upd_idx may be the d_idx of the previous step: it is read before d_idx is written.
+ * What the one call buys is one host call per iteration with all arguments checked before anything is
+ * enqueued; the kernels are those of the two calls (for rows of 8 KB and more: the tree kernel beside the
+ * copy of the new rows, then the sample).  d_upd_idx may be the d_idx of the previous step: it is read
+ * before d_idx is written.
  * Arguments and errors as for the two calls; nothing is enqueued if any argument is refused. */
 int pearl_prb_step(pearl_prb_t* prb, uint32_t B_upd, const int32_t* d_upd_idx, const float* d_td, float alpha,
                    float eps, uint32_t n, const void* d_new_obs, const void* d_new_act, const float* d_new_rew,

@@ -29,7 +29,7 @@ struct Layout {
     uint64_t off_state;
     uint64_t off_level[PRB_MAX_LEVELS];
     uint64_t off_wraw;
-    uint64_t off_handoff[2];
+    uint64_t off_handoff[kPrbHandoffs];
     uint64_t off_zero_end;                    // [0, off_zero_end) is zeroed at creation
     uint64_t off_store[PRB_NUM_FIELDS];
     uint64_t off_stage_in[PRB_NUM_FIELDS];    // staging of the *_host calls: inputs ...
@@ -75,7 +75,7 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     L->off_state = at; at = align_up(at + sizeof(PrbState));
     for (uint32_t l = 0; l <= D; ++l) { L->off_level[l] = at; at = align_up(at + L->level_alloc[l] * sizeof(float)); }
     L->off_wraw = at; at = align_up(at + (uint64_t)max_batch * sizeof(double));
-    for (int j = 0; j < 2; ++j) { L->off_handoff[j] = at; at = align_up(at + prb_handoff_bytes(max_batch)); }
+    for (uint32_t j = 0; j < kPrbHandoffs; ++j) { L->off_handoff[j] = at; at = align_up(at + prb_handoff_bytes(max_batch)); }
     L->off_zero_end = at;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_store[f] = at; at = align_up(at + capacity * L->field_bytes[f]); }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_in[f] = at; at = align_up(at + (uint64_t)max_batch * L->field_bytes[f]); }
@@ -124,12 +124,14 @@ struct pearl_prb {
     // A sample of long rows inside a stream capture is two kernels: the descents on fork.side, the row
     // copy on the caller's stream (see sample_two_kernels below).
     cudaEvent_t desc_done = nullptr;             // the descents of the running two-kernel sample are done
-    cudaEvent_t gather_done[2] = {nullptr, nullptr};   // the row copy that read hand-off area j is done
-    unsigned long long gather_capture[2] = {0, 0};     // the capture gather_done[j] was last recorded in (0: none)
+    cudaEvent_t gather_done[kPrbHandoffs] = {};   // the row copy that read hand-off area j is done
+    unsigned long long gather_capture[kPrbHandoffs] = {};    // the capture gather_done[j] was last recorded in (0: none)
     unsigned long long side_capture = 0;         // the capture fork.side has last been made part of (0: none)
     bool main_touched = true;                    // since fork.side last waited for the caller's stream, that stream
                                                  // has been given work that reads or writes the tree or the state
     uint32_t handoff_next = 0;
+    unsigned long long after_forked_tree = 0;    // the capture in which the last call was an update + insertion whose tree kernel ran on fork.side (0: it was not)
+    unsigned long long main_last_gather = 0;     // the capture in which the last kernel given to the caller's stream was such a row copy (0: it was not)
     ~pearl_prb()
     {
         destroy_fork(fork);
@@ -140,7 +142,7 @@ struct pearl_prb {
         if (subs.fork) cudaEventDestroy(subs.fork);
         if (pin_read) cudaEventDestroy(pin_read);
         if (desc_done) cudaEventDestroy(desc_done);
-        for (int j = 0; j < 2; ++j) if (gather_done[j]) cudaEventDestroy(gather_done[j]);
+        for (uint32_t j = 0; j < kPrbHandoffs; ++j) if (gather_done[j]) cudaEventDestroy(gather_done[j]);
         if (pin) cudaFreeHost(pin);
         cudaGetLastError();
     }
@@ -182,7 +184,8 @@ unsigned long long capture_of(cudaStream_t s)
 // A sample of long rows as two kernels, inside a stream capture (a captured step is replayed many
 // times, and there the time of the call is what counts, not the time of its host code).
 // The descents -- chains of dependent L2 reads that keep HBM idle -- read and write nothing of the
-// caller's: the tree, the state and a hand-off area of the slab.  So they are launched on the handle's
+// caller's: the tree, the state and a hand-off area of the slab (leaf indices and priorities; the
+// weights are formed by the row copy's spare warps).  So they are launched on the handle's
 // second stream, where they are ordered after the tree work that stream already holds (the tree kernel
 // of the update + insertion before them) but not after the rows the caller's stream is still copying:
 // in a captured step they run beside the insertion's row copy, and in back-to-back samples beside the
@@ -190,7 +193,7 @@ unsigned long long capture_of(cudaStream_t s)
 // copy, which also hands indices and weights to the caller.  Everything the caller can see is written
 // on the caller's stream, in order.  The second stream waits for the caller's stream first whenever
 // that stream has been given tree or state work since (main_touched), and once at the start of every
-// capture; the two hand-off areas are used in turn, an area not before the row copy that read it last.
+// capture; the hand-off areas are used in turn, an area not before the row copy that read it last.
 int sample_two_kernels(pearl_prb* h, unsigned long long capture, uint32_t B, float beta, uint64_t seed, int32_t* d_idx,
                        float* d_w, const PrbBatch& dst, int uniform, int buffer_norm)
 {
@@ -203,25 +206,16 @@ int sample_two_kernels(pearl_prb* h, unsigned long long capture, uint32_t B, flo
     }
     if (h->gather_capture[j] == capture && cudaStreamWaitEvent(side, h->gather_done[j], 0) != cudaSuccess) return -1;
     unsigned char* area = h->view.handoff[j];
-    PrbBatch none;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) none.ptr[f] = nullptr;
-    int k1;
-    if (!uniform && !buffer_norm) {
-        // (one small cluster, a thread per stratum, the weights' maximum over shared memory: the shortest chain)
-        const PrbSampleAhead sa = PrbSampleAhead{B, beta, seed, area};
-        k1 = prb_launch_update(h->view, 0, nullptr, nullptr, 0, 0.0f, 0.0f, side, 0, 0, nullptr, &sa);
-    } else {
-        k1 = prb_launch_sample(h->view, B, beta, seed, const_cast<int32_t*>(prb_handoff_idx(area)),
-                               const_cast<float*>(prb_handoff_w(area, h->view.max_batch)), none, side, uniform, 1, nullptr,
-                               buffer_norm, reinterpret_cast<unsigned int*>(area));
-    }
+    const int k1 = prb_launch_descend(h->view, B, seed, area, side, uniform, buffer_norm);
     if (k1 < 0) return -1;
     if (cudaEventRecord(h->desc_done, side) != cudaSuccess || cudaStreamWaitEvent(main, h->desc_done, 0) != cudaSuccess) return -1;
-    const int k2 = prb_launch_gather(h->view, B, area, d_idx, d_w, dst, main);
+    const int k2 = prb_launch_gather(h->view, B, beta, area, d_idx, d_w, dst, main, h->main_last_gather == capture);
     if (k2 < 0) return -1;
     if (cudaEventRecord(h->gather_done[j], main) != cudaSuccess) return -1;
     h->gather_capture[j] = capture;
-    h->handoff_next = j ^ 1u;
+    h->handoff_next = (j + 1u) % kPrbHandoffs;
+    h->main_last_gather = capture;
+    h->after_forked_tree = 0;
     return k1 + k2;
 }
 
@@ -270,9 +264,9 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
         }
     }
     if (cudaEventCreateWithFlags(&h->subs.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->desc_done, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->gather_done[0], cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->gather_done[1], cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
+        cudaEventCreateWithFlags(&h->desc_done, cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
+    for (uint32_t j = 0; j < kPrbHandoffs; ++j)
+        if (cudaEventCreateWithFlags(&h->gather_done[j], cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
     if (cudaHostAlloc((void**)&h->pin, 2 * kPackBytes, cudaHostAllocDefault) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->pin_read, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();                 // (not fatal: the host calls then copy array by array)
@@ -312,7 +306,7 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
         v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
     }
     v.wraw = (double*)at(h, L.off_wraw);
-    for (int j = 0; j < 2; ++j) v.handoff[j] = at(h, L.off_handoff[j]);
+    for (uint32_t j = 0; j < kPrbHandoffs; ++j) v.handoff[j] = at(h, L.off_handoff[j]);
     v.capacity = capacity;
     v.fanout = fanout;
     v.log2_fanout = 0;
@@ -365,7 +359,7 @@ int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* 
     const int k = prb_launch_insert(h->view, n, b, d_prio, h->stream);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
-    h->main_touched = true;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     return PEARL_OK;
 }
 
@@ -393,13 +387,17 @@ static int sample_common(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed, 
     if (!guard.ok) return PEARL_ERR_CUDA;
     PrbBatch b;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) b.ptr[f] = (unsigned char*)ptrs[f];
+    // Inside a capture a sample of long rows is two kernels (sample_two_kernels above) -- unless the call
+    // before it was an update + insertion whose tree kernel the descents would have to follow: that kernel
+    // ends with the row copy beside it, nothing is left for the descents to hide behind, and the one-kernel
+    // form, whose descents are the prologue of the copy, is shorter by a launch.
     const unsigned long long capture = (n_sub == 1 && prb_sample_has_long_rows(h->view, b)) ? capture_of(h->stream) : 0ull;
     int k;
-    if (capture) {
+    if (capture && h->after_forked_tree != capture) {
         k = sample_two_kernels(h, capture, B, beta, seed, d_idx, d_w, b, uniform, buffer_norm);
     } else {
         k = prb_launch_sample(h->view, B, beta, seed, d_idx, d_w, b, h->stream, uniform, n_sub, &h->subs, buffer_norm);
-        h->main_touched = true;
+        h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     }
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
@@ -453,7 +451,7 @@ static int update_common(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, const
     const int k = prb_launch_update(h->view, B, d_idx, d_val, raw, alpha, eps, h->stream, stale);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
-    h->main_touched = true;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     return PEARL_OK;
 }
 
@@ -488,7 +486,7 @@ int pearl_prb_get_priorities(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, f
     const int k = prb_launch_get_priorities(h->view, B, d_idx, d_out, h->stream);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
-    h->main_touched = true;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     return PEARL_OK;
 }
 
@@ -526,8 +524,10 @@ int pearl_prb_update_insert(pearl_prb_t* h, uint32_t B, const int32_t* d_idx, co
         // is the row copy, which touches neither the tree nor the state the descents read
         h->side_capture = capture_of(h->stream);
         h->main_touched = false;
+        h->main_last_gather = 0;
+        h->after_forked_tree = h->side_capture;
     } else {
-        h->main_touched = true;
+        h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     }
     return PEARL_OK;
 }
@@ -543,37 +543,11 @@ int pearl_prb_step(pearl_prb_t* h, uint32_t B_upd, const int32_t* d_upd_idx, con
     if (rc != PEARL_OK) return rc;
     rc = check_sample_args(h, B, beta, d_idx, d_w, out);
     if (rc != PEARL_OK) return rc;
-    PrbBatch bin, bout;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { bin.ptr[f] = (unsigned char*)in[f]; bout.ptr[f] = (unsigned char*)out[f]; }
-    if (!(prb_insert_forks(h->view, bin, B_upd) && prb_sample_has_long_rows(h->view, bout))) {
-        // short rows, or an update too large for one tree kernel: the two calls, one after the other
-        rc = pearl_prb_update_insert(h, B_upd, d_upd_idx, d_td, alpha, eps, n, d_new_obs, d_new_act, d_new_rew, d_new_next_obs,
-                                     d_new_done, d_new_prio);
-        if (rc != PEARL_OK) return rc;
-        return pearl_prb_sample(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done);
-    }
-    DeviceGuard guard(h->device);
-    if (!guard.ok) return PEARL_ERR_CUDA;
-    // Long rows.  Second stream: one tree kernel -- the update, the insertion's leaves and re-sums, then
-    // the descents and weights of the sample (its results go to a hand-off area of the slab).  Caller's
-    // stream: the copy of the new rows beside it; then, when both are done, the indexed copy of the
-    // sampled rows.  The second stream starts from an event of the caller's stream, so it is ordered after
-    // every earlier row copy that read the hand-off area.
-    const uint32_t j = h->handoff_next;
-    const PrbSampleAhead sa = PrbSampleAhead{B, beta, seed, h->view.handoff[j]};
-    bool forked = false;
-    const int k1 = prb_launch_insert(h->view, n, bin, d_new_prio, h->stream, B_upd, d_upd_idx, d_td, 0, alpha, eps, &h->fork, &forked, &sa);
-    if (k1 < 0 || !forked) return PEARL_ERR_CUDA;
-    const int k2 = prb_launch_gather(h->view, B, h->view.handoff[j], d_idx, d_w, bout, h->stream);
-    if (k2 < 0) return PEARL_ERR_CUDA;
-    const unsigned long long capture = capture_of(h->stream);
-    if (cudaEventRecord(h->gather_done[j], h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
-    h->gather_capture[j] = capture;
-    h->handoff_next = j ^ 1u;
-    h->side_capture = capture;
-    h->main_touched = false;          // (row copies only: neither touches the tree or the state the descents read)
-    h->launches += (uint64_t)(k1 + k2);
-    return PEARL_OK;
+    // (both calls' arguments have been checked: nothing is enqueued unless both go through)
+    rc = pearl_prb_update_insert(h, B_upd, d_upd_idx, d_td, alpha, eps, n, d_new_obs, d_new_act, d_new_rew, d_new_next_obs,
+                                 d_new_done, d_new_prio);
+    if (rc != PEARL_OK) return rc;
+    return pearl_prb_sample(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done);
 }
 
 // ---- host-buffer forms ---------------------------------------------------------------------
@@ -764,7 +738,7 @@ int pearl_prb_sample_static_scratch(pearl_prb_t* h, uint32_t B, float beta, uint
     const int k = prb_launch_sample(v, B, beta, seed, d_idx, d_w, b, h->stream);
     if (k < 0) return PEARL_ERR_CUDA;
     h->launches += (uint64_t)k;
-    h->main_touched = true;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     return PEARL_OK;
 }
 
@@ -778,7 +752,7 @@ int pearl_prb_sync(pearl_prb_t* h, uint32_t* status_bits)
     uint32_t st = 0;
     if (cudaMemcpyAsync(&st, &h->view.state->status, 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
     if (cudaMemsetAsync(&h->view.state->status, 0, 4, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
-    h->main_touched = true;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
     if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
     if (status_bits) *status_bits = st;
     return PEARL_OK;

@@ -27,7 +27,6 @@ constexpr uint32_t kChunk = 512;             // upper bound on granules per chun
 constexpr uint32_t kTile = kWorkers * 8;     // granules per tile of short rows
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
 constexpr uint32_t kRingBytes = 198 * 1024;  // bulk-copy ring (dynamic shared memory), <= 32 stages
-constexpr uint32_t kRingBytesBesideTree = 64 * 1024;   // ... while a tree kernel runs beside the copy
 constexpr uint32_t kRingBarBytes = 1024;     // room for the ring's mbarriers in front of its buffers
 
 struct InsertPlan {
@@ -213,7 +212,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
 
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps,
-                      const PrbFork* fork, bool* forked_out, const PrbSampleAhead* ahead)
+                      const PrbFork* fork, bool* forked_out)
 {
     if (forked_out) *forked_out = false;
     const int sm_count = prb_sm_count();
@@ -249,15 +248,10 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     bool forked = false;
     uint32_t rows_grid = 0;
     const bool fork_tree = upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr;
-    if (ahead != nullptr && !fork_tree) return -1;
     if (tasks > 0) {
-        // Beside a tree kernel the ring is shallower: a third of the depth keeps HBM as busy (measured:
-        // the copy takes the same 11-12 us) and the tree kernel's dependent reads queue behind far fewer
-        // bytes (it takes 8.7 us instead of 10.7 us).
         stage = (stage + 127u) / 128u * 128u;
         plan.ring_stage_bytes = stage;
-        plan.ring_stages = (fork_tree ? kRingBytesBesideTree : kRingBytes) / stage;
-        if (plan.ring_stages < 2) plan.ring_stages = kRingBytes / stage;
+        plan.ring_stages = kRingBytes / stage;
         if (plan.ring_stages > 32) plan.ring_stages = 32;
     }
     if (tasks > 0) {
@@ -265,7 +259,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         // their own: a copy CTA takes an SM's whole shared memory and would wait for them to leave.
         const uint32_t want = tasks + (fork_tree ? 0u : 1u);
         uint32_t room = (uint32_t)sm_count;
-        if (fork_tree && room > 2u * prb_update_ctas(v, upd.B, ahead)) room -= prb_update_ctas(v, upd.B, ahead);
+        if (fork_tree && room > 2u * prb_update_ctas(v, upd.B)) room -= prb_update_ctas(v, upd.B);
         rows_grid = want < room ? want : room;
     }
     if (fork_tree) {
@@ -273,10 +267,10 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         // row copy another on the caller's stream; neither waits for the other (each advances a
         // cursor of its own), and the caller's stream goes on when both are done.  (In one kernel the tree's chain of dependent reads, slowed by the
         // copy's traffic, was measured to outlast the copy by far.)
-        plan.tree_ctas = prb_update_ctas(v, upd.B, ahead);
+        plan.tree_ctas = prb_update_ctas(v, upd.B);
         if (cudaEventRecord(fork->fork, s) != cudaSuccess || cudaStreamWaitEvent(fork->side, fork->fork, 0) != cudaSuccess)
             return -1;
-        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, fork->side, 0, n, d_prio, ahead);
+        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, fork->side, 0, n, d_prio);
         if (k != 1 || cudaEventRecord(fork->join, fork->side) != cudaSuccess) return -1;
         upd.B = 0;
         launches = 2;
@@ -316,14 +310,4 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         if (forked && cudaStreamWaitEvent(s, fork->join, 0) != cudaSuccess) return -1;
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;
-}
-
-bool prb_insert_forks(const PrbView& v, const PrbBatch& src, uint32_t upd_B)
-{
-    if (upd_B == 0 || upd_B > PEARL_UPDATE_SUBBATCH) return false;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        if (v.field_bytes[f] == 0 || src.ptr[f] == nullptr) continue;
-        if (v.field_vec[f] == 16 && v.field_bytes[f] / 16u >= kRowMode) return true;
-    }
-    return false;
 }

@@ -5,6 +5,7 @@
 
 #define PRB_MAX_LEVELS 32       // level 0 (root) .. level D (leaves), D <= 30 for fanout 2
 #define PRB_NUM_FIELDS 5        // obs, next_obs, act, rew, done
+constexpr uint32_t kPrbHandoffs = 4;    // hand-off areas of a two-kernel sample (descents of later calls run ahead of earlier calls' row copies)
 
 enum PrbField { F_OBS = 0, F_NEXT_OBS = 1, F_ACT = 2, F_REW = 3, F_DONE = 4 };
 
@@ -41,10 +42,9 @@ struct PrbView {
     uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
     double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
     // A sample of long rows that is issued as two kernels (descents, then the row copy) hands indices
-    // and weights from the first to the second through one of two areas of the slab, used in turn:
-    // a 256-byte header whose first word says whether the sample found anything, max_batch indices,
-    // max_batch weights.
-    unsigned char* handoff[2];
+    // and leaf priorities from the first to the second through one of a few areas of the slab, used in turn:
+    // a 256-byte header (PrbHandoffHeader), max_batch indices, max_batch priorities.
+    unsigned char* handoff[kPrbHandoffs];
     uint64_t capacity;
     uint32_t fanout;                  // K
     uint32_t log2_fanout;
@@ -69,15 +69,6 @@ struct PrbFork {
     cudaEvent_t fork, join;
 };
 
-// A sample whose descents and weights a tree kernel computes right after its tree work ("sampling
-// ahead"): B strata, weights with exponent beta, Philox key `seed`; indices, weights and the found flag go
-// to `handoff` (one of PrbView::handoff).  B == 0: none.
-struct PrbSampleAhead {
-    uint32_t B;
-    float beta;
-    uint64_t seed;
-    unsigned char* handoff;
-};
 // Kernel launchers; each returns the number of kernels launched, or -1 on a launch error.
 // (upd_B > 0 runs a priority update of that batch before the insertion's tree work: in the same
 // kernel for short rows; for long rows in a tree kernel of its own on fork->side, or, without a
@@ -85,10 +76,7 @@ struct PrbSampleAhead {
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
                       int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f, const PrbFork* fork = nullptr,
-                      bool* forked_out = nullptr, const PrbSampleAhead* ahead = nullptr);
-// (ahead: only with a fork that takes place -- long rows, an update of at most PEARL_UPDATE_SUBBATCH entries --
-// which prb_insert_forks() tells beforehand; the tree kernel on fork->side then samples ahead)
-bool prb_insert_forks(const PrbView& v, const PrbBatch& src, uint32_t upd_B);
+                      bool* forked_out = nullptr);
 // Streams and events of a sample call that is issued as sub-batches (the paper's sub-batch
 // streaming, Section IV-C): sub-batch i runs on stream[i]; done[i] fires when its rows are in place.
 constexpr uint32_t kPrbMaxSubBatches = 4;
@@ -102,36 +90,49 @@ struct PrbSubStreams {
 // the leaves in a launch of its own, instead of the batch's;
 // uniform != 0: uniform replay, no tree walk, all weights 1; n_sub > 1: as that many launches, one
 // per sub-batch of consecutive strata, each on a stream of `subs`, joined back into s)
-// (found != nullptr: the call's last CTA stores 1 there if the sample found its batch, 0 if the buffer was empty)
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s, int uniform = 0, uint32_t n_sub = 1,
-                      const PrbSubStreams* subs = nullptr, int buffer_norm = 0, unsigned int* found = nullptr);
-// The second kernel of a two-kernel sample: copies the rows named by the indices in `handoff` (written by
-// a prb_launch_sample without fields that has completed) to dst, and the indices and weights to d_idx, d_w.
-int prb_launch_gather(const PrbView& v, uint32_t B, const unsigned char* handoff, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s);
-// true if a sample that writes these fields moves rows long enough for the bulk-copy ring
-bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst);
-__host__ __device__ inline const unsigned int* prb_handoff_found(const unsigned char* h) { return reinterpret_cast<const unsigned int*>(h); }
+                      const PrbSubStreams* subs = nullptr, int buffer_norm = 0);
+// A sample of long rows as two kernels.  The first walks the tree and leaves, in a hand-off area of the
+// slab (one of PrbView::handoff), what the second needs: a header, the leaf index of every stratum and
+// that leaf's priority.  The second copies the rows (and turns the priorities into weights meanwhile).
+struct PrbHandoffHeader {
+    unsigned int found;               // 1: the sample found its batch; 0: the buffer was empty, nothing is to be written
+    unsigned int buffer_norm;         // 1: weights are divided by the weight of pmin, else by the largest of the batch
+    unsigned long long fill;          // transitions stored when the sample was taken
+    float total;                      // the root then
+    float pmin;                       // smallest positive priority stored (buffer_norm only)
+};
+__host__ __device__ inline const PrbHandoffHeader* prb_handoff_header(const unsigned char* h) { return reinterpret_cast<const PrbHandoffHeader*>(h); }
 __host__ __device__ inline const int32_t* prb_handoff_idx(const unsigned char* h) { return reinterpret_cast<const int32_t*>(h + 256); }
-__host__ __device__ inline const float* prb_handoff_w(const unsigned char* h, uint32_t max_batch)
+__host__ __device__ inline const float* prb_handoff_prio(const unsigned char* h, uint32_t max_batch)
 {
     return reinterpret_cast<const float*>(h + 256 + ((uint64_t)max_batch * 4 + 255) / 256 * 256);
 }
 inline uint64_t prb_handoff_bytes(uint32_t max_batch) { return 256 + 2 * (((uint64_t)max_batch * 4 + 255) / 256 * 256); }
+// (the descents of B strata into `handoff`; uniform / buffer_norm as for prb_launch_sample)
+int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned char* handoff, cudaStream_t s, int uniform = 0,
+                       int buffer_norm = 0);
+// (the rows named by `handoff` -- written by a prb_launch_descend that has completed -- to dst, the
+// indices to d_idx, the weights with exponent beta to d_w)
+// (early_reads: the kernel before this one on s writes no rows of the store -- it is a row copy of a sample
+// too -- so this one may read rows while that one is still running)
+int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned char* handoff, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s, bool early_reads = false);
+// true if a sample that writes these fields moves rows long enough for the bulk-copy ring
+bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)
 // (ins_n > 0, B within one sub-batch: the tree part of an insertion of ins_n transitions follows
 // the update in the same kernel, which advances the tree's cursor and the fill count)
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale = 0,
-                      uint32_t ins_n = 0, const float* ins_prio = nullptr, const PrbSampleAhead* ahead = nullptr);
-// (B == 0 with `ahead`: a tree kernel that only samples ahead)
+                      uint32_t ins_n = 0, const float* ins_prio = nullptr);
 // Update batches above this many entries (one per thread of a CTA) go to one launch of many
 // co-resident CTAs instead (measured: 11-20 us for 16384 entries against 15-29 us for 4096 in one CTA);
 // an update + insertion of short rows is then two launches, the update's and the insertion's.
 constexpr uint32_t kPrbWideFrom = 1024;
-// CTAs (one cluster) of the kernel that updates a batch (or sub-batch) of b entries and then, if asked to, samples ahead
-uint32_t prb_update_ctas(const PrbView& v, uint32_t b, const PrbSampleAhead* ahead = nullptr);
+// CTAs (one cluster) of the kernel that updates a batch (or sub-batch) of b entries
+uint32_t prb_update_ctas(const PrbView& v, uint32_t b);
 int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx, float* d_out, cudaStream_t s);
 
 // Per-device facts the launchers cache: SM count, and which kernels already have their large
@@ -239,6 +240,10 @@ __device__ __forceinline__ void prb_copy_mapped(T* __restrict__ dst, const T* __
     }
     if (e < e_end) dst[dst_at(e)] = src[src_at(e)];
 }
+
+// A kernel launched as a programmatic dependent waits here until the kernel before it on its stream has
+// completed and its writes are visible; a no-op for a kernel launched the ordinary way.
+__device__ __forceinline__ void prb_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ---- bulk asynchronous copies (TMA, non-tensor form, one destination each) ----------------------
 // Long rows move global -> shared -> global as cp.async.bulk transfers.  Warp 0 of a CTA drives

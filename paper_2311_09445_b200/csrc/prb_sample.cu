@@ -55,7 +55,6 @@ struct SamplePlan {
     // leaf prefetch (when the level above the leaves is read from global memory): the first pf_groups
     // lane groups of a CTA own K*K floats each at byte pf_off of the dynamic shared memory
     uint32_t pf_groups, pf_off;
-    unsigned int* found;                     // not nullptr: the call's last CTA stores 1 there (0 if the buffer was empty)
 };
 
 // The K children of one node lie in shared memory at `row`: every lane of the group reads all of them
@@ -370,7 +369,6 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     if (tid == kThreads / 2) {
                         if (!empty) v.state->sample_calls = calls + 1;
                         if (plan.buffer_norm) v.state->pmin_bits = ~0ull;      // (ready for the next scan)
-                        if (plan.found != nullptr) *plan.found = empty ? 0u : 1u;
                         v.state->sample_ticket = 0u;
                     }
                 }
@@ -521,7 +519,6 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
         // the last CTA to finish: the call's bookkeeping (the weights are divided by a launch of their own)
         if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
         else v.state->sample_calls = calls + 1;
-        if (plan.found != nullptr) *plan.found = empty ? 0u : 1u;
         v.state->sample_ticket = 0u;
     }
 }
@@ -571,25 +568,116 @@ __global__ void prb_leaf_min_kernel(const __grid_constant__ PrbView v)
     }
 }
 
-// ---- the row copy of a two-kernel sample ----------------------------------------------------------------
-// When a sample of long rows is part of a captured sequence of calls, its descents (the kernels above,
-// launched without fields) run on the handle's second stream, where they can overlap whatever the
-// caller's stream is still copying, and leave indices and normalised weights in a hand-off area of the
-// slab; this kernel, on the caller's stream, is then nothing but the indexed copy: one CTA per SM, warp 0
-// driving the bulk-copy ring (a lane's first load goes out one L2 read -- its row's index -- after the
-// kernel starts), four more warps copying the short fields, the indices and the weights of the strata
-// whose first chunk the CTA holds.  The task numbering is that of prb_sample_kernel.
+// ---- a sample of long rows as two kernels ------------------------------------------------------------------
+// In a captured sequence of calls (a step that is replayed many times) the descents of a sample of long
+// rows run as a kernel of their own on the handle's second stream, where they can overlap whatever the
+// caller's stream is still copying, and the indexed row copy follows on the caller's stream.
+//
+// prb_descend_kernel<K>: targets and descents only, a lane group per stratum as in prb_sample_kernel, a grid
+// of at most one CTA per SM (it has to fit beside the CTAs of a row copy).  Lane 0 of a group stores the
+// leaf's index and priority in the hand-off area; the last CTA to finish (ticket) writes the header,
+// bumps the call counter and raises EMPTY if there was nothing to sample.  No weights here: the power
+// and the chain that finds their maximum are the longer half of a small sample, and nothing of the row
+// copy waits for them.
+template <int K>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+prb_descend_kernel(const __grid_constant__ PrbView v, uint32_t B, uint64_t seed, unsigned char* __restrict__ handoff,
+                   const __grid_constant__ SamplePlan plan)
+{
+    constexpr uint32_t R = kThreads / K;
+    __shared__ __align__(16) float s_top[top_floats_of(K)];
+    __shared__ __align__(16) float s_child[kThreads];
+    __shared__ unsigned long long s_calls;
+    extern __shared__ __align__(128) unsigned char s_pf[];      // leaf prefetch: K*K floats per walking group
+    const uint32_t tid = threadIdx.x;
+    const unsigned long long calls = v.state->sample_calls;
+    const unsigned long long fill = v.state->fill;
+    const float total32 = __ldg(v.level[0]);
+    {
+        const float4* src = reinterpret_cast<const float4*>(v.level[1]);
+        constexpr uint32_t kPerThread = (top_floats_of(K) / 4 + kThreads - 1) / kThreads;
+        float4 t[kPerThread];
+#pragma unroll
+        for (uint32_t u = 0; u < kPerThread; ++u)
+            if (tid + u * kThreads < plan.top_vec4) t[u] = __ldg(src + tid + u * kThreads);
+#pragma unroll
+        for (uint32_t u = 0; u < kPerThread; ++u)
+            if (tid + u * kThreads < plan.top_vec4) reinterpret_cast<float4*>(s_top)[tid + u * kThreads] = t[u];
+    }
+    if (tid == 0) s_calls = calls;        // (the value is in hand before this CTA's ticket below: the last CTA may then move the counter)
+    const bool empty = (fill == 0) || (!plan.uniform && !(total32 > 0.0f));
+    const double total = (double)total32;
+    int32_t* out_idx = const_cast<int32_t*>(prb_handoff_idx(handoff));
+    float* out_p = const_cast<float*>(prb_handoff_prio(handoff, v.max_batch));
+    const uint32_t k_lo = (uint32_t)(((uint64_t)blockIdx.x * B) / gridDim.x);
+    const uint32_t k_hi = (uint32_t)(((uint64_t)(blockIdx.x + 1) * B) / gridDim.x);
+    const uint32_t gi = tid / K, lane = tid % K;
+    __syncthreads();
+    for (uint32_t kb = k_lo; kb < k_hi && !empty; kb += R) {
+        const uint32_t n_round = min(R, k_hi - kb);
+        if ((tid / 32u) * (32u / K) < n_round) {              // warp-uniform: whole warps take part in the shuffles
+            const uint32_t k = min(kb + gi, B - 1);          // surplus groups repeat a valid stratum and write nothing
+            uint32_t leaf; float p; unsigned flags = 0;
+            if (plan.uniform) {
+                const uint32_t r0 = philox4x32_10_word0(k, 0u, (uint32_t)calls, (uint32_t)(calls >> 32), (uint32_t)seed, (uint32_t)(seed >> 32));
+                leaf = (uint32_t)(((unsigned long long)r0 * fill) >> 32);
+                p = 1.0f;
+            } else {
+                descend<K>(v, plan, s_top, s_child + (tid - lane), prb_stratum_target(k, B, total, calls, seed), lane, leaf, p, flags,
+                           gi < plan.pf_groups ? reinterpret_cast<float*>(s_pf) + gi * (K * K) : nullptr);
+            }
+            if (lane == 0 && gi < n_round) {
+                out_idx[kb + gi] = (int32_t)leaf;
+                out_p[kb + gi] = p;
+                if (flags) atomicOr(&v.state->status, flags);
+            }
+        }
+        __syncthreads();        // (a group's scratch and prefetch buffer are reused by the next round)
+    }
+    if (tid == 0 && atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) {
+        PrbHandoffHeader* hd = reinterpret_cast<PrbHandoffHeader*>(handoff);
+        hd->found = empty ? 0u : 1u;
+        hd->buffer_norm = plan.buffer_norm;
+        hd->fill = fill;
+        hd->total = total32;
+        hd->pmin = plan.buffer_norm ? __uint_as_float((unsigned)v.state->pmin_bits) : 0.0f;
+        if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
+        else v.state->sample_calls = s_calls + 1;
+        if (plan.buffer_norm) v.state->pmin_bits = ~0ull;      // (ready for the next scan)
+        v.state->sample_ticket = 0u;
+    }
+}
+
+// prb_gather_rows_kernel: the indexed copy, one CTA per SM.  Warp 0 drives the bulk-copy ring (a lane's first
+// load goes out one L2 read -- its row's index -- after the kernel starts); four more warps look after the
+// strata whose first chunk the CTA holds: the index, the short fields, and the importance-sampling weight
+//   w_k = (fill p_k / total)^-beta / max_j (fill p_j / total)^-beta = (p_k / p_min)^-beta
+// where p_min is the smallest priority of the batch (every CTA scans the B priorities in the hand-off area
+// for it: the power does not increase with p), or the smallest priority stored when the weights are
+// normalised over the buffer.  The task numbering is that of prb_sample_kernel.
+constexpr uint32_t kGatherRingBytes = 198 * 1024;      // the row copy's ring
 constexpr int kGatherWorkers = 128;
 constexpr int kGatherThreads = 32 + kGatherWorkers;
 
 __global__ void __launch_bounds__(kGatherThreads, 1)
-prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, const unsigned char* __restrict__ handoff,
+prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, const unsigned char* __restrict__ handoff,
                        int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
-                       const __grid_constant__ SamplePlan plan)
+                       const __grid_constant__ SamplePlan plan, uint32_t early_reads)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ uint32_t s_idx[kGatherWorkers];
+    __shared__ unsigned s_pmin[kGatherWorkers / 32];
     const uint32_t tid = threadIdx.x;
+    // Programmatic dependent launch, both ways.  As a primary: the kernel after this one on the stream may
+    // be scheduled as soon as every CTA here has said so, i.e. at once -- its CTAs then take over SMs one by
+    // one as CTAs of this kernel leave, instead of after the last of them.  As a secondary: this kernel may
+    // itself have started while the kernel before it on the stream was still running.  Nothing is stored
+    // before that kernel has completed (prb_dep_wait below: its writes, to the same output arrays perhaps,
+    // come first), and no row is read before then either, unless the host knows that kernel to be a row
+    // copy like this one, which writes no rows of the store (early_reads): then a CTA's whole read phase
+    // runs under the tail of the copy before it.  The hand-off area was written by a kernel this one
+    // depends on in full.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int32_t* pre_idx = prb_handoff_idx(handoff);
     const uint32_t tps = plan.tps;
     const uint32_t t_lo = (uint32_t)(((uint64_t)blockIdx.x * plan.n_tasks) / gridDim.x);
@@ -600,7 +688,9 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, const unsi
         // (the index of the lane's first row is asked for before anything else)
         int32_t leaf = t < t_hi ? __ldcg(pre_idx + t / tps) : 0;
         ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
-        if (__ldcg(prb_handoff_found(handoff)) == 0u) return;          // the buffer was empty: nothing is written
+        if (__ldcg(&prb_handoff_header(handoff)->found) == 0u) return;          // the buffer was empty: nothing is written
+        bool waited = false;
+        if (!early_reads) { prb_dep_wait(); waited = true; }
         while (t < t_hi) {
             const uint32_t k = t / tps, r = t - k * tps;
             int f = 0;
@@ -611,6 +701,7 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, const unsi
             ring.load(v.store[f] + ((uint64_t)(uint32_t)leaf * W + e0) * 16u, bytes);
             const uint32_t t_next = t + plan.ring_stages;
             const int32_t leaf_next = t_next < t_hi ? __ldcg(pre_idx + t_next / tps) : 0;
+            if (!waited) { prb_dep_wait(); waited = true; }
             ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
             t = t_next;
             leaf = leaf_next;
@@ -618,21 +709,42 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, const unsi
         ring.finish();
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
     } else if (tid >= 32) {
-        // strata whose first task lies in this CTA's range: indices, weights and short fields
         const uint32_t rank = tid - 32u;
         const uint32_t k_own = (t_lo + tps - 1) / tps, k_end = (t_hi + tps - 1) / tps;
-        if (__ldcg(prb_handoff_found(handoff)) == 0u) return;
-        const float* pre_w = prb_handoff_w(handoff, v.max_batch);
+        const PrbHandoffHeader* hd = prb_handoff_header(handoff);
+        if (__ldcg(&hd->found) == 0u) return;
+        const float* pre_p = prb_handoff_prio(handoff, v.max_batch);
+        const bool weights = out_w != nullptr && k_own < k_end;
+        float pmin = 0.0f;
+        if (weights) {
+            pmin = __ldcg(&hd->pmin);
+            if (__ldcg(&hd->buffer_norm) == 0u) {
+                unsigned best = 0xFFFFFFFFu;     // (priorities are not negative: they order like their bits)
+                for (uint32_t k = rank; k < B; k += kGatherWorkers) best = min(best, __float_as_uint(__ldcg(pre_p + k)));
+                best = __reduce_min_sync(0xFFFFFFFFu, best);
+                if ((rank & 31u) == 0) s_pmin[rank >> 5] = best;
+                asm volatile("bar.sync 1, %0;" ::"n"(kGatherWorkers) : "memory");
+#pragma unroll
+                for (int q = 0; q < kGatherWorkers / 32; ++q) best = min(best, s_pmin[q]);
+                pmin = __uint_as_float(best);
+            }
+        }
+        prb_dep_wait();
         for (uint32_t kb = k_own; kb < k_end; kb += kGatherWorkers) {
             const uint32_t n_here = min((uint32_t)kGatherWorkers, k_end - kb);
-            if (rank < n_here) {
+            const bool mine = rank < n_here;
+            float p = 1.0f;
+            if (mine) {
                 const int32_t leaf = __ldcg(pre_idx + kb + rank);
                 s_idx[rank] = (uint32_t)leaf;
                 out_idx[kb + rank] = leaf;
-                if (out_w != nullptr) out_w[kb + rank] = __ldcg(pre_w + kb + rank);
+                if (weights) p = __ldcg(pre_p + kb + rank);
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kGatherWorkers) : "memory");
             gather_short_fields(v, plan, dst, kb, n_here, s_idx, rank, kGatherWorkers);
+            // (fill p / total)^-beta / (fill pmin / total)^-beta as one power, (p / pmin)^-beta: the same number to a
+            // few units of the binary64 rounding error, exactly 1 where p is the smallest, and half the arithmetic
+            if (weights && mine) out_w[kb + rank] = (float)pow(__ddiv_rn((double)p, (double)pmin), -(double)beta);
             asm volatile("bar.sync 1, %0;" ::"n"(kGatherWorkers) : "memory");
         }
     }
@@ -662,29 +774,10 @@ static bool plan_row_mode(const PrbView& v, const PrbBatch& dst, SamplePlan& pla
     return row_mode;
 }
 
-bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst)
+// The top levels a sample kernel stages in shared memory (levels 1 .. top_levels, while they fit; the
+// levels lie one after another in the slab, each start 256-byte aligned), into the plan.
+static void plan_staged_top(const PrbView& v, bool uniform, SamplePlan& plan)
 {
-    SamplePlan plan;
-    return plan_row_mode(v, dst, plan);
-}
-
-int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs, int buffer_norm,
-                      unsigned int* found)
-{
-    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
-    const int sm_count = prb_sm_count();
-    const int dev = prb_current_device();
-    SamplePlan plan;
-    const bool row_mode = plan_row_mode(v, dst, plan);
-    plan.found = found;
-    plan.n_tasks = B * plan.tps;
-    plan.first_task = 0;
-    plan.ticket_total = 0;
-    // levels 1 .. top_levels staged in shared memory while they fit
-    // (the levels lie one after another in the slab, each start 256-byte aligned)
-    plan.uniform = uniform ? 1u : 0u;
-    plan.buffer_norm = (buffer_norm && !uniform) ? 1u : 0u;
     plan.top_levels = 0;
     plan.top_vec4 = 0;
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
@@ -695,6 +788,30 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         plan.top_vec4 = (uint32_t)((off + v.level_alloc[l] + 3) / 4);
         plan.top_levels = l;
     }
+}
+
+bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst)
+{
+    SamplePlan plan;
+    return plan_row_mode(v, dst, plan);
+}
+
+int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s, int uniform, uint32_t n_sub, const PrbSubStreams* subs, int buffer_norm)
+{
+    if (n_sub < 1 || n_sub > kPrbMaxSubBatches || n_sub > B || (n_sub > 1 && subs == nullptr)) return -1;
+    const int sm_count = prb_sm_count();
+    const int dev = prb_current_device();
+    SamplePlan plan;
+    const bool row_mode = plan_row_mode(v, dst, plan);
+    plan.n_tasks = B * plan.tps;
+    plan.first_task = 0;
+    plan.ticket_total = 0;
+    // levels 1 .. top_levels staged in shared memory while they fit
+    // (the levels lie one after another in the slab, each start 256-byte aligned)
+    plan.uniform = uniform ? 1u : 0u;
+    plan.buffer_norm = (buffer_norm && !uniform) ? 1u : 0u;
+    plan_staged_top(v, uniform != 0, plan);
     const uint32_t R = kThreads / v.fanout;
     const int ki = v.log2_fanout;
     if (!row_mode && n_sub == 1 && !uniform && !buffer_norm && B >= kWideSampleFrom) {
@@ -854,8 +971,56 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     return cudaGetLastError() == cudaSuccess ? (int)n_sub + extra_launches : -1;
 }
 
-int prb_launch_gather(const PrbView& v, uint32_t B, const unsigned char* handoff, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s)
+int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned char* handoff, cudaStream_t s, int uniform, int buffer_norm)
+{
+    const int sm_count = prb_sm_count();
+    SamplePlan plan;
+    PrbBatch none;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) none.ptr[f] = nullptr;
+    plan_row_mode(v, none, plan);
+    plan.n_tasks = B; plan.first_task = 0; plan.ticket_total = 0;
+    plan.ring_stages = 0; plan.ring_stage_bytes = 0;
+    plan.uniform = uniform ? 1u : 0u;
+    plan.buffer_norm = (buffer_norm && !uniform) ? 1u : 0u;
+    plan_staged_top(v, uniform != 0, plan);
+    int launches = 1;
+    if (plan.buffer_norm) {
+        // the scan of the leaves goes first, on the same stream
+        const uint64_t per_cta = 256ull * 16ull;
+        uint64_t ctas = (v.capacity + per_cta - 1) / per_cta;
+        if (ctas > (uint64_t)sm_count * 4) ctas = (uint64_t)sm_count * 4;
+        prb_leaf_min_kernel<<<(unsigned)ctas, 256, 0, s>>>(v);
+        launches = 2;
+    }
+    // one CTA per SM at most (the kernel has to fit beside a row copy's CTAs), each walking its strata
+    // kThreads / K at a time; a small batch is spread thin, a group or two per CTA
+    const uint32_t R = kThreads / v.fanout;
+    const uint32_t per_cta = R >= 4 ? R / 4 : 1;
+    uint32_t grid = (B + per_cta - 1) / per_cta;
+    if (grid > (uint32_t)sm_count) grid = (uint32_t)sm_count;
+    const bool prefetch = !uniform && v.depth >= 2 && plan.top_levels < v.depth - 1;
+    const uint32_t groups_per_warp = 32u / v.fanout;
+    uint32_t smem = 0;
+    plan.pf_groups = 0; plan.pf_off = 0;
+    if (prefetch) {
+        uint32_t strata = (B + grid - 1) / grid;
+        strata = (strata + groups_per_warp - 1) / groups_per_warp * groups_per_warp;      // whole warps' worth of groups
+        if (strata > R) strata = R;
+        plan.pf_groups = strata;
+        smem = strata * v.fanout * v.fanout * (uint32_t)sizeof(float);
+    }
+    switch (v.fanout) {
+    case 2: prb_descend_kernel<2><<<grid, kThreads, smem, s>>>(v, B, seed, handoff, plan); break;
+    case 4: prb_descend_kernel<4><<<grid, kThreads, smem, s>>>(v, B, seed, handoff, plan); break;
+    case 8: prb_descend_kernel<8><<<grid, kThreads, smem, s>>>(v, B, seed, handoff, plan); break;
+    case 16: prb_descend_kernel<16><<<grid, kThreads, smem, s>>>(v, B, seed, handoff, plan); break;
+    default: prb_descend_kernel<32><<<grid, kThreads, smem, s>>>(v, B, seed, handoff, plan); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned char* handoff, int32_t* d_idx, float* d_w,
+                      const PrbBatch& dst, cudaStream_t s, bool early_reads)
 {
     SamplePlan plan;
     if (!plan_row_mode(v, dst, plan)) return -1;
@@ -867,22 +1032,33 @@ int prb_launch_gather(const PrbView& v, uint32_t B, const unsigned char* handoff
     plan.uniform = 0; plan.buffer_norm = 0; plan.top_levels = 0; plan.top_vec4 = 0;
     for (uint32_t l = 0; l < PRB_MAX_LEVELS; ++l) plan.top_off[l] = 0;
     plan.pf_groups = 0; plan.pf_off = 0;
-    plan.found = nullptr;
     uint32_t stage = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) stage = plan.chunk[f] * 16u > stage ? plan.chunk[f] * 16u : stage;
     stage = (stage + 127u) / 128u * 128u;
     plan.ring_stage_bytes = stage;
-    plan.ring_stages = kRingBytes / stage;
+    plan.ring_stages = kGatherRingBytes / stage;
     if (plan.ring_stages > 32) plan.ring_stages = 32;
     const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
     static bool big_smem[kPrbMaxDevices];
     if (!big_smem[dev]) {
         if (cudaFuncSetAttribute(prb_gather_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
+                                 (int)(kRingBarBytes + kGatherRingBytes)) != cudaSuccess)
             return -1;
         big_smem[dev] = true;
     }
     const uint32_t grid = plan.n_tasks < (uint32_t)sm_count ? plan.n_tasks : (uint32_t)sm_count;
-    prb_gather_rows_kernel<<<grid, kGatherThreads, smem, s>>>(v, B, handoff, d_idx, d_w, dst, plan);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    // (launched as a programmatic dependent of the kernel before it on the stream: see the kernel)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kGatherThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint32_t early = early_reads ? 1u : 0u;
+    if (cudaLaunchKernelEx(&cfg, prb_gather_rows_kernel, v, B, beta, handoff, d_idx, d_w, dst, plan, early) != cudaSuccess) return -1;
+    return 1;
 }

@@ -8,95 +8,16 @@
 // the top of the tree, which is staged in shared memory.  More entries: one cooperative launch of
 // many CTAs (prb_update_wide_kernel, below).
 #include "prb_tree.cuh"
-#include "prb_descend.cuh"
 
 namespace {
 
-// Sampling ahead: the descents and weights of the sample that follows the tree work of this kernel, by
-// the same CTAs, as soon as that work is done (the tree's top is in CTA 0's shared memory, current, and
-// no launch or state read lies between).  Every thread walks strata of its own (prb_descend_alone); the
-// batch's largest raw weight is found over the cluster through CTA 0's shared memory; indices and
-// normalised weights go to a hand-off area of the slab, from where the kernel that copies the rows
-// (prb_gather_rows_kernel) takes them.  The results are those of prb_sample_kernel.
-template <int K>
-__device__ __forceinline__ void prb_sample_ahead(const PrbView& v, const PrbTeam& team, const PrbTop& top, const PrbSampleAhead& sa,
-                                                 unsigned long long fill, unsigned long long calls, unsigned long long* s_wmax,
-                                                 unsigned long long* s_warp)
-{
-    // the tree work of every CTA of the cluster is done and visible (the root was written by CTA 0)
-    team.phase_sync();
-    const float total32 = __ldcg(v.level[0]);
-    const bool empty = (fill == 0) || !(total32 > 0.0f);
-    const double total = (double)total32;
-    const float* s_top = top.mem;
-    if (team.parts > 1 && top.mem != nullptr)
-        s_top = reinterpret_cast<const float*>(__cluster_map_shared_rank(top.mem, 0));      // CTA 0's copy, read in place
-    int32_t* out_idx = const_cast<int32_t*>(prb_handoff_idx(sa.handoff));
-    float* out_w = const_cast<float*>(prb_handoff_w(sa.handoff, v.max_batch));
-    const uint32_t stride = team.parts * team.size, first = team.part * team.size + team.rank;
-    unsigned flags = 0u;
-    unsigned long long my_wmax = 0ull;
-    if (!empty) {
-        for (uint32_t k = first; k < sa.B; k += stride) {
-            const double x = prb_stratum_target(k, sa.B, total, calls, sa.seed);
-            uint32_t leaf; float p;
-            prb_descend_alone<K, true>(v, prb_top_levels(v, top), v.top_off, s_top, x, leaf, p, flags);
-            out_idx[k] = (int32_t)leaf;
-            const double wr = pow(__ddiv_rn(__dmul_rn((double)fill, (double)p), total), -(double)sa.beta);
-            v.wraw[k] = wr;
-            my_wmax = max(my_wmax, (unsigned long long)__double_as_longlong(wr));       // (positive binary64 values order like their bits)
-        }
-    }
-    // the largest raw weight: per warp, per CTA, then over the cluster through CTA 0's shared memory
-    // (slot `part` of its s_wmax, written and read with the cluster forms of the shared-memory accesses)
-    for (int o = 16; o > 0; o >>= 1) my_wmax = max(my_wmax, __shfl_xor_sync(0xFFFFFFFFu, my_wmax, o));
-    flags = __reduce_or_sync(0xFFFFFFFFu, flags);
-    if ((team.rank & 31u) == 0) {
-        s_warp[team.rank >> 5] = my_wmax;
-        if (flags) atomicOr(&v.state->status, flags);
-    }
-    team.sync();
-    uint32_t slots0;              // shared::cluster address of CTA 0's s_wmax
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(slots0) : "r"((uint32_t)__cvta_generic_to_shared(s_wmax)), "r"(0u));
-    if (team.rank == 0) {
-        unsigned long long m = 0ull;
-        for (uint32_t w = 0; w < team.size / 32u; ++w) m = max(m, s_warp[w]);
-        asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(slots0 + 8u * team.part), "l"(m) : "memory");
-    }
-    team.phase_sync();
-    unsigned long long wbits = 0ull;
-    for (uint32_t q = 0; q < team.parts; ++q) {
-        unsigned long long m;
-        asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(m) : "r"(slots0 + 8u * q) : "memory");
-        wbits = max(wbits, m);
-    }
-    if (!empty) {
-        const double wmax = __longlong_as_double((long long)wbits);
-        for (uint32_t k = first; k < sa.B; k += stride) out_w[k] = (float)__ddiv_rn(v.wraw[k], wmax);
-    }
-    if (team.part == 0 && team.rank == 0) {
-        if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
-        else v.state->sample_calls = calls + 1;
-        *reinterpret_cast<unsigned int*>(sa.handoff) = empty ? 0u : 1u;
-    }
-    // (no CTA of the cluster leaves while another may still read its shared memory)
-    if (team.parts > 1) team.phase_sync();
-}
-
-// kAhead: the kernel goes on to sample ahead (at most 512 threads per CTA then, so that a thread may keep
-// the 32 children of a node in registers).
-template <bool kAhead>
-__global__ void __launch_bounds__(kAhead ? 512 : 1024)
+__global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
                   const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale,
-                  uint32_t ins_n, const float* __restrict__ ins_prio, uint32_t ticket_total,
-                  const __grid_constant__ PrbSampleAhead ahead)
+                  uint32_t ins_n, const float* __restrict__ ins_prio, uint32_t ticket_total)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned long long s_cursor, s_fill;
-    __shared__ unsigned long long s_wmax[8];             // sampling ahead: the largest raw weight of each CTA of the cluster (CTA 0's copy is used)
-    __shared__ unsigned long long s_warp[32];            // ... and of each warp of this CTA
-    const unsigned long long calls = kAhead ? v.state->sample_calls : 0ull;
     PrbTeam team;
     team.rank = threadIdx.x;
     team.size = blockDim.x;
@@ -122,21 +43,7 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
         fill = v.state->fill;
         if (stale) cursor = v.state->cursor;
     }
-    if (B || ins_n)
-        prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top);
-    else
-        { prb_top_wait(); team.sync(); }                 // (sampling ahead only: the staged top has arrived)
-    if (kAhead) {
-        unsigned long long fill_after = fill + ins_n;
-        if (fill_after > v.capacity) fill_after = v.capacity;
-        switch (v.fanout) {
-        case 2: prb_sample_ahead<2>(v, team, top, ahead, fill_after, calls, s_wmax, s_warp); break;
-        case 4: prb_sample_ahead<4>(v, team, top, ahead, fill_after, calls, s_wmax, s_warp); break;
-        case 8: prb_sample_ahead<8>(v, team, top, ahead, fill_after, calls, s_wmax, s_warp); break;
-        case 16: prb_sample_ahead<16>(v, team, top, ahead, fill_after, calls, s_wmax, s_warp); break;
-        default: prb_sample_ahead<32>(v, team, top, ahead, fill_after, calls, s_wmax, s_warp); break;
-        }
-    }
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top);
 }
 
 // ---- large batches: one launch of many CTAs ------------------------------------------------------
@@ -389,13 +296,11 @@ int prb_launch_get_priorities(const PrbView& v, uint32_t B, const int32_t* d_idx
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-uint32_t prb_update_ctas(const PrbView& v, uint32_t b, const PrbSampleAhead* ahead)
+uint32_t prb_update_ctas(const PrbView& v, uint32_t b)
 {
     // Many wide child groups per level (fanout 32, hundreds of entries) are more L2 misses than
-    // one SM keeps in flight: then eight CTAs of one cluster share each level.  The same holds for
-    // the strata of a sample the kernel is to take afterwards.
-    const uint32_t most = (ahead != nullptr && ahead->B > b) ? ahead->B : b;
-    return (v.fanout * most >= 8192u) ? 8u : 1u;
+    // one SM keeps in flight: then eight CTAs of one cluster share each level.
+    return (v.fanout * b >= 8192u) ? 8u : 1u;
 }
 
 // The many-CTA update of a large batch: 1 launch, or 0 if this device cannot run it (no cooperative
@@ -438,47 +343,31 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
 
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale,
-                      uint32_t ins_n, const float* ins_prio, const PrbSampleAhead* ahead)
+                      uint32_t ins_n, const float* ins_prio)
 {
     if (ins_n && B > PEARL_UPDATE_SUBBATCH) return -1;
-    PrbSampleAhead none = PrbSampleAhead{0u, 0.0f, 0ull, nullptr};
     // a batch of more than one entry per thread of a CTA: one launch of many CTAs (values or TD errors;
     // changes keep their batch order and go sub-batch by sub-batch below)
     if (B > kPrbWideFrom && raw != 2 && ins_n == 0 && B < 0x80000000u) {
         const int k = prb_launch_update_wide(v, B, d_idx, d_val, raw, alpha, eps, s, stale);
-        if (k < 0) return k;
-        if (k > 0) {
-            if (ahead == nullptr) return k;
-            const int k2 = prb_launch_update(v, 0, d_idx, d_val, raw, alpha, eps, s, 0, 0, nullptr, ahead);
-            return k2 < 0 ? k2 : k + k2;
-        }
+        if (k != 0) return k;
     }
     static bool big_smem[kPrbMaxDevices];
     const int dev = prb_current_device();
     if (!big_smem[dev]) {
-        const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float));
-        if (cudaFuncSetAttribute(prb_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(prb_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
+        if (cudaFuncSetAttribute(prb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float))) != cudaSuccess)
             return -1;
         big_smem[dev] = true;
     }
     // A batch beyond one CTA's reach goes sub-batch by sub-batch in batch order: every launch leaves
-    // a consistent tree and later entries overwrite earlier ones, as in the whole batch.  The last
-    // launch (the only one of a tree kernel without an update) samples ahead, if asked to.
+    // a consistent tree and later entries overwrite earlier ones, as in the whole batch.
     int launches = 0;
-    for (uint32_t first = 0; first < B || (B == 0 && ahead != nullptr && launches == 0); first += PEARL_UPDATE_SUBBATCH) {
+    for (uint32_t first = 0; first < B; first += PEARL_UPDATE_SUBBATCH) {
         const uint32_t b = B - first < PEARL_UPDATE_SUBBATCH ? B - first : PEARL_UPDATE_SUBBATCH;
-        const bool last = first + b >= B;
-        const PrbSampleAhead& sa = (ahead != nullptr && last) ? *ahead : none;
         const uint32_t n2 = prb_update_n2(b);
-        uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
-        const uint32_t ctas = prb_update_ctas(v, b, sa.B ? &sa : nullptr);
-        if (sa.B) {
-            // the strata are dealt over the cluster's threads
-            uint32_t per_cta = ((sa.B + ctas - 1) / ctas + 31u) / 32u * 32u;
-            if (per_cta > threads) threads = per_cta;
-            if (threads > 512u) threads = 512u;
-        }
+        const uint32_t threads = n2 < 64 ? 64 : (n2 > 1024 ? 1024 : n2);
+        const uint32_t ctas = prb_update_ctas(v, b);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(ctas);
         cfg.blockDim = dim3(threads);
@@ -491,11 +380,9 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = sa.B ? cudaLaunchKernelEx(&cfg, prb_update_kernel<true>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
-                                                        eps, stale, ins_n, ins_prio, ctas, sa)
-                                   : cudaLaunchKernelEx(&cfg, prb_update_kernel<false>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
-                                                        eps, stale, ins_n, ins_prio, ctas, sa);
-        if (e != cudaSuccess) return -1;
+        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale,
+                               ins_n, ins_prio, ctas) != cudaSuccess)
+            return -1;
         ++launches;
     }
     return launches;
