@@ -31,9 +31,8 @@ METRIC = "PRB sample+update transitions/s at batch B"
 UNIT = "transitions/s"
 ROTATE = 8           # distinct input/output batch buffers cycled through, so inputs exceed L2 where rows are long
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) of one prb_sample_kernel launch on Atari-shaped rows with B = 512, from the
-# ncu capture summarised in profiles/prb_kernels_atari_N32768.md.  Null it if that kernel changes.
-SAMPLE_TRAFFIC_NCU = {"atari_dqn": 29.6e6}      # dram read + write of one sample launch (profiles/)
+SHORT_REGION_MS = 50.0     # a timed region shorter than this is repeated and the median taken
+REGION_REPS = 5
 
 
 def load_peak():
@@ -47,10 +46,24 @@ def load_peak():
 # ------------------------------------------------------------------------------------------
 # CPU oracle arm (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------
+def host_available_bytes():
+    """Host memory that can still be had (MemAvailable), or a cautious guess."""
+    try:
+        with open("/proc/meminfo") as f:
+            for ln in f:
+                if ln.startswith("MemAvailable:"):
+                    return int(ln.split()[1]) * 1024
+    except Exception:
+        pass
+    return 8 << 30
+
+
 def oracle_capacity(wl):
-    """Capacity the oracle is timed at: the workload's, unless its store would not fit the host."""
+    """Capacity the oracle is timed at: the workload's where its store fits in 60 % of the host memory
+    still available (the oracle keeps the whole Data Storage), else the largest power-of-two part that does."""
+    room = int(host_available_bytes() * 0.6)
     cap = wl.capacity
-    while cap * wl.transition_bytes > (6 << 30):
+    while cap > 1024 and cap * (wl.transition_bytes + 64) > room:
         cap //= 2
     return cap
 
@@ -63,9 +76,13 @@ def oracle_setup(wl, capacity):
     o = oracle.OraclePRB(capacity, wl.fanout, wl.obs_bytes, wl.act_bytes)
     plain = wk.scaled(wl, capacity, counter_rows=False)      # same shapes; bytes from numpy (content is irrelevant to time)
     chunk = max(1, min(capacity, (64 << 20) // wl.transition_bytes))
+    # one chunk of rows serves the whole prefill (only the priorities are fresh): filling 30 GB with fresh
+    # random bytes would take longer than the measurement
+    rows = wk.transitions(plain, rng, chunk)
     for first in range(0, capacity, chunk):
-        b = wk.transitions(plain, rng, min(chunk, capacity - first))
-        o.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+        n = min(chunk, capacity - first)
+        prio = wk.priorities(plain, rng, n)
+        o.insert(rows["obs"][:n], rows["act"][:n], rows["rew"][:n], rows["next_obs"][:n], rows["done"][:n], prio)
     batches = [wk.transitions(plain, rng, max(wl.n_insert, 1)) for _ in range(ROTATE)]
     tds = [wk.td_errors(wl, rng, wl.batch) for _ in range(ROTATE)]
     return o, plain, batches, tds, rng
@@ -100,7 +117,7 @@ def time_oracle(wl, steps, warmup, budget_s=None):
     sample = "%d steps of the %s step (insert %d, sample %d, update %d)" % (done, wl.name, wl.n_insert, wl.batch, wl.batch)
     if cap != wl.capacity:
         sample += " at capacity %d of %d (host memory)" % (cap, wl.capacity)
-    return done, dt, sample
+    return done, dt, sample, cap
 
 
 # ------------------------------------------------------------------------------------------
@@ -240,23 +257,37 @@ def copy_context(wl, store_rows, dev, stream):
             "note": "library kernels on the same observation bytes (read+write), indices given; context, not the product path"}
 
 
-def run_ours(args, wl, rank, world):
-    import torch
+def timed_regions(stream, run_steps, steps, world, dev):
+    """Times run_steps(steps) with CUDA events on `stream`, barrier + synchronise on both sides, maximum
+    over ranks.  A region shorter than SHORT_REGION_MS is run REGION_REPS times and all times returned
+    (the caller takes the median): a sub-millisecond region is at the mercy of one hiccup."""
     import torch.distributed as dist
+    times = []
+    for rep in range(REGION_REPS):
+        if world > 1:
+            dist.barrier()
+        ms = time_loop(stream, lambda i: run_steps(steps), 1)
+        if world > 1:
+            dist.barrier()
+            ms = max_over_ranks(ms, dev)
+        times.append(ms)
+        if ms >= SHORT_REGION_MS:
+            break
+    return times
+
+
+def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=True, e2e=True, use_graph=True, fused=True):
+    """Builds and fills one buffer for workload `wl` and times the step, its calls and the host-buffer step.
+    Returns a dict of raw measurements (milliseconds per step / per call)."""
+    import torch
     from paper_2311_09445_b200 import PrioritizedReplay
     from paper_2311_09445_b200 import workloads as wk
 
-    local = int(os.environ.get("LOCAL_RANK", 0))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda:%d" % local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    stream = torch.cuda.Stream(dev)
     rng = np.random.default_rng(wl.seed + 7919 * rank)
     B, n_ins = wl.batch, wl.n_insert
     chunk = 512 if wl.counter_rows else min(wl.capacity, 1 << 16)
     max_batch = max(B, n_ins, chunk)
-
+    m = {}
     with torch.cuda.stream(stream):
         prb = PrioritizedReplay(wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, max_batch, device=dev, stream=stream)
         # prefill the whole ring through the insert call
@@ -291,10 +322,12 @@ def run_ours(args, wl, rank, world):
             b = batches[i % ROTATE]
             prb.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
 
-        def do_sample(i):
+        def sample_args(i):
             o = outs[i % ROTATE]
-            prb.sample(B, wl.beta, wl.philox_seed, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
-                       o["rew"], o["next_obs"], o["done"])
+            return (o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None, o["rew"], o["next_obs"], o["done"])
+
+        def do_sample(i):
+            prb.sample(B, wl.beta, wl.philox_seed, *sample_args(i))
 
         def do_update(i):
             idx = upd_idx[i % ROTATE] if upd_idx else outs[i % ROTATE]["idx"]
@@ -306,7 +339,7 @@ def run_ours(args, wl, rank, world):
             prb.update_insert(idx, tds[i % ROTATE], wl.alpha, wl.eps, b["obs"], b["act"], b["rew"], b["next_obs"],
                               b["done"], b["prio"])
 
-        fused = bool(n_ins) and not args.unfused
+        fused = bool(n_ins) and fused
 
         def eager_step(i):
             # the paper's schedule (Eq. 7): sample, then update with the insertion running beside it
@@ -318,7 +351,7 @@ def run_ours(args, wl, rank, world):
                 if n_ins:
                     do_insert(i)
 
-        for i in range(max(args.warmup, 3)):
+        for i in range(max(warmup, 3)):
             eager_step(i)
         torch.cuda.synchronize()
         status = prb.sync()
@@ -327,7 +360,7 @@ def run_ours(args, wl, rank, world):
         # ROTATE consecutive steps, plus single-step graphs for a remainder of K
         l0 = prb.kernel_launches()
         eager_step(0)
-        kernels_per_step = prb.kernel_launches() - l0
+        m["kernels_per_step_eager"] = prb.kernel_launches() - l0
         torch.cuda.synchronize()
 
         def capture(calls):
@@ -337,8 +370,10 @@ def run_ours(args, wl, rank, world):
                     c()
             return g
 
-        if not args.no_graph:
+        if use_graph:
+            l0 = prb.kernel_launches()
             g_all = capture([lambda r=r: eager_step(r) for r in range(ROTATE)])
+            m["kernels_per_step"] = (prb.kernel_launches() - l0) / ROTATE
             g_one = [capture([lambda r=r: eager_step(r)]) for r in range(ROTATE)]
 
             def run_steps(k):
@@ -347,106 +382,143 @@ def run_ours(args, wl, rank, world):
                 for r in range(k % ROTATE):
                     g_one[r].replay()
         else:
+            m["kernels_per_step"] = m["kernels_per_step_eager"]
+
             def run_steps(k):
                 for i in range(k):
                     eager_step(i)
-        run_steps(max(args.warmup, 3))
+        run_steps(max(warmup, 3))
         torch.cuda.synchronize()
 
-        # ---- the timed region: exactly K steps -------------------------------------------
-        clocks = ClockSampler(local)
+        # ---- the timed region: exactly K steps (repeated, median, when it is short) ----------
+        clocks = ClockSampler(dev.index or 0)
         if rank == 0:
             clocks.start()
             time.sleep(0.3)
-        if world > 1:
-            dist.barrier()
-        ms = time_loop(stream, lambda i: run_steps(args.steps), 1)
-        if world > 1:
-            dist.barrier()
-            ms = max_over_ranks(ms, dev)
-        clk = clocks.stop() if rank == 0 else None
+        m["region_ms"] = timed_regions(stream, run_steps, steps, world, dev)
+        m["clocks"] = clocks.stop() if rank == 0 else None
 
         # ---- per-call timings (device resident), used for the roofline and the rates: a graph of
         # ROTATE back-to-back calls of one kind, replayed, so that host launch cost is not in them
-        reps = max(3, min(args.steps, 400) // ROTATE)
+        reps = max(3, min(steps, 400) // ROTATE)
 
         def per_call_ms(fn):
-            if args.no_graph:
+            if not use_graph:
                 for i in range(3):
                     fn(i)
                 return time_loop(stream, fn, reps * ROTATE) / (reps * ROTATE)
             g = capture([lambda r=r: fn(r) for r in range(ROTATE)])
             g.replay()
-            return time_loop(stream, lambda i: g.replay(), reps) / (reps * ROTATE)
+            return statistics.median(time_loop(stream, lambda i: g.replay(), reps) / (reps * ROTATE) for _ in range(3))
 
-        ms_sample = per_call_ms(do_sample)
-        ms_update = per_call_ms(do_update)
-        # the same update with its index batch in random order (the kernel has to sort it)
-        shuffled = [(upd_idx[r] if upd_idx else outs[r]["idx"])[torch.randperm(B, device=dev)] for r in range(ROTATE)]
-        ms_update_shuffled = per_call_ms(lambda i: prb.update(shuffled[i % ROTATE], tds[i % ROTATE], wl.alpha, wl.eps)) \
-            if not args.core_only else None
-        # the sample call issued as 4 sub-batches on 4 streams of the handle (whole call, all joined)
-        def do_sample_streamed(i):
-            o = outs[i % ROTATE]
-            prb.sample_streamed(B, wl.beta, wl.philox_seed, 4, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
-                                o["rew"], o["next_obs"], o["done"])
-        ms_streamed = per_call_ms(do_sample_streamed) if (B >= 4 and not args.core_only) else None
-
-        # the sample call with weights normalised over the whole buffer (a scan of the leaves goes first)
-        def do_sample_buffer_norm(i):
-            o = outs[i % ROTATE]
-            prb.sample_buffer_norm(B, wl.beta, wl.philox_seed, o["idx"], o["w"], o["obs"], o["act"] if wl.act_bytes else None,
-                                   o["rew"], o["next_obs"], o["done"])
-        ms_buffer_norm = per_call_ms(do_sample_buffer_norm) if not args.core_only else None
-        ms_insert = per_call_ms(do_insert) if n_ins else None
-        ms_fused = per_call_ms(do_update_insert) if fused else None
+        m["ms_sample"] = per_call_ms(do_sample)
+        m["ms_update"] = per_call_ms(do_update)
+        m["ms_insert"] = per_call_ms(do_insert) if n_ins else None
+        m["ms_update_insert"] = per_call_ms(do_update_insert) if fused else None
+        if extras:
+            # the same update with its index batch in random order (the kernel has to sort it)
+            shuffled = [(upd_idx[r] if upd_idx else outs[r]["idx"])[torch.randperm(B, device=dev)] for r in range(ROTATE)]
+            m["ms_update_shuffled"] = per_call_ms(lambda i: prb.update(shuffled[i % ROTATE], tds[i % ROTATE], wl.alpha, wl.eps))
+            # the sample as one kernel, whatever the call before it (the form a sample takes outside a stream
+            # capture and right after an update + insertion), through the call that always takes that form
+            if B <= 4096:
+                m["ms_sample_one_kernel"] = per_call_ms(lambda i: prb.sample_static_scratch(B, wl.beta, wl.philox_seed, *sample_args(i)))
+            # the sample issued as 4 sub-batches on 4 streams of the handle (whole call, all joined)
+            if B >= 4:
+                m["ms_sample_streamed4"] = per_call_ms(lambda i: prb.sample_streamed(B, wl.beta, wl.philox_seed, 4, *sample_args(i)))
+            # the sample with weights normalised over the whole buffer
+            m["ms_sample_buffer_norm"] = per_call_ms(lambda i: prb.sample_buffer_norm(B, wl.beta, wl.philox_seed, *sample_args(i)))
         status |= prb.sync()
 
         # ---- end to end through the host-buffer calls ----------------------------------------
-        e2e_steps = max(5, min(args.steps, 100 if wl.counter_rows else 500))
-        hb = []
-        for r in range(ROTATE):
-            d = batches[r]
-            hb.append({k: v.cpu().pin_memory() for k, v in d.items()})
-        ho = out_buffers(wl, dev, B, pinned=True)
-        htd = [t.cpu().pin_memory() for t in tds]
+        if e2e:
+            e2e_steps = max(5, min(steps, 100 if wl.counter_rows else 500))
+            hb = [{k: v.cpu().pin_memory() for k, v in batches[r].items()} for r in range(ROTATE)]
+            ho = out_buffers(wl, dev, B, pinned=True)
+            htd = [t.cpu().pin_memory() for t in tds]
 
-        def e2e_step(i):
-            if n_ins:
-                b = hb[i % ROTATE]
-                prb.insert_host(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
-            prb.sample_host(B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
-                            ho["rew"], ho["next_obs"], ho["done"])
-            prb.update_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps)
+            def e2e_step(i):
+                if n_ins:
+                    b = hb[i % ROTATE]
+                    prb.insert_host(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
+                prb.sample_host(B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
+                                ho["rew"], ho["next_obs"], ho["done"])
+                prb.update_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps)
 
-        for i in range(0 if args.no_e2e else 3):
-            e2e_step(i)
-        if world > 1:
-            dist.barrier()
-        ms_e2e = time_loop(stream, e2e_step, e2e_steps) if not args.no_e2e else float("nan")
-        if world > 1:
-            dist.barrier()
-            ms_e2e = max_over_ranks(ms_e2e, dev)
-        status |= prb.sync()
-        fill, cursor, calls, depth = prb.info()
+            for i in range(3):
+                e2e_step(i)
+            import torch.distributed as dist
+            if world > 1:
+                dist.barrier()
+            ms_e2e = time_loop(stream, e2e_step, e2e_steps)
+            if world > 1:
+                dist.barrier()
+                ms_e2e = max_over_ranks(ms_e2e, dev)
+            m["ms_e2e_step"] = ms_e2e / e2e_steps
+            m["e2e_steps"] = e2e_steps
+            status |= prb.sync()
+        m["status"] = status
+        m["depth"] = prb.info()[3]
         prb.close()
-        ctx = None
-        if rank == 0 and world == 1 and wl.obs_bytes >= 8192 and not args.no_copy_context:
-            ctx = copy_context(wl, wl.capacity, dev, stream)
+    return m
 
+
+def summary_of(wl, m, world=1):
+    """The figures the benchmark spec asks for, for one workload: step time, samples/s, updates/s, inserts/s, e2e."""
+    B, n_ins = wl.batch, wl.n_insert
+    ms_step = statistics.median(m["region_ms"]) / m["steps"]
+    out = {"us_step": ms_step * 1e3, "transitions_per_s": world * B / (ms_step * 1e-3),
+           "samples_per_s": B / (m["ms_sample"] * 1e-3), "updates_per_s": B / (m["ms_update"] * 1e-3),
+           "inserts_per_s": (n_ins / (m["ms_insert"] * 1e-3)) if m.get("ms_insert") else None,
+           "us_sample": m["ms_sample"] * 1e3, "us_update": m["ms_update"] * 1e3,
+           "us_insert": m["ms_insert"] * 1e3 if m.get("ms_insert") else None,
+           "us_update_insert": m["ms_update_insert"] * 1e3 if m.get("ms_update_insert") else None}
+    if "ms_e2e_step" in m:
+        out["e2e_transitions_per_s"] = world * B / (m["ms_e2e_step"] * 1e-3)
+    return out
+
+
+def run_ours(args, wl, rank, world):
+    import torch
+    import torch.distributed as dist
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda:%d" % local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    stream = torch.cuda.Stream(dev)
+    B, n_ins = wl.batch, wl.n_insert
+    fused = bool(n_ins) and not args.unfused
+    m = measure_workload(wl, args.steps, args.warmup, dev, stream, rank, world, extras=not args.profile,
+                         e2e=not args.profile, use_graph=not args.no_graph, fused=fused)
+    m["steps"] = args.steps
+    ctx = None
+    others = None
+    if rank == 0 and world == 1 and not args.profile:
+        if wl.obs_bytes >= 8192:
+            with torch.cuda.stream(stream):
+                ctx = copy_context(wl, wl.capacity, dev, stream)
+        others = other_workloads(wl, dev, stream)
     if world > 1:
         dist.destroy_process_group()
     if rank != 0:
         return None
 
     E = wl.transition_bytes
+    depth = m["depth"]
+    ms = statistics.median(m["region_ms"])
     h2d = (n_ins * (E + 4) if n_ins else 0) + B * 8
     d2h = B * (E + 8)
     peak, peak_kind = load_peak()
-    # algorithmic bytes of one sample launch: D child groups of K binary32 per stratum, index and
+    # algorithmic bytes of one sample call: D child groups of K binary32 per stratum, index and
     # weight written, every field of the row read once and written once
     sample_bytes = B * (depth * wl.fanout * 4 + 8 + 2 * E)
-    achieved = sample_bytes / (ms_sample * 1e-3) / 1e9
+    long_rows = wl.obs_bytes >= 8192 and wl.obs_bytes % 16 == 0
+    achieved = sample_bytes / (m["ms_sample"] * 1e-3) / 1e9
+    rates = summary_of(wl, m, world)
+    for k in ("ms_update_shuffled", "ms_sample_one_kernel", "ms_sample_streamed4", "ms_sample_buffer_norm"):
+        rates["us" + k[2:]] = m[k] * 1e3 if m.get(k) else None
     line = {
         "metric": METRIC, "value": world * B * args.steps / (ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -456,36 +528,71 @@ def run_ours(args, wl, rank, world):
                    "insert_per_step": n_ins, "transition_bytes": E, "step": "sample(idx,IS,gather) + update_insert" if fused else "sample(idx,IS,gather) + update + insert",
                    "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph,
                    "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
-        "rates": {"samples_per_s": B / (ms_sample * 1e-3), "updates_per_s": B / (ms_update * 1e-3),
-                  "inserts_per_s": (n_ins / (ms_insert * 1e-3)) if n_ins else None,
-                  "us_sample": ms_sample * 1e3, "us_update": ms_update * 1e3, "us_update_shuffled": ms_update_shuffled * 1e3 if ms_update_shuffled else None,
-                  "us_insert": ms_insert * 1e3 if n_ins else None,
-                  "us_update_insert": ms_fused * 1e3 if fused else None,
-                  "us_sample_streamed4": ms_streamed * 1e3 if ms_streamed else None,
-                  "us_sample_buffer_norm": ms_buffer_norm * 1e3 if ms_buffer_norm else None},
-        "roofline": {"kernel": "prb_sample_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "timed_region": {"repeats": len(m["region_ms"]), "ms_each": m["region_ms"],
+                         "value_from": "median" if len(m["region_ms"]) > 1 else "the one region"},
+        "rates": rates,
+        "roofline": {"kernel": "prb_gather_rows_kernel (+ prb_descend_kernel beside the copy before it)" if long_rows and not args.no_graph
+                     else "prb_sample_kernel",
+                     "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "bytes_per_launch": sample_bytes,
-                     "traffic": SAMPLE_TRAFFIC_NCU.get(wl.name) if B == 512 else None},
-        "e2e": {"value": None if args.no_e2e else world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": e2e_steps,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(kernels_per_step * args.steps),
-        "kernels_per_step": int(kernels_per_step),
-        "status_bits": int(status),
-        "clocks": clk,
+                     "timing": "captured graph of %d consecutive sample calls, replayed; per call" % ROTATE,
+                     "traffic": None,
+                     "traffic_note": "dram bytes of one launch are in profiles/ (ncu, reduced capacity); not measured in this run"},
+        "gpu_launches": int(round(m["kernels_per_step"] * args.steps)),
+        "kernels_per_step": m["kernels_per_step"],
+        "status_bits": int(m["status"]),
+        "clocks": m["clocks"],
     }
+    if "ms_e2e_step" in m:
+        line["e2e"] = {"value": world * B / (m["ms_e2e_step"] * 1e-3), "unit": UNIT, "steps": m["e2e_steps"],
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    else:
+        line["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    step_bytes = B * (depth * wl.fanout * 4 + 8 + 2 * E) + (n_ins * (2 * E + 4) if n_ins else 0)
+    line["roofline_step"] = {"bound": "hbm", "bytes_per_step": step_bytes, "achieved": step_bytes / (ms / args.steps * 1e-3) / 1e9,
+                             "peak": peak, "unit": "GB/s", "frac": step_bytes / (ms / args.steps * 1e-3) / 1e9 / peak}
     if n_ins:
         ins_bytes = n_ins * (2 * E + 4)
-        line["roofline_insert"] = {"kernel": "prb_insert_kernel", "bound": "hbm", "bytes_per_launch": ins_bytes,
-                                   "achieved": ins_bytes / (ms_insert * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
-                                   "frac": ins_bytes / (ms_insert * 1e-3) / 1e9 / peak}
+        line["roofline_insert"] = {"kernel": "prb_insert_rows_kernel" if long_rows else "prb_insert_kernel", "bound": "hbm",
+                                   "bytes_per_launch": ins_bytes,
+                                   "achieved": ins_bytes / (m["ms_insert"] * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": ins_bytes / (m["ms_insert"] * 1e-3) / 1e9 / peak}
     if ctx is not None:
         line["roofline"]["context"] = ctx
-    if world == 1 and not args.no_cpu_baseline:
-        done, dt, sample = time_oracle(wl, 10 ** 9, 2, budget_s=args.cpu_budget)
+    if others is not None:
+        line["workloads"] = others
+    if world == 1 and not args.profile:
+        done, dt, sample, cap = time_oracle(wl, 10 ** 9, 2, budget_s=args.cpu_budget)
         line["cpu_baseline"] = {"value": B * done / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-                                "host_cpus": os.cpu_count()}
+                                "capacity": cap, "host_cpus": os.cpu_count()}
     return line
+
+
+# the other workloads the benchmark spec names, and three cells of the scaling sweep: short runs after the headline's
+OTHER_SWEEP_CELLS = [(1 << 20, 16, 1024), (1 << 22, 32, 4096), (1 << 24, 4, 65536)]
+
+
+def other_workloads(headline, dev, stream):
+    import torch
+    from paper_2311_09445_b200 import workloads as wk
+    out = {}
+    todo = [w for name, w in wk.WORKLOADS.items() if name != headline.name]
+    todo += [wk.sweep_cell(n, k, b, cell_id=n % 997 + k + b) for n, k, b in OTHER_SWEEP_CELLS]
+    for wl in todo:
+        free, _ = torch.cuda.mem_get_info(dev)
+        if wl.capacity * wl.transition_bytes + (4 << 30) > free + torch.cuda.memory_reserved(dev):
+            out[wl.name] = {"skipped": "not enough free device memory"}
+            continue
+        steps = 200
+        m = measure_workload(wl, steps, 3, dev, stream, extras=False, e2e=wl.capacity <= (1 << 20))
+        m["steps"] = steps
+        d = summary_of(wl, m)
+        d.update(capacity=wl.capacity, fanout=wl.fanout, batch=wl.batch, insert_per_step=wl.n_insert, steps=steps,
+                 region_repeats=len(m["region_ms"]), status_bits=int(m["status"]))
+        out[wl.name] = d
+        torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------------------------------------
@@ -611,16 +718,28 @@ def run_reference(args, wl, rank, world):
     warm = max(args.warmup, 1)
     per_step_guess = 0.03 if wl.counter_rows else 0.001
     steps = max(1, min(args.steps, int(120 / per_step_guess)))
-    done, dt, sample = time_oracle(wl, steps, warm, budget_s=150)
+    done, dt, sample, cap = time_oracle(wl, steps, warm, budget_s=150)
     v = wl.batch * done / dt
     return {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world, "steps": done,
             "warmup": warm, "ms_per_step": dt / done * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
-            "config": {"workload": wl.name, "capacity": oracle_capacity(wl), "fanout": wl.fanout, "batch": wl.batch,
+            "config": {"workload": wl.name, "capacity": cap, "fanout": wl.fanout, "batch": wl.batch,
                        "insert_per_step": wl.n_insert, "step": "insert+sample(idx,IS,gather)+update"},
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
+
+
+def relaunch_as_ranks(n):
+    """`python bench.py --gpus N` outside a launcher: start N ranks of this script on this node and pass
+    their output through (rank 0 prints the one line)."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -632,19 +751,19 @@ def main():
     ap.add_argument("--workload", default="atari_dqn")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--unfused", action="store_true", help="update and insert as two launches instead of pearl_prb_update_insert")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--no-copy-context", action="store_true", help="skip the torch copy / index_select context timings")
-    ap.add_argument("--core-only", action="store_true",
-                    help="time only the step and its three calls (no shuffled-update, streamed or buffer-normalised sample timings)")
-    ap.add_argument("--capacity", type=int, default=0, help="override the workload's capacity (profiling runs)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
-    ap.add_argument("--sweep-fanout", type=int, default=0, help="with --sweep: this fanout only")
-    ap.add_argument("--sweep-batch", type=int, default=0, help="with --sweep: this batch size only")
     ap.add_argument("--sweep", action="store_true",
-                    help="time every cell of the capacity x fanout x batch sweep instead (one GPU; --capacity picks one capacity)")
+                    help="time every cell of the capacity x fanout x batch sweep instead (one GPU)")
+    prof = ap.add_argument_group("profiling runs (under ncu: the step and its three calls only, a smaller store)")
+    prof.add_argument("--profile", action="store_true",
+                      help="only the step and its calls: no host-buffer leg, no context timings, no other workloads, no CPU baseline")
+    prof.add_argument("--capacity", type=int, default=0, help="override the workload's capacity; with --sweep: this capacity only")
+    prof.add_argument("--sweep-fanout", type=int, default=0, help="with --sweep: this fanout only")
+    prof.add_argument("--sweep-batch", type=int, default=0, help="with --sweep: this batch size only")
     args = ap.parse_args()
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep:
+        sys.exit(relaunch_as_ranks(args.gpus))
     from paper_2311_09445_b200 import workloads as wk
     if args.sweep:
         if int(os.environ.get("RANK", 0)) == 0:
