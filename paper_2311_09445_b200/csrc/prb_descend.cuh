@@ -70,6 +70,7 @@ __device__ __forceinline__ void prb_descend_alone(const PrbView& v, uint32_t top
     for (uint32_t l = 1; l <= v.depth; ++l) {
         float c[K];
         const bool staged = l <= top_levels;
+        if (!PRB_IN_BOUNDS(v, g * K + K <= v.level_alloc[l])) { flags |= PEARL_ST_INTERNAL; g = 0; }
         prb_load_children<K, kCoherent>(staged ? s_top + top_off[l] + (uint32_t)g * K : v.level[l] + g * K, !staged, c);
         int j = -1, last_pos = -1;
         float run = 0.0f, before_j = 0.0f, before_last = 0.0f;

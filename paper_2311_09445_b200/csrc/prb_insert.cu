@@ -58,6 +58,7 @@ __device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const Pr
                            const uint32_t r = e / W;
                            uint64_t slot = cursor + r;
                            if (slot >= N) slot -= N;
+                           if (!PRB_IN_BOUNDS(v, slot < N && r < n)) slot = 0;
                            return slot * W + (e - r * W);
                        },
                        rank, nthreads);
@@ -188,6 +189,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         while (t < t_hi) {
             uint64_t slot = cursor + row;
             if (slot >= v.capacity) slot -= v.capacity;
+            if (!PRB_IN_BOUNDS(v, slot < v.capacity && row < n && e0 < W && bytes <= plan.ring_stage_bytes)) slot = 0;
             ring.store(v.store[f] + (slot * W + e0) * 16u, bytes);
             t += plan.ring_stages;
             if (t < t_hi) {

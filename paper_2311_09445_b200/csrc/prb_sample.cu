@@ -101,6 +101,7 @@ __device__ __forceinline__ void descend(const PrbView& v, const SamplePlan& plan
     int j = 0;
     for (uint32_t l = 1; l <= v.depth; ++l) {
         const float* row;
+        if (!PRB_IN_BOUNDS(v, g * K + K <= v.level_alloc[l])) { flags |= PEARL_ST_INTERNAL; g = 0; }
         if (l <= plan.top_levels) {
             row = s_top + plan.top_off[l] + (uint32_t)g * K;
         } else if (pf != nullptr && l == v.depth) {
@@ -187,7 +188,8 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
             const uint32_t e = rank + u * nthreads;
             if (e < total) {
                 const uint32_t r = (W == 1) ? e : e / W;
-                tmp[f][u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
+                if (PRB_IN_BOUNDS(v, s_idx[r] < v.capacity))
+                    tmp[f][u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
             }
         }
     }
@@ -203,7 +205,8 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
         }
         for (uint32_t e = rank + 2 * nthreads; e < total; e += nthreads) {     // the rest of a larger batch
             const uint32_t r = e / W;
-            store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec));
+            if (PRB_IN_BOUNDS(v, s_idx[r] < v.capacity))
+                store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec));
         }
     }
 }
@@ -299,9 +302,10 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
         if (tid >= kThreads / 2) {
             // raw weights, indices and flags of the strata this CTA owns (off the copy's critical path).
             // What another CTA reads -- the raw weights -- is written by atomics whose results are
-            // waited for: when a thread goes on, its value is in L2.  A fence here instead would also
-            // wait for the bulk copies the ring has in flight, and so put the ticket, and the
-            // normalisation of the weights behind it, after the whole copy.
+            // waited for, so that the values are on their way to L2 at once; the barrier below and the
+            // ticket's release/acquire pair (one thread's, not a fence in every thread, which was
+            // measured to wait for the bulk copies the ring has in flight) order them before the reads
+            // of the CTA that draws the last ticket.
             const uint32_t gi2 = tid - kThreads / 2;
             if (gi2 < n_round) {
                 if (kb + gi2 >= k_own) {
@@ -330,7 +334,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             if (tid == kThreads / 2 && last_descents) {
                 // every descent of this CTA is done and its weights are in L2: the last CTA to get
                 // here normalises the weights of the whole batch
-                s_last = (atomicAdd(&v.state->sample_ticket, 1u) == plan.ticket_total - 1) ? 1u : 0u;
+                s_last = (prb_ticket(&v.state->sample_ticket) == plan.ticket_total - 1) ? 1u : 0u;
             }
             if (last_descents) {
                 asm volatile("bar.sync 2, %0;" ::"n"(kThreads / 2) : "memory");
@@ -385,6 +389,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     const uint32_t W = v.field_bytes[f] / 16u;
                     const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
                     const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
+                    if (!PRB_IN_BOUNDS(v, s_idx[k - kb] < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes)) continue;
                     ring.load(v.store[f] + ((uint64_t)s_idx[k - kb] * W + e0) * 16u, bytes);
                     ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
                 }
@@ -431,7 +436,7 @@ __device__ __forceinline__ void gather_field_deep(const T* __restrict__ store, T
             const uint32_t e = e0 + u * nthreads;
             if (e < total) {
                 const uint32_t r = (W == 1) ? e : e / W;
-                tmp[u] = store[(uint64_t)s_idx[r] * W + (e - r * W)];
+                tmp[u] = store[(uint64_t)s_idx[r] * W + (e - r * W)];      // (s_idx comes from a descent, checked there)
             }
         }
 #pragma unroll
@@ -512,7 +517,7 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
     if (tid == 0) {
         if (s_flags) atomicOr(&v.state->status, s_flags);
         if (s_wmax) atomicMax(&v.state->wide_wmax_bits, s_wmax);
-        s_last = (atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+        s_last = (prb_ticket(&v.state->sample_ticket) == gridDim.x - 1) ? 1u : 0u;
     }
     __syncthreads();
     if (tid == 0 && s_last) {
@@ -540,7 +545,7 @@ prb_normalise_weights_kernel(const __grid_constant__ PrbView v, uint32_t B, floa
         for (uint32_t u = 0; u < 4; ++u) if (k0 + u * kThreads < B) out_w[k0 + u * kThreads] = (float)__ddiv_rn(held[u], wmax);
     }
     __syncthreads();        // every thread of the CTA has read the maximum
-    if (threadIdx.x == 0 && atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) {
+    if (threadIdx.x == 0 && prb_ticket(&v.state->sample_ticket) == gridDim.x - 1) {
         v.state->wide_wmax_bits = 0ull;
         v.state->sample_ticket = 0u;
     }
@@ -634,7 +639,7 @@ prb_descend_kernel(const __grid_constant__ PrbView v, uint32_t B, uint64_t seed,
         }
         __syncthreads();        // (a group's scratch and prefetch buffer are reused by the next round)
     }
-    if (tid == 0 && atomicAdd(&v.state->sample_ticket, 1u) == gridDim.x - 1) {
+    if (tid == 0 && prb_ticket(&v.state->sample_ticket) == gridDim.x - 1) {
         PrbHandoffHeader* hd = reinterpret_cast<PrbHandoffHeader*>(handoff);
         hd->found = empty ? 0u : 1u;
         hd->buffer_norm = plan.buffer_norm;
@@ -698,11 +703,12 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
             const uint32_t W = v.field_bytes[f] / 16u;
             const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
             const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
-            ring.load(v.store[f] + ((uint64_t)(uint32_t)leaf * W + e0) * 16u, bytes);
+            const bool inside = PRB_IN_BOUNDS(v, (uint32_t)leaf < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes);
+            if (inside) ring.load(v.store[f] + ((uint64_t)(uint32_t)leaf * W + e0) * 16u, bytes);
             const uint32_t t_next = t + plan.ring_stages;
             const int32_t leaf_next = t_next < t_hi ? __ldcg(pre_idx + t_next / tps) : 0;
             if (!waited) { prb_dep_wait(); waited = true; }
-            ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
+            if (inside) ring.store(dst.ptr[f] + ((uint64_t)k * W + e0) * 16u, bytes);
             t = t_next;
             leaf = leaf_next;
         }

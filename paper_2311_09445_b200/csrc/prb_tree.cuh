@@ -60,10 +60,10 @@ constexpr int kPrbPublishTree = 1, kPrbPublishRows = 2, kPrbPublishAll = 3;
 __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill,
                                                     uint32_t participants, int what = kPrbPublishAll)
 {
-    // no fence: the cursor and fill reads that must precede this ticket have returned their values
-    // (they were stored to shared memory before the barrier this thread has passed)
+    // (the cursor and fill reads of this CTA were stored to shared memory before the barrier this thread has
+    // passed; the ticket's release/acquire pair orders them before the last drawer's stores)
     unsigned int* ticket = (what == kPrbPublishRows) ? &v.state->row_ticket : &v.state->insert_ticket;
-    const unsigned int done = atomicAdd(ticket, 1u);
+    const unsigned int done = prb_ticket(ticket);
     if (done == participants - 1) {
         const uint64_t N = v.capacity;
         uint64_t c = cursor + n;
@@ -109,6 +109,7 @@ __device__ __forceinline__ void prb_top_wait() { asm volatile("cp.async.wait_all
 __device__ __forceinline__ void prb_resum(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T, uint32_t l, uint64_t a)
 {
     const uint32_t K = v.fanout;
+    if (!PRB_IN_BOUNDS(v, a * K + K <= v.level_alloc[l + 1] && a < v.level_alloc[l])) return;
     const float x = prb_sum_children_dyn(v.level[l + 1] + a * K, K);
     v.level[l][a] = x;
     if (l == T && l >= 1) {
@@ -154,6 +155,7 @@ __device__ __forceinline__ void prb_top_passes_k(const PrbView& v, const PrbTop&
         const float* child = top.mem + v.top_off[l + 1];
         float* own = top.mem + v.top_off[l];       // (not used for the root)
         for (uint32_t i = team.rank; i < n_l; i += team.size) {
+            if (!PRB_IN_BOUNDS(v, v.top_off[l + 1] + (i + 1) * K <= v.top_floats && i < v.level_alloc[l])) continue;
             const float x = prb_sum_staged<K>(child + (size_t)i * K);
             if (l == 0) {
                 v.level[0][0] = x;
@@ -428,9 +430,11 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
                 uint32_t s0 = rank;
                 while (s0 > 0 && sidx[s0 - 1] == slot.idx) --s0;
-                float p = __ldcg(leaves + slot.idx);
-                for (uint32_t s2 = s0; s2 <= rank; ++s2) add_change(p, vals[spos[s2]]);
-                leaves[slot.idx] = p;
+                if (PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth])) {
+                    float p = __ldcg(leaves + slot.idx);
+                    for (uint32_t s2 = s0; s2 <= rank; ++s2) add_change(p, vals[spos[s2]]);
+                    leaves[slot.idx] = p;
+                }
             }
         } else {
             for (uint32_t s1 = rank; s1 < n2; s1 += nt) {
@@ -450,7 +454,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     } else if (one_each) {
         if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
             const uint64_t ahead = slot.idx >= cursor ? slot.idx - cursor : slot.idx + N - cursor;   // distance from the cursor along the ring
-            if (!(ahead < n)) leaves[slot.idx] = vals[slot.pos];
+            if (!(ahead < n) && PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth] && slot.pos < n2)) leaves[slot.idx] = vals[slot.pos];
         }
     } else {
         for (uint32_t s = rank; s < n2; s += nt) {
@@ -459,7 +463,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             const uint32_t i = (uint32_t)(key >> 32);
             const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
             const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;
-            if (last && !(ahead < n)) leaves[i] = vals[(uint32_t)key];
+            if (last && !(ahead < n) && PRB_IN_BOUNDS(v, i < v.level_alloc[v.depth] && (uint32_t)key < n2)) leaves[i] = vals[(uint32_t)key];
         }
     }
     bool bad = false;
@@ -475,7 +479,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         float p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
         else imax = fmaxf(imax, p);
-        leaves[at] = p;
+        if (PRB_IN_BOUNDS(v, at < N)) leaves[at] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     if (n) prb_note_priorities(v.state, imax, true);      // (every CTA of a cluster wrote leaves of its own; a first default insertion writes 1)
@@ -537,7 +541,7 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
         float p = prio == nullptr ? dflt : ((pre.has_prio && t == team.rank) ? pre.prio : prio[t]);
         if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
         else imax = fmaxf(imax, p);
-        leaves[slot] = p;
+        if (PRB_IN_BOUNDS(v, slot < N)) leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     prb_note_priorities(v.state, imax, true);                       // (a first default insertion writes 1)

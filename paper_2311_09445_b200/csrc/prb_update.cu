@@ -204,7 +204,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         const PrbWideEntry e = prb_wide_classify(v, idx[b], val[b], raw, alpha, eps, fill, cursor, stale);
         if (b == gtid) first = e;
         flags |= e.flags;
-        if (e.valid) { wmax = fmaxf(wmax, e.p); atomicMax(leaf_bits + e.i, 0x80000000u | b); }
+        if (e.valid && PRB_IN_BOUNDS(v, e.i < v.level_alloc[D])) { wmax = fmaxf(wmax, e.p); atomicMax(leaf_bits + e.i, 0x80000000u | b); }
     }
     flags = __reduce_or_sync(0xFFFFFFFFu, flags);
     const unsigned mbits = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(wmax));
@@ -224,7 +224,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
     if (alive) {
         for (uint32_t b = gtid; b < B; b += gthreads) {
             const PrbWideEntry e = (b == gtid) ? first : prb_wide_classify(v, idx[b], val[b], raw, alpha, eps, fill, cursor, stale);
-            if (e.valid && __ldcg(leaf_bits + e.i) == (0x80000000u | b)) v.level[D][e.i] = e.p;
+            if (e.valid && PRB_IN_BOUNDS(v, e.i < v.level_alloc[D]) && __ldcg(leaf_bits + e.i) == (0x80000000u | b)) v.level[D][e.i] = e.p;
         }
         alive = prb_grid_barrier(v.state, passed, nctas, &s_ok);
     }
@@ -237,6 +237,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         const uint64_t n_lt = ((v.capacity - 1) >> sh) + 1;       // nodes of level lt
         if (n_lt <= 2ull * B) {
             for (uint64_t a = gtid; a < n_lt; a += gthreads) {
+                if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
                 if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
                 else prb_resum_levels(v, h, lt, a);
             }
@@ -249,6 +250,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
                     const int32_t before = idx[b - 1];
                     if (before >= 0 && (unsigned long long)before < fill && ((uint64_t)before >> sh) == a) continue;
                 }
+                if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
                 if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
                 else prb_resum_levels(v, h, lt, a);
             }
@@ -285,7 +287,7 @@ __global__ void prb_get_priorities_kernel(const __grid_constant__ PrbView v, uin
     if (b >= B) return;
     const int32_t i = idx[b];
     if (i < 0 || (unsigned long long)i >= v.state->fill) { out[b] = 0.0f; atomicOr(&v.state->status, PEARL_ST_BAD_INDEX); return; }
-    out[b] = __ldcg(v.level[v.depth] + i);
+    out[b] = PRB_IN_BOUNDS(v, (uint32_t)i < v.level_alloc[v.depth]) ? __ldcg(v.level[v.depth] + i) : 0.0f;
 }
 
 }  // namespace
