@@ -40,6 +40,7 @@ def lib():
         L = C.CDLL(build())
         vp, u32, u64, f32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_float
         L.oracle_prb_create.argtypes = [C.POINTER(vp), u64, u32, u32, u32]
+        L.oracle_prb_create_frames.argtypes = [C.POINTER(vp), u64, u32, u32, u32, u32]
         L.oracle_prb_destroy.argtypes = [vp]
         L.oracle_prb_destroy.restype = None
         L.oracle_prb_rebuild.argtypes = [vp]
@@ -114,13 +115,20 @@ def priority_pow(delta: float, eps: float, alpha: float):
 class OraclePRB:
     """The oracle buffer.  Methods mirror the product's C-ABI calls, with host arrays."""
 
-    def __init__(self, capacity: int, fanout: int, obs_bytes: int, act_bytes: int):
+    def __init__(self, capacity: int, fanout: int, obs_bytes: int, act_bytes: int, frame_stack: int = 0):
+        """frame_stack > 0: the frame-deduplicated layout; obs_bytes is then the size of a whole stack
+        (frame_stack frames) and insert takes one frame per transition in `obs`."""
         self._h = C.c_void_p()
-        rc = lib().oracle_prb_create(C.byref(self._h), capacity, fanout, obs_bytes, act_bytes)
+        if frame_stack:
+            assert obs_bytes % frame_stack == 0
+            rc = lib().oracle_prb_create_frames(C.byref(self._h), capacity, fanout, obs_bytes // frame_stack, frame_stack, act_bytes)
+        else:
+            rc = lib().oracle_prb_create(C.byref(self._h), capacity, fanout, obs_bytes, act_bytes)
         if rc != 0:
             raise ValueError("oracle_prb_create failed: %d" % rc)
         self.capacity, self.fanout = capacity, fanout
         self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
+        self.frame_stack = frame_stack
         _, _, _, self.depth = self.info()
 
     def close(self):

@@ -56,6 +56,8 @@
 #define ST_INTERNAL 16u
 #define ST_STALE 32u
 
+#define DONE_EPISODE_START 2u   /* frame-deduplicated layout: bit 1 of a slot's done byte */
+
 #define MAX_LEVELS 64
 
 typedef struct oracle_prb {
@@ -73,6 +75,9 @@ typedef struct oracle_prb {
     uint32_t obs_bytes, act_bytes;
     uint8_t *obs, *act, *next_obs, *done;
     float *rew;
+    /* Frame-deduplicated layout (stack > 0): the obs store holds ONE frame of frame_bytes per slot, the
+     * next_obs store is unused, and obs_bytes = stack * frame_bytes is the size of a rebuilt stack. */
+    uint32_t stack, frame_bytes;
     uint64_t size, cursor, sample_calls;
     uint32_t status;
     float max_priority;     /* largest priority written so far; 0 = none yet */
@@ -198,8 +203,8 @@ int oracle_priority_pow(float delta, float eps, float alpha, float *p)
 /* ------------------------------------------------------------------------ */
 static uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
 
-int oracle_prb_create(oracle_prb_t **out, uint64_t capacity, uint32_t fanout,
-                      uint32_t obs_bytes, uint32_t act_bytes)
+static int create_impl(oracle_prb_t **out, uint64_t capacity, uint32_t fanout,
+                       uint32_t obs_bytes, uint32_t act_bytes, uint32_t stack)
 {
     if (!out) return ORACLE_ERR_NULL;
     if (!(fanout == 2 || fanout == 4 || fanout == 8 || fanout == 16 || fanout == 32))
@@ -222,14 +227,49 @@ int oracle_prb_create(oracle_prb_t **out, uint64_t capacity, uint32_t fanout,
         if (!o->level[l] || !o->dirty[l] || !o->dirty_list[l]) return ORACLE_ERR_OOM;
     }
     o->obs_bytes = obs_bytes; o->act_bytes = act_bytes;
-    o->obs = (uint8_t *)malloc((size_t)capacity * obs_bytes + 1);
-    o->next_obs = (uint8_t *)malloc((size_t)capacity * obs_bytes + 1);
+    o->stack = stack; o->frame_bytes = stack ? obs_bytes / stack : 0;
+    /* (one frame per slot and no next_obs store when frames are deduplicated) */
+    o->obs = (uint8_t *)malloc((size_t)capacity * (stack ? o->frame_bytes : obs_bytes) + 1);
+    o->next_obs = (uint8_t *)malloc(stack ? 1 : (size_t)capacity * obs_bytes + 1);
     o->act = (uint8_t *)malloc((size_t)capacity * act_bytes + 1);
     o->rew = (float *)malloc((size_t)capacity * sizeof(float));
     o->done = (uint8_t *)malloc((size_t)capacity);
     if (!o->obs || !o->next_obs || !o->act || !o->rew || !o->done) return ORACLE_ERR_OOM;
     *out = o;
     return ORACLE_OK;
+}
+
+int oracle_prb_create(oracle_prb_t **out, uint64_t capacity, uint32_t fanout,
+                      uint32_t obs_bytes, uint32_t act_bytes)
+{
+    return create_impl(out, capacity, fanout, obs_bytes, act_bytes, 0);
+}
+
+/* Frame-deduplicated Data Storage (the paper's Pong workload, Table III, has 84 x 84 observations; a
+ * DQN state is a stack of the last `stack` frames, so consecutive transitions of one episode share all
+ * but one frame of obs and next_obs; Section VI-C: the Data Storage traffic is what dominates).
+ * Reading used here -- the paper does not describe such a layout:
+ *   - every slot stores ONE frame: the newest frame of its transition's next observation;
+ *   - an episode begins with a marker slot (bit 1 of its done byte set) that stores the episode's
+ *     first frame and is never sampled: its leaf is 0 whatever priority is given;
+ *   - consecutive slots of the ring are consecutive steps; for a sampled slot i, frame(b) is the frame
+ *     of slot i - min(b, c), c being the distance back to the nearest marker (or to the oldest stored
+ *     slot while the ring has not wrapped): frames "before the episode" repeat its first frame;
+ *     next_obs = [frame(S-1) .. frame(0)], obs = [frame(S) .. frame(1)], oldest frame first;
+ *   - an insertion also clears the leaves of the `stack` slots that follow the new cursor: once the
+ *     ring has wrapped they are the oldest transitions, whose history has just been overwritten;
+ *     an update that names one of them is skipped with STALE. */
+int oracle_prb_create_frames(oracle_prb_t **out, uint64_t capacity, uint32_t fanout,
+                             uint32_t frame_bytes, uint32_t stack, uint32_t act_bytes)
+{
+    if (stack < 1 || stack > 16 || frame_bytes < 1 || capacity <= stack) return ORACLE_ERR_BAD_ARG;
+    return create_impl(out, capacity, fanout, frame_bytes * stack, act_bytes, stack);
+}
+
+/* frame-deduplicated layout: is slot i one of the `stack` slots that follow the cursor? */
+static int history_less(const oracle_prb_t *o, uint64_t i)
+{
+    return o->stack && (i + o->capacity - o->cursor) % o->capacity < o->stack;
 }
 
 void oracle_prb_destroy(oracle_prb_t *o)
@@ -306,20 +346,32 @@ int oracle_prb_insert(oracle_prb_t *o, uint32_t n, const void *obs, const void *
     if (!o) return ORACLE_ERR_NULL;
     if (n == 0) return ORACLE_ERR_BAD_BATCH;
     if (n > o->capacity) return ORACLE_ERR_TOO_MANY;
+    if (o->stack && (next_obs || !done)) return ORACLE_ERR_BAD_ARG;   /* one frame per transition, in `obs`; markers live in `done` */
     uint32_t D = o->depth;
     const float dflt = default_priority(o);
+    const uint32_t row = o->stack ? o->frame_bytes : o->obs_bytes;
     for (uint32_t t = 0; t < n; ++t) {
         uint64_t slot = (o->cursor + t) % o->capacity;
-        if (obs) memcpy(o->obs + slot * o->obs_bytes, (const uint8_t *)obs + (size_t)t * o->obs_bytes, o->obs_bytes);
+        if (obs) memcpy(o->obs + slot * row, (const uint8_t *)obs + (size_t)t * row, row);
         if (next_obs) memcpy(o->next_obs + slot * o->obs_bytes, (const uint8_t *)next_obs + (size_t)t * o->obs_bytes, o->obs_bytes);
         if (act) memcpy(o->act + slot * o->act_bytes, (const uint8_t *)act + (size_t)t * o->act_bytes, o->act_bytes);
         if (rew) o->rew[slot] = rew[t];
         if (done) o->done[slot] = done[t];
         float p = prio ? prio[t] : dflt;
-        if (!valid_priority(p)) { p = 0.0f; o->status |= ST_BAD_PRIORITY; }
+        if (o->stack && (done[t] & DONE_EPISODE_START)) p = 0.0f;        /* a marker is never sampled */
+        else if (!valid_priority(p)) { p = 0.0f; o->status |= ST_BAD_PRIORITY; }
         else note_priority(o, p);
         o->level[D][slot] = p;
         mark_dirty(o, D, slot);
+    }
+    if (o->stack) {
+        /* the slots that follow the new cursor lose their history to this insertion */
+        uint64_t z = o->capacity - n < o->stack ? o->capacity - n : o->stack;
+        for (uint64_t s2 = 0; s2 < z; ++s2) {
+            uint64_t slot = (o->cursor + n + s2) % o->capacity;
+            o->level[D][slot] = 0.0f;
+            mark_dirty(o, D, slot);
+        }
     }
     resum_dirty(o);
     o->cursor = (o->cursor + n) % o->capacity;
@@ -341,6 +393,7 @@ int oracle_prb_update_priorities(oracle_prb_t *o, uint32_t B, const int32_t *idx
     uint32_t D = o->depth;
     for (uint32_t b = 0; b < B; ++b) {
         if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
+        if (history_less(o, (uint64_t)idx[b])) { o->status |= ST_STALE; continue; }
         if (!valid_priority(prio[b])) { o->status |= ST_BAD_PRIORITY; continue; }
         note_priority(o, prio[b]);
         o->level[D][idx[b]] = prio[b];
@@ -365,6 +418,7 @@ int oracle_prb_update_delta(oracle_prb_t *o, uint32_t B, const int32_t *idx, con
     uint32_t D = o->depth;
     for (uint32_t b = 0; b < B; ++b) {
         if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
+        if (history_less(o, (uint64_t)idx[b])) { o->status |= ST_STALE; continue; }
         if (!isfinite(delta[b])) { o->status |= ST_BAD_PRIORITY; continue; }
         volatile float sum = o->level[D][idx[b]] + delta[b];
         float p = sum;
@@ -386,6 +440,7 @@ int oracle_prb_update(oracle_prb_t *o, uint32_t B, const int32_t *idx, const flo
     uint32_t D = o->depth;
     for (uint32_t b = 0; b < B; ++b) {
         if (idx[b] < 0 || (uint64_t)idx[b] >= o->size) { o->status |= ST_BAD_INDEX; continue; }
+        if (history_less(o, (uint64_t)idx[b])) { o->status |= ST_STALE; continue; }
         float p;
         if (oracle_priority_pow(td[b], eps, alpha, &p)) { o->status |= ST_BAD_PRIORITY; continue; }
         note_priority(o, p);
@@ -414,7 +469,7 @@ int oracle_prb_update_after_insert(oracle_prb_t *o, uint32_t B, const int32_t *i
         /* how many slots back from the most recently written one this index lies */
         uint64_t i = (uint64_t)idx[b];
         uint64_t back = (o->cursor + o->capacity - 1 - i) % o->capacity;
-        if (back < inserted) { o->status |= ST_STALE; continue; }
+        if (back < inserted || history_less(o, i)) { o->status |= ST_STALE; continue; }
         float p;
         if (oracle_priority_pow(td[b], eps, alpha, &p)) { o->status |= ST_BAD_PRIORITY; continue; }
         note_priority(o, p);
@@ -495,6 +550,32 @@ void oracle_prb_targets(oracle_prb_t *o, uint32_t B, uint64_t seed, uint64_t cal
     }
 }
 
+/* The observations of slot i into obs / next_obs (either may be NULL): the stored rows, or, with the
+ * frame-deduplicated layout, the two stacks rebuilt from consecutive slots (see oracle_prb_create_frames). */
+static void copy_observations(const oracle_prb_t *o, uint64_t i, uint8_t *obs, uint8_t *next_obs)
+{
+    if (!o->stack) {
+        if (obs) memcpy(obs, o->obs + i * o->obs_bytes, o->obs_bytes);
+        if (next_obs) memcpy(next_obs, o->next_obs + i * o->obs_bytes, o->obs_bytes);
+        return;
+    }
+    const uint32_t S = o->stack, F = o->frame_bytes;
+    /* c: how far back frames may be taken -- to the nearest marker, or to slot 0 while the ring has not wrapped */
+    uint32_t c = S;
+    for (uint32_t d = 1; d <= S; ++d) {
+        if (o->size < o->capacity && i < d) { c = d - 1; break; }        /* nothing is stored before slot 0 */
+        uint64_t j = (i + o->capacity - d) % o->capacity;
+        if (o->done[j] & DONE_EPISODE_START) { c = d; break; }
+    }
+    for (uint32_t pos = 0; pos < S; ++pos) {          /* pos 0 = oldest frame of a stack */
+        uint32_t b_next = S - 1 - pos, b_obs = S - pos;                  /* distances back from slot i */
+        uint64_t j_next = (i + o->capacity - (b_next < c ? b_next : c)) % o->capacity;
+        uint64_t j_obs = (i + o->capacity - (b_obs < c ? b_obs : c)) % o->capacity;
+        if (next_obs) memcpy(next_obs + (size_t)pos * F, o->obs + j_next * F, F);
+        if (obs) memcpy(obs + (size_t)pos * F, o->obs + j_obs * F, F);
+    }
+}
+
 /* ------------------------------------------------------------------------ */
 /* Sample B transitions: indices (Eq. 1 per stratum), importance-sampling    */
 /* weights and the gathered batch (Listing 2: sampled_data =                 */
@@ -541,8 +622,8 @@ static int sample_impl(oracle_prb_t *o, uint32_t B, float beta, uint64_t seed,
     if (w) for (uint32_t k = 0; k < B; ++k) w[k] = (float)(wraw[k] / wmax);
     for (uint32_t k = 0; k < B; ++k) {
         uint64_t i = (uint64_t)idx[k];
-        if (obs) memcpy((uint8_t *)obs + (size_t)k * o->obs_bytes, o->obs + i * o->obs_bytes, o->obs_bytes);
-        if (next_obs) memcpy((uint8_t *)next_obs + (size_t)k * o->obs_bytes, o->next_obs + i * o->obs_bytes, o->obs_bytes);
+        copy_observations(o, i, obs ? (uint8_t *)obs + (size_t)k * o->obs_bytes : NULL,
+                          next_obs ? (uint8_t *)next_obs + (size_t)k * o->obs_bytes : NULL);
         if (act) memcpy((uint8_t *)act + (size_t)k * o->act_bytes, o->act + i * o->act_bytes, o->act_bytes);
         if (rew) rew[k] = o->rew[i];
         if (done) done[k] = o->done[i];
@@ -582,6 +663,7 @@ int oracle_prb_sample_uniform(oracle_prb_t *o, uint32_t B, uint64_t seed, int32_
 {
     if (!o || !idx) return ORACLE_ERR_NULL;
     if (B == 0) return ORACLE_ERR_BAD_BATCH;
+    if (o->stack) return ORACLE_ERR_BAD_ARG;      /* a uniform draw could name a marker or a slot without history */
     if (o->size == 0) { o->status |= ST_EMPTY; return ORACLE_OK; }
     for (uint32_t k = 0; k < B; ++k) {
         uint32_t ctr[4] = { k, 0u, (uint32_t)o->sample_calls, (uint32_t)(o->sample_calls >> 32) };
@@ -639,8 +721,8 @@ int oracle_prb_read_rows(oracle_prb_t *o, const int32_t *idx, uint32_t n, void *
     for (uint32_t k = 0; k < n; ++k) {
         if (idx[k] < 0 || (uint64_t)idx[k] >= o->capacity) return ORACLE_ERR_BAD_ARG;
         uint64_t i = (uint64_t)idx[k];
-        if (obs) memcpy((uint8_t *)obs + (size_t)k * o->obs_bytes, o->obs + i * o->obs_bytes, o->obs_bytes);
-        if (next_obs) memcpy((uint8_t *)next_obs + (size_t)k * o->obs_bytes, o->next_obs + i * o->obs_bytes, o->obs_bytes);
+        copy_observations(o, i, obs ? (uint8_t *)obs + (size_t)k * o->obs_bytes : NULL,
+                          next_obs ? (uint8_t *)next_obs + (size_t)k * o->obs_bytes : NULL);
         if (act) memcpy((uint8_t *)act + (size_t)k * o->act_bytes, o->act + i * o->act_bytes, o->act_bytes);
         if (rew) rew[k] = o->rew[i];
         if (done) done[k] = o->done[i];

@@ -137,6 +137,54 @@ def transitions(wl: Workload, rng: np.random.Generator, n: int, first_id: int = 
     return out
 
 
+class FrameTrajectory:
+    """A single actor's stream of transitions whose observations are stacks of the last `stack` frames
+    (an Atari-style environment behind a frame-stacking wrapper: at reset the stack is filled with the
+    first frame, every step pushes one new frame), handed out both ways at once:
+
+      * one frame per ring slot -- the newest frame of the transition's next observation -- with an extra
+        slot at every episode start that carries the episode's first frame and has bit 1 of `done` set
+        (the frame-deduplicated layout of the replay buffer);
+      * the same slots with whole stacks `obs` / `next_obs` (the plain layout); the rows of the extra
+        slots are zero and their priority is 0.
+
+    This is the environment side: it knows nothing of how the buffer stores or rebuilds anything."""
+
+    def __init__(self, rng: np.random.Generator, frame_bytes: int, stack: int, episode_steps=(3, 30), n_actions: int = 18):
+        self.rng, self.F, self.S = rng, frame_bytes, stack
+        self.episode_steps, self.n_actions = episode_steps, n_actions
+        self.window = None          # the current observation: `stack` frames, oldest first
+        self.left = 0               # steps left in the running episode
+
+    def _frame(self) -> np.ndarray:
+        return self.rng.integers(0, 256, size=self.F, dtype=np.uint8)
+
+    def next(self, n: int) -> Dict[str, np.ndarray]:
+        F, S = self.F, self.S
+        out = {"frame": np.zeros((n, F), np.uint8), "obs": np.zeros((n, S * F), np.uint8), "next_obs": np.zeros((n, S * F), np.uint8),
+               "act": self.rng.integers(0, self.n_actions, size=n).astype(np.int32), "rew": self.rng.integers(-1, 2, size=n).astype(np.float32),
+               "done": np.zeros(n, np.uint8), "prio": np.exp(self.rng.standard_normal(n)).astype(np.float32)}
+        for t in range(n):
+            if self.left == 0:                       # reset: the slot carries the first frame only
+                first = self._frame()
+                self.window = [first] * S
+                self.left = int(self.rng.integers(self.episode_steps[0], self.episode_steps[1] + 1))
+                out["frame"][t] = first
+                out["done"][t] = 2
+                out["prio"][t] = 0.0
+                out["act"][t], out["rew"][t] = 0, 0.0
+                continue
+            new = self._frame()
+            nxt = self.window[1:] + [new]
+            out["frame"][t] = new
+            out["obs"][t] = np.concatenate(self.window)
+            out["next_obs"][t] = np.concatenate(nxt)
+            self.window = nxt
+            self.left -= 1
+            out["done"][t] = 1 if self.left == 0 else 0
+        return out
+
+
 def update_batch(wl: Workload, rng: np.random.Generator, sampled_idx: np.ndarray):
     """The update that follows a sample: the sampled indices (with wl.dup_frac of the positions
     overwritten by a copy of another position's index) and fresh TD errors, one per position."""
