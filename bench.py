@@ -177,7 +177,12 @@ def device_batches(wl, rng, dev, n, count, first_id):
         if wl.counter_rows:
             small = wk.transitions(wl, rng, n, with_obs=False)
             ids = torch.arange(first_id + r * n, first_id + (r + 1) * n, dtype=torch.int64, device=dev)
-            d = {"obs": wk.counter_row_bytes(ids, 0, wl.obs_bytes), "next_obs": wk.counter_row_bytes(ids, 1, wl.obs_bytes)}
+            if wl.frame_stack:
+                # one frame per slot; an episode start (marker, bit 1 of done) every couple of hundred slots
+                d = {"obs": wk.counter_row_bytes(ids, 0, wl.obs_bytes // wl.frame_stack), "next_obs": None}
+                small["done"] = np.where(rng.random(n) < 0.005, 2, small["done"] & 1).astype(np.uint8)
+            else:
+                d = {"obs": wk.counter_row_bytes(ids, 0, wl.obs_bytes), "next_obs": wk.counter_row_bytes(ids, 1, wl.obs_bytes)}
             for k in ("act", "rew", "done", "prio"):
                 d[k] = torch.from_numpy(small[k]).to(dev)
         else:
@@ -289,7 +294,8 @@ def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=Tru
     max_batch = max(B, n_ins, chunk)
     m = {}
     with torch.cuda.stream(stream):
-        prb = PrioritizedReplay(wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, max_batch, device=dev, stream=stream)
+        prb = PrioritizedReplay(wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, max_batch, device=dev, stream=stream,
+                                frame_stack=wl.frame_stack)
         # prefill the whole ring through the insert call
         filled = 0
         while filled < wl.capacity:
@@ -433,7 +439,7 @@ def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=Tru
         # ---- end to end through the host-buffer calls ----------------------------------------
         if e2e:
             e2e_steps = max(5, min(steps, 100 if wl.counter_rows else 500))
-            hb = [{k: v.cpu().pin_memory() for k, v in batches[r].items()} for r in range(ROTATE)]
+            hb = [{k: (v.cpu().pin_memory() if v is not None else None) for k, v in batches[r].items()} for r in range(ROTATE)]
             ho = out_buffers(wl, dev, B, pinned=True)
             htd = [t.cpu().pin_memory() for t in tds]
 
@@ -509,12 +515,12 @@ def run_ours(args, wl, rank, world):
     depth = m["depth"]
     ms = statistics.median(m["region_ms"])
     h2d = (n_ins * (E + 4) if n_ins else 0) + B * 8
-    d2h = B * (E + 8)
+    d2h = B * (2 * wl.obs_bytes + wl.act_bytes + 5 + 8)
     peak, peak_kind = load_peak()
     # algorithmic bytes of one sample call: D child groups of K binary32 per stratum, index and
     # weight written, every field of the row read once and written once
-    sample_bytes = B * (depth * wl.fanout * 4 + 8 + 2 * E)
-    long_rows = wl.obs_bytes >= 8192 and wl.obs_bytes % 16 == 0
+    sample_bytes = B * (depth * wl.fanout * 4 + 8 + wl.sample_bytes)
+    long_rows = wl.obs_bytes >= 8192 and wl.obs_bytes % 16 == 0 and not wl.frame_stack
     achieved = sample_bytes / (m["ms_sample"] * 1e-3) / 1e9
     rates = summary_of(wl, m, world)
     for k in ("ms_update_shuffled", "ms_sample_one_kernel", "ms_sample_streamed4", "ms_sample_buffer_norm"):
@@ -549,7 +555,7 @@ def run_ours(args, wl, rank, world):
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     else:
         line["e2e"] = {"value": None, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-    step_bytes = B * (depth * wl.fanout * 4 + 8 + 2 * E) + (n_ins * (2 * E + 4) if n_ins else 0)
+    step_bytes = sample_bytes + (n_ins * (2 * E + 4) if n_ins else 0)
     line["roofline_step"] = {"bound": "hbm", "bytes_per_step": step_bytes, "achieved": step_bytes / (ms / args.steps * 1e-3) / 1e9,
                              "peak": peak, "unit": "GB/s", "frac": step_bytes / (ms / args.steps * 1e-3) / 1e9 / peak}
     if n_ins:
@@ -585,10 +591,12 @@ def other_workloads(headline, dev, stream):
             out[wl.name] = {"skipped": "not enough free device memory"}
             continue
         steps = 200
-        m = measure_workload(wl, steps, 3, dev, stream, extras=False, e2e=wl.capacity <= (1 << 20))
+        m = measure_workload(wl, steps, 3, dev, stream, extras=False, e2e=wl.capacity <= (1 << 20) or wl.frame_stack > 0)
         m["steps"] = steps
         d = summary_of(wl, m)
         d.update(capacity=wl.capacity, fanout=wl.fanout, batch=wl.batch, insert_per_step=wl.n_insert, steps=steps,
+                 stored_bytes_per_transition=wl.transition_bytes, gather_bytes_per_sample=wl.sample_bytes,
+                 gather_gbs=wl.batch * wl.sample_bytes / (m["ms_sample"] * 1e-3) / 1e9,
                  region_repeats=len(m["region_ms"]), status_bits=int(m["status"]))
         out[wl.name] = d
         torch.cuda.empty_cache()

@@ -98,6 +98,33 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout,
                      const pearl_layout_t* layout, uint32_t max_batch, int device,
                      void* cuda_stream, void* slab, uint64_t slab_bytes);
 
+/* A buffer whose Data Storage keeps ONE frame per transition instead of two stacked observations (the
+ * paper's Pong workload, Table III, has 84 x 84 observations and a DQN state stacks the last few; Section
+ * VI-C: Data Storage traffic is what dominates).  The paper describes no such layout; the one used here:
+ *   - an observation is `stack` frames (1..16) of frame_bytes each, oldest first; a sample hands out obs and
+ *     next_obs rows of stack * frame_bytes bytes, as a buffer created with pearl_prb_create would;
+ *   - consecutive ring slots hold consecutive steps of ONE trajectory.  Each slot stores the newest frame
+ *     of its transition's next observation: the insertion calls take that frame per transition in
+ *     d_obs (rows of frame_bytes), d_next_obs must be NULL and d_done must be given;
+ *   - an episode begins with a marker slot: bit 1 (value 2) of its done byte is set, its frame is the
+ *     episode's first frame, its other fields are not used, and its leaf is 0 whatever priority is given,
+ *     so it is never sampled.  Bit 0 of done keeps its meaning;
+ *   - for a sampled slot i the frame b steps back is that of slot i - min(b, c), c being the distance back
+ *     to the nearest marker (or to slot 0 while the ring has not wrapped): what lies before the episode
+ *     repeats its first frame.  next_obs = frames stack-1 .. 0 steps back, obs = frames stack .. 1 steps back;
+ *   - an insertion also clears the leaves of the `stack` slots that follow the new cursor -- once the ring
+ *     has wrapped they are the oldest transitions, whose history the insertion overwrites -- and an update
+ *     that names one of them is skipped and raises PEARL_ST_STALE;
+ *   - pearl_prb_sample_uniform is refused (PEARL_ERR_BAD_ARG): a uniform draw could name a marker.
+ * Everything else -- tree, sampling, weights, updates, status bits -- is as for pearl_prb_create.  For
+ * stack = 4 the store is an eighth of the plain layout's and an insertion writes an eighth of the bytes.
+ * capacity must exceed stack. */
+uint64_t pearl_prb_slab_bytes_frames(uint64_t capacity, uint32_t fanout, uint32_t frame_bytes, uint32_t stack,
+                                     uint32_t act_bytes, uint32_t max_batch);
+int pearl_prb_create_frames(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, uint32_t frame_bytes,
+                            uint32_t stack, uint32_t act_bytes, uint32_t max_batch, int device, void* cuda_stream,
+                            void* slab, uint64_t slab_bytes);
+
 /* Synchronises the handle's streams, frees library-owned memory, streams, events and the handle. */
 int pearl_prb_destroy(pearl_prb_t* prb);
 

@@ -35,6 +35,8 @@ _vp, _u32, _u64, _f32, _i = C.c_void_p, C.c_uint32, C.c_uint64, C.c_float, C.c_i
 SIGNATURES = {
     "pearl_prb_slab_bytes": (_u64, [_u64, _u32, C.POINTER(_Layout), _u32]),
     "pearl_prb_create": (_i, [C.POINTER(_vp), _u64, _u32, C.POINTER(_Layout), _u32, _i, _vp, _vp, _u64]),
+    "pearl_prb_slab_bytes_frames": (_u64, [_u64, _u32, _u32, _u32, _u32, _u32]),
+    "pearl_prb_create_frames": (_i, [C.POINTER(_vp), _u64, _u32, _u32, _u32, _u32, _u32, _i, _vp, _vp, _u64]),
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -118,7 +120,7 @@ class PrioritizedReplay:
     """
 
     def __init__(self, capacity: int, fanout: int, obs_bytes: int, act_bytes: int, max_batch: int,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None, frame_stack: int = 0):
         self._h = None
         lib = load_library()
         if not torch.cuda.is_available():
@@ -127,16 +129,27 @@ class PrioritizedReplay:
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         self.capacity, self.fanout, self.max_batch = capacity, fanout, max_batch
         self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
+        self.frame_stack = frame_stack          # > 0: pearl_prb_create_frames; obs_bytes is then a whole stack
         lay = _Layout(obs_bytes, act_bytes)
-        need = lib.pearl_prb_slab_bytes(capacity, fanout, C.byref(lay), max_batch)
+        if frame_stack:
+            if obs_bytes % frame_stack:
+                raise ValueError("obs_bytes must be frame_stack frames")
+            need = lib.pearl_prb_slab_bytes_frames(capacity, fanout, obs_bytes // frame_stack, frame_stack, act_bytes, max_batch)
+        else:
+            need = lib.pearl_prb_slab_bytes(capacity, fanout, C.byref(lay), max_batch)
         if need == 0:
             raise PearlError(-7, "pearl_prb_slab_bytes")
         self.slab_bytes = int(need)
         self._slab = torch.empty(self.slab_bytes, dtype=torch.uint8, device=self.device)
         h = C.c_void_p()
-        rc = lib.pearl_prb_create(C.byref(h), capacity, fanout, C.byref(lay), max_batch, self.device.index or 0,
-                                  C.c_void_p(self.stream.cuda_stream), C.c_void_p(self._slab.data_ptr()),
-                                  self.slab_bytes)
+        if frame_stack:
+            rc = lib.pearl_prb_create_frames(C.byref(h), capacity, fanout, obs_bytes // frame_stack, frame_stack, act_bytes, max_batch,
+                                             self.device.index or 0, C.c_void_p(self.stream.cuda_stream),
+                                             C.c_void_p(self._slab.data_ptr()), self.slab_bytes)
+        else:
+            rc = lib.pearl_prb_create(C.byref(h), capacity, fanout, C.byref(lay), max_batch, self.device.index or 0,
+                                      C.c_void_p(self.stream.cuda_stream), C.c_void_p(self._slab.data_ptr()),
+                                      self.slab_bytes)
         if rc != 0:
             raise PearlError(rc, "pearl_prb_create")
         self._h = h

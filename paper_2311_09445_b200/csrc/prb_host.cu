@@ -36,17 +36,22 @@ struct Layout {
     uint64_t off_stage_prio, off_stage_idx, off_stage_td;
     uint64_t off_stage_out[PRB_NUM_FIELDS];   // ... and outputs
     uint64_t off_stage_out_idx, off_stage_out_w;
-    uint32_t field_bytes[PRB_NUM_FIELDS];
+    uint32_t field_bytes[PRB_NUM_FIELDS];     // a row of the store
+    uint32_t out_bytes[PRB_NUM_FIELDS];       // a row as a sample hands it out
+    uint32_t stack;                           // frame-deduplicated layout: frames per observation (0: plain layout)
     uint64_t total;
 };
 
 bool valid_fanout(uint32_t k) { return k == 2 || k == 4 || k == 8 || k == 16 || k == 32; }
 
-bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, uint32_t max_batch, Layout* L)
+bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, uint32_t max_batch, Layout* L, uint32_t stack = 0)
 {
     if (!lay || !valid_fanout(fanout) || capacity < 1 || capacity > (1ull << 30) || max_batch < 1 ||
         max_batch > (1u << 20))
         return false;
+    if (stack > 16 || (stack && (lay->obs_bytes == 0 || capacity <= stack || (uint64_t)lay->obs_bytes * stack > 0xFFFFFFFFull)))
+        return false;
+    L->stack = stack;
     uint32_t D = 1;
     uint64_t span = fanout;
     while (span < capacity) { span *= fanout; ++D; }
@@ -58,11 +63,14 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     for (uint32_t l = 0; l <= D; ++l)
         L->level_alloc[l] = (l == 0) ? 1 : (nodes[l] + fanout - 1) / fanout * fanout;
 
+    // (with frames, lay->obs_bytes is the size of one frame)
     L->field_bytes[F_OBS] = lay->obs_bytes;
-    L->field_bytes[F_NEXT_OBS] = lay->obs_bytes;
+    L->field_bytes[F_NEXT_OBS] = stack ? 0 : lay->obs_bytes;
     L->field_bytes[F_ACT] = lay->act_bytes;
     L->field_bytes[F_REW] = 4;
     L->field_bytes[F_DONE] = 1;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) L->out_bytes[f] = L->field_bytes[f];
+    if (stack) L->out_bytes[F_OBS] = L->out_bytes[F_NEXT_OBS] = lay->obs_bytes * stack;
     // A field that is copied granule by granule (anything but rows of at least 512 16-byte granules,
     // which move as bulk copies) is indexed with 32-bit granule numbers within one batch.
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
@@ -82,7 +90,7 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     L->off_stage_prio = at; at = align_up(at + (uint64_t)max_batch * 4);
     L->off_stage_idx = at; at = align_up(at + (uint64_t)max_batch * 4);
     L->off_stage_td = at; at = align_up(at + (uint64_t)max_batch * 4);
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_out[f] = at; at = align_up(at + (uint64_t)max_batch * L->field_bytes[f]); }
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_out[f] = at; at = align_up(at + (uint64_t)max_batch * L->out_bytes[f]); }
     L->off_stage_out_idx = at; at = align_up(at + (uint64_t)max_batch * 4);
     L->off_stage_out_w = at; at = align_up(at + (uint64_t)max_batch * 4);
     L->total = at;
@@ -152,10 +160,13 @@ namespace {
 
 inline bool misaligned(const void* p, uint32_t granule) { return ((uintptr_t)p & (granule - 1)) != 0; }
 
-int check_batch_ptrs(const pearl_prb* h, const void* const ptrs[PRB_NUM_FIELDS])
+// (outputs: the pointers are a sample's outputs, whose rows are out_bytes long; else an insertion's inputs)
+int check_batch_ptrs(const pearl_prb* h, const void* const ptrs[PRB_NUM_FIELDS], bool outputs = false)
 {
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
-        if (ptrs[f] && h->view.field_bytes[f] && misaligned(ptrs[f], h->view.field_vec[f])) return PEARL_ERR_ALIGN;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        const uint32_t row = outputs ? h->view.out_bytes[f] : h->view.field_bytes[f];
+        if (ptrs[f] && row && misaligned(ptrs[f], h->view.field_vec[f])) return PEARL_ERR_ALIGN;
+    }
     return PEARL_OK;
 }
 
@@ -232,14 +243,40 @@ uint64_t pearl_prb_slab_bytes(uint64_t capacity, uint32_t fanout, const pearl_la
     return L.total;
 }
 
+uint64_t pearl_prb_slab_bytes_frames(uint64_t capacity, uint32_t fanout, uint32_t frame_bytes, uint32_t stack, uint32_t act_bytes,
+                                     uint32_t max_batch)
+{
+    Layout L;
+    const pearl_layout_t lay = { frame_bytes, act_bytes };
+    if (stack < 1 || !make_layout(capacity, fanout, &lay, max_batch, &L, stack)) return 0;
+    return L.total;
+}
+
+static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t stack,
+                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes);
+
 int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
                      uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
+{
+    return create_common(out, capacity, fanout, layout, 0, max_batch, device, cuda_stream, slab, slab_bytes);
+}
+
+int pearl_prb_create_frames(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, uint32_t frame_bytes, uint32_t stack,
+                            uint32_t act_bytes, uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
+{
+    const pearl_layout_t lay = { frame_bytes, act_bytes };
+    if (stack < 1) return PEARL_ERR_BAD_ARG;
+    return create_common(out, capacity, fanout, &lay, stack, max_batch, device, cuda_stream, slab, slab_bytes);
+}
+
+static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t stack,
+                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
 {
     if (!out || !layout) return PEARL_ERR_NULL;
     if (!valid_fanout(fanout)) return PEARL_ERR_BAD_FANOUT;
     if (max_batch < 1 || max_batch > (1u << 20)) return PEARL_ERR_BAD_BATCH;
     Layout L;
-    if (!make_layout(capacity, fanout, layout, max_batch, &L)) return PEARL_ERR_BAD_ARG;
+    if (!make_layout(capacity, fanout, layout, max_batch, &L, stack)) return PEARL_ERR_BAD_ARG;
     DeviceGuard guard(device);
     if (!guard.ok) return PEARL_ERR_CUDA;
 
@@ -303,8 +340,11 @@ int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, cons
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         v.store[f] = at(h, L.off_store[f]);
         v.field_bytes[f] = L.field_bytes[f];
+        v.out_bytes[f] = L.out_bytes[f];
         v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
     }
+    v.stack = L.stack;
+    if (v.stack) v.field_vec[F_NEXT_OBS] = v.field_vec[F_OBS];      // rebuilt from the same frames
     v.wraw = (double*)at(h, L.off_wraw);
     for (uint32_t j = 0; j < kPrbHandoffs; ++j) v.handoff[j] = at(h, L.off_handoff[j]);
     v.capacity = capacity;
@@ -348,6 +388,7 @@ int pearl_prb_insert(pearl_prb_t* h, uint32_t n, const void* d_obs, const void* 
     if (!h) return PEARL_ERR_NULL;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    if (h->view.stack && (d_next_obs || !d_done)) return PEARL_ERR_BAD_ARG;     // one frame per transition (d_obs); markers live in d_done
     const void* ptrs[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
     int rc = check_batch_ptrs(h, ptrs);
     if (rc != PEARL_OK) return rc;
@@ -369,7 +410,7 @@ static int check_sample_args(const pearl_prb_t* h, uint32_t B, float beta, const
     if (!h || !d_idx) return PEARL_ERR_NULL;
     if (B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (!finite_nonneg(beta)) return PEARL_ERR_BAD_ARG;
-    int rc = check_batch_ptrs(h, ptrs);
+    int rc = check_batch_ptrs(h, ptrs, true);
     if (rc != PEARL_OK) return rc;
     if (misaligned(d_idx, 4) || (d_w && misaligned(d_w, 4))) return PEARL_ERR_ALIGN;
     return PEARL_OK;
@@ -435,6 +476,7 @@ int pearl_prb_wait_sub_batch(pearl_prb_t* h, uint32_t sub_batch, void* cuda_stre
 int pearl_prb_sample_uniform(pearl_prb_t* h, uint32_t B, uint64_t seed, int32_t* d_idx, float* d_w, void* d_obs,
                              void* d_act, float* d_rew, void* d_next_obs, uint8_t* d_done)
 {
+    if (h && h->view.stack) return PEARL_ERR_BAD_ARG;      // (a uniform draw could name a marker or a slot without history)
     return sample_common(h, B, 0.0f, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done, 1);
 }
 
@@ -498,6 +540,7 @@ static int check_update_insert_args(const pearl_prb_t* h, uint32_t B, const int3
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
     if (!finite_nonneg(alpha) || !finite_nonneg(eps)) return PEARL_ERR_BAD_ARG;
+    if (h->view.stack && (ptrs[F_NEXT_OBS] || !ptrs[F_DONE])) return PEARL_ERR_BAD_ARG;
     int rc = check_batch_ptrs(h, ptrs);
     if (rc != PEARL_OK) return rc;
     if ((d_prio && misaligned(d_prio, 4)) || misaligned(d_idx, 4) || misaligned(d_td, 4)) return PEARL_ERR_ALIGN;
@@ -592,6 +635,7 @@ int pearl_prb_insert_host(pearl_prb_t* h, uint32_t n, const void* h_obs, const v
     if (!h) return PEARL_ERR_NULL;
     if (n == 0 || n > h->max_batch) return PEARL_ERR_BAD_BATCH;
     if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    if (h->view.stack && (h_next_obs || !h_done)) return PEARL_ERR_BAD_ARG;
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
     const void* src[PRB_NUM_FIELDS + 1] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_prio };
@@ -633,7 +677,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
     void* dst[PRB_NUM_FIELDS + 2] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_idx, h_w };
     void* dev[PRB_NUM_FIELDS + 2];
     Packing pk;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, dst[f] ? (uint64_t)B * h->view.field_bytes[f] : 0);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, dst[f] ? (uint64_t)B * h->view.out_bytes[f] : 0);
     pk.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
     pk.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
     if (h->pin && pk.total <= kPackBytes) {
@@ -652,7 +696,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
         return PEARL_OK;
     }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f)
-        dev[f] = (dst[f] && h->view.field_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
+        dev[f] = (dst[f] && h->view.out_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
     int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_out_idx);
     float* d_w = h_w ? (float*)at(h, h->lay.off_stage_out_w) : nullptr;
     int rc = pearl_prb_sample(h, B, beta, seed, d_idx, d_w, dev[F_OBS], dev[F_ACT], (float*)dev[F_REW],
@@ -662,7 +706,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
     if (h_w && cudaMemcpyAsync(h_w, d_w, (uint64_t)B * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (!dev[f]) continue;
-        if (cudaMemcpyAsync(dst[f], dev[f], (uint64_t)B * h->view.field_bytes[f], cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+        if (cudaMemcpyAsync(dst[f], dev[f], (uint64_t)B * h->view.out_bytes[f], cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
             return PEARL_ERR_CUDA;
     }
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
@@ -811,14 +855,51 @@ int pearl_prb_read_rows(pearl_prb_t* h, const int32_t* h_idx, uint32_t n, void* 
     void* dst[PRB_NUM_FIELDS] = { h_obs, h_next_obs, h_act, h_rew, h_done };
     for (uint32_t k = 0; k < n; ++k)
         if (h_idx[k] < 0 || (uint64_t)h_idx[k] >= h->view.capacity) return PEARL_ERR_BAD_ARG;
+    const uint32_t S = h->view.stack;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         const uint64_t fb = h->view.field_bytes[f];
-        if (!dst[f] || fb == 0) continue;
+        if (!dst[f] || fb == 0 || (S && f == F_OBS)) continue;
         for (uint32_t k = 0; k < n; ++k) {
             if (cudaMemcpyAsync((unsigned char*)dst[f] + k * fb, h->view.store[f] + (uint64_t)h_idx[k] * fb, fb,
                                 cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
                 return PEARL_ERR_CUDA;
         }
+    }
+    if (S && (h_obs || h_next_obs)) {
+        // frames: both observations are rebuilt the way a sample rebuilds them -- frame b steps back comes
+        // from slot i - min(b, c), c the distance back to the nearest episode-start marker (or to slot 0
+        // while the ring has not wrapped)
+        PrbState st;
+        if (cudaMemcpyAsync(&st, h->view.state, sizeof(st), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+        unsigned char* marks = (unsigned char*)malloc((size_t)n * S + 1);
+        if (!marks) return PEARL_ERR_OOM;
+        const uint64_t N = h->view.capacity, F = h->view.field_bytes[F_OBS];
+        for (uint32_t k = 0; k < n; ++k)
+            for (uint32_t d = 1; d <= S; ++d) {
+                const uint64_t j = ((uint64_t)h_idx[k] + N - d) % N;
+                if (cudaMemcpyAsync(marks + (size_t)k * S + (d - 1), h->view.store[F_DONE] + j, 1, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) {
+                    free(marks);
+                    return PEARL_ERR_CUDA;
+                }
+            }
+        if (cudaStreamSynchronize(h->stream) != cudaSuccess) { free(marks); return PEARL_ERR_CUDA; }
+        for (uint32_t k = 0; k < n; ++k) {
+            const uint64_t i = (uint64_t)h_idx[k];
+            uint32_t c = S;
+            for (uint32_t d = 1; d <= S; ++d) {
+                if (st.fill < N && i < d) { c = d - 1; break; }
+                if (marks[(size_t)k * S + (d - 1)] & kPrbEpisodeStart) { c = d; break; }
+            }
+            for (uint32_t pos = 0; pos < S; ++pos) {
+                const uint32_t b_next = S - 1 - pos, b_obs = S - pos;
+                const uint64_t j_next = (i + N - (b_next < c ? b_next : c)) % N, j_obs = (i + N - (b_obs < c ? b_obs : c)) % N;
+                if (h_next_obs && cudaMemcpyAsync((unsigned char*)h_next_obs + ((uint64_t)k * S + pos) * F, h->view.store[F_OBS] + j_next * F, F,
+                                                  cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) { free(marks); return PEARL_ERR_CUDA; }
+                if (h_obs && cudaMemcpyAsync((unsigned char*)h_obs + ((uint64_t)k * S + pos) * F, h->view.store[F_OBS] + j_obs * F, F,
+                                             cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) { free(marks); return PEARL_ERR_CUDA; }
+            }
+        }
+        free(marks);
     }
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }

@@ -119,9 +119,9 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
             if (upd.B)      // update and insertion share one re-sum pass per level
-                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top);
+                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top, src.ptr[F_DONE]);
             else
-                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp, top);
+                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp, top, src.ptr[F_DONE]);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
@@ -203,7 +203,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         PrbTeam team;
         team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
         if (blockIdx.x == 0 && plan.tree_ctas == 0)
-            prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp);
+            prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp, PrbTop{}, src.ptr[F_DONE]);
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
         for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
             copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
@@ -272,7 +272,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
         plan.tree_ctas = prb_update_ctas(v, upd.B);
         if (cudaEventRecord(fork->fork, s) != cudaSuccess || cudaStreamWaitEvent(fork->side, fork->fork, 0) != cudaSuccess)
             return -1;
-        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, fork->side, 0, n, d_prio);
+        const int k = prb_launch_update(v, upd_B, upd_idx, upd_val, upd_raw, alpha, eps, fork->side, 0, n, d_prio, src.ptr[F_DONE]);
         if (k != 1 || cudaEventRecord(fork->join, fork->side) != cudaSuccess) return -1;
         upd.B = 0;
         launches = 2;

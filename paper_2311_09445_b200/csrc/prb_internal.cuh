@@ -20,6 +20,7 @@
 constexpr uint32_t kPrbHandoffs = 4;    // hand-off areas of a two-kernel sample (descents of later calls run ahead of earlier calls' row copies)
 
 enum PrbField { F_OBS = 0, F_NEXT_OBS = 1, F_ACT = 2, F_REW = 3, F_DONE = 4 };
+constexpr unsigned char kPrbEpisodeStart = 2;      // done byte, bit 1 (frame-deduplicated layout)
 
 // Mutable state of a buffer; lives in device memory so that enqueued work never depends on
 // host-side copies of it.
@@ -52,6 +53,13 @@ struct PrbView {
     unsigned char* store[PRB_NUM_FIELDS];
     uint32_t field_bytes[PRB_NUM_FIELDS];
     uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
+    // Frame-deduplicated layout (stack > 0): the obs store keeps ONE frame of field_bytes[F_OBS] bytes per slot
+    // (the newest frame of the transition's next observation), there is no next_obs store
+    // (field_bytes[F_NEXT_OBS] == 0), and a sample rebuilds both observations, `stack` frames each, from
+    // consecutive slots.  out_bytes[f] is the size of a row of field f as a sample hands it out (equal to
+    // field_bytes[f] except for the two rebuilt fields).  Bit 1 of a slot's done byte marks an episode start.
+    uint32_t stack;
+    uint32_t out_bytes[PRB_NUM_FIELDS];
     double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
     // A sample of long rows that is issued as two kernels (descents, then the row copy) hands indices
     // and leaf priorities from the first to the second through one of a few areas of the slab, used in turn:
@@ -138,7 +146,8 @@ bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst);
 // the update in the same kernel, which advances the tree's cursor and the fill count)
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale = 0,
-                      uint32_t ins_n = 0, const float* ins_prio = nullptr);
+                      uint32_t ins_n = 0, const float* ins_prio = nullptr, const unsigned char* ins_done = nullptr);
+// (ins_done: the done bytes of the inserted batch; read with the frame-deduplicated layout only)
 // Update batches above this many entries (one per thread of a CTA) go to one launch of many
 // co-resident CTAs instead (measured: 11-20 us for 16384 entries against 15-29 us for 4096 in one CTA);
 // an update + insertion of short rows is then two launches, the update's and the insertion's.
@@ -332,7 +341,8 @@ struct PrbBulkLane {
     // wait runs out the lane is marked failed: the phase parity stays as it is (the load is still
     // outstanding), nothing is stored from the stage, and every later load and store of the lane is
     // skipped; finish() then only waits, again with a limit, for what is in flight.
-    __device__ __forceinline__ void store(void* gdst, uint32_t bytes)
+    // (gdst2 != nullptr: the stage is stored a second time, there, in the same bulk group)
+    __device__ __forceinline__ void store(void* gdst, uint32_t bytes, void* gdst2 = nullptr)
     {
         if (failed) return;
         bool done = false;
@@ -341,6 +351,9 @@ struct PrbBulkLane {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                              ::"l"(gdst), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
+                if (gdst2 != nullptr)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                                 ::"l"(gdst2), "r"(buf), "r"(bytes), "l"(stream_policy) : "memory");
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 done = true;
             }

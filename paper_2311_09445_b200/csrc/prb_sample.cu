@@ -32,6 +32,7 @@ constexpr int kThreads = 256;
 constexpr int kCtasPerSm = 2;
 constexpr uint32_t kChunk = 512;             // upper bound on granules per row chunk (8 KB)
 constexpr uint32_t kRowMode = 512;           // rows of at least this many 16-byte granules are split into chunks
+constexpr uint32_t kFrameRowMode = 64;       // ... frames of the frame-deduplicated layout from this many granules on
 constexpr uint32_t kTopFloats = 5120;        // tree entries staged in shared memory (20 KB) ...
 constexpr uint32_t kTopFloats32 = 1152;      // ... at fanout 32 only levels 1 and 2 can fit: 4.5 KB
 __host__ __device__ constexpr uint32_t top_floats_of(uint32_t K) { return K == 32 ? kTopFloats32 : kTopFloats; }
@@ -55,6 +56,9 @@ struct SamplePlan {
     // leaf prefetch (when the level above the leaves is read from global memory): the first pf_groups
     // lane groups of a CTA own K*K floats each at byte pf_off of the dynamic shared memory
     uint32_t pf_groups, pf_off;
+    // frame-deduplicated layout with frames long enough for the ring: the tasks of field F_OBS are
+    // (stack + 1) frames (0 .. stack steps back from the sampled slot) of frame_chunks chunks each
+    uint32_t frame_chunks;
 };
 
 // The K children of one node lie in shared memory at `row`: every lane of the group reads all of them
@@ -174,14 +178,41 @@ __device__ __forceinline__ void store_granule(unsigned char* base, uint64_t g, u
 // granule, by `nthreads` threads.  s_idx[r] is the leaf of stratum k_first + r.  The first two
 // granules per thread of ALL fields are loaded before anything is stored, so a small batch costs
 // one round trip instead of one per field; what is left goes field by field.
+// Frame-deduplicated layout: frame `back` steps back from slot `leaf`, no further back than `clamp` (the
+// distance to the episode's first frame): the slot that holds it.
+__device__ __forceinline__ uint64_t prb_frame_slot(const PrbView& v, uint32_t leaf, uint32_t back, uint32_t clamp)
+{
+    const uint64_t b = back < clamp ? back : clamp;
+    return ((uint64_t)leaf + v.capacity - b) % v.capacity;
+}
+
+// ... and the two observations of strata [k_first, k_first + n_rows) rebuilt granule by granule (short frames):
+// position pos (0 = oldest) of next_obs is the frame stack-1-pos steps back, of obs the frame stack-pos steps back.
+__device__ __forceinline__ void gather_short_frames(const PrbView& v, const PrbBatch& dst, uint32_t k_first, uint32_t n_rows,
+                                                    const uint32_t* s_idx, const uint32_t* s_clamp, uint32_t rank, uint32_t nthreads)
+{
+    const uint32_t vec = v.field_vec[F_OBS], W = v.field_bytes[F_OBS] / vec, S = v.stack, total = n_rows * S * W;
+    for (int f = F_OBS; f <= F_NEXT_OBS; ++f) {
+        if (dst.ptr[f] == nullptr) continue;
+        const uint64_t dbase = (uint64_t)k_first * S * W;
+        for (uint32_t e = rank; e < total; e += nthreads) {
+            const uint32_t r = e / (S * W), rem = e - r * S * W, pos = rem / W, off = rem - pos * W;
+            const uint32_t back = (f == F_NEXT_OBS) ? S - 1 - pos : S - pos;
+            const uint64_t slot = prb_frame_slot(v, s_idx[r], back, s_clamp[r]);
+            store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[F_OBS], slot * W + off, vec));
+        }
+    }
+}
+
 __device__ __forceinline__ void gather_short_fields(const PrbView& v, const SamplePlan& plan, const PrbBatch& dst,
                                                     uint32_t k_first, uint32_t n_rows, const uint32_t* s_idx,
-                                                    uint32_t rank, uint32_t nthreads)
+                                                    uint32_t rank, uint32_t nthreads, const uint32_t* s_clamp = nullptr)
 {
+    if (v.stack && plan.frame_chunks == 0) gather_short_frames(v, dst, k_first, n_rows, s_idx, s_clamp, rank, nthreads);
     uint4 tmp[PRB_NUM_FIELDS][2];
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (v.stack && f == F_OBS)) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -195,7 +226,7 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
     }
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0) continue;
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (v.stack && f == F_OBS)) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
         const uint64_t dbase = (uint64_t)k_first * W;
 #pragma unroll
@@ -225,6 +256,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     __shared__ volatile unsigned long long s_seen[R];     // answers of the atomics that publish the weights
     __shared__ float s_p[R];
     __shared__ unsigned s_flags[R];
+    __shared__ uint32_t s_clamp[R];                        // frame-deduplicated layout: how far back a stratum's frames reach
     __shared__ unsigned int s_last;
     extern __shared__ __align__(128) unsigned char s_ring[];   // long rows: mbarriers, then the ring buffers
 
@@ -292,7 +324,22 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                 if (plan.uniform) { leaf = (uint32_t)(((unsigned long long)r0 * fill) >> 32); p = 1.0f; }   // floor(u * fill)
                 else descend<K>(v, plan, s_top, s_child + (tid - lane), x, lane, leaf, p, flags,
                                 gi < plan.pf_groups ? reinterpret_cast<float*>(s_ring + plan.pf_off) + gi * (K * K) : nullptr);
-                if (lane == 0 && gi < n_round) { s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags; }
+                if (lane == 0 && gi < n_round) {
+                    s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags;
+                    if (v.stack) {
+                        // frames: the distance back to the episode's first frame -- the nearest marker among the
+                        // `stack` slots before this one (or slot 0 while the ring has not wrapped)
+                        unsigned marks = 0;
+                        for (uint32_t d = 1; d <= v.stack; ++d)
+                            marks |= (unsigned)((v.store[F_DONE][((uint64_t)leaf + v.capacity - d) % v.capacity] & kPrbEpisodeStart) ? 1u : 0u) << d;
+                        uint32_t c = v.stack;
+                        for (uint32_t d = v.stack; d >= 1; --d) {
+                            if (fill < v.capacity && leaf < d) c = d - 1;
+                            else if ((marks >> d) & 1u) c = d;
+                        }
+                        s_clamp[gi] = c;
+                    }
+                }
             }
             __syncthreads();
         }
@@ -387,6 +434,20 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     int f = 0;
                     while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
                     const uint32_t W = v.field_bytes[f] / 16u;
+                    if (plan.frame_chunks) {
+                        // one chunk of the frame `back` steps back: it is a part of next_obs (position stack-1-back)
+                        // and of obs (position stack-back): one load, up to two stores
+                        const uint32_t S = v.stack, in = r - plan.task_first[f], back = in / plan.frame_chunks;
+                        const uint32_t e0 = (in - back * plan.frame_chunks) * plan.chunk[f];
+                        const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
+                        if (!PRB_IN_BOUNDS(v, s_idx[k - kb] < v.capacity && k < B && back <= S && e0 < W && bytes <= plan.ring_stage_bytes)) continue;
+                        unsigned char* to_next = (back < S && dst.ptr[F_NEXT_OBS]) ? dst.ptr[F_NEXT_OBS] + (((uint64_t)k * S + (S - 1 - back)) * W + e0) * 16u : nullptr;
+                        unsigned char* to_obs = (back >= 1 && dst.ptr[F_OBS]) ? dst.ptr[F_OBS] + (((uint64_t)k * S + (S - back)) * W + e0) * 16u : nullptr;
+                        if (to_next == nullptr && to_obs == nullptr) continue;
+                        ring.load(v.store[F_OBS] + (prb_frame_slot(v, s_idx[k - kb], back, s_clamp[k - kb]) * W + e0) * 16u, bytes);
+                        ring.store(to_next ? to_next : to_obs, bytes, to_next ? to_obs : nullptr);
+                        continue;
+                    }
                     const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
                     const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
                     if (!PRB_IN_BOUNDS(v, s_idx[k - kb] < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes)) continue;
@@ -398,7 +459,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             const uint32_t k_flat = max(kb, k_own);
             if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
                 const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads / 2 - 32u : kThreads / 2;
-                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads);
+                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads, s_clamp + (k_flat - kb));
             }
         }
         __syncthreads();        // s_idx is rewritten by the next round
@@ -762,10 +823,24 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
 static bool plan_row_mode(const PrbView& v, const PrbBatch& dst, SamplePlan& plan)
 {
     plan.tps = 0;
+    plan.frame_chunks = 0;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         plan.task_first[f] = 0;
         plan.chunks[f] = 0;
         plan.chunk[f] = 0;
+        if (v.stack && f == F_OBS) {
+            // frames of at least 1 KB go through the ring, a frame at a time (stack + 1 frames per stratum serve
+            // both observations); shorter ones are rebuilt granule by granule
+            const uint32_t W = v.field_bytes[f] / v.field_vec[f];
+            if ((dst.ptr[F_OBS] != nullptr || dst.ptr[F_NEXT_OBS] != nullptr) && v.field_vec[f] == 16 && W >= kFrameRowMode) {
+                plan.frame_chunks = (W + kChunk - 1) / kChunk;
+                plan.chunk[f] = (W + plan.frame_chunks - 1) / plan.frame_chunks;
+                plan.chunks[f] = (v.stack + 1) * plan.frame_chunks;
+                plan.task_first[f] = plan.tps;
+                plan.tps += plan.chunks[f];
+            }
+            continue;
+        }
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
         const uint32_t W = v.field_bytes[f] / v.field_vec[f];
         if (v.field_vec[f] == 16 && W >= kRowMode) {
@@ -799,7 +874,7 @@ static void plan_staged_top(const PrbView& v, bool uniform, SamplePlan& plan)
 bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst)
 {
     SamplePlan plan;
-    return plan_row_mode(v, dst, plan);
+    return v.stack == 0 && plan_row_mode(v, dst, plan);      // (rebuilt observations: the one-kernel sample only)
 }
 
 int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, int32_t* d_idx, float* d_w,
@@ -820,7 +895,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     plan_staged_top(v, uniform != 0, plan);
     const uint32_t R = kThreads / v.fanout;
     const int ki = v.log2_fanout;
-    if (!row_mode && n_sub == 1 && !uniform && !buffer_norm && B >= kWideSampleFrom) {
+    if (!row_mode && n_sub == 1 && !uniform && !buffer_norm && B >= kWideSampleFrom && v.stack == 0) {
         // a large batch of short rows: one stratum per thread
         uint32_t grid = (B + kWideSampleStrata - 1) / kWideSampleStrata;
         const uint32_t one_wave = (uint32_t)sm_count * kCtasPerSm;

@@ -78,6 +78,22 @@ __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n
     }
 }
 
+// Frame-deduplicated layout: an insertion of n transitions at `cursor` writes n + prb_cleared_after(v, n)
+// leaves -- the last ones zero: they belong to the slots that follow the new cursor, whose history the
+// insertion overwrites once the ring has wrapped (before that they are empty and zero already) -- and the
+// leaf of an episode-start marker (bit 1 of its done byte) is zero whatever priority is given.
+__device__ __forceinline__ uint32_t prb_cleared_after(const PrbView& v, uint32_t n)
+{
+    if (v.stack == 0 || n == 0) return 0u;
+    const uint64_t room = v.capacity - n;
+    return room < v.stack ? (uint32_t)room : v.stack;
+}
+// ... and an update that names one of the `stack` slots that follow the cursor is stale.
+__device__ __forceinline__ bool prb_history_less(const PrbView& v, uint64_t cursor, uint64_t i)
+{
+    return v.stack != 0 && (i + v.capacity - cursor) % v.capacity < v.stack;
+}
+
 // The top of the tree staged in shared memory for the re-sum passes: levels 1 .. v.top_levels as
 // they lie in global memory from the start of level 1 (v.top_floats entries).  Below the staged
 // levels a pass re-sums only the parents that the batch reaches; a re-summed parent of the deepest
@@ -341,8 +357,10 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
                                                 float alpha, float eps, unsigned long long fill, unsigned char* smem,
                                                 uint32_t n = 0, const float* __restrict__ prio = nullptr,
                                                 uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
-                                                uint32_t stale = 0, PrbTop top = PrbTop{})
+                                                uint32_t stale = 0, PrbTop top = PrbTop{}, const unsigned char* __restrict__ ins_done = nullptr)
 {
+    // (frames: the insertion's dirty leaves reach past its n transitions; cursor, fill and priorities do not)
+    const uint32_t n_leaves = n + prb_cleared_after(v, n);
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
     const uint32_t rank = team.rank, nt = team.size;
@@ -368,7 +386,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             // stale: one of the `stale` slots written most recently, i.e. overwritten since it was sampled
             const uint64_t back = (i >= 0 && stale) ? (cursor + N - 1 - (uint64_t)i) % N : ~0ull;
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
-            else if (back < stale) flags |= PEARL_ST_STALE;
+            else if (back < stale || prb_history_less(v, cursor, (uint64_t)i)) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
             else { key = ((unsigned long long)(uint32_t)i << 32) | b; if (raw != 2) wmax = fmaxf(wmax, p); my_valid = true; my_idx = (uint32_t)i; }
             vals[b] = p;
@@ -454,7 +472,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     } else if (one_each) {
         if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
             const uint64_t ahead = slot.idx >= cursor ? slot.idx - cursor : slot.idx + N - cursor;   // distance from the cursor along the ring
-            if (!(ahead < n) && PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth] && slot.pos < n2)) leaves[slot.idx] = vals[slot.pos];
+            if (!(ahead < n_leaves) && PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth] && slot.pos < n2)) leaves[slot.idx] = vals[slot.pos];
         }
     } else {
         for (uint32_t s = rank; s < n2; s += nt) {
@@ -463,7 +481,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             const uint32_t i = (uint32_t)(key >> 32);
             const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
             const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;
-            if (last && !(ahead < n) && PRB_IN_BOUNDS(v, i < v.level_alloc[v.depth] && (uint32_t)key < n2)) leaves[i] = vals[(uint32_t)key];
+            if (last && !(ahead < n_leaves) && PRB_IN_BOUNDS(v, i < v.level_alloc[v.depth] && (uint32_t)key < n2)) leaves[i] = vals[(uint32_t)key];
         }
     }
     bool bad = false;
@@ -472,13 +490,16 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     // (reported by CTA 0: in a cluster the others read it after a barrier)
     if (n && prio == nullptr && team.parts > 1) { __threadfence(); team.phase_sync(); }
     const float dflt = (n && prio == nullptr) ? prb_default_priority(__ldcg(&v.state->max_prio_bits)) : 0.0f;
-    for (uint32_t t = rank; t < n; t += nt) {
+    for (uint32_t t = rank; t < n_leaves; t += nt) {
         if (!team.takes(t)) continue;
         uint64_t at = cursor + t;
         if (at >= N) at -= N;
-        float p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
-        if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
-        else imax = fmaxf(imax, p);
+        float p = 0.0f;
+        if (t < n && !(v.stack && (ins_done[t] & kPrbEpisodeStart))) {
+            p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
+            if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+            else imax = fmaxf(imax, p);
+        }
         if (PRB_IN_BOUNDS(v, at < N)) leaves[at] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
@@ -489,9 +510,9 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     // of equal ancestors does it; the insertion dirties parent range A = [a0, a1] >> sh and, if the
     // ring wrapped, B = [0, b1] >> sh
     const uint32_t lg = v.log2_fanout, T = prb_top_levels(v, top);
-    const uint64_t a0 = cursor, a1 = (n ? min(cursor + n, N) : cursor + 1) - 1;
-    const bool wrapped = cursor + n > N;
-    const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
+    const uint64_t a0 = cursor, a1 = (n ? min(cursor + n_leaves, N) : cursor + 1) - 1;
+    const bool wrapped = cursor + n_leaves > N;
+    const uint64_t b1 = wrapped ? cursor + n_leaves - N - 1 : 0;
     for (int l = (int)v.depth - 1; l >= (int)T; --l) {
         const uint32_t sh = min(lg * (v.depth - (uint32_t)l), 31u);      // (indices are below 2^31)
         if (one_each) {
@@ -527,20 +548,25 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
 __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const PrbTeam& team, uint32_t n,
                                                      const float* __restrict__ prio, uint64_t cursor,
                                                      PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
-                                                     unsigned max_bits = 0, PrbTop top = PrbTop{})
+                                                     unsigned max_bits = 0, PrbTop top = PrbTop{},
+                                                     const unsigned char* __restrict__ ins_done = nullptr)
 {
     const uint64_t N = v.capacity;
+    const uint32_t n_leaves = n + prb_cleared_after(v, n);
     const uint32_t D = v.depth, lg = v.log2_fanout, T = prb_top_levels(v, top);
     float* leaves = v.level[D];
     bool bad = false;
     float imax = 0.0f;
     const float dflt = prb_default_priority(max_bits);     // used when no priorities are given
-    for (uint32_t t = team.rank; t < n; t += team.size) {
+    for (uint32_t t = team.rank; t < n_leaves; t += team.size) {
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
-        float p = prio == nullptr ? dflt : ((pre.has_prio && t == team.rank) ? pre.prio : prio[t]);
-        if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
-        else imax = fmaxf(imax, p);
+        float p = 0.0f;
+        if (t < n && !(v.stack && (ins_done[t] & kPrbEpisodeStart))) {
+            p = prio == nullptr ? dflt : ((pre.has_prio && t == team.rank) ? pre.prio : prio[t]);
+            if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
+            else imax = fmaxf(imax, p);
+        }
         if (PRB_IN_BOUNDS(v, slot < N)) leaves[slot] = p;
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
@@ -549,9 +575,9 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
     team.sync();
     // dirty leaf ranges: A = [a0, a1]; if the ring wrapped also B = [0, b1]
     const uint64_t a0 = cursor;
-    const uint64_t a1 = min(cursor + n, N) - 1;
-    const bool wrapped = cursor + n > N;
-    const uint64_t b1 = wrapped ? cursor + n - N - 1 : 0;
+    const uint64_t a1 = min(cursor + n_leaves, N) - 1;
+    const bool wrapped = cursor + n_leaves > N;
+    const uint64_t b1 = wrapped ? cursor + n_leaves - N - 1 : 0;
     for (int l = (int)D - 1; l >= (int)T; --l) {
         const uint32_t sh = lg * (D - (uint32_t)l);
         const uint64_t pa0 = a0 >> sh, pa1 = a1 >> sh;

@@ -14,7 +14,8 @@ namespace {
 __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
                   const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale,
-                  uint32_t ins_n, const float* __restrict__ ins_prio, uint32_t ticket_total)
+                  uint32_t ins_n, const float* __restrict__ ins_prio, uint32_t ticket_total,
+                  const unsigned char* __restrict__ ins_done)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned long long s_cursor, s_fill;
@@ -41,9 +42,9 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
         if (threadIdx.x == 0) prb_publish_if_last(v, ins_n, cursor, fill, ticket_total, kPrbPublishTree);
     } else {
         fill = v.state->fill;
-        if (stale) cursor = v.state->cursor;
+        if (stale || v.stack) cursor = v.state->cursor;
     }
-    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top);
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top, ins_done);
 }
 
 // ---- large batches: one launch of many CTAs ------------------------------------------------------
@@ -80,6 +81,7 @@ __device__ __forceinline__ PrbWideEntry prb_wide_classify(const PrbView& v, int3
     if (i < 0 || (unsigned long long)i >= fill) { e.flags = PEARL_ST_BAD_INDEX; return e; }
     // one of the `stale` slots written most recently: overwritten since it was sampled
     if (stale && (cursor + N - 1 - (uint64_t)i) % N < stale) { e.flags = PEARL_ST_STALE; return e; }
+    if (prb_history_less(v, cursor, (uint64_t)i)) { e.flags = PEARL_ST_STALE; return e; }
     float p = x;
     const bool ok = raw ? prb_valid_priority(p) : prb_priority_pow(x, eps, alpha, p);
     if (!ok) { e.flags = PEARL_ST_BAD_PRIORITY; return e; }
@@ -190,7 +192,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
     const uint32_t tid = threadIdx.x, nctas = gridDim.x;
     const uint32_t gthreads = nctas * kWideThreads, gtid = blockIdx.x * kWideThreads + tid;
     const unsigned long long fill = v.state->fill;
-    const uint64_t cursor = stale ? v.state->cursor : 0ull;
+    const uint64_t cursor = (stale || v.stack) ? v.state->cursor : 0ull;
     const uint32_t K = v.fanout, lg = v.log2_fanout, D = v.depth, T = v.top_levels;
     unsigned* leaf_bits = reinterpret_cast<unsigned*>(v.level[D]);
     if (tid == 0) { s_flags = 0u; s_maxbits = 0u; }
@@ -345,7 +347,7 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
 
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
                       float alpha, float eps, cudaStream_t s, uint32_t stale,
-                      uint32_t ins_n, const float* ins_prio)
+                      uint32_t ins_n, const float* ins_prio, const unsigned char* ins_done)
 {
     if (ins_n && B > PEARL_UPDATE_SUBBATCH) return -1;
     // a batch of more than one entry per thread of a CTA: one launch of many CTAs (values or TD errors;
@@ -383,7 +385,7 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale,
-                               ins_n, ins_prio, ctas) != cudaSuccess)
+                               ins_n, ins_prio, ctas, ins_done) != cudaSuccess)
             return -1;
         ++launches;
     }

@@ -34,6 +34,7 @@ class Workload:
     eps: float = 1e-6
     philox_seed: int = 0
     counter_rows: bool = False   # observations are a function of the global insert id (too large to mirror)
+    frame_stack: int = 0         # > 0: the frame-deduplicated layout, obs_shape[0] == frame_stack frames per observation
 
     @property
     def obs_bytes(self) -> int:
@@ -45,7 +46,19 @@ class Workload:
 
     @property
     def transition_bytes(self) -> int:
+        """Bytes one transition takes in the Data Storage (and in an insertion's batch)."""
+        if self.frame_stack:
+            return self.obs_bytes // self.frame_stack + self.act_bytes + 4 + 1
         return 2 * self.obs_bytes + self.act_bytes + 4 + 1
+
+    @property
+    def sample_bytes(self) -> int:
+        """Bytes a sampled transition makes the gather read and write (both observations whole on the way out;
+        with frames, frame_stack + 1 frames on the way in)."""
+        small = self.act_bytes + 4 + 1
+        if self.frame_stack:
+            return (self.frame_stack + 1) * (self.obs_bytes // self.frame_stack) + 2 * self.obs_bytes + 2 * small
+        return 2 * (2 * self.obs_bytes + small)
 
 
 TINY = Workload("tiny", 4096, 2, (4,), "float32", (), "int32", 32, 0, 100, 1001, "normal")
@@ -54,7 +67,10 @@ DDPG = Workload("mujoco_ddpg", 1 << 20, 16, (17,), "float32", (6,), "float32", 2
                 dup_frac=0.05)
 ATARI = Workload("atari_dqn", 1 << 19, 32, (4, 84, 84), "uint8", (), "int32", 512, 512, 1_000, 1004, "normal",
                  counter_rows=True)
-WORKLOADS: Dict[str, Workload] = {w.name: w for w in (TINY, CARTPOLE, DDPG, ATARI)}
+# the Atari-shaped workload with one 84 x 84 frame stored per transition (a single actor's trajectory)
+ATARI_FRAMES = Workload("atari_dqn_frames", 1 << 19, 32, (4, 84, 84), "uint8", (), "int32", 512, 512, 1_000, 1005, "normal",
+                        counter_rows=True, frame_stack=4)
+WORKLOADS: Dict[str, Workload] = {w.name: w for w in (TINY, CARTPOLE, DDPG, ATARI, ATARI_FRAMES)}
 
 
 def sweep_cell(capacity: int, fanout: int, batch: int, cell_id: int = 0) -> Workload:
@@ -159,9 +175,11 @@ class FrameTrajectory:
     def _frame(self) -> np.ndarray:
         return self.rng.integers(0, 256, size=self.F, dtype=np.uint8)
 
-    def next(self, n: int) -> Dict[str, np.ndarray]:
+    def next(self, n: int, stacks: bool = True) -> Dict[str, np.ndarray]:
+        """n more slots.  stacks=False leaves "obs" / "next_obs" (the plain layout's rows) out."""
         F, S = self.F, self.S
-        out = {"frame": np.zeros((n, F), np.uint8), "obs": np.zeros((n, S * F), np.uint8), "next_obs": np.zeros((n, S * F), np.uint8),
+        out = {"frame": np.zeros((n, F), np.uint8), "obs": np.zeros((n if stacks else 0, S * F), np.uint8),
+               "next_obs": np.zeros((n if stacks else 0, S * F), np.uint8),
                "act": self.rng.integers(0, self.n_actions, size=n).astype(np.int32), "rew": self.rng.integers(-1, 2, size=n).astype(np.float32),
                "done": np.zeros(n, np.uint8), "prio": np.exp(self.rng.standard_normal(n)).astype(np.float32)}
         for t in range(n):
@@ -177,8 +195,9 @@ class FrameTrajectory:
             new = self._frame()
             nxt = self.window[1:] + [new]
             out["frame"][t] = new
-            out["obs"][t] = np.concatenate(self.window)
-            out["next_obs"][t] = np.concatenate(nxt)
+            if stacks:
+                out["obs"][t] = np.concatenate(self.window)
+                out["next_obs"][t] = np.concatenate(nxt)
             self.window = nxt
             self.left -= 1
             out["done"][t] = 1 if self.left == 0 else 0

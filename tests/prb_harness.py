@@ -47,12 +47,14 @@ def seed_for_sliver(oracle_mod, B, call=0, limit=1 << 22):
 
 
 class Pair:
-    def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True):
+    def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True, frame_stack=0):
+        """frame_stack > 0: both sides use the frame-deduplicated layout (obs_bytes = a whole stack; an insertion's
+        batch carries one frame per transition under "obs" and no "next_obs")."""
         from paper_2311_09445_b200 import PrioritizedReplay
-        self.gpu = PrioritizedReplay(capacity, fanout, obs_bytes, act_bytes, max_batch)
+        self.gpu = PrioritizedReplay(capacity, fanout, obs_bytes, act_bytes, max_batch, frame_stack=frame_stack)
         self.oracle_store = oracle_store
         self.ora = oracle_mod.OraclePRB(capacity, fanout, obs_bytes if oracle_store else 0,
-                                        act_bytes if oracle_store else 0)
+                                        act_bytes if oracle_store else 0, frame_stack=frame_stack)
         self.capacity, self.fanout = capacity, fanout
         self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
         self.dev = self.gpu.device
