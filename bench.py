@@ -443,13 +443,15 @@ def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=Tru
             ho = out_buffers(wl, dev, B, pinned=True)
             htd = [t.cpu().pin_memory() for t in tds]
 
+            prb.sample_host(B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
+                            ho["rew"], ho["next_obs"], ho["done"])
+
             def e2e_step(i):
-                if n_ins:
-                    b = hb[i % ROTATE]
-                    prb.insert_host(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"])
-                prb.sample_host(B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
-                                ho["rew"], ho["next_obs"], ho["done"])
-                prb.update_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps)
+                # one iteration through host buffers: the update for the batch sampled last, the new rows, the next batch
+                b = hb[i % ROTATE] if n_ins else dict.fromkeys(("obs", "act", "rew", "next_obs", "done", "prio"))
+                prb.step_host(ho["idx"], htd[i % ROTATE], wl.alpha, wl.eps, b["obs"], b["act"], b["rew"], b["next_obs"], b["done"],
+                              b["prio"], B, wl.beta, wl.philox_seed, ho["idx"], ho["w"], ho["obs"], ho["act"] if wl.act_bytes else None,
+                              ho["rew"], ho["next_obs"], ho["done"], n=n_ins)
 
             for i in range(3):
                 e2e_step(i)

@@ -227,6 +227,7 @@ int pearl_prb_update_insert(pearl_prb_t* prb, uint32_t B, const int32_t* d_idx, 
  * enqueued; the kernels are those of the two calls (for rows of 8 KB and more: the tree kernel beside the
  * copy of the new rows, then the sample).  d_upd_idx may be the d_idx of the previous step: it is read
  * before d_idx is written.
+ * n == 0 stands for an iteration without new transitions (update, then sample; the d_new_* are not read).
  * Arguments and errors as for the two calls; nothing is enqueued if any argument is refused. */
 int pearl_prb_step(pearl_prb_t* prb, uint32_t B_upd, const int32_t* d_upd_idx, const float* d_td, float alpha,
                    float eps, uint32_t n, const void* d_new_obs, const void* d_new_act, const float* d_new_rew,
@@ -274,6 +275,20 @@ int pearl_prb_sample_host(pearl_prb_t* prb, uint32_t B, float beta, uint64_t see
                           uint8_t* h_done);
 int pearl_prb_update_host(pearl_prb_t* prb, uint32_t B, const int32_t* h_idx, const float* h_td,
                           float alpha, float eps);
+
+/* pearl_prb_step through host buffers: the update for the previous batch, the insertion of the new
+ * transitions and the sample of the next batch, with every array in host memory (Section IV-A: the host
+ * runtime exchanges requests and data with the Replay Manager over PCIe).  Returns when the sampled batch is
+ * in the caller's arrays.  A step whose inputs and whose outputs come to at most 256 KB each makes no copy
+ * call: the inputs are gathered in a pinned buffer of the handle that the device reads in place, the kernels
+ * write the batch into that buffer, and the step's one synchronisation is the wait for them.  A larger step
+ * is pearl_prb_update_host, pearl_prb_insert_host and pearl_prb_sample_host one after the other.
+ * Arguments and errors as for pearl_prb_step, with host pointers. */
+int pearl_prb_step_host(pearl_prb_t* prb, uint32_t B_upd, const int32_t* h_upd_idx, const float* h_td, float alpha,
+                        float eps, uint32_t n, const void* h_new_obs, const void* h_new_act, const float* h_new_rew,
+                        const void* h_new_next_obs, const uint8_t* h_new_done, const float* h_new_prio, uint32_t B,
+                        float beta, uint64_t seed, int32_t* h_idx, float* h_w, void* h_obs, void* h_act, float* h_rew,
+                        void* h_next_obs, uint8_t* h_done);
 
 /* Largest batch pearl_prb_sample_static_scratch accepts. */
 #define PEARL_STATIC_SCRATCH_MAX_BATCH 4096u

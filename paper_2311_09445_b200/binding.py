@@ -53,6 +53,8 @@ SIGNATURES = {
     "pearl_prb_update_insert": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_step": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp,
                             _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "pearl_prb_step_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32, _u32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                 _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_insert_host": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample_host": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_update_host": (_i, [_vp, _u32, _vp, _vp, _f32, _f32]),
@@ -277,6 +279,20 @@ class PrioritizedReplay:
                                                   _hptr(next_obs, "next_obs"), _hptr(done, "done"))
         if rc != 0:
             raise PearlError(rc, "pearl_prb_sample_host")
+
+    def step_host(self, upd_idx, td, alpha: float, eps: float, new_obs, new_act, new_rew, new_next_obs, new_done, new_prio,
+                  B: int, beta: float, seed: int, idx, w=None, obs=None, act=None, rew=None, next_obs=None, done=None,
+                  n: Optional[int] = None) -> None:
+        """pearl_prb_step_host: one iteration (update, insertion, next sample) with host arrays."""
+        rc = load_library().pearl_prb_step_host(self._h, int(upd_idx.shape[0]), _hptr(upd_idx, "upd_idx"), _hptr(td, "td"), alpha,
+                                                eps, int(new_prio.shape[0]) if new_prio is not None else int(n or 0),
+                                                _hptr(new_obs, "new_obs"), _hptr(new_act, "new_act"), _hptr(new_rew, "new_rew"),
+                                                _hptr(new_next_obs, "new_next_obs"), _hptr(new_done, "new_done"),
+                                                _hptr(new_prio, "new_prio"), B, beta, seed, _hptr(idx, "idx"), _hptr(w, "w"),
+                                                _hptr(obs, "obs"), _hptr(act, "act"), _hptr(rew, "rew"),
+                                                _hptr(next_obs, "next_obs"), _hptr(done, "done"))
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_step_host")
 
     def update_host(self, idx, td, alpha: float, eps: float) -> None:
         rc = load_library().pearl_prb_update_host(self._h, int(idx.shape[0]), _hptr(idx, "idx"), _hptr(td, "td"),

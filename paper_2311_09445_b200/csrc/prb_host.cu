@@ -128,10 +128,12 @@ struct pearl_prb {
     // Small batches of the *_host calls travel packed: all arrays of a call in one pinned buffer, one
     // copy each way (2 x kPackBytes of pinned host memory; nullptr: every array is copied by itself).
     unsigned char* pin = nullptr;
+    unsigned char* pin_dev = nullptr;    // the same memory as the device sees it (mapped; nullptr if it cannot be mapped)
     cudaEvent_t pin_read = nullptr;      // the last host-to-device copy out of `pin` has been made
     // A sample of long rows inside a stream capture is two kernels: the descents on fork.side, the row
     // copy on the caller's stream (see sample_two_kernels below).
     cudaEvent_t desc_done = nullptr;             // the descents of the running two-kernel sample are done
+    cudaEvent_t relay_done = nullptr;            // ... and so is the relay behind them (see sample_two_kernels)
     cudaEvent_t gather_done[kPrbHandoffs] = {};   // the row copy that read hand-off area j is done
     unsigned long long gather_capture[kPrbHandoffs] = {};    // the capture gather_done[j] was last recorded in (0: none)
     unsigned long long side_capture = 0;         // the capture fork.side has last been made part of (0: none)
@@ -150,6 +152,7 @@ struct pearl_prb {
         if (subs.fork) cudaEventDestroy(subs.fork);
         if (pin_read) cudaEventDestroy(pin_read);
         if (desc_done) cudaEventDestroy(desc_done);
+        if (relay_done) cudaEventDestroy(relay_done);
         for (uint32_t j = 0; j < kPrbHandoffs; ++j) if (gather_done[j]) cudaEventDestroy(gather_done[j]);
         if (pin) cudaFreeHost(pin);
         cudaGetLastError();
@@ -219,7 +222,15 @@ int sample_two_kernels(pearl_prb* h, unsigned long long capture, uint32_t B, flo
     unsigned char* area = h->view.handoff[j];
     const int k1 = prb_launch_descend(h->view, B, seed, area, side, uniform, buffer_norm);
     if (k1 < 0) return -1;
-    if (cudaEventRecord(h->desc_done, side) != cudaSuccess || cudaStreamWaitEvent(main, h->desc_done, 0) != cudaSuccess) return -1;
+    // The row copy is launched as a programmatic dependent of what precedes it on the caller's stream, and an
+    // event wait joins the descents to that: it could then start before the descents' writes are flushed.  So
+    // the event it waits for is recorded behind a relay -- an empty kernel on a third stream that depends on
+    // the descents in full -- and not behind the descents themselves; the next call's descents, on the
+    // second stream, do not wait for the relay.
+    cudaStream_t third = h->subs.stream[0];
+    if (cudaEventRecord(h->desc_done, side) != cudaSuccess || cudaStreamWaitEvent(third, h->desc_done, 0) != cudaSuccess) return -1;
+    if (prb_launch_relay(third) < 0) return -1;
+    if (cudaEventRecord(h->relay_done, third) != cudaSuccess || cudaStreamWaitEvent(main, h->relay_done, 0) != cudaSuccess) return -1;
     const int k2 = prb_launch_gather(h->view, B, beta, area, d_idx, d_w, dst, main, h->main_last_gather == capture);
     if (k2 < 0) return -1;
     if (cudaEventRecord(h->gather_done[j], main) != cudaSuccess) return -1;
@@ -227,7 +238,7 @@ int sample_two_kernels(pearl_prb* h, unsigned long long capture, uint32_t B, flo
     h->handoff_next = (j + 1u) % kPrbHandoffs;
     h->main_last_gather = capture;
     h->after_forked_tree = 0;
-    return k1 + k2;
+    return k1 + k2 + 1;
 }
 
 bool finite_nonneg(float x) { return isfinite(x) && x >= 0.0f; }
@@ -301,15 +312,17 @@ static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, 
         }
     }
     if (cudaEventCreateWithFlags(&h->subs.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->desc_done, cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
+        cudaEventCreateWithFlags(&h->desc_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->relay_done, cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
     for (uint32_t j = 0; j < kPrbHandoffs; ++j)
         if (cudaEventCreateWithFlags(&h->gather_done[j], cudaEventDisableTiming) != cudaSuccess) { delete h; return PEARL_ERR_CUDA; }
-    if (cudaHostAlloc((void**)&h->pin, 2 * kPackBytes, cudaHostAllocDefault) != cudaSuccess ||
+    if (cudaHostAlloc((void**)&h->pin, 2 * kPackBytes, cudaHostAllocMapped) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->pin_read, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();                 // (not fatal: the host calls then copy array by array)
         if (h->pin) cudaFreeHost(h->pin);
         h->pin = nullptr;
     }
+    if (h->pin && cudaHostGetDevicePointer((void**)&h->pin_dev, h->pin, 0) != cudaSuccess) { cudaGetLastError(); h->pin_dev = nullptr; }
     if (slab) {
         if (slab_bytes < L.total || ((uintptr_t)slab & (kAlign - 1))) { delete h; return slab_bytes < L.total ? PEARL_ERR_OOM : PEARL_ERR_ALIGN; }
         h->base = (unsigned char*)slab;
@@ -582,13 +595,15 @@ int pearl_prb_step(pearl_prb_t* h, uint32_t B_upd, const int32_t* d_upd_idx, con
 {
     const void* in[PRB_NUM_FIELDS] = { d_new_obs, d_new_next_obs, d_new_act, d_new_rew, d_new_done };
     const void* out[PRB_NUM_FIELDS] = { d_obs, d_next_obs, d_act, d_rew, d_done };
-    int rc = check_update_insert_args(h, B_upd, d_upd_idx, d_td, alpha, eps, n, in, d_new_prio);
+    // (n == 0: an iteration without new transitions -- update, then sample)
+    int rc = check_update_insert_args(h, B_upd, d_upd_idx, d_td, alpha, eps, n ? n : 1u, in, d_new_prio);
     if (rc != PEARL_OK) return rc;
     rc = check_sample_args(h, B, beta, d_idx, d_w, out);
     if (rc != PEARL_OK) return rc;
     // (both calls' arguments have been checked: nothing is enqueued unless both go through)
-    rc = pearl_prb_update_insert(h, B_upd, d_upd_idx, d_td, alpha, eps, n, d_new_obs, d_new_act, d_new_rew, d_new_next_obs,
-                                 d_new_done, d_new_prio);
+    rc = n ? pearl_prb_update_insert(h, B_upd, d_upd_idx, d_td, alpha, eps, n, d_new_obs, d_new_act, d_new_rew, d_new_next_obs,
+                                     d_new_done, d_new_prio)
+           : pearl_prb_update(h, B_upd, d_upd_idx, d_td, alpha, eps);
     if (rc != PEARL_OK) return rc;
     return pearl_prb_sample(h, B, beta, seed, d_idx, d_w, d_obs, d_act, d_rew, d_next_obs, d_done);
 }
@@ -599,8 +614,8 @@ namespace {
 
 // Offsets of up to seven arrays packed one after another, each start 16-byte aligned.
 struct Packing {
-    uint64_t off[PRB_NUM_FIELDS + 2];
-    uint64_t bytes[PRB_NUM_FIELDS + 2];
+    uint64_t off[PRB_NUM_FIELDS + 3];
+    uint64_t bytes[PRB_NUM_FIELDS + 3];
     uint64_t total = 0;
     void add(int slot, uint64_t nbytes)
     {
@@ -735,6 +750,62 @@ int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, cons
     int rc = pearl_prb_update(h, B, d_idx, d_td, alpha, eps);
     if (rc != PEARL_OK) return rc;
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+// One iteration through host buffers as one call.  A small step (all inputs, and all outputs, within 256 KB
+// each) makes no copy call at all: the inputs are gathered in the handle's pinned buffer, which the device
+// sees mapped, the kernels read them from there and write the sampled batch into its second half, and the
+// one synchronisation of the step is the wait for that.  A larger step is the three host calls.
+int pearl_prb_step_host(pearl_prb_t* h, uint32_t B_upd, const int32_t* h_upd_idx, const float* h_td, float alpha, float eps,
+                        uint32_t n, const void* h_new_obs, const void* h_new_act, const float* h_new_rew, const void* h_new_next_obs,
+                        const uint8_t* h_new_done, const float* h_new_prio, uint32_t B, float beta, uint64_t seed, int32_t* h_idx,
+                        float* h_w, void* h_obs, void* h_act, float* h_rew, void* h_next_obs, uint8_t* h_done)
+{
+    if (!h || !h_upd_idx || !h_td || !h_idx) return PEARL_ERR_NULL;
+    if (B_upd == 0 || B_upd > h->max_batch || n > h->max_batch || B == 0 || B > h->max_batch) return PEARL_ERR_BAD_BATCH;
+    if (n > h->view.capacity) return PEARL_ERR_TOO_MANY;
+    if (!finite_nonneg(alpha) || !finite_nonneg(eps) || !finite_nonneg(beta)) return PEARL_ERR_BAD_ARG;
+    if (n && h->view.stack && (h_new_next_obs || !h_new_done)) return PEARL_ERR_BAD_ARG;
+    const void* src[PRB_NUM_FIELDS + 3] = { h_new_obs, h_new_next_obs, h_new_act, h_new_rew, h_new_done, h_new_prio, h_upd_idx, h_td };
+    void* dst[PRB_NUM_FIELDS + 2] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_idx, h_w };
+    Packing in, out;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) in.add(f, src[f] ? (uint64_t)n * h->view.field_bytes[f] : 0);
+    in.add(PRB_NUM_FIELDS, h_new_prio ? (uint64_t)n * 4 : 0);
+    in.add(PRB_NUM_FIELDS + 1, (uint64_t)B_upd * 4);
+    in.add(PRB_NUM_FIELDS + 2, (uint64_t)B_upd * 4);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) out.add(f, dst[f] ? (uint64_t)B * h->view.out_bytes[f] : 0);
+    out.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
+    out.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
+    if (!(h->pin_dev && in.total <= kPackBytes && out.total <= kPackBytes)) {
+        int rc = pearl_prb_update_host(h, B_upd, h_upd_idx, h_td, alpha, eps);
+        if (rc != PEARL_OK) return rc;
+        rc = n ? pearl_prb_insert_host(h, n, h_new_obs, h_new_act, h_new_rew, h_new_next_obs, h_new_done, h_new_prio) : PEARL_OK;
+        if (rc != PEARL_OK) return rc;
+        return pearl_prb_sample_host(h, B, beta, seed, h_idx, h_w, h_obs, h_act, h_rew, h_next_obs, h_done);
+    }
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    // the pinned buffer may still be the source of a copy an earlier *_host call left on the stream
+    if (cudaEventSynchronize(h->pin_read) != cudaSuccess) return PEARL_ERR_CUDA;
+    void* din[PRB_NUM_FIELDS + 3];
+    void* dout[PRB_NUM_FIELDS + 2];
+    for (int i = 0; i < PRB_NUM_FIELDS + 3; ++i) {
+        din[i] = nullptr;
+        if (!src[i] || in.bytes[i] == 0) continue;
+        memcpy(h->pin + in.off[i], src[i], in.bytes[i]);
+        din[i] = h->pin_dev + in.off[i];
+    }
+    for (int i = 0; i < PRB_NUM_FIELDS + 2; ++i) dout[i] = (dst[i] && out.bytes[i]) ? h->pin_dev + kPackBytes + out.off[i] : nullptr;
+    int rc = pearl_prb_step(h, B_upd, (const int32_t*)din[PRB_NUM_FIELDS + 1], (const float*)din[PRB_NUM_FIELDS + 2], alpha, eps, n,
+                            din[F_OBS], din[F_ACT], (const float*)din[F_REW], din[F_NEXT_OBS], (const uint8_t*)din[F_DONE],
+                            (const float*)din[PRB_NUM_FIELDS], B, beta, seed, (int32_t*)dout[PRB_NUM_FIELDS],
+                            (float*)dout[PRB_NUM_FIELDS + 1], dout[F_OBS], dout[F_ACT], (float*)dout[F_REW], dout[F_NEXT_OBS],
+                            (uint8_t*)dout[F_DONE]);
+    if (rc != PEARL_OK) return rc;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    for (int i = 0; i < PRB_NUM_FIELDS + 2; ++i)
+        if (dout[i]) memcpy(dst[i], h->pin + kPackBytes + out.off[i], out.bytes[i]);
+    return PEARL_OK;
 }
 
 // ---- sampling with static scratch --------------------------------------------------------------

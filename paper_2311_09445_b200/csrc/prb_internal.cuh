@@ -139,6 +139,8 @@ int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned cha
 // too -- so this one may read rows while that one is still running)
 int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned char* handoff, int32_t* d_idx, float* d_w,
                       const PrbBatch& dst, cudaStream_t s, bool early_reads = false);
+// An empty kernel: a node that depends in full on what precedes it on s, for a programmatic dependent to hang on.
+int prb_launch_relay(cudaStream_t s);
 // true if a sample that writes these fields moves rows long enough for the bulk-copy ring
 bool prb_sample_has_long_rows(const PrbView& v, const PrbBatch& dst);
 // (stale > 0: skip entries that name one of the `stale` most recently written ring slots)

@@ -430,6 +430,41 @@ def test_host_buffer_calls(oracle_mod):
     pr.close()
 
 
+@pytest.mark.parametrize("wl,N,B,n", [(wk.CARTPOLE, 5000, 64, 64), (wk.DDPG, 70_000, 256, 256), (wk.DDPG, 5000, 3000, 1000),
+                                      (wk.ATARI, 600, 16, 8)])
+def test_step_through_host_buffers(oracle_mod, wl, N, B, n):
+    # pearl_prb_step_host: a small step travels through the handle's mapped pinned buffer (no copy call), a
+    # larger one is the three host calls; either way the oracle's update, insert, sample
+    wl = wk.scaled(wl, N)
+    rng = np.random.default_rng(N + B)
+    pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096)
+    next_id = 0
+    for first in range(0, N, 1000):
+        m = min(1000, N - first)
+        pr.insert(wk.transitions(wl, rng, m, next_id), host_call=True)
+        next_id += m
+    o, g = pr.sample(B, wl.beta, 1, host_call=True)
+    for step in range(6):
+        idx, td = wk.update_batch(wl, rng, o["idx"])
+        b = wk.transitions(wl, rng, n, next_id)
+        next_id += n
+        assert pr.ora.update(idx, td, wl.alpha, wl.eps) == 0
+        assert pr.ora.insert(b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], b["prio"]) == 0
+        o = pr.ora.sample(B, wl.beta, 2 + step)
+        g = {"idx": np.full(B, -1, np.int32), "w": np.zeros(B, np.float32), "obs": np.zeros((B, wl.obs_bytes), np.uint8),
+             "act": np.zeros((B, wl.act_bytes), np.uint8), "rew": np.zeros(B, np.float32),
+             "next_obs": np.zeros((B, wl.obs_bytes), np.uint8), "done": np.zeros(B, np.uint8)}
+        c = {k: np.ascontiguousarray(v) for k, v in b.items()}
+        pr.gpu.step_host(np.ascontiguousarray(idx, np.int32), np.ascontiguousarray(td, np.float32), wl.alpha, wl.eps, c["obs"], c["act"],
+                         c["rew"], c["next_obs"], c["done"], c["prio"], B, wl.beta, 2 + step, g["idx"], g["w"], g["obs"], g["act"],
+                         g["rew"], g["next_obs"], g["done"])
+        pr.compare_sample(o, g)
+        pr.compare_tree()
+        pr.compare_state()
+    pr.compare_status()
+    pr.close()
+
+
 @pytest.mark.parametrize("wl,N,B,n", [(wk.CARTPOLE, 5000, 64, 64), (wk.DDPG, 70_000, 256, 256), (wk.DDPG, 3000, 1000, 777),
                                       (wk.ATARI, 1500, 512, 512), (wk.ATARI, 700, 37, 1), (wk.ATARI, 700, 4096, 300)])
 def test_fused_update_insert(oracle_mod, wl, N, B, n):
