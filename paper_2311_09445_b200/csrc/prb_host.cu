@@ -167,7 +167,7 @@ inline bool misaligned(const void* p, uint32_t granule) { return ((uintptr_t)p &
 int check_batch_ptrs(const pearl_prb* h, const void* const ptrs[PRB_NUM_FIELDS], bool outputs = false)
 {
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        const uint32_t row = outputs ? h->view.out_bytes[f] : h->view.field_bytes[f];
+        const uint32_t row = outputs ? h->lay.out_bytes[f] : h->view.field_bytes[f];
         if (ptrs[f] && row && misaligned(ptrs[f], h->view.field_vec[f])) return PEARL_ERR_ALIGN;
     }
     return PEARL_OK;
@@ -353,7 +353,6 @@ static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, 
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         v.store[f] = at(h, L.off_store[f]);
         v.field_bytes[f] = L.field_bytes[f];
-        v.out_bytes[f] = L.out_bytes[f];
         v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
     }
     v.stack = L.stack;
@@ -692,7 +691,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
     void* dst[PRB_NUM_FIELDS + 2] = { h_obs, h_next_obs, h_act, h_rew, h_done, h_idx, h_w };
     void* dev[PRB_NUM_FIELDS + 2];
     Packing pk;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, dst[f] ? (uint64_t)B * h->view.out_bytes[f] : 0);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) pk.add(f, dst[f] ? (uint64_t)B * h->lay.out_bytes[f] : 0);
     pk.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
     pk.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
     if (h->pin && pk.total <= kPackBytes) {
@@ -711,7 +710,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
         return PEARL_OK;
     }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f)
-        dev[f] = (dst[f] && h->view.out_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
+        dev[f] = (dst[f] && h->lay.out_bytes[f]) ? at(h, h->lay.off_stage_out[f]) : nullptr;
     int32_t* d_idx = (int32_t*)at(h, h->lay.off_stage_out_idx);
     float* d_w = h_w ? (float*)at(h, h->lay.off_stage_out_w) : nullptr;
     int rc = pearl_prb_sample(h, B, beta, seed, d_idx, d_w, dev[F_OBS], dev[F_ACT], (float*)dev[F_REW],
@@ -721,7 +720,7 @@ int pearl_prb_sample_host(pearl_prb_t* h, uint32_t B, float beta, uint64_t seed,
     if (h_w && cudaMemcpyAsync(h_w, d_w, (uint64_t)B * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (!dev[f]) continue;
-        if (cudaMemcpyAsync(dst[f], dev[f], (uint64_t)B * h->view.out_bytes[f], cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+        if (cudaMemcpyAsync(dst[f], dev[f], (uint64_t)B * h->lay.out_bytes[f], cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
             return PEARL_ERR_CUDA;
     }
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
@@ -773,7 +772,7 @@ int pearl_prb_step_host(pearl_prb_t* h, uint32_t B_upd, const int32_t* h_upd_idx
     in.add(PRB_NUM_FIELDS, h_new_prio ? (uint64_t)n * 4 : 0);
     in.add(PRB_NUM_FIELDS + 1, (uint64_t)B_upd * 4);
     in.add(PRB_NUM_FIELDS + 2, (uint64_t)B_upd * 4);
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) out.add(f, dst[f] ? (uint64_t)B * h->view.out_bytes[f] : 0);
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) out.add(f, dst[f] ? (uint64_t)B * h->lay.out_bytes[f] : 0);
     out.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
     out.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
     if (!(h->pin_dev && in.total <= kPackBytes && out.total <= kPackBytes)) {

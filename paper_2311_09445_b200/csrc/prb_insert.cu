@@ -90,6 +90,7 @@ struct FusedUpdate {
 
 // Short rows only: CTA 0 = tree (after the optional update), CTAs 1.. = a contiguous range of tiles
 // each.  Threads 0..kWorkers-1 work; thread kWorkers reads the cursor for the CTA and takes the ticket.
+template <bool kFrames>
 __global__ void __launch_bounds__(kThreadsShort, 2)
 prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
                   const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
@@ -119,9 +120,10 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
             if (upd.B)      // update and insertion share one re-sum pass per level
-                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top, src.ptr[F_DONE]);
+                prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top,
+                                src.ptr[F_DONE], kFrames ? v.stack : 0u);
             else
-                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp, top, src.ptr[F_DONE]);
+                prb_insert_tree_team(v, team, n, prio, cursor, pre, s_maxp, top, src.ptr[F_DONE], kFrames ? v.stack : 0u);
         } else {
             const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
             const uint32_t copy_ctas = gridDim.x - 1, c = blockIdx.x - 1;
@@ -137,6 +139,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
 // not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, unless a tree kernel beside
 // this one does it) and the short-field tiles (dealt round-robin, CTA 1 first).  Thread
 // 32+kWorkers: cursor and ticket.
+template <bool kFrames>
 __global__ void __launch_bounds__(kThreadsRows, 1)
 prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
                        const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
@@ -203,7 +206,8 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
         PrbTeam team;
         team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
         if (blockIdx.x == 0 && plan.tree_ctas == 0)
-            prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp, PrbTop{}, src.ptr[F_DONE]);
+            prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp, PrbTop{}, src.ptr[F_DONE],
+                                 kFrames ? v.stack : 0u);
         const uint32_t n_tiles = plan.first_tile[PRB_NUM_FIELDS];
         for (uint32_t tile = (blockIdx.x + gridDim.x - 1) % gridDim.x; tile < n_tiles; tile += gridDim.x)
             copy_tile(v, plan, src, n, cursor, tile, team.rank, team.size);
@@ -291,24 +295,30 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     if (tasks == 0) {
         static bool big_smem[kPrbMaxDevices];
         if (!big_smem[dev]) {
-            if (cudaFuncSetAttribute(prb_insert_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float))) != cudaSuccess)
+            const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float));
+            if (cudaFuncSetAttribute(prb_insert_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+                cudaFuncSetAttribute(prb_insert_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
                 return -1;
             big_smem[dev] = true;
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        prb_insert_kernel<<<copy_ctas + 1, kThreadsShort, upd_smem + v.top_floats * (uint32_t)sizeof(float), s>>>(v, n, src, d_prio, plan, upd);
+        const uint32_t smem = upd_smem + v.top_floats * (uint32_t)sizeof(float);
+        if (v.stack) prb_insert_kernel<true><<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, n, src, d_prio, plan, upd);
+        else prb_insert_kernel<false><<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, n, src, d_prio, plan, upd);
     } else {
         const uint32_t smem = kRingBarBytes + plan.ring_stages * plan.ring_stage_bytes;
         static bool big_rows[kPrbMaxDevices];
         if (!big_rows[dev]) {
-            if (cudaFuncSetAttribute(prb_insert_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(prb_insert_rows_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(kRingBarBytes + kRingBytes)) != cudaSuccess ||
+                cudaFuncSetAttribute(prb_insert_rows_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
                 return -1;
             big_rows[dev] = true;
         }
-        prb_insert_rows_kernel<<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
+        if (v.stack) prb_insert_rows_kernel<true><<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
+        else prb_insert_rows_kernel<false><<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
         if (forked && cudaStreamWaitEvent(s, fork->join, 0) != cudaSuccess) return -1;
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;

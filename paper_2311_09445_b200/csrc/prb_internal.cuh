@@ -47,24 +47,9 @@ struct PrbState {
 
 // Geometry and device addresses, passed to kernels by value.
 struct PrbView {
+    // (the scalars and the short arrays first, the per-level arrays last: a kernel reads its parameters
+    // through the constant cache, and the few lines at the front serve the start of every kernel)
     PrbState* state;
-    float* level[PRB_MAX_LEVELS];     // level[l] holds K * n_{l-1} entries (level[0]: 1)
-    uint32_t level_alloc[PRB_MAX_LEVELS];   // entries of level l, zero padding included
-    unsigned char* store[PRB_NUM_FIELDS];
-    uint32_t field_bytes[PRB_NUM_FIELDS];
-    uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
-    // Frame-deduplicated layout (stack > 0): the obs store keeps ONE frame of field_bytes[F_OBS] bytes per slot
-    // (the newest frame of the transition's next observation), there is no next_obs store
-    // (field_bytes[F_NEXT_OBS] == 0), and a sample rebuilds both observations, `stack` frames each, from
-    // consecutive slots.  out_bytes[f] is the size of a row of field f as a sample hands it out (equal to
-    // field_bytes[f] except for the two rebuilt fields).  Bit 1 of a slot's done byte marks an episode start.
-    uint32_t stack;
-    uint32_t out_bytes[PRB_NUM_FIELDS];
-    double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
-    // A sample of long rows that is issued as two kernels (descents, then the row copy) hands indices
-    // and leaf priorities from the first to the second through one of a few areas of the slab, used in turn:
-    // a 256-byte header (PrbHandoffHeader), max_batch indices, max_batch priorities.
-    unsigned char* handoff[kPrbHandoffs];
     uint64_t capacity;
     uint32_t fanout;                  // K
     uint32_t log2_fanout;
@@ -74,6 +59,22 @@ struct PrbView {
     // level 1: the part of the tree a CTA may stage in shared memory (at most kPrbTopFloats entries)
     uint32_t top_levels;
     uint32_t top_floats;
+    // Frame-deduplicated layout (stack > 0): the obs store keeps ONE frame of field_bytes[F_OBS] bytes per slot
+    // (the newest frame of the transition's next observation), there is no next_obs store
+    // (field_bytes[F_NEXT_OBS] == 0), and a sample rebuilds both observations, `stack` frames each, from
+    // consecutive slots (each output row is stack * field_bytes[F_OBS] bytes).  Bit 1 of a slot's done byte
+    // marks an episode start.
+    uint32_t stack;
+    uint32_t field_bytes[PRB_NUM_FIELDS];
+    uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
+    unsigned char* store[PRB_NUM_FIELDS];
+    double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
+    // A sample of long rows that is issued as two kernels (descents, then the row copy) hands indices
+    // and leaf priorities from the first to the second through one of a few areas of the slab, used in turn:
+    // a 256-byte header (PrbHandoffHeader), max_batch indices, max_batch priorities.
+    unsigned char* handoff[kPrbHandoffs];
+    float* level[PRB_MAX_LEVELS];     // level[l] holds K * n_{l-1} entries (level[0]: 1)
+    uint32_t level_alloc[PRB_MAX_LEVELS];   // entries of level l, zero padding included
     uint32_t top_off[PRB_MAX_LEVELS];     // entries from the start of level 1 to the start of staged level l (l >= 1)
 };
 

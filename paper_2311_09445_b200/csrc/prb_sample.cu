@@ -189,9 +189,10 @@ __device__ __forceinline__ uint64_t prb_frame_slot(const PrbView& v, uint32_t le
 // ... and the two observations of strata [k_first, k_first + n_rows) rebuilt granule by granule (short frames):
 // position pos (0 = oldest) of next_obs is the frame stack-1-pos steps back, of obs the frame stack-pos steps back.
 __device__ __forceinline__ void gather_short_frames(const PrbView& v, const PrbBatch& dst, uint32_t k_first, uint32_t n_rows,
-                                                    const uint32_t* s_idx, const uint32_t* s_clamp, uint32_t rank, uint32_t nthreads)
+                                                    const uint32_t* s_idx, const uint32_t* s_clamp, uint32_t rank, uint32_t nthreads,
+                                                    uint32_t S)
 {
-    const uint32_t vec = v.field_vec[F_OBS], W = v.field_bytes[F_OBS] / vec, S = v.stack, total = n_rows * S * W;
+    const uint32_t vec = v.field_vec[F_OBS], W = v.field_bytes[F_OBS] / vec, total = n_rows * S * W;
     for (int f = F_OBS; f <= F_NEXT_OBS; ++f) {
         if (dst.ptr[f] == nullptr) continue;
         const uint64_t dbase = (uint64_t)k_first * S * W;
@@ -206,13 +207,15 @@ __device__ __forceinline__ void gather_short_frames(const PrbView& v, const PrbB
 
 __device__ __forceinline__ void gather_short_fields(const PrbView& v, const SamplePlan& plan, const PrbBatch& dst,
                                                     uint32_t k_first, uint32_t n_rows, const uint32_t* s_idx,
-                                                    uint32_t rank, uint32_t nthreads, const uint32_t* s_clamp = nullptr)
+                                                    uint32_t rank, uint32_t nthreads, const uint32_t* s_clamp = nullptr,
+                                                    uint32_t stack = 0)
 {
-    if (v.stack && plan.frame_chunks == 0) gather_short_frames(v, dst, k_first, n_rows, s_idx, s_clamp, rank, nthreads);
+    // (stack: PrbView::stack in the kernel instantiated for the frame layout, the constant 0 elsewhere)
+    if (stack && plan.frame_chunks == 0) gather_short_frames(v, dst, k_first, n_rows, s_idx, s_clamp, rank, nthreads, stack);
     uint4 tmp[PRB_NUM_FIELDS][2];
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (v.stack && f == F_OBS)) continue;
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (stack && f == F_OBS)) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -226,7 +229,7 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
     }
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
-        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (v.stack && f == F_OBS)) continue;
+        if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (stack && f == F_OBS)) continue;
         const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
         const uint64_t dbase = (uint64_t)k_first * W;
 #pragma unroll
@@ -242,7 +245,8 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
     }
 }
 
-template <int K>
+// kFrames: the instance for the frame-deduplicated layout (it rebuilds both observations from single frames)
+template <int K, bool kFrames>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uint64_t seed,
                   int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
@@ -261,6 +265,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     extern __shared__ __align__(128) unsigned char s_ring[];   // long rows: mbarriers, then the ring buffers
 
     const uint32_t tid = threadIdx.x;
+    const uint32_t stack = kFrames ? v.stack : 0u;
     const bool bulk = plan.ring_stages > 0;
     PrbBulkLane ring;            // lanes 0 .. ring_stages-1 of warp 0 own one stage each
     const bool ring_lane = bulk && tid < plan.ring_stages;
@@ -326,14 +331,14 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                                 gi < plan.pf_groups ? reinterpret_cast<float*>(s_ring + plan.pf_off) + gi * (K * K) : nullptr);
                 if (lane == 0 && gi < n_round) {
                     s_idx[gi] = leaf; s_p[gi] = p; s_flags[gi] = flags;
-                    if (v.stack) {
+                    if (stack) {
                         // frames: the distance back to the episode's first frame -- the nearest marker among the
                         // `stack` slots before this one (or slot 0 while the ring has not wrapped)
                         unsigned marks = 0;
-                        for (uint32_t d = 1; d <= v.stack; ++d)
+                        for (uint32_t d = 1; d <= stack; ++d)
                             marks |= (unsigned)((v.store[F_DONE][((uint64_t)leaf + v.capacity - d) % v.capacity] & kPrbEpisodeStart) ? 1u : 0u) << d;
-                        uint32_t c = v.stack;
-                        for (uint32_t d = v.stack; d >= 1; --d) {
+                        uint32_t c = stack;
+                        for (uint32_t d = stack; d >= 1; --d) {
                             if (fill < v.capacity && leaf < d) c = d - 1;
                             else if ((marks >> d) & 1u) c = d;
                         }
@@ -434,10 +439,10 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                     int f = 0;
                     while (plan.chunks[f] == 0 || r >= plan.task_first[f] + plan.chunks[f]) ++f;
                     const uint32_t W = v.field_bytes[f] / 16u;
-                    if (plan.frame_chunks) {
+                    if constexpr (kFrames) { if (plan.frame_chunks) {
                         // one chunk of the frame `back` steps back: it is a part of next_obs (position stack-1-back)
                         // and of obs (position stack-back): one load, up to two stores
-                        const uint32_t S = v.stack, in = r - plan.task_first[f], back = in / plan.frame_chunks;
+                        const uint32_t S = stack, in = r - plan.task_first[f], back = in / plan.frame_chunks;
                         const uint32_t e0 = (in - back * plan.frame_chunks) * plan.chunk[f];
                         const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
                         if (!PRB_IN_BOUNDS(v, s_idx[k - kb] < v.capacity && k < B && back <= S && e0 < W && bytes <= plan.ring_stage_bytes)) continue;
@@ -447,7 +452,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
                         ring.load(v.store[F_OBS] + (prb_frame_slot(v, s_idx[k - kb], back, s_clamp[k - kb]) * W + e0) * 16u, bytes);
                         ring.store(to_next ? to_next : to_obs, bytes, to_next ? to_obs : nullptr);
                         continue;
-                    }
+                    } }
                     const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
                     const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
                     if (!PRB_IN_BOUNDS(v, s_idx[k - kb] < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes)) continue;
@@ -459,7 +464,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
             const uint32_t k_flat = max(kb, k_own);
             if (k_flat < kb + n_round && (!bulk || tid >= 32)) {
                 const uint32_t rank = bulk ? tid - 32u : tid, nthreads = bulk ? kThreads / 2 - 32u : kThreads / 2;
-                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads, s_clamp + (k_flat - kb));
+                gather_short_fields(v, plan, dst, k_flat, kb + n_round - k_flat, s_idx + (k_flat - kb), rank, nthreads, s_clamp + (k_flat - kb), stack);
             }
         }
         __syncthreads();        // s_idx is rewritten by the next round
@@ -923,15 +928,16 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     // dynamic shared memory a CTA of this kernel may have: what the device allows less its static part
     static uint32_t dyn_max[kPrbMaxDevices][6];
     if (dyn_max[dev][ki] == 0) {
+        // (the frame-layout instance has the same static shared memory: one figure serves both)
         cudaFuncAttributes fa;
         int optin = 0;
         cudaError_t e = cudaSuccess;
         switch (v.fanout) {
-        case 2: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<2>); break;
-        case 4: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<4>); break;
-        case 8: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<8>); break;
-        case 16: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<16>); break;
-        default: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<32>); break;
+        case 2: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<2, true>); break;
+        case 4: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<4, true>); break;
+        case 8: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<8, true>); break;
+        case 16: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<16, true>); break;
+        default: e = cudaFuncGetAttributes(&fa, prb_sample_kernel<32, true>); break;
         }
         if (e != cudaSuccess || cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
             return -1;
@@ -1020,7 +1026,8 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         prb_leaf_min_kernel<<<(unsigned)ctas, 256, 0, s>>>(v);
         extra_launches = 1;
     }
-    static bool big_smem[kPrbMaxDevices][6];
+    static bool big_smem[kPrbMaxDevices][2][6];
+    const int fr = v.stack ? 1 : 0;
     cudaError_t attr = cudaSuccess;
     if (n_sub > 1 && (cudaEventRecord(subs->fork, s) != cudaSuccess)) return -1;
     for (uint32_t i = 0; i < n_sub; ++i) {
@@ -1031,16 +1038,18 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         }
         const uint32_t grid = sub_grid[i], smem = sub_smem[i];
         const SamplePlan& sp = sub_plan[i];
-#define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
+#define PRB_LAUNCH_SAMPLE_AS(KK, FF)                                                                              \
     do {                                                                                                          \
-        if (max_smem && !big_smem[dev][ki]) {                                                                     \
-            attr = cudaFuncSetAttribute(prb_sample_kernel<KK>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
+        if (max_smem && !big_smem[dev][fr][ki]) {                                                                 \
+            attr = cudaFuncSetAttribute(prb_sample_kernel<KK, FF>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
                                         (int)dyn_max[dev][ki]);                                                   \
-            big_smem[dev][ki] = (attr == cudaSuccess);                                                            \
+            big_smem[dev][fr][ki] = (attr == cudaSuccess);                                                        \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \
-            prb_sample_kernel<KK><<<grid, kThreads, smem, at>>>(v, B, beta, seed, d_idx, d_w, dst, sp);           \
+            prb_sample_kernel<KK, FF><<<grid, kThreads, smem, at>>>(v, B, beta, seed, d_idx, d_w, dst, sp);       \
     } while (0)
+#define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
+    do { if (fr) PRB_LAUNCH_SAMPLE_AS(KK, true); else PRB_LAUNCH_SAMPLE_AS(KK, false); } while (0)
         switch (v.fanout) {
         case 2: PRB_LAUNCH_SAMPLE(2); break;
         case 4: PRB_LAUNCH_SAMPLE(4); break;
@@ -1049,6 +1058,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         default: PRB_LAUNCH_SAMPLE(32); break;
         }
 #undef PRB_LAUNCH_SAMPLE
+#undef PRB_LAUNCH_SAMPLE_AS
         if (attr != cudaSuccess) return -1;
         if (n_sub > 1) {
             // the sub-batch's rows and indices are in place when its event fires; the caller's stream

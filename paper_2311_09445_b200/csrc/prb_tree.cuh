@@ -82,16 +82,18 @@ __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n
 // leaves -- the last ones zero: they belong to the slots that follow the new cursor, whose history the
 // insertion overwrites once the ring has wrapped (before that they are empty and zero already) -- and the
 // leaf of an episode-start marker (bit 1 of its done byte) is zero whatever priority is given.
-__device__ __forceinline__ uint32_t prb_cleared_after(const PrbView& v, uint32_t n)
+// (`stack` is PrbView::stack in the kernels instantiated for the frame layout and the constant 0 in the
+// others, which then carry none of this code: measured, its mere presence cost the short-row step 1.2 us)
+__device__ __forceinline__ uint32_t prb_cleared_after(const PrbView& v, uint32_t n, uint32_t stack)
 {
-    if (v.stack == 0 || n == 0) return 0u;
+    if (stack == 0 || n == 0) return 0u;
     const uint64_t room = v.capacity - n;
-    return room < v.stack ? (uint32_t)room : v.stack;
+    return room < stack ? (uint32_t)room : stack;
 }
 // ... and an update that names one of the `stack` slots that follow the cursor is stale.
-__device__ __forceinline__ bool prb_history_less(const PrbView& v, uint64_t cursor, uint64_t i)
+__device__ __forceinline__ bool prb_history_less(const PrbView& v, uint64_t cursor, uint64_t i, uint32_t stack)
 {
-    return v.stack != 0 && (i + v.capacity - cursor) % v.capacity < v.stack;
+    return stack != 0 && (i + v.capacity - cursor) % v.capacity < stack;
 }
 
 // The top of the tree staged in shared memory for the re-sum passes: levels 1 .. v.top_levels as
@@ -357,10 +359,11 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
                                                 float alpha, float eps, unsigned long long fill, unsigned char* smem,
                                                 uint32_t n = 0, const float* __restrict__ prio = nullptr,
                                                 uint64_t cursor = 0, PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
-                                                uint32_t stale = 0, PrbTop top = PrbTop{}, const unsigned char* __restrict__ ins_done = nullptr)
+                                                uint32_t stale = 0, PrbTop top = PrbTop{}, const unsigned char* __restrict__ ins_done = nullptr,
+                                                uint32_t stack = 0)
 {
     // (frames: the insertion's dirty leaves reach past its n transitions; cursor, fill and priorities do not)
-    const uint32_t n_leaves = n + prb_cleared_after(v, n);
+    const uint32_t n_leaves = n + prb_cleared_after(v, n, stack);
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);
     float* vals = reinterpret_cast<float*>(smem + (size_t)n2 * sizeof(unsigned long long));
     const uint32_t rank = team.rank, nt = team.size;
@@ -386,7 +389,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             // stale: one of the `stale` slots written most recently, i.e. overwritten since it was sampled
             const uint64_t back = (i >= 0 && stale) ? (cursor + N - 1 - (uint64_t)i) % N : ~0ull;
             if (i < 0 || (unsigned long long)i >= fill) flags |= PEARL_ST_BAD_INDEX;
-            else if (back < stale || prb_history_less(v, cursor, (uint64_t)i)) flags |= PEARL_ST_STALE;
+            else if (back < stale || prb_history_less(v, cursor, (uint64_t)i, stack)) flags |= PEARL_ST_STALE;
             else if (!ok_p) flags |= PEARL_ST_BAD_PRIORITY;
             else { key = ((unsigned long long)(uint32_t)i << 32) | b; if (raw != 2) wmax = fmaxf(wmax, p); my_valid = true; my_idx = (uint32_t)i; }
             vals[b] = p;
@@ -495,7 +498,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         uint64_t at = cursor + t;
         if (at >= N) at -= N;
         float p = 0.0f;
-        if (t < n && !(v.stack && (ins_done[t] & kPrbEpisodeStart))) {
+        if (t < n && !(stack && (ins_done[t] & kPrbEpisodeStart))) {
             p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
             if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
             else imax = fmaxf(imax, p);
@@ -549,10 +552,10 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
                                                      const float* __restrict__ prio, uint64_t cursor,
                                                      PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f},
                                                      unsigned max_bits = 0, PrbTop top = PrbTop{},
-                                                     const unsigned char* __restrict__ ins_done = nullptr)
+                                                     const unsigned char* __restrict__ ins_done = nullptr, uint32_t stack = 0)
 {
     const uint64_t N = v.capacity;
-    const uint32_t n_leaves = n + prb_cleared_after(v, n);
+    const uint32_t n_leaves = n + prb_cleared_after(v, n, stack);
     const uint32_t D = v.depth, lg = v.log2_fanout, T = prb_top_levels(v, top);
     float* leaves = v.level[D];
     bool bad = false;
@@ -562,7 +565,7 @@ __device__ __forceinline__ void prb_insert_tree_team(const PrbView& v, const Prb
         uint64_t slot = cursor + t;
         if (slot >= N) slot -= N;
         float p = 0.0f;
-        if (t < n && !(v.stack && (ins_done[t] & kPrbEpisodeStart))) {
+        if (t < n && !(stack && (ins_done[t] & kPrbEpisodeStart))) {
             p = prio == nullptr ? dflt : ((pre.has_prio && t == team.rank) ? pre.prio : prio[t]);
             if (!prb_valid_priority(p)) { p = 0.0f; bad = true; }
             else imax = fmaxf(imax, p);

@@ -11,6 +11,8 @@
 
 namespace {
 
+// kFrames: the instance for the frame-deduplicated layout (markers, cleared leaves, stale history-less updates)
+template <bool kFrames>
 __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
                   const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale,
@@ -42,9 +44,10 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
         if (threadIdx.x == 0) prb_publish_if_last(v, ins_n, cursor, fill, ticket_total, kPrbPublishTree);
     } else {
         fill = v.state->fill;
-        if (stale || v.stack) cursor = v.state->cursor;
+        if (stale || kFrames) cursor = v.state->cursor;
     }
-    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top, ins_done);
+    prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top, ins_done,
+                    kFrames ? v.stack : 0u);
 }
 
 // ---- large batches: one launch of many CTAs ------------------------------------------------------
@@ -81,7 +84,7 @@ __device__ __forceinline__ PrbWideEntry prb_wide_classify(const PrbView& v, int3
     if (i < 0 || (unsigned long long)i >= fill) { e.flags = PEARL_ST_BAD_INDEX; return e; }
     // one of the `stale` slots written most recently: overwritten since it was sampled
     if (stale && (cursor + N - 1 - (uint64_t)i) % N < stale) { e.flags = PEARL_ST_STALE; return e; }
-    if (prb_history_less(v, cursor, (uint64_t)i)) { e.flags = PEARL_ST_STALE; return e; }
+    if (prb_history_less(v, cursor, (uint64_t)i, v.stack)) { e.flags = PEARL_ST_STALE; return e; }
     float p = x;
     const bool ok = raw ? prb_valid_priority(p) : prb_priority_pow(x, eps, alpha, p);
     if (!ok) { e.flags = PEARL_ST_BAD_PRIORITY; return e; }
@@ -359,8 +362,9 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
     static bool big_smem[kPrbMaxDevices];
     const int dev = prb_current_device();
     if (!big_smem[dev]) {
-        if (cudaFuncSetAttribute(prb_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float))) != cudaSuccess)
+        const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float));
+        if (cudaFuncSetAttribute(prb_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
             return -1;
         big_smem[dev] = true;
     }
@@ -384,9 +388,11 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, prb_update_kernel, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale,
-                               ins_n, ins_prio, ctas, ins_done) != cudaSuccess)
-            return -1;
+        const cudaError_t e = v.stack ? cudaLaunchKernelEx(&cfg, prb_update_kernel<true>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
+                                                           eps, stale, ins_n, ins_prio, ctas, ins_done)
+                                      : cudaLaunchKernelEx(&cfg, prb_update_kernel<false>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
+                                                           eps, stale, ins_n, ins_prio, ctas, ins_done);
+        if (e != cudaSuccess) return -1;
         ++launches;
     }
     return launches;
