@@ -61,8 +61,10 @@ typedef struct pearl_layout {
                                       partial.  After an update of more than 1024 entries that gave up, the
                                       tree is not consistent: leaves named by the batch may hold the marker
                                       bit pattern 0x80000000|entry instead of a priority, and parents may not
-                                      equal the sum of their children.  Treat the buffer as lost: destroy it
-                                      and build a new one.  No correct run raises this bit. */
+                                      equal the sum of their children; every later update of more than 1024
+                                      entries on that buffer raises the bit again and does nothing.  Treat the
+                                      buffer as lost: destroy it and build a new one.  No correct run raises
+                                      this bit. */
 #define PEARL_ST_STALE 32u         /* update_after_insert: the index was overwritten since it was sampled; entry skipped */
 
 /* The largest update batch one thread block handles.  A batch of more than 1024 priorities or TD

@@ -33,8 +33,8 @@ struct PrbState {
     unsigned int insert_ticket;       // CTAs of the running insert kernel that have finished
     unsigned int sample_ticket;       // CTAs of the running sample kernel that have finished
     unsigned int max_prio_bits;       // bits of the largest priority written so far (0: none yet)
-    unsigned int wide_arrived;        // grid barrier of the running many-CTA update: arrivals so far (cleared on the stream before each launch)
-    unsigned int wide_spare;
+    unsigned int wide_arrived;        // grid barrier of the running many-CTA update: arrivals so far (0 between launches that ended well)
+    unsigned int wide_done;           // its CTAs that have passed their last barrier
     unsigned long long wide_wmax_bits; // largest raw weight of the running large-batch sample (bits of a binary64; 0 between calls)
     // The ring cursor as the kernels that copy rows see it.  An insertion whose tree work and row copy are
     // two kernels on two streams advances `cursor` (and `fill`) from the tree kernel and `row_cursor` from
@@ -42,7 +42,8 @@ struct PrbState {
     // races with, the other's; a one-kernel insertion advances both.  Equal whenever no insertion is running.
     unsigned long long row_cursor;
     unsigned int row_ticket;          // CTAs of the running row kernel that have read row_cursor
-    unsigned int spare;
+    unsigned int wide_poisoned;       // a many-CTA update gave up at its barrier once: the barrier's state is not to be trusted, and
+                                      // neither is the tree; every later many-CTA update raises INTERNAL and does nothing
 };
 
 // Geometry and device addresses, passed to kernels by value.

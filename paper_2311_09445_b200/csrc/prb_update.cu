@@ -198,8 +198,14 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
     const uint64_t cursor = (stale || v.stack) ? v.state->cursor : 0ull;
     const uint32_t K = v.fanout, lg = v.log2_fanout, D = v.depth, T = v.top_levels;
     unsigned* leaf_bits = reinterpret_cast<unsigned*>(v.level[D]);
-    if (tid == 0) { s_flags = 0u; s_maxbits = 0u; }
+    if (tid == 0) { s_flags = 0u; s_maxbits = 0u; s_ok = (__ldcg(&v.state->wide_poisoned) == 0u) ? 1 : 0; }
     __syncthreads();
+    if (!s_ok) {
+        // an earlier launch of this kernel gave up at its barrier and left the counter (and the tree) in
+        // no known state: no launch after it pretends otherwise
+        if (tid == 0 && blockIdx.x == 0) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
+        return;
+    }
 
     // 1. validate, transform, name the last writer of every leaf (a thread's first entry stays in registers)
     PrbWideEntry first = PrbWideEntry{false, 0u, 0.0f, 0u};
@@ -264,10 +270,14 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         l -= (int)h;
     }
     if (!alive) {
-        // (the barrier's counter is cleared on the stream before every launch: a launch that gave up
-        // leaves nothing behind that the next one would trip over)
-        if (tid == 0) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
+        // (the barrier's counter is left as it is, and marked: see wide_poisoned)
+        if (tid == 0) { atomicOr(&v.state->status, PEARL_ST_INTERNAL); atomicExch(&v.state->wide_poisoned, 1u); }
         return;
+    }
+    // every CTA is past its last barrier: the last one to say so clears the barrier for the next launch
+    if (tid == 0 && atomicAdd(&v.state->wide_done, 1u) == nctas - 1) {
+        v.state->wide_arrived = 0u;
+        v.state->wide_done = 0u;
     }
     // 4. the staged levels
     if (blockIdx.x == 0 && T > 0) {
@@ -342,8 +352,6 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    // the grid barrier counts arrivals from zero: cleared here, on the stream, not by the launch before
-    if (cudaMemsetAsync(&v.state->wide_arrived, 0, sizeof(unsigned int), s) != cudaSuccess) return -1;
     if (cudaLaunchKernelEx(&cfg, prb_update_wide_kernel, v, B, d_idx, d_val, raw, alpha, eps, stale) != cudaSuccess) return -1;
     return 1;
 }
