@@ -38,6 +38,7 @@ struct Layout {
     uint64_t off_stage_out_idx, off_stage_out_w;
     uint32_t field_bytes[PRB_NUM_FIELDS];     // a row of the store
     uint32_t out_bytes[PRB_NUM_FIELDS];       // a row as a sample hands it out
+    uint32_t field_pitch[PRB_NUM_FIELDS];     // bytes from one slot's field to the next slot's (see PrbView)
     uint32_t stack;                           // frame-deduplicated layout: frames per observation (0: plain layout)
     uint64_t total;
 };
@@ -85,7 +86,31 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     L->off_wraw = at; at = align_up(at + (uint64_t)max_batch * sizeof(double));
     for (uint32_t j = 0; j < kPrbHandoffs; ++j) { L->off_handoff[j] = at; at = align_up(at + prb_handoff_bytes(max_batch)); }
     L->off_zero_end = at;
-    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_store[f] = at; at = align_up(at + capacity * L->field_bytes[f]); }
+    // Short rows (every field below the bulk-copy threshold, the record at most 512 bytes, no frames): one
+    // padded record per transition, fields at offsets aligned to their copy granules, the record a multiple
+    // of 64 bytes.  Otherwise one array per field.
+    uint64_t record = 0;
+    bool records = stack == 0;
+    uint64_t field_off[PRB_NUM_FIELDS];
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        const uint32_t g = L->field_bytes[f] ? granule_of(L->field_bytes[f]) : 1;
+        if (g == 16 && L->field_bytes[f] / g >= 512) records = false;
+        record = (record + g - 1) / g * g;
+        field_off[f] = record;
+        record += L->field_bytes[f];
+    }
+    record = (record + 63) / 64 * 64;
+    if (record > 512) records = false;
+    if (records) {
+        for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_store[f] = at + field_off[f]; L->field_pitch[f] = (uint32_t)record; }
+        at = align_up(at + capacity * record);
+    } else {
+        for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+            L->off_store[f] = at;
+            L->field_pitch[f] = L->field_bytes[f];
+            at = align_up(at + capacity * L->field_bytes[f]);
+        }
+    }
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) { L->off_stage_in[f] = at; at = align_up(at + (uint64_t)max_batch * L->field_bytes[f]); }
     L->off_stage_prio = at; at = align_up(at + (uint64_t)max_batch * 4);
     L->off_stage_idx = at; at = align_up(at + (uint64_t)max_batch * 4);
@@ -353,6 +378,7 @@ static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, 
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         v.store[f] = at(h, L.off_store[f]);
         v.field_bytes[f] = L.field_bytes[f];
+        v.field_pitch[f] = L.field_pitch[f];
         v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
     }
     v.stack = L.stack;
@@ -930,7 +956,7 @@ int pearl_prb_read_rows(pearl_prb_t* h, const int32_t* h_idx, uint32_t n, void* 
         const uint64_t fb = h->view.field_bytes[f];
         if (!dst[f] || fb == 0 || (S && f == F_OBS)) continue;
         for (uint32_t k = 0; k < n; ++k) {
-            if (cudaMemcpyAsync((unsigned char*)dst[f] + k * fb, h->view.store[f] + (uint64_t)h_idx[k] * fb, fb,
+            if (cudaMemcpyAsync((unsigned char*)dst[f] + k * fb, h->view.store[f] + (uint64_t)h_idx[k] * h->view.field_pitch[f], fb,
                                 cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
                 return PEARL_ERR_CUDA;
         }

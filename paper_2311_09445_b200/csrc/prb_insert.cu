@@ -47,7 +47,7 @@ template <typename T>
 __device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const PrbBatch& src, uint32_t n, uint64_t cursor,
                                                uint32_t tile, uint32_t rank, uint32_t nthreads)
 {
-    const uint32_t W = v.field_bytes[f] / sizeof(T);
+    const uint32_t W = v.field_bytes[f] / sizeof(T), Wp = v.field_pitch[f] / sizeof(T);     // granules per row, per slot of the store
     const uint64_t N = v.capacity;
     const uint64_t total = (uint64_t)n * W;
     const uint64_t e0 = (uint64_t)tile * kTile;
@@ -59,7 +59,7 @@ __device__ __forceinline__ void copy_flat_tile(const PrbView& v, int f, const Pr
                            uint64_t slot = cursor + r;
                            if (slot >= N) slot -= N;
                            if (!PRB_IN_BOUNDS(v, slot < N && r < n)) slot = 0;
-                           return slot * W + (e - r * W);
+                           return slot * Wp + (e - r * W);
                        },
                        rank, nthreads);
 }

@@ -68,6 +68,11 @@ struct PrbView {
     uint32_t stack;
     uint32_t field_bytes[PRB_NUM_FIELDS];
     uint32_t field_vec[PRB_NUM_FIELDS];   // copy granule in bytes: largest power of two <= 16 dividing field_bytes
+    // Bytes from slot i to slot i + 1 of field f in the store.  Long rows are stored field by field
+    // (pitch = field_bytes).  When every field is short the store is ONE padded record per transition
+    // (pitch = the record's size, a multiple of 64 bytes; store[f] points at field f of record 0), so that a
+    // sampled transition is a few consecutive sectors instead of a sector or three per field.
+    uint32_t field_pitch[PRB_NUM_FIELDS];
     unsigned char* store[PRB_NUM_FIELDS];
     double* wraw;                     // scratch: raw IS weights of the running sample call, max_batch entries
     // A sample of long rows that is issued as two kernels (descents, then the row copy) hands indices

@@ -216,21 +216,21 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (stack && f == F_OBS)) continue;
-        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, Wp = v.field_pitch[f] / vec, total = n_rows * W;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const uint32_t e = rank + u * nthreads;
             if (e < total) {
                 const uint32_t r = (W == 1) ? e : e / W;
                 if (PRB_IN_BOUNDS(v, s_idx[r] < v.capacity))
-                    tmp[f][u] = load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec);
+                    tmp[f][u] = load_granule(v.store[f], (uint64_t)s_idx[r] * Wp + (e - r * W), vec);
             }
         }
     }
 #pragma unroll
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0 || plan.chunks[f] != 0 || (stack && f == F_OBS)) continue;
-        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, Wp = v.field_pitch[f] / vec, total = n_rows * W;
         const uint64_t dbase = (uint64_t)k_first * W;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -240,7 +240,7 @@ __device__ __forceinline__ void gather_short_fields(const PrbView& v, const Samp
         for (uint32_t e = rank + 2 * nthreads; e < total; e += nthreads) {     // the rest of a larger batch
             const uint32_t r = e / W;
             if (PRB_IN_BOUNDS(v, s_idx[r] < v.capacity))
-                store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * W + (e - r * W), vec));
+                store_granule(dst.ptr[f], dbase + e, vec, load_granule(v.store[f], (uint64_t)s_idx[r] * Wp + (e - r * W), vec));
         }
     }
 }
@@ -492,7 +492,7 @@ constexpr uint32_t kWideSampleStrata = 32;      // ... spread over CTAs of at le
 // Short rows of strata [k_first, k_first + n_rows) by all `nthreads` threads, field by field, in
 // granules of type T: up to U granules per thread are loaded before the first is stored.
 template <typename T, int U>
-__device__ __forceinline__ void gather_field_deep(const T* __restrict__ store, T* __restrict__ out, uint32_t W, uint32_t total,
+__device__ __forceinline__ void gather_field_deep(const T* __restrict__ store, T* __restrict__ out, uint32_t W, uint32_t Wp, uint32_t total,
                                                   const uint32_t* s_idx, uint32_t rank, uint32_t nthreads)
 {
     for (uint32_t e0 = rank; e0 < total; e0 += nthreads * U) {
@@ -502,7 +502,7 @@ __device__ __forceinline__ void gather_field_deep(const T* __restrict__ store, T
             const uint32_t e = e0 + u * nthreads;
             if (e < total) {
                 const uint32_t r = (W == 1) ? e : e / W;
-                tmp[u] = store[(uint64_t)s_idx[r] * W + (e - r * W)];      // (s_idx comes from a descent, checked there)
+                tmp[u] = store[(uint64_t)s_idx[r] * Wp + (e - r * W)];     // (s_idx comes from a descent, checked there; Wp: granules per slot)
             }
         }
 #pragma unroll
@@ -518,15 +518,15 @@ __device__ __forceinline__ void gather_short_fields_deep(const PrbView& v, const
 {
     for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
         if (dst.ptr[f] == nullptr || v.field_bytes[f] == 0) continue;
-        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, total = n_rows * W;
+        const uint32_t vec = v.field_vec[f], W = v.field_bytes[f] / vec, Wp = v.field_pitch[f] / vec, total = n_rows * W;
         const unsigned char* src = v.store[f];
         unsigned char* out = dst.ptr[f] + (uint64_t)k_first * v.field_bytes[f];
         switch (vec) {
-        case 16: gather_field_deep<uint4, 4>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(out), W, total, s_idx, rank, nthreads); break;
-        case 8: gather_field_deep<uint2, 8>(reinterpret_cast<const uint2*>(src), reinterpret_cast<uint2*>(out), W, total, s_idx, rank, nthreads); break;
-        case 4: gather_field_deep<uint32_t, 16>(reinterpret_cast<const uint32_t*>(src), reinterpret_cast<uint32_t*>(out), W, total, s_idx, rank, nthreads); break;
-        case 2: gather_field_deep<uint16_t, 8>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(out), W, total, s_idx, rank, nthreads); break;
-        default: gather_field_deep<unsigned char, 8>(src, out, W, total, s_idx, rank, nthreads); break;
+        case 16: gather_field_deep<uint4, 4>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(out), W, Wp, total, s_idx, rank, nthreads); break;
+        case 8: gather_field_deep<uint2, 8>(reinterpret_cast<const uint2*>(src), reinterpret_cast<uint2*>(out), W, Wp, total, s_idx, rank, nthreads); break;
+        case 4: gather_field_deep<uint32_t, 16>(reinterpret_cast<const uint32_t*>(src), reinterpret_cast<uint32_t*>(out), W, Wp, total, s_idx, rank, nthreads); break;
+        case 2: gather_field_deep<uint16_t, 8>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(out), W, Wp, total, s_idx, rank, nthreads); break;
+        default: gather_field_deep<unsigned char, 8>(src, out, W, Wp, total, s_idx, rank, nthreads); break;
         }
     }
 }
