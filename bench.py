@@ -281,7 +281,8 @@ def timed_regions(stream, run_steps, steps, world, dev):
     return times
 
 
-def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=True, e2e=True, use_graph=True, fused=True):
+def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=True, e2e=True, use_graph=True, fused=True,
+                     min_tree=False):
     """Builds and fills one buffer for workload `wl` and times the step, its calls and the host-buffer step.
     Returns a dict of raw measurements (milliseconds per step / per call)."""
     import torch
@@ -295,7 +296,7 @@ def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=Tru
     m = {}
     with torch.cuda.stream(stream):
         prb = PrioritizedReplay(wl.capacity, wl.fanout, wl.obs_bytes, wl.act_bytes, max_batch, device=dev, stream=stream,
-                                frame_stack=wl.frame_stack)
+                                frame_stack=wl.frame_stack, min_tree=min_tree)
         # prefill the whole ring through the insert call
         filled = 0
         while filled < wl.capacity:
@@ -499,7 +500,7 @@ def run_ours(args, wl, rank, world):
     B, n_ins = wl.batch, wl.n_insert
     fused = bool(n_ins) and not args.unfused
     m = measure_workload(wl, args.steps, args.warmup, dev, stream, rank, world, extras=not args.profile,
-                         e2e=not args.profile, use_graph=not args.no_graph, fused=fused)
+                         e2e=not args.profile, use_graph=not args.no_graph, fused=fused, min_tree=args.min_tree)
     m["steps"] = args.steps
     ctx = None
     others = None
@@ -534,7 +535,7 @@ def run_ours(args, wl, rank, world):
         "vs_baseline": None, "dtype": "f32 tree / f64 targets / u8 rows", "data": "synthetic",
         "config": {"workload": wl.name, "capacity": wl.capacity, "fanout": wl.fanout, "depth": depth, "batch": B,
                    "insert_per_step": n_ins, "transition_bytes": E, "step": "sample(idx,IS,gather) + update_insert" if fused else "sample(idx,IS,gather) + update + insert",
-                   "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph,
+                   "parallelism": "replicas x%d" % world, "cuda_graph": not args.no_graph, "min_tree": bool(args.min_tree),
                    "l2": "inputs/outputs rotate over %d buffers (%d MB per step touched)" % (ROTATE, (2 * (n_ins + B) * E) >> 20)},
         "timed_region": {"repeats": len(m["region_ms"]), "ms_each": m["region_ms"],
                          "value_from": "median" if len(m["region_ms"]) > 1 else "the one region"},
@@ -761,6 +762,8 @@ def main():
     ap.add_argument("--workload", default="atari_dqn")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--unfused", action="store_true", help="update and insert as two launches instead of pearl_prb_update_insert")
+    ap.add_argument("--min-tree", action="store_true",
+                    help="the buffer keeps a min-tree (PEARL_OPT_MIN_TREE): rates.us_sample_buffer_norm then has no scan of the leaves")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU-oracle work for cpu_baseline")
     ap.add_argument("--sweep", action="store_true",
                     help="time every cell of the capacity x fanout x batch sweep instead (one GPU)")

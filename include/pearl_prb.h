@@ -127,6 +127,25 @@ int pearl_prb_create_frames(pearl_prb_t** out, uint64_t capacity, uint32_t fanou
                             uint32_t stack, uint32_t act_bytes, uint32_t max_batch, int device, void* cuda_stream,
                             void* slab, uint64_t slab_bytes);
 
+/* Creation with options.  frame_stack = 0 gives pearl_prb_create's layout; frame_stack >= 1 that of
+ * pearl_prb_create_frames (layout->obs_bytes is then the size of one frame).  `options` is a sum of PEARL_OPT_*
+ * bits (unknown bits: PEARL_ERR_BAD_ARG; pearl_prb_slab_bytes_opts returns 0).
+ *   PEARL_OPT_MIN_TREE  the buffer keeps, beside the sum tree, a min-tree of the same shape (Section V-A
+ *       describes the sum tree only; a min-tree is what prioritized-replay implementations use for the
+ *       weight normalisation of Schaul et al., Algorithm 1): node (l, a), l < depth, holds the smallest
+ *       positive leaf below it, 0 if there is none; the leaves serve both trees.  Every call that writes
+ *       the sum tree re-derives the min-tree's nodes above the written leaves in the same passes (the
+ *       min-tree costs one more array of the size of the inner levels, and an update or insertion about
+ *       one more read per level).  pearl_prb_sample_buffer_norm then reads the minimum at the root
+ *       instead of scanning the leaves; its results are the same either way (the minimum of a set does
+ *       not depend on the order it is taken in). */
+#define PEARL_OPT_MIN_TREE 1u
+uint64_t pearl_prb_slab_bytes_opts(uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
+                                   uint32_t frame_stack, uint32_t options, uint32_t max_batch);
+int pearl_prb_create_opts(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
+                          uint32_t frame_stack, uint32_t options, uint32_t max_batch, int device,
+                          void* cuda_stream, void* slab, uint64_t slab_bytes);
+
 /* Synchronises the handle's streams, frees library-owned memory, streams, events and the handle. */
 int pearl_prb_destroy(pearl_prb_t* prb);
 
@@ -240,7 +259,8 @@ int pearl_prb_step(pearl_prb_t* prb, uint32_t B_upd, const int32_t* d_upd_idx, c
 /* pearl_prb_sample with the weights normalised as in the prioritized-replay paper the toolkit
  * follows (Schaul et al., Algorithm 1: w_j = (N P(j))^-beta / max_i w_i, the maximum over the whole
  * memory): the divisor is the weight of the smallest positive priority stored,
- * (N p_min / total)^-beta, found by a scan of the leaves in a launch of its own before the sample.
+ * (N p_min / total)^-beta, found by a scan of the leaves in a launch of its own before the sample
+ * -- or, in a buffer created with PEARL_OPT_MIN_TREE, read from the root of its min-tree.
  * Weights are then at most 1 and do not depend on which other transitions the batch holds.  PEARL
  * itself does not say how the weights are normalised.  Everything else as pearl_prb_sample. */
 int pearl_prb_sample_buffer_norm(pearl_prb_t* prb, uint32_t B, float beta, uint64_t seed, int32_t* d_idx,
@@ -335,6 +355,8 @@ int pearl_prb_info(pearl_prb_t* prb, uint64_t* fill, uint64_t* cursor, uint64_t*
 int pearl_prb_max_priority(pearl_prb_t* prb, float* h_out);
 /* Copies the first `count` entries (padding included) of tree level `level` (0 = root). */
 int pearl_prb_read_level(pearl_prb_t* prb, uint32_t level, float* h_dst, uint64_t count);
+/* The same for level `level` < depth of the min-tree (PEARL_ERR_BAD_ARG without PEARL_OPT_MIN_TREE). */
+int pearl_prb_read_min_level(pearl_prb_t* prb, uint32_t level, float* h_dst, uint64_t count);
 /* Number of entries of a level including its zero padding; 0 for an invalid level. */
 uint64_t pearl_prb_level_alloc(pearl_prb_t* prb, uint32_t level);
 /* Copies stored rows h_idx[0..n) (slot numbers < capacity) to host arrays. */

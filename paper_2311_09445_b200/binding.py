@@ -37,6 +37,8 @@ SIGNATURES = {
     "pearl_prb_create": (_i, [C.POINTER(_vp), _u64, _u32, C.POINTER(_Layout), _u32, _i, _vp, _vp, _u64]),
     "pearl_prb_slab_bytes_frames": (_u64, [_u64, _u32, _u32, _u32, _u32, _u32]),
     "pearl_prb_create_frames": (_i, [C.POINTER(_vp), _u64, _u32, _u32, _u32, _u32, _u32, _i, _vp, _vp, _u64]),
+    "pearl_prb_slab_bytes_opts": (_u64, [_u64, _u32, C.POINTER(_Layout), _u32, _u32, _u32]),
+    "pearl_prb_create_opts": (_i, [C.POINTER(_vp), _u64, _u32, C.POINTER(_Layout), _u32, _u32, _u32, _i, _vp, _vp, _u64]),
     "pearl_prb_destroy": (_i, [_vp]),
     "pearl_prb_insert": (_i, [_vp, _u32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_sample": (_i, [_vp, _u32, _f32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -62,6 +64,7 @@ SIGNATURES = {
     "pearl_prb_info": (_i, [_vp, C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u64), C.POINTER(_u32)]),
     "pearl_prb_max_priority": (_i, [_vp, C.POINTER(_f32)]),
     "pearl_prb_read_level": (_i, [_vp, _u32, _vp, _u64]),
+    "pearl_prb_read_min_level": (_i, [_vp, _u32, _vp, _u64]),
     "pearl_prb_level_alloc": (_u64, [_vp, _u32]),
     "pearl_prb_read_rows": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_kernel_launches": (_u64, [_vp]),
@@ -122,7 +125,8 @@ class PrioritizedReplay:
     """
 
     def __init__(self, capacity: int, fanout: int, obs_bytes: int, act_bytes: int, max_batch: int,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None, frame_stack: int = 0):
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None, frame_stack: int = 0,
+                 min_tree: bool = False):
         self._h = None
         lib = load_library()
         if not torch.cuda.is_available():
@@ -132,10 +136,14 @@ class PrioritizedReplay:
         self.capacity, self.fanout, self.max_batch = capacity, fanout, max_batch
         self.obs_bytes, self.act_bytes = obs_bytes, act_bytes
         self.frame_stack = frame_stack          # > 0: pearl_prb_create_frames; obs_bytes is then a whole stack
+        self.min_tree = bool(min_tree)          # PEARL_OPT_MIN_TREE (pearl_prb_create_opts)
         lay = _Layout(obs_bytes, act_bytes)
-        if frame_stack:
-            if obs_bytes % frame_stack:
-                raise ValueError("obs_bytes must be frame_stack frames")
+        if frame_stack and obs_bytes % frame_stack:
+            raise ValueError("obs_bytes must be frame_stack frames")
+        if min_tree:
+            lay = _Layout(obs_bytes // frame_stack if frame_stack else obs_bytes, act_bytes)
+            need = lib.pearl_prb_slab_bytes_opts(capacity, fanout, C.byref(lay), frame_stack, 1, max_batch)
+        elif frame_stack:
             need = lib.pearl_prb_slab_bytes_frames(capacity, fanout, obs_bytes // frame_stack, frame_stack, act_bytes, max_batch)
         else:
             need = lib.pearl_prb_slab_bytes(capacity, fanout, C.byref(lay), max_batch)
@@ -144,7 +152,11 @@ class PrioritizedReplay:
         self.slab_bytes = int(need)
         self._slab = torch.empty(self.slab_bytes, dtype=torch.uint8, device=self.device)
         h = C.c_void_p()
-        if frame_stack:
+        if min_tree:
+            rc = lib.pearl_prb_create_opts(C.byref(h), capacity, fanout, C.byref(lay), frame_stack, 1, max_batch,
+                                           self.device.index or 0, C.c_void_p(self.stream.cuda_stream),
+                                           C.c_void_p(self._slab.data_ptr()), self.slab_bytes)
+        elif frame_stack:
             rc = lib.pearl_prb_create_frames(C.byref(h), capacity, fanout, obs_bytes // frame_stack, frame_stack, act_bytes, max_batch,
                                              self.device.index or 0, C.c_void_p(self.stream.cuda_stream),
                                              C.c_void_p(self._slab.data_ptr()), self.slab_bytes)
@@ -332,6 +344,15 @@ class PrioritizedReplay:
         rc = load_library().pearl_prb_read_level(self._h, level, C.c_void_p(out.ctypes.data), n)
         if rc != 0:
             raise PearlError(rc, "pearl_prb_read_level")
+        return out
+
+    def read_min_level(self, level: int):
+        import numpy as np
+        n = self.level_alloc(level)
+        out = np.zeros(n, dtype=np.float32)
+        rc = load_library().pearl_prb_read_min_level(self._h, level, C.c_void_p(out.ctypes.data), n)
+        if rc != 0:
+            raise PearlError(rc, "pearl_prb_read_min_level")
         return out
 
     def read_rows(self, idx):

@@ -28,6 +28,7 @@ struct Layout {
     uint64_t level_alloc[PRB_MAX_LEVELS];
     uint64_t off_state;
     uint64_t off_level[PRB_MAX_LEVELS];
+    uint64_t off_min;                         // the min-tree's levels 0 .. depth-1, laid out like the sum tree's (0: no min-tree)
     uint64_t off_wraw;
     uint64_t off_handoff[kPrbHandoffs];
     uint64_t off_zero_end;                    // [0, off_zero_end) is zeroed at creation
@@ -45,8 +46,10 @@ struct Layout {
 
 bool valid_fanout(uint32_t k) { return k == 2 || k == 4 || k == 8 || k == 16 || k == 32; }
 
-bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, uint32_t max_batch, Layout* L, uint32_t stack = 0)
+bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, uint32_t max_batch, Layout* L, uint32_t stack = 0,
+                 uint32_t options = 0)
 {
+    if (options & ~PEARL_OPT_MIN_TREE) return false;
     if (!lay || !valid_fanout(fanout) || capacity < 1 || capacity > (1ull << 30) || max_batch < 1 ||
         max_batch > (1u << 20))
         return false;
@@ -83,6 +86,8 @@ bool make_layout(uint64_t capacity, uint32_t fanout, const pearl_layout_t* lay, 
     uint64_t at = 0;
     L->off_state = at; at = align_up(at + sizeof(PrbState));
     for (uint32_t l = 0; l <= D; ++l) { L->off_level[l] = at; at = align_up(at + L->level_alloc[l] * sizeof(float)); }
+    L->off_min = 0;
+    if (options & PEARL_OPT_MIN_TREE) { L->off_min = at; at = align_up(at + (L->off_level[D] - L->off_level[0])); }
     L->off_wraw = at; at = align_up(at + (uint64_t)max_batch * sizeof(double));
     for (uint32_t j = 0; j < kPrbHandoffs; ++j) { L->off_handoff[j] = at; at = align_up(at + prb_handoff_bytes(max_batch)); }
     L->off_zero_end = at;
@@ -288,8 +293,22 @@ uint64_t pearl_prb_slab_bytes_frames(uint64_t capacity, uint32_t fanout, uint32_
     return L.total;
 }
 
+uint64_t pearl_prb_slab_bytes_opts(uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t frame_stack,
+                                   uint32_t options, uint32_t max_batch)
+{
+    Layout L;
+    if (!make_layout(capacity, fanout, layout, max_batch, &L, frame_stack, options)) return 0;
+    return L.total;
+}
+
 static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t stack,
-                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes);
+                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes, uint32_t options = 0);
+
+int pearl_prb_create_opts(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t frame_stack,
+                          uint32_t options, uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
+{
+    return create_common(out, capacity, fanout, layout, frame_stack, max_batch, device, cuda_stream, slab, slab_bytes, options);
+}
 
 int pearl_prb_create(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout,
                      uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
@@ -306,13 +325,13 @@ int pearl_prb_create_frames(pearl_prb_t** out, uint64_t capacity, uint32_t fanou
 }
 
 static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, const pearl_layout_t* layout, uint32_t stack,
-                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes)
+                         uint32_t max_batch, int device, void* cuda_stream, void* slab, uint64_t slab_bytes, uint32_t options)
 {
     if (!out || !layout) return PEARL_ERR_NULL;
     if (!valid_fanout(fanout)) return PEARL_ERR_BAD_FANOUT;
     if (max_batch < 1 || max_batch > (1u << 20)) return PEARL_ERR_BAD_BATCH;
     Layout L;
-    if (!make_layout(capacity, fanout, layout, max_batch, &L, stack)) return PEARL_ERR_BAD_ARG;
+    if (!make_layout(capacity, fanout, layout, max_batch, &L, stack, options)) return PEARL_ERR_BAD_ARG;
     DeviceGuard guard(device);
     if (!guard.ok) return PEARL_ERR_CUDA;
 
@@ -381,6 +400,7 @@ static int create_common(pearl_prb_t** out, uint64_t capacity, uint32_t fanout, 
         v.field_pitch[f] = L.field_pitch[f];
         v.field_vec[f] = L.field_bytes[f] ? granule_of(L.field_bytes[f]) : 1;
     }
+    v.min_off = L.off_min ? (L.off_min - L.off_level[0]) / sizeof(float) : 0;
     v.stack = L.stack;
     if (v.stack) v.field_vec[F_NEXT_OBS] = v.field_vec[F_OBS];      // rebuilt from the same frames
     v.wraw = (double*)at(h, L.off_wraw);
@@ -938,6 +958,17 @@ int pearl_prb_read_level(pearl_prb_t* h, uint32_t level, float* h_dst, uint64_t 
     DeviceGuard guard(h->device);
     if (!guard.ok) return PEARL_ERR_CUDA;
     if (cudaMemcpyAsync(h_dst, h->view.level[level], count * sizeof(float), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+        return PEARL_ERR_CUDA;
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+int pearl_prb_read_min_level(pearl_prb_t* h, uint32_t level, float* h_dst, uint64_t count)
+{
+    if (!h || !h_dst) return PEARL_ERR_NULL;
+    if (h->view.min_off == 0 || level >= h->view.depth || count > h->lay.level_alloc[level]) return PEARL_ERR_BAD_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    if (cudaMemcpyAsync(h_dst, h->view.level[level] + h->view.min_off, count * sizeof(float), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
         return PEARL_ERR_CUDA;
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }

@@ -90,7 +90,7 @@ struct FusedUpdate {
 
 // Short rows only: CTA 0 = tree (after the optional update), CTAs 1.. = a contiguous range of tiles
 // each.  Threads 0..kWorkers-1 work; thread kWorkers reads the cursor for the CTA and takes the ticket.
-template <bool kFrames>
+template <bool kFrames, bool kMin>
 __global__ void __launch_bounds__(kThreadsShort, 2)
 prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
                   const float* __restrict__ prio, const __grid_constant__ InsertPlan plan,
@@ -109,6 +109,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
         if (tid < upd.B) { pre.has_update = true; pre.idx = upd.idx[tid]; pre.val = upd.val[tid]; }
         if (tid < n && prio != nullptr) { pre.has_prio = true; pre.prio = prio[tid]; }
         if (v.top_levels) top.mem = reinterpret_cast<float*>(s_dyn + (upd.B ? prb_update_smem_bytes(upd.n2) : 0));
+        if (kMin && v.top_levels) top.mem_min = top.mem + v.top_floats;
         prb_top_begin(v, top, tid, kWorkers);
     }
     __syncthreads();
@@ -119,6 +120,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
         if (blockIdx.x == 0) {
             PrbTeam team;
             team.rank = tid; team.size = kWorkers; team.whole_cta = false;
+            if (kMin) team.min_off = v.min_off;
             if (upd.B)      // update and insertion share one re-sum pass per level
                 prb_update_team(v, team, upd.B, upd.n2, upd.idx, upd.val, upd.raw, upd.alpha, upd.eps, s_fill, s_dyn, n, prio, cursor, pre, 0, top,
                                 src.ptr[F_DONE], kFrames ? v.stack : 0u);
@@ -139,7 +141,7 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
 // not depend on it).  Threads 32..32+kWorkers-1: the tree work (CTA 0, unless a tree kernel beside
 // this one does it) and the short-field tiles (dealt round-robin, CTA 1 first).  Thread
 // 32+kWorkers: cursor and ticket.
-template <bool kFrames>
+template <bool kFrames, bool kMin>
 __global__ void __launch_bounds__(kThreadsRows, 1)
 prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_constant__ PrbBatch src,
                        const float* __restrict__ prio, const __grid_constant__ InsertPlan plan)
@@ -205,6 +207,7 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
     } else if (tid >= 32 && tid < kPublisher) {
         PrbTeam team;
         team.rank = tid - 32u; team.size = kWorkers; team.whole_cta = false;
+        if (kMin) team.min_off = v.min_off;
         if (blockIdx.x == 0 && plan.tree_ctas == 0)
             prb_insert_tree_team(v, team, n, prio, cursor, PrbPreloaded{false, false, 0, 0.0f, 0.0f}, s_maxp, PrbTop{}, src.ptr[F_DONE],
                                  kFrames ? v.stack : 0u);
@@ -295,30 +298,35 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     if (tasks == 0) {
         static bool big_smem[kPrbMaxDevices];
         if (!big_smem[dev]) {
-            const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float));
-            if (cudaFuncSetAttribute(prb_insert_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-                cudaFuncSetAttribute(prb_insert_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
-                return -1;
+            const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + 2 * kPrbTopFloats * sizeof(float));
+            bool ok = true;
+#define PRB_ALLOW_SMEM(FF, MM) ok = ok && cudaFuncSetAttribute(prb_insert_kernel<FF, MM>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) == cudaSuccess
+            PRB_ALLOW_SMEM(false, false); PRB_ALLOW_SMEM(true, false); PRB_ALLOW_SMEM(false, true); PRB_ALLOW_SMEM(true, true);
+#undef PRB_ALLOW_SMEM
+            if (!ok) return -1;
             big_smem[dev] = true;
         }
         const uint32_t one_wave = (uint32_t)sm_count * 2 - 1;     // CTA 0 is the tree CTA
         const uint32_t copy_ctas = tiles < one_wave ? tiles : one_wave;
-        const uint32_t smem = upd_smem + v.top_floats * (uint32_t)sizeof(float);
-        if (v.stack) prb_insert_kernel<true><<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, n, src, d_prio, plan, upd);
-        else prb_insert_kernel<false><<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, n, src, d_prio, plan, upd);
+        const uint32_t smem = upd_smem + v.top_floats * (uint32_t)sizeof(float) * (v.min_off ? 2u : 1u);
+#define PRB_LAUNCH_INSERT_AS(FF, MM) prb_insert_kernel<FF, MM><<<copy_ctas + 1, kThreadsShort, smem, s>>>(v, n, src, d_prio, plan, upd)
+        PRB_WITH_TREE_OPTIONS(v, PRB_LAUNCH_INSERT_AS);
+#undef PRB_LAUNCH_INSERT_AS
     } else {
         const uint32_t smem = kRingBarBytes + plan.ring_stages * plan.ring_stage_bytes;
         static bool big_rows[kPrbMaxDevices];
         if (!big_rows[dev]) {
-            if (cudaFuncSetAttribute(prb_insert_rows_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(kRingBarBytes + kRingBytes)) != cudaSuccess ||
-                cudaFuncSetAttribute(prb_insert_rows_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(kRingBarBytes + kRingBytes)) != cudaSuccess)
-                return -1;
+            bool ok = true;
+#define PRB_ALLOW_SMEM(FF, MM) \
+    ok = ok && cudaFuncSetAttribute(prb_insert_rows_kernel<FF, MM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kRingBarBytes + kRingBytes)) == cudaSuccess
+            PRB_ALLOW_SMEM(false, false); PRB_ALLOW_SMEM(true, false); PRB_ALLOW_SMEM(false, true); PRB_ALLOW_SMEM(true, true);
+#undef PRB_ALLOW_SMEM
+            if (!ok) return -1;
             big_rows[dev] = true;
         }
-        if (v.stack) prb_insert_rows_kernel<true><<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
-        else prb_insert_rows_kernel<false><<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan);
+#define PRB_LAUNCH_ROWS_AS(FF, MM) prb_insert_rows_kernel<FF, MM><<<rows_grid, kThreadsRows, smem, s>>>(v, n, src, d_prio, plan)
+        PRB_WITH_TREE_OPTIONS(v, PRB_LAUNCH_ROWS_AS);
+#undef PRB_LAUNCH_ROWS_AS
         if (forked && cudaStreamWaitEvent(s, fork->join, 0) != cudaSuccess) return -1;
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -79,6 +79,11 @@ struct PrbView {
     // and leaf priorities from the first to the second through one of a few areas of the slab, used in turn:
     // a 256-byte header (PrbHandoffHeader), max_batch indices, max_batch priorities.
     unsigned char* handoff[kPrbHandoffs];
+    // Min-tree (optional, PEARL_LAYOUT_MIN_TREE): node (l, a), l < depth, of a second tree holds the smallest
+    // positive leaf below it (0: none); it lies min_off entries behind the sum tree's node, level[l] + min_off
+    // (the leaves serve both trees).  0: no min-tree.  Its root is what weights normalised over the whole
+    // buffer divide by, without a scan of the leaves.
+    uint64_t min_off;
     float* level[PRB_MAX_LEVELS];     // level[l] holds K * n_{l-1} entries (level[0]: 1)
     uint32_t level_alloc[PRB_MAX_LEVELS];   // entries of level l, zero padding included
     uint32_t top_off[PRB_MAX_LEVELS];     // entries from the start of level 1 to the start of staged level l (l >= 1)
@@ -220,6 +225,62 @@ __device__ __forceinline__ float prb_sum_children_dyn(const float* c, uint32_t K
     default: return prb_sum_children<32>(c);
     }
 }
+
+// Both at once: x = the left-to-right binary32 sum of the K children at c, m = the smallest positive of the K
+// values at cm (0 if none; cm == c where the children are the leaves, which serve both trees).  All loads are
+// issued before anything is computed: one round trip through L2 for the two nodes, not two.
+template <int K>
+__device__ __forceinline__ void prb_sum_and_min(const float* c, const float* cm, float& x, float& m)
+{
+    unsigned best = 0xFFFFFFFFu;
+    auto take = [&best](float u) { if (u > 0.0f) best = min(best, __float_as_uint(u)); };
+    const bool own = cm != c;
+    if (K == 2) {
+        const float2 a = __ldcg(reinterpret_cast<const float2*>(c));
+        float2 b = a;
+        if (own) b = __ldcg(reinterpret_cast<const float2*>(cm));
+        x = __fadd_rn(a.x, a.y);
+        take(b.x); take(b.y);
+    } else {
+        constexpr int Q = K / 4 > 0 ? K / 4 : 1;
+        x = 0.0f;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const float4 a = __ldcg(reinterpret_cast<const float4*>(c) + q);
+            float4 b = a;
+            if (own) b = __ldcg(reinterpret_cast<const float4*>(cm) + q);
+            x = q ? __fadd_rn(x, a.x) : a.x;
+            x = __fadd_rn(__fadd_rn(__fadd_rn(x, a.y), a.z), a.w);
+            take(b.x); take(b.y); take(b.z); take(b.w);
+        }
+    }
+    m = best == 0xFFFFFFFFu ? 0.0f : __uint_as_float(best);
+}
+__device__ __forceinline__ void prb_sum_and_min_dyn(const float* c, const float* cm, uint32_t K, float& x, float& m)
+{
+    switch (K) {
+    case 2: prb_sum_and_min<2>(c, cm, x, m); break;
+    case 4: prb_sum_and_min<4>(c, cm, x, m); break;
+    case 8: prb_sum_and_min<8>(c, cm, x, m); break;
+    case 16: prb_sum_and_min<16>(c, cm, x, m); break;
+    default: prb_sum_and_min<32>(c, cm, x, m); break;
+    }
+}
+
+// The smallest positive priority stored, for weights normalised over the whole buffer: the min-tree's root
+// if the buffer keeps one, else what the scan launched before this kernel left in the state.
+__device__ __forceinline__ float prb_buffer_pmin(const PrbView& v)
+{
+    if (v.min_off) return __ldcg(v.level[0] + v.min_off);
+    return __uint_as_float((unsigned)v.state->pmin_bits);
+}
+
+// Runs CALL(frames, min_tree) with the two compile-time options of the tree-writing kernels that view v needs.
+#define PRB_WITH_TREE_OPTIONS(v, CALL)                                              \
+    do {                                                                            \
+        if ((v).stack) { if ((v).min_off) { CALL(true, true); } else { CALL(true, false); } }   \
+        else { if ((v).min_off) { CALL(false, true); } else { CALL(false, false); } }           \
+    } while (0)
 
 // The running maximum of written priorities: positive binary32 values order like their bit patterns.
 __device__ __forceinline__ void prb_note_priorities(PrbState* st, float local_max, bool report)

@@ -275,7 +275,7 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     const unsigned long long calls = v.state->sample_calls;
     const unsigned long long fill = v.state->fill;
     const float total32 = __ldg(v.level[0]);
-    const float pmin = plan.buffer_norm ? __uint_as_float((unsigned)v.state->pmin_bits) : 0.0f;
+    const float pmin = plan.buffer_norm ? prb_buffer_pmin(v) : 0.0f;
     {
         // stage the top levels: one contiguous run of the slab starting at level 1, 16 bytes at a time
         const float4* src = reinterpret_cast<const float4*>(v.level[1]);
@@ -711,7 +711,7 @@ prb_descend_kernel(const __grid_constant__ PrbView v, uint32_t B, uint64_t seed,
         hd->buffer_norm = plan.buffer_norm;
         hd->fill = fill;
         hd->total = total32;
-        hd->pmin = plan.buffer_norm ? __uint_as_float((unsigned)v.state->pmin_bits) : 0.0f;
+        hd->pmin = plan.buffer_norm ? prb_buffer_pmin(v) : 0.0f;
         if (empty) atomicOr(&v.state->status, PEARL_ST_EMPTY);
         else v.state->sample_calls = s_calls + 1;
         if (plan.buffer_norm) v.state->pmin_bits = ~0ull;      // (ready for the next scan)
@@ -1018,8 +1018,8 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
     }
     for (uint32_t i = 0; i < n_sub; ++i) sub_plan[i].ticket_total = ticket_total;
     int extra_launches = 0;
-    if (plan.buffer_norm) {
-        // the scan of the leaves goes first, on the caller's stream
+    if (plan.buffer_norm && v.min_off == 0) {
+        // the scan of the leaves goes first, on the caller's stream (no min-tree to read the minimum from)
         const uint64_t per_cta = 256ull * 16ull;
         uint64_t ctas = (v.capacity + per_cta - 1) / per_cta;
         if (ctas > (uint64_t)sm_count * 4) ctas = (uint64_t)sm_count * 4;
@@ -1083,8 +1083,8 @@ int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned cha
     plan.buffer_norm = (buffer_norm && !uniform) ? 1u : 0u;
     plan_staged_top(v, uniform != 0, plan);
     int launches = 1;
-    if (plan.buffer_norm) {
-        // the scan of the leaves goes first, on the same stream
+    if (plan.buffer_norm && v.min_off == 0) {
+        // the scan of the leaves goes first, on the same stream (no min-tree to read the minimum from)
         const uint64_t per_cta = 256ull * 16ull;
         uint64_t ctas = (v.capacity + per_cta - 1) / per_cta;
         if (ctas > (uint64_t)sm_count * 4) ctas = (uint64_t)sm_count * 4;

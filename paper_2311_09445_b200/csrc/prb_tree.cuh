@@ -24,6 +24,9 @@ struct PrbTeam {
     // key list, CTA `part` of `parts` takes the slots whose warp-sized group number is congruent to
     // it, and the phases are separated by the cluster's hardware barrier.  parts == 1: one CTA.
     uint32_t part = 0, parts = 1;
+    // PrbView::min_off in the kernels instantiated for a buffer with a min-tree, the constant 0 in the others
+    // (which then carry none of its code)
+    uint64_t min_off = 0;
 
     __device__ __forceinline__ void sync() const
     {
@@ -103,8 +106,10 @@ __device__ __forceinline__ bool prb_history_less(const PrbView& v, uint64_t curs
 // whole from shared memory (every parent always equals the sum of its children, so a parent none of
 // whose children changed comes out as it was): no sorted keys, no round trip through L2.
 // mem == nullptr: nothing is staged and every pass goes through global memory.
+// mem_min: the same levels of the min-tree, staged the same way (nullptr: the buffer keeps none, or nothing is staged).
 struct PrbTop {
     float* mem = nullptr;
+    float* mem_min = nullptr;
 };
 __device__ __forceinline__ uint32_t prb_top_levels(const PrbView& v, const PrbTop& top) { return top.mem ? v.top_levels : 0u; }
 
@@ -117,6 +122,23 @@ __device__ __forceinline__ void prb_top_begin(const PrbView& v, const PrbTop& to
     const float* src = v.level[1];
     for (uint32_t q = rank; q < v.top_floats / 4u; q += nthreads)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + q * 16u), "l"(src + q * 4u) : "memory");
+    if (top.mem_min == nullptr) return;
+    const uint32_t dst_min = (uint32_t)__cvta_generic_to_shared(top.mem_min);
+    for (uint32_t q = rank; q < v.top_floats / 4u; q += nthreads)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_min + q * 16u), "l"(src + v.min_off + q * 4u) : "memory");
+}
+
+// A value for the staged copy of CTA 0 (see prb_resum): a plain store by a single CTA, a store through
+// distributed shared memory by a CTA of a cluster.
+__device__ __forceinline__ void prb_store_staged(float* t, float x, const PrbTeam& team)
+{
+    if (team.parts == 1) {
+        *t = x;
+    } else {
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(t)), "r"(0u));
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(x) : "memory");
+    }
 }
 __device__ __forceinline__ void prb_top_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
@@ -128,17 +150,18 @@ __device__ __forceinline__ void prb_resum(const PrbView& v, const PrbTop& top, c
 {
     const uint32_t K = v.fanout;
     if (!PRB_IN_BOUNDS(v, a * K + K <= v.level_alloc[l + 1] && a < v.level_alloc[l])) return;
-    const float x = prb_sum_children_dyn(v.level[l + 1] + a * K, K);
+    float x, m = 0.0f;
+    if (team.min_off) {     // the min-tree's node as well: from the leaves themselves one level up, else from its own children
+        const float* c = v.level[l + 1] + a * K;
+        prb_sum_and_min_dyn(c, c + (l + 1 == v.depth ? 0 : team.min_off), K, x, m);
+        (v.level[l] + team.min_off)[a] = m;
+    } else {
+        x = prb_sum_children_dyn(v.level[l + 1] + a * K, K);
+    }
     v.level[l][a] = x;
     if (l == T && l >= 1) {
-        float* t = top.mem + v.top_off[l] + a;
-        if (team.parts == 1) {
-            *t = x;
-        } else {
-            uint32_t remote;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(t)), "r"(0u));
-            asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(x) : "memory");
-        }
+        prb_store_staged(top.mem + v.top_off[l] + a, x, team);
+        if (team.min_off) prb_store_staged(top.mem_min + v.top_off[l] + a, m, team);
     }
 }
 
@@ -160,8 +183,28 @@ __device__ __forceinline__ float prb_sum_staged(const float* c)
     }
 }
 
+// The smallest positive of K staged children (0 if none); 16-byte loads, as for the sums.
+template <int K>
+__device__ __forceinline__ float prb_min_staged(const float* c)
+{
+    unsigned best = 0xFFFFFFFFu;
+    auto take = [&best](float u) { if (u > 0.0f) best = min(best, __float_as_uint(u)); };
+    if (K == 2) {
+        const float2 f = *reinterpret_cast<const float2*>(c);
+        take(f.x); take(f.y);
+    } else {
+        float4 u[K / 4 > 0 ? K / 4 : 1];
+#pragma unroll
+        for (int q = 0; q < K / 4; ++q) u[q] = reinterpret_cast<const float4*>(c)[q];
+#pragma unroll
+        for (int q = 0; q < K / 4; ++q) { take(u[q].x); take(u[q].y); take(u[q].z); take(u[q].w); }
+    }
+    return best == 0xFFFFFFFFu ? 0.0f : __uint_as_float(best);
+}
+
 // The passes over the staged levels, by one CTA: parents of level T-1, then T-2, ... then the root,
 // each level whole; a parent that comes out different is stored, staged copy and global memory.
+// The min-tree's staged levels go through the same passes.
 template <int K>
 __device__ __forceinline__ void prb_top_passes_k(const PrbView& v, const PrbTop& top, const PrbTeam& team, uint32_t T)
 {
@@ -180,6 +223,16 @@ __device__ __forceinline__ void prb_top_passes_k(const PrbView& v, const PrbTop&
             } else if (__float_as_uint(x) != __float_as_uint(own[i])) {
                 own[i] = x;
                 v.level[l][i] = x;
+            }
+            if (team.min_off) {
+                const float m = prb_min_staged<K>(top.mem_min + v.top_off[l + 1] + (size_t)i * K);
+                float* own_min = top.mem_min + v.top_off[l];
+                if (l == 0) {
+                    (v.level[0] + team.min_off)[0] = m;
+                } else if (__float_as_uint(m) != __float_as_uint(own_min[i])) {
+                    own_min[i] = m;
+                    (v.level[l] + team.min_off)[i] = m;
+                }
             }
         }
         if (l) team.sync();

@@ -12,7 +12,8 @@
 namespace {
 
 // kFrames: the instance for the frame-deduplicated layout (markers, cleared leaves, stale history-less updates)
-template <bool kFrames>
+// kMin: the instance that maintains the min-tree beside the sum tree
+template <bool kFrames, bool kMin>
 __global__ void __launch_bounds__(1024)
 prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, const int32_t* __restrict__ idx,
                   const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale,
@@ -27,8 +28,10 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     team.whole_cta = true;
     team.part = blockIdx.x;          // CTAs of one cluster share the work (one CTA: the whole of it)
     team.parts = gridDim.x;
+    if (kMin) team.min_off = v.min_off;
     PrbTop top;
     if (v.top_levels) top.mem = reinterpret_cast<float*>(smem + prb_update_smem_bytes(n2));
+    if (kMin && v.top_levels) top.mem_min = top.mem + v.top_floats;
     if (team.part == 0) prb_top_begin(v, top, team.rank, team.size);
     unsigned long long fill, cursor = 0;
     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
@@ -146,7 +149,7 @@ __device__ __forceinline__ void prb_resum_subtree(const PrbView& v, uint32_t lt,
 __device__ __forceinline__ uint32_t prb_levels_per_pass(uint32_t K, uint32_t left, uint32_t B)
 {
     const uint32_t most = (K == 2) ? (B > 16384u ? 2u : 5u) : (K == 4) ? 2u : 1u;
-    return left < most ? left : most;
+    return left < most ? left : most;      // (with a min-tree the caller takes one level per pass)
 }
 
 __device__ __forceinline__ void prb_resum_levels(const PrbView& v, uint32_t h, uint32_t lt, uint64_t a)
@@ -157,6 +160,21 @@ __device__ __forceinline__ void prb_resum_levels(const PrbView& v, uint32_t h, u
     case 3: prb_resum_subtree<2, 3>(v, lt, a); break;
     case 4: prb_resum_subtree<2, 4>(v, lt, a); break;
     default: prb_resum_subtree<2, 5>(v, lt, a); break;
+    }
+}
+
+// One parent of level lt from its K children (and the min-tree's node beside it, if there is one).
+__device__ __forceinline__ void prb_wide_resum_one(const PrbView& v, uint32_t lt, uint64_t a)
+{
+    const uint32_t K = v.fanout;
+    const float* c = v.level[lt + 1] + a * K;
+    if (v.min_off) {
+        float x, m;
+        prb_sum_and_min_dyn(c, c + (lt + 1 == v.depth ? 0 : v.min_off), K, x, m);
+        v.level[lt][a] = x;
+        (v.level[lt] + v.min_off)[a] = m;
+    } else {
+        v.level[lt][a] = prb_sum_children_dyn(c, K);
     }
 }
 
@@ -242,14 +260,14 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
 
     // 3. the levels below the staged top, deepest first; small fanouts take several levels per pass
     for (int l = (int)D - 1; alive && l >= (int)T;) {
-        const uint32_t h = prb_levels_per_pass(K, (uint32_t)l - T + 1u, B);
+        const uint32_t h = v.min_off ? 1u : prb_levels_per_pass(K, (uint32_t)l - T + 1u, B);
         const uint32_t lt = (uint32_t)l - h + 1u;                 // the highest level this pass writes
         const uint32_t sh = lg * (D - lt);
         const uint64_t n_lt = ((v.capacity - 1) >> sh) + 1;       // nodes of level lt
         if (n_lt <= 2ull * B) {
             for (uint64_t a = gtid; a < n_lt; a += gthreads) {
                 if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
-                if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
+                if (h == 1) prb_wide_resum_one(v, lt, a);
                 else prb_resum_levels(v, h, lt, a);
             }
         } else {
@@ -262,7 +280,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
                     if (before >= 0 && (unsigned long long)before < fill && ((uint64_t)before >> sh) == a) continue;
                 }
                 if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
-                if (h == 1) v.level[lt][a] = prb_sum_children_dyn(v.level[lt + 1] + a * K, K);
+                if (h == 1) prb_wide_resum_one(v, lt, a);
                 else prb_resum_levels(v, h, lt, a);
             }
         }
@@ -283,6 +301,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
     if (blockIdx.x == 0 && T > 0) {
         PrbTop top;
         top.mem = reinterpret_cast<float*>(smem);
+        if (v.min_off) top.mem_min = top.mem + v.top_floats;
         prb_top_begin(v, top, tid, kWideThreads);
         prb_top_wait();
         __syncthreads();
@@ -290,6 +309,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         team.rank = tid;
         team.size = kWideThreads;
         team.whole_cta = true;
+        team.min_off = v.min_off;
         prb_top_passes(v, top, team, T);
     }
 }
@@ -327,7 +347,7 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
 {
     static int ctas_per_sm[kPrbMaxDevices];      // 0: not asked yet, -1: not available
     const int dev = prb_current_device();
-    const size_t smem = (size_t)kPrbTopFloats * sizeof(float);
+    const size_t smem = (size_t)kPrbTopFloats * sizeof(float) * 2;     // (room for a min-tree's staged levels too)
     if (ctas_per_sm[dev] == 0) {
         int coop = 0, nb = 0;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
@@ -345,7 +365,7 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kWideThreads);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = (size_t)v.top_floats * sizeof(float) * (v.min_off ? 2 : 1);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;
@@ -370,9 +390,11 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
     static bool big_smem[kPrbMaxDevices];
     const int dev = prb_current_device();
     if (!big_smem[dev]) {
-        const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + kPrbTopFloats * sizeof(float));
-        if (cudaFuncSetAttribute(prb_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(prb_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
+        const int most = (int)(prb_update_smem_bytes(PEARL_UPDATE_SUBBATCH) + 2 * kPrbTopFloats * sizeof(float));
+        if (cudaFuncSetAttribute(prb_update_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_update_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_update_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_update_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
             return -1;
         big_smem[dev] = true;
     }
@@ -387,7 +409,7 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(ctas);
         cfg.blockDim = dim3(threads);
-        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2) + v.top_floats * sizeof(float);
+        cfg.dynamicSmemBytes = prb_update_smem_bytes(n2) + v.top_floats * sizeof(float) * (v.min_off ? 2 : 1);
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -396,10 +418,11 @@ int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const 
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = v.stack ? cudaLaunchKernelEx(&cfg, prb_update_kernel<true>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
-                                                           eps, stale, ins_n, ins_prio, ctas, ins_done)
-                                      : cudaLaunchKernelEx(&cfg, prb_update_kernel<false>, v, b, n2, d_idx + first, d_val + first, raw, alpha,
-                                                           eps, stale, ins_n, ins_prio, ctas, ins_done);
+        cudaError_t e = cudaSuccess;
+#define PRB_LAUNCH_UPDATE_AS(FF, MM) \
+    e = cudaLaunchKernelEx(&cfg, prb_update_kernel<FF, MM>, v, b, n2, d_idx + first, d_val + first, raw, alpha, eps, stale, ins_n, ins_prio, ctas, ins_done)
+        PRB_WITH_TREE_OPTIONS(v, PRB_LAUNCH_UPDATE_AS);
+#undef PRB_LAUNCH_UPDATE_AS
         if (e != cudaSuccess) return -1;
         ++launches;
     }

@@ -47,11 +47,14 @@ def seed_for_sliver(oracle_mod, B, call=0, limit=1 << 22):
 
 
 class Pair:
-    def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True, frame_stack=0):
+    def __init__(self, oracle_mod, capacity, fanout, obs_bytes, act_bytes, max_batch, oracle_store=True, frame_stack=0,
+                 min_tree=False):
         """frame_stack > 0: both sides use the frame-deduplicated layout (obs_bytes = a whole stack; an insertion's
-        batch carries one frame per transition under "obs" and no "next_obs")."""
+        batch carries one frame per transition under "obs" and no "next_obs").  min_tree: the GPU buffer keeps a
+        min-tree (the oracle has none: it scans its leaves)."""
         from paper_2311_09445_b200 import PrioritizedReplay
-        self.gpu = PrioritizedReplay(capacity, fanout, obs_bytes, act_bytes, max_batch, frame_stack=frame_stack)
+        self.gpu = PrioritizedReplay(capacity, fanout, obs_bytes, act_bytes, max_batch, frame_stack=frame_stack,
+                                     min_tree=min_tree)
         self.oracle_store = oracle_store
         self.ora = oracle_mod.OraclePRB(capacity, fanout, obs_bytes if oracle_store else 0,
                                         act_bytes if oracle_store else 0, frame_stack=frame_stack)
@@ -191,6 +194,25 @@ class Pair:
                 bad = np.nonzero(bits(a) != bits(b))[0]
                 raise AssertionError("tree level %d differs at %d entries, first %d: oracle %r gpu %r"
                                      % (l, bad.size, bad[0], a[bad[0]], b[bad[0]]))
+
+    def compare_min_tree(self):
+        """Every node of the GPU's min-tree against its definition, written out on the ORACLE's leaves: the
+        smallest positive leaf among the fanout^(depth-l) leaves below node (l, a), 0 if none is positive."""
+        D, K = self.ora.depth, self.fanout
+        leaves = self.ora.read_level(D)
+        for l in range(D):
+            span = K ** (D - l)
+            n = self.gpu.level_alloc(l)
+            padded = np.zeros(n * span, np.float32)
+            m = min(leaves.size, padded.size)
+            padded[:m] = leaves[:m]
+            grouped = np.where(padded > 0, padded, np.float32(np.inf)).reshape(n, span).min(axis=1)
+            want = np.where(np.isinf(grouped), np.float32(0), grouped).astype(np.float32)
+            got = self.gpu.read_min_level(l)
+            if not np.array_equal(bits(want), bits(got)):
+                bad = np.nonzero(bits(want) != bits(got))[0]
+                raise AssertionError("min-tree level %d differs at %d nodes, first %d: expected %r gpu %r"
+                                     % (l, bad.size, bad[0], want[bad[0]], got[bad[0]]))
 
     def compare_state(self):
         assert self.gpu.info() == self.ora.info()

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 
 SUBSET = ("small_buffers or random_call or step or captured or fused or large_batch_sample or many_cta_update or delta or "
           "falls_off or ragged or reduced_capacity or normalised_over or streamed or uniform or default_insert or "
-          "after_insert or (sweep_cells and 65536-) or (sweep_cells and 1048576-16)")
+          "after_insert or (sweep_cells and 65536-) or (sweep_cells and 1048576-16) or min_tree")
 
 
 def test_parity_suite_against_the_checked_library():
@@ -26,6 +26,7 @@ def test_parity_suite_against_the_checked_library():
     lib = build.build(checked=True)
     env = dict(os.environ, PEARL_PRB_LIB=lib)
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join("tests", "test_gpu_parity.py"), os.path.join("tests", "test_zz_no_alloc.py"),
+                        os.path.join("tests", "test_gpu_min_tree.py"),
                         "-x", "-q", "-m", "gpu", "-k", SUBSET], cwd=ROOT, env=env, capture_output=True, text=True, timeout=1800)
     tail = r.stdout[-3000:] + r.stderr[-2000:]
     assert r.returncode == 0, tail
