@@ -304,7 +304,14 @@ int pearl_prb_update_host(pearl_prb_t* prb, uint32_t B, const int32_t* h_idx, co
  * in the caller's arrays.  A step whose inputs and whose outputs come to at most 256 KB each makes no copy
  * call: the inputs are gathered in a pinned buffer of the handle that the device reads in place, the kernels
  * write the batch into that buffer, and the step's one synchronisation is the wait for them.  A larger step
- * is pearl_prb_update_host, pearl_prb_insert_host and pearl_prb_sample_host one after the other.
+ * that inserts and samples rows of 8 KB and more (plain layout, n >= 1, B_upd <= PEARL_UPDATE_SUBBATCH) keeps
+ * both directions of the host link busy at once: the new rows travel to the device on a stream of the handle
+ * while the caller's stream updates the tree (the new priorities included), draws the batch, and sends back
+ * the rows of every stratum that drew none of the new slots; the rest -- rows of strata that did, indices,
+ * weights, short fields -- follows when the new rows are stored.  The copies overlap only if the caller's
+ * arrays are pinned (page-locked) memory; with pageable memory the step is correct and serial.  Any other
+ * large step is pearl_prb_update_host, pearl_prb_insert_host and pearl_prb_sample_host one after the other.
+ * Results are those of the three calls whichever way the step travels.
  * Arguments and errors as for pearl_prb_step, with host pointers. */
 int pearl_prb_step_host(pearl_prb_t* prb, uint32_t B_upd, const int32_t* h_upd_idx, const float* h_td, float alpha,
                         float eps, uint32_t n, const void* h_new_obs, const void* h_new_act, const float* h_new_rew,

@@ -797,10 +797,98 @@ int pearl_prb_update_host(pearl_prb_t* h, uint32_t B, const int32_t* h_idx, cons
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }
 
+namespace {
+
+inline bool long_field(const pearl_prb* h, int f)
+{
+    return h->view.field_vec[f] == 16 && h->view.field_bytes[f] / 16u >= 512u;
+}
+
+// A step of long rows through host buffers with the two directions of the host link busy at once.
+// The new transitions' long rows travel host -> device on a second stream while the caller's stream runs the
+// tree kernel (update + the insertion's tree work, which needs the new priorities only), the descents and the
+// row copy of every stratum that drew none of the new slots, and sends those rows device -> host.  When the
+// new rows have arrived and are in the store (the insertion's row kernel, second stream), the rest follows on
+// the caller's stream: rows of strata that drew new slots, indices, weights, short fields.  The first, large
+// device -> host copy carried whatever the output staging held for those few strata: their rows are copied
+// again, one by one, at the end.  Results are those of the three calls.
+int step_host_duplex(pearl_prb* h, uint32_t B_upd, const int32_t* h_upd_idx, const float* h_td, float alpha, float eps, uint32_t n,
+                     const void* const src[PRB_NUM_FIELDS], const float* h_new_prio, uint32_t B, float beta, uint64_t seed,
+                     int32_t* h_idx, float* h_w, void* const dst[PRB_NUM_FIELDS])
+{
+    const Layout& L = h->lay;
+    cudaStream_t main = h->stream, up = h->subs.stream[1];
+    PrbBatch in_b, out_b;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+        in_b.ptr[f] = (src[f] && h->view.field_bytes[f]) ? at(h, L.off_stage_in[f]) : nullptr;
+        out_b.ptr[f] = (dst[f] && L.out_bytes[f]) ? at(h, L.off_stage_out[f]) : nullptr;
+    }
+    int32_t* d_idx = (int32_t*)at(h, L.off_stage_out_idx);
+    float* d_w = h_w ? (float*)at(h, L.off_stage_out_w) : nullptr;
+    int32_t* d_uidx = (int32_t*)at(h, L.off_stage_idx);
+    float* d_td = (float*)at(h, L.off_stage_td);
+    float* d_prio = h_new_prio ? (float*)at(h, L.off_stage_prio) : nullptr;
+    auto to_dev = [](void* d, const void* s, uint64_t bytes, cudaStream_t st) {
+        return cudaMemcpyAsync(d, s, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    auto to_host = [](void* d, const void* s, uint64_t bytes, cudaStream_t st) {
+        return cudaMemcpyAsync(d, s, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    // the second stream starts where the caller's stream is (the staging areas may still be in use by its work)
+    if (cudaEventRecord(h->subs.fork, main) != cudaSuccess || cudaStreamWaitEvent(up, h->subs.fork, 0) != cudaSuccess) return PEARL_ERR_CUDA;
+    // (the tree kernel's few inputs are handed to the copy engine first: it serves copies in the order they were issued)
+    if (!to_dev(d_uidx, h_upd_idx, (uint64_t)B_upd * 4, main) || !to_dev(d_td, h_td, (uint64_t)B_upd * 4, main)) return PEARL_ERR_CUDA;
+    if (d_prio && !to_dev(d_prio, h_new_prio, (uint64_t)n * 4, main)) return PEARL_ERR_CUDA;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
+        if (in_b.ptr[f] && !to_dev(in_b.ptr[f], src[f], (uint64_t)n * h->view.field_bytes[f], up)) return PEARL_ERR_CUDA;      // (read by the row kernel only)
+    unsigned char* area = h->view.handoff[0];
+    int k = prb_launch_update(h->view, B_upd, d_uidx, d_td, 0, alpha, eps, main, 0, n, d_prio, in_b.ptr[F_DONE]);
+    if (k != 1) return PEARL_ERR_CUDA;
+    if (prb_launch_descend(h->view, B, seed, area, main, 0, 0) != 1) return PEARL_ERR_CUDA;
+    if (prb_launch_gather(h->view, B, beta, area, d_idx, d_w, out_b, main, false, 1, n) != 1) return PEARL_ERR_CUDA;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
+        if (out_b.ptr[f] && long_field(h, f) && !to_host(dst[f], out_b.ptr[f], (uint64_t)B * L.out_bytes[f], main)) return PEARL_ERR_CUDA;
+    if (prb_launch_insert(h->view, n, in_b, d_prio, up, 0, nullptr, nullptr, 0, 0.0f, 0.0f, nullptr, nullptr, true) != 1) return PEARL_ERR_CUDA;
+    if (cudaEventRecord(h->subs.done[1], up) != cudaSuccess || cudaStreamWaitEvent(main, h->subs.done[1], 0) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (prb_launch_gather(h->view, B, beta, area, d_idx, d_w, out_b, main, false, 2, n) != 1) return PEARL_ERR_CUDA;
+    h->launches += 5;
+    h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0;
+    // (the cursor comes back with the batch: into the handle's pinned buffer where there is one -- no call
+    // leaves its second half in use -- so that the copy call itself does not wait for the stream)
+    unsigned long long cursor_here = 0;
+    unsigned long long* cursor_at = h->pin ? (unsigned long long*)(h->pin + 2 * kPackBytes - 16) : &cursor_here;
+    if (!to_host(h_idx, d_idx, (uint64_t)B * 4, main) || (h_w && !to_host(h_w, d_w, (uint64_t)B * 4, main))) return PEARL_ERR_CUDA;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f)
+        if (out_b.ptr[f] && !long_field(h, f) && !to_host(dst[f], out_b.ptr[f], (uint64_t)B * L.out_bytes[f], main)) return PEARL_ERR_CUDA;
+    if (!to_host(cursor_at, &h->view.state->cursor, sizeof(unsigned long long), main)) return PEARL_ERR_CUDA;
+    if (cudaStreamSynchronize(main) != cudaSuccess) return PEARL_ERR_CUDA;
+    const unsigned long long cursor = *cursor_at;
+    // the strata that drew one of the new slots: their long rows were written after the large copy
+    const uint64_t N = h->view.capacity;
+    const uint64_t lo = cursor >= n ? cursor - n : cursor + N - n;
+    bool again = false;
+    for (uint32_t s = 0; s < B; ++s) {
+        if (h_idx[s] < 0) continue;
+        const uint64_t i = (uint64_t)h_idx[s];
+        if ((i >= lo ? i - lo : i + N - lo) >= n) continue;
+        for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+            const uint64_t row = L.out_bytes[f];
+            if (out_b.ptr[f] && long_field(h, f) && !to_host((unsigned char*)dst[f] + s * row, out_b.ptr[f] + s * row, row, main)) return PEARL_ERR_CUDA;
+        }
+        again = true;
+    }
+    if (again && cudaStreamSynchronize(main) != cudaSuccess) return PEARL_ERR_CUDA;
+    return PEARL_OK;
+}
+
+}  // namespace
+
 // One iteration through host buffers as one call.  A small step (all inputs, and all outputs, within 256 KB
 // each) makes no copy call at all: the inputs are gathered in the handle's pinned buffer, which the device
 // sees mapped, the kernels read them from there and write the sampled batch into its second half, and the
-// one synchronisation of the step is the wait for that.  A larger step is the three host calls.
+// one synchronisation of the step is the wait for that.  A larger step with long rows both ways (8 KB and
+// more, plain layout, at most PEARL_UPDATE_SUBBATCH updates) runs with both directions of the host link busy
+// at once (step_host_duplex above); any other is the three host calls.
 int pearl_prb_step_host(pearl_prb_t* h, uint32_t B_upd, const int32_t* h_upd_idx, const float* h_td, float alpha, float eps,
                         uint32_t n, const void* h_new_obs, const void* h_new_act, const float* h_new_rew, const void* h_new_next_obs,
                         const uint8_t* h_new_done, const float* h_new_prio, uint32_t B, float beta, uint64_t seed, int32_t* h_idx,
@@ -822,6 +910,17 @@ int pearl_prb_step_host(pearl_prb_t* h, uint32_t B_upd, const int32_t* h_upd_idx
     out.add(PRB_NUM_FIELDS, (uint64_t)B * 4);
     out.add(PRB_NUM_FIELDS + 1, h_w ? (uint64_t)B * 4 : 0);
     if (!(h->pin_dev && in.total <= kPackBytes && out.total <= kPackBytes)) {
+        bool long_in = false, long_out = false;
+        for (int f = 0; f < PRB_NUM_FIELDS; ++f) {
+            long_in = long_in || (src[f] && long_field(h, f));
+            long_out = long_out || (dst[f] && long_field(h, f));
+        }
+        if (n && h->view.stack == 0 && B_upd <= PEARL_UPDATE_SUBBATCH && long_in && long_out) {
+            const void* ins[PRB_NUM_FIELDS] = { h_new_obs, h_new_next_obs, h_new_act, h_new_rew, h_new_done };
+            DeviceGuard guard(h->device);
+            if (!guard.ok) return PEARL_ERR_CUDA;
+            return step_host_duplex(h, B_upd, h_upd_idx, h_td, alpha, eps, n, ins, h_new_prio, B, beta, seed, h_idx, h_w, dst);
+        }
         int rc = pearl_prb_update_host(h, B_upd, h_upd_idx, h_td, alpha, eps);
         if (rc != PEARL_OK) return rc;
         rc = n ? pearl_prb_insert_host(h, n, h_new_obs, h_new_act, h_new_rew, h_new_next_obs, h_new_done, h_new_prio) : PEARL_OK;

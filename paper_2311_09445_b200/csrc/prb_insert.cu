@@ -221,9 +221,10 @@ prb_insert_rows_kernel(const __grid_constant__ PrbView v, uint32_t n, const __gr
 
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B, const int32_t* upd_idx, const float* upd_val, int upd_raw, float alpha, float eps,
-                      const PrbFork* fork, bool* forked_out)
+                      const PrbFork* fork, bool* forked_out, bool rows_only)
 {
     if (forked_out) *forked_out = false;
+    if (rows_only && upd_B) return -1;
     const int sm_count = prb_sm_count();
     const int dev = prb_current_device();
     FusedUpdate upd;
@@ -256,6 +257,7 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     int launches = 1;
     bool forked = false;
     uint32_t rows_grid = 0;
+    if (rows_only && tasks == 0) return -1;
     const bool fork_tree = upd.B && tasks > 0 && upd.B <= PEARL_UPDATE_SUBBATCH && fork != nullptr;
     if (tasks > 0) {
         stage = (stage + 127u) / 128u * 128u;
@@ -266,12 +268,14 @@ int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const f
     if (tasks > 0) {
         // Without a tree kernel CTA 0 does the tree work and no copies; with one, its CTAs get SMs of
         // their own: a copy CTA takes an SM's whole shared memory and would wait for them to leave.
-        const uint32_t want = tasks + (fork_tree ? 0u : 1u);
+        const uint32_t want = tasks + ((fork_tree || rows_only) ? 0u : 1u);
         uint32_t room = (uint32_t)sm_count;
         if (fork_tree && room > 2u * prb_update_ctas(v, upd.B)) room -= prb_update_ctas(v, upd.B);
         rows_grid = want < room ? want : room;
     }
-    if (fork_tree) {
+    if (rows_only) {
+        plan.tree_ctas = 1;       // (CTA 0 copies like the others and the row cursor is published by itself)
+    } else if (fork_tree) {
         // Long rows: the update and the insertion's tree work are one kernel on the side stream, the
         // row copy another on the caller's stream; neither waits for the other (each advances a
         // cursor of its own), and the caller's stream goes on when both are done.  (In one kernel the tree's chain of dependent reads, slowed by the

@@ -108,7 +108,9 @@ struct PrbFork {
 int prb_launch_insert(const PrbView& v, uint32_t n, const PrbBatch& src, const float* d_prio, cudaStream_t s,
                       uint32_t upd_B = 0, const int32_t* upd_idx = nullptr, const float* upd_val = nullptr,
                       int upd_raw = 0, float alpha = 0.0f, float eps = 0.0f, const PrbFork* fork = nullptr,
-                      bool* forked_out = nullptr);
+                      bool* forked_out = nullptr, bool rows_only = false);
+// (rows_only: long rows, and the insertion's tree work is some other launch's -- a prb_launch_update with
+// ins_n = n: this one copies the rows and advances the row cursor, nothing else)
 // Streams and events of a sample call that is issued as sub-batches (the paper's sub-batch
 // streaming, Section IV-C): sub-batch i runs on stream[i]; done[i] fires when its rows are in place.
 constexpr uint32_t kPrbMaxSubBatches = 4;
@@ -150,7 +152,9 @@ int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned cha
 // (early_reads: the kernel before this one on s writes no rows of the store -- it is a row copy of a sample
 // too -- so this one may read rows while that one is still running)
 int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned char* handoff, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, bool early_reads = false);
+                      const PrbBatch& dst, cudaStream_t s, bool early_reads = false, int part = 0, uint32_t new_n = 0);
+// (part 1 / part 2: the copy as two launches around the row copy of an insertion of new_n transitions whose tree
+// work is done -- see the kernel; neither is a programmatic dependent)
 // An empty kernel: a node that depends in full on what precedes it on s, for a programmatic dependent to hang on.
 int prb_launch_relay(cudaStream_t s);
 // true if a sample that writes these fields moves rows long enough for the bulk-copy ring

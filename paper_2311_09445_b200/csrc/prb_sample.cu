@@ -730,10 +730,17 @@ constexpr uint32_t kGatherRingBytes = 198 * 1024;      // the row copy's ring
 constexpr int kGatherWorkers = 128;
 constexpr int kGatherThreads = 32 + kGatherWorkers;
 
+//
+// kPart: 0, the whole copy.  1 and 2, the copy in two launches around an insertion of new_n transitions whose
+// priorities are in the tree (so the descents may have drawn them) and whose rows are not yet in the store:
+// launch 1 moves the long rows of every stratum that drew none of the new slots -- the new_n slots before the
+// published cursor -- and launch 2, once the new rows are stored, the long rows of the others and everything
+// else (indices, weights, short fields).
+template <int kPart>
 __global__ void __launch_bounds__(kGatherThreads, 1)
 prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, const unsigned char* __restrict__ handoff,
                        int32_t* __restrict__ out_idx, float* __restrict__ out_w, const __grid_constant__ PrbBatch dst,
-                       const __grid_constant__ SamplePlan plan, uint32_t early_reads)
+                       const __grid_constant__ SamplePlan plan, uint32_t early_reads, uint32_t new_n)
 {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ uint32_t s_idx[kGatherWorkers];
@@ -762,6 +769,11 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
         if (__ldcg(&prb_handoff_header(handoff)->found) == 0u) return;          // the buffer was empty: nothing is written
         bool waited = false;
         if (!early_reads) { prb_dep_wait(); waited = true; }
+        uint64_t new_lo = 0;
+        if (kPart) {
+            const uint64_t cursor = __ldcg(&v.state->cursor);
+            new_lo = cursor >= new_n ? cursor - new_n : cursor + v.capacity - new_n;
+        }
         while (t < t_hi) {
             const uint32_t k = t / tps, r = t - k * tps;
             int f = 0;
@@ -769,7 +781,12 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
             const uint32_t W = v.field_bytes[f] / 16u;
             const uint32_t e0 = (r - plan.task_first[f]) * plan.chunk[f];
             const uint32_t bytes = min(W - e0, plan.chunk[f]) * 16u;
-            const bool inside = PRB_IN_BOUNDS(v, (uint32_t)leaf < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes);
+            bool inside = PRB_IN_BOUNDS(v, (uint32_t)leaf < v.capacity && k < B && e0 < W && bytes <= plan.ring_stage_bytes);
+            if (kPart) {
+                const uint64_t i = (uint32_t)leaf;
+                const bool is_new = (i >= new_lo ? i - new_lo : i + v.capacity - new_lo) < new_n;
+                inside = inside && (is_new == (kPart == 2));
+            }
             if (inside) ring.load(v.store[f] + ((uint64_t)(uint32_t)leaf * W + e0) * 16u, bytes);
             const uint32_t t_next = t + plan.ring_stages;
             const int32_t leaf_next = t_next < t_hi ? __ldcg(pre_idx + t_next / tps) : 0;
@@ -780,7 +797,7 @@ prb_gather_rows_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
         }
         ring.finish();
         if (ring.failed) atomicOr(&v.state->status, PEARL_ST_INTERNAL);
-    } else if (tid >= 32) {
+    } else if (tid >= 32 && kPart != 1) {
         const uint32_t rank = tid - 32u;
         const uint32_t k_own = (t_lo + tps - 1) / tps, k_end = (t_hi + tps - 1) / tps;
         const PrbHandoffHeader* hd = prb_handoff_header(handoff);
@@ -1119,8 +1136,9 @@ int prb_launch_descend(const PrbView& v, uint32_t B, uint64_t seed, unsigned cha
 }
 
 int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned char* handoff, int32_t* d_idx, float* d_w,
-                      const PrbBatch& dst, cudaStream_t s, bool early_reads)
+                      const PrbBatch& dst, cudaStream_t s, bool early_reads, int part, uint32_t new_n)
 {
+    if (part < 0 || part > 2 || (part && (early_reads || new_n == 0 || new_n > v.capacity))) return -1;
     SamplePlan plan;
     if (!plan_row_mode(v, dst, plan)) return -1;
     const int sm_count = prb_sm_count();
@@ -1140,8 +1158,10 @@ int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned c
     const uint32_t smem = kRingBarBytes + plan.ring_stages * stage;
     static bool big_smem[kPrbMaxDevices];
     if (!big_smem[dev]) {
-        if (cudaFuncSetAttribute(prb_gather_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(kRingBarBytes + kGatherRingBytes)) != cudaSuccess)
+        const int most = (int)(kRingBarBytes + kGatherRingBytes);
+        if (cudaFuncSetAttribute(prb_gather_rows_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_gather_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(prb_gather_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
             return -1;
         big_smem[dev] = true;
     }
@@ -1156,8 +1176,11 @@ int prb_launch_gather(const PrbView& v, uint32_t B, float beta, const unsigned c
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = part ? 0 : 1;      // (the two launches of a split copy depend in full on what precedes them)
     const uint32_t early = early_reads ? 1u : 0u;
-    if (cudaLaunchKernelEx(&cfg, prb_gather_rows_kernel, v, B, beta, handoff, d_idx, d_w, dst, plan, early) != cudaSuccess) return -1;
-    return 1;
+    cudaError_t e;
+    if (part == 0) e = cudaLaunchKernelEx(&cfg, prb_gather_rows_kernel<0>, v, B, beta, handoff, d_idx, d_w, dst, plan, early, 0u);
+    else if (part == 1) e = cudaLaunchKernelEx(&cfg, prb_gather_rows_kernel<1>, v, B, beta, handoff, d_idx, d_w, dst, plan, early, new_n);
+    else e = cudaLaunchKernelEx(&cfg, prb_gather_rows_kernel<2>, v, B, beta, handoff, d_idx, d_w, dst, plan, early, new_n);
+    return e == cudaSuccess ? 1 : -1;
 }

@@ -431,10 +431,13 @@ def test_host_buffer_calls(oracle_mod):
 
 
 @pytest.mark.parametrize("wl,N,B,n", [(wk.CARTPOLE, 5000, 64, 64), (wk.DDPG, 70_000, 256, 256), (wk.DDPG, 5000, 3000, 1000),
-                                      (wk.ATARI, 600, 16, 8)])
+                                      (wk.ATARI, 600, 16, 8), (wk.ATARI, 700, 512, 512), (wk.ATARI, 1500, 300, 37),
+                                      (wk.ATARI, 600, 64, 600), (wk.ATARI, 900, 4096, 100)])
 def test_step_through_host_buffers(oracle_mod, wl, N, B, n):
-    # pearl_prb_step_host: a small step travels through the handle's mapped pinned buffer (no copy call), a
-    # larger one is the three host calls; either way the oracle's update, insert, sample
+    # pearl_prb_step_host: a small step travels through the handle's mapped pinned buffer (no copy call); a
+    # larger one with long rows has its copies in both directions in flight at once, the rows of strata that
+    # drew a slot of the very insertion of the step being copied last (here: few of them, most, or all); any
+    # other is the three host calls.  Whichever way, the oracle's update, insert, sample
     wl = wk.scaled(wl, N)
     rng = np.random.default_rng(N + B)
     pr = Pair(oracle_mod, N, wl.fanout, wl.obs_bytes, wl.act_bytes, 4096)
