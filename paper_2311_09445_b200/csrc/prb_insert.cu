@@ -100,6 +100,9 @@ prb_insert_kernel(const __grid_constant__ PrbView v, uint32_t n, const __grid_co
     __shared__ unsigned long long s_cursor, s_fill;     // read once per CTA, before anything is published
     __shared__ unsigned int s_maxp;                     // running maximum of priorities at kernel start
     const uint32_t tid = threadIdx.x;
+    // (the kernel after this one on the stream, if it was launched as a programmatic dependent, may be made
+    // resident now; it waits for this kernel's completion before it reads anything)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == kWorkers) { s_cursor = v.state->cursor; s_fill = v.state->fill; s_maxp = v.state->max_prio_bits; }
     // the tree CTA fetches its first inputs now, while the cursor is on its way
     // (and starts the copy of the tree's top into shared memory, behind the update's keys)

@@ -270,6 +270,9 @@ prb_sample_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta, uin
     PrbBulkLane ring;            // lanes 0 .. ring_stages-1 of warp 0 own one stage each
     const bool ring_lane = bulk && tid < plan.ring_stages;
     if (ring_lane) ring.init(s_ring + 8u * tid, s_ring + kRingBarBytes + tid * plan.ring_stage_bytes);
+    // (launched as a programmatic dependent of the kernel before it on the stream: up to here it may have run
+    // beside that kernel; nothing has been read or written yet)
+    prb_dep_wait();
     // every thread reads the state it needs itself (same addresses: one request per warp), so the
     // targets can be formed while the staged levels are still on their way
     const unsigned long long calls = v.state->sample_calls;
@@ -1055,6 +1058,18 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
         }
         const uint32_t grid = sub_grid[i], smem = sub_smem[i];
         const SamplePlan& sp = sub_plan[i];
+        // (a whole batch is launched as a programmatic dependent of the kernel before it on the stream -- its
+        // launch is then under way while that kernel runs; it waits for that kernel before its first read)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = at;
+        cudaLaunchAttribute pss[1];
+        pss[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pss[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = pss;
+        cfg.numAttrs = n_sub == 1 ? 1 : 0;
 #define PRB_LAUNCH_SAMPLE_AS(KK, FF)                                                                              \
     do {                                                                                                          \
         if (max_smem && !big_smem[dev][fr][ki]) {                                                                 \
@@ -1063,7 +1078,7 @@ int prb_launch_sample(const PrbView& v, uint32_t B, float beta, uint64_t seed, i
             big_smem[dev][fr][ki] = (attr == cudaSuccess);                                                        \
         }                                                                                                         \
         if (attr == cudaSuccess)                                                                                  \
-            prb_sample_kernel<KK, FF><<<grid, kThreads, smem, at>>>(v, B, beta, seed, d_idx, d_w, dst, sp);       \
+            attr = cudaLaunchKernelEx(&cfg, prb_sample_kernel<KK, FF>, v, B, beta, seed, d_idx, d_w, dst, sp);     \
     } while (0)
 #define PRB_LAUNCH_SAMPLE(KK)                                                                                     \
     do { if (fr) PRB_LAUNCH_SAMPLE_AS(KK, true); else PRB_LAUNCH_SAMPLE_AS(KK, false); } while (0)

@@ -22,6 +22,9 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned long long s_cursor, s_fill;
+    // (a programmatic dependent behind this kernel may be made resident now; it waits for this kernel's
+    // completion before it reads anything)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     PrbTeam team;
     team.rank = threadIdx.x;
     team.size = blockDim.x;
