@@ -37,21 +37,18 @@ __device__ __forceinline__ double prb_stratum_target(uint32_t k, uint32_t B, dou
     return x;
 }
 
-// The K children of one node into registers.  global: from global memory -- through the read-only path,
-// or, with kCoherent, through L2 only (the kernel itself, or a CTA beside this one, has written tree
-// levels) -- else from shared memory (this CTA's, or, through a generic address, another CTA's of the cluster).
-template <int K, bool kCoherent>
+// The K children of one node into registers.  global: from global memory, through the read-only path (no
+// kernel that walks the tree writes it); else from this CTA's shared memory.
+template <int K>
 __device__ __forceinline__ void prb_load_children(const float* src, bool global, float (&c)[K])
 {
     if (K == 2) {
-        const float2 t = global ? (kCoherent ? __ldcg(reinterpret_cast<const float2*>(src)) : __ldg(reinterpret_cast<const float2*>(src)))
-                                : *reinterpret_cast<const float2*>(src);
+        const float2 t = global ? __ldg(reinterpret_cast<const float2*>(src)) : *reinterpret_cast<const float2*>(src);
         c[0] = t.x; c[1] = t.y;
     } else {
 #pragma unroll
         for (int q = 0; q < K / 4; ++q) {
-            const float4 t = global ? (kCoherent ? __ldcg(reinterpret_cast<const float4*>(src) + q) : __ldg(reinterpret_cast<const float4*>(src) + q))
-                                    : reinterpret_cast<const float4*>(src)[q];
+            const float4 t = global ? __ldg(reinterpret_cast<const float4*>(src) + q) : reinterpret_cast<const float4*>(src)[q];
             c[4 * q] = t.x; c[4 * q + 1] = t.y; c[4 * q + 2] = t.z; c[4 * q + 3] = t.w;
         }
     }
@@ -61,7 +58,7 @@ __device__ __forceinline__ void prb_load_children(const float* src, bool global,
 // K children of the node, their left-to-right binary32 prefix sums one after another, and the first
 // child whose prefix exceeds the binary64 target -- the count of prefixes the target has passed.  Levels
 // 1 .. top_levels are read from s_top (level l at top_off[l]), the others from global memory.
-template <int K, bool kCoherent>
+template <int K>
 __device__ __forceinline__ void prb_descend_alone(const PrbView& v, uint32_t top_levels, const uint32_t* top_off, const float* s_top,
                                                   double x, uint32_t& leaf, float& p_leaf, unsigned& flags)
 {
@@ -71,7 +68,7 @@ __device__ __forceinline__ void prb_descend_alone(const PrbView& v, uint32_t top
         float c[K];
         const bool staged = l <= top_levels;
         if (!PRB_IN_BOUNDS(v, g * K + K <= v.level_alloc[l])) { flags |= PEARL_ST_INTERNAL; g = 0; }
-        prb_load_children<K, kCoherent>(staged ? s_top + top_off[l] + (uint32_t)g * K : v.level[l] + g * K, !staged, c);
+        prb_load_children<K>(staged ? s_top + top_off[l] + (uint32_t)g * K : v.level[l] + g * K, !staged, c);
         int j = -1, last_pos = -1;
         float run = 0.0f, before_j = 0.0f, before_last = 0.0f;
 #pragma unroll

@@ -567,7 +567,7 @@ prb_sample_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, float beta
             // target of stratum k (Eq. 1's x, one per equal segment of the total), then the walk
             const double x = prb_stratum_target(k, B, total, calls, seed);
             uint32_t leaf; float p;
-            prb_descend_alone<K, false>(v, plan.top_levels, plan.top_off, s_top, x, leaf, p, my_flags);
+            prb_descend_alone<K>(v, plan.top_levels, plan.top_off, s_top, x, leaf, p, my_flags);
             s_idx[tid] = leaf;
             out_idx[k] = (int32_t)leaf;
             if (out_w != nullptr) {
