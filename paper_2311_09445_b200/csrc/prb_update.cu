@@ -167,15 +167,16 @@ __device__ __forceinline__ void prb_resum_levels(const PrbView& v, uint32_t h, u
 }
 
 // One parent of level lt from its K children (and the min-tree's node beside it, if there is one).
-__device__ __forceinline__ void prb_wide_resum_one(const PrbView& v, uint32_t lt, uint64_t a)
+// (min_off: PrbView::min_off in the kernel instantiated for a buffer with a min-tree, the constant 0 in the other)
+__device__ __forceinline__ void prb_wide_resum_one(const PrbView& v, uint32_t lt, uint64_t a, uint64_t min_off)
 {
     const uint32_t K = v.fanout;
     const float* c = v.level[lt + 1] + a * K;
-    if (v.min_off) {
+    if (min_off) {
         float x, m;
-        prb_sum_and_min_dyn(c, c + (lt + 1 == v.depth ? 0 : v.min_off), K, x, m);
+        prb_sum_and_min_dyn(c, c + (lt + 1 == v.depth ? 0 : min_off), K, x, m);
         v.level[lt][a] = x;
-        (v.level[lt] + v.min_off)[a] = m;
+        (v.level[lt] + min_off)[a] = m;
     } else {
         v.level[lt][a] = prb_sum_children_dyn(c, K);
     }
@@ -206,6 +207,7 @@ __device__ __forceinline__ bool prb_grid_barrier(PrbState* st, uint32_t& passed,
     return *s_ok != 0;
 }
 
+template <bool kMin>
 __global__ void __launch_bounds__(kWideThreads)
 prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int32_t* __restrict__ idx,
                        const float* __restrict__ val, int raw, float alpha, float eps, uint32_t stale)
@@ -263,14 +265,14 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
 
     // 3. the levels below the staged top, deepest first; small fanouts take several levels per pass
     for (int l = (int)D - 1; alive && l >= (int)T;) {
-        const uint32_t h = v.min_off ? 1u : prb_levels_per_pass(K, (uint32_t)l - T + 1u, B);
+        const uint32_t h = kMin ? 1u : prb_levels_per_pass(K, (uint32_t)l - T + 1u, B);
         const uint32_t lt = (uint32_t)l - h + 1u;                 // the highest level this pass writes
         const uint32_t sh = lg * (D - lt);
         const uint64_t n_lt = ((v.capacity - 1) >> sh) + 1;       // nodes of level lt
         if (n_lt <= 2ull * B) {
             for (uint64_t a = gtid; a < n_lt; a += gthreads) {
                 if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
-                if (h == 1) prb_wide_resum_one(v, lt, a);
+                if (h == 1) prb_wide_resum_one(v, lt, a, kMin ? v.min_off : 0ull);
                 else prb_resum_levels(v, h, lt, a);
             }
         } else {
@@ -283,7 +285,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
                     if (before >= 0 && (unsigned long long)before < fill && ((uint64_t)before >> sh) == a) continue;
                 }
                 if (!PRB_IN_BOUNDS(v, a < v.level_alloc[lt] && (h > 1 || a * K + K <= v.level_alloc[lt + 1]))) continue;
-                if (h == 1) prb_wide_resum_one(v, lt, a);
+                if (h == 1) prb_wide_resum_one(v, lt, a, kMin ? v.min_off : 0ull);
                 else prb_resum_levels(v, h, lt, a);
             }
         }
@@ -304,7 +306,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
     if (blockIdx.x == 0 && T > 0) {
         PrbTop top;
         top.mem = reinterpret_cast<float*>(smem);
-        if (v.min_off) top.mem_min = top.mem + v.top_floats;
+        if (kMin) top.mem_min = top.mem + v.top_floats;
         prb_top_begin(v, top, tid, kWideThreads);
         prb_top_wait();
         __syncthreads();
@@ -312,7 +314,7 @@ prb_update_wide_kernel(const __grid_constant__ PrbView v, uint32_t B, const int3
         team.rank = tid;
         team.size = kWideThreads;
         team.whole_cta = true;
-        team.min_off = v.min_off;
+        if (kMin) team.min_off = v.min_off;
         prb_top_passes(v, top, team, T);
     }
 }
@@ -354,7 +356,7 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
     if (ctas_per_sm[dev] == 0) {
         int coop = 0, nb = 0;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, prb_update_wide_kernel, (int)kWideThreads, smem) != cudaSuccess || nb < 1) {
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, prb_update_wide_kernel<true>, (int)kWideThreads, smem) != cudaSuccess || nb < 1) {
             cudaGetLastError();
             ctas_per_sm[dev] = -1;
         } else {
@@ -375,8 +377,9 @@ static int prb_launch_update_wide(const PrbView& v, uint32_t B, const int32_t* d
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, prb_update_wide_kernel, v, B, d_idx, d_val, raw, alpha, eps, stale) != cudaSuccess) return -1;
-    return 1;
+    const cudaError_t e = v.min_off ? cudaLaunchKernelEx(&cfg, prb_update_wide_kernel<true>, v, B, d_idx, d_val, raw, alpha, eps, stale)
+                                    : cudaLaunchKernelEx(&cfg, prb_update_wide_kernel<false>, v, B, d_idx, d_val, raw, alpha, eps, stale);
+    return e == cudaSuccess ? 1 : -1;
 }
 
 int prb_launch_update(const PrbView& v, uint32_t B, const int32_t* d_idx, const float* d_val, int raw,
