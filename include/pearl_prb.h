@@ -370,6 +370,26 @@ uint64_t pearl_prb_level_alloc(pearl_prb_t* prb, uint32_t level);
 int pearl_prb_read_rows(pearl_prb_t* prb, const int32_t* h_idx, uint32_t n, void* h_obs,
                         void* h_act, float* h_rew, void* h_next_obs, uint8_t* h_done);
 
+/* Checkpoint and resume.  The image of a buffer is a 256-byte header (geometry: capacity, fanout, row sizes,
+ * frame stack, options) followed by its persistent device memory as it lies in the slab: the state (ring
+ * cursor, fill count, call counter, running maximum, pending status bits), the sum tree (and the min-tree
+ * of a buffer that keeps one), and the Data Storage.  The paper keeps replay memory for the length of a
+ * training run (Section IV); a run that is to survive a restart needs it back bit for bit, because the
+ * sampled indices depend on every priority and on the call counter.
+ *   pearl_prb_image_bytes  the size of the image.
+ *   pearl_prb_export       waits for the stream, then copies bytes [offset, offset + bytes) of the image to
+ *                          h_dst (so a large image can be written out piece by piece).
+ *   pearl_prb_import       copies bytes [offset, offset + bytes) of an image into the buffer.  A piece that
+ *                          covers any of the header must cover all of it; the header is then compared with
+ *                          this buffer's geometry: PEARL_ERR_BAD_ARG if they differ (nothing is copied).
+ *                          The caller imports the whole image, the header first, before the next call
+ *                          that uses the buffer; after that the buffer behaves exactly as the exported one
+ *                          did: same samples for the same seeds, same tree, same rows.  Waits for the stream.
+ * PEARL_ERR_BAD_ARG for a range outside the image. */
+uint64_t pearl_prb_image_bytes(pearl_prb_t* prb);
+int pearl_prb_export(pearl_prb_t* prb, uint64_t offset, void* h_dst, uint64_t bytes);
+int pearl_prb_import(pearl_prb_t* prb, uint64_t offset, const void* h_src, uint64_t bytes);
+
 /* Number of kernels this handle has launched so far. */
 uint64_t pearl_prb_kernel_launches(pearl_prb_t* prb);
 

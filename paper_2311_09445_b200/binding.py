@@ -65,6 +65,9 @@ SIGNATURES = {
     "pearl_prb_max_priority": (_i, [_vp, C.POINTER(_f32)]),
     "pearl_prb_read_level": (_i, [_vp, _u32, _vp, _u64]),
     "pearl_prb_read_min_level": (_i, [_vp, _u32, _vp, _u64]),
+    "pearl_prb_image_bytes": (_u64, [_vp]),
+    "pearl_prb_export": (_i, [_vp, _u64, _vp, _u64]),
+    "pearl_prb_import": (_i, [_vp, _u64, _vp, _u64]),
     "pearl_prb_level_alloc": (_u64, [_vp, _u32]),
     "pearl_prb_read_rows": (_i, [_vp, _vp, _u32, _vp, _vp, _vp, _vp, _vp]),
     "pearl_prb_kernel_launches": (_u64, [_vp]),
@@ -354,6 +357,33 @@ class PrioritizedReplay:
         if rc != 0:
             raise PearlError(rc, "pearl_prb_read_min_level")
         return out
+
+    def export_image(self, piece_bytes: int = 1 << 28):
+        """The buffer's checkpoint image as a host array of bytes (pearl_prb_export, piece by piece)."""
+        import numpy as np
+        lib = load_library()
+        total = int(lib.pearl_prb_image_bytes(self._h))
+        out = np.empty(total, dtype=np.uint8)
+        for off in range(0, total, piece_bytes):
+            n = min(piece_bytes, total - off)
+            rc = lib.pearl_prb_export(self._h, off, C.c_void_p(out.ctypes.data + off), n)
+            if rc != 0:
+                raise PearlError(rc, "pearl_prb_export")
+        return out
+
+    def import_image(self, image, piece_bytes: int = 1 << 28) -> None:
+        """Restores the buffer from an image made by export_image (pearl_prb_import; the geometry must match)."""
+        import numpy as np
+        lib = load_library()
+        image = np.ascontiguousarray(image, dtype=np.uint8)
+        total = int(lib.pearl_prb_image_bytes(self._h))
+        if image.shape[0] != total:
+            raise PearlError(-7, "pearl_prb_import")
+        for off in range(0, total, piece_bytes):
+            n = min(piece_bytes, total - off)
+            rc = lib.pearl_prb_import(self._h, off, C.c_void_p(image.ctypes.data + off), n)
+            if rc != 0:
+                raise PearlError(rc, "pearl_prb_import")
 
     def read_rows(self, idx):
         import numpy as np

@@ -1130,6 +1130,99 @@ int pearl_prb_read_rows(pearl_prb_t* h, const int32_t* h_idx, uint32_t n, void* 
     return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
 }
 
+// ---- checkpoint and resume -----------------------------------------------------------------------
+namespace {
+
+constexpr uint64_t kImageHeaderBytes = 256;
+struct ImageHeader {
+    char magic[8];                    // "PEARLPRB"
+    uint32_t version;
+    uint32_t fanout;
+    uint64_t capacity;
+    uint32_t field_bytes[PRB_NUM_FIELDS];
+    uint32_t field_pitch[PRB_NUM_FIELDS];
+    uint32_t stack;
+    uint32_t min_tree;
+    uint64_t tree_bytes;              // state, sum tree, min-tree: slab bytes [off_state, off_wraw)
+    uint64_t store_bytes;             // Data Storage: slab bytes [off_zero_end, off_stage_in[0])
+};
+static_assert(sizeof(ImageHeader) <= kImageHeaderBytes, "the image header has 256 bytes");
+
+void fill_image_header(const pearl_prb* h, unsigned char out[kImageHeaderBytes])
+{
+    memset(out, 0, kImageHeaderBytes);
+    ImageHeader hd;
+    memset(&hd, 0, sizeof(hd));
+    memcpy(hd.magic, "PEARLPRB", 8);
+    hd.version = 1;
+    hd.fanout = h->view.fanout;
+    hd.capacity = h->view.capacity;
+    for (int f = 0; f < PRB_NUM_FIELDS; ++f) { hd.field_bytes[f] = h->lay.field_bytes[f]; hd.field_pitch[f] = h->lay.field_pitch[f]; }
+    hd.stack = h->lay.stack;
+    hd.min_tree = h->lay.off_min ? 1u : 0u;
+    hd.tree_bytes = h->lay.off_wraw - h->lay.off_state;
+    hd.store_bytes = h->lay.off_stage_in[0] - h->lay.off_zero_end;
+    memcpy(out, &hd, sizeof(hd));
+}
+
+// Copies the part of image range [offset, offset + bytes) that lies in the image's part [part_at, part_at + part_bytes),
+// which is slab range [slab_at, ...), in the direction given.
+int copy_image_part(pearl_prb* h, uint64_t offset, unsigned char* host, uint64_t bytes, uint64_t part_at, uint64_t part_bytes,
+                    uint64_t slab_at, bool to_host)
+{
+    const uint64_t lo = offset > part_at ? offset : part_at;
+    const uint64_t hi = (offset + bytes) < (part_at + part_bytes) ? (offset + bytes) : (part_at + part_bytes);
+    if (lo >= hi) return PEARL_OK;
+    unsigned char* dev = at(h, slab_at + (lo - part_at));
+    unsigned char* hp = host + (lo - offset);
+    const cudaError_t e = to_host ? cudaMemcpyAsync(hp, dev, hi - lo, cudaMemcpyDeviceToHost, h->stream)
+                                  : cudaMemcpyAsync(dev, hp, hi - lo, cudaMemcpyHostToDevice, h->stream);
+    return e == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+int image_transfer(pearl_prb* h, uint64_t offset, unsigned char* host, uint64_t bytes, bool to_host)
+{
+    unsigned char mine[kImageHeaderBytes];
+    fill_image_header(h, mine);
+    const uint64_t tree_bytes = h->lay.off_wraw - h->lay.off_state, store_bytes = h->lay.off_stage_in[0] - h->lay.off_zero_end;
+    const uint64_t total = kImageHeaderBytes + tree_bytes + store_bytes;
+    if (offset > total || bytes > total - offset) return PEARL_ERR_BAD_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return PEARL_ERR_CUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return PEARL_ERR_CUDA;
+    if (offset < kImageHeaderBytes && bytes > 0) {
+        const uint64_t n = (offset + bytes < kImageHeaderBytes ? offset + bytes : kImageHeaderBytes) - offset;
+        if (to_host) memcpy(host, mine + offset, n);
+        else if (offset != 0 || n != kImageHeaderBytes || memcmp(host, mine, kImageHeaderBytes) != 0) return PEARL_ERR_BAD_ARG;
+    }
+    int rc = copy_image_part(h, offset, host, bytes, kImageHeaderBytes, tree_bytes, h->lay.off_state, to_host);
+    if (rc == PEARL_OK)
+        rc = copy_image_part(h, offset, host, bytes, kImageHeaderBytes + tree_bytes, store_bytes, h->lay.off_zero_end, to_host);
+    if (rc != PEARL_OK) return rc;
+    if (!to_host) { h->main_touched = true; h->main_last_gather = 0; h->after_forked_tree = 0; }
+    return cudaStreamSynchronize(h->stream) == cudaSuccess ? PEARL_OK : PEARL_ERR_CUDA;
+}
+
+}  // namespace
+
+uint64_t pearl_prb_image_bytes(pearl_prb_t* h)
+{
+    if (!h) return 0;
+    return kImageHeaderBytes + (h->lay.off_wraw - h->lay.off_state) + (h->lay.off_stage_in[0] - h->lay.off_zero_end);
+}
+
+int pearl_prb_export(pearl_prb_t* h, uint64_t offset, void* h_dst, uint64_t bytes)
+{
+    if (!h || !h_dst) return PEARL_ERR_NULL;
+    return image_transfer(h, offset, (unsigned char*)h_dst, bytes, true);
+}
+
+int pearl_prb_import(pearl_prb_t* h, uint64_t offset, const void* h_src, uint64_t bytes)
+{
+    if (!h || !h_src) return PEARL_ERR_NULL;
+    return image_transfer(h, offset, (unsigned char*)h_src, bytes, false);
+}
+
 uint64_t pearl_prb_kernel_launches(pearl_prb_t* h) { return h ? h->launches : 0; }
 
 const char* pearl_prb_error_string(int code)
