@@ -148,7 +148,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, reasons = [], [], set()
+        sm, mx, watts, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.splitlines():
             p = [t.strip() for t in line.split(",")]
@@ -158,11 +158,17 @@ class ClockSampler:
                 sm.append(float(p[1])); mx.append(float(p[2]))
             except ValueError:
                 continue
+            try:
+                watts.append(float(p[3]))
+            except ValueError:
+                pass
             for name, v in zip(names, p[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons),
+                # board power while the timed region ran: context for the paper's per-watt figures (Section VI), no more
+                "power_w": statistics.median(watts) if watts else None}
 
 
 # ------------------------------------------------------------------------------------------
