@@ -482,6 +482,24 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         }
     }
 
+    // How the CTAs of a cluster share the work below the staged levels: by subtree.  A leaf, and every node
+    // above it down to the deepest staged level T, belongs to the CTA that its ancestor on level T falls to; what
+    // a pass reads was then written by the same CTA, and a barrier of that CTA separates the passes -- not the
+    // cluster's, whose release has every CTA wait until its stores have reached L2.  (Without staged levels the
+    // slots are dealt out by position and the cluster's barrier separates the passes.)
+    const uint32_t lg = v.log2_fanout, T = prb_top_levels(v, top);
+    const bool by_subtree = team.parts > 1 && T >= 1;
+    const uint32_t sh_top = min(lg * (v.depth - T), 63u);
+    auto mine = [&](uint64_t leaf, uint32_t slot_no) {
+        return by_subtree ? ((leaf >> sh_top) % team.parts) == team.part : team.takes(slot_no);
+    };
+    auto mine_node = [&](uint64_t a, uint32_t l, uint32_t slot_no) {      // node a of level l >= T
+        return by_subtree ? ((a >> (lg * (l - T))) % team.parts) == team.part : team.takes(slot_no);
+    };
+    auto pass_sync = [&](bool next_is_top) {
+        if (by_subtree && !next_is_top) team.sync();
+        else team.phase_sync();
+    };
     float* leaves = v.level[v.depth];
     if (raw == 2) {
         // Changes instead of values (n == 0): the last entry of a run of equal indices adds the run's
@@ -501,7 +519,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             team.sync();
             if (rank < n2) { sidx[rank] = slot.idx; spos[rank] = slot.pos; }
             team.sync();
-            if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
+            if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && mine(slot.idx, rank)) {
                 uint32_t s0 = rank;
                 while (s0 > 0 && sidx[s0 - 1] == slot.idx) --s0;
                 if (PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth])) {
@@ -513,7 +531,7 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         } else {
             for (uint32_t s1 = rank; s1 < n2; s1 += nt) {
                 const unsigned long long key = keys[s1];
-                if (prb_key_invalid(key) || !team.takes(s1)) continue;
+                if (prb_key_invalid(key) || !mine(key >> 32, s1)) continue;
                 const uint32_t i = (uint32_t)(key >> 32);
                 if (s1 + 1 < n2 && (uint32_t)(keys[s1 + 1] >> 32) == i) continue;      // not the last of its run
                 uint32_t s0 = s1;
@@ -526,14 +544,14 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         if (refused) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
         prb_note_priorities(v.state, dmax, true);
     } else if (one_each) {
-        if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && team.takes(rank)) {
+        if (slot.idx != 0xFFFFFFFFu && slot.next != slot.idx && mine(slot.idx, rank)) {
             const uint64_t ahead = slot.idx >= cursor ? slot.idx - cursor : slot.idx + N - cursor;   // distance from the cursor along the ring
             if (!(ahead < n_leaves) && PRB_IN_BOUNDS(v, slot.idx < v.level_alloc[v.depth] && slot.pos < n2)) leaves[slot.idx] = vals[slot.pos];
         }
     } else {
         for (uint32_t s = rank; s < n2; s += nt) {
             const unsigned long long key = keys[s];
-            if (prb_key_invalid(key) || !team.takes(s)) continue;
+            if (prb_key_invalid(key) || !mine(key >> 32, s)) continue;
             const uint32_t i = (uint32_t)(key >> 32);
             const bool last = (s + 1 == n2) || ((uint32_t)(keys[s + 1] >> 32) != i);
             const uint64_t ahead = i >= cursor ? i - cursor : i + N - cursor;
@@ -547,9 +565,9 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     if (n && prio == nullptr && team.parts > 1) { __threadfence(); team.phase_sync(); }
     const float dflt = (n && prio == nullptr) ? prb_default_priority(__ldcg(&v.state->max_prio_bits)) : 0.0f;
     for (uint32_t t = rank; t < n_leaves; t += nt) {
-        if (!team.takes(t)) continue;
         uint64_t at = cursor + t;
         if (at >= N) at -= N;
+        if (!mine(at, t)) continue;
         float p = 0.0f;
         if (t < n && !(stack && (ins_done[t] & kPrbEpisodeStart))) {
             p = prio == nullptr ? dflt : ((pre.has_prio && t == rank) ? pre.prio : prio[t]);
@@ -560,12 +578,11 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
     }
     if (bad) atomicOr(&v.state->status, PEARL_ST_BAD_PRIORITY);
     if (n) prb_note_priorities(v.state, imax, true);      // (every CTA of a cluster wrote leaves of its own; a first default insertion writes 1)
-    team.phase_sync();
+    pass_sync(false);
 
     // re-sum the ancestors below the staged levels, deepest level first: the first entry of every run
     // of equal ancestors does it; the insertion dirties parent range A = [a0, a1] >> sh and, if the
     // ring wrapped, B = [0, b1] >> sh
-    const uint32_t lg = v.log2_fanout, T = prb_top_levels(v, top);
     const uint64_t a0 = cursor, a1 = (n ? min(cursor + n_leaves, N) : cursor + 1) - 1;
     const bool wrapped = cursor + n_leaves > N;
     const uint64_t b1 = wrapped ? cursor + n_leaves - N - 1 : 0;
@@ -573,12 +590,13 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
         const uint32_t sh = min(lg * (v.depth - (uint32_t)l), 31u);      // (indices are below 2^31)
         if (one_each) {
             const uint32_t a = slot.idx >> sh;
-            if (slot.idx != 0xFFFFFFFFu && (slot.prev >> sh) != a && team.takes(rank)) prb_resum(v, top, team, T, (uint32_t)l, a);
+            if (slot.idx != 0xFFFFFFFFu && (slot.prev >> sh) != a && mine_node(a, (uint32_t)l, rank)) prb_resum(v, top, team, T, (uint32_t)l, a);
         } else {
             for (uint32_t s = rank; s < n2; s += nt) {
                 const unsigned long long key = keys[s];
-                if (prb_key_invalid(key) || !team.takes(s)) continue;
+                if (prb_key_invalid(key)) continue;
                 const uint32_t a = (uint32_t)(key >> 32) >> sh;
+                if (!mine_node(a, (uint32_t)l, s)) continue;
                 const bool first = (s == 0) || (((uint32_t)(keys[s - 1] >> 32) >> sh) != a);
                 if (first) prb_resum(v, top, team, T, (uint32_t)l, a);
             }
@@ -588,11 +606,11 @@ __device__ __forceinline__ void prb_update_team(const PrbView& v, const PrbTeam&
             uint64_t cntB = 0;
             if (wrapped) cntB = (pa0 == 0) ? 0 : min(b1 >> sh, pa0 - 1) + 1;     // parents of B not already in A
             for (uint64_t i = rank; i < cntA + cntB; i += nt) {
-                if (!team.takes((uint32_t)i)) continue;
-                prb_resum(v, top, team, T, (uint32_t)l, (i < cntA) ? pa0 + i : i - cntA);
+                const uint64_t a = (i < cntA) ? pa0 + i : i - cntA;
+                if (mine_node(a, (uint32_t)l, (uint32_t)i)) prb_resum(v, top, team, T, (uint32_t)l, a);
             }
         }
-        team.phase_sync();
+        pass_sync((uint32_t)l == T);
     }
     // the staged levels: CTA 0 alone
     if (team.part == 0) prb_top_passes(v, top, team, T);
