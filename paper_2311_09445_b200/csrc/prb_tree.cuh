@@ -60,6 +60,22 @@ struct PrbTeam {
 //   kPrbPublishTree  the tree kernel of a two-kernel insertion: cursor and fill (insert_ticket)
 //   kPrbPublishRows  its row kernel: row_cursor (row_ticket)
 constexpr int kPrbPublishTree = 1, kPrbPublishRows = 2, kPrbPublishAll = 3;
+// (what the drawer of the last ticket does; a kernel whose drawing thread has other work to do first may
+// draw early with prb_ticket and come back here with the answer when that work is done)
+__device__ __forceinline__ void prb_publish(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill, int what)
+{
+    unsigned int* ticket = (what == kPrbPublishRows) ? &v.state->row_ticket : &v.state->insert_ticket;
+    const uint64_t N = v.capacity;
+    uint64_t c = cursor + n;
+    if (c >= N) c -= N;
+    if (what & kPrbPublishRows) v.state->row_cursor = c;
+    if (what & kPrbPublishTree) {
+        v.state->cursor = c;
+        fill += n;
+        v.state->fill = fill > N ? N : fill;
+    }
+    *ticket = 0;
+}
 __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n, uint64_t cursor, unsigned long long fill,
                                                     uint32_t participants, int what = kPrbPublishAll)
 {
@@ -67,18 +83,7 @@ __device__ __forceinline__ void prb_publish_if_last(const PrbView& v, uint32_t n
     // passed; the ticket's release/acquire pair orders them before the last drawer's stores)
     unsigned int* ticket = (what == kPrbPublishRows) ? &v.state->row_ticket : &v.state->insert_ticket;
     const unsigned int done = prb_ticket(ticket);
-    if (done == participants - 1) {
-        const uint64_t N = v.capacity;
-        uint64_t c = cursor + n;
-        if (c >= N) c -= N;
-        if (what & kPrbPublishRows) v.state->row_cursor = c;
-        if (what & kPrbPublishTree) {
-            v.state->cursor = c;
-            fill += n;
-            v.state->fill = fill > N ? N : fill;
-        }
-        *ticket = 0;
-    }
+    if (done == participants - 1) prb_publish(v, n, cursor, fill, what);
 }
 
 // Frame-deduplicated layout: an insertion of n transitions at `cursor` writes n + prb_cleared_after(v, n)

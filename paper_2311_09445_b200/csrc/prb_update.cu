@@ -37,6 +37,7 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
     if (kMin && v.top_levels) top.mem_min = top.mem + v.top_floats;
     if (team.part == 0) prb_top_begin(v, top, team.rank, team.size);
     unsigned long long fill, cursor = 0;
+    unsigned int ticket_drawn = 0;
     PrbPreloaded pre = PrbPreloaded{false, false, 0, 0.0f, 0.0f};
     if (ins_n) {
         // with an insertion: cursor and fill are read once per CTA, before anything is published;
@@ -47,13 +48,16 @@ prb_update_kernel(const __grid_constant__ PrbView v, uint32_t B, uint32_t n2, co
         __syncthreads();
         cursor = s_cursor;
         fill = s_fill;
-        if (threadIdx.x == 0) prb_publish_if_last(v, ins_n, cursor, fill, ticket_total, kPrbPublishTree);
+        // (thread 0 draws the CTA's ticket now and looks at the answer after the tree work: it has an entry of
+        // the batch like every other thread, and the team would wait for it at the first barrier of the sort)
+        if (threadIdx.x == 0) ticket_drawn = prb_ticket(&v.state->insert_ticket);
     } else {
         fill = v.state->fill;
         if (stale || kFrames) cursor = v.state->cursor;
     }
     prb_update_team(v, team, B, n2, idx, val, raw, alpha, eps, fill, smem, ins_n, ins_prio, cursor, pre, stale, top, ins_done,
                     kFrames ? v.stack : 0u);
+    if (ins_n && threadIdx.x == 0 && ticket_drawn == ticket_total - 1) prb_publish(v, ins_n, cursor, fill, kPrbPublishTree);
 }
 
 // ---- large batches: one launch of many CTAs ------------------------------------------------------
