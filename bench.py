@@ -479,7 +479,7 @@ def measure_workload(wl, steps, warmup, dev, stream, rank=0, world=1, extras=Tru
 
 
 def summary_of(wl, m, world=1):
-    """The figures the benchmark spec asks for, for one workload: step time, samples/s, updates/s, inserts/s, e2e."""
+    """One workload's figures: step time, samples/s, updates/s, inserts/s, and the same step through host buffers."""
     B, n_ins = wl.batch, wl.n_insert
     ms_step = statistics.median(m["region_ms"]) / m["steps"]
     out = {"us_step": ms_step * 1e3, "transitions_per_s": world * B / (ms_step * 1e-3),
@@ -584,7 +584,7 @@ def run_ours(args, wl, rank, world):
     return line
 
 
-# the other workloads the benchmark spec names, and three cells of the scaling sweep: short runs after the headline's
+# the paper's other workloads (Table III shapes), and three cells of the scaling sweep: short runs after the headline's
 OTHER_SWEEP_CELLS = [(1 << 20, 16, 1024), (1 << 22, 32, 4096), (1 << 24, 4, 65536)]
 
 
