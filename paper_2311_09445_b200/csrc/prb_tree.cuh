@@ -21,8 +21,9 @@ struct PrbTeam {
     uint32_t rank, size;     // this thread's rank in the team, number of threads (multiple of 32)
     bool whole_cta;          // the team is the whole CTA: plain __syncthreads; otherwise named barrier 1
     // Several CTAs of one thread-block cluster may share the tree work: each holds the full sorted
-    // key list, CTA `part` of `parts` takes the slots whose warp-sized group number is congruent to
-    // it, and the phases are separated by the cluster's hardware barrier.  parts == 1: one CTA.
+    // key list and CTA `part` of `parts` takes its share -- by subtree where the tree has staged levels
+    // (see prb_update_team), else the slots whose warp-sized group number is congruent to it, the
+    // phases then separated by the cluster's hardware barrier.  parts == 1: one CTA.
     uint32_t part = 0, parts = 1;
     // PrbView::min_off in the kernels instantiated for a buffer with a min-tree, the constant 0 in the others
     // (which then carry none of its code)
