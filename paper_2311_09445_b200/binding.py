@@ -97,12 +97,14 @@ def _lib_error_string(code: int) -> str:
         return "error"
 
 
+# (addresses are handed to ctypes as plain integers: every pointer parameter is declared c_void_p, which takes
+# an int or None, and a step makes fifteen of these conversions)
 def _dptr(t: Optional[torch.Tensor], what: str):
     if t is None:
         return None
     if not t.is_cuda or not t.is_contiguous():
         raise ValueError("%s must be a contiguous CUDA tensor" % what)
-    return C.c_void_p(t.data_ptr())
+    return t.data_ptr()
 
 
 def _hptr(t, what: str):
@@ -111,8 +113,8 @@ def _hptr(t, what: str):
     if isinstance(t, torch.Tensor):
         if t.is_cuda or not t.is_contiguous():
             raise ValueError("%s must be a contiguous host tensor" % what)
-        return C.c_void_p(t.data_ptr())
-    return C.c_void_p(t.ctypes.data)      # numpy array
+        return t.data_ptr()
+    return t.ctypes.data      # numpy array
 
 
 def _row_bytes(t: torch.Tensor, n: int) -> int:
